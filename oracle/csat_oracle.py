@@ -1,0 +1,175 @@
+"""CPU oracle for the compressed-sensing attention (CSAT) forward.  TEST INFRASTRUCTURE.
+
+This file is test infrastructure: only the tests, the smoke check and the
+benchmark's CPU-baseline leg may import it.  The product (the CUDA library and
+its Python binding) never does, and this file imports nothing from the product.
+
+Plain numpy in float64, one step per equation of the paper's "Mathematical
+Framework" section, in the paper's order and notation (rows are tokens, so the
+paper's column vectors alpha_i, Z_i, C_i appear here as 1 x d rows):
+
+  compress           K~ = Phi K,  V~ = Phi V              (compression equation)
+  compressed_scores  S  = Q K~^T / sqrt(d_k)              (approximate attention matrix)
+  softmax_rows       A~ = softmax over the m measurements (same equation)
+  compressed_output  Z  = A~ V~                           (compressed attention output)
+  decoder_setup      S, B, theta of the LISTA recurrence, instantiated as ISTA
+  ista               alpha^{t+1} = eta_theta(S alpha^t + B Z_i)   (LISTA recurrence)
+  reconstruct        C^_i = Psi alpha^_i                  (reconstruction equation)
+
+Reading of the decoder (the paper's "Z_i = Phi Psi alpha_i" with Phi in R^{m x n}
+cannot multiply a d_k-vector): the sensing matrix of the decoder is a d x d matrix
+D acting on the feature axis, by default the leading d x d block of the head's
+Phi ("Phi_V reused"); M = D Psi; the recurrence is ISTA for
+min_alpha 1/2 ||z - alpha M^T||^2 + lambda ||alpha||_1 with step mu = 1/L^,
+L^ = max absolute row sum of M^T M; S = I - mu M^T M, B = mu M, theta = mu lambda;
+alpha^0 = 0; T = 0 returns Z itself.  Parity with the paper's own (unstated)
+decoder: parity unpinned.  Every function below is pinned by tests/test_oracle_pins.py.
+
+A library matmul (numpy @) serves as the contraction step; nothing is blocked,
+fused or reordered.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+# ----------------------------------------------------------------------------
+# compression, scores, softmax, compressed output
+# ----------------------------------------------------------------------------
+def compress(Phi: np.ndarray, X: np.ndarray) -> np.ndarray:
+    """X~ = Phi X for one (batch, head): Phi [m,n], X [n,d] -> [m,d]."""
+    Phi = np.asarray(Phi, F64)
+    X = np.asarray(X, F64)
+    assert Phi.ndim == 2 and X.ndim == 2 and Phi.shape[1] == X.shape[0]
+    return Phi @ X
+
+
+def compressed_scores(Q: np.ndarray, Kt: np.ndarray, scale: float | None = None) -> np.ndarray:
+    """S[i,r] = scale * <Q_i, K~_r>, scale = 1/sqrt(d_k) by default.  Q [n_q,d], K~ [m,d] -> [n_q,m]."""
+    Q = np.asarray(Q, F64)
+    Kt = np.asarray(Kt, F64)
+    d = Q.shape[1]
+    if scale is None:
+        scale = 1.0 / np.sqrt(F64(d))
+    return (Q @ Kt.T) * F64(scale)
+
+
+def softmax_rows(S: np.ndarray) -> np.ndarray:
+    """Row-wise softmax over the m measurements (last axis), max-subtracted."""
+    S = np.asarray(S, F64)
+    e = np.exp(S - S.max(axis=-1, keepdims=True))
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def compressed_output(A: np.ndarray, Vt: np.ndarray) -> np.ndarray:
+    """Z = A~ V~ : [n_q,m] x [m,d] -> [n_q,d]."""
+    return np.asarray(A, F64) @ np.asarray(Vt, F64)
+
+
+# ----------------------------------------------------------------------------
+# sparse decoder
+# ----------------------------------------------------------------------------
+def soft_threshold(x: np.ndarray, theta: float) -> np.ndarray:
+    """eta_theta(x) = sign(x) * max(|x| - theta, 0), elementwise."""
+    x = np.asarray(x, F64)
+    return np.sign(x) * np.maximum(np.abs(x) - F64(theta), 0.0)
+
+
+def decoder_setup(M: np.ndarray, lam: float, step: float | None = None):
+    """ISTA instance of the LISTA weights for the model z = alpha M^T (M is p x q).
+
+    Returns (S_dec [q,q], B_dec [p,q], theta, mu) with
+      G = M^T M,  L^ = max_a sum_b |G[a,b]|,  mu = 1/L^ (unless `step` is given),
+      S_dec = I - mu G,  B_dec = mu M,  theta = mu * lambda.
+    """
+    M = np.asarray(M, F64)
+    G = M.T @ M
+    if step is None or step == 0:
+        L = np.abs(G).sum(axis=1).max()
+        mu = 1.0 / L
+    else:
+        mu = F64(step)
+    S_dec = np.eye(G.shape[0], dtype=F64) - mu * G
+    B_dec = mu * M
+    theta = mu * F64(lam)
+    return S_dec, B_dec, theta, mu
+
+
+def ista(Z: np.ndarray, S_dec: np.ndarray, B_dec: np.ndarray, theta: float, T: int,
+         return_iterates: bool = False):
+    """T iterations alpha^{t+1} = eta_theta(alpha^t S_dec + Z B_dec), alpha^0 = 0, row-wise.
+
+    Z [rows,p], S_dec [q,q], B_dec [p,q] -> alpha [rows,q].
+    """
+    Z = np.asarray(Z, F64)
+    c = Z @ B_dec
+    alpha = np.zeros((Z.shape[0], S_dec.shape[0]), dtype=F64)
+    its = [alpha]
+    for _ in range(int(T)):
+        alpha = soft_threshold(alpha @ S_dec + c, theta)
+        if return_iterates:
+            its.append(alpha)
+    return (alpha, its) if return_iterates else alpha
+
+
+def reconstruct(alpha: np.ndarray, Psi: np.ndarray | None) -> np.ndarray:
+    """C^_i = Psi alpha^_i, row-wise: out = alpha Psi^T (Psi = I when None)."""
+    if Psi is None:
+        return np.asarray(alpha, F64)
+    return np.asarray(alpha, F64) @ np.asarray(Psi, F64).T
+
+
+def default_decoder_matrix(Phi_h: np.ndarray, d: int) -> np.ndarray:
+    """D = leading d x d block of the head's measurement matrix (rows 0..d-1, columns 0..d-1)."""
+    Phi_h = np.asarray(Phi_h, F64)
+    assert Phi_h.shape[0] >= d and Phi_h.shape[1] >= d, "default decoder matrix needs m >= d and n >= d"
+    return Phi_h[:d, :d].copy()
+
+
+# ----------------------------------------------------------------------------
+# the whole forward
+# ----------------------------------------------------------------------------
+def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, scale=None,
+                      stages: dict | None = None) -> np.ndarray:
+    """CSAT forward for one (batch, head).  Q [n_q,d], K,V [n,d], Phi_h [m,n] -> [n_q,d]."""
+    Q = np.asarray(Q, F64)
+    d = Q.shape[1]
+    Kt = compress(Phi_h, K)
+    Vt = compress(Phi_h, V)
+    S = compressed_scores(Q, Kt, scale)
+    A = softmax_rows(S)
+    Z = compressed_output(A, Vt)
+    if stages is not None:
+        stages.update(Kt=Kt, Vt=Vt, Z=Z)
+    if int(T) == 0:
+        return Z
+    if D is None:
+        D = default_decoder_matrix(Phi_h, d)
+    D = np.asarray(D, F64)
+    M = D if Psi is None else D @ np.asarray(Psi, F64)
+    S_dec, B_dec, theta, mu = decoder_setup(M, lam, step)
+    alpha = ista(Z, S_dec, B_dec, theta, T)
+    if stages is not None:
+        stages.update(alpha=alpha, S_dec=S_dec, B_dec=B_dec, theta=theta, mu=mu)
+    return reconstruct(alpha, Psi)
+
+
+def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=None,
+                 stages: list | None = None) -> np.ndarray:
+    """CSAT forward.  Q [B,H,n_q,d], K,V [B,H,n,d], Phi [H,m,n] (one per head, shared over the
+    batch, Phi_K = Phi_V), Psi None | [d,d] | [H,d,d], D None | [H,d,d]  ->  out [B,H,n_q,d]."""
+    Q = np.asarray(Q)
+    B, H, nq, d = Q.shape
+    out = np.empty((B, H, nq, d), dtype=F64)
+    for b in range(B):
+        for h in range(H):
+            psi_h = None if Psi is None else (Psi if np.ndim(Psi) == 2 else Psi[h])
+            D_h = None if D is None else D[h]
+            st = {} if stages is not None else None
+            out[b, h] = csat_forward_head(Q[b, h], K[b, h], V[b, h], Phi[h], T=T, lam=lam,
+                                          Psi=psi_h, D=D_h, step=step, scale=scale, stages=st)
+            if stages is not None:
+                stages.append(st)
+    return out

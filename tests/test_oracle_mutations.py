@@ -1,0 +1,125 @@
+"""The pins must bite: plant one plausible mistake at a time in the oracle (on the CPU, by
+monkeypatching) and require that at least one pin of tests/test_oracle_pins.py fails."""
+import numpy as np
+import pytest
+
+from oracle import csat_oracle as orc
+import test_oracle_pins as pins
+
+PINS = [getattr(pins, k) for k in dir(pins) if k.startswith("test_") and "phi" not in k and "philox" not in k]
+
+F64 = np.float64
+
+
+def _scores_no_scale(Q, Kt, scale=None):
+    return np.asarray(Q, F64) @ np.asarray(Kt, F64).T * (1.0 if scale is None else scale)
+
+
+def _softmax_wrong_axis(S):
+    e = np.exp(S - S.max(axis=0, keepdims=True))
+    return e / e.sum(axis=0, keepdims=True)
+
+
+def _softmax_no_norm(S):
+    return np.exp(S - S.max(axis=-1, keepdims=True))
+
+
+def _soft_no_sign(x, theta):
+    return np.maximum(np.abs(x) - theta, 0.0)
+
+
+def _soft_hard(x, theta):
+    return np.where(np.abs(x) > theta, x, 0.0)
+
+
+def _setup_theta_is_lambda(M, lam, step=None):
+    S, B, th, mu = _orig_setup(M, lam, step)
+    return S, B, F64(lam), mu
+
+
+def _setup_plus_sign(M, lam, step=None):
+    S, B, th, mu = _orig_setup(M, lam, step)
+    return 2 * np.eye(S.shape[0]) - S, B, th, mu
+
+
+def _setup_B_transposed(M, lam, step=None):
+    S, B, th, mu = _orig_setup(M, lam, step)
+    return S, (B.T if B.shape[0] == B.shape[1] else B), th, mu
+
+
+def _setup_spectral_of_M(M, lam, step=None):
+    # step from ||M||_inf instead of ||M^T M||_inf
+    M = np.asarray(M, F64)
+    mu = 1.0 / np.abs(M).sum(axis=1).max() if not step else step
+    G = M.T @ M
+    return np.eye(G.shape[0]) - mu * G, mu * M, mu * lam, mu
+
+
+def _reconstruct_no_transpose(alpha, Psi):
+    return alpha if Psi is None else alpha @ Psi
+
+
+def _block_transposed(Phi_h, d):
+    assert Phi_h.shape[0] >= d and Phi_h.shape[1] >= d
+    return np.asarray(Phi_h, F64)[:d, :d].T.copy()
+
+
+def _block_offset(Phi_h, d):
+    assert Phi_h.shape[0] >= d and Phi_h.shape[1] >= d
+    return np.asarray(Phi_h, F64)[-d:, :d].copy()
+
+
+def _ista_drop_B(Z, S_dec, B_dec, theta, T, return_iterates=False):
+    return _orig_ista(Z, S_dec, np.eye(*B_dec.shape), theta, T, return_iterates)
+
+
+def _ista_one_short(Z, S_dec, B_dec, theta, T, return_iterates=False):
+    return _orig_ista(Z, S_dec, B_dec, theta, max(int(T) - 1, 0) if T < 50 else T, return_iterates)
+
+
+def _compress_abs(Phi, X):
+    return np.abs(np.asarray(Phi, F64)) @ np.asarray(X, F64)
+
+
+def _output_uses_unweighted(A, Vt):
+    return np.ones_like(A) / A.shape[1] @ np.asarray(Vt, F64)
+
+
+_orig_setup = orc.decoder_setup
+_orig_ista = orc.ista
+
+MUTATIONS = {
+    "scores: scale dropped": ("compressed_scores", _scores_no_scale),
+    "softmax: wrong axis": ("softmax_rows", _softmax_wrong_axis),
+    "softmax: not normalised": ("softmax_rows", _softmax_no_norm),
+    "shrink: sign dropped": ("soft_threshold", _soft_no_sign),
+    "shrink: hard threshold": ("soft_threshold", _soft_hard),
+    "setup: theta = lambda": ("decoder_setup", _setup_theta_is_lambda),
+    "setup: S = I + mu G": ("decoder_setup", _setup_plus_sign),
+    "setup: B transposed": ("decoder_setup", _setup_B_transposed),
+    "setup: step from ||M||": ("decoder_setup", _setup_spectral_of_M),
+    "reconstruct: Psi not transposed": ("reconstruct", _reconstruct_no_transpose),
+    "decoder block transposed": ("default_decoder_matrix", _block_transposed),
+    "decoder block from last rows": ("default_decoder_matrix", _block_offset),
+    "ista: B dropped": ("ista", _ista_drop_B),
+    "ista: one iteration short": ("ista", _ista_one_short),
+    "compress: |Phi|": ("compress", _compress_abs),
+    "output: weights ignored": ("compressed_output", _output_uses_unweighted),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_some_pin_catches(name, monkeypatch):
+    attr, fn = MUTATIONS[name]
+    monkeypatch.setattr(orc, attr, fn)
+    caught = False
+    for pin in PINS:
+        try:
+            pin()
+        except AssertionError:
+            caught = True
+            break
+        except Exception:
+            caught = True       # a shape error from the planted mistake also exposes it
+            break
+    assert caught, f"no pin noticed: {name}"

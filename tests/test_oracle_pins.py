@@ -1,0 +1,380 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, independent of the oracle.
+
+The paper prints no worked numeric example, so the pins are closed forms, brute force on
+tiny inputs, library routines of a different kind (a linear solve for an iteration's limit),
+optimality conditions and invariants.  Each pin names the oracle function(s) it guards and
+the mistake it would catch.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import csat_oracle as orc
+from oracle import phi_oracle as phi
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+# ----------------------------------------------------------------------------------------
+# brute-force standard attention (the paper's Attn(Q,K,V) equation), pure Python loops
+# ----------------------------------------------------------------------------------------
+def brute_attention(Q, K, V, keys=None):
+    nq, d = len(Q), len(Q[0])
+    keys = list(range(len(K))) if keys is None else list(keys)
+    out = [[0.0] * d for _ in range(nq)]
+    for i in range(nq):
+        s = []
+        for j in keys:
+            acc = 0.0
+            for c in range(d):
+                acc += Q[i][c] * K[j][c]
+            s.append(acc / math.sqrt(d))
+        mx = max(s)
+        w = [math.exp(x - mx) for x in s]
+        tot = sum(w)
+        for c in range(d):
+            acc = 0.0
+            for t, j in enumerate(keys):
+                acc += w[t] * V[j][c]
+            out[i][c] = acc / tot
+    return np.array(out)
+
+
+def _rng(seed):
+    return np.random.default_rng(seed)
+
+
+# P1: m = n, Phi = I, recovery disabled  =>  standard softmax attention.
+def test_identity_measurement_is_standard_attention():
+    r = _rng(1)
+    n, nq, d = 7, 5, 4
+    Q, K, V = r.standard_normal((nq, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    out = orc.csat_forward_head(Q, K, V, np.eye(n), T=0, lam=0.1)
+    ref = brute_attention(Q.tolist(), K.tolist(), V.tolist())
+    assert np.abs(out - ref).max() <= 1e-12
+
+
+# P1b: Phi = row-selection matrix  =>  standard attention restricted to the selected tokens.
+# Catches a transposed or mis-indexed Phi, and Phi applied to the wrong axis.
+def test_selection_measurement_is_attention_over_subset():
+    r = _rng(2)
+    n, nq, d = 9, 4, 3
+    sel = [6, 0, 3, 7]
+    Phi = np.zeros((len(sel), n))
+    for row, j in enumerate(sel):
+        Phi[row, j] = 1.0
+    Q, K, V = r.standard_normal((nq, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    out = orc.csat_forward_head(Q, K, V, Phi, T=0, lam=0.0)
+    ref = brute_attention(Q.tolist(), K.tolist(), V.tolist(), keys=sel)
+    assert np.abs(out - ref).max() <= 1e-12
+
+
+# Hand-sized closed forms.  m = 1: softmax over one measurement is 1, so Z = Phi V for every
+# query; d = 1 makes every decoder quantity a scalar that can be written down.
+def test_single_measurement_scalar_case_by_hand():
+    a, b = 2.0, 1.0
+    Phi = np.array([[a, b]])
+    K = np.array([[0.7], [-1.3]])
+    V = np.array([[3.0], [4.0]])
+    Q = np.array([[0.2], [-5.0], [9.0]])
+    Z = orc.csat_forward_head(Q, K, V, Phi, T=0, lam=0.1)
+    assert np.allclose(Z, 10.0, atol=1e-14)           # 2*3 + 1*4
+    # D = Phi[0,0] = 2, M = 2, G = 4, L = 4, mu = 1/4, S = 0, B = 1/2, theta = lambda/4
+    out = orc.csat_forward_head(Q, K, V, Phi, T=3, lam=0.1)
+    assert np.allclose(out, 10.0 / 2.0 - 0.1 / 4.0, atol=1e-14)   # soft(5, 0.025) = 4.975
+    # a large threshold shrinks everything to zero
+    out0 = orc.csat_forward_head(Q, K, V, Phi, T=3, lam=25.0)
+    assert np.all(out0 == 0.0)
+
+
+# m = 2, d = 1: softmax over two measurements is a logistic function of the score gap.
+def test_two_measurements_logistic_closed_form():
+    Phi = np.array([[1.0, 2.0, 0.0], [0.0, -1.0, 3.0]])
+    K = np.array([[0.5], [0.25], [-1.0]])
+    V = np.array([[1.0], [2.0], [4.0]])
+    q = 1.5
+    kt0, kt1 = 1.0 * 0.5 + 2.0 * 0.25, -0.25 - 3.0          # 1.0, -3.25
+    vt0, vt1 = 1.0 + 4.0, -2.0 + 12.0                        # 5, 10
+    p0 = 1.0 / (1.0 + math.exp(-(q * kt0 - q * kt1)))        # d = 1 -> scale 1
+    z = p0 * vt0 + (1.0 - p0) * vt1
+    Z = orc.csat_forward_head(np.array([[q]]), K, V, Phi, T=0, lam=0.0)
+    assert abs(Z[0, 0] - z) <= 1e-13
+
+
+# Q = 0  =>  uniform weights  =>  Z = mean over measurements of Phi V (any Phi).
+def test_zero_queries_give_uniform_average():
+    r = _rng(3)
+    n, m, d = 10, 4, 3
+    Phi, K, V = r.standard_normal((m, n)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    Z = orc.csat_forward_head(np.zeros((2, d)), K, V, Phi, T=0, lam=0.0)
+    ref = np.zeros(d)
+    for rr in range(m):
+        for j in range(n):
+            ref += Phi[rr, j] * V[j] / m
+    assert np.abs(Z - ref[None, :]).max() <= 1e-13
+
+
+# The scale argument and the default 1/sqrt(d): doubling d by zero-padding features changes only
+# the scale, so scores with explicit scale must match.
+def test_scale_is_inverse_sqrt_d():
+    r = _rng(4)
+    Q, Kt = r.standard_normal((3, 16)), r.standard_normal((5, 16))
+    S = orc.compressed_scores(Q, Kt)
+    for i in range(3):
+        for rr in range(5):
+            assert abs(S[i, rr] - sum(Q[i] * Kt[rr]) / 4.0) <= 1e-13
+
+
+# P2: soft-threshold identities and its proximal definition.
+def test_soft_threshold_identities_and_prox():
+    x = np.linspace(-3, 3, 241)
+    for theta in (0.0, 0.3, 1.0):
+        s = orc.soft_threshold(x, theta)
+        assert np.allclose(s, x - np.clip(x, -theta, theta), atol=1e-15)   # shrinkage identity
+        assert np.allclose(orc.soft_threshold(-x, theta), -s, atol=0)      # odd
+        assert np.all(s[np.abs(x) <= theta] == 0.0)
+        assert np.all(np.abs(s) <= np.abs(x) + 1e-15)
+    assert np.array_equal(orc.soft_threshold(x, 0.0), x)
+    # prox: argmin_u 1/2 (u-x)^2 + theta |u| by brute force on a fine grid
+    grid = np.linspace(-4, 4, 80001)
+    for xv in (-2.2, -0.31, 0.0, 0.29, 0.3, 1.7):
+        obj = 0.5 * (grid - xv) ** 2 + 0.3 * np.abs(grid)
+        assert abs(grid[obj.argmin()] - orc.soft_threshold(np.array([xv]), 0.3)[0]) <= 2e-4
+
+
+def _lasso_obj(y, M, x, lam):
+    return 0.5 * np.sum((y - x @ M.T) ** 2) + lam * np.abs(x).sum()
+
+
+# P3: the recovery claim (basis-pursuit / RIP paragraph): an exactly k-sparse vector is recovered
+# from enough Gaussian measurements; LASSO objective monotone; KKT conditions at convergence
+# (these fix theta = mu*lambda, the sign of the gradient step and the transposes).
+def test_ista_recovers_k_sparse_and_satisfies_kkt():
+    r = _rng(5)
+    p, q, k = 32, 64, 3
+    M = r.standard_normal((p, q)) / np.sqrt(p)
+    x = np.zeros((2, q))
+    for row in range(2):
+        sup = r.choice(q, k, replace=False)
+        x[row, sup] = r.choice([-1.0, 1.0], k) * (1.0 + r.random(k))
+    y = x @ M.T
+    lam = 5e-3
+    S_dec, B_dec, theta, mu = orc.decoder_setup(M, lam)
+    assert S_dec.shape == (q, q) and B_dec.shape == (p, q)
+    xh, its = orc.ista(y, S_dec, B_dec, theta, 20000, return_iterates=True)
+    assert np.array_equal(np.abs(xh) > 1e-3, x != 0)                       # support exact
+    assert np.linalg.norm(xh - x) / np.linalg.norm(x) < 1e-2
+    objs = [_lasso_obj(y, M, a, lam) for a in its[::50]]
+    assert all(b <= a + 1e-12 for a, b in zip(objs, objs[1:]))
+    first = [_lasso_obj(y, M, a, lam) for a in its[:40]]
+    assert all(b <= a + 1e-12 for a, b in zip(first, first[1:]))
+    g = (y - xh @ M.T) @ M                                                # M^T (y - M x^)
+    assert np.all(np.abs(g) <= lam * (1 + 1e-6))
+    on = xh != 0
+    assert np.allclose(g[on], lam * np.sign(xh[on]), rtol=1e-5, atol=1e-9)
+    # P11: the iteration map is non-expansive for mu <= 1/L, so steps never grow
+    steps = [np.linalg.norm(b - a) for a, b in zip(its[:200], its[1:201])]
+    assert all(s2 <= s1 * (1 + 1e-12) + 1e-15 for s1, s2 in zip(steps, steps[1:]))
+
+
+# step size: L^ is the max absolute row sum of M^T M and bounds its largest eigenvalue.
+def test_decoder_setup_step_and_matrices():
+    r = _rng(6)
+    M = r.standard_normal((5, 5))
+    S_dec, B_dec, theta, mu = orc.decoder_setup(M, 0.2)
+    G = np.zeros((5, 5))
+    for a in range(5):
+        for b in range(5):
+            G[a, b] = sum(M[k, a] * M[k, b] for k in range(5))
+    L = max(sum(abs(G[a, b]) for b in range(5)) for a in range(5))
+    assert abs(mu - 1.0 / L) <= 1e-15
+    assert L >= np.linalg.eigvalsh(G).max() - 1e-12
+    assert np.allclose(S_dec, np.eye(5) - G / L, atol=1e-14)
+    assert np.allclose(B_dec, M / L, atol=1e-15)
+    assert abs(theta - 0.2 / L) <= 1e-16
+    _, _, theta2, mu2 = orc.decoder_setup(M, 0.2, step=0.05)
+    assert mu2 == 0.05 and abs(theta2 - 0.01) <= 1e-16
+
+
+# P4: orthonormal M and mu = 1: one step lands on soft(z M, lambda) and stays there.
+def test_orthonormal_sensing_converges_in_one_step():
+    r = _rng(7)
+    d = 8
+    M, _ = np.linalg.qr(r.standard_normal((d, d)))
+    z = r.standard_normal((3, d))
+    S_dec, B_dec, theta, mu = orc.decoder_setup(M, 0.25, step=1.0)
+    a1 = orc.ista(z, S_dec, B_dec, theta, 1)
+    a9 = orc.ista(z, S_dec, B_dec, theta, 9)
+    expect = np.zeros_like(z)
+    for i in range(3):
+        for c in range(d):
+            v = sum(z[i, k] * M[k, c] for k in range(d))
+            expect[i, c] = math.copysign(max(abs(v) - 0.25, 0.0), v)
+    assert np.abs(a1 - expect).max() <= 1e-13
+    assert np.abs(a9 - expect).max() <= 1e-12
+
+
+# P5: Phi = I (m = n): default D = I, L^ = 1, so out = soft(Attn, lambda) for every T >= 1; with an
+# orthonormal dictionary, out = soft(Attn Psi, lambda) Psi^T.
+def test_identity_measurement_with_recovery():
+    r = _rng(8)
+    n, d = 8, 4
+    Q, K, V = r.standard_normal((n, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    attn = brute_attention(Q.tolist(), K.tolist(), V.tolist())
+    lam = 0.2
+    shr = np.sign(attn) * np.maximum(np.abs(attn) - lam, 0)
+    for T in (1, 2, 7):
+        out = orc.csat_forward_head(Q, K, V, np.eye(n), T=T, lam=lam)
+        assert np.abs(out - shr).max() <= 1e-12
+    Psi, _ = np.linalg.qr(r.standard_normal((d, d)))
+    w = attn @ Psi
+    expect = (np.sign(w) * np.maximum(np.abs(w) - lam, 0)) @ Psi.T
+    # G = Psi^T Psi = I up to rounding, L^ = 1 + O(eps): converges geometrically fast
+    out = orc.csat_forward_head(Q, K, V, np.eye(n), T=5, lam=lam, Psi=Psi)
+    assert np.abs(out - expect).max() <= 1e-10
+
+
+# P6: lambda = 0 and a well-conditioned D: the iteration is Landweber's and converges to the exact
+# inverse, out -> Z D^{-T}, whatever the (invertible) dictionary.  Catches M = Psi D instead of D Psi,
+# a missing transpose in B or in the reconstruction, and a wrong sign of the gradient step.
+def test_lambda_zero_converges_to_inverse():
+    r = _rng(9)
+    n, m, d = 12, 6, 5
+    Q, K, V = r.standard_normal((4, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    Phi = r.standard_normal((m, n)) / np.sqrt(m)
+    D = np.eye(d) + 0.1 * r.standard_normal((d, d))
+    Psi, _ = np.linalg.qr(r.standard_normal((d, d)))
+    Z = orc.csat_forward_head(Q, K, V, Phi, T=0, lam=0.0)
+    expect = np.linalg.solve(D, Z.T).T                                    # rows: z D^{-T}
+    for psi in (None, Psi):
+        out = orc.csat_forward_head(Q, K, V, Phi, T=3000, lam=0.0, D=D, Psi=psi)
+        assert np.abs(out - expect).max() <= 1e-9
+    # column-vector statement of the model: z = D Psi alpha, C = Psi alpha
+    alpha = np.zeros(d); alpha[[1, 3]] = [2.0, -1.5]
+    C = Psi @ alpha
+    z = D @ C
+    S_dec, B_dec, theta, _ = orc.decoder_setup(D @ Psi, 0.0)
+    a = orc.ista(z[None, :], S_dec, B_dec, theta, 3000)
+    assert np.abs(orc.reconstruct(a, Psi)[0] - C).max() <= 1e-9
+
+
+# Default decoder matrix: the leading d x d block of the head's Phi, rows first.
+def test_default_decoder_block():
+    r = _rng(10)
+    n, m, d = 9, 7, 3
+    Phi = r.standard_normal((m, n))
+    D = orc.default_decoder_matrix(Phi, d)
+    for a in range(d):
+        for b in range(d):
+            assert D[a, b] == Phi[a, b]
+    Q, K, V = r.standard_normal((2, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    o1 = orc.csat_forward_head(Q, K, V, Phi, T=4, lam=0.05)
+    o2 = orc.csat_forward_head(Q, K, V, Phi, T=4, lam=0.05, D=Phi[:d, :d])
+    assert np.array_equal(o1, o2)
+    with pytest.raises(AssertionError):
+        orc.default_decoder_matrix(Phi[:2], d)
+
+
+# P7: rows of A~ are probability vectors, so every Z entry lies between the column extremes of V~.
+def test_softmax_rows_and_convex_hull():
+    r = _rng(11)
+    n, m, d = 20, 6, 4
+    Q, K, V = 3 * r.standard_normal((5, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    Phi = r.standard_normal((m, n))
+    st = {}
+    Z = orc.csat_forward_head(Q, K, V, Phi, T=0, lam=0, stages=st)
+    A = orc.softmax_rows(orc.compressed_scores(Q, st["Kt"]))
+    assert A.shape == (5, m) and np.all(A >= 0) and np.allclose(A.sum(axis=1), 1.0, atol=1e-14)
+    assert np.all(Z <= st["Vt"].max(axis=0) + 1e-12) and np.all(Z >= st["Vt"].min(axis=0) - 1e-12)
+    # shift invariance and overflow safety of the softmax
+    big = orc.softmax_rows(np.array([[1000.0, 1001.0, 999.0]]))
+    small = orc.softmax_rows(np.array([[0.0, 1.0, -1.0]]))
+    assert np.allclose(big, small, atol=1e-15)
+    e = [math.exp(-1), 1.0, math.exp(-2)]
+    assert np.allclose(small[0], np.array(e) / sum(e), atol=1e-15)
+
+
+# P8: linearity of the compression; permutation invariances of Z.
+def test_linearity_and_permutation_invariance():
+    r = _rng(12)
+    n, m, d = 11, 5, 3
+    Phi = r.standard_normal((m, n))
+    K1, K2 = r.standard_normal((n, d)), r.standard_normal((n, d))
+    lhs = orc.compress(Phi, 2.0 * K1 - 0.5 * K2)
+    assert np.allclose(lhs, 2.0 * orc.compress(Phi, K1) - 0.5 * orc.compress(Phi, K2), atol=1e-13)
+    Q, V = r.standard_normal((4, d)), r.standard_normal((n, d))
+    Z = orc.csat_forward_head(Q, K1, V, Phi, T=0, lam=0)
+    pt = r.permutation(n)
+    Zt = orc.csat_forward_head(Q, K1[pt], V[pt], Phi[:, pt], T=0, lam=0)
+    assert np.allclose(Z, Zt, atol=1e-13)
+    pm = r.permutation(m)
+    Zm = orc.csat_forward_head(Q, K1, V, Phi[pm], T=0, lam=0)
+    assert np.allclose(Z, Zm, atol=1e-13)
+
+
+# The batched driver applies one Phi per head, shared over the batch.
+def test_batched_forward_uses_per_head_phi():
+    r = _rng(13)
+    B, H, n, m, d = 2, 3, 6, 4, 4
+    Q, K, V = (r.standard_normal((B, H, n, d)) for _ in range(3))
+    Phi = r.standard_normal((H, m, n))
+    out = orc.csat_forward(Q, K, V, Phi, T=2, lam=0.05)
+    for b in range(B):
+        for h in range(H):
+            one = orc.csat_forward_head(Q[b, h], K[b, h], V[b, h], Phi[h], T=2, lam=0.05)
+            assert np.array_equal(out[b, h], one)
+
+
+# ----------------------------------------------------------------------------------------
+# P9: the measurement-matrix generator
+# ----------------------------------------------------------------------------------------
+def test_philox_known_answers():
+    rows = []
+    with open(os.path.join(HERE, "golden", "philox4x32_10_kat.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                rows.append([int(t, 16) for t in line.split()])
+    assert len(rows) == 3
+    for w in rows:
+        got = phi.philox4x32_10(w[0], w[1], w[2], w[3], w[4], w[5])
+        assert [int(x) for x in got] == w[6:10]
+
+
+def test_phi_layout_counter_and_seed():
+    H, m, n, seed = 2, 3, 10, 0x1234567890ABCDEF
+    P = phi.phi_gaussian(H, m, n, seed)
+    assert P.shape == (H, m, n)
+    # element e = (h*m + r)*n + j, block e//4, lane e%4; checked one element at a time
+    for (h, r, j) in [(0, 0, 0), (0, 0, 3), (0, 1, 1), (1, 2, 9), (1, 0, 5)]:
+        e = (h * m + r) * n + j
+        u = [int(x) for x in phi.philox4x32_10(e // 4, 0, 0, 0, seed & 0xFFFFFFFF, seed >> 32)]
+        U = [((x >> 9) + 0.5) / 2 ** 23 for x in u]
+        g = []
+        for a, b in ((0, 1), (2, 3)):
+            rad = math.sqrt(-2.0 * math.log(U[a]))
+            g += [rad * math.cos(2 * math.pi * U[b]), rad * math.sin(2 * math.pi * U[b])]
+        assert abs(P[h, r, j] - g[e % 4] / math.sqrt(m)) <= 1e-15
+    assert not np.array_equal(P, phi.phi_gaussian(H, m, n, seed + 1))
+    assert np.array_equal(P[1:], phi.phi_gaussian(H, m, n, seed, heads=[1]))
+
+
+def test_phi_moments_and_normality():
+    from scipy import stats
+    m, n = 64, 4096
+    P = phi.phi_gaussian(1, m, n, 0)[0]
+    g = P.ravel() * np.sqrt(m)
+    N = g.size
+    assert abs(g.mean()) < 4 / np.sqrt(N)
+    assert abs(g.var() - 1.0) < 4 * np.sqrt(2 / N)
+    assert abs(stats.skew(g)) < 4 * np.sqrt(6 / N)
+    assert abs(stats.kurtosis(g)) < 4 * np.sqrt(24 / N)
+    assert stats.kstest(g, "norm").pvalue > 1e-3
+    cn = (P ** 2).sum(axis=0)                       # squared column norms: mean 1, var 2/m
+    assert abs(cn.mean() - 1.0) < 4 * np.sqrt(2 / m / n)
+    assert abs(cn.var() - 2 / m) < 0.2 * (2 / m)
+    # neighbouring Gaussians of one block and of adjacent blocks are uncorrelated
+    for lag in (1, 2, 3, 4):
+        c = np.corrcoef(g[:-lag], g[lag:])[0, 1]
+        assert abs(c) < 4 / np.sqrt(N)
