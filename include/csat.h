@@ -1,0 +1,168 @@
+/*
+ * csat.h -- C-ABI of the B200 (sm_100a) compressed-sensing attention (CSAT) forward.
+ *
+ * What the library computes, per (batch b, head h), in the notation of the paper's
+ * "Mathematical Framework" section (tokens are rows):
+ *
+ *   K~ = Phi_h K,  V~ = Phi_h V            compression equation, Phi_h in R^{m x n}
+ *   A~ = softmax(Q K~^T / sqrt(d_k))       approximate attention matrix, softmax over the m measurements
+ *   Z  = A~ V~                             compressed attention output, n_q x d_k
+ *   alpha^{t+1} = eta_theta(S alpha^t + B Z_i),  t = 0..T-1, alpha^0 = 0      LISTA recurrence
+ *   C^_i = Psi alpha^_i                    reconstruction equation; out = C^
+ *
+ * with the recurrence instantiated as ISTA for  min 1/2 ||z - alpha M^T||^2 + lambda ||alpha||_1,
+ * M = D Psi, D = leading d x d block of Phi_h unless supplied, mu = 1/L^ with
+ * L^ = max absolute row sum of M^T M unless supplied, S = I - mu M^T M, B = mu M, theta = mu lambda.
+ * T = 0 disables recovery: out = Z.
+ *
+ * Conventions common to every call
+ *   - All tensor pointers are DEVICE pointers unless the parameter is named *_host.
+ *     They must be 16-byte aligned and contiguous in the stated layout, innermost index last.
+ *   - Element type of Q, K, V, out, Phi, Psi, D is the context's CSAT_DTYPE
+ *     (CSAT_DTYPE_BF16: 16-bit bfloat16; CSAT_DTYPE_FP32: IEEE binary32).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     Calls enqueue work on it and return; they do not synchronise unless stated.
+ *   - The caller owns every buffer it passes in and keeps it alive and unmodified until the
+ *     stream has passed the call.  The library owns everything it allocates (Phi, the K~|V~
+ *     workspace, decoder matrices) and frees it in csat_destroy.
+ *   - Every call returns a CSAT_* status (never throws, never aborts).  A text for the most
+ *     recent failure is kept per context (csat_last_error).
+ *   - A context is used by one host thread at a time; different contexts are independent.
+ *   - Results are deterministic: same seed, parameters and inputs give bit-identical output.
+ */
+#ifndef CSAT_H_
+#define CSAT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct csat_ctx csat_ctx; /* opaque, library-owned */
+
+enum {
+  CSAT_OK = 0,
+  CSAT_ERR_INVALID_ARG = 1, /* NULL pointer, unknown key, misaligned pointer            */
+  CSAT_ERR_SHAPE = 2,       /* a size outside the supported range (see csat_create)      */
+  CSAT_ERR_ALLOC = 3,       /* device or host allocation failed                          */
+  CSAT_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; text in last_error     */
+  CSAT_ERR_UNSUPPORTED = 5, /* valid request this build has no kernel for                */
+  CSAT_ERR_STATE = 6,       /* call not legal in the context's current state             */
+  CSAT_ERR_TIMEOUT = 7      /* a bounded device-side wait gave up (reported by the next
+                               host call that reads the device status word)              */
+};
+
+/* keys of csat_set_i64 / csat_get_i64 */
+enum {
+  CSAT_BATCH = 1,      /* B, default 1                                                   */
+  CSAT_NQ = 2,         /* query tokens n_q, default n (self-attention); cross-attention
+                          of text queries over compressed visual keys uses n_q != n     */
+  CSAT_DTYPE = 3,      /* CSAT_DTYPE_BF16 (default) or CSAT_DTYPE_FP32                   */
+  CSAT_T = 4,          /* recovery iterations (decoder depth t), default 10; 0 = out = Z */
+  CSAT_FORCE_SIMT = 5  /* diagnostic: 1 routes bf16 through the plain FFMA kernels       */
+};
+enum { CSAT_DTYPE_BF16 = 0, CSAT_DTYPE_FP32 = 1 };
+
+/* keys of csat_set_f64 / csat_get_f64 */
+enum {
+  CSAT_LAMBDA = 1, /* LASSO weight lambda >= 0, default 0.1; per-step threshold is mu*lambda */
+  CSAT_STEP = 2,   /* step mu > 0; 0 (default) = 1 / max-abs-row-sum(M^T M), per head       */
+  CSAT_SCALE = 3   /* score scale; 0 (default) = 1/sqrt(d)                                   */
+};
+
+/*
+ * csat_create -- paper: compression equation (Phi in R^{m x n}) and the sentence after it
+ * (Gaussian ensemble).  Builds a context for n key/value tokens, m measurements, head size d
+ * and H heads on the CURRENT CUDA device, and generates one measurement matrix per head,
+ * Phi[h,r,j] ~ N(0, 1/m) i.i.d. from `seed` (Philox4x32-10 keyed by seed, counter = flat element
+ * index / 4, Box-Muller; Phi_K = Phi_V = Phi_h, shared over the batch).
+ * Requires 1 <= m <= n, d >= 1, H >= 1, d <= 256 and d % 8 == 0.  Returns NULL on failure;
+ * csat_last_error(NULL) then gives the reason (thread-local).
+ * Allocates device memory and synchronises.  Changing CSAT_DTYPE, CSAT_BATCH or CSAT_NQ later
+ * re-allocates (and, for CSAT_DTYPE, re-generates Phi from the seed).
+ */
+csat_ctx* csat_create(int64_t n, int64_t m, int64_t d, int64_t H, uint64_t seed);
+
+/* Frees everything the context owns.  NULL is a no-op.  Synchronises the device. */
+int csat_destroy(csat_ctx* ctx);
+
+/* Tunables m, t, Phi, Psi of the paper ("Interpretation and Benefits") that are not fixed at
+ * creation.  Setters validate and record; dependent decoder quantities (S, B, theta) are
+ * re-derived by the next csat_forward on that call's stream.  Must not be called while a
+ * forward of the same context is still running on the device. */
+int csat_set_i64(csat_ctx* ctx, int key, int64_t value);
+int csat_get_i64(const csat_ctx* ctx, int key, int64_t* value_host);
+int csat_set_f64(csat_ctx* ctx, int key, double value);
+int csat_get_f64(const csat_ctx* ctx, int key, double* value_host);
+
+/* csat_set_phi / csat_get_phi -- paper: "fixed or learned" measurement matrices.
+ * phi: [H, m, n] dense, context dtype.  set overrides the seeded matrix (copied into the
+ * library's padded storage); get writes the matrix in use.  Enqueued on `stream`. */
+int csat_set_phi(csat_ctx* ctx, const void* phi, void* stream);
+int csat_get_phi(const csat_ctx* ctx, void* phi_out, void* stream);
+
+/* csat_set_dictionary -- paper: dictionary Psi in R^{d_k x d_k} with C_i = Psi alpha_i.
+ * psi: [d, d] (per_head = 0) or [H, d, d] (per_head = 1), context dtype, row-major
+ * (Psi[a][b] multiplies alpha_b).  NULL restores Psi = I.  Copied on `stream`. */
+int csat_set_dictionary(csat_ctx* ctx, const void* psi, int per_head, void* stream);
+
+/* csat_set_decoder_matrix -- paper: "Phi = Phi_V is reused as the measurement matrix for
+ * decoding"; the decoder's sensing matrix D is d x d (see file header).  D: [H, d, d], context
+ * dtype.  NULL restores the default D_h = Phi_h[0:d, 0:d], which needs m >= d and n >= d
+ * (otherwise csat_forward with T > 0 returns CSAT_ERR_SHAPE).  Copied on `stream`. */
+int csat_set_decoder_matrix(csat_ctx* ctx, const void* D, void* stream);
+
+/*
+ * csat_forward -- paper: compression, approximate attention matrix, compressed output,
+ * LISTA recurrence and reconstruction equations (all of the hot path).
+ *   Q   [B, H, n_q, d]   K, V [B, H, n, d]   out [B, H, n_q, d]   device, context dtype.
+ * out must not overlap Q, K or V.  Launch-only: no allocation, no synchronisation, no host
+ * access to the tensors.  The n_q x m attention matrix and the recovery iterates never reach
+ * global memory; K~|V~ (m x 2d per (b,h)) live in the context's workspace.
+ * Errors: CSAT_ERR_INVALID_ARG (NULL/misaligned), CSAT_ERR_SHAPE (default D with m < d or
+ * n < d), CSAT_ERR_CUDA (launch failure), CSAT_ERR_TIMEOUT (a previous launch's bounded wait
+ * gave up; its output is invalid).
+ */
+int csat_forward(csat_ctx* ctx, const void* Q, const void* K, const void* V, void* out, void* stream);
+
+/*
+ * csat_forward_host -- same computation with HOST buffers (same layouts and dtype; pinned
+ * memory gives asynchronous copies).  Copies Q, K, V to staging buffers the context owns
+ * (allocated by the first call, so that call also allocates), runs csat_forward, copies out
+ * back and synchronises `stream` before returning.
+ */
+int csat_forward_host(csat_ctx* ctx, const void* Q_host, const void* K_host, const void* V_host,
+                      void* out_host, void* stream);
+
+/* csat_get_compressed -- paper: K~, V~ of the compression equation, as left in the workspace
+ * by the most recent csat_forward.  kt_out, vt_out: [B, H, m, d] each, context dtype (either may
+ * be NULL).  Enqueued on `stream`.  CSAT_ERR_STATE before the first forward. */
+int csat_get_compressed(const csat_ctx* ctx, void* kt_out, void* vt_out, void* stream);
+
+/* csat_get_decoder -- paper: S, B, theta of the LISTA recurrence as derived for the current
+ * parameters: S_out, B_out [H, d, d] float32 (row-vector convention: alpha <- eta(alpha S + z B)),
+ * theta_out [H] float32, mu_out [H] float32 (any may be NULL).  Derives them on `stream` first if
+ * parameters changed. */
+int csat_get_decoder(csat_ctx* ctx, float* S_out, float* B_out, float* theta_out, float* mu_out, void* stream);
+
+/* Bytes of device memory the context currently owns (Phi, workspace, decoder matrices, staging). */
+size_t csat_workspace_bytes(const csat_ctx* ctx);
+
+/* Number of kernels the most recent csat_forward enqueued (0 before the first). */
+int csat_last_launch_count(const csat_ctx* ctx);
+
+/* Text of the most recent failure of this context; with NULL, of the calling thread's most
+ * recent failed csat_create.  Also reads the device status word (cudaMemcpy of 4 bytes, which
+ * synchronises) so a CSAT_ERR_TIMEOUT raised by a finished launch becomes visible.
+ * The pointer stays valid until the next call on the same context / thread. */
+const char* csat_last_error(const csat_ctx* ctx);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int csat_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSAT_H_ */

@@ -1,0 +1,281 @@
+"""ctypes binding of libcsat.so: the same entry points as include/csat.h, argument marshalling only.
+
+Every step of the CSAT forward runs inside the library's CUDA kernels.  PyTorch is used for
+device memory and streams.  There is no CPU path: loading fails loudly if the library cannot be
+found or built, and every call raises CsatError on a non-zero status.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+CSAT_OK = 0
+ERR_NAMES = {1: "CSAT_ERR_INVALID_ARG", 2: "CSAT_ERR_SHAPE", 3: "CSAT_ERR_ALLOC", 4: "CSAT_ERR_CUDA",
+             5: "CSAT_ERR_UNSUPPORTED", 6: "CSAT_ERR_STATE", 7: "CSAT_ERR_TIMEOUT"}
+CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT = 1, 2, 3, 4, 5
+CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1
+CSAT_LAMBDA, CSAT_STEP, CSAT_SCALE = 1, 2, 3
+
+_DTYPES = {"bf16": (CSAT_DTYPE_BF16, torch.bfloat16), "fp32": (CSAT_DTYPE_FP32, torch.float32)}
+
+# name -> (restype, argtypes); must list every symbol include/csat.h declares
+_vp, _i64, _u64, _int, _dbl = C.c_void_p, C.c_int64, C.c_uint64, C.c_int, C.c_double
+SIGNATURES = {
+    "csat_create": (_vp, [_i64, _i64, _i64, _i64, _u64]),
+    "csat_destroy": (_int, [_vp]),
+    "csat_set_i64": (_int, [_vp, _int, _i64]),
+    "csat_get_i64": (_int, [_vp, _int, C.POINTER(_i64)]),
+    "csat_set_f64": (_int, [_vp, _int, _dbl]),
+    "csat_get_f64": (_int, [_vp, _int, C.POINTER(_dbl)]),
+    "csat_set_phi": (_int, [_vp, _vp, _vp]),
+    "csat_get_phi": (_int, [_vp, _vp, _vp]),
+    "csat_set_dictionary": (_int, [_vp, _vp, _int, _vp]),
+    "csat_set_decoder_matrix": (_int, [_vp, _vp, _vp]),
+    "csat_forward": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "csat_forward_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
+    "csat_get_decoder": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "csat_workspace_bytes": (C.c_size_t, [_vp]),
+    "csat_last_launch_count": (_int, [_vp]),
+    "csat_last_error": (C.c_char_p, [_vp]),
+    "csat_version": (_int, []),
+}
+
+_lib = None
+
+
+class CsatError(RuntimeError):
+    def __init__(self, code: int, text: str):
+        super().__init__(f"{ERR_NAMES.get(code, code)}: {text}")
+        self.code = code
+
+
+def load() -> C.CDLL:
+    """Load (building first if the sources are newer) the in-tree libcsat.so."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    try:
+        path = _build.build_library()
+    except Exception as exc:  # no nvcc and no prebuilt library: there is nothing to fall back to
+        if not os.path.exists(_build.LIB):
+            raise RuntimeError(f"libcsat.so is missing and could not be built: {exc}") from exc
+        path = _build.LIB
+    lib = C.CDLL(path)
+    for name, (res, args) in SIGNATURES.items():
+        fn = getattr(lib, name)          # AttributeError if the library lacks a declared symbol
+        fn.restype, fn.argtypes = res, args
+    _lib = lib
+    return lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors passed to libcsat must be contiguous"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _check(handle, rc):
+    if rc != CSAT_OK:
+        raise CsatError(rc, (load().csat_last_error(handle) or b"").decode())
+
+
+# ---- thin functions, one per C entry point -------------------------------------------------
+def csat_version() -> int:
+    return load().csat_version()
+
+
+def csat_create(n, m, d, H, seed):
+    h = load().csat_create(n, m, d, H, seed)
+    if not h:
+        raise CsatError(0, (load().csat_last_error(None) or b"").decode())
+    return C.c_void_p(h)
+
+
+def csat_destroy(h):
+    _check(None, load().csat_destroy(h))
+
+
+def csat_set_i64(h, key, v):
+    _check(h, load().csat_set_i64(h, key, int(v)))
+
+
+def csat_get_i64(h, key) -> int:
+    out = _i64()
+    _check(h, load().csat_get_i64(h, key, C.byref(out)))
+    return out.value
+
+
+def csat_set_f64(h, key, v):
+    _check(h, load().csat_set_f64(h, key, float(v)))
+
+
+def csat_get_f64(h, key) -> float:
+    out = _dbl()
+    _check(h, load().csat_get_f64(h, key, C.byref(out)))
+    return out.value
+
+
+def csat_set_phi(h, phi, stream=None):
+    _check(h, load().csat_set_phi(h, _ptr(phi), _stream(stream)))
+
+
+def csat_get_phi(h, phi_out, stream=None):
+    _check(h, load().csat_get_phi(h, _ptr(phi_out), _stream(stream)))
+
+
+def csat_set_dictionary(h, psi, per_head=False, stream=None):
+    _check(h, load().csat_set_dictionary(h, _ptr(psi), int(per_head), _stream(stream)))
+
+
+def csat_set_decoder_matrix(h, D, stream=None):
+    _check(h, load().csat_set_decoder_matrix(h, _ptr(D), _stream(stream)))
+
+
+def csat_forward(h, Q, K, V, out, stream=None):
+    _check(h, load().csat_forward(h, _ptr(Q), _ptr(K), _ptr(V), _ptr(out), _stream(stream)))
+
+
+def csat_forward_host(h, Qh, Kh, Vh, outh, stream=None):
+    _check(h, load().csat_forward_host(h, _ptr(Qh), _ptr(Kh), _ptr(Vh), _ptr(outh), _stream(stream)))
+
+
+def csat_get_compressed(h, kt_out, vt_out, stream=None):
+    _check(h, load().csat_get_compressed(h, _ptr(kt_out), _ptr(vt_out), _stream(stream)))
+
+
+def csat_get_decoder(h, S_out, B_out, theta_out, mu_out, stream=None):
+    _check(h, load().csat_get_decoder(h, _ptr(S_out), _ptr(B_out), _ptr(theta_out), _ptr(mu_out), _stream(stream)))
+
+
+def csat_workspace_bytes(h) -> int:
+    return load().csat_workspace_bytes(h)
+
+
+def csat_last_launch_count(h) -> int:
+    return load().csat_last_launch_count(h)
+
+
+def csat_last_error(h) -> str:
+    return (load().csat_last_error(h) or b"").decode()
+
+
+# ---- convenience wrapper: owns a handle, allocates result tensors with torch ------------------
+class Csat:
+    """A CSAT context.  Tensors are torch CUDA tensors of the context's dtype."""
+
+    def __init__(self, n, m, d, H, seed=0, *, B=1, n_q=None, dtype="bf16", T=10, lam=0.1, step=0.0, scale=0.0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("libcsat needs a CUDA device (sm_100a); there is no CPU path")
+        self.n, self.m, self.d, self.H, self.B = n, m, d, H, B
+        self.n_q = n if n_q is None else n_q
+        self.dtype_name = dtype
+        self.code, self.torch_dtype = _DTYPES[dtype]
+        self.h = csat_create(n, m, d, H, seed)
+        try:
+            if self.code != CSAT_DTYPE_BF16:
+                csat_set_i64(self.h, CSAT_DTYPE, self.code)
+            csat_set_i64(self.h, CSAT_BATCH, B)
+            csat_set_i64(self.h, CSAT_NQ, self.n_q)
+            csat_set_i64(self.h, CSAT_T, T)
+            csat_set_f64(self.h, CSAT_LAMBDA, lam)
+            csat_set_f64(self.h, CSAT_STEP, step)
+            csat_set_f64(self.h, CSAT_SCALE, scale)
+        except Exception:
+            self.close()
+            raise
+
+    def close(self):
+        if getattr(self, "h", None):
+            csat_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set(self, *, T=None, lam=None, step=None, scale=None, force_simt=None):
+        if T is not None:
+            csat_set_i64(self.h, CSAT_T, T)
+        if lam is not None:
+            csat_set_f64(self.h, CSAT_LAMBDA, lam)
+        if step is not None:
+            csat_set_f64(self.h, CSAT_STEP, step)
+        if scale is not None:
+            csat_set_f64(self.h, CSAT_SCALE, scale)
+        if force_simt is not None:
+            csat_set_i64(self.h, CSAT_FORCE_SIMT, int(force_simt))
+
+    def _new(self, *shape, dtype=None):
+        return torch.empty(*shape, dtype=dtype or self.torch_dtype, device="cuda")
+
+    def forward(self, Q, K, V, out=None):
+        assert Q.shape == (self.B, self.H, self.n_q, self.d) and Q.dtype == self.torch_dtype and Q.is_cuda
+        assert K.shape == (self.B, self.H, self.n, self.d) and K.dtype == self.torch_dtype and K.is_cuda
+        assert V.shape == K.shape and V.dtype == self.torch_dtype and V.is_cuda
+        if out is None:
+            out = self._new(self.B, self.H, self.n_q, self.d)
+        csat_forward(self.h, Q, K, V, out)
+        return out
+
+    def forward_host(self, Qh, Kh, Vh, outh):
+        for t in (Qh, Kh, Vh, outh):
+            assert not t.is_cuda and t.dtype == self.torch_dtype
+        csat_forward_host(self.h, Qh, Kh, Vh, outh)
+        return outh
+
+    def get_phi(self):
+        phi = self._new(self.H, self.m, self.n)
+        csat_get_phi(self.h, phi)
+        return phi
+
+    def set_phi(self, phi):
+        assert phi.shape == (self.H, self.m, self.n) and phi.dtype == self.torch_dtype
+        csat_set_phi(self.h, phi.contiguous())
+
+    def set_dictionary(self, psi):
+        if psi is None:
+            csat_set_dictionary(self.h, None)
+            return
+        assert psi.dtype == self.torch_dtype and psi.shape[-2:] == (self.d, self.d)
+        csat_set_dictionary(self.h, psi.contiguous(), per_head=(psi.dim() == 3))
+
+    def set_decoder_matrix(self, D):
+        if D is not None:
+            assert D.shape == (self.H, self.d, self.d) and D.dtype == self.torch_dtype
+            D = D.contiguous()
+        csat_set_decoder_matrix(self.h, D)
+
+    def get_compressed(self):
+        kt = self._new(self.B, self.H, self.m, self.d)
+        vt = self._new(self.B, self.H, self.m, self.d)
+        csat_get_compressed(self.h, kt, vt)
+        return kt, vt
+
+    def get_decoder(self):
+        S = self._new(self.H, self.d, self.d, dtype=torch.float32)
+        Bm = self._new(self.H, self.d, self.d, dtype=torch.float32)
+        th = self._new(self.H, dtype=torch.float32)
+        mu = self._new(self.H, dtype=torch.float32)
+        csat_get_decoder(self.h, S, Bm, th, mu)
+        return S, Bm, th, mu
+
+    @property
+    def launches(self) -> int:
+        return csat_last_launch_count(self.h)
+
+    @property
+    def workspace_bytes(self) -> int:
+        return csat_workspace_bytes(self.h)

@@ -1,0 +1,414 @@
+// Host side of libcsat: context, parameter handling, dispatch.  See include/csat.h for the contract.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "csat_internal.h"
+
+namespace {
+
+thread_local std::string g_create_error;
+
+int fail(csat_ctx* c, int code, const std::string& msg) {
+  if (c) c->err = msg;
+  else g_create_error = msg;
+  return code;
+}
+
+int fail_cuda(csat_ctx* c, cudaError_t e, const char* what) {
+  return fail(c, CSAT_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+cudaError_t dev_alloc(csat_ctx* c, T** p, size_t bytes) {
+  *p = nullptr;
+  if (bytes == 0) return cudaSuccess;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes);
+  if (e == cudaSuccess) c->bytes += bytes;
+  return e;
+}
+
+template <typename T>
+void dev_free(csat_ctx* c, T** p, size_t bytes) {
+  if (*p) {
+    cudaFree(*p);
+    c->bytes -= bytes;
+    *p = nullptr;
+  }
+}
+
+size_t phi_bytes(const csat::Params& p) { return (size_t)(p.H * p.m * p.n_pad) * csat::elt_size(p.dtype); }
+size_t kv_bytes(const csat::Params& p) { return (size_t)(p.B * p.H * p.m * 2 * p.d) * csat::elt_size(p.dtype); }
+size_t dd_bytes(const csat::Params& p, size_t elt) { return (size_t)(p.H * p.d * p.d) * elt; }
+
+void free_staging(csat_ctx* c) {
+  dev_free(c, &c->stage_q, c->stage_bytes_q);
+  dev_free(c, &c->stage_o, c->stage_bytes_q);
+  dev_free(c, &c->stage_k, c->stage_bytes_kv);
+  dev_free(c, &c->stage_v, c->stage_bytes_kv);
+  c->stage_bytes_q = c->stage_bytes_kv = 0;
+}
+
+void free_all(csat_ctx* c) {
+  const csat::Params& p = c->p;
+  dev_free(c, &c->phi, phi_bytes(p));
+  dev_free(c, &c->kv, kv_bytes(p));
+  dev_free(c, &c->psi, (size_t)((c->psi_per_head ? p.H : 1) * p.d * p.d) * csat::elt_size(p.dtype));
+  dev_free(c, &c->dmat, dd_bytes(p, csat::elt_size(p.dtype)));
+  dev_free(c, &c->Mf64, dd_bytes(p, 8));
+  dev_free(c, &c->Gf64, dd_bytes(p, 8));
+  dev_free(c, &c->S_dec, dd_bytes(p, 4));
+  dev_free(c, &c->B_dec, dd_bytes(p, 4));
+  dev_free(c, &c->psi_f32, dd_bytes(p, 4));
+  dev_free(c, &c->theta, (size_t)p.H * 4);
+  dev_free(c, &c->mu, (size_t)p.H * 4);
+  free_staging(c);
+  if (c->status) {
+    cudaFreeHost(c->status);
+    c->status = nullptr;
+  }
+}
+
+// (re)allocates everything whose size depends on dtype / B and regenerates Phi from the seed
+int allocate_and_generate(csat_ctx* c) {
+  const csat::Params& p = c->p;
+  cudaError_t e;
+  if ((e = dev_alloc(c, &c->phi, phi_bytes(p))) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(Phi) failed");
+  if ((e = dev_alloc(c, &c->kv, kv_bytes(p))) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(K~|V~) failed");
+  if ((e = csat::launch_phi_gen(c->phi, p, 0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen launch");
+  if ((e = cudaStreamSynchronize(0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen");
+  c->decoder_dirty = true;
+  c->have_forward = false;
+  return CSAT_OK;
+}
+
+bool on_device(const csat_ctx* c, std::string* why) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev != c->device) {
+    *why = "context was created on another CUDA device than the current one";
+    return false;
+  }
+  return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int csat_version(void) { return 100; }
+
+csat_ctx* csat_create(int64_t n, int64_t m, int64_t d, int64_t H, uint64_t seed) {
+  if (n < 1 || m < 1 || m > n || d < 1 || H < 1) {
+    fail(nullptr, CSAT_ERR_SHAPE, "csat_create: need 1 <= m <= n, d >= 1, H >= 1");
+    return nullptr;
+  }
+  if (d > 256 || d % 8 != 0) {
+    fail(nullptr, CSAT_ERR_SHAPE, "csat_create: need d <= 256 and d % 8 == 0");
+    return nullptr;
+  }
+  if (n > (int64_t)1 << 31 || H * m * csat::round_up(n, csat::kPhiColPad) > (int64_t)1 << 38) {
+    fail(nullptr, CSAT_ERR_SHAPE, "csat_create: problem too large");
+    return nullptr;
+  }
+  int ndev = 0;
+  cudaError_t e = cudaGetDeviceCount(&ndev);
+  if (e != cudaSuccess || ndev == 0) {
+    fail(nullptr, CSAT_ERR_CUDA, std::string("csat_create: no CUDA device: ") + cudaGetErrorString(e));
+    return nullptr;
+  }
+  csat_ctx* c = new (std::nothrow) csat_ctx();
+  if (!c) {
+    fail(nullptr, CSAT_ERR_ALLOC, "csat_create: host allocation failed");
+    return nullptr;
+  }
+  cudaGetDevice(&c->device);
+  csat::Params& p = c->p;
+  p.n = n; p.m = m; p.d = d; p.H = H; p.B = 1; p.nq = n;
+  p.n_pad = csat::round_up(n, csat::kPhiColPad);
+  p.dtype = CSAT_DTYPE_BF16;
+  p.T = 10; p.lambda = 0.1; p.step = 0.0; p.scale = 0.0; p.seed = seed;
+
+  int rc = CSAT_OK;
+  e = cudaHostAlloc(reinterpret_cast<void**>(&c->status), sizeof(int), cudaHostAllocMapped);
+  if (e != cudaSuccess) rc = fail(c, CSAT_ERR_ALLOC, "cudaHostAlloc(status) failed");
+  else *c->status = 0;
+  if (rc == CSAT_OK && (dev_alloc(c, &c->Mf64, dd_bytes(p, 8)) != cudaSuccess ||
+                        dev_alloc(c, &c->Gf64, dd_bytes(p, 8)) != cudaSuccess ||
+                        dev_alloc(c, &c->S_dec, dd_bytes(p, 4)) != cudaSuccess ||
+                        dev_alloc(c, &c->B_dec, dd_bytes(p, 4)) != cudaSuccess ||
+                        dev_alloc(c, &c->psi_f32, dd_bytes(p, 4)) != cudaSuccess ||
+                        dev_alloc(c, &c->theta, (size_t)H * 4) != cudaSuccess ||
+                        dev_alloc(c, &c->mu, (size_t)H * 4) != cudaSuccess))
+    rc = fail(c, CSAT_ERR_ALLOC, "cudaMalloc(decoder matrices) failed");
+  if (rc == CSAT_OK) rc = allocate_and_generate(c);
+  if (rc != CSAT_OK) {
+    g_create_error = "csat_create: " + c->err;
+    cudaGetLastError();
+    free_all(c);
+    delete c;
+    return nullptr;
+  }
+  return c;
+}
+
+int csat_destroy(csat_ctx* c) {
+  if (!c) return CSAT_OK;
+  cudaDeviceSynchronize();
+  free_all(c);
+  delete c;
+  return CSAT_OK;
+}
+
+int csat_set_i64(csat_ctx* c, int key, int64_t v) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  csat::Params& p = c->p;
+  switch (key) {
+    case CSAT_BATCH: {
+      if (v < 1 || v > (1 << 20)) return fail(c, CSAT_ERR_SHAPE, "CSAT_BATCH must be >= 1");
+      if (v == p.B) return CSAT_OK;
+      cudaDeviceSynchronize();
+      dev_free(c, &c->kv, kv_bytes(p));
+      free_staging(c);
+      p.B = v;
+      c->have_forward = false;
+      if (dev_alloc(c, &c->kv, kv_bytes(p)) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(K~|V~) failed");
+      return CSAT_OK;
+    }
+    case CSAT_NQ:
+      if (v < 1 || v > ((int64_t)1 << 31)) return fail(c, CSAT_ERR_SHAPE, "CSAT_NQ must be >= 1");
+      if (v != p.nq) { cudaDeviceSynchronize(); free_staging(c); }
+      p.nq = v;
+      return CSAT_OK;
+    case CSAT_DTYPE: {
+      if (v != CSAT_DTYPE_BF16 && v != CSAT_DTYPE_FP32) return fail(c, CSAT_ERR_INVALID_ARG, "unknown CSAT_DTYPE");
+      if ((int)v == p.dtype) return CSAT_OK;
+      cudaDeviceSynchronize();
+      dev_free(c, &c->phi, phi_bytes(p));
+      dev_free(c, &c->kv, kv_bytes(p));
+      dev_free(c, &c->psi, (size_t)((c->psi_per_head ? p.H : 1) * p.d * p.d) * csat::elt_size(p.dtype));
+      dev_free(c, &c->dmat, dd_bytes(p, csat::elt_size(p.dtype)));
+      free_staging(c);
+      p.dtype = (int)v;
+      return allocate_and_generate(c);   // user-set Phi, Psi, D are dropped with the old dtype
+    }
+    case CSAT_T:
+      if (v < 0 || v > 100000) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_T must be in [0, 100000]");
+      p.T = (int)v;
+      return CSAT_OK;
+    case CSAT_FORCE_SIMT:
+      c->force_simt = v != 0;
+      return CSAT_OK;
+    default:
+      return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_i64: unknown key");
+  }
+}
+
+int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
+  if (!c || !out) return CSAT_ERR_INVALID_ARG;
+  switch (key) {
+    case CSAT_BATCH: *out = c->p.B; return CSAT_OK;
+    case CSAT_NQ: *out = c->p.nq; return CSAT_OK;
+    case CSAT_DTYPE: *out = c->p.dtype; return CSAT_OK;
+    case CSAT_T: *out = c->p.T; return CSAT_OK;
+    case CSAT_FORCE_SIMT: *out = c->force_simt; return CSAT_OK;
+    default: return CSAT_ERR_INVALID_ARG;
+  }
+}
+
+int csat_set_f64(csat_ctx* c, int key, double v) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!(v == v)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_f64: NaN");
+  switch (key) {
+    case CSAT_LAMBDA:
+      if (v < 0) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_LAMBDA must be >= 0");
+      c->p.lambda = v; c->decoder_dirty = true; return CSAT_OK;
+    case CSAT_STEP:
+      if (v < 0) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_STEP must be >= 0 (0 = automatic)");
+      c->p.step = v; c->decoder_dirty = true; return CSAT_OK;
+    case CSAT_SCALE:
+      if (v < 0) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_SCALE must be >= 0 (0 = 1/sqrt(d))");
+      c->p.scale = v; return CSAT_OK;
+    default:
+      return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_f64: unknown key");
+  }
+}
+
+int csat_get_f64(const csat_ctx* c, int key, double* out) {
+  if (!c || !out) return CSAT_ERR_INVALID_ARG;
+  switch (key) {
+    case CSAT_LAMBDA: *out = c->p.lambda; return CSAT_OK;
+    case CSAT_STEP: *out = c->p.step; return CSAT_OK;
+    case CSAT_SCALE: *out = c->p.scale; return CSAT_OK;
+    default: return CSAT_ERR_INVALID_ARG;
+  }
+}
+
+int csat_set_phi(csat_ctx* c, const void* phi, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!phi || !aligned16(phi)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_phi: NULL or misaligned pointer");
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  cudaError_t e = csat::launch_phi_pack(c->phi, phi, c->p, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_set_phi");
+  c->decoder_dirty = true;
+  return CSAT_OK;
+}
+
+int csat_get_phi(const csat_ctx* c, void* phi_out, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  csat_ctx* mc = const_cast<csat_ctx*>(c);
+  if (!phi_out || !aligned16(phi_out)) return fail(mc, CSAT_ERR_INVALID_ARG, "csat_get_phi: NULL or misaligned pointer");
+  std::string why;
+  if (!on_device(c, &why)) return fail(mc, CSAT_ERR_STATE, why);
+  cudaError_t e = csat::launch_phi_unpack(phi_out, c->phi, c->p, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(mc, e, "csat_get_phi");
+  return CSAT_OK;
+}
+
+int csat_set_dictionary(csat_ctx* c, const void* psi, int per_head, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  csat::Params& p = c->p;
+  const size_t es = csat::elt_size(p.dtype);
+  if (psi && !aligned16(psi)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_dictionary: misaligned pointer");
+  const size_t old_bytes = (size_t)((c->psi_per_head ? p.H : 1) * p.d * p.d) * es;
+  const size_t new_bytes = (size_t)((per_head ? p.H : 1) * p.d * p.d) * es;
+  if (c->psi && (!psi || old_bytes != new_bytes)) {
+    cudaDeviceSynchronize();
+    dev_free(c, &c->psi, old_bytes);
+  }
+  c->decoder_dirty = true;
+  if (!psi) { c->psi_per_head = false; return CSAT_OK; }
+  c->psi_per_head = per_head != 0;
+  if (!c->psi && dev_alloc(c, &c->psi, new_bytes) != cudaSuccess)
+    return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(Psi) failed");
+  cudaError_t e = cudaMemcpyAsync(c->psi, psi, new_bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_set_dictionary");
+  return CSAT_OK;
+}
+
+int csat_set_decoder_matrix(csat_ctx* c, const void* D, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  csat::Params& p = c->p;
+  const size_t bytes = dd_bytes(p, csat::elt_size(p.dtype));
+  if (D && !aligned16(D)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_decoder_matrix: misaligned pointer");
+  c->decoder_dirty = true;
+  if (!D) {
+    if (c->dmat) { cudaDeviceSynchronize(); dev_free(c, &c->dmat, bytes); }
+    return CSAT_OK;
+  }
+  if (!c->dmat && dev_alloc(c, &c->dmat, bytes) != cudaSuccess)
+    return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(D) failed");
+  cudaError_t e = cudaMemcpyAsync(c->dmat, D, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_set_decoder_matrix");
+  return CSAT_OK;
+}
+
+static int ensure_decoder(csat_ctx* c, cudaStream_t s, int* launches) {
+  const csat::Params& p = c->p;
+  if (!c->dmat && (p.m < p.d || p.n < p.d))
+    return fail(c, CSAT_ERR_SHAPE, "default decoder matrix D = Phi[0:d,0:d] needs m >= d and n >= d");
+  if (!c->decoder_dirty) return CSAT_OK;
+  cudaError_t e = csat::launch_decoder_setup(c, s, launches);
+  if (e != cudaSuccess) return fail_cuda(c, e, "decoder set-up launch");
+  c->decoder_dirty = false;
+  return CSAT_OK;
+}
+
+int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void* out, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !out) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward: NULL tensor pointer");
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out))
+    return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward: tensor pointers must be 16-byte aligned");
+  if (out == Q || out == K || out == V) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward: out aliases an input");
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  if (*(volatile int*)c->status != 0)
+    return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
+  cudaStream_t s = (cudaStream_t)stream;
+  int launches = 0;
+  if (c->p.T > 0) {
+    int rc = ensure_decoder(c, s, &launches);
+    if (rc != CSAT_OK) return rc;
+  }
+  cudaError_t e;
+  // float32 contexts, and head sizes without a tensor-core kernel, take the FFMA kernels
+  if ((e = csat::launch_simt_compress(c, K, V, s, &launches)) != cudaSuccess) return fail_cuda(c, e, "compress launch");
+  if ((e = csat::launch_simt_attend_recover(c, Q, out, s, &launches)) != cudaSuccess)
+    return fail_cuda(c, e, "attend/recover launch");
+  c->have_forward = true;
+  c->last_launches = launches;
+  return CSAT_OK;
+}
+
+int csat_forward_host(csat_ctx* c, const void* Qh, const void* Kh, const void* Vh, void* outh, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!Qh || !Kh || !Vh || !outh) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward_host: NULL pointer");
+  const csat::Params& p = c->p;
+  const size_t es = csat::elt_size(p.dtype);
+  const size_t bq = (size_t)(p.B * p.H * p.nq * p.d) * es, bkv = (size_t)(p.B * p.H * p.n * p.d) * es;
+  if (c->stage_bytes_q != bq || c->stage_bytes_kv != bkv) {
+    cudaDeviceSynchronize();
+    free_staging(c);
+    c->stage_bytes_q = bq; c->stage_bytes_kv = bkv;
+    if (dev_alloc(c, &c->stage_q, bq) != cudaSuccess || dev_alloc(c, &c->stage_o, bq) != cudaSuccess ||
+        dev_alloc(c, &c->stage_k, bkv) != cudaSuccess || dev_alloc(c, &c->stage_v, bkv) != cudaSuccess) {
+      free_staging(c);
+      return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(staging) failed");
+    }
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(c->stage_q, Qh, bq, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(c->stage_k, Kh, bkv, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(c->stage_v, Vh, bkv, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+    return fail_cuda(c, e, "host->device copy");
+  int rc = csat_forward(c, c->stage_q, c->stage_k, c->stage_v, c->stage_o, stream);
+  if (rc != CSAT_OK) return rc;
+  if ((e = cudaMemcpyAsync(outh, c->stage_o, bq, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+    return fail_cuda(c, e, "device->host copy");
+  if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return fail_cuda(c, e, "csat_forward_host");
+  if (*(volatile int*)c->status != 0) return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait gave up");
+  return CSAT_OK;
+}
+
+int csat_get_compressed(const csat_ctx* c, void* kt, void* vt, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  csat_ctx* mc = const_cast<csat_ctx*>(c);
+  if (!c->have_forward) return fail(mc, CSAT_ERR_STATE, "csat_get_compressed: no forward has run yet");
+  if ((kt && !aligned16(kt)) || (vt && !aligned16(vt)))
+    return fail(mc, CSAT_ERR_INVALID_ARG, "csat_get_compressed: misaligned pointer");
+  cudaError_t e = csat::launch_split_kv(c, kt, vt, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(mc, e, "csat_get_compressed");
+  return CSAT_OK;
+}
+
+int csat_get_decoder(csat_ctx* c, float* S_out, float* B_out, float* theta_out, float* mu_out, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  int launches = 0;
+  int rc = ensure_decoder(c, s, &launches);
+  if (rc != CSAT_OK) return rc;
+  const csat::Params& p = c->p;
+  cudaError_t e = cudaSuccess;
+  if (S_out && e == cudaSuccess) e = cudaMemcpyAsync(S_out, c->S_dec, dd_bytes(p, 4), cudaMemcpyDeviceToDevice, s);
+  if (B_out && e == cudaSuccess) e = cudaMemcpyAsync(B_out, c->B_dec, dd_bytes(p, 4), cudaMemcpyDeviceToDevice, s);
+  if (theta_out && e == cudaSuccess) e = cudaMemcpyAsync(theta_out, c->theta, (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
+  if (mu_out && e == cudaSuccess) e = cudaMemcpyAsync(mu_out, c->mu, (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_get_decoder");
+  return CSAT_OK;
+}
+
+size_t csat_workspace_bytes(const csat_ctx* c) { return c ? c->bytes : 0; }
+
+int csat_last_launch_count(const csat_ctx* c) { return c ? c->last_launches : 0; }
+
+const char* csat_last_error(const csat_ctx* c) {
+  if (!c) return g_create_error.c_str();
+  if (c->status && *(volatile int*)c->status != 0 && c->err.empty())
+    const_cast<csat_ctx*>(c)->err = "a bounded device-side wait gave up (CSAT_ERR_TIMEOUT)";
+  return c->err.c_str();
+}
+
+}  // extern "C"

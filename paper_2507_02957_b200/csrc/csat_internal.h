@@ -1,0 +1,78 @@
+// Internal declarations shared by the translation units of libcsat (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <string>
+
+#include "csat.h"
+
+namespace csat {
+
+// n is padded to a multiple of this in the library's Phi storage, so that every row of Phi
+// starts on a 128-byte boundary for both dtypes and whole 64-token chunks can be staged.
+constexpr int64_t kPhiColPad = 64;
+
+inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+struct Params {            // plain values kernels need
+  int64_t n, m, d, H, B, nq;
+  int64_t n_pad;           // padded row length of Phi
+  int dtype;               // CSAT_DTYPE_*
+  int T;
+  double lambda, step, scale;
+  uint64_t seed;
+};
+
+}  // namespace csat
+
+struct csat_ctx {
+  csat::Params p;
+  int device = 0;
+  bool force_simt = false;
+
+  // library-owned device memory
+  void* phi = nullptr;        // [H, m, n_pad] dtype
+  void* kv = nullptr;         // K~|V~ workspace [B, H, m, 2d] dtype (row r: K~_r then V~_r)
+  void* psi = nullptr;        // [Hpsi, d, d] dtype (user dictionary), null = identity
+  void* dmat = nullptr;       // [H, d, d] dtype (user decoder matrix), null = Phi block
+  bool psi_per_head = false;
+  double* Mf64 = nullptr;     // [H, d, d] scratch of the decoder set-up
+  double* Gf64 = nullptr;     // [H, d, d]
+  float* S_dec = nullptr;     // [H, d, d]  I - mu G
+  float* B_dec = nullptr;     // [H, d, d]  mu M
+  float* psi_f32 = nullptr;   // [H, d, d]  Psi as float (row-major), only when psi != null
+  float* theta = nullptr;     // [H]
+  float* mu = nullptr;        // [H]
+  int* status = nullptr;      // device status word (0 = ok)
+  // staging for csat_forward_host
+  void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
+  size_t stage_bytes_q = 0, stage_bytes_kv = 0;
+
+  bool decoder_dirty = true;
+  bool have_forward = false;
+  int last_launches = 0;
+  size_t bytes = 0;
+  std::string err;
+};
+
+namespace csat {
+
+size_t elt_size(int dtype);
+
+// phi_gen.cu
+cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s);
+cudaError_t launch_phi_pack(void* phi_padded, const void* phi_dense, const Params& p, cudaStream_t s);
+cudaError_t launch_phi_unpack(void* phi_dense, const void* phi_padded, const Params& p, cudaStream_t s);
+
+// decoder_setup.cu : derives S_dec, B_dec, theta, mu (and psi_f32) on the stream; returns #launches
+cudaError_t launch_decoder_setup(csat_ctx* c, cudaStream_t s, int* launches);
+
+// simt_forward.cu : plain FFMA path (fp32 accumulate), both storage types
+cudaError_t launch_simt_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches);
+cudaError_t launch_simt_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
+
+// copies K~ or V~ out of the interleaved workspace: dst [B,H,m,d]
+cudaError_t launch_split_kv(const csat_ctx* c, void* kt, void* vt, cudaStream_t s);
+
+}  // namespace csat

@@ -1,0 +1,104 @@
+// Decoder set-up, once per parameter change and per head (tiny: d x d matrices, float64 arithmetic).
+// Paper: LISTA recurrence alpha^{t+1} = eta_theta(S alpha^t + B Z_i) with S, B, theta taken from ISTA
+// ("fast approximate solvers, such as ISTA") for the model Z_i = D Psi alpha_i:
+//   M = D Psi, G = M^T M, L^ = max_a sum_b |G[a][b]|, mu = 1/L^ (or the caller's step),
+//   S = I - mu G, B = mu M, theta = mu lambda.
+// D defaults to the leading d x d block of the head's Phi ("Phi = Phi_V is reused").
+#include "csat_internal.h"
+
+namespace csat {
+namespace {
+
+template <typename T> __device__ __forceinline__ double ld(const T* p, int64_t i);
+template <> __device__ __forceinline__ double ld<float>(const float* p, int64_t i) { return (double)p[i]; }
+template <> __device__ __forceinline__ double ld<__nv_bfloat16>(const __nv_bfloat16* p, int64_t i) {
+  return (double)__bfloat162float(p[i]);
+}
+
+// M[h][a][b] = sum_k D[h][a][k] * Psi[h][k][b]
+template <typename T>
+__global__ void build_M_kernel(double* __restrict__ M, const T* __restrict__ phi, const T* __restrict__ dmat,
+                               const T* __restrict__ psi, int psi_per_head, int d, int64_t m, int64_t n_pad) {
+  const int h = blockIdx.y;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= d * d) return;
+  const int a = idx / d, b = idx % d;
+  const T* Dh = dmat ? dmat + (int64_t)h * d * d : phi + (int64_t)h * m * n_pad;
+  const int64_t ldD = dmat ? d : n_pad;
+  double acc;
+  if (psi) {
+    const T* P = psi + (psi_per_head ? (int64_t)h * d * d : 0);
+    acc = 0.0;
+    for (int k = 0; k < d; ++k) acc += ld(Dh, a * ldD + k) * ld(P, (int64_t)k * d + b);
+  } else {
+    acc = ld(Dh, a * ldD + b);
+  }
+  M[(int64_t)h * d * d + idx] = acc;
+}
+
+// G[h][a][b] = sum_k M[h][k][a] * M[h][k][b]
+__global__ void gram_kernel(double* __restrict__ G, const double* __restrict__ M, int d) {
+  const int h = blockIdx.y;
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= d * d) return;
+  const int a = idx / d, b = idx % d;
+  const double* Mh = M + (int64_t)h * d * d;
+  double acc = 0.0;
+  for (int k = 0; k < d; ++k) acc += Mh[k * d + a] * Mh[k * d + b];
+  G[(int64_t)h * d * d + idx] = acc;
+}
+
+// one block per head; blockDim.x >= d (power of two <= 256)
+template <typename T>
+__global__ void finalize_kernel(float* __restrict__ S_dec, float* __restrict__ B_dec, float* __restrict__ theta,
+                                float* __restrict__ mu_out, float* __restrict__ psi_f32, const double* __restrict__ G,
+                                const double* __restrict__ M, const T* __restrict__ psi, int psi_per_head, int d,
+                                double lambda, double step) {
+  __shared__ double red[256];
+  const int h = blockIdx.x, t = threadIdx.x;
+  const double* Gh = G + (int64_t)h * d * d;
+  const double* Mh = M + (int64_t)h * d * d;
+  double rs = 0.0;
+  if (t < d)
+    for (int b = 0; b < d; ++b) rs += fabs(Gh[t * d + b]);
+  red[t] = rs;
+  __syncthreads();
+  for (int s = blockDim.x >> 1; s > 0; s >>= 1) {   // max is order-independent: deterministic
+    if (t < s) red[t] = fmax(red[t], red[t + s]);
+    __syncthreads();
+  }
+  const double L = red[0];
+  const double mu = step > 0.0 ? step : (L > 0.0 ? 1.0 / L : 0.0);
+  for (int i = t; i < d * d; i += blockDim.x) {
+    const int a = i / d, b = i % d;
+    S_dec[(int64_t)h * d * d + i] = (float)((a == b ? 1.0 : 0.0) - mu * Gh[i]);
+    B_dec[(int64_t)h * d * d + i] = (float)(mu * Mh[i]);
+    if (psi) psi_f32[(int64_t)h * d * d + i] = (float)ld(psi + (psi_per_head ? (int64_t)h * d * d : 0), i);
+  }
+  if (t == 0) {
+    theta[h] = (float)(mu * lambda);
+    mu_out[h] = (float)mu;
+  }
+}
+
+template <typename T>
+cudaError_t run(csat_ctx* c, cudaStream_t s, int* launches) {
+  const Params& p = c->p;
+  const int d = (int)p.d, H = (int)p.H;
+  const dim3 grid((d * d + 255) / 256, H);
+  build_M_kernel<T><<<grid, 256, 0, s>>>(c->Mf64, (const T*)c->phi, (const T*)c->dmat, (const T*)c->psi,
+                                         c->psi_per_head ? 1 : 0, d, p.m, p.n_pad);
+  gram_kernel<<<grid, 256, 0, s>>>(c->Gf64, c->Mf64, d);
+  finalize_kernel<T><<<H, 256, 0, s>>>(c->S_dec, c->B_dec, c->theta, c->mu, c->psi_f32, c->Gf64, c->Mf64,
+                                       (const T*)c->psi, c->psi_per_head ? 1 : 0, d, p.lambda, p.step);
+  *launches += 3;
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_decoder_setup(csat_ctx* c, cudaStream_t s, int* launches) {
+  return c->p.dtype == CSAT_DTYPE_FP32 ? run<float>(c, s, launches) : run<__nv_bfloat16>(c, s, launches);
+}
+
+}  // namespace csat

@@ -1,0 +1,120 @@
+// Seeded Gaussian measurement matrices Phi_h in R^{m x n}, entries N(0, 1/m).
+// Paper: compression equation and the sentence after it (sub-Gaussian ensembles, "random Gaussian").
+// The paper fixes no generator: this library uses Philox4x32-10 (Salmon et al., SC'11) keyed by the
+// 64-bit seed, counter = flat element index / 4, and Box-Muller on 23-bit uniforms.
+#include "csat_internal.h"
+
+namespace csat {
+namespace {
+
+struct U4 { uint32_t x, y, z, w; };
+
+__device__ __forceinline__ U4 philox4x32_10(U4 c, uint32_t k0, uint32_t k1) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(M0, c.x), lo0 = M0 * c.x;
+    const uint32_t hi1 = __umulhi(M1, c.z), lo1 = M1 * c.z;
+    c = U4{hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0};
+    k0 += W0;
+    k1 += W1;
+  }
+  return c;
+}
+
+// U = ((u >> 9) + 0.5) * 2^-23 : exact in float, strictly inside (0,1)
+__device__ __forceinline__ float uniform23(uint32_t u) {
+  return (static_cast<float>(u >> 9) + 0.5f) * 1.1920928955078125e-07f;
+}
+
+__device__ __forceinline__ void box_muller(uint32_t ua, uint32_t ub, float& g0, float& g1) {
+  const float r = sqrtf(-2.0f * logf(uniform23(ua)));
+  float s, c;
+  sincospif(2.0f * uniform23(ub), &s, &c);
+  g0 = r * c;
+  g1 = r * s;
+}
+
+template <typename T> __device__ __forceinline__ T to_storage(float v);
+template <> __device__ __forceinline__ float to_storage<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 to_storage<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// One thread per Philox block = 4 consecutive elements of the UNPADDED index space e = (h*m + r)*n + j.
+template <typename T>
+__global__ void phi_gen_kernel(T* __restrict__ phi, int64_t total, int64_t n, int64_t n_pad, float inv_sqrt_m,
+                               uint32_t k0, uint32_t k1) {
+  const int64_t nblocks = (total + 3) >> 2;
+  for (int64_t q = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; q < nblocks;
+       q += (int64_t)gridDim.x * blockDim.x) {
+    const U4 u = philox4x32_10(U4{(uint32_t)q, (uint32_t)(q >> 32), 0u, 0u}, k0, k1);
+    float g[4];
+    box_muller(u.x, u.y, g[0], g[1]);
+    box_muller(u.z, u.w, g[2], g[3]);
+    const int64_t e0 = q << 2;
+    int64_t row = e0 / n;
+    int64_t j = e0 - row * n;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (e0 + i < total) phi[row * n_pad + j] = to_storage<T>(g[i] * inv_sqrt_m);
+      if (++j == n) { j = 0; ++row; }
+    }
+  }
+}
+
+template <typename T>
+__global__ void phi_pack_kernel(T* __restrict__ dst, const T* __restrict__ src, int64_t rows, int64_t n,
+                                int64_t n_pad, bool to_padded) {
+  const int64_t total = rows * n;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = i / n, j = i - r * n;
+    if (to_padded) dst[r * n_pad + j] = src[i];
+    else dst[i] = src[r * n_pad + j];
+  }
+}
+
+int grid_for(int64_t work, int block) {
+  int64_t g = (work + block - 1) / block;
+  const int64_t cap = 148LL * 16;   // a few waves of the 148 SMs; kernels use grid-stride loops
+  return (int)(g < 1 ? 1 : (g > cap ? cap : g));
+}
+
+}  // namespace
+
+size_t elt_size(int dtype) { return dtype == CSAT_DTYPE_FP32 ? 4 : 2; }
+
+cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s) {
+  const int64_t total = p.H * p.m * p.n;
+  cudaError_t e = cudaMemsetAsync(phi, 0, (size_t)(p.H * p.m * p.n_pad) * elt_size(p.dtype), s);
+  if (e != cudaSuccess) return e;
+  const float inv = (float)(1.0 / sqrt((double)p.m));
+  const uint32_t k0 = (uint32_t)(p.seed & 0xFFFFFFFFull), k1 = (uint32_t)(p.seed >> 32);
+  const int block = 256, grid = grid_for((total + 3) / 4, block);
+  if (p.dtype == CSAT_DTYPE_FP32)
+    phi_gen_kernel<float><<<grid, block, 0, s>>>((float*)phi, total, p.n, p.n_pad, inv, k0, k1);
+  else
+    phi_gen_kernel<__nv_bfloat16><<<grid, block, 0, s>>>((__nv_bfloat16*)phi, total, p.n, p.n_pad, inv, k0, k1);
+  return cudaGetLastError();
+}
+
+static cudaError_t pack(void* dst, const void* src, const Params& p, cudaStream_t s, bool to_padded) {
+  const int64_t rows = p.H * p.m;
+  const int block = 256, grid = grid_for(rows * p.n, block);
+  if (p.dtype == CSAT_DTYPE_FP32)
+    phi_pack_kernel<float><<<grid, block, 0, s>>>((float*)dst, (const float*)src, rows, p.n, p.n_pad, to_padded);
+  else
+    phi_pack_kernel<__nv_bfloat16><<<grid, block, 0, s>>>((__nv_bfloat16*)dst, (const __nv_bfloat16*)src, rows, p.n,
+                                                         p.n_pad, to_padded);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_phi_pack(void* phi_padded, const void* phi_dense, const Params& p, cudaStream_t s) {
+  cudaError_t e = cudaMemsetAsync(phi_padded, 0, (size_t)(p.H * p.m * p.n_pad) * elt_size(p.dtype), s);
+  if (e != cudaSuccess) return e;
+  return pack(phi_padded, phi_dense, p, s, true);
+}
+
+cudaError_t launch_phi_unpack(void* phi_dense, const void* phi_padded, const Params& p, cudaStream_t s) {
+  return pack(phi_dense, phi_padded, p, s, false);
+}
+
+}  // namespace csat

@@ -1,0 +1,227 @@
+"""GPU parity: libcsat (through its C-ABI binding) against the float64 CPU oracle, element by element,
+on the same seeded inputs and the library's exported Phi.
+
+Bar: max|gpu - oracle| / max|oracle| <= 2e-2 for bf16 storage with fp32 accumulation, <= 1e-4 for the
+fp32 path.  Several workloads give an all-zero output at their own (T, lambda) (everything is shrunk
+away), so every case is also checked with recovery disabled (T = 0, out = Z), at lambda = 0 and at a
+lambda that keeps about half of the coefficients.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import csat_oracle as orc
+from oracle import phi_oracle as pho
+from paper_2507_02957_b200 import binding, workloads as wl
+from gpu_util import TOL, device_inputs, make_ctx, rel_err, to_dev, to_np
+
+pytestmark = pytest.mark.gpu
+
+C = wl.CONFIGS
+
+SMALL_CASES = {
+    "c1_full_fp32": C["c1"],
+    "c1_as_bf16": wl.shrink(C["c1"], dtype="bf16"),
+    "c2_vit_B2_H3": wl.shrink(C["c2"], B=2, H=3),
+    "c3_video_B1_H2": wl.shrink(C["c3"], B=1, H=2),
+    "c4_cross_B2_H2": wl.shrink(C["c4"], B=2, H=2),
+    "c5_long_n2048_nq700": wl.shrink(C["c5"], B=1, H=2, n=2048, n_q=700, m=128),
+    "c5_long_n4096_m256": wl.shrink(C["c5"], B=1, H=1, n=4096, n_q=1000, m=256),
+    "ragged_fp32_d72": wl.Workload("ragged", 2, 2, 203, 37, 72, 75, "fp32", 5, 0.02, "iid", 77),
+    "ragged_bf16_d40": wl.Workload("ragged16", 1, 3, 131, 67, 40, 41, "bf16", 4, 0.02, "iid", 78),
+}
+
+
+def oracle_all(w, inp, phi, T, lam, stages=None):
+    return orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=lam, Psi=inp["Psi"], stages=stages)
+
+
+def median_lambda(w, inp, phi):
+    """lambda that shrinks about half of the first-iteration coefficients (from the oracle only)."""
+    st = []
+    orc.csat_forward(inp["Q"][:1, :1], inp["K"][:1, :1], inp["V"][:1, :1], phi[:1], T=1, lam=0.0,
+                     Psi=inp["Psi"], stages=st)
+    s = st[0]
+    return float(np.median(np.abs(s["Z"] @ s["B_dec"])) / s["mu"])
+
+
+@pytest.mark.parametrize("name", sorted(SMALL_CASES))
+def test_forward_matches_oracle(name):
+    w = SMALL_CASES[name]
+    inp = wl.make_inputs(w)
+    Q, K, V, Psi = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    if Psi is not None:
+        ctx.set_dictionary(Psi)
+    phi = to_np(ctx.get_phi())
+    tol = TOL[w.dtype]
+    lam_med = median_lambda(w, inp, phi)
+    for T, lam in [(0, w.lam), (w.T, w.lam), (w.T, 0.0), (w.T, lam_med), (1, lam_med)]:
+        ctx.set(T=T, lam=lam)
+        out = to_np(ctx.forward(Q, K, V))
+        stages = []
+        ref = oracle_all(w, inp, phi, T, lam, stages)
+        if np.abs(ref).max() == 0.0:
+            theta = max(s["theta"] for s in stages)
+            assert np.abs(out).max() <= theta * tol, (name, T, lam)
+        else:
+            err = rel_err(out, ref)
+            assert err <= tol, (name, T, lam, err)
+        assert ctx.launches >= 2
+    # compression stage on its own: K~, V~ as left in the workspace
+    kt, vt = (to_np(t) for t in ctx.get_compressed())
+    kt_ref = np.stack([[s["Kt"]] for s in stages]).reshape(kt.shape)
+    vt_ref = np.stack([[s["Vt"]] for s in stages]).reshape(vt.shape)
+    assert rel_err(kt, kt_ref) <= (4e-3 if w.dtype == "bf16" else 2e-6)
+    assert rel_err(vt, vt_ref) <= (4e-3 if w.dtype == "bf16" else 2e-6)
+    ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_identity_measurement_is_softmax_attention(dtype):
+    """m = n, Phi = I: recovery disabled gives standard attention; T >= 1 gives soft(Attn, lambda)."""
+    w = wl.shrink(C["c1"], m=256, dtype=dtype)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w, T=0)
+    ctx.set_phi(to_dev(np.eye(w.n, dtype=np.float32)[None], dtype))
+    Qd, Kd, Vd = (inp[k][0, 0].astype(np.float64) for k in "QKV")
+    A = np.exp(Qd @ Kd.T / 8.0 - (Qd @ Kd.T / 8.0).max(axis=1, keepdims=True))
+    attn = (A / A.sum(axis=1, keepdims=True)) @ Vd
+    out = to_np(ctx.forward(Q, K, V))[0, 0]
+    assert rel_err(out, attn) <= TOL[dtype]
+    ctx.set(T=3, lam=0.1)
+    out = to_np(ctx.forward(Q, K, V))[0, 0]
+    shr = np.sign(attn) * np.maximum(np.abs(attn) - 0.1, 0.0)
+    assert rel_err(out, shr) <= TOL[dtype]
+    ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_phi_matches_oracle_generator(dtype):
+    for (H, m, n, seed) in [(1, 64, 256, 0), (3, 20, 197, 0xDEADBEEF12345678), (2, 7, 64, 5)]:
+        ctx = binding.Csat(n, m, 8, H, seed, dtype=dtype)
+        got = to_np(ctx.get_phi())
+        exact = pho.phi_gaussian(H, m, n, seed)
+        ref = wl.round_to_storage(exact.astype(np.float32), dtype).astype(np.float64)
+        if dtype == "fp32":
+            # float32 transcendentals vs float64: a few ulp, plus cancellation near sin/cos zeros
+            assert np.all(np.abs(got - exact) <= 4e-6 * np.abs(exact) + 2e-7 / np.sqrt(m))
+        else:
+            bad = got != ref
+            assert bad.mean() <= 1e-3
+            assert np.all(np.abs(got - ref)[bad] <= np.abs(ref[bad]) * 2.0 ** -7)   # one bf16 ulp
+        ctx.close()
+
+
+def test_decoder_matrices_match_oracle():
+    w = wl.shrink(C["c4"], B=1, H=3, n=392, m=98)
+    inp = wl.make_inputs(w)
+    ctx = make_ctx(w)
+    Psi = to_dev(inp["Psi"], w.dtype)
+    phi = to_np(ctx.get_phi())
+    for psi_dev, psi_np in ((None, None), (Psi, inp["Psi"].astype(np.float64))):
+        ctx.set_dictionary(psi_dev)
+        for step in (0.0, 0.3):
+            ctx.set(step=step)
+            S, Bm, th, mu = (to_np(t) for t in ctx.get_decoder())
+            for h in range(w.H):
+                D = phi[h, :w.d, :w.d]
+                M = D if psi_np is None else D @ psi_np
+                S_ref, B_ref, th_ref, mu_ref = orc.decoder_setup(M, w.lam, step)
+                assert np.abs(S[h] - S_ref).max() <= 1e-6
+                assert np.abs(Bm[h] - B_ref).max() <= 1e-6 * max(1.0, np.abs(B_ref).max())
+                assert abs(th[h] - th_ref) <= 1e-6 * th_ref and abs(mu[h] - mu_ref) <= 1e-6 * mu_ref
+    # a caller-supplied decoder matrix replaces the Phi block
+    r = np.random.default_rng(3)
+    Dn = wl.round_to_storage((np.eye(w.d) + 0.1 * r.standard_normal((w.H, w.d, w.d))).astype(np.float32), w.dtype)
+    ctx.set_dictionary(None)
+    ctx.set(step=0.0)
+    ctx.set_decoder_matrix(to_dev(Dn, w.dtype))
+    S, Bm, th, mu = (to_np(t) for t in ctx.get_decoder())
+    for h in range(w.H):
+        S_ref, B_ref, _, _ = orc.decoder_setup(Dn[h].astype(np.float64), w.lam)
+        assert np.abs(S[h] - S_ref).max() <= 1e-6 and np.abs(Bm[h] - B_ref).max() <= 1e-6
+    Q, K, V, _ = device_inputs(w, inp)
+    out = to_np(ctx.forward(Q, K, V))
+    ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=w.T, lam=w.lam, D=Dn.astype(np.float64))
+    assert rel_err(out, ref) <= TOL[w.dtype]
+    ctx.close()
+
+
+def test_edge_shapes():
+    """Single query, single measurement (needs a supplied D), tiny ragged sizes, huge lambda."""
+    r = np.random.default_rng(11)
+    for dtype in ("fp32", "bf16"):
+        for (B, H, n, nq, d, m) in [(1, 1, 8, 1, 8, 1), (2, 1, 9, 3, 8, 9), (1, 2, 300, 5, 16, 2), (1, 1, 64, 129, 64, 64)]:
+            w = wl.Workload("edge", B, H, n, nq, d, m, dtype, 3, 0.01, "iid", 5)
+            inp = wl.make_inputs(w)
+            Q, K, V, _ = device_inputs(w, inp)
+            ctx = make_ctx(w)
+            Dn = wl.round_to_storage((np.eye(d) + 0.2 * r.standard_normal((H, d, d))).astype(np.float32), dtype)
+            ctx.set_decoder_matrix(to_dev(Dn, dtype))
+            phi = to_np(ctx.get_phi())
+            for T, lam in [(0, 0.0), (3, 0.01), (2, 1e6)]:
+                ctx.set(T=T, lam=lam)
+                out = to_np(ctx.forward(Q, K, V))
+                ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=lam, D=Dn.astype(np.float64))
+                if lam == 1e6:
+                    assert np.all(out == 0.0) and np.all(ref == 0.0)
+                else:
+                    assert rel_err(out, ref) <= TOL[dtype], (dtype, B, H, n, nq, d, m, T)
+            ctx.close()
+
+
+def test_abi_errors_and_determinism():
+    w = wl.shrink(C["c2"], B=1, H=2)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w, lam=0.0)
+    out1 = ctx.forward(Q, K, V).clone()
+    out2 = ctx.forward(Q, K, V)
+    assert torch.equal(out1, out2)                                    # bit-identical run to run
+    lib = binding.load()
+    s = torch.cuda.current_stream().cuda_stream
+    p = lambda t: t.data_ptr()
+    assert lib.csat_forward(ctx.h, None, p(K), p(V), p(out2), s) == 1
+    assert lib.csat_forward(ctx.h, p(Q) + 2, p(K), p(V), p(out2), s) == 1     # misaligned
+    assert lib.csat_forward(ctx.h, p(Q), p(K), p(V), p(Q), s) == 1            # out aliases Q
+    assert "alias" in binding.csat_last_error(ctx.h)
+    assert lib.csat_set_i64(ctx.h, 99, 1) == 1
+    assert lib.csat_set_i64(ctx.h, binding.CSAT_T, -1) == 1
+    assert lib.csat_set_f64(ctx.h, binding.CSAT_LAMBDA, -0.5) == 1
+    assert lib.csat_set_i64(ctx.h, binding.CSAT_BATCH, 0) == 2
+    assert binding.csat_get_i64(ctx.h, binding.CSAT_T) == w.T
+    assert binding.csat_get_f64(ctx.h, binding.CSAT_LAMBDA) == 0.0
+    assert ctx.workspace_bytes > 0
+    torch.cuda.synchronize()
+    assert torch.equal(ctx.forward(Q, K, V), out1)                    # failed calls left the context usable
+    ctx.close()
+    # default decoder matrix needs m >= d
+    small = binding.Csat(64, 8, 64, 1, 0, dtype="fp32", T=2)
+    q = torch.zeros(1, 1, 64, 64, device="cuda")
+    with pytest.raises(binding.CsatError) as ei:
+        small.forward(q, q.clone(), q.clone())
+    assert ei.value.code == 2
+    small.set(T=0)
+    small.forward(q, q.clone(), q.clone())                            # recovery disabled: legal
+    small.close()
+    with pytest.raises(binding.CsatError):
+        c = binding.Csat(64, 8, 64, 1, 0)
+        try:
+            binding.csat_get_compressed(c.h, q, q)                    # before any forward
+        finally:
+            c.close()
+
+
+def test_forward_host_equals_forward():
+    w = wl.shrink(C["c3"], B=1, H=2, n=392, n_q=392, m=64)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    out = ctx.forward(Q, K, V)
+    Qh, Kh, Vh = (t.cpu().pin_memory() for t in (Q, K, V))
+    oh = torch.empty_like(Qh).pin_memory()
+    ctx.forward_host(Qh, Kh, Vh, oh)
+    assert torch.equal(oh, out.cpu())
+    ctx.close()
