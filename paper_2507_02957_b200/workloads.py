@@ -61,7 +61,11 @@ def sweep_config(n: int) -> Workload:
 
 
 def shrink(w: Workload, **kw) -> Workload:
-    """A smaller instance of the same recipe (used by parity tests)."""
+    """A smaller instance of the same recipe (used by parity tests).  For the frame-structured
+    workloads a new n keeps the patches per frame and changes the number of frames."""
+    if "n" in kw and w.patches and "frames" not in kw:
+        assert kw["n"] % w.patches == 0, "n must stay a whole number of frames"
+        kw["frames"] = kw["n"] // w.patches
     return replace(w, **kw)
 
 
