@@ -61,7 +61,18 @@ enum {
                           of text queries over compressed visual keys uses n_q != n     */
   CSAT_DTYPE = 3,      /* CSAT_DTYPE_BF16 (default) or CSAT_DTYPE_FP32                   */
   CSAT_T = 4,          /* recovery iterations (decoder depth t), default 10; 0 = out = Z */
-  CSAT_FORCE_SIMT = 5  /* diagnostic: 1 routes bf16 through the plain FFMA kernels       */
+  CSAT_FORCE_SIMT = 5, /* diagnostic: 1 routes bf16 through the plain FFMA kernels       */
+  CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls
+                          (0 = off, default; at most 4096).  Setting it creates/destroys
+                          events, so set it outside the timed region                    */
+};
+
+/* kernel ids reported by csat_get_profile */
+enum {
+  CSAT_KERNEL_DECODER_SETUP = 0, /* the three small set-up launches, timed together      */
+  CSAT_KERNEL_COMPRESS = 1,      /* K~|V~ = Phi [K|V]                                    */
+  CSAT_KERNEL_ATTEND_RECOVER = 2,/* softmax(Q K~^T) V~, recovery iterations, Psi         */
+  CSAT_KERNEL_SPLIT_REDUCE = 3   /* fixed-order sum of token-axis partial K~|V~ tiles    */
 };
 enum { CSAT_DTYPE_BF16 = 0, CSAT_DTYPE_FP32 = 1 };
 
@@ -147,6 +158,15 @@ int csat_get_compressed(const csat_ctx* ctx, void* kt_out, void* vt_out, void* s
  * parameters changed. */
 int csat_get_decoder(csat_ctx* ctx, float* S_out, float* B_out, float* theta_out, float* mu_out, void* stream);
 
+/* csat_get_profile -- measurement aid, no counterpart in the paper.  With CSAT_PROFILE = v > 0
+ * every csat_forward records CUDA events on its stream before the first and after each of its
+ * kernels.  call_index counts forward calls since CSAT_PROFILE was set (0-based; only the most
+ * recent v are kept).  Writes up to `cap` kernel ids and their durations in milliseconds to the
+ * HOST arrays and the number of kernels to *count_host.  Synchronises on the call's last event.
+ * CSAT_ERR_STATE if profiling is off or the call is no longer / not yet recorded. */
+int csat_get_profile(const csat_ctx* ctx, int64_t call_index, int cap, int* kernel_ids_host, float* ms_host,
+                     int* count_host);
+
 /* Bytes of device memory the context currently owns (Phi, workspace, decoder matrices, staging). */
 size_t csat_workspace_bytes(const csat_ctx* ctx);
 
@@ -154,9 +174,10 @@ size_t csat_workspace_bytes(const csat_ctx* ctx);
 int csat_last_launch_count(const csat_ctx* ctx);
 
 /* Text of the most recent failure of this context; with NULL, of the calling thread's most
- * recent failed csat_create.  Also reads the device status word (cudaMemcpy of 4 bytes, which
- * synchronises) so a CSAT_ERR_TIMEOUT raised by a finished launch becomes visible.
- * The pointer stays valid until the next call on the same context / thread. */
+ * recent failed csat_create.  Also looks at the status word kernels write when a bounded wait
+ * gives up (host-mapped memory, read without synchronising), so a CSAT_ERR_TIMEOUT raised by a
+ * finished launch becomes visible.  The pointer stays valid until the next call on the same
+ * context / thread. */
 const char* csat_last_error(const csat_ctx* ctx);
 
 /* Library version: major*10000 + minor*100 + patch. */

@@ -16,7 +16,8 @@ from . import build as _build
 CSAT_OK = 0
 ERR_NAMES = {1: "CSAT_ERR_INVALID_ARG", 2: "CSAT_ERR_SHAPE", 3: "CSAT_ERR_ALLOC", 4: "CSAT_ERR_CUDA",
              5: "CSAT_ERR_UNSUPPORTED", 6: "CSAT_ERR_STATE", 7: "CSAT_ERR_TIMEOUT"}
-CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT = 1, 2, 3, 4, 5
+CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE = 1, 2, 3, 4, 5, 6
+KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover", 3: "split_reduce"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1
 CSAT_LAMBDA, CSAT_STEP, CSAT_SCALE = 1, 2, 3
 
@@ -39,6 +40,7 @@ SIGNATURES = {
     "csat_forward_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
     "csat_get_decoder": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "csat_get_profile": (_int, [_vp, _i64, _int, C.POINTER(_int), C.POINTER(C.c_float), C.POINTER(_int)]),
     "csat_workspace_bytes": (C.c_size_t, [_vp]),
     "csat_last_launch_count": (_int, [_vp]),
     "csat_last_error": (C.c_char_p, [_vp]),
@@ -156,6 +158,14 @@ def csat_get_compressed(h, kt_out, vt_out, stream=None):
 
 def csat_get_decoder(h, S_out, B_out, theta_out, mu_out, stream=None):
     _check(h, load().csat_get_decoder(h, _ptr(S_out), _ptr(B_out), _ptr(theta_out), _ptr(mu_out), _stream(stream)))
+
+
+def csat_get_profile(h, call_index):
+    """[(kernel id, milliseconds), ...] of one recorded forward call."""
+    cap = 8
+    ids, ms, cnt = (_int * cap)(), (C.c_float * cap)(), _int()
+    _check(h, load().csat_get_profile(h, call_index, cap, ids, ms, C.byref(cnt)))
+    return [(ids[i], ms[i]) for i in range(min(cnt.value, cap))]
 
 
 def csat_workspace_bytes(h) -> int:

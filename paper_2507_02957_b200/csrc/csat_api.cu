@@ -43,6 +43,8 @@ size_t phi_bytes(const csat::Params& p) { return (size_t)(p.H * p.m * p.n_pad) *
 size_t kv_bytes(const csat::Params& p) { return (size_t)(p.B * p.H * p.m * 2 * p.d) * csat::elt_size(p.dtype); }
 size_t dd_bytes(const csat::Params& p, size_t elt) { return (size_t)(p.H * p.d * p.d) * elt; }
 
+void prof_destroy(csat_ctx* c);
+
 void free_staging(csat_ctx* c) {
   dev_free(c, &c->stage_q, c->stage_bytes_q);
   dev_free(c, &c->stage_o, c->stage_bytes_q);
@@ -65,6 +67,7 @@ void free_all(csat_ctx* c) {
   dev_free(c, &c->theta, (size_t)p.H * 4);
   dev_free(c, &c->mu, (size_t)p.H * 4);
   free_staging(c);
+  prof_destroy(c);
   if (c->status) {
     cudaFreeHost(c->status);
     c->status = nullptr;
@@ -82,6 +85,32 @@ int allocate_and_generate(csat_ctx* c) {
   c->decoder_dirty = true;
   c->have_forward = false;
   return CSAT_OK;
+}
+
+void prof_destroy(csat_ctx* c) {
+  for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
+  c->prof_events.clear();
+  c->prof_ids.clear();
+  c->prof_count.clear();
+  c->prof_slots = 0;
+  c->prof_calls = 0;
+}
+
+// records the event that closes kernel `id` of the current call (id < 0: the opening event)
+void prof_mark(csat_ctx* c, cudaStream_t s, int id) {
+  if (c->prof_slots == 0) return;
+  const int K = csat_ctx::kProfMaxKernels;
+  const int slot = (int)(c->prof_calls % c->prof_slots);
+  if (id < 0) {
+    c->prof_count[slot] = 0;
+    cudaEventRecord(c->prof_events[(size_t)slot * (K + 1)], s);
+    return;
+  }
+  int& n = c->prof_count[slot];
+  if (n >= K) return;
+  c->prof_ids[(size_t)slot * K + n] = id;
+  cudaEventRecord(c->prof_events[(size_t)slot * (K + 1) + n + 1], s);
+  ++n;
 }
 
 bool on_device(const csat_ctx* c, std::string* why) {
@@ -200,6 +229,25 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
     case CSAT_FORCE_SIMT:
       c->force_simt = v != 0;
       return CSAT_OK;
+    case CSAT_PROFILE: {
+      if (v < 0 || v > 4096) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_PROFILE must be in [0, 4096]");
+      cudaDeviceSynchronize();
+      prof_destroy(c);
+      const int K = csat_ctx::kProfMaxKernels;
+      c->prof_events.reserve((size_t)v * (K + 1));
+      for (int64_t i = 0; i < v * (K + 1); ++i) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) {
+          prof_destroy(c);
+          return fail(c, CSAT_ERR_ALLOC, "cudaEventCreate failed");
+        }
+        c->prof_events.push_back(e);
+      }
+      c->prof_ids.assign((size_t)v * K, 0);
+      c->prof_count.assign((size_t)v, 0);
+      c->prof_slots = (int)v;
+      return CSAT_OK;
+    }
     default:
       return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_i64: unknown key");
   }
@@ -213,6 +261,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
     case CSAT_DTYPE: *out = c->p.dtype; return CSAT_OK;
     case CSAT_T: *out = c->p.T; return CSAT_OK;
     case CSAT_FORCE_SIMT: *out = c->force_simt; return CSAT_OK;
+    case CSAT_PROFILE: *out = c->prof_slots; return CSAT_OK;
     default: return CSAT_ERR_INVALID_ARG;
   }
 }
@@ -328,15 +377,21 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
     return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
   cudaStream_t s = (cudaStream_t)stream;
   int launches = 0;
+  prof_mark(c, s, -1);
   if (c->p.T > 0) {
+    const bool was_dirty = c->decoder_dirty;
     int rc = ensure_decoder(c, s, &launches);
     if (rc != CSAT_OK) return rc;
+    if (was_dirty) prof_mark(c, s, CSAT_KERNEL_DECODER_SETUP);
   }
   cudaError_t e;
   // float32 contexts, and head sizes without a tensor-core kernel, take the FFMA kernels
   if ((e = csat::launch_simt_compress(c, K, V, s, &launches)) != cudaSuccess) return fail_cuda(c, e, "compress launch");
+  prof_mark(c, s, CSAT_KERNEL_COMPRESS);
   if ((e = csat::launch_simt_attend_recover(c, Q, out, s, &launches)) != cudaSuccess)
     return fail_cuda(c, e, "attend/recover launch");
+  prof_mark(c, s, CSAT_KERNEL_ATTEND_RECOVER);
+  if (c->prof_slots) ++c->prof_calls;
   c->have_forward = true;
   c->last_launches = launches;
   return CSAT_OK;
@@ -397,6 +452,26 @@ int csat_get_decoder(csat_ctx* c, float* S_out, float* B_out, float* theta_out, 
   if (theta_out && e == cudaSuccess) e = cudaMemcpyAsync(theta_out, c->theta, (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
   if (mu_out && e == cudaSuccess) e = cudaMemcpyAsync(mu_out, c->mu, (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_get_decoder");
+  return CSAT_OK;
+}
+
+int csat_get_profile(const csat_ctx* c, int64_t call_index, int cap, int* ids, float* ms, int* count) {
+  if (!c || !count || cap < 0 || (cap > 0 && (!ids || !ms))) return CSAT_ERR_INVALID_ARG;
+  csat_ctx* mc = const_cast<csat_ctx*>(c);
+  if (c->prof_slots == 0) return fail(mc, CSAT_ERR_STATE, "csat_get_profile: CSAT_PROFILE is off");
+  if (call_index < 0 || call_index >= c->prof_calls || call_index < c->prof_calls - c->prof_slots)
+    return fail(mc, CSAT_ERR_STATE, "csat_get_profile: that call is not recorded");
+  const int K = csat_ctx::kProfMaxKernels;
+  const int slot = (int)(call_index % c->prof_slots);
+  const int n = c->prof_count[slot];
+  const cudaEvent_t* ev = &c->prof_events[(size_t)slot * (K + 1)];
+  cudaError_t e = cudaEventSynchronize(ev[n]);
+  if (e != cudaSuccess) return fail_cuda(mc, e, "csat_get_profile");
+  *count = n;
+  for (int i = 0; i < n && i < cap; ++i) {
+    ids[i] = c->prof_ids[(size_t)slot * K + i];
+    if ((e = cudaEventElapsedTime(&ms[i], ev[i], ev[i + 1])) != cudaSuccess) return fail_cuda(mc, e, "csat_get_profile");
+  }
   return CSAT_OK;
 }
 

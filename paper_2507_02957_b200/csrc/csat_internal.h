@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <string>
+#include <vector>
 
 #include "csat.h"
 
@@ -48,6 +49,14 @@ struct csat_ctx {
   // staging for csat_forward_host
   void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
   size_t stage_bytes_q = 0, stage_bytes_kv = 0;
+
+  // per-kernel CUDA-event timing of the most recent `prof_slots` forward calls (CSAT_PROFILE)
+  static constexpr int kProfMaxKernels = 8;
+  int prof_slots = 0;
+  int64_t prof_calls = 0;                       // forward calls since profiling was switched on
+  std::vector<cudaEvent_t> prof_events;         // [slots][kProfMaxKernels + 1]
+  std::vector<int> prof_ids;                    // [slots][kProfMaxKernels]
+  std::vector<int> prof_count;                  // [slots]
 
   bool decoder_dirty = true;
   bool have_forward = false;

@@ -123,12 +123,25 @@ def _redundant_frames(rng, B, H, frames, patches, d) -> np.ndarray:
     return (base + noise).reshape(B, H, frames * patches, d)
 
 
-def make_inputs(w: Workload) -> dict:
+def flops(w: Workload, with_psi: bool | None = None) -> dict:
+    """Algorithmic floating-point operations of one forward (all B*H pairs), per stage."""
+    bh = w.B * w.H
+    psi = (w.kind == "crossmodal") if with_psi is None else with_psi
+    compress = 4 * w.m * w.n * w.d * bh
+    attend = 4 * w.n_q * w.m * w.d * bh
+    recover = (2 * w.n_q * w.d * w.d * (w.T + 1) + (2 * w.n_q * w.d * w.d if psi else 0)) * bh if w.T > 0 else 0
+    return {"compress": compress, "attend": attend, "recover": recover, "total": compress + attend + recover}
+
+
+def make_inputs(w: Workload, rounded: bool = True) -> dict:
     """Draw Q, K, V (and Psi for the cross-modal workload) for a workload.
 
-    Returns float32 arrays already rounded to the storage type:
+    Returns float32 arrays, rounded to the storage type unless rounded=False (a caller that
+    converts with another round-to-nearest-even routine gets the same values):
       Q [B,H,n_q,d], K [B,H,n,d], V [B,H,n,d], Psi [d,d] or None.
     """
+    if not rounded:
+        w = replace(w, dtype="fp32")
     rng = np.random.Generator(np.random.PCG64(w.data_seed))
     B, H, n, nq, d = w.B, w.H, w.n, w.n_q, w.d
     psi = None
