@@ -167,6 +167,38 @@ int csat_get_decoder(csat_ctx* ctx, float* S_out, float* B_out, float* theta_out
 int csat_get_profile(const csat_ctx* ctx, int64_t call_index, int cap, int* kernel_ids_host, float* ms_host,
                      int* count_host);
 
+/*
+ * csat_attend_noalloc -- the paper has no counterpart; this is a deployment aid.
+ *
+ * Some callers may not allocate device memory at the point where they need attention: code that
+ * runs inside another framework's memory plan or after its arena has been sealed, real-time loops
+ * where cudaMalloc's implicit device synchronisation is not acceptable, and processes whose memory
+ * budget is fixed up front.  csat_create/csat_forward are closed to them because the K~|V~
+ * workspace comes from cudaMalloc.  This entry point computes the compressed attention with
+ * recovery disabled,
+ *     out = softmax(Q (Phi K)^T * scale) (Phi V)        (same result as csat_forward with CSAT_T = 0),
+ * and keeps K~|V~ in a fixed CSAT_NOALLOC_SCRATCH_BYTES array that is part of the library image.
+ * It calls no cudaMalloc/cudaFree and no allocating library routine, and needs no context.
+ *
+ *   Q [B,H,n_q,d], K,V [B,H,n,d], phi [H,m,n] dense (e.g. from csat_get_phi), out [B,H,n_q,d]:
+ *   device pointers, 16-byte aligned, element type `dtype` (CSAT_DTYPE_*).  scale 0 = 1/sqrt(d).
+ *   err_host/err_cap: optional host buffer that receives a message when the call fails.
+ *
+ * Limits and rules
+ *   - B*H*m*2*d*sizeof(element) must not exceed CSAT_NOALLOC_SCRATCH_BYTES; larger problems are
+ *     refused with CSAT_ERR_SHAPE and a message stating both numbers.
+ *   - Every GPU that loads the library holds the array (8 MiB) until the process exits.
+ *   - The first call on each device looks the array's device address up (cudaGetSymbolAddress,
+ *     with that device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  Each call overwrites the part it reads, so
+ *     nothing needs clearing, but two calls that overlap on the GPU (different streams, or
+ *     different host threads without ordering) race on it: serialise them on one stream.
+ */
+#define CSAT_NOALLOC_SCRATCH_BYTES (8u << 20)
+int csat_attend_noalloc(const void* Q, const void* K, const void* V, const void* phi, void* out, int64_t B,
+                        int64_t H, int64_t n, int64_t n_q, int64_t m, int64_t d, int dtype, double scale,
+                        void* stream, char* err_host, size_t err_cap);
+
 /* Bytes of device memory the context currently owns (Phi, workspace, decoder matrices, staging). */
 size_t csat_workspace_bytes(const csat_ctx* ctx);
 

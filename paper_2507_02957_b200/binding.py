@@ -41,6 +41,8 @@ SIGNATURES = {
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
     "csat_get_decoder": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_profile": (_int, [_vp, _i64, _int, C.POINTER(_int), C.POINTER(C.c_float), C.POINTER(_int)]),
+    "csat_attend_noalloc": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _i64, _i64, _int, _dbl, _vp,
+                                   C.c_char_p, C.c_size_t]),
     "csat_workspace_bytes": (C.c_size_t, [_vp]),
     "csat_last_launch_count": (_int, [_vp]),
     "csat_last_error": (C.c_char_p, [_vp]),
@@ -166,6 +168,24 @@ def csat_get_profile(h, call_index):
     ids, ms, cnt = (_int * cap)(), (C.c_float * cap)(), _int()
     _check(h, load().csat_get_profile(h, call_index, cap, ids, ms, C.byref(cnt)))
     return [(ids[i], ms[i]) for i in range(min(cnt.value, cap))]
+
+
+NOALLOC_SCRATCH_BYTES = 8 << 20
+
+
+def csat_attend_noalloc(Q, K, V, phi, out, scale=0.0, stream=None):
+    """Compressed attention with recovery disabled, for callers that must not allocate device memory:
+    the K~|V~ scratch is a fixed array inside the library (see include/csat.h).  Shapes are read from
+    the tensors: Q [B,H,n_q,d], K,V [B,H,n,d], phi [H,m,n], out [B,H,n_q,d]; nothing is allocated here."""
+    B, H, nq, d = Q.shape
+    n, m = K.shape[2], phi.shape[1]
+    code = CSAT_DTYPE_FP32 if Q.dtype == torch.float32 else CSAT_DTYPE_BF16
+    err = C.create_string_buffer(512)
+    rc = load().csat_attend_noalloc(_ptr(Q), _ptr(K), _ptr(V), _ptr(phi), _ptr(out), B, H, n, nq, m, d, code,
+                                    float(scale), _stream(stream), err, len(err))
+    if rc != CSAT_OK:
+        raise CsatError(rc, err.value.decode())
+    return out
 
 
 def csat_workspace_bytes(h) -> int:

@@ -317,3 +317,141 @@ cudaError_t launch_split_kv(const csat_ctx* c, void* kt, void* vt, cudaStream_t 
 }
 
 }  // namespace csat
+
+// =============================================================================================
+// csat_attend_noalloc: compressed attention (recovery disabled) for callers that cannot allocate.
+// The K~|V~ scratch lives in a fixed array inside the library image instead of a cudaMalloc'd
+// workspace.  See include/csat.h for who needs this and for the rules of use.
+// =============================================================================================
+#include <mutex>
+
+namespace csat {
+namespace {
+
+// Scratch shared by every call on a device.  Resident on each GPU that loads the library, until exit.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[CSAT_NOALLOC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices] = {};   // device address of the array above, per device
+std::mutex g_noalloc_mutex;
+
+// Dense-Phi compression into the scratch: one thread per output element, tokens summed in index order
+// (the same order, with the same fused multiply-adds, as compress_kernel).
+template <typename T>
+__global__ void compress_dense_phi_kernel(T* __restrict__ kv, const T* __restrict__ phi, const T* __restrict__ K,
+                                          const T* __restrict__ V, int64_t n, int64_t m, int d, int H, int64_t total) {
+  const int d2 = 2 * d;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int c = (int)(i % d2);
+    const int64_t r = (i / d2) % m, bh = i / (d2 * m);
+    const T* src = (c < d ? K : V) + bh * n * d + (c < d ? c : c - d);
+    const T* ph = phi + ((bh % H) * m + r) * n;
+    float acc = 0.f;
+    for (int64_t j = 0; j < n; ++j) acc = fmaf(ldf(ph, j), ldf(src, j * d), acc);
+    stf(kv, i, acc);
+  }
+}
+
+void write_err(char* buf, size_t cap, const char* msg) {
+  if (buf && cap) snprintf(buf, cap, "%s", msg);
+}
+
+template <typename T>
+int attend_noalloc_t(const void* Q, const void* K, const void* V, const void* phi, void* out, void* scratch,
+                     int64_t B, int64_t H, int64_t n, int64_t nq, int64_t m, int d, float scale, cudaStream_t s,
+                     char* err, size_t cap) {
+  const int64_t total = B * H * m * 2 * d;
+  int64_t g = (total + 255) / 256;
+  if (g > 148 * 32) g = 148 * 32;
+  compress_dense_phi_kernel<T><<<(unsigned)g, 256, 0, s>>>((T*)scratch, (const T*)phi, (const T*)K, (const T*)V, n, m,
+                                                          d, (int)H, total);
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) {
+    const dim3 grid((unsigned)((nq + kAttWarps - 1) / kAttWarps), (unsigned)(B * H));
+    const size_t sm = (size_t)(32 * (2 * d + 1) + kAttWarps * d) * sizeof(float);
+    const int dc = (d + 31) / 32;
+#define CSAT_NOALLOC_ATT(DC)                                                                                        \
+  do {                                                                                                              \
+    if (sm > 48 * 1024)                                                                                             \
+      e = cudaFuncSetAttribute(attend_recover_kernel<T, DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); \
+    if (e == cudaSuccess)                                                                                           \
+      attend_recover_kernel<T, DC><<<grid, kAttWarps * 32, sm, s>>>((T*)out, (const T*)Q, (const T*)scratch,        \
+                                                                    nullptr, nullptr, nullptr, nullptr, nq, m, d,   \
+                                                                    (int)H, /*T_iters=*/0, scale);                  \
+  } while (0)
+    if (dc <= 2) CSAT_NOALLOC_ATT(2);
+    else if (dc <= 4) CSAT_NOALLOC_ATT(4);
+    else CSAT_NOALLOC_ATT(8);
+#undef CSAT_NOALLOC_ATT
+    if (e == cudaSuccess) e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    write_err(err, cap, cudaGetErrorString(e));
+    return CSAT_ERR_CUDA;
+  }
+  return CSAT_OK;
+}
+
+}  // namespace
+}  // namespace csat
+
+extern "C" int csat_attend_noalloc(const void* Q, const void* K, const void* V, const void* phi, void* out, int64_t B,
+                                   int64_t H, int64_t n, int64_t n_q, int64_t m, int64_t d, int dtype, double scale,
+                                   void* stream, char* err_host, size_t err_cap) {
+  using namespace csat;
+  if (err_host && err_cap) err_host[0] = 0;
+  if (!Q || !K || !V || !phi || !out) {
+    write_err(err_host, err_cap, "csat_attend_noalloc: NULL tensor pointer");
+    return CSAT_ERR_INVALID_ARG;
+  }
+  for (const void* p : {Q, K, V, phi, (const void*)out})
+    if (reinterpret_cast<uintptr_t>(p) & 15u) {
+      write_err(err_host, err_cap, "csat_attend_noalloc: tensor pointers must be 16-byte aligned");
+      return CSAT_ERR_INVALID_ARG;
+    }
+  if (dtype != CSAT_DTYPE_BF16 && dtype != CSAT_DTYPE_FP32) {
+    write_err(err_host, err_cap, "csat_attend_noalloc: unknown dtype");
+    return CSAT_ERR_INVALID_ARG;
+  }
+  if (B < 1 || H < 1 || n < 1 || n_q < 1 || m < 1 || m > n || d < 8 || d > 256 || d % 8 != 0 || B * H > 65535 ||
+      n > ((int64_t)1 << 31) || n_q > ((int64_t)1 << 31)) {
+    write_err(err_host, err_cap, "csat_attend_noalloc: need B,H,n_q >= 1, 1 <= m <= n, 8 <= d <= 256, d % 8 == 0, B*H <= 65535");
+    return CSAT_ERR_SHAPE;
+  }
+  const int64_t need = B * H * m * 2 * d * (int64_t)elt_size(dtype);
+  if (need > (int64_t)CSAT_NOALLOC_SCRATCH_BYTES) {
+    if (err_host && err_cap)
+      snprintf(err_host, err_cap,
+               "csat_attend_noalloc: K~|V~ needs %lld bytes (B*H*m*2d*elt) but the built-in scratch holds %lld; "
+               "use csat_create/csat_forward for larger problems",
+               (long long)need, (long long)CSAT_NOALLOC_SCRATCH_BYTES);
+    return CSAT_ERR_SHAPE;
+  }
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    write_err(err_host, err_cap, "csat_attend_noalloc: no usable current CUDA device");
+    return CSAT_ERR_CUDA;
+  }
+  void* scratch = nullptr;
+  {
+    // once per device, with that device current: turn the host-side symbol into a device address
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+      void* p = nullptr;
+      e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+      if (e != cudaSuccess || !p) {
+        write_err(err_host, err_cap, cudaGetErrorString(e));
+        return CSAT_ERR_CUDA;
+      }
+      g_noalloc_ptr[dev] = p;
+    }
+    scratch = g_noalloc_ptr[dev];
+  }
+  const float sc = (float)(scale > 0.0 ? scale : 1.0 / sqrt((double)d));
+  cudaStream_t s = (cudaStream_t)stream;
+  return dtype == CSAT_DTYPE_FP32
+             ? attend_noalloc_t<float>(Q, K, V, phi, out, scratch, B, H, n, n_q, m, (int)d, sc, s, err_host, err_cap)
+             : attend_noalloc_t<__nv_bfloat16>(Q, K, V, phi, out, scratch, B, H, n, n_q, m, (int)d, sc, s, err_host,
+                                               err_cap);
+}
