@@ -1,0 +1,189 @@
+// K~|V~ = Phi_h [K|V]  (paper: compression equation) on the sm_100a tensor cores.
+//
+// Per (batch, head) this is one GEMM  C[m, 2d] = Phi_h[m, n] * [K|V][n, 2d]  with the token axis n as the
+// reduction.  One CTA owns a 128 x 2d tile of C (128 measurements, all K and V columns) in tensor memory
+// and walks the tokens in chunks of 64:
+//   warp 0   : TMA producer.  Phi tile {64 tokens x 128 rows} (K-major A operand) and {64 cols x 64 tokens}
+//              boxes of K and V (MN-major B operand: tokens are the rows of K and V as the caller stores
+//              them, so no transpose pass is needed), 128-byte swizzle, ring of kStages buffers.
+//   warp 1   : allocates tensor memory; one elected thread issues tcgen05.mma (M=128, N=2d, K=16, bf16
+//              in, fp32 accumulate) and commits to the ring's "empty" barriers.
+//   warps 2-5: epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), round to bf16, store
+//              row r of the tile as K~_r | V~_r into the workspace.
+// Rows of Phi beyond m and tokens beyond n are zero-filled by TMA (and Phi's padded columns hold zeros).
+#include "csat_internal.h"
+#include "sm100_ptx.cuh"
+#include "tma_host.h"
+
+namespace csat {
+namespace {
+
+using namespace ptx;
+
+constexpr int kTileM = 128;      // measurements per CTA
+constexpr int kChunk = 64;       // tokens per pipeline stage (one 128-byte swizzled row of bf16)
+constexpr int kThreads = 192;
+constexpr uint32_t kABytes = kTileM * kChunk * 2;     // 16 KB
+constexpr uint32_t kBoxBytes = 64 * kChunk * 2;       // 8 KB: 64 columns x 64 tokens
+
+template <int D> struct Cfg {
+  static constexpr int kN = 2 * D;                    // accumulator columns
+  static constexpr int kBoxes = kN / 64;              // B boxes per stage
+  static constexpr int kStages = (D == 64) ? 6 : 4;
+  static constexpr uint32_t kStageBytes = kABytes + kBoxes * kBoxBytes;
+  static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1)
+compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_k,
+                      const __grid_constant__ CUtensorMap tmap_v, __nv_bfloat16* __restrict__ kv, int m, int n, int H,
+                      int* status) {
+  using C = Cfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* a_buf = smem;                                      // [stages][16 KB]
+  uint8_t* b_buf = smem + C::kStages * kABytes;               // [stages][boxes][8 KB]
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::kStages * C::kStageBytes);
+  uint64_t* empty = full + C::kStages;
+  uint64_t* acc_done = empty + C::kStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int mtile = blockIdx.x, bh = blockIdx.y, h = bh % H;
+  const int nchunks = (n + kChunk - 1) / kChunk;
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tmap_phi);
+    prefetch_tmap(&tmap_k);
+    prefetch_tmap(&tmap_v);
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(acc_done, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, C::kN);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (elect_one()) {
+      int issued = 0;
+      bool ok = true;
+      for (int i = 0; i < nchunks && ok; ++i) {
+        const int s = i % C::kStages;
+        ok = mbar_wait(&empty[s], ((i / C::kStages) & 1) ^ 1, status, 101);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&full[s], C::kStageBytes);
+        tma_load_3d(a_buf + s * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, h);
+#pragma unroll
+        for (int g = 0; g < C::kBoxes; ++g) {
+          const bool is_v = g >= C::kBoxes / 2;
+          tma_load_3d(b_buf + (s * C::kBoxes + g) * kBoxBytes, is_v ? &tmap_v : &tmap_k, &full[s],
+                      (g % (C::kBoxes / 2)) * 64, i * kChunk, bh);
+        }
+        ++issued;
+      }
+      if (!ok) {
+        // gave up: let copies that are still in flight land before the CTA's shared memory goes away
+        for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
+          mbar_wait(&full[i % C::kStages], (i / C::kStages) & 1, status, 102);
+      }
+    }
+  } else if (warp == 1) {
+    if (elect_one()) {
+      constexpr uint32_t idesc = make_idesc_bf16(kTileM, C::kN, /*A MN-major*/ false, /*B MN-major*/ true);
+      bool ok = true;
+      for (int i = 0; i < nchunks; ++i) {
+        const int s = i % C::kStages;
+        ok = mbar_wait(&full[s], (i / C::kStages) & 1, status, 103);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t a_desc = make_smem_desc(smem_u32(a_buf + s * kABytes), 16, 1024);
+        const uint64_t b_desc = make_smem_desc(smem_u32(b_buf + s * C::kBoxes * kBoxBytes), kBoxBytes, 1024);
+#pragma unroll
+        for (int k = 0; k < kChunk / 16; ++k)   // +32 B along K for A, +2048 B (16 token rows) for B
+          mma_f16_ss(tmem_base, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, (i | k) != 0);
+        mma_commit(&empty[s]);                  // stage reusable once these MMAs have read it
+      }
+      mma_commit(acc_done);                     // arrives when every MMA above has finished (also after a give-up)
+    }
+  } else {
+    const int q = warp & 3;                     // this warp may touch TMEM lanes [32q, 32q+32)
+    if (mbar_wait(acc_done, 0, status, 104) && *(volatile int*)status == 0) {
+      tc_fence_after();
+      const int row = mtile * kTileM + q * 32 + lane;
+      __nv_bfloat16* dst = kv + ((int64_t)bh * m + row) * C::kN;
+#pragma unroll 1
+      for (int c0 = 0; c0 < C::kN; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+        tmem_wait_ld();
+        if (row < m) {
+          uint4* o = reinterpret_cast<uint4*>(dst + c0);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              __nv_bfloat162 p = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2 * j]),
+                                                       __uint_as_float(r[v * 8 + 2 * j + 1]));
+              w[j] = *reinterpret_cast<uint32_t*>(&p);
+            }
+            o[v] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem_base, C::kN);
+}
+
+template <int D>
+cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
+  using C = Cfg<D>;
+  const Params& p = c->p;
+  CUtensorMap tk, tv;
+  const uint64_t kd[3] = {(uint64_t)D, (uint64_t)p.n, (uint64_t)(p.B * p.H)};
+  const uint64_t ks[2] = {(uint64_t)D * 2, (uint64_t)p.n * D * 2};
+  const uint32_t kb[3] = {64, (uint32_t)kChunk, 1};
+  cudaError_t e;
+  if ((e = make_tmap_bf16_3d(&tk, K, kd, ks, kb)) != cudaSuccess) return e;
+  if ((e = make_tmap_bf16_3d(&tv, V, kd, ks, kb)) != cudaSuccess) return e;
+  static bool attr_set = false;
+  if (!attr_set) {
+    e = cudaFuncSetAttribute(compress_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(p.B * p.H));
+  compress_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
+                                                                 (int)p.n, (int)p.H, c->status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t make_phi_tmap(csat_ctx* c) {
+  const Params& p = c->p;
+  const uint64_t d[3] = {(uint64_t)p.n_pad, (uint64_t)p.m, (uint64_t)p.H};
+  const uint64_t st[2] = {(uint64_t)p.n_pad * 2, (uint64_t)p.m * p.n_pad * 2};
+  const uint32_t b[3] = {(uint32_t)kChunk, (uint32_t)kTileM, 1};
+  return make_tmap_bf16_3d(&c->tmap_phi, c->phi, d, st, b);
+}
+
+cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches) {
+  *launches += 1;
+  return c->p.d == 64 ? launch<64>(c, K, V, s) : launch<128>(c, K, V, s);
+}
+
+}  // namespace csat

@@ -82,6 +82,11 @@ int allocate_and_generate(csat_ctx* c) {
   if ((e = dev_alloc(c, &c->kv, kv_bytes(p))) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(K~|V~) failed");
   if ((e = csat::launch_phi_gen(c->phi, p, 0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen launch");
   if ((e = cudaStreamSynchronize(0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen");
+  c->tmap_phi_valid = false;
+  if (p.dtype == CSAT_DTYPE_BF16 && (p.d == 64 || p.d == 128)) {
+    if ((e = csat::make_phi_tmap(c)) != cudaSuccess) return fail_cuda(c, e, "tensor map for Phi");
+    c->tmap_phi_valid = true;
+  }
   c->decoder_dirty = true;
   c->have_forward = false;
   return CSAT_OK;
@@ -386,7 +391,9 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   }
   cudaError_t e;
   // float32 contexts, and head sizes without a tensor-core kernel, take the FFMA kernels
-  if ((e = csat::launch_simt_compress(c, K, V, s, &launches)) != cudaSuccess) return fail_cuda(c, e, "compress launch");
+  const bool tensor_path = c->tmap_phi_valid && !c->force_simt;
+  e = tensor_path ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
+  if (e != cudaSuccess) return fail_cuda(c, e, "compress launch");
   prof_mark(c, s, CSAT_KERNEL_COMPRESS);
   if ((e = csat::launch_simt_attend_recover(c, Q, out, s, &launches)) != cudaSuccess)
     return fail_cuda(c, e, "attend/recover launch");

@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libcsat (not part of the ABI).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -38,6 +39,8 @@ struct csat_ctx {
   void* psi = nullptr;        // [Hpsi, d, d] dtype (user dictionary), null = identity
   void* dmat = nullptr;       // [H, d, d] dtype (user decoder matrix), null = Phi block
   bool psi_per_head = false;
+  CUtensorMap tmap_phi;       // TMA view of phi for the tensor-core compress kernel (bf16, d in {64,128})
+  bool tmap_phi_valid = false;
   double* Mf64 = nullptr;     // [H, d, d] scratch of the decoder set-up
   double* Gf64 = nullptr;     // [H, d, d]
   float* S_dec = nullptr;     // [H, d, d]  I - mu G
@@ -80,6 +83,10 @@ cudaError_t launch_decoder_setup(csat_ctx* c, cudaStream_t s, int* launches);
 // simt_forward.cu : plain FFMA path (fp32 accumulate), both storage types
 cudaError_t launch_simt_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches);
 cudaError_t launch_simt_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
+
+// compress_sm100.cu : tcgen05 / TMEM / TMA compression (bf16, d in {64, 128})
+cudaError_t make_phi_tmap(csat_ctx* c);
+cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches);
 
 // copies K~ or V~ out of the interleaved workspace: dst [B,H,m,d]
 cudaError_t launch_split_kv(const csat_ctx* c, void* kt, void* vt, cudaStream_t s);
