@@ -61,7 +61,8 @@ enum {
                           of text queries over compressed visual keys uses n_q != n     */
   CSAT_DTYPE = 3,      /* CSAT_DTYPE_BF16 (default) or CSAT_DTYPE_FP32                   */
   CSAT_T = 4,          /* recovery iterations (decoder depth t), default 10; 0 = out = Z */
-  CSAT_FORCE_SIMT = 5, /* diagnostic: 1 routes bf16 through the plain FFMA kernels       */
+  CSAT_FORCE_SIMT = 5, /* diagnostic: 1 routes bf16 through the plain FFMA kernels, 2 only
+                          the attention/recovery stage; 0 (default) = tensor-core kernels */
   CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls
                           (0 = off, default; at most 4096).  Setting it creates/destroys
                           events, so set it outside the timed region                    */

@@ -48,6 +48,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
   uint64_t* empty = full + C::kStages;
   uint64_t* acc_done = empty + C::kStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_done + 1);
+  int* cta_abort = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int mtile = blockIdx.x, bh = blockIdx.y, h = bh % H;
@@ -62,6 +63,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
       mbar_init(&empty[s], 1);
     }
     mbar_init(acc_done, 1);
+    *cta_abort = 0;
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -79,7 +81,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
       bool ok = true;
       for (int i = 0; i < nchunks && ok; ++i) {
         const int s = i % C::kStages;
-        ok = mbar_wait(&empty[s], ((i / C::kStages) & 1) ^ 1, status, 101);
+        ok = mbar_wait(&empty[s], ((i / C::kStages) & 1) ^ 1, status, 101, cta_abort);
         if (!ok) break;
         mbar_arrive_expect_tx(&full[s], C::kStageBytes);
         tma_load_3d(a_buf + s * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, h);
@@ -94,7 +96,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
       if (!ok) {
         // gave up: let copies that are still in flight land before the CTA's shared memory goes away
         for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
-          mbar_wait(&full[i % C::kStages], (i / C::kStages) & 1, status, 102);
+          mbar_wait(&full[i % C::kStages], (i / C::kStages) & 1, status, 102, cta_abort);
       }
     }
   } else if (warp == 1) {
@@ -103,7 +105,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
       bool ok = true;
       for (int i = 0; i < nchunks; ++i) {
         const int s = i % C::kStages;
-        ok = mbar_wait(&full[s], (i / C::kStages) & 1, status, 103);
+        ok = mbar_wait(&full[s], (i / C::kStages) & 1, status, 103, cta_abort);
         if (!ok) break;
         tc_fence_after();
         const uint64_t a_desc = make_smem_desc(smem_u32(a_buf + s * kABytes), 16, 1024);
@@ -117,7 +119,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
     }
   } else {
     const int q = warp & 3;                     // this warp may touch TMEM lanes [32q, 32q+32)
-    if (mbar_wait(acc_done, 0, status, 104) && *(volatile int*)status == 0) {
+    if (mbar_wait(acc_done, 0, status, 104, cta_abort) && *(volatile int*)cta_abort == 0) {
       tc_fence_after();
       const int row = mtile * kTileM + q * 32 + lane;
       __nv_bfloat16* dst = kv + ((int64_t)bh * m + row) * C::kN;

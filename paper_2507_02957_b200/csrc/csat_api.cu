@@ -66,6 +66,7 @@ void free_all(csat_ctx* c) {
   dev_free(c, &c->psi_f32, dd_bytes(p, 4));
   dev_free(c, &c->theta, (size_t)p.H * 4);
   dev_free(c, &c->mu, (size_t)p.H * 4);
+  dev_free(c, &c->mats_bf16, 3 * dd_bytes(p, 2));
   free_staging(c);
   prof_destroy(c);
   if (c->status) {
@@ -85,6 +86,7 @@ int allocate_and_generate(csat_ctx* c) {
   c->tmap_phi_valid = false;
   if (p.dtype == CSAT_DTYPE_BF16 && (p.d == 64 || p.d == 128)) {
     if ((e = csat::make_phi_tmap(c)) != cudaSuccess) return fail_cuda(c, e, "tensor map for Phi");
+    if ((e = csat::make_attend_tmaps(c)) != cudaSuccess) return fail_cuda(c, e, "tensor maps for K~|V~");
     c->tmap_phi_valid = true;
   }
   c->decoder_dirty = true;
@@ -174,7 +176,8 @@ csat_ctx* csat_create(int64_t n, int64_t m, int64_t d, int64_t H, uint64_t seed)
                         dev_alloc(c, &c->B_dec, dd_bytes(p, 4)) != cudaSuccess ||
                         dev_alloc(c, &c->psi_f32, dd_bytes(p, 4)) != cudaSuccess ||
                         dev_alloc(c, &c->theta, (size_t)H * 4) != cudaSuccess ||
-                        dev_alloc(c, &c->mu, (size_t)H * 4) != cudaSuccess))
+                        dev_alloc(c, &c->mu, (size_t)H * 4) != cudaSuccess ||
+                        dev_alloc(c, &c->mats_bf16, 3 * dd_bytes(p, 2)) != cudaSuccess))
     rc = fail(c, CSAT_ERR_ALLOC, "cudaMalloc(decoder matrices) failed");
   if (rc == CSAT_OK) rc = allocate_and_generate(c);
   if (rc != CSAT_OK) {
@@ -208,6 +211,10 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       p.B = v;
       c->have_forward = false;
       if (dev_alloc(c, &c->kv, kv_bytes(p)) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(K~|V~) failed");
+      if (c->tmap_phi_valid && csat::make_attend_tmaps(c) != cudaSuccess) {
+        c->tmap_phi_valid = false;
+        return fail(c, CSAT_ERR_CUDA, "tensor maps for K~|V~");
+      }
       return CSAT_OK;
     }
     case CSAT_NQ:
@@ -232,7 +239,8 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       p.T = (int)v;
       return CSAT_OK;
     case CSAT_FORCE_SIMT:
-      c->force_simt = v != 0;
+      if (v < 0 || v > 2) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_FORCE_SIMT must be 0, 1 or 2");
+      c->force_simt = (int)v;
       return CSAT_OK;
     case CSAT_PROFILE: {
       if (v < 0 || v > 4096) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_PROFILE must be in [0, 4096]");
@@ -391,12 +399,14 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   }
   cudaError_t e;
   // float32 contexts, and head sizes without a tensor-core kernel, take the FFMA kernels
-  const bool tensor_path = c->tmap_phi_valid && !c->force_simt;
-  e = tensor_path ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
+  const bool tc_compress = c->tmap_phi_valid && c->force_simt != 1;
+  const bool tc_attend = c->tmap_phi_valid && c->force_simt == 0;
+  e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
   if (e != cudaSuccess) return fail_cuda(c, e, "compress launch");
   prof_mark(c, s, CSAT_KERNEL_COMPRESS);
-  if ((e = csat::launch_simt_attend_recover(c, Q, out, s, &launches)) != cudaSuccess)
-    return fail_cuda(c, e, "attend/recover launch");
+  e = tc_attend ? csat::launch_sm100_attend_recover(c, Q, out, s, &launches)
+                : csat::launch_simt_attend_recover(c, Q, out, s, &launches);
+  if (e != cudaSuccess) return fail_cuda(c, e, "attend/recover launch");
   prof_mark(c, s, CSAT_KERNEL_ATTEND_RECOVER);
   if (c->prof_slots) ++c->prof_calls;
   c->have_forward = true;

@@ -31,7 +31,7 @@ struct Params {            // plain values kernels need
 struct csat_ctx {
   csat::Params p;
   int device = 0;
-  bool force_simt = false;
+  int force_simt = 0;         // diagnostic: 1 = FFMA kernels for everything, 2 = for attention/recovery only
 
   // library-owned device memory
   void* phi = nullptr;        // [H, m, n_pad] dtype
@@ -41,6 +41,11 @@ struct csat_ctx {
   bool psi_per_head = false;
   CUtensorMap tmap_phi;       // TMA view of phi for the tensor-core compress kernel (bf16, d in {64,128})
   bool tmap_phi_valid = false;
+  CUtensorMap tmap_kv;        // TMA view of the K~|V~ workspace
+  CUtensorMap tmap_mats;      // TMA view of mats_bf16
+  // bf16 operand copies of the decoder matrices for the tensor-core path: [H][3][d][d], each stored
+  // [output column][k] (k contiguous): 0 = mu G (symmetric), 1 = (mu M)^T, 2 = Psi
+  __nv_bfloat16* mats_bf16 = nullptr;
   double* Mf64 = nullptr;     // [H, d, d] scratch of the decoder set-up
   double* Gf64 = nullptr;     // [H, d, d]
   float* S_dec = nullptr;     // [H, d, d]  I - mu G
@@ -87,6 +92,10 @@ cudaError_t launch_simt_attend_recover(csat_ctx* c, const void* Q, void* out, cu
 // compress_sm100.cu : tcgen05 / TMEM / TMA compression (bf16, d in {64, 128})
 cudaError_t make_phi_tmap(csat_ctx* c);
 cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches);
+
+// attend_recover_sm100.cu : tcgen05 compressed attention + recovery (bf16, d in {64, 128})
+cudaError_t make_attend_tmaps(csat_ctx* c);
+cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
 
 // copies K~ or V~ out of the interleaved workspace: dst [B,H,m,d]
 cudaError_t launch_split_kv(const csat_ctx* c, void* kt, void* vt, cudaStream_t s);

@@ -53,7 +53,7 @@ template <typename T>
 __global__ void finalize_kernel(float* __restrict__ S_dec, float* __restrict__ B_dec, float* __restrict__ theta,
                                 float* __restrict__ mu_out, float* __restrict__ psi_f32, const double* __restrict__ G,
                                 const double* __restrict__ M, const T* __restrict__ psi, int psi_per_head, int d,
-                                double lambda, double step) {
+                                double lambda, double step, __nv_bfloat16* __restrict__ mats_bf16) {
   __shared__ double red[256];
   const int h = blockIdx.x, t = threadIdx.x;
   const double* Gh = G + (int64_t)h * d * d;
@@ -74,6 +74,14 @@ __global__ void finalize_kernel(float* __restrict__ S_dec, float* __restrict__ B
     S_dec[(int64_t)h * d * d + i] = (float)((a == b ? 1.0 : 0.0) - mu * Gh[i]);
     B_dec[(int64_t)h * d * d + i] = (float)(mu * Mh[i]);
     if (psi) psi_f32[(int64_t)h * d * d + i] = (float)ld(psi + (psi_per_head ? (int64_t)h * d * d : 0), i);
+    if (mats_bf16) {
+      // tensor-core operand copies, each stored [output column][k]: mu G (symmetric), (mu M)^T, Psi
+      __nv_bfloat16* mh = mats_bf16 + (int64_t)h * 3 * d * d;
+      mh[i] = __float2bfloat16_rn((float)(mu * Gh[i]));
+      mh[d * d + i] = __float2bfloat16_rn((float)(mu * Mh[b * d + a]));
+      mh[2 * d * d + i] =
+          psi ? __float2bfloat16_rn((float)ld(psi + (psi_per_head ? (int64_t)h * d * d : 0), i)) : __float2bfloat16_rn(0.f);
+    }
   }
   if (t == 0) {
     theta[h] = (float)(mu * lambda);
@@ -90,7 +98,7 @@ cudaError_t run(csat_ctx* c, cudaStream_t s, int* launches) {
                                          c->psi_per_head ? 1 : 0, d, p.m, p.n_pad);
   gram_kernel<<<grid, 256, 0, s>>>(c->Gf64, c->Mf64, d);
   finalize_kernel<T><<<H, 256, 0, s>>>(c->S_dec, c->B_dec, c->theta, c->mu, c->psi_f32, c->Gf64, c->Mf64,
-                                       (const T*)c->psi, c->psi_per_head ? 1 : 0, d, p.lambda, p.step);
+                                       (const T*)c->psi, c->psi_per_head ? 1 : 0, d, p.lambda, p.step, c->mats_bf16);
   *launches += 3;
   return cudaGetLastError();
 }
