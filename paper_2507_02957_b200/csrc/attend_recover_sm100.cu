@@ -4,17 +4,30 @@
 // alpha^{t+1} = eta_theta(S alpha^t + B Z_i) (LISTA recurrence with S = I - mu G, B = mu M); C^_i = Psi alpha^_i.
 // Neither the 128 x m block of A~ nor any iterate alpha^t leaves the SM.
 //
-// CTA = 10 warps:
+// Two CTAs are resident per SM (<= 96 registers, ~100 KB shared memory, 256 tensor-memory columns each), so
+// that one tile's MMAs run while the other tile's threads do the softmax / shrinkage arithmetic.
+//
+// CTA = 9 warps:
 //   warps 0-7 (256 threads): two threads per query row (TMEM lane = row; warps w and w+4 share the lane
-//             quarter w and split the columns).  Softmax statistics, exp2, P -> bf16 -> shared memory,
+//             quarter w and split the columns).  Softmax statistics, exp2, P -> bf16 -> tensor memory,
 //             Z accumulation in fp32 registers, soft-threshold, output.
-//   warp 8  : TMA producer (Q tile, K~|V~ chunks of kMC measurements, decoder matrices).
-//   warp 9  : TMEM allocation; one elected thread issues every tcgen05.mma.
-// Attention phase, per chunk j of measurements:  S_j = Q K~_j^T (TMEM, double buffered) -> threads read
-// S_j, update the running row maximum, write P_j = exp2(S_j - max) as the bf16 A operand ->
-// Zc_j = P_j V~_j (TMEM, fresh accumulator) -> threads fold it in: z = z * corr_j + Zc_j.
-// Recovery phase: c = z B (one MMA), alpha^1 = eta(c); then T-1 times R = alpha_bf16 (mu G),
-// alpha <- eta(alpha - R + c); alpha and c stay in fp32 registers, only the MMA operand copy is bf16.
+//   warp 8  : allocates tensor memory; one elected thread issues every TMA copy and every tcgen05.mma.
+//
+// Attention phase, per chunk j of 64 measurements:
+//   S_j = Q K~_j^T            (SS MMA, accumulator S[j&1] in tensor memory)
+//   threads read S_j, update the running row maximum, write P_j = exp2(S_j - max) as packed bf16 over the
+//   first half of S[j&1]'s columns
+//   Zc_j = P_j V~_j           (TS MMA: A operand from tensor memory, fresh accumulator)
+//   threads fold it in: z = z * corr_j + Zc_j.
+// MMAs of one CTA execute in issue order (S_0, S_1, PV_0, S_2, PV_1, ...), so S_{j+2} overwrites S[j&1] only
+// after PV_j has read P_j from it.
+//
+// Recovery phase.  The accumulator holds r_t = c - a^_t (mu G), where c = z B and a^_t is the sum of the bf16
+// increments fed to the tensor cores so far:
+//   r_0 = z_bf16 B (one MMA);  alpha^{t+1} = eta_theta(alpha^t + r_t);
+//   r_{t+1} = r_t + bf16(alpha^t - alpha^{t+1}) (mu G)     (one accumulating MMA per iteration).
+// This is the paper's S alpha + B z with S = I - mu G: the identity part stays exact in fp32 registers, only
+// the increment that multiplies mu G is rounded to bf16, and c never needs registers of its own.
 #include "csat_internal.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -27,51 +40,52 @@ using namespace ptx;
 constexpr int kRows = 128;            // queries per CTA
 constexpr int kMC = 64;               // measurements per chunk
 constexpr int kComputeThreads = 256;
-constexpr int kThreads = 320;
-constexpr int kKvStages = 3;
+constexpr int kThreads = 288;
+constexpr int kMaxStages = 4;
 
 template <int D> struct Cfg {
   static constexpr int kDBoxes = D / 64;                          // 64-column boxes across the head dimension
-  static constexpr uint32_t kABytes = kDBoxes * kRows * 128;      // Q tile / bf16 operand copy of z, alpha
-  static constexpr uint32_t kKHalf = kDBoxes * kMC * 128;         // K~ chunk (= V~ chunk)
-  static constexpr uint32_t kStageBytes = 2 * kKHalf;
-  static constexpr uint32_t kPBytes = kRows * 128;                // P chunk: 128 x 64 bf16
-  static constexpr uint32_t kMatBytes = kDBoxes * D * 128;        // one d x d bf16 matrix
-  static constexpr uint32_t kOffA = 0;
-  static constexpr uint32_t kOffKv = kOffA + kABytes;
-  static constexpr uint32_t kOffP = kOffKv + kKvStages * kStageBytes;
-  static constexpr uint32_t kOffG = kOffP + 2 * kPBytes;
-  static constexpr uint32_t kOffB = kOffG + kMatBytes;
-  static constexpr uint32_t kOffBar = kOffB + kMatBytes;
-  static constexpr uint32_t kBarBytes = 256 + 2048;               // barriers | row statistics exchange
+  static constexpr int kStages = (D == 64) ? 4 : 2;               // K~ / V~ chunks in flight
+  static constexpr uint32_t kQBytes = kDBoxes * kRows * 128;      // Q tile; later the matrix B
+  static constexpr uint32_t kBoxBytes = kMC * 128;                // one 64-column box of a K~ or V~ chunk
+  static constexpr uint32_t kSlotBytes = kDBoxes * kBoxBytes;     // K~ chunk (= V~ chunk)
+  static constexpr uint32_t kMatBoxBytes = D * 128;               // one 64-column box of a d x d bf16 matrix
+  static constexpr uint32_t kMatBytes = kDBoxes * kMatBoxBytes;
+  static constexpr uint32_t kOffQ = 0;
+  static constexpr uint32_t kOffRing = kOffQ + kQBytes;           // [stage][K~ slot | V~ slot]
+  static constexpr uint32_t kOffBar = kOffRing + kStages * 2 * kSlotBytes;
+  static constexpr uint32_t kBarBytes = 256 + 2048;               // barriers | row-maximum exchange
   static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes;     // base must be 1024-byte aligned (checked)
-  // TMEM columns: S[2] | Zc[2]; the recovery accumulator R reuses Zc[0]
-  static constexpr uint32_t kColS = 0, kColZ = 2 * kMC, kTmemCols = (2 * kMC + 2 * D <= 256) ? 256 : 512;
-  static_assert(2 * kMC + 2 * D <= 512, "TMEM budget");
-  static_assert(kMatBytes <= kStageBytes, "Psi is staged in a K~|V~ buffer");
-  static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+  // TMEM columns: S[0] | S[1] | accumulator (Zc, then r_t).  P_j overlays S[j&1]; the recovery operand S[0].
+  static constexpr uint32_t kColS = 0, kColAcc = 2 * kMC, kTmemCols = 256;
+  static_assert(2 * kMC + D <= 256, "TMEM budget");
+  static_assert(D / 2 <= 2 * kMC, "recovery operand fits in the S columns");
+  static_assert(kStages >= kDBoxes && kStages <= kMaxStages, "mu G and Psi are staged box by box in ring slots");
+  static_assert(kMatBoxBytes <= kSlotBytes && kMatBytes <= kQBytes, "decoder matrices fit where they are staged");
+  static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two CTAs per SM");
 };
 
 struct Bars {
-  uint64_t q_full, mats_full, psi_full, attn_done;
-  uint64_t kv_full[kKvStages], kv_empty[kKvStages];
-  uint64_t s_full[2], s_empty[2], p_full[2], p_empty[2], zc_full[2], zc_empty[2];
+  uint64_t q_full, mats_full, psi_full;
+  uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
+  uint64_t s_full[2], p_full[2], zc_full, zc_empty;
   uint64_t a_full, r_full;
   uint32_t tmem_slot;
   int abort;
 };
+static_assert(sizeof(Bars) <= 256, "barrier block");
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-__device__ __forceinline__ float soft(float x, float th) { return x - fminf(fmaxf(x, -th), th); }
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&p);
 }
-__device__ __forceinline__ void named_barrier_256() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// warps q and q+4 (the two halves of the same 32 rows) meet here
+__device__ __forceinline__ void pair_barrier(int q) { asm volatile("bar.sync %0, 64;" ::"r"(q + 1) : "memory"); }
 
 // A wait that never blocks for more than the time-out and turns into a no-op once anything gave up.
 struct Waiter {
@@ -84,14 +98,8 @@ struct Waiter {
   }
 };
 
-// writes 8 consecutive bf16 (one 16-byte chunk) of row r into a K-major 128-byte-swizzled box
-__device__ __forceinline__ void st_chunk(uint8_t* box, int r, int chunk, const float* v) {
-  uint4 w = make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
-  *reinterpret_cast<uint4*>(box + r * 128 + ((chunk ^ (r & 7)) << 4)) = w;
-}
-
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int nq, int m, int H, int T, int has_psi,
@@ -103,17 +111,16 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     if (threadIdx.x == 0) atomicCAS(status, 0, 200);
     return;
   }
-  uint8_t* a_buf = smem + C::kOffA;
-  uint8_t* kv_buf = smem + C::kOffKv;
-  uint8_t* p_buf = smem + C::kOffP;
-  uint8_t* g_buf = smem + C::kOffG;
-  uint8_t* b_buf = smem + C::kOffB;
+  uint8_t* q_buf = smem + C::kOffQ;
+  uint8_t* ring = smem + C::kOffRing;
   Bars* bars = reinterpret_cast<Bars*>(smem + C::kOffBar);
   float* xch = reinterpret_cast<float*>(smem + C::kOffBar + 256);   // [2 buffers][2 halves][128 rows] floats
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int qtile = blockIdx.x, bh = blockIdx.y, h = bh % H;
   const int nchunks = (m + kMC - 1) / kMC;
   Waiter w{status, &bars->abort};
+  auto k_slot = [&](int s) { return ring + (2 * s) * C::kSlotBytes; };
+  auto v_slot = [&](int s) { return ring + (2 * s + 1) * C::kSlotBytes; };
 
   if (threadIdx.x == 0) {
     prefetch_tmap(&tmap_q);
@@ -122,19 +129,19 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     mbar_init(&bars->q_full, 1);
     mbar_init(&bars->mats_full, 1);
     mbar_init(&bars->psi_full, 1);
-    mbar_init(&bars->attn_done, kComputeThreads);
-    for (int s = 0; s < kKvStages; ++s) { mbar_init(&bars->kv_full[s], 1); mbar_init(&bars->kv_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&bars->s_full[s], 1);  mbar_init(&bars->s_empty[s], kComputeThreads);
-      mbar_init(&bars->p_full[s], kComputeThreads);  mbar_init(&bars->p_empty[s], 1);
-      mbar_init(&bars->zc_full[s], 1); mbar_init(&bars->zc_empty[s], kComputeThreads);
+    for (int s = 0; s < C::kStages; ++s) {
+      mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1);
+      mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
     }
+    for (int s = 0; s < 2; ++s) { mbar_init(&bars->s_full[s], 1); mbar_init(&bars->p_full[s], kComputeThreads); }
+    mbar_init(&bars->zc_full, 1);
+    mbar_init(&bars->zc_empty, kComputeThreads);
     mbar_init(&bars->a_full, kComputeThreads);
     mbar_init(&bars->r_full, 1);
     bars->abort = 0;
     fence_mbar_init();
   }
-  if (warp == 9) {
+  if (warp == 8) {
     tmem_alloc(&bars->tmem_slot, C::kTmemCols);
     tmem_relinquish();
   }
@@ -144,95 +151,162 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   const uint32_t tmem = bars->tmem_slot;
 
   if (warp == 8) {
-    // ------------------------------------------------ TMA producer ------------------------------------------------
-    if (elect_one()) {
-      mbar_arrive_expect_tx(&bars->q_full, C::kABytes);
-      for (int g = 0; g < C::kDBoxes; ++g)
-        tma_load_3d(a_buf + g * kRows * 128, &tmap_q, &bars->q_full, g * 64, qtile * kRows, bh);
-      if (T > 0) {
-        mbar_arrive_expect_tx(&bars->mats_full, 2 * C::kMatBytes);
-        for (int g = 0; g < C::kDBoxes; ++g) {
-          tma_load_3d(g_buf + g * D * 128, &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 0);
-          tma_load_3d(b_buf + g * D * 128, &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 1);
-        }
-      }
-      for (int j = 0; j < nchunks; ++j) {
-        const int s = j % kKvStages;
-        w.wait(&bars->kv_empty[s], ((j / kKvStages) & 1) ^ 1, 201);
-        if (w.dead) break;
-        uint8_t* st = kv_buf + s * C::kStageBytes;
-        mbar_arrive_expect_tx(&bars->kv_full[s], C::kStageBytes);
-        for (int g = 0; g < C::kDBoxes; ++g) {
-          tma_load_3d(st + g * kMC * 128, &tmap_kv, &bars->kv_full[s], g * 64, j * kMC, bh);                  // K~
-          tma_load_3d(st + C::kKHalf + g * kMC * 128, &tmap_kv, &bars->kv_full[s], D + g * 64, j * kMC, bh);  // V~
-        }
-      }
-      if (T > 0 && has_psi) {
-        // Psi is staged in K~|V~ buffer 0 once the attention phase no longer needs it
-        w.wait(&bars->attn_done, 0, 202);
-        if (!w.dead) {
-          mbar_arrive_expect_tx(&bars->psi_full, C::kMatBytes);
-          for (int g = 0; g < C::kDBoxes; ++g)
-            tma_load_3d(kv_buf + g * D * 128, &tmap_mats, &bars->psi_full, g * 64, 0, h * 3 + 2);
-        }
-      }
-    }
-  } else if (warp == 9) {
-    // ------------------------------------------------ MMA issuer --------------------------------------------------
+    // ------------------------------------ TMA copies and MMA issue (one thread) -----------------------------------
     if (elect_one()) {
       constexpr uint32_t idesc_s = make_idesc_bf16(kRows, kMC, false, false);   // S  = Q  K~^T : both K-major
       constexpr uint32_t idesc_z = make_idesc_bf16(kRows, D, false, true);      // Zc = P  V~   : V~ is MN-major
-      constexpr uint32_t idesc_r = make_idesc_bf16(kRows, D, false, false);     // R  = a  W^T  : both K-major
-      auto issue_pv = [&](int i) {
-        const int s = i % kKvStages, b = i & 1;
-        w.wait(&bars->p_full[b], (i >> 1) & 1, 211);
-        w.wait(&bars->zc_empty[b], ((i >> 1) & 1) ^ 1, 212);
-        tc_fence_after();
-        const uint64_t a_desc = make_smem_desc(smem_u32(p_buf + b * C::kPBytes), 16, 1024);
-        const uint64_t b_desc = make_smem_desc(smem_u32(kv_buf + s * C::kStageBytes + C::kKHalf), kMC * 128, 1024);
-#pragma unroll
-        for (int k = 0; k < kMC / 16; ++k)
-          mma_f16_ss(tmem + C::kColZ + b * D, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc_z, k != 0);
-        mma_commit(&bars->zc_full[b]);
-        mma_commit(&bars->kv_empty[s]);
-        mma_commit(&bars->p_empty[b]);
+      constexpr uint32_t idesc_r = make_idesc_bf16(kRows, D, false, false);     // r  = a  W^T  : both K-major
+      int next_k = 0, next_v = 0;           // next chunk whose K~ / V~ copy has not been issued
+      int seen_k = 0, seen_v = 0;           // chunks whose copy this thread has waited for
+      bool q_issued = false, mats_issued = false, psi_issued = false, mats_seen = false, psi_seen = false;
+
+      auto issue_k = [&](int c) {
+        const int s = c % C::kStages;
+        mbar_arrive_expect_tx(&bars->k_full[s], C::kSlotBytes);
+        for (int g = 0; g < C::kDBoxes; ++g)
+          tma_load_3d(k_slot(s) + g * C::kBoxBytes, &tmap_kv, &bars->k_full[s], g * 64, c * kMC, bh);
       };
+      auto issue_v = [&](int c) {
+        const int s = c % C::kStages;
+        mbar_arrive_expect_tx(&bars->v_full[s], C::kSlotBytes);
+        for (int g = 0; g < C::kDBoxes; ++g)
+          tma_load_3d(v_slot(s) + g * C::kBoxBytes, &tmap_kv, &bars->v_full[s], D + g * 64, c * kMC, bh);
+      };
+      // issues every copy whose slot is free right now; never blocks
+      auto service = [&]() {
+        while (next_k < nchunks) {
+          const int s = next_k % C::kStages, use = next_k / C::kStages;
+          if (use > 0 && !mbar_try_wait(&bars->k_empty[s], (use - 1) & 1)) break;
+          issue_k(next_k++);
+        }
+        while (next_v < nchunks) {
+          const int s = next_v % C::kStages, use = next_v / C::kStages;
+          if (use > 0 && !mbar_try_wait(&bars->v_empty[s], (use - 1) & 1)) break;
+          issue_v(next_v++);
+        }
+      };
+      // bounded wait that keeps the copies flowing while it spins
+      auto wait_serving = [&](uint64_t* bar, uint32_t parity, int code) {
+        if (w.dead) return;
+        if (mbar_try_wait(bar, parity)) return;
+        const unsigned long long t0 = globaltimer();
+        uint32_t spins = 0;
+        while (!mbar_try_wait(bar, parity)) {
+          service();
+          if ((++spins & 0xff) == 0) {
+            if (*(volatile int*)&bars->abort != 0) { w.dead = true; return; }
+            if (globaltimer() - t0 > kWaitTimeoutNs) {
+              *(volatile int*)&bars->abort = 1;
+              atomicCAS(status, 0, code);
+              w.dead = true;
+              return;
+            }
+          }
+        }
+      };
+      // the copies of chunk c must have been issued before their barrier is waited for
+      auto ensure_k = [&](int c) {
+        while (next_k <= c && !w.dead) {
+          const int s = next_k % C::kStages, use = next_k / C::kStages;
+          if (use > 0) w.wait(&bars->k_empty[s], (use - 1) & 1, 201);
+          if (!w.dead) issue_k(next_k++);
+        }
+      };
+      auto ensure_v = [&](int c) {
+        while (next_v <= c && !w.dead) {
+          const int s = next_v % C::kStages, use = next_v / C::kStages;
+          if (use > 0) w.wait(&bars->v_empty[s], (use - 1) & 1, 202);
+          if (!w.dead) issue_v(next_v++);
+        }
+      };
+      auto issue_pv = [&](int i) {
+        const int s = i % C::kStages, b = i & 1;
+        ensure_v(i);
+        wait_serving(&bars->v_full[s], (i / C::kStages) & 1, 211);
+        if (!w.dead) seen_v = i + 1;
+        wait_serving(&bars->p_full[b], (i >> 1) & 1, 212);
+        if (i > 0) wait_serving(&bars->zc_empty, (i - 1) & 1, 213);   // Zc_{i-1} has been folded
+        tc_fence_after();
+        const uint64_t b_desc = make_smem_desc(smem_u32(v_slot(s)), C::kBoxBytes, 1024);
+#pragma unroll
+        for (int k = 0; k < kMC / 16; ++k)     // P: 8 packed columns per 16 measurements; V~: +16 rows = 2048 B
+          mma_f16_ts(tmem + C::kColAcc, tmem + C::kColS + b * kMC + k * 8, b_desc + (uint64_t)(k * 128), idesc_z, k != 0);
+        mma_commit(&bars->zc_full);
+        mma_commit(&bars->v_empty[s]);
+      };
+
+      mbar_arrive_expect_tx(&bars->q_full, C::kQBytes);
+      for (int g = 0; g < C::kDBoxes; ++g)
+        tma_load_3d(q_buf + g * kRows * 128, &tmap_q, &bars->q_full, g * 64, qtile * kRows, bh);
+      q_issued = true;
+      service();
       w.wait(&bars->q_full, 0, 210);
       for (int j = 0; j < nchunks; ++j) {
-        const int s = j % kKvStages, b = j & 1;
-        w.wait(&bars->kv_full[s], (j / kKvStages) & 1, 213);
-        w.wait(&bars->s_empty[b], ((j >> 1) & 1) ^ 1, 214);
+        const int s = j % C::kStages, b = j & 1;
+        ensure_k(j);
+        wait_serving(&bars->k_full[s], (j / C::kStages) & 1, 214);
+        if (!w.dead) seen_k = j + 1;
         tc_fence_after();
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) {
-          const uint64_t a_desc = make_smem_desc(smem_u32(a_buf + (k / 4) * kRows * 128), 16, 1024) + (uint64_t)((k % 4) * 2);
-          const uint64_t b_desc =
-              make_smem_desc(smem_u32(kv_buf + s * C::kStageBytes + (k / 4) * kMC * 128), 16, 1024) + (uint64_t)((k % 4) * 2);
+          const uint64_t a_desc = make_smem_desc(smem_u32(q_buf + (k / 4) * kRows * 128), 16, 1024) + (uint64_t)((k % 4) * 2);
+          const uint64_t b_desc = make_smem_desc(smem_u32(k_slot(s) + (k / 4) * C::kBoxBytes), 16, 1024) + (uint64_t)((k % 4) * 2);
           mma_f16_ss(tmem + C::kColS + b * kMC, a_desc, b_desc, idesc_s, k != 0);
         }
         mma_commit(&bars->s_full[b]);
+        mma_commit(&bars->k_empty[s]);
         if (j > 0) issue_pv(j - 1);
+        service();
+      }
+      if (T > 0) {
+        // every S MMA has finished once the last one has: Q and the K~ slots are free for mu G and B
+        const int last = nchunks - 1;
+        wait_serving(&bars->k_empty[last % C::kStages], (last / C::kStages) & 1, 215);
+        if (!w.dead) {
+          mbar_arrive_expect_tx(&bars->mats_full, 2 * C::kMatBytes);
+          for (int g = 0; g < C::kDBoxes; ++g) {
+            tma_load_3d(k_slot(g), &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 0);                          // mu G
+            tma_load_3d(q_buf + g * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 1);       // B
+          }
+          mats_issued = true;
+        }
       }
       issue_pv(nchunks - 1);
       if (T > 0) {
-        w.wait(&bars->mats_full, 0, 215);
-        const int n_mma = T + (has_psi ? 1 : 0);            // c = zB, then T-1 products with mu G, then Psi
-        for (int i = 0; i < n_mma; ++i) {
-          const uint8_t* wsm = (i == 0) ? b_buf : g_buf;
-          if (has_psi && i == n_mma - 1) {
-            w.wait(&bars->psi_full, 0, 216);
-            wsm = kv_buf;
+        if (has_psi) {
+          // Psi goes to the V~ slots once the last P V~ product has read them
+          const int last = nchunks - 1;
+          w.wait(&bars->v_empty[last % C::kStages], (last / C::kStages) & 1, 216);
+          if (!w.dead) {
+            mbar_arrive_expect_tx(&bars->psi_full, C::kMatBytes);
+            for (int g = 0; g < C::kDBoxes; ++g)
+              tma_load_3d(v_slot(g), &tmap_mats, &bars->psi_full, g * 64, 0, h * 3 + 2);
+            psi_issued = true;
           }
-          w.wait(&bars->a_full, i & 1, 217);
+        }
+        const int n_mma = T + (has_psi ? 1 : 0);            // r_0 = z B, then T-1 increments with mu G, then Psi
+        for (int i = 0; i < n_mma; ++i) {
+          const bool first = (i == 0), psi_step = has_psi && i == n_mma - 1;
+          if (first) { w.wait(&bars->mats_full, 0, 217); if (!w.dead) mats_seen = true; }
+          if (psi_step) { w.wait(&bars->psi_full, 0, 218); if (!w.dead) psi_seen = true; }
+          w.wait(&bars->a_full, i & 1, 219);
           tc_fence_after();
 #pragma unroll
           for (int k = 0; k < D / 16; ++k) {
-            const uint64_t a_desc = make_smem_desc(smem_u32(a_buf + (k / 4) * kRows * 128), 16, 1024) + (uint64_t)((k % 4) * 2);
-            const uint64_t b_desc = make_smem_desc(smem_u32(wsm + (k / 4) * D * 128), 16, 1024) + (uint64_t)((k % 4) * 2);
-            mma_f16_ss(tmem + C::kColZ, a_desc, b_desc, idesc_r, k != 0);
+            const uint8_t* box = first ? q_buf + (k / 4) * C::kMatBoxBytes : (psi_step ? v_slot(k / 4) : k_slot(k / 4));
+            const uint64_t b_desc = make_smem_desc(smem_u32(box), 16, 1024) + (uint64_t)((k % 4) * 2);
+            mma_f16_ts(tmem + C::kColAcc, tmem + C::kColS + k * 8, b_desc, idesc_r, (first || psi_step) ? (k != 0) : 1u);
           }
           mma_commit(&bars->r_full);
         }
+      }
+      if (w.dead) {
+        // gave up: let the copies that are still in flight land before the CTA's shared memory goes away
+        if (q_issued) mbar_wait_drain(&bars->q_full, 0);
+        for (int c = seen_k; c < next_k; ++c) mbar_wait_drain(&bars->k_full[c % C::kStages], (c / C::kStages) & 1);
+        for (int c = seen_v; c < next_v; ++c) mbar_wait_drain(&bars->v_full[c % C::kStages], (c / C::kStages) & 1);
+        if (mats_issued && !mats_seen) mbar_wait_drain(&bars->mats_full, 0);
+        if (psi_issued && !psi_seen) mbar_wait_drain(&bars->psi_full, 0);
       }
     }
   } else {
@@ -246,19 +320,18 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     float run_max = -INFINITY, run_sum = 0.f, corr_prev = 0.f;
 
     auto fold_zc = [&](int i, float corr) {
-      const int b = i & 1;
-      w.wait(&bars->zc_full[b], (i >> 1) & 1, 221);
+      w.wait(&bars->zc_full, i & 1, 221);
       tc_fence_after();
 #pragma unroll
-      for (int c0 = 0; c0 < HC; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(tmem + lane_addr + C::kColZ + b * D + half * HC + c0, r);
+      for (int c0 = 0; c0 < HC; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(tmem + lane_addr + C::kColAcc + half * HC + c0, r);
         tmem_wait_ld();
 #pragma unroll
-        for (int e = 0; e < 32; ++e) z[c0 + e] = fmaf(z[c0 + e], corr, __uint_as_float(r[e]));
+        for (int e = 0; e < 16; ++e) z[c0 + e] = fmaf(z[c0 + e], corr, __uint_as_float(r[e]));
       }
       tc_fence_before();
-      mbar_arrive(&bars->zc_empty[b]);
+      mbar_arrive(&bars->zc_empty);
     };
 
     for (int j = 0; j < nchunks; ++j) {
@@ -268,98 +341,119 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       uint32_t r[32];
       tmem_ld_32x32b_x32(tmem + lane_addr + C::kColS + b * kMC + half * 32, r);
       tmem_wait_ld();
-      tc_fence_before();
-      mbar_arrive(&bars->s_empty[b]);
       // scores in the log2 domain; measurements beyond m are masked out
-      float t[32], mx = -INFINITY;
+      float mx = -INFINITY;
       const int col0 = j * kMC + half * 32;
+      if (col0 + 32 <= m) {
 #pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        t[e] = (col0 + e < m) ? __uint_as_float(r[e]) * scale_log2 : -INFINITY;
-        mx = fmaxf(mx, t[e]);
+        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
+      } else {
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          if (col0 + e >= m) r[e] = 0xff800000u;                // -inf
+          mx = fmaxf(mx, __uint_as_float(r[e]));
+        }
       }
+      mx *= scale_log2;                                         // scale > 0: the maximum commutes with it
       float* slot = xch + b * 256;
       slot[half * 128 + row] = mx;
-      named_barrier_256();
+      pair_barrier(q);              // also orders this thread's S read before its partner's P write below
       mx = fmaxf(mx, slot[(half ^ 1) * 128 + row]);
       const float new_max = fmaxf(run_max, mx);                 // finite: chunk 0 has a valid measurement
       const float corr = ex2(run_max - new_max);
       run_max = new_max;
       float sum = 0.f;
+      uint32_t pk[16];
 #pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        t[e] = ex2(t[e] - new_max);
-        sum += t[e];
+      for (int e = 0; e < 32; e += 2) {
+        const float p0 = ex2(fmaf(__uint_as_float(r[e]), scale_log2, -new_max));
+        const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), scale_log2, -new_max));
+        sum += p0 + p1;
+        pk[e >> 1] = pack_bf16(p0, p1);
       }
       run_sum = fmaf(run_sum, corr, sum);
-      w.wait(&bars->p_empty[b], ((j >> 1) & 1) ^ 1, 222);       // P buffer free again
-#pragma unroll
-      for (int c = 0; c < 4; ++c) st_chunk(p_buf + b * C::kPBytes, row, half * 4 + c, &t[c * 8]);
-      fence_proxy_async();
+      // P_j over the first 32 columns of S[b]: this half's 32 measurements are packed columns [16 half, +16)
+      tmem_st_32x32b_x16(tmem + lane_addr + C::kColS + b * kMC + half * 16, pk);
+      tmem_wait_st();
+      tc_fence_before();
       mbar_arrive(&bars->p_full[b]);
       if (j > 0) fold_zc(j - 1, corr_prev);
       corr_prev = corr;
     }
     fold_zc(nchunks - 1, corr_prev);
     // the two halves of a row share max and corr; their partial sums are added once
-    float* slot = xch;               // reused once every thread is past the last chunk's exchange
-    named_barrier_256();
+    float* slot = xch + (nchunks & 1) * 256;   // the buffer the last chunk did not use
     slot[half * 128 + row] = run_sum;
-    named_barrier_256();
+    pair_barrier(q);
     const float inv = 1.f / (run_sum + slot[(half ^ 1) * 128 + row]);
 #pragma unroll
     for (int i = 0; i < HC; ++i) z[i] *= inv;
-    mbar_arrive(&bars->attn_done);
 
     if (T > 0) {
       const float th = theta[h];
-      // the thread's HC columns sit in box (half*HC)/64 at chunks ((half*HC)%64)/8 ...
-      uint8_t* box = a_buf + ((half * HC) / 64) * kRows * 128;
-      const int chunk0 = ((half * HC) % 64) / 8;
-      auto publish = [&](const float* v) {                      // bf16 operand copy for the next MMA
-#pragma unroll
-        for (int c = 0; c < HC / 8; ++c) st_chunk(box, row, chunk0 + c, v + c * 8);
-        fence_proxy_async();
-        tc_fence_before();
-        mbar_arrive(&bars->a_full);
-      };
-      float cvec[HC];
-      int phase = 0;
-      publish(z);
-      w.wait(&bars->r_full, phase & 1, 230); ++phase;
-      tc_fence_after();
+      const uint32_t op_addr = tmem + lane_addr + C::kColS + half * (HC / 2);   // this thread's operand columns
+      // z as the bf16 A operand of r_0 = z B
 #pragma unroll
       for (int c0 = 0; c0 < HC; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(tmem + lane_addr + C::kColZ + half * HC + c0, r);
-        tmem_wait_ld();
+        uint32_t pk[16];
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          cvec[c0 + e] = __uint_as_float(r[e]);
-          z[c0 + e] = soft(cvec[c0 + e], th);                   // alpha^1 (alpha^0 = 0)
-        }
+        for (int e = 0; e < 32; e += 2) pk[e >> 1] = pack_bf16(z[c0 + e], z[c0 + e + 1]);
+        tmem_st_32x32b_x16(op_addr + c0 / 2, pk);
       }
-      for (int it = 1; it < T; ++it) {
-        publish(z);
-        w.wait(&bars->r_full, phase & 1, 231); ++phase;
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars->a_full);
+#pragma unroll
+      for (int i = 0; i < HC; ++i) z[i] = 0.f;                  // z now holds alpha (alpha^0 = 0)
+      int phase = 0;
+      for (int it = 0; it < T; ++it) {
+        w.wait(&bars->r_full, phase & 1, 230); ++phase;
         tc_fence_after();
+        const bool more = it + 1 < T;
 #pragma unroll
-        for (int c0 = 0; c0 < HC; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld_32x32b_x32(tmem + lane_addr + C::kColZ + half * HC + c0, r);
+        for (int c0 = 0; c0 < HC; c0 += 16) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(tmem + lane_addr + C::kColAcc + half * HC + c0, r);
           tmem_wait_ld();
+          uint32_t pk[8];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) z[c0 + e] = soft(z[c0 + e] - __uint_as_float(r[e]) + cvec[c0 + e], th);
+          for (int e = 0; e < 16; e += 2) {
+            float nd[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const float rv = __uint_as_float(r[e + u]);
+              const float x = z[c0 + e + u] + rv;               // alpha^t S + z B, identity part in fp32
+              const float cl = fminf(fmaxf(x, -th), th);
+              z[c0 + e + u] = x - cl;                           // eta_theta(x)
+              nd[u] = cl - rv;                                  // alpha^t - alpha^{t+1}
+            }
+            pk[e >> 1] = pack_bf16(nd[0], nd[1]);
+          }
+          if (more) tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+        }
+        if (more) {
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&bars->a_full);
         }
       }
       if (has_psi) {
-        publish(z);
+#pragma unroll
+        for (int c0 = 0; c0 < HC; c0 += 32) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) pk[e >> 1] = pack_bf16(z[c0 + e], z[c0 + e + 1]);
+          tmem_st_32x32b_x16(op_addr + c0 / 2, pk);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bars->a_full);
         w.wait(&bars->r_full, phase & 1, 232); ++phase;
         tc_fence_after();
 #pragma unroll
         for (int c0 = 0; c0 < HC; c0 += 32) {
           uint32_t r[32];
-          tmem_ld_32x32b_x32(tmem + lane_addr + C::kColZ + half * HC + c0, r);
+          tmem_ld_32x32b_x32(tmem + lane_addr + C::kColAcc + half * HC + c0, r);
           tmem_wait_ld();
 #pragma unroll
           for (int e = 0; e < 32; ++e) z[c0 + e] = __uint_as_float(r[e]);
@@ -367,7 +461,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       }
     }
     const int grow = qtile * kRows + row;
-    if (grow < nq && !w.dead) {
+    if (grow < nq && !w.dead && *(volatile int*)&bars->abort == 0) {
       uint4* o = reinterpret_cast<uint4*>(out + ((int64_t)bh * nq + grow) * D + half * HC);
 #pragma unroll
       for (int c = 0; c < HC / 8; ++c)
@@ -377,7 +471,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 9) tmem_dealloc(tmem, C::kTmemCols);
+  if (warp == 8) tmem_dealloc(tmem, C::kTmemCols);
 }
 
 template <int D>
@@ -394,6 +488,10 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   if (!attr_set) {
     e = cudaFuncSetAttribute(attend_recover_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)C::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    // two CTAs per SM need the large shared-memory carve-out
+    e = cudaFuncSetAttribute(attend_recover_sm100_kernel<D>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                             (int)cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
