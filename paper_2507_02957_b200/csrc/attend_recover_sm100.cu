@@ -1,33 +1,41 @@
-// Compressed attention and sparse recovery for one tile of 128 queries, on the sm_100a tensor cores.
+// Compressed attention and sparse recovery for two tiles of 128 queries per CTA, on the sm_100a tensor cores.
 //
 // Paper, in order: A~ = softmax(Q K~^T / sqrt(d_k)) over the m measurements; Z = A~ V~;
 // alpha^{t+1} = eta_theta(S alpha^t + B Z_i) (LISTA recurrence with S = I - mu G, B = mu M); C^_i = Psi alpha^_i.
-// Neither the 128 x m block of A~ nor any iterate alpha^t leaves the SM.
+// Neither the n_q x m matrix A~ nor any iterate alpha^t leaves the SM.
 //
-// Two CTAs are resident per SM (<= 96 registers, ~100 KB shared memory, 256 tensor-memory columns each), so
-// that one tile's MMAs run while the other tile's threads do the softmax / shrinkage arithmetic.
+// One CTA per SM works on 256 consecutive queries of one (batch, head) as two independent tiles A and B that
+// share the stream of K~|V~ chunks.  While the tensor cores run one tile's MMAs the other tile's threads do
+// their softmax / shrinkage arithmetic, and the other way round.
 //
-// CTA = 9 warps:
-//   warps 0-7 (256 threads): two threads per query row (TMEM lane = row; warps w and w+4 share the lane
-//             quarter w and split the columns).  Softmax statistics, exp2, P -> bf16 -> tensor memory,
-//             Z accumulation in fp32 registers, soft-threshold, output.
-//   warp 8  : allocates tensor memory; one elected thread issues every TMA copy and every tcgen05.mma.
+// CTA = 12 warps in three warpgroups (registers are re-divided between them with setmaxnreg: the two
+// compute warpgroups hold a whole row of alpha per thread, the control warps need very few):
+//   warps 0-3 : tile A, one thread per query row (TMEM lane = row).  Softmax reference and sum, exp2,
+//               P -> bf16 -> tensor memory, soft-threshold, output.  The whole row of alpha is in registers.
+//   warps 4-7 : tile B, the same.
+//   warp 8    : allocates tensor memory; one elected thread issues every tcgen05.mma.
+//   warp 9    : one elected thread issues every TMA copy.
+//   warps 10-11: idle (they only complete the control warpgroup).
 //
-// Attention phase, per chunk j of 64 measurements:
+// Attention phase, per tile and per chunk j of 64 measurements:
 //   S_j = Q K~_j^T            (SS MMA, accumulator S[j&1] in tensor memory)
-//   threads read S_j, update the running row maximum, write P_j = exp2(S_j - max) as packed bf16 over the
-//   first half of S[j&1]'s columns
-//   Zc_j = P_j V~_j           (TS MMA: A operand from tensor memory, fresh accumulator)
-//   threads fold it in: z = z * corr_j + Zc_j.
-// MMAs of one CTA execute in issue order (S_0, S_1, PV_0, S_2, PV_1, ...), so S_{j+2} overwrites S[j&1] only
-// after PV_j has read P_j from it.
+//   the row's thread reads S_j and writes P_j = exp2(S_j - ref) as packed bf16 over the first half of
+//   S[j&1]'s columns
+//   Zacc += P_j V~_j          (TS MMA: A operand from tensor memory, one accumulator for all chunks)
+// ref is the row's reference maximum.  It only has to keep exp2 in range, so it is raised (and the row of
+// Zacc and the running sum rescaled by exp2(old - new)) only when a chunk's maximum exceeds it by more than
+// 8, i.e. when some P would exceed 2^8; the final division by the row sum cancels ref exactly.
+// All MMAs of the CTA execute in issue order, so S_{j+2} overwrites S[j&1] only after P_j V~_j has read P_j.
 //
-// Recovery phase.  The accumulator holds r_t = c - a^_t (mu G), where c = z B and a^_t is the sum of the bf16
-// increments fed to the tensor cores so far:
-//   r_0 = z_bf16 B (one MMA);  alpha^{t+1} = eta_theta(alpha^t + r_t);
-//   r_{t+1} = r_t + bf16(alpha^t - alpha^{t+1}) (mu G)     (one accumulating MMA per iteration).
+// Recovery phase, per tile.  The accumulator holds r_t = theta + c - a^_t (mu G), where c = z B and a^_t is
+// the sum of the bf16 increments fed to the tensor cores so far; the registers hold b_t = alpha^t - theta:
+//   r_0 = theta + z_bf16 B (threads store theta, one accumulating MMA);
+//   x = b_t + r_t = alpha^t S + z B;   b_{t+1} = eta_theta(x) - theta = x - 2 theta sat(x / (2 theta) + 1/2);
+//   r_{t+1} = r_t + bf16(b_t - b_{t+1}) (mu G)             (one accumulating MMA per iteration).
 // This is the paper's S alpha + B z with S = I - mu G: the identity part stays exact in fp32 registers, only
-// the increment that multiplies mu G is rounded to bf16, and c never needs registers of its own.
+// the increment that multiplies mu G is rounded to bf16, and c never needs registers of its own.  The
+// saturating form of the shrinkage runs on the FMA pipe (two-element packed instructions where they exist);
+// it leaves O(1e-7 theta) instead of exact zeros, so the last iteration uses the exact min/max form.
 #include "csat_internal.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -37,43 +45,46 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kRows = 128;            // queries per CTA
+constexpr int kRows = 128;            // queries per tile
+constexpr int kTiles = 2;             // tiles per CTA
 constexpr int kMC = 64;               // measurements per chunk
-constexpr int kComputeThreads = 256;
-constexpr int kThreads = 288;
-constexpr int kMaxStages = 4;
+constexpr int kTileThreads = 128;
+constexpr int kThreads = 384;          // three warpgroups: tile A, tile B, control
+constexpr int kMmaWarp = 8, kTmaWarp = 9;
+constexpr int kMaxStages = 6;
 
 template <int D> struct Cfg {
   static constexpr int kDBoxes = D / 64;                          // 64-column boxes across the head dimension
-  static constexpr int kStages = (D == 64) ? 4 : 2;               // K~ / V~ chunks in flight
-  static constexpr uint32_t kQBytes = kDBoxes * kRows * 128;      // Q tile; later the matrix B
+  static constexpr int kStages = (D == 64) ? 6 : 4;               // K~ / V~ chunks in flight
+  static constexpr uint32_t kQBytes = kDBoxes * kRows * 128;      // one Q tile; tile A's buffer later holds B
   static constexpr uint32_t kBoxBytes = kMC * 128;                // one 64-column box of a K~ or V~ chunk
   static constexpr uint32_t kSlotBytes = kDBoxes * kBoxBytes;     // K~ chunk (= V~ chunk)
   static constexpr uint32_t kMatBoxBytes = D * 128;               // one 64-column box of a d x d bf16 matrix
   static constexpr uint32_t kMatBytes = kDBoxes * kMatBoxBytes;
-  static constexpr uint32_t kOffQ = 0;
-  static constexpr uint32_t kOffRing = kOffQ + kQBytes;           // [stage][K~ slot | V~ slot]
+  static constexpr uint32_t kOffQ = 0;                            // [tile]
+  static constexpr uint32_t kOffRing = kOffQ + kTiles * kQBytes;  // [stage][K~ slot | V~ slot]
   static constexpr uint32_t kOffBar = kOffRing + kStages * 2 * kSlotBytes;
-  static constexpr uint32_t kBarBytes = 256 + 2048;               // barriers | row-maximum exchange
+  static constexpr uint32_t kBarBytes = 512;
   static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes;     // base must be 1024-byte aligned (checked)
-  // TMEM columns: S[0] | S[1] | accumulator (Zc, then r_t).  P_j overlays S[j&1]; the recovery operand S[0].
-  static constexpr uint32_t kColS = 0, kColAcc = 2 * kMC, kTmemCols = 256;
+  // TMEM columns per tile (tile t starts at column 256 t): S[0] | S[1] | accumulator (Zacc, then r_t).
+  // P_j overlays S[j&1]; the recovery operand overlays S[0].
+  static constexpr uint32_t kTileCols = 256, kColS = 0, kColAcc = 2 * kMC, kTmemCols = 512;
   static_assert(2 * kMC + D <= 256, "TMEM budget");
   static_assert(D / 2 <= 2 * kMC, "recovery operand fits in the S columns");
   static_assert(kStages >= kDBoxes && kStages <= kMaxStages, "mu G and Psi are staged box by box in ring slots");
   static_assert(kMatBoxBytes <= kSlotBytes && kMatBytes <= kQBytes, "decoder matrices fit where they are staged");
-  static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two CTAs per SM");
+  static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 };
 
 struct Bars {
-  uint64_t q_full, mats_full, psi_full;
+  uint64_t q_full[kTiles], mats_full, psi_full;
   uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
-  uint64_t s_full[2], p_full[2], zc_full, zc_empty;
-  uint64_t a_full, r_full;
+  uint64_t s_full[kTiles][2], p_full[kTiles][2], zc_full[kTiles];
+  uint64_t a_full[kTiles], r_full[kTiles];
   uint32_t tmem_slot;
   int abort;
 };
-static_assert(sizeof(Bars) <= 256, "barrier block");
+static_assert(sizeof(Bars) <= 512, "barrier block");
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -84,8 +95,54 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&p);
 }
-// warps q and q+4 (the two halves of the same 32 rows) meet here
-__device__ __forceinline__ void pair_barrier(int q) { asm volatile("bar.sync %0, 64;" ::"r"(q + 1) : "memory"); }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {   // clamps the result to [0, 1]
+  float y;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
+// two-element packed fp32 arithmetic (one instruction for both halves of a 64-bit register pair)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
+// warpgroup-wide change of the per-thread register allowance (every warp of the warpgroup executes it)
+template <int N> __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // A wait that never blocks for more than the time-out and turns into a no-op once anything gave up.
 struct Waiter {
@@ -99,24 +156,23 @@ struct Waiter {
 };
 
 template <int D>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int nq, int m, int H, int T, int has_psi,
                             float scale_log2, int* status) {
   using C = Cfg<D>;
-  constexpr int HC = D / 2;                    // feature columns per thread
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
     if (threadIdx.x == 0) atomicCAS(status, 0, 200);
     return;
   }
-  uint8_t* q_buf = smem + C::kOffQ;
+  uint8_t* q_buf = smem + C::kOffQ;             // [tile]
   uint8_t* ring = smem + C::kOffRing;
   Bars* bars = reinterpret_cast<Bars*>(smem + C::kOffBar);
-  float* xch = reinterpret_cast<float*>(smem + C::kOffBar + 256);   // [2 buffers][2 halves][128 rows] floats
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int qtile = blockIdx.x, bh = blockIdx.y, h = bh % H;
+  const int row0 = blockIdx.x * (kTiles * kRows), bh = blockIdx.y, h = bh % H;
+  const int ntiles = (nq - row0 > kRows) ? 2 : 1;               // the last CTA of a (batch, head) may hold one tile
   const int nchunks = (m + kMC - 1) / kMC;
   Waiter w{status, &bars->abort};
   auto k_slot = [&](int s) { return ring + (2 * s) * C::kSlotBytes; };
@@ -126,22 +182,23 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     prefetch_tmap(&tmap_q);
     prefetch_tmap(&tmap_kv);
     prefetch_tmap(&tmap_mats);
-    mbar_init(&bars->q_full, 1);
     mbar_init(&bars->mats_full, 1);
     mbar_init(&bars->psi_full, 1);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1);
       mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
     }
-    for (int s = 0; s < 2; ++s) { mbar_init(&bars->s_full[s], 1); mbar_init(&bars->p_full[s], kComputeThreads); }
-    mbar_init(&bars->zc_full, 1);
-    mbar_init(&bars->zc_empty, kComputeThreads);
-    mbar_init(&bars->a_full, kComputeThreads);
-    mbar_init(&bars->r_full, 1);
+    for (int t = 0; t < kTiles; ++t) {
+      mbar_init(&bars->q_full[t], 1);
+      for (int s = 0; s < 2; ++s) { mbar_init(&bars->s_full[t][s], 1); mbar_init(&bars->p_full[t][s], kTileThreads); }
+      mbar_init(&bars->zc_full[t], 1);
+      mbar_init(&bars->a_full[t], kTileThreads);
+      mbar_init(&bars->r_full[t], 1);
+    }
     bars->abort = 0;
     fence_mbar_init();
   }
-  if (warp == 8) {
+  if (warp == kMmaWarp) {
     tmem_alloc(&bars->tmem_slot, C::kTmemCols);
     tmem_relinquish();
   }
@@ -150,133 +207,49 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   tc_fence_after();
   const uint32_t tmem = bars->tmem_slot;
 
-  if (warp == 8) {
-    // ------------------------------------ TMA copies and MMA issue (one thread) -----------------------------------
+  // 2 x 128 x 224 + 128 x 56 = 64512 registers; each branch below starts with its own setmaxnreg
+  if (warp >= kMmaWarp) {
+  reg_dealloc<56>();
+  if (warp == kTmaWarp) {
+    // ------------------------------------------------ TMA producer ------------------------------------------------
     if (elect_one()) {
-      constexpr uint32_t idesc_s = make_idesc_bf16(kRows, kMC, false, false);   // S  = Q  K~^T : both K-major
-      constexpr uint32_t idesc_z = make_idesc_bf16(kRows, D, false, true);      // Zc = P  V~   : V~ is MN-major
-      constexpr uint32_t idesc_r = make_idesc_bf16(kRows, D, false, false);     // r  = a  W^T  : both K-major
-      int next_k = 0, next_v = 0;           // next chunk whose K~ / V~ copy has not been issued
-      int seen_k = 0, seen_v = 0;           // chunks whose copy this thread has waited for
-      bool q_issued = false, mats_issued = false, psi_issued = false, mats_seen = false, psi_seen = false;
-
-      auto issue_k = [&](int c) {
-        const int s = c % C::kStages;
+      int issued_k = 0, issued_v = 0;
+      bool mats_issued = false, psi_issued = false;
+      for (int t = 0; t < ntiles; ++t) {
+        mbar_arrive_expect_tx(&bars->q_full[t], C::kQBytes);
+        for (int g = 0; g < C::kDBoxes; ++g)
+          tma_load_3d(q_buf + t * C::kQBytes + g * kRows * 128, &tmap_q, &bars->q_full[t], g * 64, row0 + t * kRows, bh);
+      }
+      for (int j = 0; j < nchunks; ++j) {
+        const int s = j % C::kStages, use = j / C::kStages;
+        if (use > 0) w.wait(&bars->k_empty[s], (use - 1) & 1, 201);
+        if (w.dead) break;
         mbar_arrive_expect_tx(&bars->k_full[s], C::kSlotBytes);
         for (int g = 0; g < C::kDBoxes; ++g)
-          tma_load_3d(k_slot(s) + g * C::kBoxBytes, &tmap_kv, &bars->k_full[s], g * 64, c * kMC, bh);
-      };
-      auto issue_v = [&](int c) {
-        const int s = c % C::kStages;
+          tma_load_3d(k_slot(s) + g * C::kBoxBytes, &tmap_kv, &bars->k_full[s], g * 64, j * kMC, bh);
+        issued_k = j + 1;
+        if (use > 0) w.wait(&bars->v_empty[s], (use - 1) & 1, 202);
+        if (w.dead) break;
         mbar_arrive_expect_tx(&bars->v_full[s], C::kSlotBytes);
         for (int g = 0; g < C::kDBoxes; ++g)
-          tma_load_3d(v_slot(s) + g * C::kBoxBytes, &tmap_kv, &bars->v_full[s], D + g * 64, c * kMC, bh);
-      };
-      // issues every copy whose slot is free right now; never blocks
-      auto service = [&]() {
-        while (next_k < nchunks) {
-          const int s = next_k % C::kStages, use = next_k / C::kStages;
-          if (use > 0 && !mbar_try_wait(&bars->k_empty[s], (use - 1) & 1)) break;
-          issue_k(next_k++);
-        }
-        while (next_v < nchunks) {
-          const int s = next_v % C::kStages, use = next_v / C::kStages;
-          if (use > 0 && !mbar_try_wait(&bars->v_empty[s], (use - 1) & 1)) break;
-          issue_v(next_v++);
-        }
-      };
-      // bounded wait that keeps the copies flowing while it spins
-      auto wait_serving = [&](uint64_t* bar, uint32_t parity, int code) {
-        if (w.dead) return;
-        if (mbar_try_wait(bar, parity)) return;
-        const unsigned long long t0 = globaltimer();
-        uint32_t spins = 0;
-        while (!mbar_try_wait(bar, parity)) {
-          service();
-          if ((++spins & 0xff) == 0) {
-            if (*(volatile int*)&bars->abort != 0) { w.dead = true; return; }
-            if (globaltimer() - t0 > kWaitTimeoutNs) {
-              *(volatile int*)&bars->abort = 1;
-              atomicCAS(status, 0, code);
-              w.dead = true;
-              return;
-            }
-          }
-        }
-      };
-      // the copies of chunk c must have been issued before their barrier is waited for
-      auto ensure_k = [&](int c) {
-        while (next_k <= c && !w.dead) {
-          const int s = next_k % C::kStages, use = next_k / C::kStages;
-          if (use > 0) w.wait(&bars->k_empty[s], (use - 1) & 1, 201);
-          if (!w.dead) issue_k(next_k++);
-        }
-      };
-      auto ensure_v = [&](int c) {
-        while (next_v <= c && !w.dead) {
-          const int s = next_v % C::kStages, use = next_v / C::kStages;
-          if (use > 0) w.wait(&bars->v_empty[s], (use - 1) & 1, 202);
-          if (!w.dead) issue_v(next_v++);
-        }
-      };
-      auto issue_pv = [&](int i) {
-        const int s = i % C::kStages, b = i & 1;
-        ensure_v(i);
-        wait_serving(&bars->v_full[s], (i / C::kStages) & 1, 211);
-        if (!w.dead) seen_v = i + 1;
-        wait_serving(&bars->p_full[b], (i >> 1) & 1, 212);
-        if (i > 0) wait_serving(&bars->zc_empty, (i - 1) & 1, 213);   // Zc_{i-1} has been folded
-        tc_fence_after();
-        const uint64_t b_desc = make_smem_desc(smem_u32(v_slot(s)), C::kBoxBytes, 1024);
-#pragma unroll
-        for (int k = 0; k < kMC / 16; ++k)     // P: 8 packed columns per 16 measurements; V~: +16 rows = 2048 B
-          mma_f16_ts(tmem + C::kColAcc, tmem + C::kColS + b * kMC + k * 8, b_desc + (uint64_t)(k * 128), idesc_z, k != 0);
-        mma_commit(&bars->zc_full);
-        mma_commit(&bars->v_empty[s]);
-      };
-
-      mbar_arrive_expect_tx(&bars->q_full, C::kQBytes);
-      for (int g = 0; g < C::kDBoxes; ++g)
-        tma_load_3d(q_buf + g * kRows * 128, &tmap_q, &bars->q_full, g * 64, qtile * kRows, bh);
-      q_issued = true;
-      service();
-      w.wait(&bars->q_full, 0, 210);
-      for (int j = 0; j < nchunks; ++j) {
-        const int s = j % C::kStages, b = j & 1;
-        ensure_k(j);
-        wait_serving(&bars->k_full[s], (j / C::kStages) & 1, 214);
-        if (!w.dead) seen_k = j + 1;
-        tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) {
-          const uint64_t a_desc = make_smem_desc(smem_u32(q_buf + (k / 4) * kRows * 128), 16, 1024) + (uint64_t)((k % 4) * 2);
-          const uint64_t b_desc = make_smem_desc(smem_u32(k_slot(s) + (k / 4) * C::kBoxBytes), 16, 1024) + (uint64_t)((k % 4) * 2);
-          mma_f16_ss(tmem + C::kColS + b * kMC, a_desc, b_desc, idesc_s, k != 0);
-        }
-        mma_commit(&bars->s_full[b]);
-        mma_commit(&bars->k_empty[s]);
-        if (j > 0) issue_pv(j - 1);
-        service();
+          tma_load_3d(v_slot(s) + g * C::kBoxBytes, &tmap_kv, &bars->v_full[s], D + g * 64, j * kMC, bh);
+        issued_v = j + 1;
       }
       if (T > 0) {
-        // every S MMA has finished once the last one has: Q and the K~ slots are free for mu G and B
+        // every S MMA has finished once the last one has: tile A's Q buffer and the K~ slots are free for B, mu G
         const int last = nchunks - 1;
-        wait_serving(&bars->k_empty[last % C::kStages], (last / C::kStages) & 1, 215);
+        w.wait(&bars->k_empty[last % C::kStages], (last / C::kStages) & 1, 203);
         if (!w.dead) {
           mbar_arrive_expect_tx(&bars->mats_full, 2 * C::kMatBytes);
           for (int g = 0; g < C::kDBoxes; ++g) {
-            tma_load_3d(k_slot(g), &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 0);                          // mu G
-            tma_load_3d(q_buf + g * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 1);       // B
+            tma_load_3d(k_slot(g), &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 0);                      // mu G
+            tma_load_3d(q_buf + g * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 1);   // B
           }
           mats_issued = true;
         }
-      }
-      issue_pv(nchunks - 1);
-      if (T > 0) {
         if (has_psi) {
           // Psi goes to the V~ slots once the last P V~ product has read them
-          const int last = nchunks - 1;
-          w.wait(&bars->v_empty[last % C::kStages], (last / C::kStages) & 1, 216);
+          w.wait(&bars->v_empty[last % C::kStages], (last / C::kStages) & 1, 204);
           if (!w.dead) {
             mbar_arrive_expect_tx(&bars->psi_full, C::kMatBytes);
             for (int g = 0; g < C::kDBoxes; ++g)
@@ -284,194 +257,326 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             psi_issued = true;
           }
         }
-        const int n_mma = T + (has_psi ? 1 : 0);            // r_0 = z B, then T-1 increments with mu G, then Psi
-        for (int i = 0; i < n_mma; ++i) {
-          const bool first = (i == 0), psi_step = has_psi && i == n_mma - 1;
-          if (first) { w.wait(&bars->mats_full, 0, 217); if (!w.dead) mats_seen = true; }
-          if (psi_step) { w.wait(&bars->psi_full, 0, 218); if (!w.dead) psi_seen = true; }
-          w.wait(&bars->a_full, i & 1, 219);
-          tc_fence_after();
-#pragma unroll
-          for (int k = 0; k < D / 16; ++k) {
-            const uint8_t* box = first ? q_buf + (k / 4) * C::kMatBoxBytes : (psi_step ? v_slot(k / 4) : k_slot(k / 4));
-            const uint64_t b_desc = make_smem_desc(smem_u32(box), 16, 1024) + (uint64_t)((k % 4) * 2);
-            mma_f16_ts(tmem + C::kColAcc, tmem + C::kColS + k * 8, b_desc, idesc_r, (first || psi_step) ? (k != 0) : 1u);
-          }
-          mma_commit(&bars->r_full);
-        }
       }
       if (w.dead) {
         // gave up: let the copies that are still in flight land before the CTA's shared memory goes away
-        if (q_issued) mbar_wait_drain(&bars->q_full, 0);
-        for (int c = seen_k; c < next_k; ++c) mbar_wait_drain(&bars->k_full[c % C::kStages], (c / C::kStages) & 1);
-        for (int c = seen_v; c < next_v; ++c) mbar_wait_drain(&bars->v_full[c % C::kStages], (c / C::kStages) & 1);
-        if (mats_issued && !mats_seen) mbar_wait_drain(&bars->mats_full, 0);
-        if (psi_issued && !psi_seen) mbar_wait_drain(&bars->psi_full, 0);
+        for (int t = 0; t < ntiles; ++t) mbar_wait_drain(&bars->q_full[t], 0);
+        for (int c = issued_k > C::kStages ? issued_k - C::kStages : 0; c < issued_k; ++c)
+          mbar_wait_drain(&bars->k_full[c % C::kStages], (c / C::kStages) & 1);
+        for (int c = issued_v > C::kStages ? issued_v - C::kStages : 0; c < issued_v; ++c)
+          mbar_wait_drain(&bars->v_full[c % C::kStages], (c / C::kStages) & 1);
+        if (mats_issued) mbar_wait_drain(&bars->mats_full, 0);
+        if (psi_issued) mbar_wait_drain(&bars->psi_full, 0);
       }
     }
-  } else {
-    // ------------------------------------------------ compute threads ---------------------------------------------
-    const int q = warp & 3, half = warp >> 2;
-    const int row = q * 32 + lane;                              // row of the tile = TMEM lane
-    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    float z[HC];
+  } else if (warp == kMmaWarp) {
+    // ------------------------------------------------ MMA issuer --------------------------------------------------
+    // One thread issues every MMA of both tiles, so the issue path is kept short: descriptors of buffers that
+    // do not move are built once, the others differ from a base by compile-time constants.
+    if (elect_one()) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(kRows, kMC, false, false);   // S  = Q  K~^T : both K-major
+      constexpr uint32_t idesc_z = make_idesc_bf16(kRows, D, false, true);      // Z += P  V~   : V~ is MN-major
+      constexpr uint32_t idesc_r = make_idesc_bf16(kRows, D, false, false);     // r += a  W^T  : both K-major
+      // K-major operand: K step k (16 columns) lies in 64-column box k / 4, 32 (k % 4) bytes into each row
+      auto kstep = [](int k, uint32_t box_bytes) { return (uint64_t)((k / 4) * (box_bytes >> 4) + (k % 4) * 2); };
+      const uint64_t q_desc0 = make_smem_desc(smem_u32(q_buf), 16, 1024);
+      const uint64_t ring_k0 = make_smem_desc(smem_u32(ring), 16, 1024);
+      const uint64_t ring_v0 = make_smem_desc(smem_u32(ring + C::kSlotBytes), C::kBoxBytes, 1024);
+      constexpr uint64_t kStageStep = (2 * C::kSlotBytes) >> 4;                 // descriptor distance between stages
+      auto issue_pv = [&](int i) {
+        const int s = i % C::kStages, b = i & 1;
+        w.wait(&bars->v_full[s], (i / C::kStages) & 1, 211);
+        const uint64_t b_desc = ring_v0 + (uint64_t)s * kStageStep;
+        const uint32_t acc = (i != 0);
 #pragma unroll
-    for (int i = 0; i < HC; ++i) z[i] = 0.f;
-    float run_max = -INFINITY, run_sum = 0.f, corr_prev = 0.f;
-
-    auto fold_zc = [&](int i, float corr) {
-      w.wait(&bars->zc_full, i & 1, 221);
-      tc_fence_after();
+        for (int t = 0; t < kTiles; ++t) {
+          if (t < ntiles) {
+            w.wait(&bars->p_full[t][b], (i >> 1) & 1, 212);
+            tc_fence_after();
+            const uint32_t tb = tmem + t * C::kTileCols;
+            // P: 8 packed columns per 16 measurements; V~: +16 rows = 2048 B
+            mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC, b_desc, idesc_z, acc);
 #pragma unroll
-      for (int c0 = 0; c0 < HC; c0 += 16) {
-        uint32_t r[16];
-        tmem_ld_32x32b_x16(tmem + lane_addr + C::kColAcc + half * HC + c0, r);
-        tmem_wait_ld();
+            for (int k = 1; k < kMC / 16; ++k)
+              mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC + k * 8, b_desc + (uint64_t)(k * 128), idesc_z, 1u);
+            mma_commit(&bars->zc_full[t]);
+          }
+        }
+        mma_commit(&bars->v_empty[s]);
+      };
 #pragma unroll
-        for (int e = 0; e < 16; ++e) z[c0 + e] = fmaf(z[c0 + e], corr, __uint_as_float(r[e]));
+      for (int t = 0; t < kTiles; ++t)
+        if (t < ntiles) w.wait(&bars->q_full[t], 0, 210);
+      for (int j = 0; j < nchunks; ++j) {
+        const int s = j % C::kStages, b = j & 1;
+        w.wait(&bars->k_full[s], (j / C::kStages) & 1, 213);
+        tc_fence_after();
+        const uint64_t kd = ring_k0 + (uint64_t)s * kStageStep;
+#pragma unroll
+        for (int t = 0; t < kTiles; ++t) {
+          if (t < ntiles) {
+            const uint64_t qd = q_desc0 + (uint64_t)(t * (C::kQBytes >> 4));
+            const uint32_t ds = tmem + t * C::kTileCols + C::kColS + b * kMC;
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k)
+              mma_f16_ss(ds, qd + kstep(k, kRows * 128), kd + kstep(k, C::kBoxBytes), idesc_s, k != 0);
+            mma_commit(&bars->s_full[t][b]);
+          }
+        }
+        mma_commit(&bars->k_empty[s]);
+        if (j > 0) issue_pv(j - 1);
       }
-      tc_fence_before();
-      mbar_arrive(&bars->zc_empty);
-    };
-
-    for (int j = 0; j < nchunks; ++j) {
-      const int b = j & 1;
-      w.wait(&bars->s_full[b], (j >> 1) & 1, 220);
-      tc_fence_after();
-      uint32_t r[32];
-      tmem_ld_32x32b_x32(tmem + lane_addr + C::kColS + b * kMC + half * 32, r);
-      tmem_wait_ld();
-      // scores in the log2 domain; measurements beyond m are masked out
-      float mx = -INFINITY;
-      const int col0 = j * kMC + half * 32;
-      if (col0 + 32 <= m) {
+      issue_pv(nchunks - 1);
+      if (T > 0) {
+        const int n_mma = T + (has_psi ? 1 : 0);    // r_0 = theta + z B, then T-1 increments with mu G, then Psi
+        for (int i = 0; i < n_mma; ++i) {
+          const bool first = (i == 0), psi_step = has_psi && i == n_mma - 1;
+          if (first) w.wait(&bars->mats_full, 0, 214);
+          if (psi_step) w.wait(&bars->psi_full, 0, 215);
+          // B sits in tile A's Q buffer (boxes of d rows), mu G in the K~ slots and Psi in the V~ slots of the
+          // first stages (one box per stage)
+          const uint64_t w0 = first ? q_desc0 : (psi_step ? ring_k0 + (uint64_t)(C::kSlotBytes >> 4) : ring_k0);
+          const uint64_t wbox = first ? (uint64_t)(C::kMatBoxBytes >> 4) : kStageStep;
+          const uint32_t acc0 = psi_step ? 0u : 1u;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, __uint_as_float(r[e]));
-      } else {
+          for (int t = 0; t < kTiles; ++t) {
+            if (t < ntiles) {
+              w.wait(&bars->a_full[t], i & 1, 216);
+              tc_fence_after();
+              const uint32_t tb = tmem + t * C::kTileCols;
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          if (col0 + e >= m) r[e] = 0xff800000u;                // -inf
-          mx = fmaxf(mx, __uint_as_float(r[e]));
+              for (int k = 0; k < D / 16; ++k)
+                mma_f16_ts(tb + C::kColAcc, tb + C::kColS + k * 8, w0 + (uint64_t)(k / 4) * wbox + (uint64_t)((k % 4) * 2),
+                           idesc_r, k == 0 ? acc0 : 1u);
+              mma_commit(&bars->r_full[t]);
+            }
+          }
         }
       }
-      mx *= scale_log2;                                         // scale > 0: the maximum commutes with it
-      float* slot = xch + b * 256;
-      slot[half * 128 + row] = mx;
-      pair_barrier(q);              // also orders this thread's S read before its partner's P write below
-      mx = fmaxf(mx, slot[(half ^ 1) * 128 + row]);
-      const float new_max = fmaxf(run_max, mx);                 // finite: chunk 0 has a valid measurement
-      const float corr = ex2(run_max - new_max);
-      run_max = new_max;
-      float sum = 0.f;
-      uint32_t pk[16];
-#pragma unroll
-      for (int e = 0; e < 32; e += 2) {
-        const float p0 = ex2(fmaf(__uint_as_float(r[e]), scale_log2, -new_max));
-        const float p1 = ex2(fmaf(__uint_as_float(r[e + 1]), scale_log2, -new_max));
-        sum += p0 + p1;
-        pk[e >> 1] = pack_bf16(p0, p1);
-      }
-      run_sum = fmaf(run_sum, corr, sum);
-      // P_j over the first 32 columns of S[b]: this half's 32 measurements are packed columns [16 half, +16)
-      tmem_st_32x32b_x16(tmem + lane_addr + C::kColS + b * kMC + half * 16, pk);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&bars->p_full[b]);
-      if (j > 0) fold_zc(j - 1, corr_prev);
-      corr_prev = corr;
     }
-    fold_zc(nchunks - 1, corr_prev);
-    // the two halves of a row share max and corr; their partial sums are added once
-    float* slot = xch + (nchunks & 1) * 256;   // the buffer the last chunk did not use
-    slot[half * 128 + row] = run_sum;
-    pair_barrier(q);
-    const float inv = 1.f / (run_sum + slot[(half ^ 1) * 128 + row]);
-#pragma unroll
-    for (int i = 0; i < HC; ++i) z[i] *= inv;
+  }
+  } else {
+    reg_alloc<224>();
+    // ------------------------------------------------ compute threads ---------------------------------------------
+    const int t = warp >> 2, wq = warp & 3;                     // tile, lane quarter
+    if (t < ntiles) {
+      const int row = wq * 32 + lane;                           // row of the tile = TMEM lane
+      const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + t * C::kTileCols;
+      const uint32_t acc_addr = tbase + C::kColAcc;
+      float ref = -INFINITY;                                    // reference maximum of the row (log2 domain)
+      uint64_t sum2 = pack2(0.f, 0.f);                          // running sum of P, two partial sums
+      const uint64_t sc2 = pack2(scale_log2, scale_log2);
+      int zc_seen = 0;                                          // phases of zc_full[t] this thread has waited for
 
-    if (T > 0) {
-      const float th = theta[h];
-      const uint32_t op_addr = tmem + lane_addr + C::kColS + half * (HC / 2);   // this thread's operand columns
-      // z as the bf16 A operand of r_0 = z B
-#pragma unroll
-      for (int c0 = 0; c0 < HC; c0 += 32) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int e = 0; e < 32; e += 2) pk[e >> 1] = pack_bf16(z[c0 + e], z[c0 + e + 1]);
-        tmem_st_32x32b_x16(op_addr + c0 / 2, pk);
-      }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(&bars->a_full);
-#pragma unroll
-      for (int i = 0; i < HC; ++i) z[i] = 0.f;                  // z now holds alpha (alpha^0 = 0)
-      int phase = 0;
-      for (int it = 0; it < T; ++it) {
-        w.wait(&bars->r_full, phase & 1, 230); ++phase;
+      for (int j = 0; j < nchunks; ++j) {
+        const int b = j & 1;
+        w.wait(&bars->s_full[t][b], (j >> 1) & 1, 220);
         tc_fence_after();
-        const bool more = it + 1 < T;
+        uint32_t ra[32], rb[32];                                // columns [0, 32) and [32, 64) of S_j
+        tmem_ld_32x32b_x32(tbase + C::kColS + b * kMC, ra);
+        tmem_ld_32x32b_x32(tbase + C::kColS + b * kMC + 32, rb);
+        tmem_wait_ld();
+        // scores in the log2 domain; measurements beyond m are masked out
+        float mx = -INFINITY;
+        if ((j + 1) * kMC <= m) {
+          float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;   // independent chains
 #pragma unroll
-        for (int c0 = 0; c0 < HC; c0 += 16) {
-          uint32_t r[16];
-          tmem_ld_32x32b_x16(tmem + lane_addr + C::kColAcc + half * HC + c0, r);
+          for (int e = 0; e < 32; e += 4) {
+            m0 = max3(m0, __uint_as_float(ra[e]), __uint_as_float(ra[e + 1]));
+            m1 = max3(m1, __uint_as_float(ra[e + 2]), __uint_as_float(ra[e + 3]));
+            m2 = max3(m2, __uint_as_float(rb[e]), __uint_as_float(rb[e + 1]));
+            m3 = max3(m3, __uint_as_float(rb[e + 2]), __uint_as_float(rb[e + 3]));
+          }
+          mx = fmaxf(max3(m0, m1, m2), m3);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            if (j * kMC + e >= m) ra[e] = 0xff800000u;          // -inf
+            if (j * kMC + 32 + e >= m) rb[e] = 0xff800000u;
+            mx = max3(mx, __uint_as_float(ra[e]), __uint_as_float(rb[e]));
+          }
+        }
+        mx *= scale_log2;           // scale > 0: the maximum commutes with it; finite: the chunk has a valid column
+        if (j == 0) {
+          ref = mx;
+        } else {
+          const bool raise = mx > ref + 8.f;
+          if (__any_sync(0xffffffffu, raise)) {
+            // rare: rescale this warp's rows of the accumulator (factor 1 for rows that keep their reference)
+            w.wait(&bars->zc_full[t], (j - 1) & 1, 221);        // P_{j-1} V~_{j-1} has been added
+            zc_seen = j;
+            tc_fence_after();
+            const float f = raise ? ex2(ref - mx) : 1.f;
+            if (raise) ref = mx;
+            sum2 = mul2(sum2, pack2(f, f));
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 16) {
+              uint32_t a[16];
+              tmem_ld_32x32b_x16(acc_addr + c0, a);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 16; ++e) a[e] = __float_as_uint(__uint_as_float(a[e]) * f);
+              tmem_st_32x32b_x16(acc_addr + c0, a);
+            }
+          }
+        }
+        const uint64_t nref2 = pack2(-ref, -ref);
+        // P_j over the first 32 columns of S[b] (two bf16 per column)
+        auto exp_half = [&](const uint32_t (&r)[32], uint32_t col) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            float t0, t1;
+            unpack2(fma2(pack2u(r[e], r[e + 1]), sc2, nref2), t0, t1);
+            const float p0 = ex2(t0), p1 = ex2(t1);
+            sum2 = add2(sum2, pack2(p0, p1));
+            pk[e >> 1] = pack_bf16(p0, p1);
+          }
+          tmem_st_32x32b_x16(tbase + C::kColS + b * kMC + col, pk);
+        };
+        exp_half(ra, 0);
+        exp_half(rb, 16);
+        tmem_wait_st();                                         // also covers a rescale's stores
+        tc_fence_before();
+        // A parity wait is only safe when the waiter is at most one phase behind, so every phase of zc_full is
+        // observed in order: phase j-1 here (it cannot be two ahead, since P_j V~_j needs the arrival below;
+        // normally it completed long ago), phase j after the next chunk, the last one after the loop.
+        if (j > 0 && zc_seen < j) {
+          w.wait(&bars->zc_full[t], (j - 1) & 1, 223);
+          zc_seen = j;
+        }
+        mbar_arrive(&bars->p_full[t][b]);
+      }
+      float inv;
+      {
+        float s0, s1;
+        unpack2(sum2, s0, s1);
+        inv = 1.f / (s0 + s1);
+      }
+      w.wait(&bars->zc_full[t], (nchunks - 1) & 1, 222);        // every P V~ product has been added
+      tc_fence_after();
+      // v2 holds, in turn: Z, b_t = alpha^t - theta, alpha^T, Psi alpha^T  (pairs of adjacent columns)
+      uint64_t v2[D / 2];
+      {
+        const uint64_t inv2 = pack2(inv, inv);
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t a[16];
+          tmem_ld_32x32b_x16(acc_addr + c0, a);
           tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) v2[(c0 + e) >> 1] = mul2(pack2u(a[e], a[e + 1]), inv2);
+        }
+      }
+      auto publish = [&]() {                                    // v2 as the bf16 A operand of the next MMA
+        const uint32_t op_addr = tbase + C::kColS;
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
           uint32_t pk[8];
 #pragma unroll
           for (int e = 0; e < 16; e += 2) {
-            float nd[2];
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const float rv = __uint_as_float(r[e + u]);
-              const float x = z[c0 + e + u] + rv;               // alpha^t S + z B, identity part in fp32
-              const float cl = fminf(fmaxf(x, -th), th);
-              z[c0 + e + u] = x - cl;                           // eta_theta(x)
-              nd[u] = cl - rv;                                  // alpha^t - alpha^{t+1}
-            }
-            pk[e >> 1] = pack_bf16(nd[0], nd[1]);
+            float x0, x1;
+            unpack2(v2[(c0 + e) >> 1], x0, x1);
+            pk[e >> 1] = pack_bf16(x0, x1);
           }
-          if (more) tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
-        }
-        if (more) {
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(&bars->a_full);
-        }
-      }
-      if (has_psi) {
-#pragma unroll
-        for (int c0 = 0; c0 < HC; c0 += 32) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) pk[e >> 1] = pack_bf16(z[c0 + e], z[c0 + e + 1]);
-          tmem_st_32x32b_x16(op_addr + c0 / 2, pk);
+          tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
         }
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(&bars->a_full);
-        w.wait(&bars->r_full, phase & 1, 232); ++phase;
+        mbar_arrive(&bars->a_full[t]);
+      };
+
+      if (T > 0) {
+        const float th = theta[h];
+        const float inv2th = th > 0.f ? 0.5f / th : 0.f;        // theta = 0: sat(1/2) = 1/2 and b' = x
+        const uint64_t m2th2 = pack2(-2.f * th, -2.f * th);
+        const uint32_t op_addr = tbase + C::kColS;
+        // accumulator := theta (r_0 = theta + z B), and z as the bf16 A operand
+        {
+          uint32_t tb[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) tb[e] = __float_as_uint(th);
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) tmem_st_32x32b_x16(acc_addr + c0, tb);
+        }
+        publish();
+#pragma unroll
+        for (int i = 0; i < D / 2; ++i) v2[i] = pack2(-th, -th);        // b = alpha - theta, alpha^0 = 0
+        int phase = 0;
+        for (int it = 0; it + 1 < T; ++it) {
+          w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
+          tc_fence_after();
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(acc_addr + c0, r);
+            tmem_wait_ld();
+            uint32_t pk[16];
+#pragma unroll
+            for (int e = 0; e < 32; e += 2) {
+              const uint64_t bo = v2[(c0 + e) >> 1];
+              const uint64_t x2 = add2(bo, pack2u(r[e], r[e + 1]));          // alpha^t S + z B
+              float x0, x1;
+              unpack2(x2, x0, x1);
+              const uint64_t t2 = pack2(fma_sat(x0, inv2th, 0.5f), fma_sat(x1, inv2th, 0.5f));
+              const uint64_t bn = fma2(t2, m2th2, x2);                       // eta_theta(x) - theta
+              v2[(c0 + e) >> 1] = bn;
+              float d0, d1;
+              unpack2(sub2(bo, bn), d0, d1);                                 // alpha^t - alpha^{t+1}
+              pk[e >> 1] = pack_bf16(d0, d1);
+            }
+            tmem_st_32x32b_x16(op_addr + c0 / 2, pk);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&bars->a_full[t]);
+        }
+        // last iteration, exact shrinkage: alpha^T = eta_theta(x)
+        w.wait(&bars->r_full[t], phase & 1, 231); ++phase;
         tc_fence_after();
 #pragma unroll
-        for (int c0 = 0; c0 < HC; c0 += 32) {
-          uint32_t r[32];
-          tmem_ld_32x32b_x32(tmem + lane_addr + C::kColAcc + half * HC + c0, r);
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(acc_addr + c0, r);
           tmem_wait_ld();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) z[c0 + e] = __uint_as_float(r[e]);
+          for (int e = 0; e < 16; e += 2) {
+            float b0, b1;
+            unpack2(v2[(c0 + e) >> 1], b0, b1);
+            const float x0 = b0 + __uint_as_float(r[e]), x1 = b1 + __uint_as_float(r[e + 1]);
+            v2[(c0 + e) >> 1] = pack2(x0 - fminf(fmaxf(x0, -th), th), x1 - fminf(fmaxf(x1, -th), th));
+          }
+        }
+        if (has_psi) {
+          publish();
+          w.wait(&bars->r_full[t], phase & 1, 232); ++phase;
+          tc_fence_after();
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld_32x32b_x16(acc_addr + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) v2[(c0 + e) >> 1] = pack2u(r[e], r[e + 1]);
+          }
         }
       }
-    }
-    const int grow = qtile * kRows + row;
-    if (grow < nq && !w.dead && *(volatile int*)&bars->abort == 0) {
-      uint4* o = reinterpret_cast<uint4*>(out + ((int64_t)bh * nq + grow) * D + half * HC);
+      const int grow = row0 + t * kRows + row;
+      if (grow < nq && !w.dead && *(volatile int*)&bars->abort == 0) {
+        uint4* o = reinterpret_cast<uint4*>(out + ((int64_t)bh * nq + grow) * D);
 #pragma unroll
-      for (int c = 0; c < HC / 8; ++c)
-        o[c] = make_uint4(pack_bf16(z[c * 8], z[c * 8 + 1]), pack_bf16(z[c * 8 + 2], z[c * 8 + 3]),
-                          pack_bf16(z[c * 8 + 4], z[c * 8 + 5]), pack_bf16(z[c * 8 + 6], z[c * 8 + 7]));
+        for (int c = 0; c < D / 8; ++c) {
+          float x[8];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) unpack2(v2[c * 4 + u], x[2 * u], x[2 * u + 1]);
+          o[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+        }
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 8) tmem_dealloc(tmem, C::kTmemCols);
+  if (warp == kMmaWarp) tmem_dealloc(tmem, C::kTmemCols);
 }
 
 template <int D>
@@ -489,15 +594,12 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
     e = cudaFuncSetAttribute(attend_recover_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)C::kSmemBytes);
     if (e != cudaSuccess) return e;
-    // two CTAs per SM need the large shared-memory carve-out
-    e = cudaFuncSetAttribute(attend_recover_sm100_kernel<D>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                             (int)cudaSharedmemCarveoutMaxShared);
-    if (e != cudaSuccess) return e;
     attr_set = true;
   }
   const double scale = p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)D);
   const float scale_log2 = (float)(scale * 1.4426950408889634);
-  const dim3 grid((unsigned)((p.nq + kRows - 1) / kRows), (unsigned)(p.B * p.H));
+  const int64_t rows_per_cta = kTiles * kRows;
+  const dim3 grid((unsigned)((p.nq + rows_per_cta - 1) / rows_per_cta), (unsigned)(p.B * p.H));
   attend_recover_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(
       tq, c->tmap_kv, c->tmap_mats, (__nv_bfloat16*)out, c->theta, (int)p.nq, (int)p.m, (int)p.H, p.T,
       c->psi ? 1 : 0, scale_log2, c->status);
