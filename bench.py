@@ -80,7 +80,7 @@ class ClockSampler:
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", sel, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", sel, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=self.tmp, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -245,7 +245,7 @@ def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3) -> dict:
 def run_csat(args, w: wl.Workload) -> dict:
     import torch
     import torch.distributed as dist
-    from paper_2507_02957_b200 import binding
+    from paper_2507_02957_b200 import binding, parallel
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -283,11 +283,7 @@ def run_csat(args, w: wl.Workload) -> dict:
     torch.cuda.synchronize()
     barrier()
     clocks = sampler.stop() if sampler else None
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = parallel.max_over_ranks(e0.elapsed_time(e1), device="cuda")
     ms_step = ms_total / K
 
     # per-kernel CUDA-event times recorded inside the timed region
@@ -323,11 +319,7 @@ def run_csat(args, w: wl.Workload) -> dict:
     for _ in range(K):
         ctx.forward_host(host["Q"], host["K"], host["V"], oh)
     torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = parallel.max_over_ranks(time.perf_counter() - t0, device="cuda")
     h2d = sum(host[k].numel() * host[k].element_size() for k in "QKV")
     d2h = oh.numel() * oh.element_size()
     ctx.close()
@@ -375,7 +367,7 @@ def run_csat(args, w: wl.Workload) -> dict:
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c5", help="c1..c5 or c5_sweep_n<N>")
     ap.add_argument("--impl", default="csat", choices=["csat", "reference"])
