@@ -506,14 +506,11 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         for (int it = 0; it + 1 < T; ++it) {
           w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
           tc_fence_after();
+          // 16 columns at a time, the next piece's TMEM load in flight while this one is shrunk
+          auto shrink16 = [&](const uint32_t (&r)[16], int c0) {
+            uint32_t pk[8];
 #pragma unroll
-          for (int c0 = 0; c0 < D; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld_32x32b_x32(acc_addr + c0, r);
-            tmem_wait_ld();
-            uint32_t pk[16];
-#pragma unroll
-            for (int e = 0; e < 32; e += 2) {
+            for (int e = 0; e < 16; e += 2) {
               const uint64_t bo = v2[(c0 + e) >> 1];
               const uint64_t x2 = add2(bo, pack2u(r[e], r[e + 1]));          // alpha^t S + z B
               float x0, x1;
@@ -525,7 +522,18 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
               unpack2(sub2(bo, bn), d0, d1);                                 // alpha^t - alpha^{t+1}
               pk[e >> 1] = pack_bf16(d0, d1);
             }
-            tmem_st_32x32b_x16(op_addr + c0 / 2, pk);
+            tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+          };
+          uint32_t r0[16], r1[16];
+          tmem_ld_32x32b_x16(acc_addr, r0);
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            tmem_wait_ld();
+            tmem_ld_32x32b_x16(acc_addr + c0 + 16, r1);
+            shrink16(r0, c0);
+            tmem_wait_ld();
+            if (c0 + 32 < D) tmem_ld_32x32b_x16(acc_addr + c0 + 32, r0);
+            shrink16(r1, c0 + 16);
           }
           tmem_wait_st();
           tc_fence_before();
