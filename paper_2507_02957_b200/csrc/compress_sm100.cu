@@ -38,7 +38,7 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, __nv_bfloat16* __restrict__ kv, int m, int n, int H,
-                      int* status) {
+                      int B, int* status) {
   using C = Cfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -51,7 +51,9 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
   int* cta_abort = reinterpret_cast<int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int mtile = blockIdx.x, bh = blockIdx.y, h = bh % H;
+  // blockIdx.y walks the batch fastest, so that the CTAs that stream the same tile of Phi_h (one per batch
+  // element) are scheduled together and all but the first find it in L2
+  const int mtile = blockIdx.x, h = blockIdx.y / B, bh = (blockIdx.y % B) * H + h;
   const int nchunks = (n + kChunk - 1) / kChunk;
 
   if (threadIdx.x == 0) {
@@ -169,7 +171,7 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
   }
   const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(p.B * p.H));
   compress_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
-                                                                 (int)p.n, (int)p.H, c->status);
+                                                                 (int)p.n, (int)p.H, (int)p.B, c->status);
   return cudaGetLastError();
 }
 

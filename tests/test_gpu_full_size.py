@@ -1,0 +1,48 @@
+"""GPU parity at the full workload sizes, in the launch configuration bench.py times.
+
+The float64 oracle cannot run a whole workload in seconds, but every (batch, head) pair is independent, so a
+few sampled pairs are checked in full, element by element, against the oracle (same seeded inputs, the
+library's exported Phi), with recovery disabled, at the workload's own (T, lambda) and at lambda = 0 (dense
+output).  Properties that hold at any size cover the rest: no NaN/Inf anywhere, and bit-identical reruns.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import csat_oracle as orc
+from paper_2507_02957_b200 import workloads as wl
+from gpu_util import TOL, device_inputs, make_ctx, rel_err, to_np
+
+pytestmark = pytest.mark.gpu
+
+SAMPLES = {"c2": [(0, 0), (17, 5), (31, 11)], "c3": [(0, 0), (7, 11)], "c4": [(0, 0), (15, 7)], "c5": [(1, 9)]}
+
+
+@pytest.mark.parametrize("key", sorted(SAMPLES))
+def test_sampled_pairs_of_the_full_workload(key):
+    w = wl.CONFIGS[key]
+    inp = wl.make_inputs(w)
+    Q, K, V, Psi = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    if Psi is not None:
+        ctx.set_dictionary(Psi)
+    phi = ctx.get_phi()
+    tol = TOL[w.dtype]
+    psi64 = None if inp["Psi"] is None else inp["Psi"].astype(np.float64)
+    for T, lam in [(0, w.lam), (w.T, w.lam), (w.T, 0.0)]:
+        ctx.set(T=T, lam=lam)
+        out = ctx.forward(Q, K, V)
+        assert torch.isfinite(out).all()
+        if (T, lam) == (w.T, w.lam):
+            assert torch.equal(out, ctx.forward(Q, K, V))          # deterministic at full size
+        for (b, h) in SAMPLES[key]:
+            st = {}
+            ref = orc.csat_forward_head(inp["Q"][b, h], inp["K"][b, h], inp["V"][b, h], to_np(phi[h]), T=T, lam=lam,
+                                        Psi=psi64, stages=st)
+            got = to_np(out[b, h])
+            if np.abs(ref).max() == 0.0:
+                assert np.abs(got).max() <= st["theta"] * tol, (key, b, h, T, lam)
+            else:
+                err = rel_err(got, ref)
+                assert err <= tol, (key, b, h, T, lam, err)
+    ctx.close()
