@@ -52,6 +52,7 @@ constexpr int kTileThreads = 128;
 constexpr int kThreads = 384;          // three warpgroups: tile A, tile B, control
 constexpr int kMmaWarp = 8, kTmaWarp = 9;
 constexpr int kMaxStages = 6;
+constexpr int kPolyEvery = 4;          // every 4th pair of scores takes the polynomial exp2 (measured best of 1, 2, 3, 4, none)
 
 template <int D> struct Cfg {
   static constexpr int kDBoxes = D / 64;                          // 64-column boxes across the head dimension
@@ -138,6 +139,27 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
   uint64_t r;
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
   return r;
+}
+
+// exp2 of both halves on the FMA pipe (the MUFU unit is the bottleneck of the softmax: 4 lanes per clock and
+// sub-core).  x <= ~9; anything below -120 (masked columns are -inf) gives 2^-120.  Round-to-nearest split
+// x = i + f, f in [-1/2, 1/2]; 2^f by a cubic fitted to 7.5e-5 relative error (P is rounded to bf16, 3.9e-3,
+// and the row sum tolerates far more); 2^i by adding i to the exponent field.
+__device__ __forceinline__ void exp2_poly2(uint64_t x2, float& p0, float& p1) {
+  float x0, x1;
+  unpack2(x2, x0, x1);
+  x2 = pack2(fmaxf(x0, -120.f), fmaxf(x1, -120.f));
+  const uint64_t magic = pack2(12582912.f, 12582912.f);          // 1.5 * 2^23: the sum's low mantissa bits hold i
+  const uint64_t t2 = add2(x2, magic);
+  const uint64_t f2 = sub2(x2, sub2(t2, magic));
+  uint64_t q2 = fma2(f2, pack2(0.055171459913253784f, 0.055171459913253784f), pack2(0.2426108568906784f, 0.2426108568906784f));
+  q2 = fma2(q2, f2, pack2(0.6932609677314758f, 0.6932609677314758f));
+  q2 = fma2(q2, f2, pack2(0.9999281167984009f, 0.9999281167984009f));
+  float t0, t1, q0, q1;
+  unpack2(t2, t0, t1);
+  unpack2(q2, q0, q1);
+  p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+  p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
 }
 
 // warpgroup-wide change of the per-thread register allowance (every warp of the warpgroup executes it)
@@ -426,9 +448,16 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           uint32_t pk[16];
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            float t0, t1;
-            unpack2(fma2(pack2u(r[e], r[e + 1]), sc2, nref2), t0, t1);
-            const float p0 = ex2(t0), p1 = ex2(t1);
+            const uint64_t x2 = fma2(pack2u(r[e], r[e + 1]), sc2, nref2);
+            float p0, p1;
+            if ((e >> 1) % kPolyEvery == kPolyEvery - 1) {       // this pair on the FMA pipe, the others on the MUFU
+              exp2_poly2(x2, p0, p1);
+            } else {
+              float t0, t1;
+              unpack2(x2, t0, t1);
+              p0 = ex2(t0);
+              p1 = ex2(t1);
+            }
             sum2 = add2(sum2, pack2(p0, p1));
             pk[e >> 1] = pack_bf16(p0, p1);
           }
