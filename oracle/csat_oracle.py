@@ -13,7 +13,8 @@ paper's column vectors alpha_i, Z_i, C_i appear here as 1 x d rows):
   softmax_rows       A~ = softmax over the m measurements (same equation)
   compressed_output  Z  = A~ V~                           (compressed attention output)
   decoder_setup      S, B, theta of the LISTA recurrence, instantiated as ISTA
-  ista               alpha^{t+1} = eta_theta(S alpha^t + B Z_i)   (LISTA recurrence)
+  ista               alpha^{t+1} = eta_theta(S alpha^t + B Z_i)   (LISTA recurrence, ISTA weights)
+  lista              the same recurrence with supplied S, B and per-layer theta_t
   reconstruct        C^_i = Psi alpha^_i                  (reconstruction equation)
 
 Reading of the decoder (the paper's "Z_i = Phi Psi alpha_i" with Phi in R^{m x n}
@@ -114,6 +115,25 @@ def ista(Z: np.ndarray, S_dec: np.ndarray, B_dec: np.ndarray, theta: float, T: i
     return (alpha, its) if return_iterates else alpha
 
 
+def lista(Z: np.ndarray, S: np.ndarray, B: np.ndarray, thetas, return_iterates: bool = False):
+    """LISTA recurrence with supplied ("learned") weights, row-wise:
+    alpha^{t+1} = eta_{theta_t}(alpha^t S + Z B), t = 0 .. T-1, alpha^0 = 0, T = len(thetas).
+
+    Z [rows,p], S [q,q], B [p,q], thetas: sequence of T thresholds (one per layer) -> alpha [rows,q].
+    The paper's S, B carry no layer index (shared over the t layers); eta_theta may differ per layer.
+    """
+    Z = np.asarray(Z, F64)
+    S = np.asarray(S, F64)
+    c = Z @ np.asarray(B, F64)
+    alpha = np.zeros((Z.shape[0], S.shape[0]), dtype=F64)
+    its = [alpha]
+    for th in thetas:
+        alpha = soft_threshold(alpha @ S + c, th)
+        if return_iterates:
+            its.append(alpha)
+    return (alpha, its) if return_iterates else alpha
+
+
 def reconstruct(alpha: np.ndarray, Psi: np.ndarray | None) -> np.ndarray:
     """C^_i = Psi alpha^_i, row-wise: out = alpha Psi^T (Psi = I when None)."""
     if Psi is None:
@@ -132,8 +152,10 @@ def default_decoder_matrix(Phi_h: np.ndarray, d: int) -> np.ndarray:
 # the whole forward
 # ----------------------------------------------------------------------------
 def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, scale=None,
-                      stages: dict | None = None) -> np.ndarray:
-    """CSAT forward for one (batch, head).  Q [n_q,d], K,V [n,d], Phi_h [m,n] -> [n_q,d]."""
+                      stages: dict | None = None, weights=None) -> np.ndarray:
+    """CSAT forward for one (batch, head).  Q [n_q,d], K,V [n,d], Phi_h [m,n] -> [n_q,d].
+    weights = (S [d,d], B [d,d], thetas [T]) replaces the ISTA-derived decoder by supplied LISTA weights
+    (lam, D and step are then unused)."""
     Q = np.asarray(Q, F64)
     d = Q.shape[1]
     Kt = compress(Phi_h, K)
@@ -145,6 +167,13 @@ def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, sc
         stages.update(Kt=Kt, Vt=Vt, Z=Z)
     if int(T) == 0:
         return Z
+    if weights is not None:
+        S_w, B_w, thetas = weights
+        assert len(thetas) == int(T)
+        alpha = lista(Z, S_w, B_w, thetas)
+        if stages is not None:
+            stages.update(alpha=alpha)
+        return reconstruct(alpha, Psi)
     if D is None:
         D = default_decoder_matrix(Phi_h, d)
     D = np.asarray(D, F64)
@@ -157,7 +186,7 @@ def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, sc
 
 
 def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=None,
-                 stages: list | None = None) -> np.ndarray:
+                 stages: list | None = None, weights=None) -> np.ndarray:
     """CSAT forward.  Q [B,H,n_q,d], K,V [B,H,n,d], Phi [H,m,n] (one per head, shared over the
     batch, Phi_K = Phi_V), Psi None | [d,d] | [H,d,d], D None | [H,d,d]  ->  out [B,H,n_q,d]."""
     Q = np.asarray(Q)
@@ -168,8 +197,10 @@ def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=Non
             psi_h = None if Psi is None else (Psi if np.ndim(Psi) == 2 else Psi[h])
             D_h = None if D is None else D[h]
             st = {} if stages is not None else None
+            # weights = (S [H,d,d], B [H,d,d], thetas [T,H])
+            w_h = None if weights is None else (weights[0][h], weights[1][h], [th[h] for th in weights[2]])
             out[b, h] = csat_forward_head(Q[b, h], K[b, h], V[b, h], Phi[h], T=T, lam=lam,
-                                          Psi=psi_h, D=D_h, step=step, scale=scale, stages=st)
+                                          Psi=psi_h, D=D_h, step=step, scale=scale, stages=st, weights=w_h)
             if stages is not None:
                 stages.append(st)
     return out

@@ -85,6 +85,25 @@ def _output_uses_unweighted(A, Vt):
     return np.ones_like(A) / A.shape[1] @ np.asarray(Vt, F64)
 
 
+def _lista_S_transposed(Z, S, B, thetas, return_iterates=False):
+    return _orig_lista(Z, np.asarray(S, F64).T, B, thetas, return_iterates)
+
+
+def _lista_first_theta_everywhere(Z, S, B, thetas, return_iterates=False):
+    thetas = list(thetas)
+    return _orig_lista(Z, S, B, [thetas[0]] * len(thetas), return_iterates)
+
+
+def _lista_drop_input(Z, S, B, thetas, return_iterates=False):
+    # Z B only feeds the first layer
+    Z = np.asarray(Z, F64)
+    alpha = np.zeros((Z.shape[0], np.asarray(S).shape[0]))
+    for i, th in enumerate(thetas):
+        alpha = orc.soft_threshold(alpha @ S + (Z @ B if i == 0 else 0.0), th)
+    return alpha
+
+
+_orig_lista = orc.lista
 _orig_setup = orc.decoder_setup
 _orig_ista = orc.ista
 
@@ -103,6 +122,9 @@ MUTATIONS = {
     "decoder block from last rows": ("default_decoder_matrix", _block_offset),
     "ista: B dropped": ("ista", _ista_drop_B),
     "ista: one iteration short": ("ista", _ista_one_short),
+    "lista: S transposed": ("lista", _lista_S_transposed),
+    "lista: per-layer thresholds ignored": ("lista", _lista_first_theta_everywhere),
+    "lista: input only in the first layer": ("lista", _lista_drop_input),
     "compress: |Phi|": ("compress", _compress_abs),
     "output: weights ignored": ("compressed_output", _output_uses_unweighted),
 }

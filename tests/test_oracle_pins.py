@@ -13,6 +13,7 @@ import pytest
 
 from oracle import csat_oracle as orc
 from oracle import phi_oracle as phi
+from paper_2507_02957_b200 import workloads as wl
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 
@@ -378,3 +379,67 @@ def test_phi_moments_and_normality():
     for lag in (1, 2, 3, 4):
         c = np.corrcoef(g[:-lag], g[lag:])[0, 1]
         assert abs(c) < 4 / np.sqrt(N)
+
+
+# ---------------------------------------------------------------------------------------------------
+# LISTA recurrence with supplied weights (paper: alpha^{t+1} = eta_theta(S alpha^t + B Z_i), learned S, B, theta)
+# ---------------------------------------------------------------------------------------------------
+def test_lista_with_ista_weights_is_ista():
+    r = np.random.default_rng(21)
+    M = r.standard_normal((12, 9)) / 3.0
+    Z = r.standard_normal((7, 12))
+    S_dec, B_dec, theta, _ = orc.decoder_setup(M, 0.07)
+    for T in (1, 2, 9):
+        assert np.array_equal(orc.lista(Z, S_dec, B_dec, [theta] * T), orc.ista(Z, S_dec, B_dec, theta, T))
+
+
+def test_lista_matches_scalar_loops_with_per_layer_thresholds():
+    """Brute force: every coordinate by Python loops, non-symmetric S, thresholds that differ per layer."""
+    r = np.random.default_rng(22)
+    p, q, rows = 3, 4, 2
+    S = r.standard_normal((q, q)) * 0.4
+    B = r.standard_normal((p, q))
+    Z = r.standard_normal((rows, p))
+    thetas = [0.3, 0.05, 0.2]
+    alpha = [[0.0] * q for _ in range(rows)]
+    for th in thetas:
+        new = [[0.0] * q for _ in range(rows)]
+        for i in range(rows):
+            for b in range(q):
+                x = sum(alpha[i][a] * S[a][b] for a in range(q)) + sum(Z[i][a] * B[a][b] for a in range(p))
+                new[i][b] = (abs(x) - th) * (1 if x > 0 else -1) if abs(x) > th else 0.0
+        alpha = new
+    assert np.allclose(orc.lista(Z, S, B, thetas), np.array(alpha), rtol=0, atol=1e-14)
+
+
+def test_lista_special_cases():
+    r = np.random.default_rng(23)
+    Z = r.standard_normal((5, 6))
+    B = r.standard_normal((6, 6))
+    # S = 0: every layer forgets the previous iterate, the result is the last layer's shrinkage of Z B
+    out = orc.lista(Z, np.zeros((6, 6)), B, [0.5, 0.1, 0.25])
+    assert np.array_equal(out, orc.soft_threshold(Z @ B, 0.25))
+    # theta = 0, S = I - B (B symmetric positive definite, ||I - B|| < 1): Neumann series, alpha^T -> Z
+    A = r.standard_normal((6, 6))
+    Bs = 0.5 * np.eye(6) + 0.05 * (A @ A.T) / 6
+    out = orc.lista(Z, np.eye(6) - Bs, Bs, [0.0] * 400)
+    assert np.allclose(out, Z, atol=1e-9)
+    # transposed S must give a different answer (row-vector convention alpha S)
+    Sn = r.standard_normal((6, 6)) * 0.3
+    assert not np.allclose(orc.lista(Z, Sn, B, [0.1] * 3), orc.lista(Z, Sn.T, B, [0.1] * 3))
+
+
+def test_forward_with_supplied_weights_uses_them():
+    w = wl.shrink(wl.CONFIGS["c1"], n=32, n_q=8, m=16, d=8)
+    inp = wl.make_inputs(w)
+    Phi = phi.phi_gaussian(1, w.m, w.n, 0)
+    r = np.random.default_rng(24)
+    S = r.standard_normal((1, 8, 8)) * 0.2
+    B = r.standard_normal((1, 8, 8)) * 0.5
+    thetas = [[0.05], [0.02]]
+    st = []
+    out = orc.csat_forward(inp["Q"], inp["K"], inp["V"], Phi, T=2, lam=123.0, weights=(S, B, thetas), stages=st)
+    Z = st[0]["Z"]
+    a1 = orc.soft_threshold(Z @ B[0], 0.05)
+    a2 = orc.soft_threshold(a1 @ S[0] + Z @ B[0], 0.02)
+    assert np.allclose(out[0, 0], a2, atol=1e-14)
