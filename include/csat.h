@@ -126,6 +126,17 @@ int csat_set_dictionary(csat_ctx* ctx, const void* psi, int per_head, void* stre
  * (otherwise csat_forward with T > 0 returns CSAT_ERR_SHAPE).  Copied on `stream`. */
 int csat_set_decoder_matrix(csat_ctx* ctx, const void* D, void* stream);
 
+/* csat_set_lista_weights -- paper: LISTA recurrence alpha^{t+1} = eta_theta(S alpha^t + B Z_i), where "S, B and
+ * eta_theta are learned weight matrices and nonlinearities" shared by the t layers.  Replaces the ISTA-derived
+ * decoder by supplied weights, row-vector convention alpha <- eta(alpha S + z B):
+ *   S, Bm   [H, d, d], context dtype, device (row-major: S[a][b] multiplies alpha_a into column b)
+ *   theta   [layers, H] float32, device, every entry >= 0; layers = 1 uses the same threshold in every
+ *           layer, otherwise layers must equal CSAT_T when csat_forward runs (else CSAT_ERR_STATE).
+ * The weights are copied on `stream`.  CSAT_LAMBDA, CSAT_STEP and the decoder matrix D are ignored while supplied
+ * weights are in force; the dictionary Psi still applies to the reconstruction.  S = NULL restores the
+ * ISTA-derived decoder.  On the bf16 tensor-core path S enters as I - W with W = I - S rounded to bf16. */
+int csat_set_lista_weights(csat_ctx* ctx, const void* S, const void* Bm, const float* theta, int layers, void* stream);
+
 /*
  * csat_forward -- paper: compression, approximate attention matrix, compressed output,
  * LISTA recurrence and reconstruction equations (all of the hot path).

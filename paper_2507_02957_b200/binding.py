@@ -36,6 +36,7 @@ SIGNATURES = {
     "csat_get_phi": (_int, [_vp, _vp, _vp]),
     "csat_set_dictionary": (_int, [_vp, _vp, _int, _vp]),
     "csat_set_decoder_matrix": (_int, [_vp, _vp, _vp]),
+    "csat_set_lista_weights": (_int, [_vp, _vp, _vp, _vp, _int, _vp]),
     "csat_forward": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_forward_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
@@ -144,6 +145,10 @@ def csat_set_dictionary(h, psi, per_head=False, stream=None):
 
 def csat_set_decoder_matrix(h, D, stream=None):
     _check(h, load().csat_set_decoder_matrix(h, _ptr(D), _stream(stream)))
+
+
+def csat_set_lista_weights(h, S, Bm, theta, layers, stream=None):
+    _check(h, load().csat_set_lista_weights(h, _ptr(S), _ptr(Bm), _ptr(theta), int(layers), _stream(stream)))
 
 
 def csat_forward(h, Q, K, V, out, stream=None):
@@ -287,6 +292,16 @@ class Csat:
             assert D.shape == (self.H, self.d, self.d) and D.dtype == self.torch_dtype
             D = D.contiguous()
         csat_set_decoder_matrix(self.h, D)
+
+    def set_lista_weights(self, S, Bm=None, theta=None):
+        """Supplied LISTA weights: S, Bm [H,d,d] (context dtype), theta [layers,H] or [H] float32; S=None restores
+        the ISTA-derived decoder."""
+        if S is None:
+            csat_set_lista_weights(self.h, None, None, None, 1)
+            return
+        assert S.shape == (self.H, self.d, self.d) and Bm.shape == S.shape and S.dtype == self.torch_dtype == Bm.dtype
+        theta = theta.reshape(-1, self.H).to(torch.float32).contiguous()
+        csat_set_lista_weights(self.h, S.contiguous(), Bm.contiguous(), theta, theta.shape[0])
 
     def get_compressed(self):
         kt = self._new(self.B, self.H, self.m, self.d)

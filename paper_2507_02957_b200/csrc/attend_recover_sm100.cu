@@ -28,7 +28,8 @@
 // All MMAs of the CTA execute in issue order, so S_{j+2} overwrites S[j&1] only after P_j V~_j has read P_j.
 //
 // Recovery phase, per tile.  The accumulator holds r_t = theta + c - a^_t (mu G), where c = z B and a^_t is
-// the sum of the bf16 increments fed to the tensor cores so far; the registers hold b_t = alpha^t - theta:
+// the sum of the bf16 increments fed to the tensor cores so far; the registers hold b_t = alpha^t - theta
+// (theta = the first layer's threshold where the thresholds differ per layer; eta then uses the layer's own):
 //   r_0 = theta + z_bf16 B (threads store theta, one accumulating MMA);
 //   x = b_t + r_t = alpha^t S + z B;   b_{t+1} = eta_theta(x) - theta = x - 2 theta sat(x / (2 theta) + 1/2);
 //   r_{t+1} = r_t + bf16(b_t - b_{t+1}) (mu G)             (one accumulating MMA per iteration).
@@ -39,6 +40,8 @@
 #include "csat_internal.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
+
+#include <type_traits>
 
 namespace csat {
 namespace {
@@ -181,8 +184,8 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
-                            const float* __restrict__ theta, int nq, int m, int H, int T, int has_psi,
-                            float scale_log2, int* status) {
+                            const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
+                            int has_psi, float scale_log2, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
@@ -516,58 +519,69 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       };
 
       if (T > 0) {
-        const float th = theta[h];
-        const float inv2th = th > 0.f ? 0.5f / th : 0.f;        // theta = 0: sat(1/2) = 1/2 and b' = x
-        const uint64_t m2th2 = pack2(-2.f * th, -2.f * th);
+        // layer t uses theta[t * theta_stride + h] (stride 0: one threshold for all layers).  The accumulator is
+        // biased by kappa = theta of layer 0 and the registers hold b = alpha - kappa throughout.
+        const float kappa = theta[h];
         const uint32_t op_addr = tbase + C::kColS;
-        // accumulator := theta (r_0 = theta + z B), and z as the bf16 A operand
+        // accumulator := kappa (r_0 = kappa + z B), and z as the bf16 A operand
         {
           uint32_t tb[16];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) tb[e] = __float_as_uint(th);
+          for (int e = 0; e < 16; ++e) tb[e] = __float_as_uint(kappa);
 #pragma unroll
           for (int c0 = 0; c0 < D; c0 += 16) tmem_st_32x32b_x16(acc_addr + c0, tb);
         }
         publish();
 #pragma unroll
-        for (int i = 0; i < D / 2; ++i) v2[i] = pack2(-th, -th);        // b = alpha - theta, alpha^0 = 0
+        for (int i = 0; i < D / 2; ++i) v2[i] = pack2(-kappa, -kappa);  // alpha^0 = 0
         int phase = 0;
-        for (int it = 0; it + 1 < T; ++it) {
-          w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
-          tc_fence_after();
-          // 16 columns at a time, the next piece's TMEM load in flight while this one is shrunk
-          auto shrink16 = [&](const uint32_t (&r)[16], int c0) {
-            uint32_t pk[8];
+        // per_layer is a compile-time tag: with one threshold for all layers theta_t - kappa = 0 and the add of it
+        // is left out of the inner loop
+        auto iterate = [&](auto per_layer) {
+          for (int it = 0; it + 1 < T; ++it) {
+            const float th = per_layer.value ? theta[(int64_t)it * theta_stride + h] : kappa;
+            const float inv2th = th > 0.f ? 0.5f / th : 0.f;        // theta = 0: sat(1/2) = 1/2 and eta(x) = x
+            const uint64_t m2th2 = pack2(-2.f * th, -2.f * th);
+            const uint64_t dk2 = pack2(th - kappa, th - kappa);
+            w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
+            tc_fence_after();
+            // 16 columns at a time, the next piece's TMEM load in flight while this one is shrunk
+            auto shrink16 = [&](const uint32_t (&r)[16], int c0) {
+              uint32_t pk[8];
 #pragma unroll
-            for (int e = 0; e < 16; e += 2) {
-              const uint64_t bo = v2[(c0 + e) >> 1];
-              const uint64_t x2 = add2(bo, pack2u(r[e], r[e + 1]));          // alpha^t S + z B
-              float x0, x1;
-              unpack2(x2, x0, x1);
-              const uint64_t t2 = pack2(fma_sat(x0, inv2th, 0.5f), fma_sat(x1, inv2th, 0.5f));
-              const uint64_t bn = fma2(t2, m2th2, x2);                       // eta_theta(x) - theta
-              v2[(c0 + e) >> 1] = bn;
-              float d0, d1;
-              unpack2(sub2(bo, bn), d0, d1);                                 // alpha^t - alpha^{t+1}
-              pk[e >> 1] = pack_bf16(d0, d1);
+              for (int e = 0; e < 16; e += 2) {
+                const uint64_t bo = v2[(c0 + e) >> 1];
+                const uint64_t x2 = add2(bo, pack2u(r[e], r[e + 1]));          // alpha^t S + z B
+                float x0, x1;
+                unpack2(x2, x0, x1);
+                const uint64_t t2 = pack2(fma_sat(x0, inv2th, 0.5f), fma_sat(x1, inv2th, 0.5f));
+                uint64_t bn = fma2(t2, m2th2, x2);                             // eta_theta(x) - theta
+                if (per_layer.value) bn = add2(bn, dk2);                       // ... - kappa
+                v2[(c0 + e) >> 1] = bn;
+                float d0, d1;
+                unpack2(sub2(bo, bn), d0, d1);                                 // alpha^t - alpha^{t+1}
+                pk[e >> 1] = pack_bf16(d0, d1);
+              }
+              tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+            };
+            uint32_t r0[16], r1[16];
+            tmem_ld_32x32b_x16(acc_addr, r0);
+#pragma unroll
+            for (int c0 = 0; c0 < D; c0 += 32) {
+              tmem_wait_ld();
+              tmem_ld_32x32b_x16(acc_addr + c0 + 16, r1);
+              shrink16(r0, c0);
+              tmem_wait_ld();
+              if (c0 + 32 < D) tmem_ld_32x32b_x16(acc_addr + c0 + 32, r0);
+              shrink16(r1, c0 + 16);
             }
-            tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
-          };
-          uint32_t r0[16], r1[16];
-          tmem_ld_32x32b_x16(acc_addr, r0);
-#pragma unroll
-          for (int c0 = 0; c0 < D; c0 += 32) {
-            tmem_wait_ld();
-            tmem_ld_32x32b_x16(acc_addr + c0 + 16, r1);
-            shrink16(r0, c0);
-            tmem_wait_ld();
-            if (c0 + 32 < D) tmem_ld_32x32b_x16(acc_addr + c0 + 32, r0);
-            shrink16(r1, c0 + 16);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(&bars->a_full[t]);
           }
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(&bars->a_full[t]);
-        }
+        };
+        if (theta_stride != 0) iterate(std::true_type{}); else iterate(std::false_type{});
+        const float th = theta[(int64_t)(T - 1) * theta_stride + h];
         // last iteration, exact shrinkage: alpha^T = eta_theta(x)
         w.wait(&bars->r_full[t], phase & 1, 231); ++phase;
         tc_fence_after();
@@ -638,7 +652,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   const int64_t rows_per_cta = kTiles * kRows;
   const dim3 grid((unsigned)((p.nq + rows_per_cta - 1) / rows_per_cta), (unsigned)(p.B * p.H));
   attend_recover_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(
-      tq, c->tmap_kv, c->tmap_mats, (__nv_bfloat16*)out, c->theta, (int)p.nq, (int)p.m, (int)p.H, p.T,
+      tq, c->tmap_kv, c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, p.T,
       c->psi ? 1 : 0, scale_log2, c->status);
   return cudaGetLastError();
 }

@@ -45,6 +45,14 @@ size_t dd_bytes(const csat::Params& p, size_t elt) { return (size_t)(p.H * p.d *
 
 void prof_destroy(csat_ctx* c);
 
+void free_lista(csat_ctx* c) {
+  const csat::Params& p = c->p;
+  dev_free(c, &c->w_S, dd_bytes(p, csat::elt_size(p.dtype)));
+  dev_free(c, &c->w_B, dd_bytes(p, csat::elt_size(p.dtype)));
+  dev_free(c, &c->w_theta, (size_t)c->w_layers * p.H * 4);
+  c->w_layers = 0;
+}
+
 void free_staging(csat_ctx* c) {
   dev_free(c, &c->stage_q, c->stage_bytes_q);
   dev_free(c, &c->stage_o, c->stage_bytes_q);
@@ -67,6 +75,7 @@ void free_all(csat_ctx* c) {
   dev_free(c, &c->theta, (size_t)p.H * 4);
   dev_free(c, &c->mu, (size_t)p.H * 4);
   dev_free(c, &c->mats_bf16, 3 * dd_bytes(p, 2));
+  free_lista(c);
   free_staging(c);
   prof_destroy(c);
   if (c->status) {
@@ -230,6 +239,7 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       dev_free(c, &c->kv, kv_bytes(p));
       dev_free(c, &c->psi, (size_t)((c->psi_per_head ? p.H : 1) * p.d * p.d) * csat::elt_size(p.dtype));
       dev_free(c, &c->dmat, dd_bytes(p, csat::elt_size(p.dtype)));
+      free_lista(c);
       free_staging(c);
       p.dtype = (int)v;
       return allocate_and_generate(c);   // user-set Phi, Psi, D are dropped with the old dtype
@@ -367,9 +377,39 @@ int csat_set_decoder_matrix(csat_ctx* c, const void* D, void* stream) {
   return CSAT_OK;
 }
 
+int csat_set_lista_weights(csat_ctx* c, const void* S, const void* Bm, const float* theta, int layers, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  csat::Params& p = c->p;
+  c->decoder_dirty = true;
+  if (!S) {
+    if (c->w_S) { cudaDeviceSynchronize(); free_lista(c); }
+    return CSAT_OK;
+  }
+  if (!Bm || !theta) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_lista_weights: NULL pointer");
+  if (!aligned16(S) || !aligned16(Bm)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_lista_weights: misaligned pointer");
+  if (layers < 1 || layers > 100000) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_lista_weights: layers must be >= 1");
+  const size_t mat_bytes = dd_bytes(p, csat::elt_size(p.dtype));
+  if (c->w_S && c->w_layers != layers) { cudaDeviceSynchronize(); free_lista(c); }
+  if (!c->w_S) {
+    c->w_layers = layers;
+    if (dev_alloc(c, &c->w_S, mat_bytes) != cudaSuccess || dev_alloc(c, &c->w_B, mat_bytes) != cudaSuccess ||
+        dev_alloc(c, &c->w_theta, (size_t)layers * p.H * 4) != cudaSuccess) {
+      free_lista(c);
+      return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(LISTA weights) failed");
+    }
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(c->w_S, S, mat_bytes, cudaMemcpyDeviceToDevice, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(c->w_B, Bm, mat_bytes, cudaMemcpyDeviceToDevice, s)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(c->w_theta, theta, (size_t)layers * p.H * 4, cudaMemcpyDeviceToDevice, s)) != cudaSuccess)
+    return fail_cuda(c, e, "csat_set_lista_weights");
+  return CSAT_OK;
+}
+
 static int ensure_decoder(csat_ctx* c, cudaStream_t s, int* launches) {
   const csat::Params& p = c->p;
-  if (!c->dmat && (p.m < p.d || p.n < p.d))
+  if (!c->w_S && !c->dmat && (p.m < p.d || p.n < p.d))
     return fail(c, CSAT_ERR_SHAPE, "default decoder matrix D = Phi[0:d,0:d] needs m >= d and n >= d");
   if (!c->decoder_dirty) return CSAT_OK;
   cudaError_t e = csat::launch_decoder_setup(c, s, launches);
@@ -391,6 +431,8 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   cudaStream_t s = (cudaStream_t)stream;
   int launches = 0;
   prof_mark(c, s, -1);
+  if (c->p.T > 0 && c->w_S && c->w_layers != 1 && c->w_layers != c->p.T)
+    return fail(c, CSAT_ERR_STATE, "csat_set_lista_weights was given thresholds for a number of layers other than CSAT_T");
   if (c->p.T > 0) {
     const bool was_dirty = c->decoder_dirty;
     int rc = ensure_decoder(c, s, &launches);
@@ -466,7 +508,7 @@ int csat_get_decoder(csat_ctx* c, float* S_out, float* B_out, float* theta_out, 
   cudaError_t e = cudaSuccess;
   if (S_out && e == cudaSuccess) e = cudaMemcpyAsync(S_out, c->S_dec, dd_bytes(p, 4), cudaMemcpyDeviceToDevice, s);
   if (B_out && e == cudaSuccess) e = cudaMemcpyAsync(B_out, c->B_dec, dd_bytes(p, 4), cudaMemcpyDeviceToDevice, s);
-  if (theta_out && e == cudaSuccess) e = cudaMemcpyAsync(theta_out, c->theta, (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
+  if (theta_out && e == cudaSuccess) e = cudaMemcpyAsync(theta_out, c->thr(), (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
   if (mu_out && e == cudaSuccess) e = cudaMemcpyAsync(mu_out, c->mu, (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_get_decoder");
   return CSAT_OK;

@@ -51,7 +51,12 @@ struct csat_ctx {
   float* S_dec = nullptr;     // [H, d, d]  I - mu G
   float* B_dec = nullptr;     // [H, d, d]  mu M
   float* psi_f32 = nullptr;   // [H, d, d]  Psi as float (row-major), only when psi != null
-  float* theta = nullptr;     // [H]
+  float* theta = nullptr;     // [H] (ISTA-derived) 
+  // supplied LISTA weights (csat_set_lista_weights); null = ISTA-derived decoder
+  void* w_S = nullptr;        // [H, d, d] dtype
+  void* w_B = nullptr;        // [H, d, d] dtype
+  float* w_theta = nullptr;   // [w_layers, H]
+  int w_layers = 0;
   float* mu = nullptr;        // [H]
   int* status = nullptr;      // device status word (0 = ok)
   // staging for csat_forward_host
@@ -65,6 +70,10 @@ struct csat_ctx {
   std::vector<cudaEvent_t> prof_events;         // [slots][kProfMaxKernels + 1]
   std::vector<int> prof_ids;                    // [slots][kProfMaxKernels]
   std::vector<int> prof_count;                  // [slots]
+
+  // thresholds the kernels read: theta_t of head h at thr()[t * thr_stride() + h]
+  const float* thr() const { return w_S ? w_theta : theta; }
+  int thr_stride() const { return (w_S && w_layers > 1) ? (int)p.H : 0; }
 
   bool decoder_dirty = true;
   bool have_forward = false;

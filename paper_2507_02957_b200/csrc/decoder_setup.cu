@@ -89,11 +89,42 @@ __global__ void finalize_kernel(float* __restrict__ S_dec, float* __restrict__ B
   }
 }
 
+// Supplied LISTA weights: S, B as given (float32 copies for the FFMA kernels), and the tensor-core operand
+// copies, each stored [output column][k]: W = I - S (so that alpha S = alpha - alpha W), B, Psi.
+template <typename T>
+__global__ void weights_kernel(float* __restrict__ S_dec, float* __restrict__ B_dec, float* __restrict__ mu_out,
+                               float* __restrict__ psi_f32, const T* __restrict__ S, const T* __restrict__ Bm,
+                               const T* __restrict__ psi, int psi_per_head, int d,
+                               __nv_bfloat16* __restrict__ mats_bf16) {
+  const int h = blockIdx.y;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= d * d) return;
+  const int a = i / d, b = i % d;
+  const int64_t base = (int64_t)h * d * d;
+  S_dec[base + i] = (float)ld(S, base + i);
+  B_dec[base + i] = (float)ld(Bm, base + i);
+  const T* P = psi ? psi + (psi_per_head ? base : 0) : nullptr;
+  if (P) psi_f32[base + i] = (float)ld(P, i);
+  if (mats_bf16) {
+    __nv_bfloat16* mh = mats_bf16 + base * 3;
+    mh[i] = __float2bfloat16_rn((float)((a == b ? 1.0 : 0.0) - ld(S, base + (int64_t)b * d + a)));   // W[b][a]
+    mh[d * d + i] = __float2bfloat16_rn((float)ld(Bm, base + (int64_t)b * d + a));                    // B[b][a]
+    mh[2 * d * d + i] = P ? __float2bfloat16_rn((float)ld(P, i)) : __float2bfloat16_rn(0.f);
+  }
+  if (i == 0) mu_out[h] = 0.f;
+}
+
 template <typename T>
 cudaError_t run(csat_ctx* c, cudaStream_t s, int* launches) {
   const Params& p = c->p;
   const int d = (int)p.d, H = (int)p.H;
   const dim3 grid((d * d + 255) / 256, H);
+  if (c->w_S) {
+    weights_kernel<T><<<grid, 256, 0, s>>>(c->S_dec, c->B_dec, c->mu, c->psi_f32, (const T*)c->w_S, (const T*)c->w_B,
+                                           (const T*)c->psi, c->psi_per_head ? 1 : 0, d, c->mats_bf16);
+    *launches += 1;
+    return cudaGetLastError();
+  }
   build_M_kernel<T><<<grid, 256, 0, s>>>(c->Mf64, (const T*)c->phi, (const T*)c->dmat, (const T*)c->psi,
                                          c->psi_per_head ? 1 : 0, d, p.m, p.n_pad);
   gram_kernel<<<grid, 256, 0, s>>>(c->Gf64, c->Mf64, d);
