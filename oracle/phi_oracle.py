@@ -85,3 +85,24 @@ def phi_gaussian(H: int, m: int, n: int, seed: int, heads=None) -> np.ndarray:
              + np.arange(m * n, dtype=np.uint64)).reshape(m, n)
         out[i] = gaussian_elements(e, seed) / np.sqrt(np.float64(m))
     return out
+
+
+def phi_rademacher(H: int, m: int, n: int, seed: int, heads=None) -> np.ndarray:
+    """Rademacher ensemble (the paper's second example of a sub-Gaussian measurement matrix):
+    Phi[h,r,j] = +-1/sqrt(m), float64 (unrounded).
+
+    Reading (the paper fixes no generator): element e = (h*m + r)*n + j takes bit e % 32 of word (e // 32) % 4
+    of the Philox4x32-10 block with counter (q low, q high, 1, 0), q = e // 128, key = seed; a set bit means
+    -1/sqrt(m).  (The third counter word is 1 so that the stream differs from the Gaussian ensemble's.)
+    """
+    heads = range(H) if heads is None else heads
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    out = np.empty((len(heads), m, n), dtype=np.float64)
+    for i, h in enumerate(heads):
+        e = np.uint64(h) * np.uint64(m) * np.uint64(n) + np.arange(m * n, dtype=np.uint64)
+        q = e >> np.uint64(7)
+        words = np.stack(philox4x32_10(q & _MASK, q >> _S32, 1, 0, seed & 0xFFFFFFFF, seed >> 32), axis=-1)
+        word = np.take_along_axis(words, ((e >> np.uint64(5)) & np.uint64(3)).astype(np.int64)[:, None], axis=-1)[:, 0]
+        bit = (word >> (e & np.uint64(31))) & np.uint64(1)
+        out[i] = ((1.0 - 2.0 * bit.astype(np.float64)) / np.sqrt(np.float64(m))).reshape(m, n)
+    return out

@@ -443,3 +443,49 @@ def test_forward_with_supplied_weights_uses_them():
     a1 = orc.soft_threshold(Z @ B[0], 0.05)
     a2 = orc.soft_threshold(a1 @ S[0] + Z @ B[0], 0.02)
     assert np.allclose(out[0, 0], a2, atol=1e-14)
+
+
+# ---------------------------------------------------------------------------------------------------
+# Rademacher measurement matrices (paper: "random Gaussian, Rademacher, or structured Hadamard matrices")
+# ---------------------------------------------------------------------------------------------------
+def _philox_scalar(ctr, key):
+    """Philox4x32-10 on Python ints, written from the published round function (checked against the
+    known-answer vectors below before it is used)."""
+    c = list(ctr)
+    k0, k1 = key
+    for _ in range(10):
+        p0, p1 = 0xD2511F53 * c[0], 0xCD9E8D57 * c[2]
+        c = [(p1 >> 32) ^ c[1] ^ k0, p1 & 0xFFFFFFFF, (p0 >> 32) ^ c[3] ^ k1, p0 & 0xFFFFFFFF]
+        k0, k1 = (k0 + 0x9E3779B9) & 0xFFFFFFFF, (k1 + 0xBB67AE85) & 0xFFFFFFFF
+    return c
+
+
+def test_rademacher_layout_by_scalar_brute_force():
+    # the scalar routine reproduces the published known-answer vectors
+    assert _philox_scalar([0, 0, 0, 0], [0, 0]) == [0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8]
+    assert _philox_scalar([0xFFFFFFFF] * 4, [0xFFFFFFFF] * 2) == [0x408F276D, 0x41C83B0E, 0xA20BC7C6, 0x6D5451FD]
+    H, m, n, seed = 2, 5, 77, 0x0123456789ABCDEF
+    got = phi.phi_rademacher(H, m, n, seed)
+    for (h, r, j) in [(0, 0, 0), (0, 0, 31), (0, 0, 32), (0, 1, 50), (0, 4, 76), (1, 0, 0), (1, 3, 5), (1, 4, 76)]:
+        e = (h * m + r) * n + j
+        q = e // 128
+        words = _philox_scalar([q & 0xFFFFFFFF, q >> 32, 1, 0], [seed & 0xFFFFFFFF, seed >> 32])
+        bit = (words[(e // 32) % 4] >> (e % 32)) & 1
+        assert got[h, r, j] == (-1.0 if bit else 1.0) / math.sqrt(m)
+
+
+def test_rademacher_is_a_sign_matrix_with_unit_columns():
+    H, m, n = 3, 64, 500
+    P = phi.phi_rademacher(H, m, n, 7)
+    assert np.array_equal(np.abs(P), np.full_like(P, 1.0 / 8.0))
+    assert np.allclose((P ** 2).sum(axis=1), 1.0, atol=1e-15)                 # every column has norm exactly 1
+    assert abs(P.mean()) * 8.0 < 4.0 / math.sqrt(P.size)                      # balanced signs (4 sigma)
+    # rows are nearly orthogonal: off-diagonal Gram entries are sums of n independent signs / m
+    G = P[0] @ P[0].T
+    off = G[~np.eye(m, dtype=bool)]
+    assert np.abs(off).max() < 5.0 * math.sqrt(n) / m and abs(off.mean()) < 5.0 * math.sqrt(n) / m / math.sqrt(off.size) * 2
+    # another seed, another head: different matrices
+    assert not np.array_equal(P[0], P[1])
+    assert not np.array_equal(P, phi.phi_rademacher(H, m, n, 8))
+    # and not the Gaussian ensemble's sign pattern
+    assert not np.array_equal(np.sign(P), np.sign(phi.phi_gaussian(H, m, n, 7)))
