@@ -63,6 +63,9 @@ enum {
   CSAT_T = 4,          /* recovery iterations (decoder depth t), default 10; 0 = out = Z */
   CSAT_FORCE_SIMT = 5, /* diagnostic: 1 routes bf16 through the plain FFMA kernels, 2 only
                           the attention/recovery stage; 0 (default) = tensor-core kernels */
+  CSAT_ENSEMBLE = 7,   /* measurement ensemble: CSAT_ENSEMBLE_GAUSSIAN (default), N(0, 1/m) entries, or
+                          CSAT_ENSEMBLE_RADEMACHER, +-1/sqrt(m) entries (paper: "random Gaussian,
+                          Rademacher, ...").  Changing it regenerates Phi from the seed           */
   CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls
                           (0 = off, default; at most 4096).  Setting it creates/destroys
                           events, so set it outside the timed region                    */
@@ -76,6 +79,7 @@ enum {
   CSAT_KERNEL_SPLIT_REDUCE = 3   /* fixed-order sum of token-axis partial K~|V~ tiles    */
 };
 enum { CSAT_DTYPE_BF16 = 0, CSAT_DTYPE_FP32 = 1 };
+enum { CSAT_ENSEMBLE_GAUSSIAN = 0, CSAT_ENSEMBLE_RADEMACHER = 1 };
 
 /* keys of csat_set_f64 / csat_get_f64 */
 enum {
@@ -89,7 +93,9 @@ enum {
  * (Gaussian ensemble).  Builds a context for n key/value tokens, m measurements, head size d
  * and H heads on the CURRENT CUDA device, and generates one measurement matrix per head,
  * Phi[h,r,j] ~ N(0, 1/m) i.i.d. from `seed` (Philox4x32-10 keyed by seed, counter = flat element
- * index / 4, Box-Muller; Phi_K = Phi_V = Phi_h, shared over the batch).
+ * index / 4, Box-Muller; Phi_K = Phi_V = Phi_h, shared over the batch).  With CSAT_ENSEMBLE_RADEMACHER the
+ * entries are +-1/sqrt(m): element e takes bit e % 32 of word (e / 32) % 4 of the Philox block with counter
+ * (e / 128, 0, 1, 0) as (low, high, third, fourth) words; a set bit means the negative sign.
  * Requires 1 <= m <= n, d >= 1, H >= 1, d <= 256 and d % 8 == 0.  Returns NULL on failure;
  * csat_last_error(NULL) then gives the reason (thread-local).
  * Allocates device memory and synchronises.  Changing CSAT_DTYPE, CSAT_BATCH or CSAT_NQ later

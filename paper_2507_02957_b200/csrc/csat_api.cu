@@ -173,6 +173,7 @@ csat_ctx* csat_create(int64_t n, int64_t m, int64_t d, int64_t H, uint64_t seed)
   p.n = n; p.m = m; p.d = d; p.H = H; p.B = 1; p.nq = n;
   p.n_pad = csat::round_up(n, csat::kPhiColPad);
   p.dtype = CSAT_DTYPE_BF16;
+  p.ensemble = CSAT_ENSEMBLE_GAUSSIAN;
   p.T = 10; p.lambda = 0.1; p.step = 0.0; p.scale = 0.0; p.seed = seed;
 
   int rc = CSAT_OK;
@@ -244,6 +245,18 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       p.dtype = (int)v;
       return allocate_and_generate(c);   // user-set Phi, Psi, D are dropped with the old dtype
     }
+    case CSAT_ENSEMBLE: {
+      if (v != CSAT_ENSEMBLE_GAUSSIAN && v != CSAT_ENSEMBLE_RADEMACHER)
+        return fail(c, CSAT_ERR_INVALID_ARG, "unknown CSAT_ENSEMBLE");
+      if ((int)v == p.ensemble) return CSAT_OK;
+      cudaDeviceSynchronize();
+      p.ensemble = (int)v;
+      cudaError_t e = csat::launch_phi_gen(c->phi, p, 0);      // a Phi set by csat_set_phi is replaced as well
+      if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+      if (e != cudaSuccess) return fail_cuda(c, e, "phi_gen");
+      c->decoder_dirty = true;
+      return CSAT_OK;
+    }
     case CSAT_T:
       if (v < 0 || v > 100000) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_T must be in [0, 100000]");
       p.T = (int)v;
@@ -283,6 +296,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
     case CSAT_NQ: *out = c->p.nq; return CSAT_OK;
     case CSAT_DTYPE: *out = c->p.dtype; return CSAT_OK;
     case CSAT_T: *out = c->p.T; return CSAT_OK;
+    case CSAT_ENSEMBLE: *out = c->p.ensemble; return CSAT_OK;
     case CSAT_FORCE_SIMT: *out = c->force_simt; return CSAT_OK;
     case CSAT_PROFILE: *out = c->prof_slots; return CSAT_OK;
     default: return CSAT_ERR_INVALID_ARG;

@@ -21,6 +21,7 @@ struct Params {            // plain values kernels need
   int64_t n, m, d, H, B, nq;
   int64_t n_pad;           // padded row length of Phi
   int dtype;               // CSAT_DTYPE_*
+  int ensemble;            // CSAT_ENSEMBLE_*
   int T;
   double lambda, step, scale;
   uint64_t seed;

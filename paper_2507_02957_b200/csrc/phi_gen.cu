@@ -61,6 +61,81 @@ __global__ void phi_gen_kernel(T* __restrict__ phi, int64_t total, int64_t n, in
   }
 }
 
+// Rademacher ensemble: one sign bit per element of the unpadded index space, 128 elements per Philox block,
+// counter (q, 0, 1, 0) as (low, high, third, fourth) words.  A warp takes 32 consecutive blocks (4096
+// elements): lane l computes block l, and in step s the word (s % 4) of lane s / 4 is broadcast so that lane l
+// writes element 32 s + l: consecutive lanes write consecutive elements.  Write-bound.
+template <typename T>
+__global__ void phi_rademacher_kernel(T* __restrict__ phi, int64_t total, int64_t n, int64_t n_pad, float inv_sqrt_m,
+                                      uint32_t k0, uint32_t k1) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int64_t nspans = (total + 4095) >> 12;
+  const T pos = to_storage<T>(inv_sqrt_m), neg = to_storage<T>(-inv_sqrt_m);
+  for (int64_t span = warp; span < nspans; span += nwarps) {
+    const int64_t q = (span << 5) + lane;
+    const U4 u = philox4x32_10(U4{(uint32_t)q, (uint32_t)(q >> 32), 1u, 0u}, k0, k1);
+    int64_t e = (span << 12) + lane;
+    int64_t row = e / n;
+    int64_t j = e - row * n;
+#pragma unroll 4
+    for (int s = 0; s < 128; ++s) {
+      const int w = s & 3;
+      const uint32_t mine = w == 0 ? u.x : (w == 1 ? u.y : (w == 2 ? u.z : u.w));
+      const uint32_t bits = __shfl_sync(0xffffffffu, mine, s >> 2);
+      if (e < total) phi[row * n_pad + j] = ((bits >> lane) & 1u) ? neg : pos;
+      e += 32;
+      j += 32;
+      while (j >= n) { j -= n; ++row; }
+    }
+  }
+}
+
+// Same stream, n % 8 == 0: every lane writes 8 consecutive elements (one 16-byte store for bf16, two for
+// float) that never straddle a row.  A warp step covers 256 elements = 2 Philox blocks; lane l needs byte
+// (l % 4) of word (l / 4) % 4 of block 2 s + l / 16.
+template <typename T>
+__global__ void phi_rademacher_vec_kernel(T* __restrict__ phi, int64_t total, int64_t n, int64_t n_pad,
+                                          float inv_sqrt_m, uint32_t k0, uint32_t k1) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int64_t nspans = (total + 4095) >> 12;
+  const T pos = to_storage<T>(inv_sqrt_m), neg = to_storage<T>(-inv_sqrt_m);
+  for (int64_t span = warp; span < nspans; span += nwarps) {
+    const int64_t q = (span << 5) + lane;
+    const U4 u = philox4x32_10(U4{(uint32_t)q, (uint32_t)(q >> 32), 1u, 0u}, k0, k1);
+    int64_t e = (span << 12) + lane * 8;
+    int64_t row = e / n;
+    int64_t j = e - row * n;
+#pragma unroll 4
+    for (int s = 0; s < 16; ++s) {
+      const int src = 2 * s + (lane >> 4);
+      const uint32_t wx = __shfl_sync(0xffffffffu, u.x, src), wy = __shfl_sync(0xffffffffu, u.y, src);
+      const uint32_t wz = __shfl_sync(0xffffffffu, u.z, src), ww = __shfl_sync(0xffffffffu, u.w, src);
+      const int wi = (lane >> 2) & 3;
+      const uint32_t word = wi == 0 ? wx : (wi == 1 ? wy : (wi == 2 ? wz : ww));
+      const uint32_t byte = (word >> ((lane & 3) * 8)) & 0xffu;
+      if (e < total) {                      // total % 8 == 0: all 8 elements exist
+        alignas(16) T v[8];
+#pragma unroll
+        for (int b = 0; b < 8; ++b) v[b] = ((byte >> b) & 1u) ? neg : pos;
+        T* dst = phi + row * n_pad + j;
+        if (sizeof(T) == 2) {
+          *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(v);
+        } else {
+          reinterpret_cast<uint4*>(dst)[0] = reinterpret_cast<const uint4*>(v)[0];
+          reinterpret_cast<uint4*>(dst)[1] = reinterpret_cast<const uint4*>(v)[1];
+        }
+      }
+      e += 256;
+      j += 256;
+      while (j >= n) { j -= n; ++row; }
+    }
+  }
+}
+
 template <typename T>
 __global__ void phi_pack_kernel(T* __restrict__ dst, const T* __restrict__ src, int64_t rows, int64_t n,
                                 int64_t n_pad, bool to_padded) {
@@ -88,6 +163,20 @@ cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   const float inv = (float)(1.0 / sqrt((double)p.m));
   const uint32_t k0 = (uint32_t)(p.seed & 0xFFFFFFFFull), k1 = (uint32_t)(p.seed >> 32);
+  if (p.ensemble == CSAT_ENSEMBLE_RADEMACHER) {
+    const int rb = 256, rg = grid_for((total + 127) / 128, rb);
+    const bool vec = p.n % 8 == 0;
+    if (p.dtype == CSAT_DTYPE_FP32) {
+      if (vec) phi_rademacher_vec_kernel<float><<<rg, rb, 0, s>>>((float*)phi, total, p.n, p.n_pad, inv, k0, k1);
+      else phi_rademacher_kernel<float><<<rg, rb, 0, s>>>((float*)phi, total, p.n, p.n_pad, inv, k0, k1);
+    } else {
+      if (vec)
+        phi_rademacher_vec_kernel<__nv_bfloat16><<<rg, rb, 0, s>>>((__nv_bfloat16*)phi, total, p.n, p.n_pad, inv, k0, k1);
+      else
+        phi_rademacher_kernel<__nv_bfloat16><<<rg, rb, 0, s>>>((__nv_bfloat16*)phi, total, p.n, p.n_pad, inv, k0, k1);
+    }
+    return cudaGetLastError();
+  }
   const int block = 256, grid = grid_for((total + 3) / 4, block);
   if (p.dtype == CSAT_DTYPE_FP32)
     phi_gen_kernel<float><<<grid, block, 0, s>>>((float*)phi, total, p.n, p.n_pad, inv, k0, k1);

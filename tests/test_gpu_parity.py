@@ -270,3 +270,32 @@ def test_supplied_lista_weights_match_oracle(name):
         again = to_np(ctx.forward(Q, K, V))
         assert rel_err(again, base) <= 1e-5
     ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_rademacher_ensemble_is_bit_exact_and_runs(dtype):
+    """Integer work: the library's Rademacher Phi equals the oracle's bit for bit; a forward with it matches
+    the oracle; switching back restores the Gaussian matrix."""
+    for (H, m, n, seed) in [(1, 64, 256, 0), (3, 20, 197, 0xDEADBEEF12345678), (2, 7, 4099, 5), (2, 9, 4104, 6), (5, 33, 1568, 1)]:
+        ctx = binding.Csat(n, m, 8, H, seed, dtype=dtype)
+        gauss = ctx.get_phi().clone()
+        ctx.set(ensemble="rademacher")
+        got = to_np(ctx.get_phi())
+        ref = wl.round_to_storage(pho.phi_rademacher(H, m, n, seed).astype(np.float32), dtype).astype(np.float64)
+        assert np.array_equal(got, ref)
+        ctx.set(ensemble="gaussian")
+        assert torch.equal(ctx.get_phi(), gauss)
+        ctx.close()
+    w = wl.shrink(C["c3"], B=1, H=2, n=784, n_q=300, m=128) if dtype == "bf16" else C["c1"]
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    ctx.set(ensemble="rademacher")
+    phi = to_np(ctx.get_phi())
+    assert np.array_equal(np.abs(phi), np.full_like(phi, np.abs(phi[0, 0, 0])))
+    for T, lam in [(0, 0.0), (w.T, w.lam)]:
+        ctx.set(T=T, lam=lam)
+        out = to_np(ctx.forward(Q, K, V))
+        ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=lam)
+        assert rel_err(out, ref) <= TOL[dtype], (dtype, T)
+    ctx.close()
