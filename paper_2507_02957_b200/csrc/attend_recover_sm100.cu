@@ -4,8 +4,9 @@
 // alpha^{t+1} = eta_theta(S alpha^t + B Z_i) (LISTA recurrence with S = I - mu G, B = mu M); C^_i = Psi alpha^_i.
 // Neither the n_q x m matrix A~ nor any iterate alpha^t leaves the SM.
 //
-// One CTA per SM works on 256 consecutive queries of one (batch, head) as two independent tiles A and B that
-// share the stream of K~|V~ chunks.  While the tensor cores run one tile's MMAs the other tile's threads do
+// One persistent CTA per SM walks work items of 256 consecutive queries of one (batch, head), each as two
+// independent tiles A and B that share the stream of K~|V~ chunks; the TMA and MMA warps run ahead into the
+// next item (its Q tiles, first chunks and first S MMAs) while the compute threads finish the current one.  While the tensor cores run one tile's MMAs the other tile's threads do
 // their softmax / shrinkage arithmetic, and the other way round.
 //
 // CTA = 12 warps in three warpgroups (registers are re-divided between them with setmaxnreg: the two
@@ -81,7 +82,7 @@ template <int D> struct Cfg {
 };
 
 struct Bars {
-  uint64_t q_full[kTiles], mats_full, psi_full;
+  uint64_t q_full[kTiles], q_free[kTiles], mats_full;
   uint64_t k_full[kMaxStages], k_empty[kMaxStages], v_full[kMaxStages], v_empty[kMaxStages];
   uint64_t s_full[kTiles][2], p_full[kTiles][2], zc_full[kTiles];
   uint64_t a_full[kTiles], r_full[kTiles];
@@ -185,7 +186,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
-                            int has_psi, float scale_log2, int* status) {
+                            int has_psi, float scale_log2, int items_x, int n_items, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
@@ -196,9 +197,13 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   uint8_t* ring = smem + C::kOffRing;
   Bars* bars = reinterpret_cast<Bars*>(smem + C::kOffBar);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int row0 = blockIdx.x * (kTiles * kRows), bh = blockIdx.y, h = bh % H;
-  const int ntiles = (nq - row0 > kRows) ? 2 : 1;               // the last CTA of a (batch, head) may hold one tile
+  // Work items: item = bh * items_x + x covers queries [256 x, 256 x + 256) of (batch, head) bh.  The CTA is
+  // persistent: it takes items blockIdx.x, blockIdx.x + gridDim.x, ...  Every role walks the same sequence with
+  // its own free-running counters (ring position, chunks and recovery MMAs per tile), from which the barrier
+  // parities follow, so that the TMA and MMA warps can run ahead into the next item while the compute threads
+  // finish the current one.
   const int nchunks = (m + kMC - 1) / kMC;
+  const int nvirt = T > 0 ? C::kDBoxes : 0;     // ring positions an item's decoder matrices take after its chunks
   Waiter w{status, &bars->abort};
   auto k_slot = [&](int s) { return ring + (2 * s) * C::kSlotBytes; };
   auto v_slot = [&](int s) { return ring + (2 * s + 1) * C::kSlotBytes; };
@@ -208,13 +213,13 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     prefetch_tmap(&tmap_kv);
     prefetch_tmap(&tmap_mats);
     mbar_init(&bars->mats_full, 1);
-    mbar_init(&bars->psi_full, 1);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1);
       mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
     }
     for (int t = 0; t < kTiles; ++t) {
       mbar_init(&bars->q_full[t], 1);
+      mbar_init(&bars->q_free[t], 1);
       for (int s = 0; s < 2; ++s) { mbar_init(&bars->s_full[t][s], 1); mbar_init(&bars->p_full[t][s], kTileThreads); }
       mbar_init(&bars->zc_full[t], 1);
       mbar_init(&bars->a_full[t], kTileThreads);
@@ -237,61 +242,91 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   reg_dealloc<56>();
   if (warp == kTmaWarp) {
     // ------------------------------------------------ TMA producer ------------------------------------------------
+    // Ring position g counts the chunks loaded so far (stage g % kStages, use g / kStages).  After an item's
+    // chunks come nvirt "virtual chunks": the boxes of mu G go to their K~ slots and those of Psi to their V~
+    // slots, under the same full / empty barriers.  B goes to tile A's Q buffer once the item's S MMAs are done.
     if (elect_one()) {
-      int issued_k = 0, issued_v = 0;
-      bool mats_issued = false, psi_issued = false;
-      for (int t = 0; t < ntiles; ++t) {
-        mbar_arrive_expect_tx(&bars->q_full[t], C::kQBytes);
-        for (int g = 0; g < C::kDBoxes; ++g)
-          tma_load_3d(q_buf + t * C::kQBytes + g * kRows * 128, &tmap_q, &bars->q_full[t], g * 64, row0 + t * kRows, bh);
-      }
-      for (int j = 0; j < nchunks; ++j) {
-        const int s = j % C::kStages, use = j / C::kStages;
-        if (use > 0) w.wait(&bars->k_empty[s], (use - 1) & 1, 201);
-        if (w.dead) break;
-        mbar_arrive_expect_tx(&bars->k_full[s], C::kSlotBytes);
-        for (int g = 0; g < C::kDBoxes; ++g)
-          tma_load_3d(k_slot(s) + g * C::kBoxBytes, &tmap_kv, &bars->k_full[s], g * 64, j * kMC, bh);
-        issued_k = j + 1;
-        if (use > 0) w.wait(&bars->v_empty[s], (use - 1) & 1, 202);
-        if (w.dead) break;
-        mbar_arrive_expect_tx(&bars->v_full[s], C::kSlotBytes);
-        for (int g = 0; g < C::kDBoxes; ++g)
-          tma_load_3d(v_slot(s) + g * C::kBoxBytes, &tmap_kv, &bars->v_full[s], D + g * 64, j * kMC, bh);
-        issued_v = j + 1;
-      }
-      if (T > 0) {
-        // every S MMA has finished once the last one has: tile A's Q buffer and the K~ slots are free for B, mu G
-        const int last = nchunks - 1;
-        w.wait(&bars->k_empty[last % C::kStages], (last / C::kStages) & 1, 203);
-        if (!w.dead) {
-          mbar_arrive_expect_tx(&bars->mats_full, 2 * C::kMatBytes);
-          for (int g = 0; g < C::kDBoxes; ++g) {
-            tma_load_3d(k_slot(g), &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 0);                      // mu G
-            tma_load_3d(q_buf + g * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, g * 64, 0, h * 3 + 1);   // B
+      uint32_t g = 0, items_done = 0;
+      uint32_t q_loads[kTiles] = {0, 0};
+      uint64_t k_hist = 0, v_hist = 0;        // bit i: the copy into the K~ / V~ slot of ring position g-1-i was issued
+      uint32_t mats_loads = 0;
+      auto ring_wait_k = [&](uint32_t pos, int code) {
+        if (pos >= (uint32_t)C::kStages) w.wait(&bars->k_empty[pos % C::kStages], (pos / C::kStages - 1) & 1, code);
+      };
+      auto ring_wait_v = [&](uint32_t pos, int code) {
+        if (pos >= (uint32_t)C::kStages) w.wait(&bars->v_empty[pos % C::kStages], (pos / C::kStages - 1) & 1, code);
+      };
+      for (int item = blockIdx.x; item < n_items && !w.dead; item += gridDim.x, ++items_done) {
+        const int bh = item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
+        const int ntiles = (nq - row0 > kRows) ? 2 : 1;
+#pragma unroll
+        for (int t = 0; t < kTiles; ++t) {
+          if (t < ntiles) {
+            if (q_loads[t] > 0) w.wait(&bars->q_free[t], (q_loads[t] - 1) & 1, 205);   // released by the last user
+            if (w.dead) break;
+            mbar_arrive_expect_tx(&bars->q_full[t], C::kQBytes);
+            for (int gx = 0; gx < C::kDBoxes; ++gx)
+              tma_load_3d(q_buf + t * C::kQBytes + gx * kRows * 128, &tmap_q, &bars->q_full[t], gx * 64, row0 + t * kRows, bh);
+            ++q_loads[t];
           }
-          mats_issued = true;
         }
-        if (has_psi) {
-          // Psi goes to the V~ slots once the last P V~ product has read them
-          w.wait(&bars->v_empty[last % C::kStages], (last / C::kStages) & 1, 204);
+        for (int j = 0; j < nchunks && !w.dead; ++j, ++g) {
+          const int s = g % C::kStages;
+          ring_wait_k(g, 201);
+          if (w.dead) break;
+          mbar_arrive_expect_tx(&bars->k_full[s], C::kSlotBytes);
+          for (int gx = 0; gx < C::kDBoxes; ++gx)
+            tma_load_3d(k_slot(s) + gx * C::kBoxBytes, &tmap_kv, &bars->k_full[s], gx * 64, j * kMC, bh);
+          k_hist = (k_hist << 1) | 1u;
+          v_hist <<= 1;
+          ring_wait_v(g, 202);
+          if (w.dead) { ++g; break; }
+          mbar_arrive_expect_tx(&bars->v_full[s], C::kSlotBytes);
+          for (int gx = 0; gx < C::kDBoxes; ++gx)
+            tma_load_3d(v_slot(s) + gx * C::kBoxBytes, &tmap_kv, &bars->v_full[s], D + gx * 64, j * kMC, bh);
+          v_hist |= 1u;
+        }
+        if (T > 0 && !w.dead) {
+          // every S MMA of the item has finished once the last one has: tile A's Q buffer is free for B
+          const uint32_t gl = g - 1;
+          w.wait(&bars->k_empty[gl % C::kStages], (gl / C::kStages) & 1, 203);
           if (!w.dead) {
-            mbar_arrive_expect_tx(&bars->psi_full, C::kMatBytes);
-            for (int g = 0; g < C::kDBoxes; ++g)
-              tma_load_3d(v_slot(g), &tmap_mats, &bars->psi_full, g * 64, 0, h * 3 + 2);
-            psi_issued = true;
+            mbar_arrive_expect_tx(&bars->mats_full, C::kMatBytes);
+            for (int gx = 0; gx < C::kDBoxes; ++gx)
+              tma_load_3d(q_buf + gx * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, gx * 64, 0, h * 3 + 1);
+            ++mats_loads;
+          }
+          for (int gx = 0; gx < C::kDBoxes && !w.dead; ++gx, ++g) {
+            const int s = g % C::kStages;
+            ring_wait_k(g, 206);
+            if (w.dead) break;
+            mbar_arrive_expect_tx(&bars->k_full[s], C::kMatBoxBytes);
+            tma_load_3d(k_slot(s), &tmap_mats, &bars->k_full[s], gx * 64, 0, h * 3 + 0);          // mu G
+            k_hist = (k_hist << 1) | 1u;
+            v_hist <<= 1;
+            ring_wait_v(g, 207);
+            if (w.dead) { ++g; break; }
+            if (has_psi) {
+              mbar_arrive_expect_tx(&bars->v_full[s], C::kMatBoxBytes);
+              tma_load_3d(v_slot(s), &tmap_mats, &bars->v_full[s], gx * 64, 0, h * 3 + 2);        // Psi
+              v_hist |= 1u;
+            } else {
+              mbar_arrive(&bars->v_full[s]);     // nothing to load: complete the phase so that the parities stay in step
+            }
           }
         }
       }
       if (w.dead) {
         // gave up: let the copies that are still in flight land before the CTA's shared memory goes away
-        for (int t = 0; t < ntiles; ++t) mbar_wait_drain(&bars->q_full[t], 0);
-        for (int c = issued_k > C::kStages ? issued_k - C::kStages : 0; c < issued_k; ++c)
-          mbar_wait_drain(&bars->k_full[c % C::kStages], (c / C::kStages) & 1);
-        for (int c = issued_v > C::kStages ? issued_v - C::kStages : 0; c < issued_v; ++c)
-          mbar_wait_drain(&bars->v_full[c % C::kStages], (c / C::kStages) & 1);
-        if (mats_issued) mbar_wait_drain(&bars->mats_full, 0);
-        if (psi_issued) mbar_wait_drain(&bars->psi_full, 0);
+#pragma unroll
+        for (int t = 0; t < kTiles; ++t)
+          if (q_loads[t] > 0) mbar_wait_drain(&bars->q_full[t], (q_loads[t] - 1) & 1);
+        for (uint32_t i = 0; i < (uint32_t)C::kStages && i < g; ++i) {
+          const uint32_t pos = g - 1 - i;
+          if ((k_hist >> i) & 1u) mbar_wait_drain(&bars->k_full[pos % C::kStages], (pos / C::kStages) & 1);
+          if ((v_hist >> i) & 1u) mbar_wait_drain(&bars->v_full[pos % C::kStages], (pos / C::kStages) & 1);
+        }
+        if (mats_loads > 0) mbar_wait_drain(&bars->mats_full, (mats_loads - 1) & 1);
       }
     }
   } else if (warp == kMmaWarp) {
@@ -308,75 +343,110 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       const uint64_t ring_k0 = make_smem_desc(smem_u32(ring), 16, 1024);
       const uint64_t ring_v0 = make_smem_desc(smem_u32(ring + C::kSlotBytes), C::kBoxBytes, 1024);
       constexpr uint64_t kStageStep = (2 * C::kSlotBytes) >> 4;                 // descriptor distance between stages
-      auto issue_pv = [&](int i) {
-        const int s = i % C::kStages, b = i & 1;
-        w.wait(&bars->v_full[s], (i / C::kStages) & 1, 211);
-        const uint64_t b_desc = ring_v0 + (uint64_t)s * kStageStep;
-        const uint32_t acc = (i != 0);
-#pragma unroll
-        for (int t = 0; t < kTiles; ++t) {
-          if (t < ntiles) {
-            w.wait(&bars->p_full[t][b], (i >> 1) & 1, 212);
-            tc_fence_after();
-            const uint32_t tb = tmem + t * C::kTileCols;
-            // P: 8 packed columns per 16 measurements; V~: +16 rows = 2048 B
-            mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC, b_desc, idesc_z, acc);
-#pragma unroll
-            for (int k = 1; k < kMC / 16; ++k)
-              mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC + k * 8, b_desc + (uint64_t)(k * 128), idesc_z, 1u);
-            mma_commit(&bars->zc_full[t]);
-          }
-        }
-        mma_commit(&bars->v_empty[s]);
-      };
-#pragma unroll
-      for (int t = 0; t < kTiles; ++t)
-        if (t < ntiles) w.wait(&bars->q_full[t], 0, 210);
-      for (int j = 0; j < nchunks; ++j) {
-        const int s = j % C::kStages, b = j & 1;
-        w.wait(&bars->k_full[s], (j / C::kStages) & 1, 213);
-        tc_fence_after();
-        const uint64_t kd = ring_k0 + (uint64_t)s * kStageStep;
-#pragma unroll
-        for (int t = 0; t < kTiles; ++t) {
-          if (t < ntiles) {
-            const uint64_t qd = q_desc0 + (uint64_t)(t * (C::kQBytes >> 4));
-            const uint32_t ds = tmem + t * C::kTileCols + C::kColS + b * kMC;
-#pragma unroll
-            for (int k = 0; k < D / 16; ++k)
-              mma_f16_ss(ds, qd + kstep(k, kRows * 128), kd + kstep(k, C::kBoxBytes), idesc_s, k != 0);
-            mma_commit(&bars->s_full[t][b]);
-          }
-        }
-        mma_commit(&bars->k_empty[s]);
-        if (j > 0) issue_pv(j - 1);
-      }
-      issue_pv(nchunks - 1);
-      if (T > 0) {
-        const int n_mma = T + (has_psi ? 1 : 0);    // r_0 = theta + z B, then T-1 increments with mu G, then Psi
-        for (int i = 0; i < n_mma; ++i) {
-          const bool first = (i == 0), psi_step = has_psi && i == n_mma - 1;
-          if (first) w.wait(&bars->mats_full, 0, 214);
-          if (psi_step) w.wait(&bars->psi_full, 0, 215);
-          // B sits in tile A's Q buffer (boxes of d rows), mu G in the K~ slots and Psi in the V~ slots of the
-          // first stages (one box per stage)
-          const uint64_t w0 = first ? q_desc0 : (psi_step ? ring_k0 + (uint64_t)(C::kSlotBytes >> 4) : ring_k0);
-          const uint64_t wbox = first ? (uint64_t)(C::kMatBoxBytes >> 4) : kStageStep;
-          const uint32_t acc0 = psi_step ? 0u : 1u;
+      uint32_t g = 0, items_done = 0;          // ring position of the item's first chunk; items of this CTA so far
+      uint32_t cb[kTiles] = {0, 0};            // chunks of earlier items, per tile (S / P buffer and parities)
+      uint32_t ab[kTiles] = {0, 0};            // recovery MMAs of earlier items, per tile
+      uint32_t q_uses[kTiles] = {0, 0};
+      for (int item = blockIdx.x; item < n_items && !w.dead; item += gridDim.x, ++items_done) {
+        const int row0 = (item % items_x) * (kTiles * kRows);
+        const int ntiles = (nq - row0 > kRows) ? 2 : 1;
+        auto issue_pv = [&](int i) {
+          const uint32_t pos = g + i;
+          const int s = pos % C::kStages;
+          w.wait(&bars->v_full[s], (pos / C::kStages) & 1, 211);
+          const uint64_t b_desc = ring_v0 + (uint64_t)s * kStageStep;
+          const uint32_t acc = (i != 0);
 #pragma unroll
           for (int t = 0; t < kTiles; ++t) {
             if (t < ntiles) {
-              w.wait(&bars->a_full[t], i & 1, 216);
+              const uint32_t c = cb[t] + i;
+              const int b = c & 1;
+              w.wait(&bars->p_full[t][b], (c >> 1) & 1, 212);
               tc_fence_after();
               const uint32_t tb = tmem + t * C::kTileCols;
+              // P: 8 packed columns per 16 measurements; V~: +16 rows = 2048 B
+              mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC, b_desc, idesc_z, acc);
 #pragma unroll
-              for (int k = 0; k < D / 16; ++k)
-                mma_f16_ts(tb + C::kColAcc, tb + C::kColS + k * 8, w0 + (uint64_t)(k / 4) * wbox + (uint64_t)((k % 4) * 2),
-                           idesc_r, k == 0 ? acc0 : 1u);
-              mma_commit(&bars->r_full[t]);
+              for (int k = 1; k < kMC / 16; ++k)
+                mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC + k * 8, b_desc + (uint64_t)(k * 128), idesc_z, 1u);
+              mma_commit(&bars->zc_full[t]);
             }
           }
+          mma_commit(&bars->v_empty[s]);
+        };
+#pragma unroll
+        for (int t = 0; t < kTiles; ++t)
+          if (t < ntiles) { w.wait(&bars->q_full[t], q_uses[t] & 1, 210); ++q_uses[t]; }
+        for (int j = 0; j < nchunks; ++j) {
+          const uint32_t pos = g + j;
+          const int s = pos % C::kStages;
+          w.wait(&bars->k_full[s], (pos / C::kStages) & 1, 213);
+          tc_fence_after();
+          const uint64_t kd = ring_k0 + (uint64_t)s * kStageStep;
+#pragma unroll
+          for (int t = 0; t < kTiles; ++t) {
+            if (t < ntiles) {
+              const int b = (cb[t] + j) & 1;
+              const uint64_t qd = q_desc0 + (uint64_t)(t * (C::kQBytes >> 4));
+              const uint32_t ds = tmem + t * C::kTileCols + C::kColS + b * kMC;
+#pragma unroll
+              for (int k = 0; k < D / 16; ++k)
+                mma_f16_ss(ds, qd + kstep(k, kRows * 128), kd + kstep(k, C::kBoxBytes), idesc_s, k != 0);
+              mma_commit(&bars->s_full[t][b]);
+            }
+          }
+          mma_commit(&bars->k_empty[s]);
+          if (j == nchunks - 1) {
+            // the Q buffers have been read for the last time (tile A's still takes B when there is a recovery)
+            if (ntiles == 2) mma_commit(&bars->q_free[1]);
+            if (T == 0) mma_commit(&bars->q_free[0]);
+          }
+          if (j > 0) issue_pv(j - 1);
         }
+        issue_pv(nchunks - 1);
+        if (T > 0) {
+          const uint32_t gv = g + nchunks;            // ring position of the first box of mu G / Psi
+          const int n_mma = T + (has_psi ? 1 : 0);    // r_0 = theta + z B, then T-1 increments with mu G, then Psi
+          for (int i = 0; i < n_mma; ++i) {
+            const bool first = (i == 0), psi_step = has_psi && i == n_mma - 1;
+            if (first) w.wait(&bars->mats_full, items_done & 1, 214);
+            if (i == 1 || psi_step)
+              for (int gx = 0; gx < C::kDBoxes; ++gx) {
+                const uint32_t pos = gv + gx;
+                w.wait(psi_step ? &bars->v_full[pos % C::kStages] : &bars->k_full[pos % C::kStages],
+                       (pos / C::kStages) & 1, 215);
+              }
+            const uint32_t acc0 = psi_step ? 0u : 1u;
+#pragma unroll
+            for (int t = 0; t < kTiles; ++t) {
+              if (t < ntiles) {
+                w.wait(&bars->a_full[t], (ab[t] + i) & 1, 216);
+                tc_fence_after();
+                const uint32_t tb = tmem + t * C::kTileCols;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                  // B: boxes of d rows in tile A's Q buffer; mu G / Psi: box k / 4 in the K~ / V~ slot of ring
+                  // position gv + k / 4
+                  const uint64_t wd = first ? q_desc0 + (uint64_t)((k / 4) * (C::kMatBoxBytes >> 4))
+                                            : ring_k0 + (uint64_t)((gv + k / 4) % C::kStages) * kStageStep +
+                                                  (psi_step ? (uint64_t)(C::kSlotBytes >> 4) : 0);
+                  mma_f16_ts(tb + C::kColAcc, tb + C::kColS + k * 8, wd + (uint64_t)((k % 4) * 2), idesc_r,
+                             k == 0 ? acc0 : 1u);
+                }
+                mma_commit(&bars->r_full[t]);
+              }
+            }
+            if (first) mma_commit(&bars->q_free[0]);      // B has been read: tile A's Q buffer is free
+          }
+          for (int gx = 0; gx < C::kDBoxes; ++gx) {       // release the ring positions of mu G / Psi
+            mma_commit(&bars->k_empty[(gv + gx) % C::kStages]);
+            mma_commit(&bars->v_empty[(gv + gx) % C::kStages]);
+          }
+        }
+        g += nchunks + nvirt;
+#pragma unroll
+        for (int t = 0; t < kTiles; ++t)
+          if (t < ntiles) { cb[t] += nchunks; ab[t] += T > 0 ? T + (has_psi ? 1 : 0) : 0; }
       }
     }
   }
@@ -384,18 +454,24 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     reg_alloc<224>();
     // ------------------------------------------------ compute threads ---------------------------------------------
     const int t = warp >> 2, wq = warp & 3;                     // tile, lane quarter
-    if (t < ntiles) {
-      const int row = wq * 32 + lane;                           // row of the tile = TMEM lane
-      const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + t * C::kTileCols;
-      const uint32_t acc_addr = tbase + C::kColAcc;
+    const int row = wq * 32 + lane;                             // row of the tile = TMEM lane
+    const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + t * C::kTileCols;
+    const uint32_t acc_addr = tbase + C::kColAcc;
+    const uint64_t sc2 = pack2(scale_log2, scale_log2);
+    uint32_t cb = 0;                                            // chunks of this tile's earlier items
+    uint32_t zc_seen = 0;                                       // phases of zc_full[t] this thread has waited for
+    int phase = 0;                                              // phases of r_full[t] this thread has waited for
+    for (int item = blockIdx.x; item < n_items && !w.dead; item += gridDim.x) {
+      const int bh = item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
+      if (t >= ((nq - row0 > kRows) ? 2 : 1)) continue;         // this item has no second tile
       float ref = -INFINITY;                                    // reference maximum of the row (log2 domain)
       uint64_t sum2 = pack2(0.f, 0.f);                          // running sum of P, two partial sums
-      const uint64_t sc2 = pack2(scale_log2, scale_log2);
-      int zc_seen = 0;                                          // phases of zc_full[t] this thread has waited for
+      const float kappa = T > 0 ? theta[h] : 0.f;               // loaded now, needed after the attention phase
 
       for (int j = 0; j < nchunks; ++j) {
-        const int b = j & 1;
-        w.wait(&bars->s_full[t][b], (j >> 1) & 1, 220);
+        const uint32_t c = cb + j;                              // chunk count of this tile over all its items
+        const int b = c & 1;
+        w.wait(&bars->s_full[t][b], (c >> 1) & 1, 220);
         tc_fence_after();
         uint32_t ra[32], rb[32];                                // columns [0, 32) and [32, 64) of S_j
         tmem_ld_32x32b_x32(tbase + C::kColS + b * kMC, ra);
@@ -428,8 +504,8 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           const bool raise = mx > ref + 8.f;
           if (__any_sync(0xffffffffu, raise)) {
             // rare: rescale this warp's rows of the accumulator (factor 1 for rows that keep their reference)
-            w.wait(&bars->zc_full[t], (j - 1) & 1, 221);        // P_{j-1} V~_{j-1} has been added
-            zc_seen = j;
+            w.wait(&bars->zc_full[t], (c - 1) & 1, 221);        // P_{j-1} V~_{j-1} has been added
+            zc_seen = c;
             tc_fence_after();
             const float f = raise ? ex2(ref - mx) : 1.f;
             if (raise) ref = mx;
@@ -473,9 +549,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         // A parity wait is only safe when the waiter is at most one phase behind, so every phase of zc_full is
         // observed in order: phase j-1 here (it cannot be two ahead, since P_j V~_j needs the arrival below;
         // normally it completed long ago), phase j after the next chunk, the last one after the loop.
-        if (j > 0 && zc_seen < j) {
-          w.wait(&bars->zc_full[t], (j - 1) & 1, 223);
-          zc_seen = j;
+        if (j > 0 && zc_seen < c) {
+          w.wait(&bars->zc_full[t], (c - 1) & 1, 223);
+          zc_seen = c;
         }
         mbar_arrive(&bars->p_full[t][b]);
       }
@@ -485,7 +561,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         unpack2(sum2, s0, s1);
         inv = 1.f / (s0 + s1);
       }
-      w.wait(&bars->zc_full[t], (nchunks - 1) & 1, 222);        // every P V~ product has been added
+      w.wait(&bars->zc_full[t], (cb + nchunks - 1) & 1, 222);   // every P V~ product has been added
+      cb += nchunks;
+      zc_seen = cb;
       tc_fence_after();
       // v2 holds, in turn: Z, b_t = alpha^t - theta, alpha^T, Psi alpha^T  (pairs of adjacent columns)
       uint64_t v2[D / 2];
@@ -521,7 +599,6 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       if (T > 0) {
         // layer t uses theta[t * theta_stride + h] (stride 0: one threshold for all layers).  The accumulator is
         // biased by kappa = theta of layer 0 and the registers hold b = alpha - kappa throughout.
-        const float kappa = theta[h];
         const uint32_t op_addr = tbase + C::kColS;
         // accumulator := kappa (r_0 = kappa + z B), and z as the bf16 A operand
         {
@@ -534,7 +611,6 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         publish();
 #pragma unroll
         for (int i = 0; i < D / 2; ++i) v2[i] = pack2(-kappa, -kappa);  // alpha^0 = 0
-        int phase = 0;
         // per_layer is a compile-time tag: with one threshold for all layers theta_t - kappa = 0 and the add of it
         // is left out of the inner loop
         auto iterate = [&](auto per_layer) {
@@ -649,11 +725,21 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   }
   const double scale = p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)D);
   const float scale_log2 = (float)(scale * 1.4426950408889634);
-  const int64_t rows_per_cta = kTiles * kRows;
-  const dim3 grid((unsigned)((p.nq + rows_per_cta - 1) / rows_per_cta), (unsigned)(p.B * p.H));
+  // persistent CTAs, one per SM, each walking the work items (256 queries of one (batch, head)) it owns
+  const int64_t rows_per_item = kTiles * kRows;
+  const int64_t items_x = (p.nq + rows_per_item - 1) / rows_per_item, n_items = items_x * p.B * p.H;
+  if (n_items > (int64_t)1 << 30) return cudaErrorInvalidValue;
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+      sms = 148;
+  }
+  const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
   attend_recover_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(
       tq, c->tmap_kv, c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, p.T,
-      c->psi ? 1 : 0, scale_log2, c->status);
+      c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, c->status);
   return cudaGetLastError();
 }
 
