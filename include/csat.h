@@ -217,6 +217,17 @@ int csat_attend_noalloc(const void* Q, const void* K, const void* V, const void*
                         int64_t H, int64_t n, int64_t n_q, int64_t m, int64_t d, int dtype, double scale,
                         void* stream, char* err_host, size_t err_cap);
 
+/* csat_selftest_wait_timeout / csat_clear_status -- failure-detection aids, no counterpart in the paper.
+ * Every device-side wait of this library is bounded; when one gives up, the kernel records a code in the
+ * context's status word and returns, and host calls report CSAT_ERR_TIMEOUT from then on.
+ * csat_selftest_wait_timeout launches a one-thread kernel that waits `limit_us` microseconds (1 .. 1000000) on a
+ * barrier nothing arrives at, synchronises `stream` and returns CSAT_ERR_TIMEOUT if (as it must) the wait gave
+ * up and the status word was set, CSAT_ERR_STATE if it was not.  The context stays usable for queries; its
+ * csat_forward calls return CSAT_ERR_TIMEOUT until csat_clear_status, which synchronises the device, resets the
+ * status word and returns the code it held (0 = none). */
+int csat_selftest_wait_timeout(csat_ctx* ctx, int64_t limit_us, void* stream);
+int csat_clear_status(csat_ctx* ctx, int* code_host);
+
 /* Bytes of device memory the context currently owns (Phi, workspace, decoder matrices, staging). */
 size_t csat_workspace_bytes(const csat_ctx* ctx);
 

@@ -45,6 +45,8 @@ SIGNATURES = {
     "csat_get_profile": (_int, [_vp, _i64, _int, C.POINTER(_int), C.POINTER(C.c_float), C.POINTER(_int)]),
     "csat_attend_noalloc": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _i64, _i64, _int, _dbl, _vp,
                                    C.c_char_p, C.c_size_t]),
+    "csat_selftest_wait_timeout": (_int, [_vp, _i64, _vp]),
+    "csat_clear_status": (_int, [_vp, C.POINTER(_int)]),
     "csat_workspace_bytes": (C.c_size_t, [_vp]),
     "csat_last_launch_count": (_int, [_vp]),
     "csat_last_error": (C.c_char_p, [_vp]),
@@ -192,6 +194,17 @@ def csat_attend_noalloc(Q, K, V, phi, out, scale=0.0, stream=None):
     if rc != CSAT_OK:
         raise CsatError(rc, err.value.decode())
     return out
+
+
+def csat_selftest_wait_timeout(h, limit_us, stream=None) -> int:
+    """Returns the status code (CSAT_ERR_TIMEOUT = 7 when the bounded wait reported its time-out as it must)."""
+    return load().csat_selftest_wait_timeout(h, int(limit_us), _stream(stream))
+
+
+def csat_clear_status(h) -> int:
+    code = _int()
+    _check(h, load().csat_clear_status(h, C.byref(code)))
+    return code.value
 
 
 def csat_workspace_bytes(h) -> int:

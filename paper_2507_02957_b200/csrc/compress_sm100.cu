@@ -152,6 +152,19 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
   if (warp == 1) tmem_dealloc(tmem_base, C::kN);
 }
 
+// Self-test of the bounded wait: one thread waits on a barrier that nothing arrives at.  The wait gives up after
+// limit_ns, writes code 999 into the status word and the kernel returns normally (no trap, no endless loop).
+__global__ void wait_timeout_selftest_kernel(int* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int cta_abort;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    cta_abort = 0;
+    fence_mbar_init();
+    mbar_wait(&bar, 0, status, 999, &cta_abort, limit_ns);
+  }
+}
+
 template <int D>
 cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
   using C = Cfg<D>;
@@ -176,6 +189,11 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
 }
 
 }  // namespace
+
+cudaError_t launch_wait_timeout_selftest(csat_ctx* c, unsigned long long limit_ns, cudaStream_t s) {
+  wait_timeout_selftest_kernel<<<1, 32, 0, s>>>(c->status, limit_ns);
+  return cudaGetLastError();
+}
 
 cudaError_t make_phi_tmap(csat_ctx* c) {
   const Params& p = c->p;

@@ -548,6 +548,28 @@ int csat_get_profile(const csat_ctx* c, int64_t call_index, int cap, int* ids, f
   return CSAT_OK;
 }
 
+int csat_selftest_wait_timeout(csat_ctx* c, int64_t limit_us, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (limit_us < 1 || limit_us > 1000000) return fail(c, CSAT_ERR_INVALID_ARG, "csat_selftest_wait_timeout: limit_us must be in [1, 1000000]");
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = csat::launch_wait_timeout_selftest(c, (unsigned long long)limit_us * 1000ull, s);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_selftest_wait_timeout");
+  if (*(volatile int*)c->status == 0) return fail(c, CSAT_ERR_STATE, "the bounded wait did not report its time-out");
+  return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait gave up (self-test)");
+}
+
+int csat_clear_status(csat_ctx* c, int* code_host) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  if (code_host) *code_host = *(volatile int*)c->status;
+  *(volatile int*)c->status = 0;
+  c->err.clear();
+  return CSAT_OK;
+}
+
 size_t csat_workspace_bytes(const csat_ctx* c) { return c ? c->bytes : 0; }
 
 int csat_last_launch_count(const csat_ctx* c) { return c ? c->last_launches : 0; }

@@ -101,6 +101,7 @@ cudaError_t launch_simt_attend_recover(csat_ctx* c, const void* Q, void* out, cu
 
 // compress_sm100.cu : tcgen05 / TMEM / TMA compression (bf16, d in {64, 128})
 cudaError_t make_phi_tmap(csat_ctx* c);
+cudaError_t launch_wait_timeout_selftest(csat_ctx* c, unsigned long long limit_ns, cudaStream_t s);
 cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches);
 
 // attend_recover_sm100.cu : tcgen05 compressed attention + recovery (bf16, d in {64, 128})

@@ -56,14 +56,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  On time-out writes (code) into *status (if still 0; status may live in host-mapped
 // memory, so it is only touched on failure), raises the CTA's shared-memory abort flag and returns false.
 // Waits of the same CTA that are still spinning see the flag and give up as well.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code, int* cta_abort) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status, int code, int* cta_abort,
+                                          unsigned long long limit_ns = kWaitTimeoutNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 0x3ff) == 0) {
       if (*(volatile int*)cta_abort != 0) return false;        // somebody in this CTA already gave up
-      if (globaltimer() - t0 > kWaitTimeoutNs) {
+      if (globaltimer() - t0 > limit_ns) {
         *(volatile int*)cta_abort = 1;
         atomicCAS(status, 0, code);
         return false;

@@ -299,3 +299,22 @@ def test_rademacher_ensemble_is_bit_exact_and_runs(dtype):
         ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=lam)
         assert rel_err(out, ref) <= TOL[dtype], (dtype, T)
     ctx.close()
+
+
+def test_bounded_wait_reports_a_timeout_and_the_context_recovers():
+    """A wait that can never complete (nothing arrives at its barrier) gives up after its limit, the status
+    word turns every later forward into CSAT_ERR_TIMEOUT, and clearing it restores the context."""
+    w = wl.shrink(C["c2"], B=1, H=2)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w, lam=0.0)
+    good = ctx.forward(Q, K, V).clone()
+    assert binding.csat_selftest_wait_timeout(ctx.h, 1000) == 7          # 1 ms limit
+    assert "gave up" in binding.csat_last_error(ctx.h)
+    with pytest.raises(binding.CsatError) as ei:
+        ctx.forward(Q, K, V)
+    assert ei.value.code == 7
+    assert binding.csat_clear_status(ctx.h) == 999                        # the self-test's code
+    assert binding.csat_clear_status(ctx.h) == 0
+    assert torch.equal(ctx.forward(Q, K, V), good)
+    ctx.close()
