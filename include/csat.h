@@ -65,7 +65,10 @@ enum {
                           the attention/recovery stage; 0 (default) = tensor-core kernels */
   CSAT_ENSEMBLE = 7,   /* measurement ensemble: CSAT_ENSEMBLE_GAUSSIAN (default), N(0, 1/m) entries, or
                           CSAT_ENSEMBLE_RADEMACHER, +-1/sqrt(m) entries (paper: "random Gaussian,
-                          Rademacher, ...").  Changing it regenerates Phi from the seed           */
+                          Rademacher, or structured Hadamard matrices"), or CSAT_ENSEMBLE_HADAMARD:
+                          m rows (a r + b mod N, a odd) of the N x N Sylvester-Hadamard matrix, N the
+                          smallest power of two >= n, columns truncated to n, a random sign per
+                          column, scaled by 1/sqrt(m).  Changing it regenerates Phi from the seed  */
   CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls
                           (0 = off, default; at most 4096).  Setting it creates/destroys
                           events, so set it outside the timed region                    */
@@ -79,7 +82,7 @@ enum {
   CSAT_KERNEL_SPLIT_REDUCE = 3   /* fixed-order sum of token-axis partial K~|V~ tiles    */
 };
 enum { CSAT_DTYPE_BF16 = 0, CSAT_DTYPE_FP32 = 1 };
-enum { CSAT_ENSEMBLE_GAUSSIAN = 0, CSAT_ENSEMBLE_RADEMACHER = 1 };
+enum { CSAT_ENSEMBLE_GAUSSIAN = 0, CSAT_ENSEMBLE_RADEMACHER = 1, CSAT_ENSEMBLE_HADAMARD = 2 };
 
 /* keys of csat_set_f64 / csat_get_f64 */
 enum {

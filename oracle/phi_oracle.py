@@ -106,3 +106,46 @@ def phi_rademacher(H: int, m: int, n: int, seed: int, heads=None) -> np.ndarray:
         bit = (word >> (e & np.uint64(31))) & np.uint64(1)
         out[i] = ((1.0 - 2.0 * bit.astype(np.float64)) / np.sqrt(np.float64(m))).reshape(m, n)
     return out
+
+
+def hadamard_rows(H: int, m: int, n: int, seed: int):
+    """Row indices i_r of the subsampled Hadamard ensemble: N = smallest power of two >= n; for head h,
+    i_r = (a r + b) mod N with a = 2 u0 + 1 (odd, so r -> i_r is injective for r < N) and b = u1, where u0, u1
+    are the first two words of the Philox block with counter (h, 0, 3, 0).  Returns (N, rows [H, m])."""
+    N = 1
+    while N < n:
+        N *= 2
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    rows = np.empty((H, m), dtype=np.int64)
+    for h in range(H):
+        u0, u1, _, _ = philox4x32_10(h, 0, 3, 0, seed & 0xFFFFFFFF, seed >> 32)
+        a, b = 2 * int(u0) + 1, int(u1)
+        rows[h] = [(a * r + b) % N for r in range(m)]
+    return N, rows
+
+
+def phi_hadamard(H: int, m: int, n: int, seed: int, heads=None) -> np.ndarray:
+    """Structured Hadamard ensemble (the paper's third example): m rows of the N x N Sylvester-Hadamard matrix
+    W (W[i,j] = (-1)^popcount(i & j)), columns truncated to n, with a random sign per column:
+        Phi[h,r,j] = s[h,j] * W[i_r, j] / sqrt(m),   float64 (unrounded),
+    rows i_r from hadamard_rows, column signs s[h,j] = -1 where bit e % 32 of word (e // 32) % 4 of the Philox
+    block with counter (e // 128, 0, 2, 0) is set, e = h*n + j.  Needs m <= N."""
+    heads = range(H) if heads is None else heads
+    seed = int(seed) & 0xFFFFFFFFFFFFFFFF
+    N, rows = hadamard_rows(H, m, n, seed)
+    assert m <= N
+    out = np.empty((len(heads), m, n), dtype=np.float64)
+    j = np.arange(n, dtype=np.uint64)
+    for i, h in enumerate(heads):
+        e = np.uint64(h) * np.uint64(n) + j
+        q = e >> np.uint64(7)
+        words = np.stack(philox4x32_10(q & _MASK, q >> _S32, 2, 0, seed & 0xFFFFFFFF, seed >> 32), axis=-1)
+        word = np.take_along_axis(words, ((e >> np.uint64(5)) & np.uint64(3)).astype(np.int64)[:, None], axis=-1)[:, 0]
+        s = 1.0 - 2.0 * ((word >> (e & np.uint64(31))) & np.uint64(1)).astype(np.float64)
+        for r in range(m):
+            x = np.uint64(rows[h, r]) & j
+            par = np.zeros(n, dtype=np.uint64)
+            for sh in range(40):                                    # parity of popcount, bit by bit
+                par ^= (x >> np.uint64(sh)) & np.uint64(1)
+            out[i, r] = s * (1.0 - 2.0 * par.astype(np.float64)) / np.sqrt(np.float64(m))
+    return out

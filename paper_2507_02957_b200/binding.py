@@ -17,7 +17,7 @@ CSAT_OK = 0
 ERR_NAMES = {1: "CSAT_ERR_INVALID_ARG", 2: "CSAT_ERR_SHAPE", 3: "CSAT_ERR_ALLOC", 4: "CSAT_ERR_CUDA",
              5: "CSAT_ERR_UNSUPPORTED", 6: "CSAT_ERR_STATE", 7: "CSAT_ERR_TIMEOUT"}
 CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE, CSAT_ENSEMBLE = 1, 2, 3, 4, 5, 6, 7
-CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER = 0, 1
+CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER, CSAT_ENSEMBLE_HADAMARD = 0, 1, 2
 KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover", 3: "split_reduce"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1
 CSAT_LAMBDA, CSAT_STEP, CSAT_SCALE = 1, 2, 3
@@ -257,7 +257,7 @@ class Csat:
 
     def set(self, *, T=None, lam=None, step=None, scale=None, force_simt=None, ensemble=None):
         if ensemble is not None:
-            csat_set_i64(self.h, CSAT_ENSEMBLE, {"gaussian": 0, "rademacher": 1}[ensemble])
+            csat_set_i64(self.h, CSAT_ENSEMBLE, {"gaussian": 0, "rademacher": 1, "hadamard": 2}[ensemble])
         if T is not None:
             csat_set_i64(self.h, CSAT_T, T)
         if lam is not None:

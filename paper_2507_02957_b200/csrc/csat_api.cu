@@ -246,7 +246,7 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       return allocate_and_generate(c);   // user-set Phi, Psi, D are dropped with the old dtype
     }
     case CSAT_ENSEMBLE: {
-      if (v != CSAT_ENSEMBLE_GAUSSIAN && v != CSAT_ENSEMBLE_RADEMACHER)
+      if (v != CSAT_ENSEMBLE_GAUSSIAN && v != CSAT_ENSEMBLE_RADEMACHER && v != CSAT_ENSEMBLE_HADAMARD)
         return fail(c, CSAT_ERR_INVALID_ARG, "unknown CSAT_ENSEMBLE");
       if ((int)v == p.ensemble) return CSAT_OK;
       cudaDeviceSynchronize();

@@ -136,6 +136,42 @@ __global__ void phi_rademacher_vec_kernel(T* __restrict__ phi, int64_t total, in
   }
 }
 
+// Structured Hadamard ensemble: Phi[h,r,j] = s[h,j] (-1)^popcount(i_r & j) / sqrt(m), i_r = (a r + b) mod N with
+// a = 2 u0 + 1, b = u1 from the Philox block (h, 0, 3, 0); column sign s[h,j] from bit e % 32 of word (e / 32) % 4 of
+// block (e / 128, 0, 2, 0), e = h n + j.  One thread per V consecutive columns of one row (V = 8 when n % 8 == 0:
+// the eight sign bits are one byte of one word, and the store is one 16-byte vector for bf16).
+template <typename T, int V>
+__global__ void phi_hadamard_kernel(T* __restrict__ phi, int64_t n, int64_t n_pad, int64_t m, uint32_t log2N,
+                                    float inv_sqrt_m, uint32_t k0, uint32_t k1) {
+  const int64_t row = blockIdx.y;                        // h * m + r
+  const int64_t h = row / m, r = row - h * m;
+  const int64_t j0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * V;
+  if (j0 >= n) return;
+  const U4 ab = philox4x32_10(U4{(uint32_t)h, 0u, 3u, 0u}, k0, k1);
+  const uint64_t a = 2ull * ab.x + 1ull, b = ab.y;
+  const uint32_t ir = (uint32_t)((a * (uint64_t)r + b) & ((1ull << log2N) - 1ull));
+  const int64_t e0 = h * n + j0;
+  const U4 u = philox4x32_10(U4{(uint32_t)(e0 >> 7), (uint32_t)(e0 >> 39), 2u, 0u}, k0, k1);
+  const uint32_t wi = (uint32_t)(e0 >> 5) & 3u;
+  const uint32_t word = wi == 0 ? u.x : (wi == 1 ? u.y : (wi == 2 ? u.z : u.w));
+  const T pos = to_storage<T>(inv_sqrt_m), neg = to_storage<T>(-inv_sqrt_m);
+  alignas(16) T v[V];
+#pragma unroll
+  for (int i = 0; i < V; ++i) {
+    const uint32_t sbit = (word >> (((uint32_t)e0 & 31u) + i)) & 1u;          // V = 8: e0 % 8 == 0, the bits share a byte
+    const uint32_t par = __popc(ir & (uint32_t)(j0 + i)) & 1u;
+    v[i] = (sbit ^ par) ? neg : pos;
+  }
+  T* dst = phi + row * n_pad + j0;
+  if (V == 8) {
+    const uint4* src = reinterpret_cast<const uint4*>(v);
+    reinterpret_cast<uint4*>(dst)[0] = src[0];
+    if (sizeof(T) == 4) reinterpret_cast<uint4*>(dst)[1] = src[1];
+  } else {
+    dst[0] = v[0];
+  }
+}
+
 template <typename T>
 __global__ void phi_pack_kernel(T* __restrict__ dst, const T* __restrict__ src, int64_t rows, int64_t n,
                                 int64_t n_pad, bool to_padded) {
@@ -163,6 +199,20 @@ cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   const float inv = (float)(1.0 / sqrt((double)p.m));
   const uint32_t k0 = (uint32_t)(p.seed & 0xFFFFFFFFull), k1 = (uint32_t)(p.seed >> 32);
+  if (p.ensemble == CSAT_ENSEMBLE_HADAMARD) {
+    uint32_t log2N = 0;
+    while (((int64_t)1 << log2N) < p.n) ++log2N;
+    const int64_t rows = p.H * p.m;
+    if (rows > 65535) return cudaErrorInvalidValue;      // one grid row per row of Phi
+    const bool vec = p.n % 8 == 0;
+    const int64_t per_row = vec ? p.n / 8 : p.n;
+    const dim3 grid((unsigned)((per_row + 127) / 128), (unsigned)rows);
+#define CSAT_HAD(T, V) phi_hadamard_kernel<T, V><<<grid, 128, 0, s>>>((T*)phi, p.n, p.n_pad, p.m, log2N, inv, k0, k1)
+    if (p.dtype == CSAT_DTYPE_FP32) { if (vec) CSAT_HAD(float, 8); else CSAT_HAD(float, 1); }
+    else { if (vec) CSAT_HAD(__nv_bfloat16, 8); else CSAT_HAD(__nv_bfloat16, 1); }
+#undef CSAT_HAD
+    return cudaGetLastError();
+  }
   if (p.ensemble == CSAT_ENSEMBLE_RADEMACHER) {
     const int rb = 256, rg = grid_for((total + 127) / 128, rb);
     const bool vec = p.n % 8 == 0;

@@ -318,3 +318,26 @@ def test_bounded_wait_reports_a_timeout_and_the_context_recovers():
     assert binding.csat_clear_status(ctx.h) == 0
     assert torch.equal(ctx.forward(Q, K, V), good)
     ctx.close()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_hadamard_ensemble_is_bit_exact_and_runs(dtype):
+    for (H, m, n, seed) in [(1, 64, 256, 0), (3, 20, 197, 0xDEADBEEF12345678), (2, 9, 4104, 6), (4, 33, 1568, 1)]:
+        ctx = binding.Csat(n, m, 8, H, seed, dtype=dtype)
+        ctx.set(ensemble="hadamard")
+        got = to_np(ctx.get_phi())
+        ref = wl.round_to_storage(pho.phi_hadamard(H, m, n, seed).astype(np.float32), dtype).astype(np.float64)
+        assert np.array_equal(got, ref), (H, m, n)
+        ctx.close()
+    w = wl.shrink(C["c3"], B=1, H=2, n=784, n_q=300, m=128) if dtype == "bf16" else C["c1"]
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    ctx.set(ensemble="hadamard")
+    phi = to_np(ctx.get_phi())
+    for T, lam in [(0, 0.0), (w.T, w.lam)]:
+        ctx.set(T=T, lam=lam)
+        out = to_np(ctx.forward(Q, K, V))
+        ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=lam)
+        assert rel_err(out, ref) <= TOL[dtype], (dtype, T)
+    ctx.close()

@@ -489,3 +489,29 @@ def test_rademacher_is_a_sign_matrix_with_unit_columns():
     assert not np.array_equal(P, phi.phi_rademacher(H, m, n, 8))
     # and not the Gaussian ensemble's sign pattern
     assert not np.array_equal(np.sign(P), np.sign(phi.phi_gaussian(H, m, n, 7)))
+
+
+# ---------------------------------------------------------------------------------------------------
+# Structured Hadamard measurement matrices
+# ---------------------------------------------------------------------------------------------------
+def test_hadamard_ensemble_against_the_library_hadamard_matrix():
+    from scipy.linalg import hadamard
+    H, m, n, seed = 2, 24, 64, 11
+    P = phi.phi_hadamard(H, m, n, seed)
+    N, rows = phi.hadamard_rows(H, m, n, seed)
+    assert N == 64 and all(len(set(rows[h])) == m for h in range(H))      # distinct rows
+    W = hadamard(N).astype(np.float64)
+    for h in range(H):
+        signs = P[h, 0] * math.sqrt(m) * W[rows[h, 0]]                     # recovers the column signs from row 0
+        assert np.array_equal(np.abs(signs), np.ones(n))
+        assert np.array_equal(P[h], W[rows[h]] * signs[None, :] / math.sqrt(m))
+        assert np.allclose(P[h] @ P[h].T, np.eye(m) * n / m, atol=1e-12)  # orthogonal rows when n is a power of two
+        assert abs(signs.sum()) < n                                        # not all the same sign
+    assert not np.array_equal(rows[0], rows[1])
+    # truncated columns (n not a power of two): still a sign matrix with unit columns, rows of the 256 x 256 matrix
+    P = phi.phi_hadamard(1, 16, 197, 3)
+    N, rows = phi.hadamard_rows(1, 16, 197, 3)
+    assert N == 256 and np.array_equal(np.abs(P), np.full_like(P, 0.25))
+    W = hadamard(256).astype(np.float64)
+    G = (P[0] * 4.0) * W[rows[0]][:, :197]                                 # = column signs in every row
+    assert np.array_equal(G, np.tile(G[:1], (16, 1)))
