@@ -257,11 +257,12 @@ def run_csat(args, w: wl.Workload) -> dict:
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the CSAT library has no CPU path")
     torch.cuda.set_device(local)
-    if world > 1:
+    under_torchrun = "RANK" in os.environ and "MASTER_ADDR" in os.environ
+    if world > 1 or under_torchrun:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     def barrier():
-        if world > 1:
+        if dist.is_initialized():
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -362,7 +363,7 @@ def run_csat(args, w: wl.Workload) -> dict:
                 "value": oracle_tokens_per_s(w, sec, len(pairs)), "unit": UNIT, "cores": blas_threads(),
                 "kind": "oracle", "seconds": sec,
                 "sample": f"{len(pairs)} of {w.B * w.H} (batch, head) pairs in full, scaled to the whole job"}
-    if world > 1:
+    if dist.is_initialized():
         dist.barrier()
         dist.destroy_process_group()
     return result if rank == 0 else {}
