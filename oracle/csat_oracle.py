@@ -152,14 +152,17 @@ def default_decoder_matrix(Phi_h: np.ndarray, d: int) -> np.ndarray:
 # the whole forward
 # ----------------------------------------------------------------------------
 def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, scale=None,
-                      stages: dict | None = None, weights=None) -> np.ndarray:
+                      stages: dict | None = None, weights=None, Phi_v_h=None) -> np.ndarray:
     """CSAT forward for one (batch, head).  Q [n_q,d], K,V [n,d], Phi_h [m,n] -> [n_q,d].
+    Phi_v_h: separate measurement matrix for the values (the paper's Phi_V; Phi_h is then Phi_K).  The decoder's
+    default D is taken from Phi_V ("Phi = Phi_V is reused as the measurement matrix for decoding").
     weights = (S [d,d], B [d,d], thetas [T]) replaces the ISTA-derived decoder by supplied LISTA weights
     (lam, D and step are then unused)."""
     Q = np.asarray(Q, F64)
     d = Q.shape[1]
+    Phi_v = Phi_h if Phi_v_h is None else Phi_v_h
     Kt = compress(Phi_h, K)
-    Vt = compress(Phi_h, V)
+    Vt = compress(Phi_v, V)
     S = compressed_scores(Q, Kt, scale)
     A = softmax_rows(S)
     Z = compressed_output(A, Vt)
@@ -175,7 +178,7 @@ def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, sc
             stages.update(alpha=alpha)
         return reconstruct(alpha, Psi)
     if D is None:
-        D = default_decoder_matrix(Phi_h, d)
+        D = default_decoder_matrix(Phi_v, d)
     D = np.asarray(D, F64)
     M = D if Psi is None else D @ np.asarray(Psi, F64)
     S_dec, B_dec, theta, mu = decoder_setup(M, lam, step)
@@ -186,7 +189,7 @@ def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, sc
 
 
 def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=None,
-                 stages: list | None = None, weights=None) -> np.ndarray:
+                 stages: list | None = None, weights=None, Phi_V=None) -> np.ndarray:
     """CSAT forward.  Q [B,H,n_q,d], K,V [B,H,n,d], Phi [H,m,n] (one per head, shared over the
     batch, Phi_K = Phi_V), Psi None | [d,d] | [H,d,d], D None | [H,d,d]  ->  out [B,H,n_q,d]."""
     Q = np.asarray(Q)
@@ -200,7 +203,8 @@ def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=Non
             # weights = (S [H,d,d], B [H,d,d], thetas [T,H])
             w_h = None if weights is None else (weights[0][h], weights[1][h], [th[h] for th in weights[2]])
             out[b, h] = csat_forward_head(Q[b, h], K[b, h], V[b, h], Phi[h], T=T, lam=lam,
-                                          Psi=psi_h, D=D_h, step=step, scale=scale, stages=st, weights=w_h)
+                                          Psi=psi_h, D=D_h, step=step, scale=scale, stages=st, weights=w_h,
+                                          Phi_v_h=None if Phi_V is None else Phi_V[h])
             if stages is not None:
                 stages.append(st)
     return out

@@ -515,3 +515,30 @@ def test_hadamard_ensemble_against_the_library_hadamard_matrix():
     W = hadamard(256).astype(np.float64)
     G = (P[0] * 4.0) * W[rows[0]][:, :197]                                 # = column signs in every row
     assert np.array_equal(G, np.tile(G[:1], (16, 1)))
+
+
+# ---------------------------------------------------------------------------------------------------
+# Separate measurement matrices for keys and values (paper: K~ = Phi_K K, V~ = Phi_V V)
+# ---------------------------------------------------------------------------------------------------
+def test_separate_value_matrix():
+    w = wl.shrink(wl.CONFIGS["c1"], n=40, n_q=6, m=12, d=8)
+    inp = wl.make_inputs(w)
+    both = phi.phi_gaussian(2, w.m, w.n, 5)
+    Pk, Pv = both[:1], both[1:]
+    # the same matrix passed twice is the shared-matrix forward
+    a = orc.csat_forward(inp["Q"], inp["K"], inp["V"], Pk, T=3, lam=0.01)
+    b = orc.csat_forward(inp["Q"], inp["K"], inp["V"], Pk, T=3, lam=0.01, Phi_V=Pk)
+    assert np.array_equal(a, b)
+    # different matrices: scores from Phi_K K, values from Phi_V V, by hand
+    st = []
+    out = orc.csat_forward(inp["Q"], inp["K"], inp["V"], Pk, T=0, lam=0.0, Phi_V=Pv, stages=st)
+    Q, K, V = (inp[k][0, 0].astype(np.float64) for k in "QKV")
+    S = Q @ (Pk[0] @ K).T / math.sqrt(w.d)
+    A = np.exp(S - S.max(axis=1, keepdims=True)); A /= A.sum(axis=1, keepdims=True)
+    assert np.allclose(out[0, 0], A @ (Pv[0] @ V), atol=1e-13)
+    assert not np.allclose(out, orc.csat_forward(inp["Q"], inp["K"], inp["V"], Pv, T=0, lam=0.0, Phi_V=Pk))
+    # the decoder's default matrix is the block of Phi_V
+    st = []
+    orc.csat_forward(inp["Q"], inp["K"], inp["V"], Pk, T=2, lam=0.01, Phi_V=Pv, stages=st)
+    S_ref, B_ref, th_ref, mu_ref = orc.decoder_setup(Pv[0][:w.d, :w.d], 0.01)
+    assert np.array_equal(st[0]["B_dec"], B_ref) and st[0]["theta"] == th_ref
