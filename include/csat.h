@@ -69,6 +69,11 @@ enum {
                           m rows (a r + b mod N, a odd) of the N x N Sylvester-Hadamard matrix, N the
                           smallest power of two >= n, columns truncated to n, a random sign per
                           column, scaled by 1/sqrt(m).  Changing it regenerates Phi from the seed  */
+  CSAT_SEPARATE_PHI = 8, /* 0 (default): one matrix per head, Phi_K = Phi_V.  1: separate Phi_K and Phi_V per head
+                          (paper: K~ = Phi_K K, V~ = Phi_V V); Phi_V of head h is drawn as head H + h of the
+                          same seeded generator, the decoder's default D is the block of Phi_V, and
+                          csat_set_phi / csat_get_phi then move [2H, m, n]: the H matrices Phi_K, then the H
+                          matrices Phi_V.  Changing it regenerates both from the seed                 */
   CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls
                           (0 = off, default; at most 4096).  Setting it creates/destroys
                           events, so set it outside the timed region                    */

@@ -16,7 +16,7 @@ from . import build as _build
 CSAT_OK = 0
 ERR_NAMES = {1: "CSAT_ERR_INVALID_ARG", 2: "CSAT_ERR_SHAPE", 3: "CSAT_ERR_ALLOC", 4: "CSAT_ERR_CUDA",
              5: "CSAT_ERR_UNSUPPORTED", 6: "CSAT_ERR_STATE", 7: "CSAT_ERR_TIMEOUT"}
-CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE, CSAT_ENSEMBLE = 1, 2, 3, 4, 5, 6, 7
+CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE, CSAT_ENSEMBLE, CSAT_SEPARATE_PHI = 1, 2, 3, 4, 5, 6, 7, 8
 CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER, CSAT_ENSEMBLE_HADAMARD = 0, 1, 2
 KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover", 3: "split_reduce"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1
@@ -255,7 +255,10 @@ class Csat:
         except Exception:
             pass
 
-    def set(self, *, T=None, lam=None, step=None, scale=None, force_simt=None, ensemble=None):
+    def set(self, *, T=None, lam=None, step=None, scale=None, force_simt=None, ensemble=None, separate_phi=None):
+        if separate_phi is not None:
+            csat_set_i64(self.h, CSAT_SEPARATE_PHI, int(bool(separate_phi)))
+            self.phi_heads = self.H * (2 if separate_phi else 1)
         if ensemble is not None:
             csat_set_i64(self.h, CSAT_ENSEMBLE, {"gaussian": 0, "rademacher": 1, "hadamard": 2}[ensemble])
         if T is not None:
@@ -288,12 +291,12 @@ class Csat:
         return outh
 
     def get_phi(self):
-        phi = self._new(self.H, self.m, self.n)
+        phi = self._new(getattr(self, "phi_heads", self.H), self.m, self.n)
         csat_get_phi(self.h, phi)
         return phi
 
     def set_phi(self, phi):
-        assert phi.shape == (self.H, self.m, self.n) and phi.dtype == self.torch_dtype
+        assert phi.shape == (getattr(self, "phi_heads", self.H), self.m, self.n) and phi.dtype == self.torch_dtype
         csat_set_phi(self.h, phi.contiguous())
 
     def set_dictionary(self, psi):

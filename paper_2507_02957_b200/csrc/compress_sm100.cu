@@ -26,24 +26,27 @@ constexpr int kThreads = 192;
 constexpr uint32_t kABytes = kTileM * kChunk * 2;     // 16 KB
 constexpr uint32_t kBoxBytes = 64 * kChunk * 2;       // 8 KB: 64 columns x 64 tokens
 
-template <int D> struct Cfg {
+// SEP: separate measurement matrices for keys and values (a second A tile per stage, Phi_V, which multiplies the
+// V columns; the K columns keep Phi_K)
+template <int D, bool SEP> struct Cfg {
   static constexpr int kN = 2 * D;                    // accumulator columns
   static constexpr int kBoxes = kN / 64;              // B boxes per stage
-  static constexpr int kStages = (D == 64) ? 6 : 4;
-  static constexpr uint32_t kStageBytes = kABytes + kBoxes * kBoxBytes;
+  static constexpr int kATiles = SEP ? 2 : 1;
+  static constexpr int kStages = (D == 64) ? (SEP ? 4 : 6) : (SEP ? 3 : 4);
+  static constexpr uint32_t kStageBytes = kATiles * kABytes + kBoxes * kBoxBytes;
   static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <int D>
+template <int D, bool SEP>
 __global__ void __launch_bounds__(kThreads, 1)
 compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, __nv_bfloat16* __restrict__ kv, int m, int n, int H,
                       int B, int* status) {
-  using C = Cfg<D>;
+  using C = Cfg<D, SEP>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* a_buf = smem;                                      // [stages][16 KB]
-  uint8_t* b_buf = smem + C::kStages * kABytes;               // [stages][boxes][8 KB]
+  uint8_t* a_buf = smem;                                      // [stages][A tiles][16 KB]
+  uint8_t* b_buf = smem + C::kStages * C::kATiles * kABytes;  // [stages][boxes][8 KB]
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::kStages * C::kStageBytes);
   uint64_t* empty = full + C::kStages;
   uint64_t* acc_done = empty + C::kStages;
@@ -86,7 +89,8 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
         ok = mbar_wait(&empty[s], ((i / C::kStages) & 1) ^ 1, status, 101, cta_abort);
         if (!ok) break;
         mbar_arrive_expect_tx(&full[s], C::kStageBytes);
-        tma_load_3d(a_buf + s * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, h);
+        tma_load_3d(a_buf + s * C::kATiles * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, h);
+        if (SEP) tma_load_3d(a_buf + (s * C::kATiles + 1) * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, H + h);
 #pragma unroll
         for (int g = 0; g < C::kBoxes; ++g) {
           const bool is_v = g >= C::kBoxes / 2;
@@ -103,18 +107,22 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
     }
   } else if (warp == 1) {
     if (elect_one()) {
-      constexpr uint32_t idesc = make_idesc_bf16(kTileM, C::kN, /*A MN-major*/ false, /*B MN-major*/ true);
+      constexpr uint32_t idesc = make_idesc_bf16(kTileM, SEP ? D : C::kN, /*A MN-major*/ false, /*B MN-major*/ true);
       bool ok = true;
       for (int i = 0; i < nchunks; ++i) {
         const int s = i % C::kStages;
         ok = mbar_wait(&full[s], (i / C::kStages) & 1, status, 103, cta_abort);
         if (!ok) break;
         tc_fence_after();
-        const uint64_t a_desc = make_smem_desc(smem_u32(a_buf + s * kABytes), 16, 1024);
+        const uint64_t a_desc = make_smem_desc(smem_u32(a_buf + s * C::kATiles * kABytes), 16, 1024);
         const uint64_t b_desc = make_smem_desc(smem_u32(b_buf + s * C::kBoxes * kBoxBytes), kBoxBytes, 1024);
 #pragma unroll
-        for (int k = 0; k < kChunk / 16; ++k)   // +32 B along K for A, +2048 B (16 token rows) for B
+        for (int k = 0; k < kChunk / 16; ++k) { // +32 B along K for A, +2048 B (16 token rows) for B
           mma_f16_ss(tmem_base, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, (i | k) != 0);
+          if (SEP)                              // V columns: the second A tile, the V boxes, accumulator columns [d, 2d)
+            mma_f16_ss(tmem_base + D, a_desc + (uint64_t)((kABytes >> 4) + k * 2),
+                       b_desc + (uint64_t)(((C::kBoxes / 2) * kBoxBytes >> 4) + k * 128), idesc, (i | k) != 0);
+        }
         mma_commit(&empty[s]);                  // stage reusable once these MMAs have read it
       }
       mma_commit(acc_done);                     // arrives when every MMA above has finished (also after a give-up)
@@ -165,9 +173,9 @@ __global__ void wait_timeout_selftest_kernel(int* status, unsigned long long lim
   }
 }
 
-template <int D>
+template <int D, bool SEP>
 cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
-  using C = Cfg<D>;
+  using C = Cfg<D, SEP>;
   const Params& p = c->p;
   CUtensorMap tk, tv;
   const uint64_t kd[3] = {(uint64_t)D, (uint64_t)p.n, (uint64_t)(p.B * p.H)};
@@ -178,12 +186,12 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
   if ((e = make_tmap_bf16_3d(&tv, V, kd, ks, kb)) != cudaSuccess) return e;
   static bool attr_set = false;
   if (!attr_set) {
-    e = cudaFuncSetAttribute(compress_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
+    e = cudaFuncSetAttribute(compress_sm100_kernel<D, SEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(p.B * p.H));
-  compress_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
+  compress_sm100_kernel<D, SEP><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
                                                                  (int)p.n, (int)p.H, (int)p.B, c->status);
   return cudaGetLastError();
 }
@@ -197,7 +205,7 @@ cudaError_t launch_wait_timeout_selftest(csat_ctx* c, unsigned long long limit_n
 
 cudaError_t make_phi_tmap(csat_ctx* c) {
   const Params& p = c->p;
-  const uint64_t d[3] = {(uint64_t)p.n_pad, (uint64_t)p.m, (uint64_t)p.H};
+  const uint64_t d[3] = {(uint64_t)p.n_pad, (uint64_t)p.m, (uint64_t)c->phi_heads()};
   const uint64_t st[2] = {(uint64_t)p.n_pad * 2, (uint64_t)p.m * p.n_pad * 2};
   const uint32_t b[3] = {(uint32_t)kChunk, (uint32_t)kTileM, 1};
   return make_tmap_bf16_3d(&c->tmap_phi, c->phi, d, st, b);
@@ -205,7 +213,8 @@ cudaError_t make_phi_tmap(csat_ctx* c) {
 
 cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches) {
   *launches += 1;
-  return c->p.d == 64 ? launch<64>(c, K, V, s) : launch<128>(c, K, V, s);
+  if (c->p.separate_phi) return c->p.d == 64 ? launch<64, true>(c, K, V, s) : launch<128, true>(c, K, V, s);
+  return c->p.d == 64 ? launch<64, false>(c, K, V, s) : launch<128, false>(c, K, V, s);
 }
 
 }  // namespace csat

@@ -39,7 +39,15 @@ void dev_free(csat_ctx* c, T** p, size_t bytes) {
   }
 }
 
-size_t phi_bytes(const csat::Params& p) { return (size_t)(p.H * p.m * p.n_pad) * csat::elt_size(p.dtype); }
+size_t phi_bytes(const csat::Params& p) {
+  return (size_t)(p.H * (p.separate_phi ? 2 : 1) * p.m * p.n_pad) * csat::elt_size(p.dtype);
+}
+// the generators see Phi_V of head h as head H + h
+csat::Params gen_params(const csat::Params& p) {
+  csat::Params g = p;
+  g.H = p.H * (p.separate_phi ? 2 : 1);
+  return g;
+}
 size_t kv_bytes(const csat::Params& p) { return (size_t)(p.B * p.H * p.m * 2 * p.d) * csat::elt_size(p.dtype); }
 size_t dd_bytes(const csat::Params& p, size_t elt) { return (size_t)(p.H * p.d * p.d) * elt; }
 
@@ -90,7 +98,7 @@ int allocate_and_generate(csat_ctx* c) {
   cudaError_t e;
   if ((e = dev_alloc(c, &c->phi, phi_bytes(p))) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(Phi) failed");
   if ((e = dev_alloc(c, &c->kv, kv_bytes(p))) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(K~|V~) failed");
-  if ((e = csat::launch_phi_gen(c->phi, p, 0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen launch");
+  if ((e = csat::launch_phi_gen(c->phi, gen_params(p), 0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen launch");
   if ((e = cudaStreamSynchronize(0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen");
   c->tmap_phi_valid = false;
   if (p.dtype == CSAT_DTYPE_BF16 && (p.d == 64 || p.d == 128)) {
@@ -174,6 +182,7 @@ csat_ctx* csat_create(int64_t n, int64_t m, int64_t d, int64_t H, uint64_t seed)
   p.n_pad = csat::round_up(n, csat::kPhiColPad);
   p.dtype = CSAT_DTYPE_BF16;
   p.ensemble = CSAT_ENSEMBLE_GAUSSIAN;
+  p.separate_phi = 0;
   p.T = 10; p.lambda = 0.1; p.step = 0.0; p.scale = 0.0; p.seed = seed;
 
   int rc = CSAT_OK;
@@ -251,11 +260,20 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       if ((int)v == p.ensemble) return CSAT_OK;
       cudaDeviceSynchronize();
       p.ensemble = (int)v;
-      cudaError_t e = csat::launch_phi_gen(c->phi, p, 0);      // a Phi set by csat_set_phi is replaced as well
+      cudaError_t e = csat::launch_phi_gen(c->phi, gen_params(p), 0);   // a Phi set by csat_set_phi is replaced as well
       if (e == cudaSuccess) e = cudaStreamSynchronize(0);
       if (e != cudaSuccess) return fail_cuda(c, e, "phi_gen");
       c->decoder_dirty = true;
       return CSAT_OK;
+    }
+    case CSAT_SEPARATE_PHI: {
+      if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_SEPARATE_PHI must be 0 or 1");
+      if ((int)v == p.separate_phi) return CSAT_OK;
+      cudaDeviceSynchronize();
+      dev_free(c, &c->phi, phi_bytes(p));
+      dev_free(c, &c->kv, kv_bytes(p));
+      p.separate_phi = (int)v;
+      return allocate_and_generate(c);
     }
     case CSAT_T:
       if (v < 0 || v > 100000) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_T must be in [0, 100000]");
@@ -297,6 +315,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
     case CSAT_DTYPE: *out = c->p.dtype; return CSAT_OK;
     case CSAT_T: *out = c->p.T; return CSAT_OK;
     case CSAT_ENSEMBLE: *out = c->p.ensemble; return CSAT_OK;
+    case CSAT_SEPARATE_PHI: *out = c->p.separate_phi; return CSAT_OK;
     case CSAT_FORCE_SIMT: *out = c->force_simt; return CSAT_OK;
     case CSAT_PROFILE: *out = c->prof_slots; return CSAT_OK;
     default: return CSAT_ERR_INVALID_ARG;
@@ -336,7 +355,7 @@ int csat_set_phi(csat_ctx* c, const void* phi, void* stream) {
   if (!phi || !aligned16(phi)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_phi: NULL or misaligned pointer");
   std::string why;
   if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
-  cudaError_t e = csat::launch_phi_pack(c->phi, phi, c->p, (cudaStream_t)stream);
+  cudaError_t e = csat::launch_phi_pack(c->phi, phi, gen_params(c->p), (cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_set_phi");
   c->decoder_dirty = true;
   return CSAT_OK;
@@ -348,7 +367,7 @@ int csat_get_phi(const csat_ctx* c, void* phi_out, void* stream) {
   if (!phi_out || !aligned16(phi_out)) return fail(mc, CSAT_ERR_INVALID_ARG, "csat_get_phi: NULL or misaligned pointer");
   std::string why;
   if (!on_device(c, &why)) return fail(mc, CSAT_ERR_STATE, why);
-  cudaError_t e = csat::launch_phi_unpack(phi_out, c->phi, c->p, (cudaStream_t)stream);
+  cudaError_t e = csat::launch_phi_unpack(phi_out, c->phi, gen_params(c->p), (cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(mc, e, "csat_get_phi");
   return CSAT_OK;
 }

@@ -22,6 +22,7 @@ struct Params {            // plain values kernels need
   int64_t n_pad;           // padded row length of Phi
   int dtype;               // CSAT_DTYPE_*
   int ensemble;            // CSAT_ENSEMBLE_*
+  int separate_phi;        // 1: Phi holds 2H matrices, Phi_K of every head then Phi_V of every head
   int T;
   double lambda, step, scale;
   uint64_t seed;
@@ -31,6 +32,7 @@ struct Params {            // plain values kernels need
 
 struct csat_ctx {
   csat::Params p;
+  int64_t phi_heads() const { return p.H * (p.separate_phi ? 2 : 1); }   // matrices stored in phi
   int device = 0;
   int force_simt = 0;         // diagnostic: 1 = FFMA kernels for everything, 2 = for attention/recovery only
 

@@ -18,12 +18,12 @@ template <> __device__ __forceinline__ double ld<__nv_bfloat16>(const __nv_bfloa
 // M[h][a][b] = sum_k D[h][a][k] * Psi[h][k][b]
 template <typename T>
 __global__ void build_M_kernel(double* __restrict__ M, const T* __restrict__ phi, const T* __restrict__ dmat,
-                               const T* __restrict__ psi, int psi_per_head, int d, int64_t m, int64_t n_pad) {
+                               const T* __restrict__ psi, int psi_per_head, int d, int64_t m, int64_t n_pad, int phi_head0) {
   const int h = blockIdx.y;
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   if (idx >= d * d) return;
   const int a = idx / d, b = idx % d;
-  const T* Dh = dmat ? dmat + (int64_t)h * d * d : phi + (int64_t)h * m * n_pad;
+  const T* Dh = dmat ? dmat + (int64_t)h * d * d : phi + (int64_t)(phi_head0 + h) * m * n_pad;   // block of Phi_V
   const int64_t ldD = dmat ? d : n_pad;
   double acc;
   if (psi) {
@@ -126,7 +126,7 @@ cudaError_t run(csat_ctx* c, cudaStream_t s, int* launches) {
     return cudaGetLastError();
   }
   build_M_kernel<T><<<grid, 256, 0, s>>>(c->Mf64, (const T*)c->phi, (const T*)c->dmat, (const T*)c->psi,
-                                         c->psi_per_head ? 1 : 0, d, p.m, p.n_pad);
+                                         c->psi_per_head ? 1 : 0, d, p.m, p.n_pad, p.separate_phi ? (int)p.H : 0);
   gram_kernel<<<grid, 256, 0, s>>>(c->Gf64, c->Mf64, d);
   finalize_kernel<T><<<H, 256, 0, s>>>(c->S_dec, c->B_dec, c->theta, c->mu, c->psi_f32, c->Gf64, c->Mf64,
                                        (const T*)c->psi, c->psi_per_head ? 1 : 0, d, p.lambda, p.step, c->mats_bf16);

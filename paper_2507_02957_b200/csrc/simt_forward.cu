@@ -30,10 +30,12 @@ constexpr int kCmpRows = 32, kCmpChunk = 16;
 template <typename T, int KC>   // KC = ceil(2d / 32) column slots per lane
 __global__ void __launch_bounds__(256) compress_kernel(T* __restrict__ kv, const T* __restrict__ phi,
                                                        const T* __restrict__ K, const T* __restrict__ V, int64_t n,
-                                                       int64_t n_pad, int64_t m, int d, int H) {
+                                                       int64_t n_pad, int64_t m, int d, int H, int phi_v_head0) {
+  // phi_v_head0: index of the first Phi_V matrix in phi (0 when Phi_V = Phi_K, H when they are separate)
   extern __shared__ float smem[];
-  float* phis = smem;                              // [32][17]
-  float* kvs = smem + kCmpRows * (kCmpChunk + 1);  // [16][2d]
+  float* phis = smem;                              // [2][32][17]: Phi_K tile, Phi_V tile
+  float* phiv = smem + kCmpRows * (kCmpChunk + 1);
+  float* kvs = smem + 2 * kCmpRows * (kCmpChunk + 1);  // [16][2d]
   const int d2 = 2 * d;
   const int bh = blockIdx.y, h = bh % H;
   const int64_t r0 = (int64_t)blockIdx.x * kCmpRows;
@@ -41,6 +43,7 @@ __global__ void __launch_bounds__(256) compress_kernel(T* __restrict__ kv, const
   const T* Kb = K + (int64_t)bh * n * d;
   const T* Vb = V + (int64_t)bh * n * d;
   const T* Ph = phi + (int64_t)h * m * n_pad;
+  const T* Pv = phi + (int64_t)(phi_v_head0 + h) * m * n_pad;
   float acc[4][KC];
 #pragma unroll
   for (int i = 0; i < 4; ++i)
@@ -52,6 +55,7 @@ __global__ void __launch_bounds__(256) compress_kernel(T* __restrict__ kv, const
       const int rr = i / kCmpChunk, jj = i % kCmpChunk;
       const int64_t r = r0 + rr;
       phis[rr * (kCmpChunk + 1) + jj] = (r < m) ? ldf(Ph, r * n_pad + j0 + jj) : 0.f;   // padded columns hold 0
+      phiv[rr * (kCmpChunk + 1) + jj] = (r < m) ? ldf(Pv, r * n_pad + j0 + jj) : 0.f;
     }
     for (int i = threadIdx.x; i < kCmpChunk * d2; i += 256) {
       const int jj = i / d2, c = i % d2;
@@ -63,15 +67,18 @@ __global__ void __launch_bounds__(256) compress_kernel(T* __restrict__ kv, const
     __syncthreads();
 #pragma unroll 4
     for (int jj = 0; jj < kCmpChunk; ++jj) {
-      float a[4];
+      float a[4], av[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = phis[(ty * 4 + i) * (kCmpChunk + 1) + jj];
+      for (int i = 0; i < 4; ++i) {
+        a[i] = phis[(ty * 4 + i) * (kCmpChunk + 1) + jj];
+        av[i] = phiv[(ty * 4 + i) * (kCmpChunk + 1) + jj];
+      }
 #pragma unroll
       for (int k = 0; k < KC; ++k) {
         const int c = tx + 32 * k;
         const float b = (c < d2) ? kvs[jj * d2 + c] : 0.f;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) acc[i][k] = fmaf(a[i], b, acc[i][k]);
+        for (int i = 0; i < 4; ++i) acc[i][k] = fmaf(c < d ? a[i] : av[i], b, acc[i][k]);   // K columns, then V columns
       }
     }
     __syncthreads();
@@ -254,11 +261,11 @@ cudaError_t compress_t(csat_ctx* c, const void* K, const void* V, cudaStream_t s
   const Params& p = c->p;
   const int d = (int)p.d;
   const dim3 grid((unsigned)((p.m + kCmpRows - 1) / kCmpRows), (unsigned)(p.B * p.H));
-  const size_t sm = (size_t)(kCmpRows * (kCmpChunk + 1) + kCmpChunk * 2 * d) * sizeof(float);
+  const size_t sm = (size_t)(2 * kCmpRows * (kCmpChunk + 1) + kCmpChunk * 2 * d) * sizeof(float);
   const int kc = (2 * d + 31) / 32;
 #define CSAT_CMP(KC)                                                                                         \
   compress_kernel<T, KC><<<grid, 256, sm, s>>>((T*)c->kv, (const T*)c->phi, (const T*)K, (const T*)V, p.n, \
-                                               p.n_pad, p.m, d, (int)p.H)
+                                               p.n_pad, p.m, d, (int)p.H, p.separate_phi ? (int)p.H : 0)
   if (kc <= 4) CSAT_CMP(4);
   else if (kc <= 8) CSAT_CMP(8);
   else CSAT_CMP(16);

@@ -341,3 +341,43 @@ def test_hadamard_ensemble_is_bit_exact_and_runs(dtype):
         ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=lam)
         assert rel_err(out, ref) <= TOL[dtype], (dtype, T)
     ctx.close()
+
+
+@pytest.mark.parametrize("name", ["c1_full_fp32", "c3_video_B1_H2", "c5_long_n2048_nq700", "c4_cross_B2_H2", "ragged_bf16_d40"])
+def test_separate_key_and_value_matrices(name):
+    """CSAT_SEPARATE_PHI: K~ = Phi_K K, V~ = Phi_V V with Phi_V drawn as heads H .. 2H-1 of the same generator;
+    the decoder's default matrix is the block of Phi_V."""
+    w = SMALL_CASES[name]
+    inp = wl.make_inputs(w)
+    Q, K, V, Psi = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    if Psi is not None:
+        ctx.set_dictionary(Psi)
+    shared = ctx.get_phi().clone()
+    ctx.set(separate_phi=True)
+    both = ctx.get_phi()
+    assert both.shape[0] == 2 * w.H and torch.equal(both[:w.H], shared)       # Phi_K is the shared matrix
+    assert not torch.equal(both[w.H:], both[:w.H])
+    phi = to_np(both)
+    for T, lam in [(0, w.lam), (w.T, w.lam), (w.T, 0.0)]:
+        ctx.set(T=T, lam=lam)
+        out = to_np(ctx.forward(Q, K, V))
+        stages = []
+        ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi[:w.H], T=T, lam=lam, Psi=inp["Psi"],
+                               Phi_V=phi[w.H:], stages=stages)
+        if np.abs(ref).max() == 0.0:
+            assert np.abs(out).max() <= max(s["theta"] for s in stages) * TOL[w.dtype]
+        else:
+            assert rel_err(out, ref) <= TOL[w.dtype], (name, T, lam)
+    kt, vt = (to_np(t) for t in ctx.get_compressed())
+    vt_ref = np.stack([[s["Vt"]] for s in stages]).reshape(vt.shape)
+    assert rel_err(vt, vt_ref) <= (4e-3 if w.dtype == "bf16" else 2e-6)
+    # Rademacher: both halves bit-exact against the oracle's 2H-head generator
+    ctx.set(ensemble="rademacher")
+    ref = wl.round_to_storage(pho.phi_rademacher(2 * w.H, w.m, w.n, w.phi_seed).astype(np.float32), w.dtype)
+    assert np.array_equal(to_np(ctx.get_phi()), ref.astype(np.float64))
+    # back to one matrix per head
+    ctx.set(ensemble="gaussian")
+    ctx.set(separate_phi=False)
+    assert torch.equal(ctx.get_phi(), shared)
+    ctx.close()
