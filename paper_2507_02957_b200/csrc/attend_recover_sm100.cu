@@ -6,8 +6,9 @@
 //
 // One persistent CTA per SM walks work items of 256 consecutive queries of one (batch, head), each as two
 // independent tiles A and B that share the stream of K~|V~ chunks; the TMA and MMA warps run ahead into the
-// next item (its Q tiles, first chunks and first S MMAs) while the compute threads finish the current one.  While the tensor cores run one tile's MMAs the other tile's threads do
-// their softmax / shrinkage arithmetic, and the other way round.
+// next item (its Q tiles, first chunks and first S MMAs) while the compute threads finish the current one.
+// While the tensor cores run one tile's MMAs the other tile's threads do their softmax / shrinkage
+// arithmetic, and the other way round.
 //
 // CTA = 12 warps in three warpgroups (registers are re-divided between them with setmaxnreg: the two
 // compute warpgroups hold a whole row of alpha per thread, the control warps need very few):
