@@ -28,21 +28,26 @@ constexpr uint32_t kBoxBytes = 64 * kChunk * 2;       // 8 KB: 64 columns x 64 t
 
 // SEP: separate measurement matrices for keys and values (a second A tile per stage, Phi_V, which multiplies the
 // V columns; the K columns keep Phi_K)
-template <int D, bool SEP> struct Cfg {
-  static constexpr int kN = 2 * D;                    // accumulator columns
+// BG: batch elements per CTA.  They share the Phi tile; their K (then their V) columns sit side by side in the B
+// operand and the accumulator: [K of element 0 .. K of element BG-1 | V of element 0 .. V of element BG-1].  With
+// d = 64 one element gives an N = 128 MMA, which needs 32 KB of operands per 256 cycles of tensor work: right at
+// what an SM can load; two elements (N = 256) halve the operand bytes per flop and the L2 reads of Phi.
+template <int D, bool SEP, int BG> struct Cfg {
+  static constexpr int kN = 2 * D * BG;               // accumulator columns
   static constexpr int kBoxes = kN / 64;              // B boxes per stage
   static constexpr int kATiles = SEP ? 2 : 1;
-  static constexpr int kStages = (D == 64) ? (SEP ? 4 : 6) : (SEP ? 3 : 4);
+  static constexpr int kStages = (D == 64 && BG == 1) ? (SEP ? 4 : 6) : (SEP ? 3 : 4);
+  static_assert(kN <= 256, "one MMA covers the accumulator");
   static constexpr uint32_t kStageBytes = kATiles * kABytes + kBoxes * kBoxBytes;
   static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <int D, bool SEP>
+template <int D, bool SEP, int BG>
 __global__ void __launch_bounds__(kThreads, 1)
 compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, __nv_bfloat16* __restrict__ kv, int m, int n, int H,
                       int B, int* status) {
-  using C = Cfg<D, SEP>;
+  using C = Cfg<D, SEP, BG>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a_buf = smem;                                      // [stages][A tiles][16 KB]
@@ -56,7 +61,11 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // blockIdx.y walks the batch fastest, so that the CTAs that stream the same tile of Phi_h (one per batch
   // element) are scheduled together and all but the first find it in L2
-  const int mtile = blockIdx.x, h = blockIdx.y / B, bh = (blockIdx.y % B) * H + h;
+  // (with BG > 1 blockIdx.y counts groups of BG batch elements; a group that runs past the batch repeats its
+  // last element and does not store it)
+  const int groups = (B + BG - 1) / BG;
+  const int mtile = blockIdx.x, h = blockIdx.y / groups, b0 = (blockIdx.y % groups) * BG;
+  auto bh_of = [&](int e) { return (b0 + e < B ? b0 + e : B - 1) * H + h; };
   const int nchunks = (n + kChunk - 1) / kChunk;
 
   if (threadIdx.x == 0) {
@@ -94,8 +103,9 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
 #pragma unroll
         for (int g = 0; g < C::kBoxes; ++g) {
           const bool is_v = g >= C::kBoxes / 2;
+          const int gg = g % (C::kBoxes / 2);               // box within the K (or V) half: element, then 64-column box
           tma_load_3d(b_buf + (s * C::kBoxes + g) * kBoxBytes, is_v ? &tmap_v : &tmap_k, &full[s],
-                      (g % (C::kBoxes / 2)) * 64, i * kChunk, bh);
+                      (gg % (D / 64)) * 64, i * kChunk, bh_of(gg / (D / 64)));
         }
         ++issued;
       }
@@ -107,7 +117,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
     }
   } else if (warp == 1) {
     if (elect_one()) {
-      constexpr uint32_t idesc = make_idesc_bf16(kTileM, SEP ? D : C::kN, /*A MN-major*/ false, /*B MN-major*/ true);
+      constexpr uint32_t idesc = make_idesc_bf16(kTileM, SEP ? C::kN / 2 : C::kN, /*A MN-major*/ false, /*B MN-major*/ true);
       bool ok = true;
       for (int i = 0; i < nchunks; ++i) {
         const int s = i % C::kStages;
@@ -120,7 +130,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
         for (int k = 0; k < kChunk / 16; ++k) { // +32 B along K for A, +2048 B (16 token rows) for B
           mma_f16_ss(tmem_base, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 128), idesc, (i | k) != 0);
           if (SEP)                              // V columns: the second A tile, the V boxes, accumulator columns [d, 2d)
-            mma_f16_ss(tmem_base + D, a_desc + (uint64_t)((kABytes >> 4) + k * 2),
+            mma_f16_ss(tmem_base + C::kN / 2, a_desc + (uint64_t)((kABytes >> 4) + k * 2),
                        b_desc + (uint64_t)(((C::kBoxes / 2) * kBoxBytes >> 4) + k * 128), idesc, (i | k) != 0);
         }
         mma_commit(&empty[s]);                  // stage reusable once these MMAs have read it
@@ -132,14 +142,15 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
     if (mbar_wait(acc_done, 0, status, 104, cta_abort) && *(volatile int*)cta_abort == 0) {
       tc_fence_after();
       const int row = mtile * kTileM + q * 32 + lane;
-      __nv_bfloat16* dst = kv + ((int64_t)bh * m + row) * C::kN;
 #pragma unroll 1
       for (int c0 = 0; c0 < C::kN; c0 += 32) {
         uint32_t r[32];
         tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
         tmem_wait_ld();
-        if (row < m) {
-          uint4* o = reinterpret_cast<uint4*>(dst + c0);
+        // accumulator column c0: K half or V half, batch element e of the group, feature column
+        const int half = c0 / (C::kN / 2), e = (c0 % (C::kN / 2)) / D, col = c0 % D;
+        if (row < m && b0 + e < B) {
+          uint4* o = reinterpret_cast<uint4*>(kv + ((int64_t)bh_of(e) * m + row) * (2 * D) + half * D + col);
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             uint32_t w[4];
@@ -173,9 +184,9 @@ __global__ void wait_timeout_selftest_kernel(int* status, unsigned long long lim
   }
 }
 
-template <int D, bool SEP>
+template <int D, bool SEP, int BG>
 cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
-  using C = Cfg<D, SEP>;
+  using C = Cfg<D, SEP, BG>;
   const Params& p = c->p;
   CUtensorMap tk, tv;
   const uint64_t kd[3] = {(uint64_t)D, (uint64_t)p.n, (uint64_t)(p.B * p.H)};
@@ -186,12 +197,12 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
   if ((e = make_tmap_bf16_3d(&tv, V, kd, ks, kb)) != cudaSuccess) return e;
   static bool attr_set = false;
   if (!attr_set) {
-    e = cudaFuncSetAttribute(compress_sm100_kernel<D, SEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
+    e = cudaFuncSetAttribute(compress_sm100_kernel<D, SEP, BG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(p.B * p.H));
-  compress_sm100_kernel<D, SEP><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
+  const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(((p.B + BG - 1) / BG) * p.H));
+  compress_sm100_kernel<D, SEP, BG><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
                                                                  (int)p.n, (int)p.H, (int)p.B, c->status);
   return cudaGetLastError();
 }
@@ -213,8 +224,11 @@ cudaError_t make_phi_tmap(csat_ctx* c) {
 
 cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches) {
   *launches += 1;
-  if (c->p.separate_phi) return c->p.d == 64 ? launch<64, true>(c, K, V, s) : launch<128, true>(c, K, V, s);
-  return c->p.d == 64 ? launch<64, false>(c, K, V, s) : launch<128, false>(c, K, V, s);
+  // d = 64: two batch elements per CTA where the batch has them (N = 256 MMAs)
+  if (c->p.d == 64 && c->p.B >= 2)
+    return c->p.separate_phi ? launch<64, true, 2>(c, K, V, s) : launch<64, false, 2>(c, K, V, s);
+  if (c->p.separate_phi) return c->p.d == 64 ? launch<64, true, 1>(c, K, V, s) : launch<128, true, 1>(c, K, V, s);
+  return c->p.d == 64 ? launch<64, false, 1>(c, K, V, s) : launch<128, false, 1>(c, K, V, s);
 }
 
 }  // namespace csat

@@ -24,6 +24,7 @@ SMALL_CASES = {
     "c1_as_bf16": wl.shrink(C["c1"], dtype="bf16"),
     "c2_vit_B2_H3": wl.shrink(C["c2"], B=2, H=3),
     "c3_video_B1_H2": wl.shrink(C["c3"], B=1, H=2),
+    "c3_video_B3_H1_odd_batch": wl.shrink(C["c3"], B=3, H=1, n=392, n_q=200, m=200),
     "c4_cross_B2_H2": wl.shrink(C["c4"], B=2, H=2),
     "c5_long_n2048_nq700": wl.shrink(C["c5"], B=1, H=2, n=2048, n_q=700, m=128),
     "c5_long_n4096_m256": wl.shrink(C["c5"], B=1, H=1, n=4096, n_q=1000, m=256),
