@@ -382,3 +382,40 @@ def test_separate_key_and_value_matrices(name):
     ctx.set(separate_phi=False)
     assert torch.equal(ctx.get_phi(), shared)
     ctx.close()
+
+
+def test_tensor_core_edge_shapes():
+    """Shapes that stress the tcgen05 kernels' tails: partial query tiles and measurement chunks at d = 128,
+    a single query, fewer measurements than one chunk, a dictionary with one iteration, many iterations."""
+    r = np.random.default_rng(17)
+    cases = [  # B, H, n, n_q, d, m, T, with_psi
+        (3, 2, 200, 130, 128, 136, 3, False),
+        (1, 1, 128, 1, 128, 128, 2, True),
+        (2, 1, 300, 257, 128, 9, 1, True),
+        (1, 2, 90, 40, 64, 1, 4, False),
+        (2, 3, 520, 513, 64, 200, 1, True),
+        (1, 1, 256, 100, 128, 192, 60, False),
+    ]
+    for (B, H, n, nq, d, m, T, with_psi) in cases:
+        w = wl.Workload("tc_edge", B, H, n, nq, d, m, "bf16", T, 0.02, "iid", 5)
+        inp = wl.make_inputs(w)
+        Q, K, V, _ = device_inputs(w, inp)
+        ctx = make_ctx(w)
+        Dn = wl.round_to_storage((np.eye(d) + 0.1 * r.standard_normal((H, d, d))).astype(np.float32), "bf16")
+        ctx.set_decoder_matrix(to_dev(Dn, "bf16"))           # m may be smaller than d
+        psi = None
+        if with_psi:
+            psi = wl.orthonormal_basis(d, 99 + d)
+            psi = wl.round_to_storage(psi, "bf16")
+            ctx.set_dictionary(to_dev(psi, "bf16"))
+        phi = to_np(ctx.get_phi())
+        for T_run, lam in [(0, 0.0), (T, 0.02), (T, 0.0)]:
+            ctx.set(T=T_run, lam=lam)
+            out = ctx.forward(Q, K, V)
+            assert torch.isfinite(out).all()
+            ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T_run, lam=lam, D=Dn.astype(np.float64),
+                                   Psi=None if psi is None else psi.astype(np.float64))
+            assert np.abs(ref).max() > 0
+            err = rel_err(to_np(out), ref)
+            assert err <= TOL["bf16"], (B, H, n, nq, d, m, T_run, lam, err)
+        ctx.close()
