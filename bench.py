@@ -310,7 +310,7 @@ def run_csat(args, w: wl.Workload) -> dict:
     top = kernels[0]
     peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
     if w.dtype == "fp32":
-        peak_tf = peak_tf / 32.0   # FFMA path: no fp32 tensor-core kernel
+        peak_tf = peak_tf / 32.0   # FFMA path: no fp32 tensor-core kernel; fp32 FMA peak taken as 1/32 of the bf16 tensor peak
     roofline = {"kernel": top["kernel"], "bound": "tensor", "achieved": top["tflops"], "peak": peak_tf,
                 "unit": "TFLOP/s", "frac": top["tflops"] / peak_tf, "peak_source": f"{peak_kind} bf16 sustained",
                 "traffic": NCU_TRAFFIC_BYTES.get((top["kernel"], w.name)),

@@ -48,7 +48,7 @@ enum {
   CSAT_ERR_SHAPE = 2,       /* a size outside the supported range (see csat_create)      */
   CSAT_ERR_ALLOC = 3,       /* device or host allocation failed                          */
   CSAT_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; text in last_error     */
-  CSAT_ERR_UNSUPPORTED = 5, /* valid request this build has no kernel for                */
+  CSAT_ERR_UNSUPPORTED = 5, /* valid request this library has no kernel for              */
   CSAT_ERR_STATE = 6,       /* call not legal in the context's current state             */
   CSAT_ERR_TIMEOUT = 7      /* a bounded device-side wait gave up (reported by the next
                                host call that reads the device status word)              */

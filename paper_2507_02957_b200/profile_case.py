@@ -1,0 +1,88 @@
+"""Runs a few CSAT forwards of a given shape and prints the library's per-kernel CUDA-event times.
+
+    python -m paper_2507_02957_b200.profile_case forward N M D B H T [--nq NQ] [--iters I] [--dtype bf16|fp32]
+    python -m paper_2507_02957_b200.profile_case workload c1|c2|c3|c4|c5 [--iters I]
+    python -m paper_2507_02957_b200.profile_case ensembles N M D H        (regenerates Phi with every ensemble)
+
+A small driver to put under a profiler (ncu -k regex:<kernel> ...): 3 warm-up forwards, then I timed ones.
+Inputs are seeded random tensors (N(0, 1/d) for `forward`, the workload's own recipe for `workload`).
+"""
+from __future__ import annotations
+
+import argparse
+import time
+
+import numpy as np
+import torch
+
+from . import binding, workloads as wl
+
+
+def _timed_forwards(ctx, Q, K, V, iters):
+    out = torch.empty_like(Q)
+    for _ in range(3):
+        ctx.forward(Q, K, V, out)
+    torch.cuda.synchronize()
+    binding.csat_set_i64(ctx.h, binding.CSAT_PROFILE, iters)
+    for _ in range(iters):
+        ctx.forward(Q, K, V, out)
+    torch.cuda.synchronize()
+    per = {}
+    for i in range(iters):
+        for kid, ms in binding.csat_get_profile(ctx.h, i):
+            per.setdefault(binding.KERNEL_NAMES.get(kid, str(kid)), []).append(ms)
+    return {k: round(float(np.median(v)), 5) for k, v in per.items()}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    sub = ap.add_subparsers(dest="cmd", required=True)
+    f = sub.add_parser("forward")
+    for name in ("n", "m", "d", "B", "H", "T"):
+        f.add_argument(name, type=int)
+    f.add_argument("--nq", type=int, default=None)
+    f.add_argument("--iters", type=int, default=5)
+    f.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
+    w_ = sub.add_parser("workload")
+    w_.add_argument("name")
+    w_.add_argument("--iters", type=int, default=5)
+    e = sub.add_parser("ensembles")
+    for name in ("n", "m", "d", "H"):
+        e.add_argument(name, type=int)
+    a = ap.parse_args()
+
+    if a.cmd == "forward":
+        nq = a.nq or a.n
+        dt = torch.bfloat16 if a.dtype == "bf16" else torch.float32
+        g = torch.Generator(device="cuda")
+        g.manual_seed(1)
+        s = 1.0 / np.sqrt(a.d)
+        Q = (torch.randn(a.B, a.H, nq, a.d, device="cuda", generator=g) * s).to(dt)
+        K = (torch.randn(a.B, a.H, a.n, a.d, device="cuda", generator=g) * s).to(dt)
+        V = (torch.randn(a.B, a.H, a.n, a.d, device="cuda", generator=g) * s).to(dt)
+        ctx = binding.Csat(a.n, a.m, a.d, a.H, 0, B=a.B, n_q=nq, dtype=a.dtype, T=a.T, lam=0.05)
+        print(vars(a), _timed_forwards(ctx, Q, K, V, a.iters))
+        ctx.close()
+    elif a.cmd == "workload":
+        w = wl.CONFIGS[a.name]
+        inp = wl.make_inputs(w)
+        dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        Q, K, V = (torch.from_numpy(inp[k]).cuda().to(dt) for k in "QKV")
+        ctx = binding.Csat(w.n, w.m, w.d, w.H, w.phi_seed, B=w.B, n_q=w.n_q, dtype=w.dtype, T=w.T, lam=w.lam)
+        if inp["Psi"] is not None:
+            ctx.set_dictionary(torch.from_numpy(inp["Psi"]).cuda().to(dt))
+        print(w.name, _timed_forwards(ctx, Q, K, V, a.iters))
+        ctx.close()
+    else:
+        ctx = binding.Csat(a.n, a.m, a.d, a.H, 0, dtype="bf16")
+        for ens in ("rademacher", "gaussian", "hadamard", "gaussian", "rademacher"):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            ctx.set(ensemble=ens)
+            torch.cuda.synchronize()
+            print(ens, "regenerated (memset + kernel + synchronise):", round((time.perf_counter() - t0) * 1e3, 3), "ms")
+        ctx.close()
+
+
+if __name__ == "__main__":
+    main()
