@@ -165,10 +165,12 @@ int csat_set_lista_weights(csat_ctx* ctx, const void* S, const void* Bm, const f
 int csat_forward(csat_ctx* ctx, const void* Q, const void* K, const void* V, void* out, void* stream);
 
 /*
- * csat_forward_host -- same computation with HOST buffers (same layouts and dtype; pinned
- * memory gives asynchronous copies).  Copies Q, K, V to staging buffers the context owns
- * (allocated by the first call, so that call also allocates), runs csat_forward, copies out
- * back and synchronises `stream` before returning.
+ * csat_forward_host -- same computation with HOST buffers (same layouts and dtype; pinned memory gives
+ * asynchronous copies).  Copies Q, K, V to staging buffers the context owns (allocated by the first call, so
+ * that call also allocates), computes, copies out back and returns once `stream` has reached the end of all of
+ * it.  On the tensor-core path (and with CSAT_PROFILE off) the job is pipelined in chunks of a few heads of one
+ * batch element over three internal streams (copy in, compute, copy out) ordered after `stream`, so that the
+ * copies overlap the compute and each other; otherwise everything runs in order on `stream`.
  */
 int csat_forward_host(csat_ctx* ctx, const void* Q_host, const void* K_host, const void* V_host,
                       void* out_host, void* stream);

@@ -187,7 +187,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
-                            int has_psi, float scale_log2, int items_x, int n_items, int* status) {
+                            int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
@@ -258,7 +258,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         if (pos >= (uint32_t)C::kStages) w.wait(&bars->v_empty[pos % C::kStages], (pos / C::kStages - 1) & 1, code);
       };
       for (int item = blockIdx.x; item < n_items && !w.dead; item += gridDim.x, ++items_done) {
-        const int bh = item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
+        const int bh = bh0 + item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
         const int ntiles = (nq - row0 > kRows) ? 2 : 1;
 #pragma unroll
         for (int t = 0; t < kTiles; ++t) {
@@ -463,7 +463,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     uint32_t zc_seen = 0;                                       // phases of zc_full[t] this thread has waited for
     int phase = 0;                                              // phases of r_full[t] this thread has waited for
     for (int item = blockIdx.x; item < n_items && !w.dead; item += gridDim.x) {
-      const int bh = item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
+      const int bh = bh0 + item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
       if (t >= ((nq - row0 > kRows) ? 2 : 1)) continue;         // this item has no second tile
       float ref = -INFINITY;                                    // reference maximum of the row (log2 domain)
       uint64_t sum2 = pack2(0.f, 0.f);                          // running sum of P, two partial sums
@@ -728,7 +728,8 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   const float scale_log2 = (float)(scale * 1.4426950408889634);
   // persistent CTAs, one per SM, each walking the work items (256 queries of one (batch, head)) it owns
   const int64_t rows_per_item = kTiles * kRows;
-  const int64_t items_x = (p.nq + rows_per_item - 1) / rows_per_item, n_items = items_x * p.B * p.H;
+  const int64_t items_x = (p.nq + rows_per_item - 1) / rows_per_item;
+  const int64_t n_items = items_x * (c->bh_cnt ? c->bh_cnt : p.B * p.H);    // all (batch, head) pairs, or a sub-range
   if (n_items > (int64_t)1 << 30) return cudaErrorInvalidValue;
   static int sms = 0;
   if (sms == 0) {
@@ -740,7 +741,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
   attend_recover_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(
       tq, c->tmap_kv, c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, p.T,
-      c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, c->status);
+      c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, (int)c->bh0, c->status);
   return cudaGetLastError();
 }
 

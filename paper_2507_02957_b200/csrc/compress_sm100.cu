@@ -46,7 +46,7 @@ template <int D, bool SEP, int BG>
 __global__ void __launch_bounds__(kThreads, 1)
 compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, __nv_bfloat16* __restrict__ kv, int m, int n, int H,
-                      int B, int* status) {
+                      int B, int bh0, int* status) {
   using C = Cfg<D, SEP, BG>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -65,7 +65,10 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
   // last element and does not store it)
   const int groups = (B + BG - 1) / BG;
   const int mtile = blockIdx.x, h = blockIdx.y / groups, b0 = (blockIdx.y % groups) * BG;
-  auto bh_of = [&](int e) { return (b0 + e < B ? b0 + e : B - 1) * H + h; };
+  // bh0: first (batch, head) pair of a sub-range launch (then B = 1 and blockIdx.y counts its heads); 0 otherwise
+  const int hl = h;
+  auto bh_of = [&](int e) { return bh0 + (b0 + e < B ? b0 + e : B - 1) * H + hl; };
+  const int hphi = bh_of(0) % H;                    // head whose Phi this CTA streams
   const int nchunks = (n + kChunk - 1) / kChunk;
 
   if (threadIdx.x == 0) {
@@ -98,8 +101,8 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
         ok = mbar_wait(&empty[s], ((i / C::kStages) & 1) ^ 1, status, 101, cta_abort);
         if (!ok) break;
         mbar_arrive_expect_tx(&full[s], C::kStageBytes);
-        tma_load_3d(a_buf + s * C::kATiles * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, h);
-        if (SEP) tma_load_3d(a_buf + (s * C::kATiles + 1) * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, H + h);
+        tma_load_3d(a_buf + s * C::kATiles * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, hphi);
+        if (SEP) tma_load_3d(a_buf + (s * C::kATiles + 1) * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, H + hphi);
 #pragma unroll
         for (int g = 0; g < C::kBoxes; ++g) {
           const bool is_v = g >= C::kBoxes / 2;
@@ -201,9 +204,11 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(((p.B + BG - 1) / BG) * p.H));
+  // whole batch, or a range of heads of one batch element
+  const int64_t Bl = c->bh_cnt ? 1 : p.B, Hl = c->bh_cnt ? c->bh_cnt : p.H;
+  const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(((Bl + BG - 1) / BG) * Hl));
   compress_sm100_kernel<D, SEP, BG><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
-                                                                 (int)p.n, (int)p.H, (int)p.B, c->status);
+                                                                 (int)p.n, (int)p.H, (int)Bl, (int)c->bh0, c->status);
   return cudaGetLastError();
 }
 
@@ -225,7 +230,7 @@ cudaError_t make_phi_tmap(csat_ctx* c) {
 cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches) {
   *launches += 1;
   // d = 64: two batch elements per CTA where the batch has them (N = 256 MMAs)
-  if (c->p.d == 64 && c->p.B >= 2)
+  if (c->p.d == 64 && c->p.B >= 2 && c->bh_cnt == 0)
     return c->p.separate_phi ? launch<64, true, 2>(c, K, V, s) : launch<64, false, 2>(c, K, V, s);
   if (c->p.separate_phi) return c->p.d == 64 ? launch<64, true, 1>(c, K, V, s) : launch<128, true, 1>(c, K, V, s);
   return c->p.d == 64 ? launch<64, false, 1>(c, K, V, s) : launch<128, false, 1>(c, K, V, s);

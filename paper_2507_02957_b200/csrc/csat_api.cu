@@ -86,6 +86,11 @@ void free_all(csat_ctx* c) {
   free_lista(c);
   free_staging(c);
   prof_destroy(c);
+  if (c->pipe_ready) {
+    for (int i = 0; i < 3; ++i) cudaStreamDestroy(c->pipe_stream[i]);
+    for (int i = 0; i < csat_ctx::kPipeEvents; ++i) cudaEventDestroy(c->pipe_event[i]);
+    c->pipe_ready = false;
+  }
   if (c->status) {
     cudaFreeHost(c->status);
     c->status = nullptr;
@@ -489,6 +494,18 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   return CSAT_OK;
 }
 
+// streams and events of the pipelined host-buffer forward (created by its first call)
+static int ensure_pipeline(csat_ctx* c) {
+  if (c->pipe_ready) return CSAT_OK;
+  cudaError_t e = cudaSuccess;
+  for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaStreamCreateWithFlags(&c->pipe_stream[i], cudaStreamNonBlocking);
+  for (int i = 0; i < csat_ctx::kPipeEvents && e == cudaSuccess; ++i)
+    e = cudaEventCreateWithFlags(&c->pipe_event[i], cudaEventDisableTiming);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_forward_host: stream/event creation");
+  c->pipe_ready = true;
+  return CSAT_OK;
+}
+
 int csat_forward_host(csat_ctx* c, const void* Qh, const void* Kh, const void* Vh, void* outh, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
   if (!Qh || !Kh || !Vh || !outh) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward_host: NULL pointer");
@@ -507,15 +524,75 @@ int csat_forward_host(csat_ctx* c, const void* Qh, const void* Kh, const void* V
   }
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e;
-  if ((e = cudaMemcpyAsync(c->stage_q, Qh, bq, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(c->stage_k, Kh, bkv, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
-      (e = cudaMemcpyAsync(c->stage_v, Vh, bkv, cudaMemcpyHostToDevice, s)) != cudaSuccess)
-    return fail_cuda(c, e, "host->device copy");
-  int rc = csat_forward(c, c->stage_q, c->stage_k, c->stage_v, c->stage_o, stream);
+  const bool tensor_core_path = c->tmap_phi_valid && c->force_simt == 0;
+  if (!tensor_core_path || c->prof_slots != 0) {
+    // plain order: copy everything in, compute, copy out
+    if ((e = cudaMemcpyAsync(c->stage_q, Qh, bq, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(c->stage_k, Kh, bkv, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(c->stage_v, Vh, bkv, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+      return fail_cuda(c, e, "host->device copy");
+    int rc = csat_forward(c, c->stage_q, c->stage_k, c->stage_v, c->stage_o, stream);
+    if (rc != CSAT_OK) return rc;
+    if ((e = cudaMemcpyAsync(outh, c->stage_o, bq, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+      return fail_cuda(c, e, "device->host copy");
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return fail_cuda(c, e, "csat_forward_host");
+    if (*(volatile int*)c->status != 0) return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait gave up");
+    return CSAT_OK;
+  }
+
+  // Pipelined: the job is cut into chunks of a few heads of one batch element (contiguous in every tensor); chunk
+  // i's host->device copies, its two kernels and its device->host copy run on three streams, so that the copies
+  // of neighbouring chunks overlap the compute and each other (the two directions of the bus are independent).
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  if (*(volatile int*)c->status != 0)
+    return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
+  int rc = ensure_pipeline(c);
   if (rc != CSAT_OK) return rc;
-  if ((e = cudaMemcpyAsync(outh, c->stage_o, bq, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
-    return fail_cuda(c, e, "device->host copy");
-  if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return fail_cuda(c, e, "csat_forward_host");
+  cudaStream_t s_in = c->pipe_stream[0], s_run = c->pipe_stream[1], s_out = c->pipe_stream[2];
+  cudaEvent_t ev_start = c->pipe_event[0], ev_done = c->pipe_event[1];
+  // order after the caller's stream
+  if ((e = cudaEventRecord(ev_start, s)) != cudaSuccess || (e = cudaStreamWaitEvent(s_in, ev_start, 0)) != cudaSuccess ||
+      (e = cudaStreamWaitEvent(s_run, ev_start, 0)) != cudaSuccess || (e = cudaStreamWaitEvent(s_out, ev_start, 0)) != cudaSuccess)
+    return fail_cuda(c, e, "csat_forward_host: stream ordering");
+  int launches = 0;
+  if (p.T > 0) {
+    rc = ensure_decoder(c, s_run, &launches);
+    if (rc != CSAT_OK) return rc;
+  }
+  int64_t hg = (p.H + 3) / 4;                         // heads per chunk: about four chunks per batch element
+  const int max_chunks = (csat_ctx::kPipeEvents - 2) / 2;
+  while (p.B * ((p.H + hg - 1) / hg) > max_chunks) ++hg;
+  int chunk = 0;
+  for (int64_t b = 0; b < p.B; ++b) {
+    for (int64_t h0 = 0; h0 < p.H; h0 += hg, ++chunk) {
+      const int64_t cnt = p.H - h0 < hg ? p.H - h0 : hg, bh0 = b * p.H + h0;
+      const size_t oq = (size_t)(bh0 * p.nq * p.d) * es, okv = (size_t)(bh0 * p.n * p.d) * es;
+      const size_t nq_b = (size_t)(cnt * p.nq * p.d) * es, nkv_b = (size_t)(cnt * p.n * p.d) * es;
+      cudaEvent_t ev_in = c->pipe_event[2 + 2 * chunk], ev_run = c->pipe_event[3 + 2 * chunk];
+      if ((e = cudaMemcpyAsync((char*)c->stage_k + okv, (const char*)Kh + okv, nkv_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
+          (e = cudaMemcpyAsync((char*)c->stage_v + okv, (const char*)Vh + okv, nkv_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
+          (e = cudaMemcpyAsync((char*)c->stage_q + oq, (const char*)Qh + oq, nq_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
+          (e = cudaEventRecord(ev_in, s_in)) != cudaSuccess || (e = cudaStreamWaitEvent(s_run, ev_in, 0)) != cudaSuccess)
+        return fail_cuda(c, e, "csat_forward_host: host->device copy");
+      c->bh0 = bh0;
+      c->bh_cnt = cnt;
+      e = csat::launch_sm100_compress(c, c->stage_k, c->stage_v, s_run, &launches);
+      if (e == cudaSuccess) e = csat::launch_sm100_attend_recover(c, c->stage_q, c->stage_o, s_run, &launches);
+      c->bh0 = 0;
+      c->bh_cnt = 0;
+      if (e != cudaSuccess) return fail_cuda(c, e, "csat_forward_host: launch");
+      if ((e = cudaEventRecord(ev_run, s_run)) != cudaSuccess || (e = cudaStreamWaitEvent(s_out, ev_run, 0)) != cudaSuccess ||
+          (e = cudaMemcpyAsync((char*)outh + oq, (const char*)c->stage_o + oq, nq_b, cudaMemcpyDeviceToHost, s_out)) != cudaSuccess)
+        return fail_cuda(c, e, "csat_forward_host: device->host copy");
+    }
+  }
+  // the caller's stream continues after the last copy; this call returns once everything has landed
+  if ((e = cudaEventRecord(ev_done, s_out)) != cudaSuccess || (e = cudaStreamWaitEvent(s, ev_done, 0)) != cudaSuccess ||
+      (e = cudaStreamSynchronize(s)) != cudaSuccess)
+    return fail_cuda(c, e, "csat_forward_host");
+  c->have_forward = true;
+  c->last_launches = launches;
   if (*(volatile int*)c->status != 0) return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait gave up");
   return CSAT_OK;
 }

@@ -65,6 +65,11 @@ struct csat_ctx {
   // staging for csat_forward_host
   void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
   size_t stage_bytes_q = 0, stage_bytes_kv = 0;
+  // streams (copy in, compute, copy out) and events of the pipelined csat_forward_host
+  static constexpr int kPipeEvents = 2 + 2 * 64;
+  cudaStream_t pipe_stream[3] = {};
+  cudaEvent_t pipe_event[kPipeEvents] = {};
+  bool pipe_ready = false;
 
   // per-kernel CUDA-event timing of the most recent `prof_slots` forward calls (CSAT_PROFILE)
   static constexpr int kProfMaxKernels = 8;
@@ -77,6 +82,10 @@ struct csat_ctx {
   // thresholds the kernels read: theta_t of head h at thr()[t * thr_stride() + h]
   const float* thr() const { return w_S ? w_theta : theta; }
   int thr_stride() const { return (w_S && w_layers > 1) ? (int)p.H : 0; }
+
+  // (batch, head) pairs [bh0, bh0 + bh_cnt) the next kernel launches cover; bh_cnt = 0 means all B*H.  A sub-range
+  // lies inside one batch element (csat_forward_host pipelines copies and compute chunk by chunk)
+  int64_t bh0 = 0, bh_cnt = 0;
 
   bool decoder_dirty = true;
   bool have_forward = false;

@@ -419,3 +419,31 @@ def test_tensor_core_edge_shapes():
             err = rel_err(to_np(out), ref)
             assert err <= TOL["bf16"], (B, H, n, nq, d, m, T_run, lam, err)
         ctx.close()
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_pipelined_host_forward_is_bit_identical(d):
+    """csat_forward_host cuts the job into chunks of heads of one batch element (here 2 + 2 + 1 heads per batch
+    element) on its own streams; the result must equal csat_forward on device buffers bit for bit, twice in a row,
+    and with a caller stream other than the default one."""
+    w = wl.Workload("host_pipe", 2, 5, 448, 300, d, 128, "bf16", 3, 0.01, "iid", 41)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    ref = ctx.forward(Q, K, V).cpu()
+    Qh, Kh, Vh = (t.cpu().pin_memory() for t in (Q, K, V))
+    for rep in range(2):
+        oh = torch.full_like(Qh, float("nan")).pin_memory()
+        ctx.forward_host(Qh, Kh, Vh, oh)
+        assert torch.equal(oh, ref), rep
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        oh = torch.full_like(Qh, float("nan")).pin_memory()
+        ctx.forward_host(Qh, Kh, Vh, oh)
+    assert torch.equal(oh, ref)
+    ctx.set(T=0)
+    ref0 = ctx.forward(Q, K, V).cpu()
+    oh = torch.empty_like(Qh).pin_memory()
+    ctx.forward_host(Qh, Kh, Vh, oh)
+    assert torch.equal(oh, ref0)
+    ctx.close()
