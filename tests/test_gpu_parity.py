@@ -447,3 +447,30 @@ def test_pipelined_host_forward_is_bit_identical(d):
     ctx.forward_host(Qh, Kh, Vh, oh)
     assert torch.equal(oh, ref0)
     ctx.close()
+
+
+def test_forward_can_be_captured_in_a_cuda_graph():
+    """csat_forward only enqueues work (no allocation, no synchronisation), so a stream capture records it; replays
+    with new input values in the same buffers give the same output as eager calls."""
+    w = wl.shrink(C["c2"], B=2, H=3)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w, lam=0.0)
+    out = torch.empty_like(Q)
+    ctx.forward(Q, K, V, out)                     # first call: derives the decoder matrices outside the capture
+    torch.cuda.synchronize()
+    eager1 = out.clone()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        ctx.forward(Q, K, V, out)
+    out.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, eager1)
+    Q.copy_(torch.flip(Q, dims=[2]))              # new values, same buffers
+    graph.replay()
+    torch.cuda.synchronize()
+    replayed = out.clone()
+    assert torch.equal(ctx.forward(Q, K, V), replayed)
+    assert not torch.equal(replayed, eager1)
+    ctx.close()
