@@ -117,18 +117,26 @@ def ista(Z: np.ndarray, S_dec: np.ndarray, B_dec: np.ndarray, theta: float, T: i
 
 def lista(Z: np.ndarray, S: np.ndarray, B: np.ndarray, thetas, return_iterates: bool = False):
     """LISTA recurrence with supplied ("learned") weights, row-wise:
-    alpha^{t+1} = eta_{theta_t}(alpha^t S + Z B), t = 0 .. T-1, alpha^0 = 0, T = len(thetas).
+    alpha^{t+1} = eta_{theta_t}(alpha^t S_t + Z B_t), t = 0 .. T-1, alpha^0 = 0, T = len(thetas).
 
-    Z [rows,p], S [q,q], B [p,q], thetas: sequence of T thresholds (one per layer) -> alpha [rows,q].
-    The paper's S, B carry no layer index (shared over the t layers); eta_theta may differ per layer.
+    Z [rows,p]; thetas: sequence of T thresholds (one per layer) -> alpha [rows,q].
+    S [q,q] and B [p,q] (the paper's S, B carry no layer index: shared over the T layers), or one matrix per
+    layer, S [T,q,q] and B [T,p,q] (untied layers: layer t uses S[t], B[t]).
     """
     Z = np.asarray(Z, F64)
     S = np.asarray(S, F64)
-    c = Z @ np.asarray(B, F64)
-    alpha = np.zeros((Z.shape[0], S.shape[0]), dtype=F64)
+    B = np.asarray(B, F64)
+    thetas = list(thetas)
+    if S.ndim != B.ndim:
+        raise ValueError("S and B are both shared over the layers or both per layer")
+    if S.ndim == 3 and not (S.shape[0] == B.shape[0] == len(thetas)):
+        raise ValueError("per-layer weights need one S, one B and one threshold per layer")
+    alpha = np.zeros((Z.shape[0], S.shape[-1]), dtype=F64)
     its = [alpha]
-    for th in thetas:
-        alpha = soft_threshold(alpha @ S + c, th)
+    for t, th in enumerate(thetas):
+        S_t = S[t] if S.ndim == 3 else S
+        B_t = B[t] if B.ndim == 3 else B
+        alpha = soft_threshold(alpha @ S_t + Z @ B_t, th)
         if return_iterates:
             its.append(alpha)
     return (alpha, its) if return_iterates else alpha
@@ -156,8 +164,8 @@ def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, sc
     """CSAT forward for one (batch, head).  Q [n_q,d], K,V [n,d], Phi_h [m,n] -> [n_q,d].
     Phi_v_h: separate measurement matrix for the values (the paper's Phi_V; Phi_h is then Phi_K).  The decoder's
     default D is taken from Phi_V ("Phi = Phi_V is reused as the measurement matrix for decoding").
-    weights = (S [d,d], B [d,d], thetas [T]) replaces the ISTA-derived decoder by supplied LISTA weights
-    (lam, D and step are then unused)."""
+    weights = (S, B, thetas [T]) with S, B [d,d] or per layer [T,d,d] replaces the ISTA-derived decoder by
+    supplied LISTA weights (lam, D and step are then unused)."""
     Q = np.asarray(Q, F64)
     d = Q.shape[1]
     Phi_v = Phi_h if Phi_v_h is None else Phi_v_h
@@ -200,8 +208,12 @@ def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=Non
             psi_h = None if Psi is None else (Psi if np.ndim(Psi) == 2 else Psi[h])
             D_h = None if D is None else D[h]
             st = {} if stages is not None else None
-            # weights = (S [H,d,d], B [H,d,d], thetas [T,H])
-            w_h = None if weights is None else (weights[0][h], weights[1][h], [th[h] for th in weights[2]])
+            # weights = (S, B, thetas [T,H]) with S, B [H,d,d] (shared over the layers) or [T,H,d,d] (per layer)
+            w_h = None
+            if weights is not None:
+                per_layer = np.ndim(weights[0]) == 4
+                w_h = (np.asarray(weights[0])[:, h] if per_layer else weights[0][h],
+                       np.asarray(weights[1])[:, h] if per_layer else weights[1][h], [th[h] for th in weights[2]])
             out[b, h] = csat_forward_head(Q[b, h], K[b, h], V[b, h], Phi[h], T=T, lam=lam,
                                           Psi=psi_h, D=D_h, step=step, scale=scale, stages=st, weights=w_h,
                                           Phi_v_h=None if Phi_V is None else Phi_V[h])

@@ -103,6 +103,27 @@ def _lista_drop_input(Z, S, B, thetas, return_iterates=False):
     return alpha
 
 
+def _lista_first_layer_everywhere(Z, S, B, thetas, return_iterates=False):
+    S, B = np.asarray(S, F64), np.asarray(B, F64)
+    if S.ndim == 3:
+        S, B = S[0], B[0]
+    return _orig_lista(Z, S, B, thetas, return_iterates)
+
+
+def _lista_B_one_layer_late(Z, S, B, thetas, return_iterates=False):
+    B = np.asarray(B, F64)
+    if B.ndim == 3:
+        B = np.roll(B, 1, axis=0)
+    return _orig_lista(Z, S, B, thetas, return_iterates)
+
+
+def _lista_layers_reversed(Z, S, B, thetas, return_iterates=False):
+    S, B = np.asarray(S, F64), np.asarray(B, F64)
+    if S.ndim == 3:
+        S, B = S[::-1], B[::-1]
+    return _orig_lista(Z, S, B, thetas, return_iterates)
+
+
 _orig_lista = orc.lista
 _orig_setup = orc.decoder_setup
 _orig_ista = orc.ista
@@ -125,6 +146,9 @@ MUTATIONS = {
     "lista: S transposed": ("lista", _lista_S_transposed),
     "lista: per-layer thresholds ignored": ("lista", _lista_first_theta_everywhere),
     "lista: input only in the first layer": ("lista", _lista_drop_input),
+    "lista: first layer's matrices in every layer": ("lista", _lista_first_layer_everywhere),
+    "lista: B of the layer before": ("lista", _lista_B_one_layer_late),
+    "lista: layers in reverse order": ("lista", _lista_layers_reversed),
     "compress: |Phi|": ("compress", _compress_abs),
     "output: weights ignored": ("compressed_output", _output_uses_unweighted),
 }

@@ -429,6 +429,78 @@ def test_lista_special_cases():
     assert not np.allclose(orc.lista(Z, Sn, B, [0.1] * 3), orc.lista(Z, Sn.T, B, [0.1] * 3))
 
 
+def test_lista_per_layer_weights_match_scalar_loops():
+    """Brute force with a different S_t, B_t and theta_t in every layer."""
+    r = np.random.default_rng(24)
+    p, q, rows, T = 3, 4, 2, 3
+    S = r.standard_normal((T, q, q)) * 0.4
+    B = r.standard_normal((T, p, q))
+    Z = r.standard_normal((rows, p))
+    thetas = [0.25, 0.02, 0.15]
+    alpha = [[0.0] * q for _ in range(rows)]
+    for t in range(T):
+        new = [[0.0] * q for _ in range(rows)]
+        for i in range(rows):
+            for b in range(q):
+                x = sum(alpha[i][a] * S[t][a][b] for a in range(q)) + sum(Z[i][a] * B[t][a][b] for a in range(p))
+                new[i][b] = (abs(x) - thetas[t]) * (1 if x > 0 else -1) if abs(x) > thetas[t] else 0.0
+        alpha = new
+    assert np.allclose(orc.lista(Z, S, B, thetas), np.array(alpha), rtol=0, atol=1e-14)
+
+
+def test_lista_per_layer_weights_closed_forms():
+    r = np.random.default_rng(25)
+    T, q = 4, 5
+    Z = r.standard_normal((6, q))
+    S = r.standard_normal((T, q, q)) * 0.5
+    B = r.standard_normal((T, q, q))
+    # theta = 0: the recurrence is linear, alpha^T = sum_t Z B_t S_{t+1} S_{t+2} ... S_{T-1}
+    want = np.zeros((6, q))
+    for t in range(T):
+        term = Z @ B[t]
+        for u in range(t + 1, T):
+            term = term @ S[u]
+        want += term
+    assert np.allclose(orc.lista(Z, S, B, [0.0] * T), want, rtol=0, atol=1e-12)
+    # the layers do not commute: the reversed stack gives something else
+    assert not np.allclose(orc.lista(Z, S[::-1], B[::-1], [0.0] * T), want)
+    # S_t = 0 in the last layer: only that layer's B and threshold count
+    S0 = S.copy()
+    S0[-1] = 0.0
+    assert np.array_equal(orc.lista(Z, S0, B, [0.3, 0.2, 0.1, 0.05]), orc.soft_threshold(Z @ B[-1], 0.05))
+    # the same matrix in every layer is the shared form
+    th = [0.2, 0.1, 0.3, 0.05]
+    tied = orc.lista(Z, S[1], B[2], th)
+    assert np.array_equal(orc.lista(Z, np.stack([S[1]] * T), np.stack([B[2]] * T), th), tied)
+    # one S, one B and one threshold per layer, or an error
+    for bad in [(S[:3], B, th), (S, B[:3], th), (S, B, th[:3]), (S, B[0], th)]:
+        try:
+            orc.lista(Z, *bad)
+        except ValueError:
+            continue
+        raise AssertionError("inconsistent per-layer weights accepted")
+
+
+def test_forward_with_per_layer_weights_uses_them():
+    """The whole forward hands layer t of head h its own matrices: equal to the stages composed by hand."""
+    r = np.random.default_rng(26)
+    Bt, H, n, nq, d, m, T = 2, 2, 12, 5, 4, 6, 3
+    Q, K, V = (r.standard_normal((Bt, H, s, d)) for s in (nq, n, n))
+    Phi = r.standard_normal((H, m, n)) / np.sqrt(m)
+    S = r.standard_normal((T, H, d, d)) * 0.4
+    Bm = r.standard_normal((T, H, d, d)) * 0.6
+    th = np.abs(r.standard_normal((T, H))) * 0.05
+    Psi = r.standard_normal((d, d))
+    out = orc.csat_forward(Q, K, V, Phi, T=T, lam=0.0, Psi=Psi, weights=(S, Bm, list(th)))
+    for b in range(Bt):
+        for h in range(H):
+            Z = orc.csat_forward_head(Q[b, h], K[b, h], V[b, h], Phi[h], T=0, lam=0.0)
+            a = np.zeros((nq, d))
+            for t in range(T):
+                a = orc.soft_threshold(a @ S[t, h] + Z @ Bm[t, h], th[t, h])
+            assert np.allclose(out[b, h], a @ Psi.T, rtol=0, atol=1e-13)
+
+
 def test_forward_with_supplied_weights_uses_them():
     w = wl.shrink(wl.CONFIGS["c1"], n=32, n_q=8, m=16, d=8)
     inp = wl.make_inputs(w)
