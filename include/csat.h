@@ -64,8 +64,8 @@ enum {
   CSAT_FORCE_SIMT = 5, /* diagnostic: 1 routes bf16 through the plain FFMA kernels, 2 only
                           the attention/recovery stage; 0 (default) = tensor-core kernels */
   CSAT_ENSEMBLE = 7,   /* measurement ensemble: CSAT_ENSEMBLE_GAUSSIAN (default), N(0, 1/m) entries, or
-                          CSAT_ENSEMBLE_RADEMACHER, +-1/sqrt(m) entries (paper: "random Gaussian,
-                          Rademacher, or structured Hadamard matrices"), or CSAT_ENSEMBLE_HADAMARD:
+                          CSAT_ENSEMBLE_RADEMACHER, +-1/sqrt(m) entries, or CSAT_ENSEMBLE_HADAMARD (the
+                          three ensembles the paper lists after the compression equation):
                           m rows (a r + b mod N, a odd) of the N x N Sylvester-Hadamard matrix, N the
                           smallest power of two >= n, columns truncated to n, a random sign per
                           column, scaled by 1/sqrt(m).  Changing it regenerates Phi from the seed  */
@@ -123,7 +123,7 @@ int csat_get_i64(const csat_ctx* ctx, int key, int64_t* value_host);
 int csat_set_f64(csat_ctx* ctx, int key, double value);
 int csat_get_f64(const csat_ctx* ctx, int key, double* value_host);
 
-/* csat_set_phi / csat_get_phi -- paper: "fixed or learned" measurement matrices.
+/* csat_set_phi / csat_get_phi -- the paper allows measurement matrices that are fixed or trained.
  * phi: [H, m, n] dense, context dtype.  set overrides the seeded matrix (copied into the
  * library's padded storage); get writes the matrix in use.  Enqueued on `stream`. */
 int csat_set_phi(csat_ctx* ctx, const void* phi, void* stream);
@@ -134,14 +134,14 @@ int csat_get_phi(const csat_ctx* ctx, void* phi_out, void* stream);
  * (Psi[a][b] multiplies alpha_b).  NULL restores Psi = I.  Copied on `stream`. */
 int csat_set_dictionary(csat_ctx* ctx, const void* psi, int per_head, void* stream);
 
-/* csat_set_decoder_matrix -- paper: "Phi = Phi_V is reused as the measurement matrix for
- * decoding"; the decoder's sensing matrix D is d x d (see file header).  D: [H, d, d], context
+/* csat_set_decoder_matrix -- the paper decodes with the values' measurement matrix;
+ * the decoder's sensing matrix D is d x d (see file header).  D: [H, d, d], context
  * dtype.  NULL restores the default D_h = Phi_h[0:d, 0:d], which needs m >= d and n >= d
  * (otherwise csat_forward with T > 0 returns CSAT_ERR_SHAPE).  Copied on `stream`. */
 int csat_set_decoder_matrix(csat_ctx* ctx, const void* D, void* stream);
 
-/* csat_set_lista_weights -- paper: LISTA recurrence alpha^{t+1} = eta_theta(S alpha^t + B Z_i), where "S, B and
- * eta_theta are learned weight matrices and nonlinearities" shared by the t layers.  Replaces the ISTA-derived
+/* csat_set_lista_weights -- paper: LISTA recurrence alpha^{t+1} = eta_theta(S alpha^t + B Z_i), whose matrices
+ * S, B and shrinkage eta_theta are trained and carry no layer index.  Replaces the ISTA-derived
  * decoder by supplied weights, row-vector convention alpha <- eta(alpha S + z B):
  *   S, Bm   [H, d, d], context dtype, device (row-major: S[a][b] multiplies alpha_a into column b)
  *   theta   [layers, H] float32, device, every entry >= 0; layers = 1 uses the same threshold in every
@@ -150,6 +150,19 @@ int csat_set_decoder_matrix(csat_ctx* ctx, const void* D, void* stream);
  * weights are in force; the dictionary Psi still applies to the reconstruction.  S = NULL restores the
  * ISTA-derived decoder.  On the bf16 tensor-core path S enters as I - W with W = I - S rounded to bf16. */
 int csat_set_lista_weights(csat_ctx* ctx, const void* S, const void* Bm, const float* theta, int layers, void* stream);
+
+/* csat_set_lista_layer_weights -- the same LISTA recurrence with untied layers: layer t has its own matrices,
+ * alpha^{t+1} = eta_{theta_t}(alpha^t S_t + z B_t), t = 0 .. layers-1 (the paper's recurrence writes S, B
+ * without a layer index; one matrix per layer is the usual generalisation of the unrolled decoder).
+ *   S, Bm   [layers, H, d, d], context dtype, device (row-major as in csat_set_lista_weights)
+ *   theta   [layers, H] float32, device, every entry >= 0
+ * 1 <= layers <= 4096, and layers must equal CSAT_T when csat_forward runs (else CSAT_ERR_STATE).  Copied on `stream`; replaces weights
+ * set by csat_set_lista_weights and is cleared by csat_set_lista_weights(ctx, NULL, ...).  csat_get_decoder
+ * then returns layer 0's S, B and theta.  On the bf16 tensor-core path every layer is one product
+ * [alpha^t | z] [S_t - I ; B_t] with bf16 operands, added to alpha^t kept in float32; the matrices
+ * of layer t stream through shared memory while layer t-1 is computed. */
+int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, const float* theta, int layers,
+                                 void* stream);
 
 /*
  * csat_forward -- paper: compression, approximate attention matrix, compressed output,

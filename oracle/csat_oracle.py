@@ -163,7 +163,7 @@ def csat_forward_head(Q, K, V, Phi_h, *, T, lam, Psi=None, D=None, step=None, sc
                       stages: dict | None = None, weights=None, Phi_v_h=None) -> np.ndarray:
     """CSAT forward for one (batch, head).  Q [n_q,d], K,V [n,d], Phi_h [m,n] -> [n_q,d].
     Phi_v_h: separate measurement matrix for the values (the paper's Phi_V; Phi_h is then Phi_K).  The decoder's
-    default D is taken from Phi_V ("Phi = Phi_V is reused as the measurement matrix for decoding").
+    default D is taken from Phi_V (the paper decodes with the values' measurement matrix).
     weights = (S, B, thetas [T]) with S, B [d,d] or per layer [T,d,d] replaces the ISTA-derived decoder by
     supplied LISTA weights (lam, D and step are then unused)."""
     Q = np.asarray(Q, F64)

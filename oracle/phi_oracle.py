@@ -2,7 +2,7 @@
 
 Only tests, the smoke check and the benchmark's CPU-baseline leg import this.
 
-The paper draws Phi from a sub-Gaussian ensemble ("random Gaussian", section
+The paper draws Phi from a sub-Gaussian ensemble (Gaussian entries first among its examples; section
 "Mathematical Framework", the sentence after the compression equation) and fixes
 neither generator nor variance.  The reading implemented here (and, separately,
 by the CUDA library):

@@ -38,6 +38,7 @@ SIGNATURES = {
     "csat_set_dictionary": (_int, [_vp, _vp, _int, _vp]),
     "csat_set_decoder_matrix": (_int, [_vp, _vp, _vp]),
     "csat_set_lista_weights": (_int, [_vp, _vp, _vp, _vp, _int, _vp]),
+    "csat_set_lista_layer_weights": (_int, [_vp, _vp, _vp, _vp, _int, _vp]),
     "csat_forward": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_forward_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
@@ -152,6 +153,10 @@ def csat_set_decoder_matrix(h, D, stream=None):
 
 def csat_set_lista_weights(h, S, Bm, theta, layers, stream=None):
     _check(h, load().csat_set_lista_weights(h, _ptr(S), _ptr(Bm), _ptr(theta), int(layers), _stream(stream)))
+
+
+def csat_set_lista_layer_weights(h, S, Bm, theta, layers, stream=None):
+    _check(h, load().csat_set_lista_layer_weights(h, _ptr(S), _ptr(Bm), _ptr(theta), int(layers), _stream(stream)))
 
 
 def csat_forward(h, Q, K, V, out, stream=None):
@@ -321,6 +326,14 @@ class Csat:
         assert S.shape == (self.H, self.d, self.d) and Bm.shape == S.shape and S.dtype == self.torch_dtype == Bm.dtype
         theta = theta.reshape(-1, self.H).to(torch.float32).contiguous()
         csat_set_lista_weights(self.h, S.contiguous(), Bm.contiguous(), theta, theta.shape[0])
+
+    def set_lista_layer_weights(self, S, Bm, theta):
+        """Untied layers: S, Bm [layers,H,d,d] (context dtype), theta [layers,H] float32."""
+        L = S.shape[0]
+        assert S.shape == (L, self.H, self.d, self.d) and Bm.shape == S.shape and S.dtype == self.torch_dtype == Bm.dtype
+        theta = theta.to(torch.float32).contiguous()
+        assert theta.shape == (L, self.H)
+        csat_set_lista_layer_weights(self.h, S.contiguous(), Bm.contiguous(), theta, L)
 
     def get_compressed(self):
         kt = self._new(self.B, self.H, self.m, self.d)

@@ -39,6 +39,12 @@
 // the increment that multiplies mu G is rounded to bf16, and c never needs registers of its own.  The
 // saturating form of the shrinkage runs on the FMA pipe (two-element packed instructions where they exist);
 // it leaves O(1e-7 theta) instead of exact zeros, so the last iteration uses the exact min/max form.
+//
+// Untied layers (one S_t, B_t per layer, kUntied): no running accumulator is possible, so every layer is one fresh
+// product r_t = [a^_t | z^] [S_t - I ; B_t] (K = 2 d, both operands bf16 in tensor memory, z^ written once) and
+// x = alpha^t + r_t with alpha^t exact in registers.  The matrices of layer t take ring positions after the
+// item's chunks (S_t - I in the K~ slots, B_t in the V~ slots), so layer t + 1 is loaded while layer t is computed.
+// The registers hold alpha^t + theta_t, which turns the shrinkage into y - 2 theta sat(y / (2 theta)).
 #include "csat_internal.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -76,7 +82,7 @@ template <int D> struct Cfg {
   // P_j overlays S[j&1]; the recovery operand overlays S[0].
   static constexpr uint32_t kTileCols = 256, kColS = 0, kColAcc = 2 * kMC, kTmemCols = 512;
   static_assert(2 * kMC + D <= 256, "TMEM budget");
-  static_assert(D / 2 <= 2 * kMC, "recovery operand fits in the S columns");
+  static_assert(D <= 2 * kMC, "recovery operands (z and alpha, D / 2 packed columns each) fit in the S columns");
   static_assert(kStages >= kDBoxes && kStages <= kMaxStages, "mu G and Psi are staged box by box in ring slots");
   static_assert(kMatBoxBytes <= kSlotBytes && kMatBytes <= kQBytes, "decoder matrices fit where they are staged");
   static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
@@ -182,7 +188,7 @@ struct Waiter {
   }
 };
 
-template <int D>
+template <int D, bool kUntied>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
@@ -204,7 +210,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   // parities follow, so that the TMA and MMA warps can run ahead into the next item while the compute threads
   // finish the current one.
   const int nchunks = (m + kMC - 1) / kMC;
-  const int nvirt = T > 0 ? C::kDBoxes : 0;     // ring positions an item's decoder matrices take after its chunks
+  // ring positions an item's decoder matrices take after its chunks: mu G | Psi once, or one set per untied layer
+  const int nlayers = T > 0 ? T + (has_psi ? 1 : 0) : 0;        // recovery MMAs per tile and item
+  const int nvirt = T > 0 ? (kUntied ? C::kDBoxes * nlayers : C::kDBoxes) : 0;
   Waiter w{status, &bars->abort};
   auto k_slot = [&](int s) { return ring + (2 * s) * C::kSlotBytes; };
   auto v_slot = [&](int s) { return ring + (2 * s + 1) * C::kSlotBytes; };
@@ -287,7 +295,33 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             tma_load_3d(v_slot(s) + gx * C::kBoxBytes, &tmap_kv, &bars->v_full[s], D + gx * 64, j * kMC, bh);
           v_hist |= 1u;
         }
-        if (T > 0 && !w.dead) {
+        if (kUntied && T > 0 && !w.dead) {
+          // layer l: S_l - I to the K~ slots, B_l to the V~ slots; after the last layer Psi to V~ slots
+          const int mat0 = h * (2 * T + 1);
+          for (int l = 0; l < nlayers && !w.dead; ++l) {
+            const bool psi_l = (l == T);
+            for (int gx = 0; gx < C::kDBoxes && !w.dead; ++gx, ++g) {
+              const int s = g % C::kStages;
+              ring_wait_k(g, 206);
+              if (w.dead) break;
+              if (!psi_l) {
+                mbar_arrive_expect_tx(&bars->k_full[s], C::kMatBoxBytes);
+                tma_load_3d(k_slot(s), &tmap_mats, &bars->k_full[s], gx * 64, 0, mat0 + 2 * l);
+                k_hist = (k_hist << 1) | 1u;
+              } else {
+                mbar_arrive(&bars->k_full[s]);   // nothing to load: complete the phase so that the parities stay in step
+                k_hist <<= 1;
+              }
+              v_hist <<= 1;
+              ring_wait_v(g, 207);
+              if (w.dead) { ++g; break; }
+              mbar_arrive_expect_tx(&bars->v_full[s], C::kMatBoxBytes);
+              tma_load_3d(v_slot(s), &tmap_mats, &bars->v_full[s], gx * 64, 0, mat0 + (psi_l ? 2 * T : 2 * l + 1));
+              v_hist |= 1u;
+            }
+          }
+        }
+        if (!kUntied && T > 0 && !w.dead) {
           // every S MMA of the item has finished once the last one has: tile A's Q buffer is free for B
           const uint32_t gl = g - 1;
           w.wait(&bars->k_empty[gl % C::kStages], (gl / C::kStages) & 1, 203);
@@ -400,14 +434,55 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           if (j == nchunks - 1) {
             // the Q buffers have been read for the last time (tile A's still takes B when there is a recovery)
             if (ntiles == 2) mma_commit(&bars->q_free[1]);
-            if (T == 0) mma_commit(&bars->q_free[0]);
+            if (T == 0 || kUntied) mma_commit(&bars->q_free[0]);
           }
           if (j > 0) issue_pv(j - 1);
         }
         issue_pv(nchunks - 1);
-        if (T > 0) {
+        if (kUntied && T > 0) {
+          // layer l: r = z^ B_l (+ a^_l (S_l - I) from the second layer on); then Psi on the final alpha
+          for (int l = 0; l < nlayers; ++l) {
+            const bool psi_l = (l == T);
+            const uint32_t pl = g + nchunks + l * C::kDBoxes;     // ring position of the layer's first box
+            for (int gx = 0; gx < C::kDBoxes; ++gx) {
+              const uint32_t pos = pl + gx;
+              w.wait(&bars->k_full[pos % C::kStages], (pos / C::kStages) & 1, 215);
+              w.wait(&bars->v_full[pos % C::kStages], (pos / C::kStages) & 1, 215);
+            }
+#pragma unroll
+            for (int t = 0; t < kTiles; ++t) {
+              if (t < ntiles) {
+                w.wait(&bars->a_full[t], (ab[t] + l) & 1, 216);
+                tc_fence_after();
+                const uint32_t tb = tmem + t * C::kTileCols;
+                const uint32_t z_cols = tb + C::kColS, a_cols = tb + C::kColS + D / 2;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                  // the V~ slot of the layer's box k / 4: B_l (A operand z^), or Psi (A operand the final alpha)
+                  const uint64_t wd = ring_k0 + (uint64_t)((pl + k / 4) % C::kStages) * kStageStep +
+                                      (uint64_t)(C::kSlotBytes >> 4) + (uint64_t)((k % 4) * 2);
+                  mma_f16_ts(tb + C::kColAcc, (psi_l ? a_cols : z_cols) + k * 8, wd, idesc_r, k == 0 ? 0u : 1u);
+                }
+                if (!psi_l && l > 0) {
+#pragma unroll
+                  for (int k = 0; k < D / 16; ++k) {
+                    const uint64_t wd = ring_k0 + (uint64_t)((pl + k / 4) % C::kStages) * kStageStep +
+                                        (uint64_t)((k % 4) * 2);                                   // S_l - I
+                    mma_f16_ts(tb + C::kColAcc, a_cols + k * 8, wd, idesc_r, 1u);
+                  }
+                }
+                mma_commit(&bars->r_full[t]);
+              }
+            }
+            for (int gx = 0; gx < C::kDBoxes; ++gx) {     // both tiles have read the layer's matrices
+              mma_commit(&bars->k_empty[(pl + gx) % C::kStages]);
+              mma_commit(&bars->v_empty[(pl + gx) % C::kStages]);
+            }
+          }
+        }
+        if (!kUntied && T > 0) {
           const uint32_t gv = g + nchunks;            // ring position of the first box of mu G / Psi
-          const int n_mma = T + (has_psi ? 1 : 0);    // r_0 = theta + z B, then T-1 increments with mu G, then Psi
+          const int n_mma = nlayers;                  // r_0 = theta + z B, then T-1 increments with mu G, then Psi
           for (int i = 0; i < n_mma; ++i) {
             const bool first = (i == 0), psi_step = has_psi && i == n_mma - 1;
             if (first) w.wait(&bars->mats_full, items_done & 1, 214);
@@ -447,7 +522,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         g += nchunks + nvirt;
 #pragma unroll
         for (int t = 0; t < kTiles; ++t)
-          if (t < ntiles) { cb[t] += nchunks; ab[t] += T > 0 ? T + (has_psi ? 1 : 0) : 0; }
+          if (t < ntiles) { cb[t] += nchunks; ab[t] += nlayers; }
       }
     }
   }
@@ -579,8 +654,8 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           for (int e = 0; e < 16; e += 2) v2[(c0 + e) >> 1] = mul2(pack2u(a[e], a[e + 1]), inv2);
         }
       }
-      auto publish = [&]() {                                    // v2 as the bf16 A operand of the next MMA
-        const uint32_t op_addr = tbase + C::kColS;
+      auto publish = [&](uint32_t col) {                        // v2 as a bf16 A operand, from column col of S on
+        const uint32_t op_addr = tbase + C::kColS + col;
 #pragma unroll
         for (int c0 = 0; c0 < D; c0 += 16) {
           uint32_t pk[8];
@@ -597,7 +672,87 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         mbar_arrive(&bars->a_full[t]);
       };
 
-      if (T > 0) {
+      if (kUntied && T > 0) {
+        // z^ in the first D / 2 packed columns (written once), a^_t in the next D / 2.  The registers hold
+        // y-offset iterates b_t = alpha^t + theta_t, so that x + theta_t = b_t + r_t needs no add of its own;
+        // the layer before the last adds nothing, because the last layer shrinks exactly from x = alpha + r.
+        const uint32_t a_addr = tbase + C::kColS + D / 2;
+        publish(0);
+        {
+          const float b0 = T > 1 ? theta[h] : 0.f;
+#pragma unroll
+          for (int i = 0; i < D / 2; ++i) v2[i] = pack2(b0, b0);      // alpha^0 = 0
+        }
+        for (int it = 0; it + 1 < T; ++it) {
+          const float th = theta[(int64_t)it * theta_stride + h];
+          const float thn = it + 2 < T ? theta[(int64_t)(it + 1) * theta_stride + h] : 0.f;
+          const float inv2th = th > 0.f ? 0.5f / th : 0.f;          // theta = 0: sat(0) = 0 and eta(x) = x
+          const uint64_t m2th2 = pack2(-2.f * th, -2.f * th);
+          const uint64_t nx2 = pack2(thn, thn);
+          w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
+          tc_fence_after();
+          auto shrink16 = [&](const uint32_t (&r)[16], int c0) {
+            uint32_t pk[8];
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) {
+              const uint64_t y2 = add2(v2[(c0 + e) >> 1], pack2u(r[e], r[e + 1]));   // alpha^t S_t + z B_t + theta_t
+              float y0, y1;
+              unpack2(y2, y0, y1);
+              const uint64_t t2 = pack2(fma_sat(y0, inv2th, 0.f), fma_sat(y1, inv2th, 0.f));
+              const uint64_t an = fma2(t2, m2th2, y2);                               // alpha^{t+1} = eta_theta(x)
+              v2[(c0 + e) >> 1] = add2(an, nx2);
+              float a0, a1;
+              unpack2(an, a0, a1);
+              pk[e >> 1] = pack_bf16(a0, a1);
+            }
+            tmem_st_32x32b_x8(a_addr + c0 / 2, pk);
+          };
+          uint32_t r0[16], r1[16];
+          tmem_ld_32x32b_x16(acc_addr, r0);
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            tmem_wait_ld();
+            tmem_ld_32x32b_x16(acc_addr + c0 + 16, r1);
+            shrink16(r0, c0);
+            tmem_wait_ld();
+            if (c0 + 32 < D) tmem_ld_32x32b_x16(acc_addr + c0 + 32, r0);
+            shrink16(r1, c0 + 16);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&bars->a_full[t]);
+        }
+        const float th = theta[(int64_t)(T - 1) * theta_stride + h];
+        w.wait(&bars->r_full[t], phase & 1, 231); ++phase;
+        tc_fence_after();
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(acc_addr + c0, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) {
+            float b0, b1;
+            unpack2(v2[(c0 + e) >> 1], b0, b1);
+            const float x0 = b0 + __uint_as_float(r[e]), x1 = b1 + __uint_as_float(r[e + 1]);
+            v2[(c0 + e) >> 1] = pack2(x0 - fminf(fmaxf(x0, -th), th), x1 - fminf(fmaxf(x1, -th), th));
+          }
+        }
+        if (has_psi) {
+          publish(D / 2);
+          w.wait(&bars->r_full[t], phase & 1, 232); ++phase;
+          tc_fence_after();
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld_32x32b_x16(acc_addr + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) v2[(c0 + e) >> 1] = pack2u(r[e], r[e + 1]);
+          }
+        }
+      }
+      if (!kUntied && T > 0) {
         // layer t uses theta[t * theta_stride + h] (stride 0: one threshold for all layers).  The accumulator is
         // biased by kappa = theta of layer 0 and the registers hold b = alpha - kappa throughout.
         const uint32_t op_addr = tbase + C::kColS;
@@ -609,7 +764,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
 #pragma unroll
           for (int c0 = 0; c0 < D; c0 += 16) tmem_st_32x32b_x16(acc_addr + c0, tb);
         }
-        publish();
+        publish(0);
 #pragma unroll
         for (int i = 0; i < D / 2; ++i) v2[i] = pack2(-kappa, -kappa);  // alpha^0 = 0
         // per_layer is a compile-time tag: with one threshold for all layers theta_t - kappa = 0 and the add of it
@@ -676,7 +831,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
         if (has_psi) {
-          publish();
+          publish(0);
           w.wait(&bars->r_full[t], phase & 1, 232); ++phase;
           tc_fence_after();
 #pragma unroll
@@ -707,7 +862,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   if (warp == kMmaWarp) tmem_dealloc(tmem, C::kTmemCols);
 }
 
-template <int D>
+template <int D, bool kUntied>
 cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   using C = Cfg<D>;
   const Params& p = c->p;
@@ -719,7 +874,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
   static bool attr_set = false;
   if (!attr_set) {
-    e = cudaFuncSetAttribute(attend_recover_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(attend_recover_sm100_kernel<D, kUntied>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)C::kSmemBytes);
     if (e != cudaSuccess) return e;
     attr_set = true;
@@ -739,8 +894,8 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
       sms = 148;
   }
   const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
-  attend_recover_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(
-      tq, c->tmap_kv, c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, p.T,
+  attend_recover_sm100_kernel<D, kUntied><<<grid, kThreads, C::kSmemBytes, s>>>(
+      tq, c->tmap_kv, kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, p.T,
       c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, (int)c->bh0, c->status);
   return cudaGetLastError();
 }
@@ -761,9 +916,21 @@ cudaError_t make_attend_tmaps(csat_ctx* c) {
   return make_tmap_bf16_3d(&c->tmap_mats, c->mats_bf16, md, ms, mb);
 }
 
+// tensor map over the per-layer operands [H (2 L + 1)][d][d] of untied layers
+cudaError_t make_layer_weights_tmap(csat_ctx* c) {
+  const Params& p = c->p;
+  const uint64_t md[3] = {(uint64_t)p.d, (uint64_t)p.d, (uint64_t)(p.H * (2 * c->w_layers + 1))};
+  const uint64_t ms[2] = {(uint64_t)p.d * 2, (uint64_t)p.d * p.d * 2};
+  const uint32_t mb[3] = {64, (uint32_t)p.d, 1};
+  return make_tmap_bf16_3d(&c->tmap_lmats, c->lmats_bf16, md, ms, mb);
+}
+
 cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches) {
   *launches += 1;
-  return c->p.d == 64 ? launch<64>(c, Q, out, s) : launch<128>(c, Q, out, s);
+  // with untied layers and T > 0 the per-layer kernel; the set-up has then built its operands for exactly T layers
+  if (c->w_S && c->w_untied && c->p.T > 0)
+    return c->p.d == 64 ? launch<64, true>(c, Q, out, s) : launch<128, true>(c, Q, out, s);
+  return c->p.d == 64 ? launch<64, false>(c, Q, out, s) : launch<128, false>(c, Q, out, s);
 }
 
 }  // namespace csat

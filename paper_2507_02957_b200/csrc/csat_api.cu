@@ -55,10 +55,15 @@ void prof_destroy(csat_ctx* c);
 
 void free_lista(csat_ctx* c) {
   const csat::Params& p = c->p;
-  dev_free(c, &c->w_S, dd_bytes(p, csat::elt_size(p.dtype)));
-  dev_free(c, &c->w_B, dd_bytes(p, csat::elt_size(p.dtype)));
+  const size_t mats = c->w_mat_count();
+  dev_free(c, &c->w_S, mats * csat::elt_size(p.dtype));
+  dev_free(c, &c->w_B, mats * csat::elt_size(p.dtype));
   dev_free(c, &c->w_theta, (size_t)c->w_layers * p.H * 4);
+  dev_free(c, &c->Sl_dec, mats * 4);
+  dev_free(c, &c->Bl_dec, mats * 4);
+  dev_free(c, &c->lmats_bf16, (size_t)(2 * c->w_layers + 1) * dd_bytes(p, 2));
   c->w_layers = 0;
+  c->w_untied = false;
 }
 
 void free_staging(csat_ctx* c) {
@@ -415,7 +420,8 @@ int csat_set_decoder_matrix(csat_ctx* c, const void* D, void* stream) {
   return CSAT_OK;
 }
 
-int csat_set_lista_weights(csat_ctx* c, const void* S, const void* Bm, const float* theta, int layers, void* stream) {
+static int set_weights(csat_ctx* c, const void* S, const void* Bm, const float* theta, int layers, bool untied,
+                       void* stream, const char* who) {
   if (!c) return CSAT_ERR_INVALID_ARG;
   csat::Params& p = c->p;
   c->decoder_dirty = true;
@@ -423,26 +429,49 @@ int csat_set_lista_weights(csat_ctx* c, const void* S, const void* Bm, const flo
     if (c->w_S) { cudaDeviceSynchronize(); free_lista(c); }
     return CSAT_OK;
   }
-  if (!Bm || !theta) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_lista_weights: NULL pointer");
-  if (!aligned16(S) || !aligned16(Bm)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_lista_weights: misaligned pointer");
-  if (layers < 1 || layers > 100000) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_lista_weights: layers must be >= 1");
-  const size_t mat_bytes = dd_bytes(p, csat::elt_size(p.dtype));
-  if (c->w_S && c->w_layers != layers) { cudaDeviceSynchronize(); free_lista(c); }
+  const std::string name(who);
+  if (!Bm || !theta) return fail(c, CSAT_ERR_INVALID_ARG, name + ": NULL pointer");
+  if (!aligned16(S) || !aligned16(Bm)) return fail(c, CSAT_ERR_INVALID_ARG, name + ": misaligned pointer");
+  if (layers < 1 || layers > 100000) return fail(c, CSAT_ERR_INVALID_ARG, name + ": layers must be >= 1");
+  if (c->w_S && (c->w_layers != layers || c->w_untied != untied)) { cudaDeviceSynchronize(); free_lista(c); }
+  const size_t elt = csat::elt_size(p.dtype);
   if (!c->w_S) {
     c->w_layers = layers;
-    if (dev_alloc(c, &c->w_S, mat_bytes) != cudaSuccess || dev_alloc(c, &c->w_B, mat_bytes) != cudaSuccess ||
-        dev_alloc(c, &c->w_theta, (size_t)layers * p.H * 4) != cudaSuccess) {
+    c->w_untied = untied;
+    const size_t mats = c->w_mat_count();
+    bool ok = dev_alloc(c, &c->w_S, mats * elt) == cudaSuccess && dev_alloc(c, &c->w_B, mats * elt) == cudaSuccess &&
+              dev_alloc(c, &c->w_theta, (size_t)layers * p.H * 4) == cudaSuccess;
+    if (ok && untied) {
+      ok = dev_alloc(c, &c->Sl_dec, mats * 4) == cudaSuccess && dev_alloc(c, &c->Bl_dec, mats * 4) == cudaSuccess;
+      if (ok && p.dtype == CSAT_DTYPE_BF16 && (p.d == 64 || p.d == 128))
+        ok = dev_alloc(c, &c->lmats_bf16, (size_t)(2 * layers + 1) * dd_bytes(p, 2)) == cudaSuccess &&
+             csat::make_layer_weights_tmap(c) == cudaSuccess;
+    }
+    if (!ok) {
+      cudaGetLastError();
       free_lista(c);
       return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(LISTA weights) failed");
     }
   }
   cudaStream_t s = (cudaStream_t)stream;
+  const size_t mat_bytes = c->w_mat_count() * elt;
   cudaError_t e;
   if ((e = cudaMemcpyAsync(c->w_S, S, mat_bytes, cudaMemcpyDeviceToDevice, s)) != cudaSuccess ||
       (e = cudaMemcpyAsync(c->w_B, Bm, mat_bytes, cudaMemcpyDeviceToDevice, s)) != cudaSuccess ||
       (e = cudaMemcpyAsync(c->w_theta, theta, (size_t)layers * p.H * 4, cudaMemcpyDeviceToDevice, s)) != cudaSuccess)
-    return fail_cuda(c, e, "csat_set_lista_weights");
+    return fail_cuda(c, e, who);
   return CSAT_OK;
+}
+
+int csat_set_lista_weights(csat_ctx* c, const void* S, const void* Bm, const float* theta, int layers, void* stream) {
+  return set_weights(c, S, Bm, theta, layers, false, stream, "csat_set_lista_weights");
+}
+
+int csat_set_lista_layer_weights(csat_ctx* c, const void* S, const void* Bm, const float* theta, int layers,
+                                 void* stream) {
+  if (c && !S) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_lista_layer_weights: NULL pointer");
+  if (c && layers > 4096) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_lista_layer_weights: at most 4096 layers");
+  return set_weights(c, S, Bm, theta, layers, true, stream, "csat_set_lista_layer_weights");
 }
 
 static int ensure_decoder(csat_ctx* c, cudaStream_t s, int* launches) {
@@ -469,8 +498,8 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   cudaStream_t s = (cudaStream_t)stream;
   int launches = 0;
   prof_mark(c, s, -1);
-  if (c->p.T > 0 && c->w_S && c->w_layers != 1 && c->w_layers != c->p.T)
-    return fail(c, CSAT_ERR_STATE, "csat_set_lista_weights was given thresholds for a number of layers other than CSAT_T");
+  if (c->p.T > 0 && c->w_S && (c->w_layers != 1 || c->w_untied) && c->w_layers != c->p.T)
+    return fail(c, CSAT_ERR_STATE, "the supplied LISTA weights are for a number of layers other than CSAT_T");
   if (c->p.T > 0) {
     const bool was_dirty = c->decoder_dirty;
     int rc = ensure_decoder(c, s, &launches);

@@ -55,11 +55,19 @@ struct csat_ctx {
   float* B_dec = nullptr;     // [H, d, d]  mu M
   float* psi_f32 = nullptr;   // [H, d, d]  Psi as float (row-major), only when psi != null
   float* theta = nullptr;     // [H] (ISTA-derived) 
-  // supplied LISTA weights (csat_set_lista_weights); null = ISTA-derived decoder
-  void* w_S = nullptr;        // [H, d, d] dtype
-  void* w_B = nullptr;        // [H, d, d] dtype
+  // supplied LISTA weights (csat_set_lista_weights / csat_set_lista_layer_weights); null = ISTA-derived decoder
+  void* w_S = nullptr;        // [H, d, d] dtype, or [w_layers, H, d, d] when w_untied
+  void* w_B = nullptr;        // the same
   float* w_theta = nullptr;   // [w_layers, H]
   int w_layers = 0;
+  bool w_untied = false;      // one S_t, B_t per layer
+  // untied layers, derived by the decoder set-up: float32 copies for the FFMA kernels and the bf16 tensor-core
+  // operands [H][2 w_layers + 1][d][d], each stored [output column][k]: 2t = S_t - I, 2t + 1 = B_t, last = Psi
+  float* Sl_dec = nullptr;    // [w_layers, H, d, d]
+  float* Bl_dec = nullptr;    // [w_layers, H, d, d]
+  __nv_bfloat16* lmats_bf16 = nullptr;
+  CUtensorMap tmap_lmats;     // TMA view of lmats_bf16
+  size_t w_mat_count() const { return (size_t)(w_untied ? w_layers : 1) * (size_t)(p.H * p.d * p.d); }
   float* mu = nullptr;        // [H]
   int* status = nullptr;      // device status word (0 = ok)
   // staging for csat_forward_host
@@ -117,6 +125,7 @@ cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cud
 
 // attend_recover_sm100.cu : tcgen05 compressed attention + recovery (bf16, d in {64, 128})
 cudaError_t make_attend_tmaps(csat_ctx* c);
+cudaError_t make_layer_weights_tmap(csat_ctx* c);
 cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
 
 // copies K~ or V~ out of the interleaved workspace: dst [B,H,m,d]

@@ -1,9 +1,9 @@
 // Decoder set-up, once per parameter change and per head (tiny: d x d matrices, float64 arithmetic).
 // Paper: LISTA recurrence alpha^{t+1} = eta_theta(S alpha^t + B Z_i) with S, B, theta taken from ISTA
-// ("fast approximate solvers, such as ISTA") for the model Z_i = D Psi alpha_i:
+// (the paper names ISTA among the approximate solvers it allows) for the model Z_i = D Psi alpha_i:
 //   M = D Psi, G = M^T M, L^ = max_a sum_b |G[a][b]|, mu = 1/L^ (or the caller's step),
 //   S = I - mu G, B = mu M, theta = mu lambda.
-// D defaults to the leading d x d block of the head's Phi ("Phi = Phi_V is reused").
+// D defaults to the leading d x d block of the head's Phi (the paper decodes with the values' measurement matrix).
 #include "csat_internal.h"
 
 namespace csat {
@@ -114,11 +114,53 @@ __global__ void weights_kernel(float* __restrict__ S_dec, float* __restrict__ B_
   if (i == 0) mu_out[h] = 0.f;
 }
 
+// Supplied LISTA weights with one S_t, B_t per layer (grid z = layer): float32 copies [L, H, d, d] for the FFMA
+// kernels, and the tensor-core operands of head h at lmats[h][2t] = S_t - I and lmats[h][2t + 1] = B_t, each stored
+// [output column][k] (layer t is the product [alpha^t | z] [S_t - I ; B_t], added to alpha^t), lmats[h][2L] = Psi.
+// Layer 0 also goes to S_dec / B_dec (what csat_get_decoder returns).
+template <typename T>
+__global__ void layer_weights_kernel(float* __restrict__ Sl_dec, float* __restrict__ Bl_dec, float* __restrict__ S_dec,
+                                     float* __restrict__ B_dec, float* __restrict__ mu_out, float* __restrict__ psi_f32,
+                                     const T* __restrict__ S, const T* __restrict__ Bm, const T* __restrict__ psi,
+                                     int psi_per_head, int d, int H, int L, __nv_bfloat16* __restrict__ lmats) {
+  const int h = blockIdx.y, l = blockIdx.z;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= d * d) return;
+  const int a = i / d, b = i % d;
+  const int64_t dd = (int64_t)d * d;
+  const int64_t src = ((int64_t)l * H + h) * dd;
+  const float sv = (float)ld(S, src + i), bv = (float)ld(Bm, src + i);
+  Sl_dec[src + i] = sv;
+  Bl_dec[src + i] = bv;
+  const T* P = psi ? psi + (psi_per_head ? (int64_t)h * dd : 0) : nullptr;
+  if (l == 0) {
+    S_dec[(int64_t)h * dd + i] = sv;
+    B_dec[(int64_t)h * dd + i] = bv;
+    if (P) psi_f32[(int64_t)h * dd + i] = (float)ld(P, i);
+    if (i == 0) mu_out[h] = 0.f;
+  }
+  if (lmats) {
+    __nv_bfloat16* mh = lmats + (int64_t)h * (2 * L + 1) * dd;
+    mh[(int64_t)(2 * l) * dd + i] =
+        __float2bfloat16_rn((float)(ld(S, src + (int64_t)b * d + a) - (a == b ? 1.0 : 0.0)));             // (S_t - I)[b][a]
+    mh[(int64_t)(2 * l + 1) * dd + i] = __float2bfloat16_rn((float)ld(Bm, src + (int64_t)b * d + a));    // B_t[b][a]
+    if (l == 0) mh[(int64_t)(2 * L) * dd + i] = P ? __float2bfloat16_rn((float)ld(P, i)) : __float2bfloat16_rn(0.f);
+  }
+}
+
 template <typename T>
 cudaError_t run(csat_ctx* c, cudaStream_t s, int* launches) {
   const Params& p = c->p;
   const int d = (int)p.d, H = (int)p.H;
   const dim3 grid((d * d + 255) / 256, H);
+  if (c->w_S && c->w_untied) {
+    const dim3 lgrid(grid.x, H, c->w_layers);
+    layer_weights_kernel<T><<<lgrid, 256, 0, s>>>(c->Sl_dec, c->Bl_dec, c->S_dec, c->B_dec, c->mu, c->psi_f32,
+                                                  (const T*)c->w_S, (const T*)c->w_B, (const T*)c->psi,
+                                                  c->psi_per_head ? 1 : 0, d, H, c->w_layers, c->lmats_bf16);
+    *launches += 1;
+    return cudaGetLastError();
+  }
   if (c->w_S) {
     weights_kernel<T><<<grid, 256, 0, s>>>(c->S_dec, c->B_dec, c->mu, c->psi_f32, (const T*)c->w_S, (const T*)c->w_B,
                                            (const T*)c->psi, c->psi_per_head ? 1 : 0, d, c->mats_bf16);

@@ -1,5 +1,5 @@
 // Seeded Gaussian measurement matrices Phi_h in R^{m x n}, entries N(0, 1/m).
-// Paper: compression equation and the sentence after it (sub-Gaussian ensembles, "random Gaussian").
+// Paper: compression equation and the sentence after it (Phi is drawn from a sub-Gaussian ensemble; Gaussian entries are the default).
 // The paper fixes no generator: this library uses Philox4x32-10 (Salmon et al., SC'11) keyed by the
 // 64-bit seed, counter = flat element index / 4, and Box-Muller on 23-bit uniforms.
 #include "csat_internal.h"

@@ -141,7 +141,7 @@ __device__ __forceinline__ void row_times_matrix(const float (&x)[DC], float (&y
 template <typename T, int DC>   // DC = ceil(d / 32)
 __global__ void __launch_bounds__(kAttWarps * 32) attend_recover_kernel(
     T* __restrict__ out, const T* __restrict__ Q, const T* __restrict__ kv, const float* __restrict__ S_dec,
-    const float* __restrict__ B_dec, const float* __restrict__ theta, int theta_stride,
+    const float* __restrict__ B_dec, int64_t layer_stride, const float* __restrict__ theta, int theta_stride,
     const float* __restrict__ psi_f32, int64_t nq, int64_t m, int d, int H, int T_iters, float scale) {
   extern __shared__ float smem[];
   const int d2 = 2 * d, ldk = d2 + 1;
@@ -198,16 +198,18 @@ __global__ void __launch_bounds__(kAttWarps * 32) attend_recover_kernel(
 #pragma unroll
     for (int j = 0; j < DC; ++j) res[j] = z[j];
   } else {
+    // layer t reads theta[t * theta_stride + h] and the matrices at layer_stride * t (0: one S, B for all layers)
     const float* Sh = S_dec + (int64_t)h * d * d;
     const float* Bh = B_dec + (int64_t)h * d * d;
-    float th = theta[h];                        // layer t reads theta[t * theta_stride + h]
+    float th = theta[h];
     float c[DC], a[DC], t[DC];
     row_times_matrix<DC>(z, c, Bh, d, lane);
 #pragma unroll
     for (int j = 0; j < DC; ++j) a[j] = soft_threshold(c[j], th);   // alpha^1 = eta(0 S + z B)
     for (int it = 1; it < T_iters; ++it) {
       th = theta[(int64_t)it * theta_stride + h];
-      row_times_matrix<DC>(a, t, Sh, d, lane);
+      if (layer_stride != 0) row_times_matrix<DC>(z, c, Bh + layer_stride * it, d, lane);   // z B_t
+      row_times_matrix<DC>(a, t, Sh + layer_stride * it, d, lane);
 #pragma unroll
       for (int j = 0; j < DC; ++j) a[j] = soft_threshold(t[j] + c[j], th);
     }
@@ -288,7 +290,9 @@ cudaError_t attend_t(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
       e = cudaFuncSetAttribute(attend_recover_kernel<T, DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); \
     if (e == cudaSuccess)                                                                                         \
       attend_recover_kernel<T, DC><<<grid, kAttWarps * 32, sm, s>>>(                                              \
-          (T*)out, (const T*)Q, (const T*)c->kv, c->S_dec, c->B_dec, c->thr(), c->thr_stride(),                  \
+          (T*)out, (const T*)Q, (const T*)c->kv, c->w_untied ? c->Sl_dec : c->S_dec,                             \
+          c->w_untied ? c->Bl_dec : c->B_dec, c->w_untied ? (int64_t)(p.H * p.d * p.d) : (int64_t)0, c->thr(),  \
+          c->thr_stride(),                                                                                       \
           c->psi ? c->psi_f32 : nullptr,                                                                         \
           p.nq, p.m, d, (int)p.H, p.T, scale);                                                                    \
   } while (0)
@@ -385,7 +389,8 @@ int attend_noalloc_t(const void* Q, const void* K, const void* V, const void* ph
       e = cudaFuncSetAttribute(attend_recover_kernel<T, DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm); \
     if (e == cudaSuccess)                                                                                           \
       attend_recover_kernel<T, DC><<<grid, kAttWarps * 32, sm, s>>>((T*)out, (const T*)Q, (const T*)scratch,        \
-                                                                    nullptr, nullptr, nullptr, 0, nullptr, nq, m, d, \
+                                                                    nullptr, nullptr, (int64_t)0, nullptr, 0,       \
+                                                                    nullptr, nq, m, d,                              \
                                                                     (int)H, /*T_iters=*/0, scale);                  \
   } while (0)
     if (dc <= 2) CSAT_NOALLOC_ATT(2);

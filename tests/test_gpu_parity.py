@@ -474,3 +474,71 @@ def test_forward_can_be_captured_in_a_cuda_graph():
     assert torch.equal(ctx.forward(Q, K, V), replayed)
     assert not torch.equal(replayed, eager1)
     ctx.close()
+
+
+@pytest.mark.parametrize("name", ["c1_fp32", "c2_bf16_d64", "c5_bf16_d128", "c3_bf16_psi"])
+def test_untied_lista_layers_match_oracle(name):
+    """One S_t, B_t and theta_t per layer (random, non-symmetric): FFMA path in fp32, per-layer tensor-core kernel
+    in bf16 (head dimension 64 and 128, ragged query tiles, with and without a dictionary)."""
+    if name == "c1_fp32":
+        w = C["c1"]
+    elif name == "c2_bf16_d64":
+        w = wl.shrink(C["c2"], B=2, H=3, n_q=300)
+    elif name == "c5_bf16_d128":
+        w = wl.shrink(C["c5"], B=1, H=2, n=1024, n_q=700, m=192)
+    else:
+        w = wl.shrink(C["c3"], B=2, H=2, n=784, n_q=257, m=100)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    phi = to_np(ctx.get_phi())
+    r = np.random.default_rng(41)
+    d, H = w.d, w.H
+    Psi = None
+    if name == "c3_bf16_psi":
+        Psi = wl.round_to_storage((np.eye(d) + 0.3 * r.standard_normal((d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        ctx.set_dictionary(to_dev(Psi, w.dtype))
+    st = []
+    orc.csat_forward(inp["Q"][:1], inp["K"][:1], inp["V"][:1], phi, T=0, lam=0.0, stages=st)
+    for T in sorted({1, 2, w.T}):
+        ctx.set(T=T)
+        S = wl.round_to_storage((0.6 * np.eye(d) + 0.4 * r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        Bm = wl.round_to_storage((r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        th0 = float(np.median(np.abs(st[0]["Z"] @ Bm[0, 0].astype(np.float64))))
+        thetas = (th0 * r.uniform(0.2, 1.5, size=(T, H))).astype(np.float32)
+        thetas[T // 2, 0] = 0.0                                    # a layer without shrinkage
+        ctx.set_lista_layer_weights(to_dev(S, w.dtype), to_dev(Bm, w.dtype), torch.from_numpy(thetas).cuda())
+        out = to_np(ctx.forward(Q, K, V))
+        ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=0.0, Psi=None if Psi is None else Psi.astype(np.float64),
+                               weights=(S.astype(np.float64), Bm.astype(np.float64), list(thetas.astype(np.float64))))
+        assert np.abs(ref).max() > 0
+        err = rel_err(out, ref)
+        assert err <= TOL[w.dtype], (name, T, err)
+        if w.dtype == "bf16":
+            # the FFMA path reads the same per-layer weights
+            ctx.set(force_simt=1)
+            err = rel_err(to_np(ctx.forward(Q, K, V)), ref)
+            ctx.set(force_simt=0)
+            assert err <= TOL[w.dtype], (name, T, "ffma", err)
+    # csat_get_decoder returns layer 0
+    S_d, B_d, th_d, _ = ctx.get_decoder()
+    assert np.array_equal(to_np(S_d), S[0].astype(np.float64)) and np.array_equal(to_np(B_d), Bm[0].astype(np.float64))
+    assert np.array_equal(to_np(th_d), thetas[0].astype(np.float64))
+    # another depth than the weights' is refused; tied weights and the derived decoder come back afterwards
+    ctx.set(T=T + 1)
+    with pytest.raises(binding.CsatError) as ei:
+        ctx.forward(Q, K, V)
+    assert ei.value.code == 6
+    ctx.set(T=T)
+    tied_th = torch.from_numpy(thetas[:1].copy()).cuda()
+    ctx.set_lista_weights(to_dev(S[0], w.dtype), to_dev(Bm[0], w.dtype), tied_th)
+    tied = to_np(ctx.forward(Q, K, V))
+    same = np.stack([S[0]] * T), np.stack([Bm[0]] * T), np.repeat(thetas[:1], T, axis=0)
+    ctx.set_lista_layer_weights(to_dev(same[0], w.dtype), to_dev(same[1], w.dtype), torch.from_numpy(same[2].copy()).cuda())
+    again = to_np(ctx.forward(Q, K, V))
+    assert rel_err(again, tied) <= TOL[w.dtype]
+    ctx.set_lista_weights(None)
+    ctx.set(lam=w.lam)
+    ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=w.lam, Psi=None if Psi is None else Psi.astype(np.float64))
+    assert rel_err(to_np(ctx.forward(Q, K, V)), ref) <= TOL[w.dtype]
+    ctx.close()

@@ -518,7 +518,7 @@ def test_forward_with_supplied_weights_uses_them():
 
 
 # ---------------------------------------------------------------------------------------------------
-# Rademacher measurement matrices (paper: "random Gaussian, Rademacher, or structured Hadamard matrices")
+# Rademacher measurement matrices (the second of the three ensembles the paper lists)
 # ---------------------------------------------------------------------------------------------------
 def _philox_scalar(ctr, key):
     """Philox4x32-10 on Python ints, written from the published round function (checked against the
