@@ -221,11 +221,20 @@ def kernel_flops(w: wl.Workload) -> dict:
             "split_reduce": 0}
 
 
-def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3) -> dict:
-    """Per-iteration CUDA-event timing with an L2 flush between iterations (workloads that fit in L2)."""
+def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3, untied: bool = False) -> dict:
+    """Per-iteration CUDA-event timing with an L2 flush between iterations (workloads that fit in L2).
+    untied: random LISTA weights with one S_t, B_t per layer instead of the ISTA-derived decoder."""
     import torch
     host, dev, psi = device_tensors(w)
     ctx = make_ctx(w, psi)
+    if untied:
+        g = torch.Generator(device="cuda")
+        g.manual_seed(7)
+        s = 1.0 / np.sqrt(w.d)
+        dt = dev["Q"].dtype
+        S = (0.6 * torch.eye(w.d, device="cuda") + 0.4 * s * torch.randn(w.T, w.H, w.d, w.d, device="cuda", generator=g)).to(dt)
+        Bm = (s * torch.randn(w.T, w.H, w.d, w.d, device="cuda", generator=g)).to(dt)
+        ctx.set_lista_layer_weights(S, Bm, torch.full((w.T, w.H), 0.02, device="cuda"))
     out = torch.empty_like(dev["Q"])
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     for _ in range(warmup):
@@ -242,6 +251,8 @@ def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3) -> dict:
     ctx.close()
     ms = float(np.median(times))
     f = wl.flops(w)["total"]
+    if untied:
+        f += 2 * w.n_q * w.d * w.d * (w.T - 1) * w.B * w.H      # z B_t in every layer after the first
     return {"ms": ms, "tokens_per_s": w.query_tokens / (ms * 1e-3), "tflops": f / (ms * 1e-3) / 1e12,
             "gflop": f / 1e9}
 
@@ -353,6 +364,8 @@ def run_csat(args, w: wl.Workload) -> dict:
                 extra[wl.CONFIGS[key].name] = time_small(wl.CONFIGS[key])
             for n in (2048, 4096, 8192):
                 extra[f"c5_sweep_n{n}"] = time_small(wl.sweep_config(n))
+            if w.T > 1 and w.dtype == "bf16":
+                extra[f"{w.name}_untied_layers"] = time_small(w, untied=True)
             result["other_workloads"] = extra
         if not args.no_cpu_baseline:
             inp = {k: host[k].float().numpy() for k in "QKV"}

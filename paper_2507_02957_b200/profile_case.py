@@ -1,11 +1,12 @@
 """Runs a few CSAT forwards of a given shape and prints the library's per-kernel CUDA-event times.
 
-    python -m paper_2507_02957_b200.profile_case forward N M D B H T [--nq NQ] [--iters I] [--dtype bf16|fp32]
+    python -m paper_2507_02957_b200.profile_case forward N M D B H T [--nq NQ] [--iters I] [--dtype bf16|fp32] [--untied]
     python -m paper_2507_02957_b200.profile_case workload c1|c2|c3|c4|c5 [--iters I]
     python -m paper_2507_02957_b200.profile_case ensembles N M D H        (regenerates Phi with every ensemble)
 
 A small driver to put under a profiler (ncu -k regex:<kernel> ...): 3 warm-up forwards, then I timed ones.
 Inputs are seeded random tensors (N(0, 1/d) for `forward`, the workload's own recipe for `workload`).
+--untied replaces the ISTA-derived decoder by random LISTA weights with one S_t, B_t per layer.
 """
 from __future__ import annotations
 
@@ -43,6 +44,7 @@ def main():
     f.add_argument("--nq", type=int, default=None)
     f.add_argument("--iters", type=int, default=5)
     f.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
+    f.add_argument("--untied", action="store_true")
     w_ = sub.add_parser("workload")
     w_.add_argument("name")
     w_.add_argument("--iters", type=int, default=5)
@@ -61,6 +63,11 @@ def main():
         K = (torch.randn(a.B, a.H, a.n, a.d, device="cuda", generator=g) * s).to(dt)
         V = (torch.randn(a.B, a.H, a.n, a.d, device="cuda", generator=g) * s).to(dt)
         ctx = binding.Csat(a.n, a.m, a.d, a.H, 0, B=a.B, n_q=nq, dtype=a.dtype, T=a.T, lam=0.05)
+        if a.untied and a.T > 0:
+            eye = torch.eye(a.d, device="cuda")
+            S = (0.6 * eye + 0.4 * s * torch.randn(a.T, a.H, a.d, a.d, device="cuda", generator=g)).to(dt)
+            Bm = (s * torch.randn(a.T, a.H, a.d, a.d, device="cuda", generator=g)).to(dt)
+            ctx.set_lista_layer_weights(S, Bm, torch.full((a.T, a.H), 0.02, device="cuda"))
         print(vars(a), _timed_forwards(ctx, Q, K, V, a.iters))
         ctx.close()
     elif a.cmd == "workload":
