@@ -33,8 +33,9 @@
 // the sum of the bf16 increments fed to the tensor cores so far; the registers hold b_t = alpha^t - theta
 // (theta = the first layer's threshold where the thresholds differ per layer; eta then uses the layer's own):
 //   r_0 = theta + z_bf16 B (threads store theta, one accumulating MMA);
-//   x = b_t + r_t = alpha^t S + z B;   b_{t+1} = eta_theta(x) - theta = x - 2 theta sat(x / (2 theta) + 1/2);
-//   r_{t+1} = r_t + bf16(b_t - b_{t+1}) (mu G)             (one accumulating MMA per iteration).
+//   x = b_t + r_t = alpha^t S + z B;   s = sat(x / (2 theta) + 1/2);   b_{t+1} = eta_theta(x) - theta = x - 2 theta s;
+//   increment b_{t+1} - b_t = r_t - 2 theta s   (from r_t, so that b_{t+1} can overwrite b_t at once);
+//   r_{t+1} = r_t + bf16(b_{t+1} - b_t) (-mu G)            (one accumulating MMA per iteration; -mu G is stored).
 // This is the paper's S alpha + B z with S = I - mu G: the identity part stays exact in fp32 registers, only
 // the increment that multiplies mu G is rounded to bf16, and c never needs registers of its own.  The
 // saturating form of the shrinkage runs on the FMA pipe (two-element packed instructions where they exist);
@@ -336,7 +337,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             ring_wait_k(g, 206);
             if (w.dead) break;
             mbar_arrive_expect_tx(&bars->k_full[s], C::kMatBoxBytes);
-            tma_load_3d(k_slot(s), &tmap_mats, &bars->k_full[s], gx * 64, 0, h * 3 + 0);          // mu G
+            tma_load_3d(k_slot(s), &tmap_mats, &bars->k_full[s], gx * 64, 0, h * 3 + 0);          // -mu G
             k_hist = (k_hist << 1) | 1u;
             v_hist <<= 1;
             ring_wait_v(g, 207);
@@ -371,7 +372,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     if (elect_one()) {
       constexpr uint32_t idesc_s = make_idesc_bf16(kRows, kMC, false, false);   // S  = Q  K~^T : both K-major
       constexpr uint32_t idesc_z = make_idesc_bf16(kRows, D, false, true);      // Z += P  V~   : V~ is MN-major
-      constexpr uint32_t idesc_r = make_idesc_bf16(kRows, D, false, false);     // r += a  W^T  : both K-major
+      constexpr uint32_t idesc_r = make_idesc_bf16(kRows, D, false, false);     // r += a (-W)^T: both K-major
       // K-major operand: K step k (16 columns) lies in 64-column box k / 4, 32 (k % 4) bytes into each row
       auto kstep = [](int k, uint32_t box_bytes) { return (uint64_t)((k / 4) * (box_bytes >> 4) + (k % 4) * 2); };
       const uint64_t q_desc0 = make_smem_desc(smem_u32(q_buf), 16, 1024);
@@ -782,16 +783,17 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
               uint32_t pk[8];
 #pragma unroll
               for (int e = 0; e < 16; e += 2) {
-                const uint64_t bo = v2[(c0 + e) >> 1];
-                const uint64_t x2 = add2(bo, pack2u(r[e], r[e + 1]));          // alpha^t S + z B
+                const uint64_t r2 = pack2u(r[e], r[e + 1]);
+                const uint64_t x2 = add2(v2[(c0 + e) >> 1], r2);               // alpha^t S + z B
                 float x0, x1;
                 unpack2(x2, x0, x1);
                 const uint64_t t2 = pack2(fma_sat(x0, inv2th, 0.5f), fma_sat(x1, inv2th, 0.5f));
                 uint64_t bn = fma2(t2, m2th2, x2);                             // eta_theta(x) - theta
-                if (per_layer.value) bn = add2(bn, dk2);                       // ... - kappa
+                uint64_t dn = fma2(t2, m2th2, r2);                             // alpha^{t+1} - alpha^t
+                if (per_layer.value) { bn = add2(bn, dk2); dn = add2(dn, dk2); }   // ... - kappa
                 v2[(c0 + e) >> 1] = bn;
                 float d0, d1;
-                unpack2(sub2(bo, bn), d0, d1);                                 // alpha^t - alpha^{t+1}
+                unpack2(dn, d0, d1);
                 pk[e >> 1] = pack_bf16(d0, d1);
               }
               tmem_st_32x32b_x8(op_addr + c0 / 2, pk);

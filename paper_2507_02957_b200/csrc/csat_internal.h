@@ -47,7 +47,7 @@ struct csat_ctx {
   CUtensorMap tmap_kv;        // TMA view of the K~|V~ workspace
   CUtensorMap tmap_mats;      // TMA view of mats_bf16
   // bf16 operand copies of the decoder matrices for the tensor-core path: [H][3][d][d], each stored
-  // [output column][k] (k contiguous): 0 = mu G (symmetric), 1 = (mu M)^T, 2 = Psi
+  // [output column][k] (k contiguous): 0 = -mu G = S - I (symmetric for ISTA), 1 = B^T = (mu M)^T, 2 = Psi
   __nv_bfloat16* mats_bf16 = nullptr;
   double* Mf64 = nullptr;     // [H, d, d] scratch of the decoder set-up
   double* Gf64 = nullptr;     // [H, d, d]

@@ -75,9 +75,9 @@ __global__ void finalize_kernel(float* __restrict__ S_dec, float* __restrict__ B
     B_dec[(int64_t)h * d * d + i] = (float)(mu * Mh[i]);
     if (psi) psi_f32[(int64_t)h * d * d + i] = (float)ld(psi + (psi_per_head ? (int64_t)h * d * d : 0), i);
     if (mats_bf16) {
-      // tensor-core operand copies, each stored [output column][k]: mu G (symmetric), (mu M)^T, Psi
+      // tensor-core operand copies, each stored [output column][k]: -mu G (symmetric), (mu M)^T, Psi
       __nv_bfloat16* mh = mats_bf16 + (int64_t)h * 3 * d * d;
-      mh[i] = __float2bfloat16_rn((float)(mu * Gh[i]));
+      mh[i] = __float2bfloat16_rn((float)(-mu * Gh[i]));
       mh[d * d + i] = __float2bfloat16_rn((float)(mu * Mh[b * d + a]));
       mh[2 * d * d + i] =
           psi ? __float2bfloat16_rn((float)ld(psi + (psi_per_head ? (int64_t)h * d * d : 0), i)) : __float2bfloat16_rn(0.f);
@@ -90,7 +90,7 @@ __global__ void finalize_kernel(float* __restrict__ S_dec, float* __restrict__ B
 }
 
 // Supplied LISTA weights: S, B as given (float32 copies for the FFMA kernels), and the tensor-core operand
-// copies, each stored [output column][k]: W = I - S (so that alpha S = alpha - alpha W), B, Psi.
+// copies, each stored [output column][k]: S - I (so that alpha S = alpha + alpha (S - I)), B, Psi.
 template <typename T>
 __global__ void weights_kernel(float* __restrict__ S_dec, float* __restrict__ B_dec, float* __restrict__ mu_out,
                                float* __restrict__ psi_f32, const T* __restrict__ S, const T* __restrict__ Bm,
@@ -107,7 +107,7 @@ __global__ void weights_kernel(float* __restrict__ S_dec, float* __restrict__ B_
   if (P) psi_f32[base + i] = (float)ld(P, i);
   if (mats_bf16) {
     __nv_bfloat16* mh = mats_bf16 + base * 3;
-    mh[i] = __float2bfloat16_rn((float)((a == b ? 1.0 : 0.0) - ld(S, base + (int64_t)b * d + a)));   // W[b][a]
+    mh[i] = __float2bfloat16_rn((float)(ld(S, base + (int64_t)b * d + a) - (a == b ? 1.0 : 0.0)));   // (S - I)[b][a]
     mh[d * d + i] = __float2bfloat16_rn((float)ld(Bm, base + (int64_t)b * d + a));                    // B[b][a]
     mh[2 * d * d + i] = P ? __float2bfloat16_rn((float)ld(P, i)) : __float2bfloat16_rn(0.f);
   }
