@@ -15,9 +15,10 @@
 //   warps 0-3 : tile A, one thread per query row (TMEM lane = row).  Softmax reference and sum, exp2,
 //               P -> bf16 -> tensor memory, soft-threshold, output.  The whole row of alpha is in registers.
 //   warps 4-7 : tile B, the same.
-//   warp 8    : allocates tensor memory; one elected thread issues every tcgen05.mma.
+//   warp 8    : allocates tensor memory; one elected thread issues tile A's tcgen05.mma.
 //   warp 9    : one elected thread issues every TMA copy.
-//   warps 10-11: idle (they only complete the control warpgroup).
+//   warp 10   : one elected thread issues tile B's tcgen05.mma.
+//   warp 11   : idle (it only completes the control warpgroup).
 //
 // Attention phase, per tile and per chunk j of 64 measurements:
 //   S_j = Q K~_j^T            (SS MMA, accumulator S[j&1] in tensor memory)
@@ -27,7 +28,8 @@
 // ref is the row's reference maximum.  It only has to keep exp2 in range, so it is raised (and the row of
 // Zacc and the running sum rescaled by exp2(old - new)) only when a chunk's maximum exceeds it by more than
 // 8, i.e. when some P would exceed 2^8; the final division by the row sum cancels ref exactly.
-// All MMAs of the CTA execute in issue order, so S_{j+2} overwrites S[j&1] only after P_j V~_j has read P_j.
+// The MMAs of one tile are issued by one thread and execute in issue order, so S_{j+2} overwrites S[j&1] only
+// after P_j V~_j has read P_j.
 //
 // Recovery phase, per tile.  The accumulator holds r_t = theta + c - a^_t (mu G), where c = z B and a^_t is
 // the sum of the bf16 increments fed to the tensor cores so far; the registers hold b_t = alpha^t - theta
@@ -62,7 +64,7 @@ constexpr int kTiles = 2;             // tiles per CTA
 constexpr int kMC = 64;               // measurements per chunk
 constexpr int kTileThreads = 128;
 constexpr int kThreads = 384;          // three warpgroups: tile A, tile B, control
-constexpr int kMmaWarp = 8, kTmaWarp = 9;
+constexpr int kMmaWarp = 8, kTmaWarp = 9, kMmaWarpB = 10;   // tile A's MMA issuer, TMA producer, tile B's MMA issuer
 constexpr int kMaxStages = 6;
 constexpr int kPolyEvery = 4;          // every 4th pair of scores takes the polynomial exp2 (measured best of 1, 2, 3, 4, none)
 
@@ -224,12 +226,12 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     prefetch_tmap(&tmap_mats);
     mbar_init(&bars->mats_full, 1);
     for (int s = 0; s < C::kStages; ++s) {
-      mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], 1);
-      mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], 1);
+      mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], kTiles);     // released by both MMA issuers
+      mbar_init(&bars->v_full[s], 1); mbar_init(&bars->v_empty[s], kTiles);
     }
     for (int t = 0; t < kTiles; ++t) {
       mbar_init(&bars->q_full[t], 1);
-      mbar_init(&bars->q_free[t], 1);
+      mbar_init(&bars->q_free[t], t == 0 ? kTiles : 1);     // tile A's buffer also holds B, which both tiles read
       for (int s = 0; s < 2; ++s) { mbar_init(&bars->s_full[t][s], 1); mbar_init(&bars->p_full[t][s], kTileThreads); }
       mbar_init(&bars->zc_full[t], 1);
       mbar_init(&bars->a_full[t], kTileThreads);
@@ -365,10 +367,15 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         if (mats_loads > 0) mbar_wait_drain(&bars->mats_full, (mats_loads - 1) & 1);
       }
     }
-  } else if (warp == kMmaWarp) {
-    // ------------------------------------------------ MMA issuer --------------------------------------------------
-    // One thread issues every MMA of both tiles, so the issue path is kept short: descriptors of buffers that
-    // do not move are built once, the others differ from a base by compile-time constants.
+  } else if (warp == kMmaWarp || warp == kMmaWarpB) {
+    // ------------------------------------------------ MMA issuers -------------------------------------------------
+    // One elected thread per tile issues that tile's MMAs (tile A: warp 8, tile B: warp 10, on different
+    // sub-cores): issuing is a serial stream of a few dozen cycles per MMA, and one thread for both tiles was the
+    // critical path of the attention phase.  Barriers that release something both tiles read (ring slots, tile
+    // A's Q buffer when it holds B) count two arrivals, one per issuer; where an item has no second tile, tile
+    // B's issuer walks the same ring positions and arrives without issuing anything.
+    // Descriptors of buffers that do not move are built once, the others differ from a base by constants.
+    const int t = (warp == kMmaWarp) ? 0 : 1;
     if (elect_one()) {
       constexpr uint32_t idesc_s = make_idesc_bf16(kRows, kMC, false, false);   // S  = Q  K~^T : both K-major
       constexpr uint32_t idesc_z = make_idesc_bf16(kRows, D, false, true);      // Z += P  V~   : V~ is MN-major
@@ -376,66 +383,60 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       // K-major operand: K step k (16 columns) lies in 64-column box k / 4, 32 (k % 4) bytes into each row
       auto kstep = [](int k, uint32_t box_bytes) { return (uint64_t)((k / 4) * (box_bytes >> 4) + (k % 4) * 2); };
       const uint64_t q_desc0 = make_smem_desc(smem_u32(q_buf), 16, 1024);
+      const uint64_t qd = q_desc0 + (uint64_t)(t * (C::kQBytes >> 4));
       const uint64_t ring_k0 = make_smem_desc(smem_u32(ring), 16, 1024);
       const uint64_t ring_v0 = make_smem_desc(smem_u32(ring + C::kSlotBytes), C::kBoxBytes, 1024);
       constexpr uint64_t kStageStep = (2 * C::kSlotBytes) >> 4;                 // descriptor distance between stages
+      const uint32_t tb = tmem + t * C::kTileCols;
       uint32_t g = 0, items_done = 0;          // ring position of the item's first chunk; items of this CTA so far
-      uint32_t cb[kTiles] = {0, 0};            // chunks of earlier items, per tile (S / P buffer and parities)
-      uint32_t ab[kTiles] = {0, 0};            // recovery MMAs of earlier items, per tile
-      uint32_t q_uses[kTiles] = {0, 0};
+      uint32_t cb = 0;                         // chunks of this tile's earlier items (S / P buffer and parities)
+      uint32_t ab = 0;                         // recovery MMAs of this tile's earlier items
+      uint32_t q_uses = 0;
       for (int item = blockIdx.x; item < n_items && !w.dead; item += gridDim.x, ++items_done) {
         const int row0 = (item % items_x) * (kTiles * kRows);
-        const int ntiles = (nq - row0 > kRows) ? 2 : 1;
+        const bool active = t == 0 || nq - row0 > kRows;          // the item has this tile
+        // releases a buffer both issuers account for: after this thread's MMAs, or at once when it has none
+        auto release = [&](uint64_t* bar) { if (active) mma_commit(bar); else mbar_arrive(bar); };
         auto issue_pv = [&](int i) {
           const uint32_t pos = g + i;
           const int s = pos % C::kStages;
           w.wait(&bars->v_full[s], (pos / C::kStages) & 1, 211);
-          const uint64_t b_desc = ring_v0 + (uint64_t)s * kStageStep;
-          const uint32_t acc = (i != 0);
+          if (active) {
+            const uint64_t b_desc = ring_v0 + (uint64_t)s * kStageStep;
+            const uint32_t c = cb + i;
+            const int b = c & 1;
+            w.wait(&bars->p_full[t][b], (c >> 1) & 1, 212);
+            tc_fence_after();
+            // P: 8 packed columns per 16 measurements; V~: +16 rows = 2048 B
+            mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC, b_desc, idesc_z, (uint32_t)(i != 0));
 #pragma unroll
-          for (int t = 0; t < kTiles; ++t) {
-            if (t < ntiles) {
-              const uint32_t c = cb[t] + i;
-              const int b = c & 1;
-              w.wait(&bars->p_full[t][b], (c >> 1) & 1, 212);
-              tc_fence_after();
-              const uint32_t tb = tmem + t * C::kTileCols;
-              // P: 8 packed columns per 16 measurements; V~: +16 rows = 2048 B
-              mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC, b_desc, idesc_z, acc);
-#pragma unroll
-              for (int k = 1; k < kMC / 16; ++k)
-                mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC + k * 8, b_desc + (uint64_t)(k * 128), idesc_z, 1u);
-              mma_commit(&bars->zc_full[t]);
-            }
+            for (int k = 1; k < kMC / 16; ++k)
+              mma_f16_ts(tb + C::kColAcc, tb + C::kColS + b * kMC + k * 8, b_desc + (uint64_t)(k * 128), idesc_z, 1u);
+            mma_commit(&bars->zc_full[t]);
           }
-          mma_commit(&bars->v_empty[s]);
+          release(&bars->v_empty[s]);
         };
-#pragma unroll
-        for (int t = 0; t < kTiles; ++t)
-          if (t < ntiles) { w.wait(&bars->q_full[t], q_uses[t] & 1, 210); ++q_uses[t]; }
+        if (active) { w.wait(&bars->q_full[t], q_uses & 1, 210); ++q_uses; }
         for (int j = 0; j < nchunks; ++j) {
           const uint32_t pos = g + j;
           const int s = pos % C::kStages;
           w.wait(&bars->k_full[s], (pos / C::kStages) & 1, 213);
-          tc_fence_after();
-          const uint64_t kd = ring_k0 + (uint64_t)s * kStageStep;
+          if (active) {
+            tc_fence_after();
+            const uint64_t kd = ring_k0 + (uint64_t)s * kStageStep;
+            const int b = (cb + j) & 1;
+            const uint32_t ds = tb + C::kColS + b * kMC;
 #pragma unroll
-          for (int t = 0; t < kTiles; ++t) {
-            if (t < ntiles) {
-              const int b = (cb[t] + j) & 1;
-              const uint64_t qd = q_desc0 + (uint64_t)(t * (C::kQBytes >> 4));
-              const uint32_t ds = tmem + t * C::kTileCols + C::kColS + b * kMC;
-#pragma unroll
-              for (int k = 0; k < D / 16; ++k)
-                mma_f16_ss(ds, qd + kstep(k, kRows * 128), kd + kstep(k, C::kBoxBytes), idesc_s, k != 0);
-              mma_commit(&bars->s_full[t][b]);
-            }
+            for (int k = 0; k < D / 16; ++k)
+              mma_f16_ss(ds, qd + kstep(k, kRows * 128), kd + kstep(k, C::kBoxBytes), idesc_s, k != 0);
+            mma_commit(&bars->s_full[t][b]);
           }
-          mma_commit(&bars->k_empty[s]);
+          release(&bars->k_empty[s]);
           if (j == nchunks - 1) {
-            // the Q buffers have been read for the last time (tile A's still takes B when there is a recovery)
-            if (ntiles == 2) mma_commit(&bars->q_free[1]);
-            if (T == 0 || kUntied) mma_commit(&bars->q_free[0]);
+            // the Q buffers have been read for the last time (tile A's still takes B when there is a recovery
+            // with one S, B for all layers)
+            if (t == 1 && active) mma_commit(&bars->q_free[1]);
+            if (T == 0 || kUntied) release(&bars->q_free[0]);
           }
           if (j > 0) issue_pv(j - 1);
         }
@@ -450,40 +451,36 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
               w.wait(&bars->k_full[pos % C::kStages], (pos / C::kStages) & 1, 215);
               w.wait(&bars->v_full[pos % C::kStages], (pos / C::kStages) & 1, 215);
             }
+            if (active) {
+              w.wait(&bars->a_full[t], (ab + l) & 1, 216);
+              tc_fence_after();
+              const uint32_t z_cols = tb + C::kColS, a_cols = tb + C::kColS + D / 2;
 #pragma unroll
-            for (int t = 0; t < kTiles; ++t) {
-              if (t < ntiles) {
-                w.wait(&bars->a_full[t], (ab[t] + l) & 1, 216);
-                tc_fence_after();
-                const uint32_t tb = tmem + t * C::kTileCols;
-                const uint32_t z_cols = tb + C::kColS, a_cols = tb + C::kColS + D / 2;
+              for (int k = 0; k < D / 16; ++k) {
+                // the V~ slot of the layer's box k / 4: B_l (A operand z^), or Psi (A operand the final alpha)
+                const uint64_t wd = ring_k0 + (uint64_t)((pl + k / 4) % C::kStages) * kStageStep +
+                                    (uint64_t)(C::kSlotBytes >> 4) + (uint64_t)((k % 4) * 2);
+                mma_f16_ts(tb + C::kColAcc, (psi_l ? a_cols : z_cols) + k * 8, wd, idesc_r, k == 0 ? 0u : 1u);
+              }
+              if (!psi_l && l > 0) {
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                  // the V~ slot of the layer's box k / 4: B_l (A operand z^), or Psi (A operand the final alpha)
                   const uint64_t wd = ring_k0 + (uint64_t)((pl + k / 4) % C::kStages) * kStageStep +
-                                      (uint64_t)(C::kSlotBytes >> 4) + (uint64_t)((k % 4) * 2);
-                  mma_f16_ts(tb + C::kColAcc, (psi_l ? a_cols : z_cols) + k * 8, wd, idesc_r, k == 0 ? 0u : 1u);
+                                      (uint64_t)((k % 4) * 2);                                   // S_l - I
+                  mma_f16_ts(tb + C::kColAcc, a_cols + k * 8, wd, idesc_r, 1u);
                 }
-                if (!psi_l && l > 0) {
-#pragma unroll
-                  for (int k = 0; k < D / 16; ++k) {
-                    const uint64_t wd = ring_k0 + (uint64_t)((pl + k / 4) % C::kStages) * kStageStep +
-                                        (uint64_t)((k % 4) * 2);                                   // S_l - I
-                    mma_f16_ts(tb + C::kColAcc, a_cols + k * 8, wd, idesc_r, 1u);
-                  }
-                }
-                mma_commit(&bars->r_full[t]);
               }
+              mma_commit(&bars->r_full[t]);
             }
-            for (int gx = 0; gx < C::kDBoxes; ++gx) {     // both tiles have read the layer's matrices
-              mma_commit(&bars->k_empty[(pl + gx) % C::kStages]);
-              mma_commit(&bars->v_empty[(pl + gx) % C::kStages]);
+            for (int gx = 0; gx < C::kDBoxes; ++gx) {     // this tile has read the layer's matrices
+              release(&bars->k_empty[(pl + gx) % C::kStages]);
+              release(&bars->v_empty[(pl + gx) % C::kStages]);
             }
           }
         }
         if (!kUntied && T > 0) {
-          const uint32_t gv = g + nchunks;            // ring position of the first box of mu G / Psi
-          const int n_mma = nlayers;                  // r_0 = theta + z B, then T-1 increments with mu G, then Psi
+          const uint32_t gv = g + nchunks;            // ring position of the first box of -mu G / Psi
+          const int n_mma = nlayers;                  // r_0 = theta + z B, then T-1 increments with -mu G, then Psi
           for (int i = 0; i < n_mma; ++i) {
             const bool first = (i == 0), psi_step = has_psi && i == n_mma - 1;
             if (first) w.wait(&bars->mats_full, items_done & 1, 214);
@@ -493,37 +490,34 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                 w.wait(psi_step ? &bars->v_full[pos % C::kStages] : &bars->k_full[pos % C::kStages],
                        (pos / C::kStages) & 1, 215);
               }
-            const uint32_t acc0 = psi_step ? 0u : 1u;
+            if (active) {
+              const uint32_t acc0 = psi_step ? 0u : 1u;
+              w.wait(&bars->a_full[t], (ab + i) & 1, 216);
+              tc_fence_after();
 #pragma unroll
-            for (int t = 0; t < kTiles; ++t) {
-              if (t < ntiles) {
-                w.wait(&bars->a_full[t], (ab[t] + i) & 1, 216);
-                tc_fence_after();
-                const uint32_t tb = tmem + t * C::kTileCols;
-#pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                  // B: boxes of d rows in tile A's Q buffer; mu G / Psi: box k / 4 in the K~ / V~ slot of ring
-                  // position gv + k / 4
-                  const uint64_t wd = first ? q_desc0 + (uint64_t)((k / 4) * (C::kMatBoxBytes >> 4))
-                                            : ring_k0 + (uint64_t)((gv + k / 4) % C::kStages) * kStageStep +
-                                                  (psi_step ? (uint64_t)(C::kSlotBytes >> 4) : 0);
-                  mma_f16_ts(tb + C::kColAcc, tb + C::kColS + k * 8, wd + (uint64_t)((k % 4) * 2), idesc_r,
-                             k == 0 ? acc0 : 1u);
-                }
-                mma_commit(&bars->r_full[t]);
+              for (int k = 0; k < D / 16; ++k) {
+                // B: boxes of d rows in tile A's Q buffer; -mu G / Psi: box k / 4 in the K~ / V~ slot of ring
+                // position gv + k / 4
+                const uint64_t wd = first ? q_desc0 + (uint64_t)((k / 4) * (C::kMatBoxBytes >> 4))
+                                          : ring_k0 + (uint64_t)((gv + k / 4) % C::kStages) * kStageStep +
+                                                (psi_step ? (uint64_t)(C::kSlotBytes >> 4) : 0);
+                mma_f16_ts(tb + C::kColAcc, tb + C::kColS + k * 8, wd + (uint64_t)((k % 4) * 2), idesc_r,
+                           k == 0 ? acc0 : 1u);
               }
+              mma_commit(&bars->r_full[t]);
             }
-            if (first) mma_commit(&bars->q_free[0]);      // B has been read: tile A's Q buffer is free
+            if (first) release(&bars->q_free[0]);         // B has been read: tile A's Q buffer is free
           }
-          for (int gx = 0; gx < C::kDBoxes; ++gx) {       // release the ring positions of mu G / Psi
-            mma_commit(&bars->k_empty[(gv + gx) % C::kStages]);
-            mma_commit(&bars->v_empty[(gv + gx) % C::kStages]);
+          for (int gx = 0; gx < C::kDBoxes; ++gx) {       // release the ring positions of -mu G / Psi; a position
+            const uint32_t pos = gv + gx;                 // that was never read is waited for first, so that no
+            if (T == 1) w.wait(&bars->k_full[pos % C::kStages], (pos / C::kStages) & 1, 215);   // phase is skipped
+            if (!has_psi) w.wait(&bars->v_full[pos % C::kStages], (pos / C::kStages) & 1, 215);
+            release(&bars->k_empty[pos % C::kStages]);
+            release(&bars->v_empty[pos % C::kStages]);
           }
         }
         g += nchunks + nvirt;
-#pragma unroll
-        for (int t = 0; t < kTiles; ++t)
-          if (t < ntiles) { cb[t] += nchunks; ab[t] += nlayers; }
+        if (active) { cb += nchunks; ab += nlayers; }
       }
     }
   }
