@@ -120,6 +120,12 @@ __device__ __forceinline__ float fma_sat(float a, float b, float c) {   // clamp
   asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
+// 32-byte store (the address is 32-byte aligned)
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&r)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]),
+               "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
+}
 // two-element packed fp32 arithmetic (one instruction for both halves of a 64-bit register pair)
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
   uint64_t r;
@@ -842,13 +848,30 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       }
       const int grow = row0 + t * kRows + row;
       if (grow < nq && !w.dead && *(volatile int*)&bars->abort == 0) {
-        uint4* o = reinterpret_cast<uint4*>(out + ((int64_t)bh * nq + grow) * D);
+        // a row is a multiple of 128 bytes; where the output is 32-byte aligned every store covers whole
+        // 32-byte sectors (the lanes of a warp write different rows), otherwise 16-byte stores
+        __nv_bfloat16* orow = out + ((int64_t)bh * nq + grow) * D;
+        if ((reinterpret_cast<uintptr_t>(out) & 31u) == 0) {
 #pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
-          float x[8];
+          for (int c = 0; c < D / 16; ++c) {
+            uint32_t pk[8];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) unpack2(v2[c * 4 + u], x[2 * u], x[2 * u + 1]);
-          o[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+            for (int u = 0; u < 8; ++u) {
+              float x0, x1;
+              unpack2(v2[c * 8 + u], x0, x1);
+              pk[u] = pack_bf16(x0, x1);
+            }
+            st_global_v8(orow + c * 16, pk);
+          }
+        } else {
+          uint4* o = reinterpret_cast<uint4*>(orow);
+#pragma unroll
+          for (int c = 0; c < D / 8; ++c) {
+            float x[8];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) unpack2(v2[c * 4 + u], x[2 * u], x[2 * u + 1]);
+            o[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+          }
         }
       }
     }
