@@ -542,3 +542,21 @@ def test_untied_lista_layers_match_oracle(name):
     ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=T, lam=w.lam, Psi=None if Psi is None else Psi.astype(np.float64))
     assert rel_err(to_np(ctx.forward(Q, K, V)), ref) <= TOL[w.dtype]
     ctx.close()
+
+
+def test_output_aligned_to_16_bytes_only_gives_the_same_result():
+    """The tensor-core kernel stores 32 bytes per lane where the output allows it and 16 bytes otherwise: an
+    output that starts 16 bytes into an allocation must come out bit-identical."""
+    for w in (wl.shrink(C["c2"], B=2, H=3, n_q=300), wl.shrink(C["c5"], B=1, H=2, n=1024, n_q=700, m=192)):
+        inp = wl.make_inputs(w)
+        Q, K, V, _ = device_inputs(w, inp)
+        ctx = make_ctx(w)
+        ref = ctx.forward(Q, K, V)
+        flat = torch.zeros(Q.numel() + 8, dtype=Q.dtype, device="cuda")
+        out = flat[8:].view(Q.shape)
+        assert out.data_ptr() % 32 == 16 and out.is_contiguous()
+        ctx.forward(Q, K, V, out)
+        torch.cuda.synchronize()
+        assert torch.equal(out, ref)
+        assert float(flat[:8].abs().max()) == 0.0
+        ctx.close()
