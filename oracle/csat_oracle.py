@@ -16,6 +16,7 @@ paper's column vectors alpha_i, Z_i, C_i appear here as 1 x d rows):
   ista               alpha^{t+1} = eta_theta(S alpha^t + B Z_i)   (LISTA recurrence, ISTA weights)
   lista              the same recurrence with supplied S, B and per-layer theta_t
   reconstruct        C^_i = Psi alpha^_i                  (reconstruction equation)
+  project_qkv        Q = X W^Q, K = X W^K, V = X W^V      (projection equation, one set of d_k columns per head)
 
 Reading of the decoder (the paper's "Z_i = Phi Psi alpha_i" with Phi in R^{m x n}
 cannot multiply a d_k-vector): the sensing matrix of the decoder is a d x d matrix
@@ -34,6 +35,28 @@ from __future__ import annotations
 import numpy as np
 
 F64 = np.float64
+
+
+# ----------------------------------------------------------------------------
+# input projections
+# ----------------------------------------------------------------------------
+def project_qkv(X: np.ndarray, W: np.ndarray, H: int, d: int):
+    """Q = X W^Q, K = X W^K, V = X W^V for every head.  X [B,n,d_model]; W [d_model, 3*H*d] holds the projection
+    matrices side by side: columns [0, H*d) are W^Q of heads 0..H-1 (d columns each), then W^K, then W^V.
+    Returns Q, K, V, each [B,H,n,d]."""
+    X = np.asarray(X, F64)
+    W = np.asarray(W, F64)
+    B, n, dm = X.shape
+    assert W.shape == (dm, 3 * H * d)
+    out = []
+    for which in range(3):
+        P = np.empty((B, H, n, d), dtype=F64)
+        for h in range(H):
+            Wh = W[:, (which * H + h) * d:(which * H + h + 1) * d]      # [d_model, d] of this head
+            for b in range(B):
+                P[b, h] = X[b] @ Wh
+        out.append(P)
+    return tuple(out)
 
 
 # ----------------------------------------------------------------------------

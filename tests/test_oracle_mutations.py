@@ -124,7 +124,19 @@ def _lista_layers_reversed(Z, S, B, thetas, return_iterates=False):
     return _orig_lista(Z, S, B, thetas, return_iterates)
 
 
+def _project_heads_interleaved(X, W, H, d):
+    # columns taken as [head][which] instead of [which][head]
+    Wp = np.asarray(W, F64).reshape(W.shape[0], H, 3, d).transpose(0, 2, 1, 3).reshape(W.shape[0], 3 * H * d)
+    return _orig_project(X, Wp, H, d)
+
+
+def _project_W_transposed_per_head(X, W, H, d):
+    Q, K, V = _orig_project(X, W, H, d)
+    return K, Q, V
+
+
 _orig_lista = orc.lista
+_orig_project = orc.project_qkv
 _orig_setup = orc.decoder_setup
 _orig_ista = orc.ista
 
@@ -149,6 +161,8 @@ MUTATIONS = {
     "lista: first layer's matrices in every layer": ("lista", _lista_first_layer_everywhere),
     "lista: B of the layer before": ("lista", _lista_B_one_layer_late),
     "lista: layers in reverse order": ("lista", _lista_layers_reversed),
+    "project: head and q/k/v order swapped": ("project_qkv", _project_heads_interleaved),
+    "project: queries and keys exchanged": ("project_qkv", _project_W_transposed_per_head),
     "compress: |Phi|": ("compress", _compress_abs),
     "output: weights ignored": ("compressed_output", _output_uses_unweighted),
 }

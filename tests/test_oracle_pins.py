@@ -614,3 +614,34 @@ def test_separate_value_matrix():
     orc.csat_forward(inp["Q"], inp["K"], inp["V"], Pk, T=2, lam=0.01, Phi_V=Pv, stages=st)
     S_ref, B_ref, th_ref, mu_ref = orc.decoder_setup(Pv[0][:w.d, :w.d], 0.01)
     assert np.array_equal(st[0]["B_dec"], B_ref) and st[0]["theta"] == th_ref
+
+
+# ---------------------------------------------------------------------------------------------------
+# input projections (paper: Q = X W^Q, K = X W^K, V = X W^V)
+# ---------------------------------------------------------------------------------------------------
+def test_project_qkv_matches_scalar_loops_and_layout():
+    r = np.random.default_rng(61)
+    B, n, dm, H, d = 2, 3, 5, 2, 4
+    X = r.standard_normal((B, n, dm))
+    W = r.standard_normal((dm, 3 * H * d))
+    Q, K, V = orc.project_qkv(X, W, H, d)
+    for which, P in enumerate((Q, K, V)):
+        assert P.shape == (B, H, n, d)
+        for b in range(B):
+            for h in range(H):
+                for i in range(n):
+                    for c in range(d):
+                        want = sum(X[b][i][k] * W[k][(which * H + h) * d + c] for k in range(dm))
+                        assert abs(P[b, h, i, c] - want) < 1e-13
+    # closed forms: a one-hot token picks a row of W; an identity-like W copies X into the heads
+    E = np.zeros((1, 1, dm)); E[0, 0, 3] = 1.0
+    Q1, K1, V1 = orc.project_qkv(E, W, H, d)
+    assert np.array_equal(Q1[0, :, 0, :].reshape(-1), W[3, :H * d])
+    assert np.array_equal(K1[0, :, 0, :].reshape(-1), W[3, H * d:2 * H * d])
+    assert np.array_equal(V1[0, :, 0, :].reshape(-1), W[3, 2 * H * d:])
+    Wi = np.zeros((H * d, 3 * H * d)); Wi[:, :H * d] = np.eye(H * d); Wi[:, H * d:2 * H * d] = 2 * np.eye(H * d)
+    Xi = r.standard_normal((B, n, H * d))
+    Q2, K2, V2 = orc.project_qkv(Xi, Wi, H, d)
+    assert np.array_equal(Q2.transpose(0, 2, 1, 3).reshape(B, n, H * d), Xi)
+    assert np.array_equal(K2.transpose(0, 2, 1, 3).reshape(B, n, H * d), 2 * Xi)
+    assert not V2.any()
