@@ -164,6 +164,19 @@ int csat_set_lista_weights(csat_ctx* ctx, const void* S, const void* Bm, const f
 int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, const float* theta, int layers,
                                  void* stream);
 
+/* csat_project_qkv -- paper: the projection equation Q = X W^Q, K = X W^K, V = X W^V ("Mathematical Framework"),
+ * for all heads at once, written in the layout csat_forward reads.
+ *   Xq   [B, n_q, d_model]  tokens the queries come from           (context dtype, device)
+ *   Xkv  [B, n,   d_model]  tokens the keys and values come from; the same pointer as Xq for self-attention
+ *   W    [d_model, 3 H d]   row-major; columns [0, H d) = W^Q of heads 0..H-1 (d columns each), then W^K, then W^V
+ *   Q    [B, H, n_q, d]   K, V  [B, H, n, d]                        (outputs, context dtype)
+ * Float32 accumulation, outputs rounded to the context dtype.  With Xq == Xkv and n_q == n this is one launch over
+ * all 3 H d columns, otherwise one for Q and one for K and V.  Enqueued on `stream`, no allocation.  bf16 with
+ * d in {64, 128} and d_model a multiple of 8 runs on the tensor cores; everything else on a plain FFMA kernel.
+ * All pointers 16-byte aligned, else CSAT_ERR_INVALID_ARG. */
+int csat_project_qkv(csat_ctx* ctx, const void* Xq, const void* Xkv, const void* W, int64_t d_model, void* Q, void* K,
+                     void* V, void* stream);
+
 /*
  * csat_forward -- paper: compression, approximate attention matrix, compressed output,
  * LISTA recurrence and reconstruction equations (all of the hot path).

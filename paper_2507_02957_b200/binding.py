@@ -39,6 +39,7 @@ SIGNATURES = {
     "csat_set_decoder_matrix": (_int, [_vp, _vp, _vp]),
     "csat_set_lista_weights": (_int, [_vp, _vp, _vp, _vp, _int, _vp]),
     "csat_set_lista_layer_weights": (_int, [_vp, _vp, _vp, _vp, _int, _vp]),
+    "csat_project_qkv": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp]),
     "csat_forward": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_forward_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
@@ -157,6 +158,11 @@ def csat_set_lista_weights(h, S, Bm, theta, layers, stream=None):
 
 def csat_set_lista_layer_weights(h, S, Bm, theta, layers, stream=None):
     _check(h, load().csat_set_lista_layer_weights(h, _ptr(S), _ptr(Bm), _ptr(theta), int(layers), _stream(stream)))
+
+
+def csat_project_qkv(h, Xq, Xkv, W, d_model, Q, K, V, stream=None):
+    _check(h, load().csat_project_qkv(h, _ptr(Xq), _ptr(Xkv), _ptr(W), int(d_model), _ptr(Q), _ptr(K), _ptr(V),
+                                      _stream(stream)))
 
 
 def csat_forward(h, Q, K, V, out, stream=None):
@@ -326,6 +332,19 @@ class Csat:
         assert S.shape == (self.H, self.d, self.d) and Bm.shape == S.shape and S.dtype == self.torch_dtype == Bm.dtype
         theta = theta.reshape(-1, self.H).to(torch.float32).contiguous()
         csat_set_lista_weights(self.h, S.contiguous(), Bm.contiguous(), theta, theta.shape[0])
+
+    def project_qkv(self, X, W, Xkv=None):
+        """Q, K, V [B,H,tokens,d] from tokens X [B,n_q,d_model] (and Xkv [B,n,d_model] for cross-attention; default X)
+        and W [d_model, 3*H*d] = [W^Q heads | W^K heads | W^V heads]."""
+        Xkv = X if Xkv is None else Xkv
+        dm = X.shape[-1]
+        assert X.shape == (self.B, self.n_q, dm) and Xkv.shape == (self.B, self.n, dm)
+        assert W.shape == (dm, 3 * self.H * self.d) and X.dtype == self.torch_dtype == W.dtype == Xkv.dtype
+        Q = self._new(self.B, self.H, self.n_q, self.d)
+        K = self._new(self.B, self.H, self.n, self.d)
+        V = self._new(self.B, self.H, self.n, self.d)
+        csat_project_qkv(self.h, X, Xkv, W, dm, Q, K, V)
+        return Q, K, V
 
     def set_lista_layer_weights(self, S, Bm, theta):
         """Untied layers: S, Bm [layers,H,d,d] (context dtype), theta [layers,H] float32."""

@@ -626,6 +626,34 @@ int csat_forward_host(csat_ctx* c, const void* Qh, const void* Kh, const void* V
   return CSAT_OK;
 }
 
+int csat_project_qkv(csat_ctx* c, const void* Xq, const void* Xkv, const void* W, int64_t d_model, void* Q, void* K,
+                     void* V, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!Xq || !Xkv || !W || !Q || !K || !V) return fail(c, CSAT_ERR_INVALID_ARG, "csat_project_qkv: NULL pointer");
+  if (!aligned16(Xq) || !aligned16(Xkv) || !aligned16(W) || !aligned16(Q) || !aligned16(K) || !aligned16(V))
+    return fail(c, CSAT_ERR_INVALID_ARG, "csat_project_qkv: pointers must be 16-byte aligned");
+  if (d_model < 1 || d_model > (1 << 20)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_project_qkv: d_model out of range");
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  if (*(volatile int*)c->status != 0)
+    return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
+  const csat::Params& p = c->p;
+  if (3 * p.H * p.d > (1 << 24)) return fail(c, CSAT_ERR_SHAPE, "csat_project_qkv: 3 H d too large");
+  cudaStream_t s = (cudaStream_t)stream;
+  const int hd = (int)(p.H * p.d);
+  int launches = 0;
+  cudaError_t e;
+  if (Xq == Xkv && p.nq == p.n) {
+    e = csat::launch_project(c, Xq, W, p.n, d_model, 0, 3 * hd, Q, K, V, s, &launches);
+  } else {
+    e = csat::launch_project(c, Xq, W, p.nq, d_model, 0, hd, Q, K, V, s, &launches);
+    if (e == cudaSuccess) e = csat::launch_project(c, Xkv, W, p.n, d_model, hd, 2 * hd, Q, K, V, s, &launches);
+  }
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_project_qkv launch");
+  c->last_launches = launches;
+  return CSAT_OK;
+}
+
 int csat_get_compressed(const csat_ctx* c, void* kt, void* vt, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
   csat_ctx* mc = const_cast<csat_ctx*>(c);

@@ -128,6 +128,11 @@ cudaError_t make_attend_tmaps(csat_ctx* c);
 cudaError_t make_layer_weights_tmap(csat_ctx* c);
 cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
 
+// project_sm100.cu : input projections; one launch applies columns [col0, col0 + ncols) of W [dm, 3 H d] to
+// X [B, n_tok, dm] and writes the heads of Q / K / V those columns belong to
+cudaError_t launch_project(csat_ctx* c, const void* X, const void* W, int64_t n_tok, int64_t dm, int col0, int ncols,
+                           void* Q, void* K, void* V, cudaStream_t s, int* launches);
+
 // copies K~ or V~ out of the interleaved workspace: dst [B,H,m,d]
 cudaError_t launch_split_kv(const csat_ctx* c, void* kt, void* vt, cudaStream_t s);
 

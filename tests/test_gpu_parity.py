@@ -560,3 +560,41 @@ def test_output_aligned_to_16_bytes_only_gives_the_same_result():
         assert torch.equal(out, ref)
         assert float(flat[:8].abs().max()) == 0.0
         ctx.close()
+
+
+@pytest.mark.parametrize("case", ["bf16_d64_self", "bf16_d128_self", "bf16_d64_cross", "bf16_ragged_k", "fp32", "bf16_ffma"])
+def test_project_qkv_matches_oracle(case):
+    """Q = X W^Q, K = X W^K, V = X W^V for all heads, in the layout csat_forward reads: tensor-core kernel over
+    several 128 x 256 tiles with ragged tokens, columns and reduction length; cross-attention (two launches);
+    the FFMA kernel for float32 and for forced bf16."""
+    r = np.random.default_rng(71)
+    cfg = {
+        "bf16_d64_self":  dict(dtype="bf16", B=2, H=3, d=64, n=197, n_q=197, dm=192),
+        "bf16_d128_self": dict(dtype="bf16", B=1, H=3, d=128, n=300, n_q=300, dm=256),
+        "bf16_d64_cross": dict(dtype="bf16", B=2, H=5, d=64, n=260, n_q=77, dm=128),
+        "bf16_ragged_k":  dict(dtype="bf16", B=1, H=2, d=64, n=130, n_q=130, dm=72),
+        "fp32":           dict(dtype="fp32", B=2, H=2, d=32, n=50, n_q=20, dm=40),
+        "bf16_ffma":      dict(dtype="bf16", B=1, H=2, d=64, n=70, n_q=70, dm=64),
+    }[case]
+    dt, B, H, d, n, nq, dm = (cfg[k] for k in ("dtype", "B", "H", "d", "n", "n_q", "dm"))
+    ctx = binding.Csat(n, 16, d, H, 3, B=B, n_q=nq, dtype=dt, T=0)
+    if case == "bf16_ffma":
+        ctx.set(force_simt=1)
+    X = wl.round_to_storage(r.standard_normal((B, nq, dm)).astype(np.float32), dt)
+    Xkv = X if nq == n else wl.round_to_storage(r.standard_normal((B, n, dm)).astype(np.float32), dt)
+    W = wl.round_to_storage((r.standard_normal((dm, 3 * H * d)) / np.sqrt(dm)).astype(np.float32), dt)
+    Xd, Wd = to_dev(X, dt), to_dev(W, dt)
+    Xkvd = Xd if nq == n else to_dev(Xkv, dt)
+    Q, K, V = ctx.project_qkv(Xd, Wd, None if nq == n else Xkvd)
+    HD = H * d
+    Qr = orc.project_qkv(X, W, H, d)[0]
+    _, Kr, Vr = orc.project_qkv(Xkv, W, H, d)
+    for name, got, ref in (("Q", Q, Qr), ("K", K, Kr), ("V", V, Vr)):
+        err = rel_err(to_np(got), ref)
+        assert err <= (1e-5 if dt == "fp32" else 8e-3), (case, name, err)     # bf16: output rounding, 2^-8 of max
+    assert binding.csat_last_launch_count(ctx.h) == (1 if nq == n else 2)
+    # the projected tensors feed the forward as they are
+    out = to_np(ctx.forward(Q, K, V))
+    ref = orc.csat_forward(to_np(Q), to_np(K), to_np(V), to_np(ctx.get_phi()), T=0, lam=0.0)
+    assert rel_err(out, ref) <= TOL[dt]
+    ctx.close()
