@@ -257,6 +257,36 @@ def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3, untied: bool = 
             "gflop": f / 1e9}
 
 
+def time_projection(w: wl.Workload, iters: int = 10, warmup: int = 3) -> dict:
+    """The Q, K, V projections in front of the path (csat_project_qkv) for the workload's shape, d_model = H d,
+    self-attention form (one GEMM over 3 H d columns); L2 flushed between iterations."""
+    import torch
+    from paper_2507_02957_b200 import binding
+    dm = w.H * w.d
+    g = torch.Generator(device="cuda")
+    g.manual_seed(11)
+    X = torch.randn(w.B, w.n, dm, device="cuda", generator=g).to(torch.bfloat16)
+    W = (torch.randn(dm, 3 * dm, device="cuda", generator=g) / np.sqrt(dm)).to(torch.bfloat16)
+    ctx = binding.Csat(w.n, w.m, w.d, w.H, w.phi_seed, B=w.B, dtype="bf16", T=0)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    Q, K, V = (torch.empty(w.B, w.H, w.n, w.d, dtype=torch.bfloat16, device="cuda") for _ in range(3))
+    for _ in range(warmup):
+        binding.csat_project_qkv(ctx.h, X, X, W, dm, Q, K, V)
+    times = []
+    for _ in range(iters):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        binding.csat_project_qkv(ctx.h, X, X, W, dm, Q, K, V)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ctx.close()
+    ms = float(np.median(times))
+    f = 2.0 * w.B * w.n * dm * 3 * dm
+    return {"ms": ms, "tflops": f / (ms * 1e-3) / 1e12, "gflop": f / 1e9, "d_model": dm}
+
+
 def run_csat(args, w: wl.Workload) -> dict:
     import torch
     import torch.distributed as dist
@@ -366,6 +396,8 @@ def run_csat(args, w: wl.Workload) -> dict:
                 extra[f"c5_sweep_n{n}"] = time_small(wl.sweep_config(n))
             if w.T > 1 and w.dtype == "bf16":
                 extra[f"{w.name}_untied_layers"] = time_small(w, untied=True)
+            if w.dtype == "bf16" and w.n == w.n_q:
+                extra[f"{w.name}_qkv_projection"] = time_projection(w)
             result["other_workloads"] = extra
         if not args.no_cpu_baseline:
             inp = {k: host[k].float().numpy() for k in "QKV"}

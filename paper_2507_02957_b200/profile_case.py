@@ -3,6 +3,7 @@
     python -m paper_2507_02957_b200.profile_case forward N M D B H T [--nq NQ] [--iters I] [--dtype bf16|fp32] [--untied]
     python -m paper_2507_02957_b200.profile_case workload c1|c2|c3|c4|c5 [--iters I]
     python -m paper_2507_02957_b200.profile_case ensembles N M D H        (regenerates Phi with every ensemble)
+    python -m paper_2507_02957_b200.profile_case project N D B H DMODEL [--iters I]   (the Q, K, V projections)
 
 A small driver to put under a profiler (ncu -k regex:<kernel> ...): 3 warm-up forwards, then I timed ones.
 Inputs are seeded random tensors (N(0, 1/d) for `forward`, the workload's own recipe for `workload`).
@@ -51,6 +52,10 @@ def main():
     e = sub.add_parser("ensembles")
     for name in ("n", "m", "d", "H"):
         e.add_argument(name, type=int)
+    pj = sub.add_parser("project")
+    for name in ("n", "d", "B", "H", "dm"):
+        pj.add_argument(name, type=int)
+    pj.add_argument("--iters", type=int, default=10)
     a = ap.parse_args()
 
     if a.cmd == "forward":
@@ -79,6 +84,29 @@ def main():
         if inp["Psi"] is not None:
             ctx.set_dictionary(torch.from_numpy(inp["Psi"]).cuda().to(dt))
         print(w.name, _timed_forwards(ctx, Q, K, V, a.iters))
+        ctx.close()
+    elif a.cmd == "project":
+        g = torch.Generator(device="cuda")
+        g.manual_seed(1)
+        X = torch.randn(a.B, a.n, a.dm, device="cuda", generator=g).to(torch.bfloat16)
+        W = (torch.randn(a.dm, 3 * a.H * a.d, device="cuda", generator=g) / np.sqrt(a.dm)).to(torch.bfloat16)
+        ctx = binding.Csat(a.n, min(64, a.n), a.d, a.H, 0, B=a.B, dtype="bf16", T=0)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        Q, K, V = (torch.empty(a.B, a.H, a.n, a.d, dtype=torch.bfloat16, device="cuda") for _ in range(3))
+        for _ in range(3):
+            binding.csat_project_qkv(ctx.h, X, X, W, a.dm, Q, K, V)
+        times = []
+        for _ in range(a.iters):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            binding.csat_project_qkv(ctx.h, X, X, W, a.dm, Q, K, V)
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = float(np.median(times))
+        fl = 2.0 * a.B * a.n * a.dm * 3 * a.H * a.d
+        print(vars(a), {"ms": round(ms, 4), "tflops": round(fl / ms / 1e9, 1)})
         ctx.close()
     else:
         ctx = binding.Csat(a.n, a.m, a.d, a.H, 0, dtype="bf16")
