@@ -17,6 +17,8 @@ paper's column vectors alpha_i, Z_i, C_i appear here as 1 x d rows):
   lista              the same recurrence with supplied S, B and per-layer theta_t
   reconstruct        C^_i = Psi alpha^_i                  (reconstruction equation)
   project_qkv        Q = X W^Q, K = X W^K, V = X W^V      (projection equation, one set of d_k columns per head)
+  csat_backward      gradients of the forward with respect to Q, K, V (chain rule through the equations above,
+                     last to first; the paper trains through the unrolled decoder but prints no backward pass)
 
 Reading of the decoder (the paper's "Z_i = Phi Psi alpha_i" with Phi in R^{m x n}
 cannot multiply a d_k-vector): the sensing matrix of the decoder is a d x d matrix
@@ -243,3 +245,98 @@ def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=Non
             if stages is not None:
                 stages.append(st)
     return out
+
+
+# ----------------------------------------------------------------------------
+# backward: d out / d (Q, K, V), chain rule through the forward's equations in reverse order
+# ----------------------------------------------------------------------------
+def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None, scale=None, weights=None,
+                       Phi_v_h=None, stages: dict | None = None):
+    """Vector-Jacobian product of csat_forward_head for one (batch, head): given G = dL/d out [n_q,d], returns
+    (dL/dQ [n_q,d], dL/dK [n,d], dL/dV [n,d]).  Phi, Psi and the decoder weights are constants.
+    The shrinkage eta_theta has derivative 1 where |x| > theta and 0 elsewhere (0 is taken at |x| = theta).
+    stages (optional dict) receives min_margin [n_q] = min over layers and columns of | |x_t| - theta_t |, which
+    tells how close a row came to a kink of eta."""
+    Q = np.asarray(Q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    G = np.asarray(G, F64)
+    Phi_h = np.asarray(Phi_h, F64)
+    d = Q.shape[1]
+    Phi_v = Phi_h if Phi_v_h is None else np.asarray(Phi_v_h, F64)
+    sc = (1.0 / np.sqrt(d)) if scale is None else float(scale)
+    # forward, keeping what the backward needs
+    Kt = compress(Phi_h, K)
+    Vt = compress(Phi_v, V)
+    A = softmax_rows(compressed_scores(Q, Kt, scale))
+    Z = compressed_output(A, Vt)
+    margin = np.full(Q.shape[0], np.inf)
+    if int(T) == 0:
+        dZ = G.copy()
+    else:
+        if weights is not None:
+            S_w, B_w, thetas = weights
+            S_w, B_w = np.asarray(S_w, F64), np.asarray(B_w, F64)
+            S_l = [S_w[t] if S_w.ndim == 3 else S_w for t in range(int(T))]
+            B_l = [B_w[t] if B_w.ndim == 3 else B_w for t in range(int(T))]
+            thetas = [float(th) for th in thetas]
+        else:
+            Dm = default_decoder_matrix(Phi_v, d) if D is None else np.asarray(D, F64)
+            M = Dm if Psi is None else Dm @ np.asarray(Psi, F64)
+            S_dec, B_dec, theta, _ = decoder_setup(M, lam, step)
+            S_l, B_l, thetas = [S_dec] * int(T), [B_dec] * int(T), [float(theta)] * int(T)
+        alpha = np.zeros_like(Z)
+        xs = []
+        for t in range(int(T)):
+            x = alpha @ S_l[t] + Z @ B_l[t]
+            xs.append(x)
+            margin = np.minimum(margin, np.abs(np.abs(x) - thetas[t]).min(axis=1))
+            alpha = soft_threshold(x, thetas[t])
+        # out = alpha Psi^T  ->  d alpha = G Psi
+        d_alpha = G if Psi is None else G @ np.asarray(Psi, F64)
+        dZ = np.zeros_like(Z)
+        for t in range(int(T) - 1, -1, -1):
+            dx = d_alpha * (np.abs(xs[t]) > thetas[t])          # through eta_theta
+            dZ += dx @ B_l[t].T                                  # x_t = alpha_t S_t + Z B_t
+            d_alpha = dx @ S_l[t].T
+    if stages is not None:
+        stages.update(min_margin=margin, dZ=dZ, A=A, Z=Z)
+    # Z = A~ V~
+    dA = dZ @ Vt.T
+    dVt = A.T @ dZ
+    # A~ = softmax(S) row-wise:  dS = A o (dA - rowsum(dA o A))
+    dS = A * (dA - (dA * A).sum(axis=1, keepdims=True))
+    # S = sc Q K~^T
+    dQ = sc * (dS @ Kt)
+    dKt = sc * (dS.T @ Q)
+    # K~ = Phi K, V~ = Phi_V V
+    dK = Phi_h.T @ dKt
+    dV = Phi_v.T @ dVt
+    return dQ, dK, dV
+
+
+def csat_backward(Q, K, V, Phi, G, *, T, lam, Psi=None, D=None, step=None, scale=None, weights=None, Phi_V=None,
+                  stages: list | None = None):
+    """Vector-Jacobian product of csat_forward: G [B,H,n_q,d] -> (dQ [B,H,n_q,d], dK [B,H,n,d], dV [B,H,n,d])."""
+    Q = np.asarray(Q)
+    B, H, nq, d = Q.shape
+    n = np.asarray(K).shape[2]
+    dQ = np.empty((B, H, nq, d), dtype=F64)
+    dK = np.empty((B, H, n, d), dtype=F64)
+    dV = np.empty((B, H, n, d), dtype=F64)
+    for b in range(B):
+        for h in range(H):
+            psi_h = None if Psi is None else (Psi if np.ndim(Psi) == 2 else Psi[h])
+            D_h = None if D is None else D[h]
+            w_h = None
+            if weights is not None:
+                per_layer = np.ndim(weights[0]) == 4
+                w_h = (np.asarray(weights[0])[:, h] if per_layer else weights[0][h],
+                       np.asarray(weights[1])[:, h] if per_layer else weights[1][h], [th[h] for th in weights[2]])
+            st = {} if stages is not None else None
+            dQ[b, h], dK[b, h], dV[b, h] = csat_backward_head(
+                Q[b, h], K[b, h], V[b, h], Phi[h], G[b, h], T=T, lam=lam, Psi=psi_h, D=D_h, step=step, scale=scale,
+                weights=w_h, Phi_v_h=None if Phi_V is None else Phi_V[h], stages=st)
+            if stages is not None:
+                stages.append(st)
+    return dQ, dK, dV

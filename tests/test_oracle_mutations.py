@@ -135,8 +135,29 @@ def _project_W_transposed_per_head(X, W, H, d):
     return K, Q, V
 
 
+def _backward_scale_dropped(Q, K, V, Phi_h, G, **kw):
+    dQ, dK, dV = _orig_backward_head(Q, K, V, Phi_h, G, **kw)
+    s = np.sqrt(np.asarray(Q).shape[1]) if kw.get("scale") is None else 1.0 / kw["scale"]
+    return dQ * s, dK * s, dV
+
+
+def _backward_softmax_without_row_term(Q, K, V, Phi_h, G, **kw):
+    # dS = A o dA, the projection onto the simplex's tangent space forgotten
+    st = {}
+    _orig_backward_head(Q, K, V, Phi_h, G, **{**kw, "stages": st})
+    Phi_h = np.asarray(Phi_h, F64)
+    Phi_v = Phi_h if kw.get("Phi_v_h") is None else np.asarray(kw["Phi_v_h"], F64)
+    Kt, Vt = Phi_h @ np.asarray(K, F64), Phi_v @ np.asarray(V, F64)
+    sc = 1.0 / np.sqrt(np.asarray(Q).shape[1]) if kw.get("scale") is None else kw["scale"]
+    dS = st["A"] * (st["dZ"] @ Vt.T)
+    if kw.get("stages") is not None:
+        kw["stages"].update(st)
+    return sc * dS @ Kt, Phi_h.T @ (sc * dS.T @ np.asarray(Q, F64)), Phi_v.T @ (st["A"].T @ st["dZ"])
+
+
 _orig_lista = orc.lista
 _orig_project = orc.project_qkv
+_orig_backward_head = orc.csat_backward_head
 _orig_setup = orc.decoder_setup
 _orig_ista = orc.ista
 
@@ -163,6 +184,8 @@ MUTATIONS = {
     "lista: layers in reverse order": ("lista", _lista_layers_reversed),
     "project: head and q/k/v order swapped": ("project_qkv", _project_heads_interleaved),
     "project: queries and keys exchanged": ("project_qkv", _project_W_transposed_per_head),
+    "backward: score scale dropped": ("csat_backward_head", _backward_scale_dropped),
+    "backward: softmax Jacobian without the row term": ("csat_backward_head", _backward_softmax_without_row_term),
     "compress: |Phi|": ("compress", _compress_abs),
     "output: weights ignored": ("compressed_output", _output_uses_unweighted),
 }

@@ -645,3 +645,115 @@ def test_project_qkv_matches_scalar_loops_and_layout():
     assert np.array_equal(Q2.transpose(0, 2, 1, 3).reshape(B, n, H * d), Xi)
     assert np.array_equal(K2.transpose(0, 2, 1, 3).reshape(B, n, H * d), 2 * Xi)
     assert not V2.any()
+
+
+# ---------------------------------------------------------------------------------------------------
+# backward (vector-Jacobian product of the forward with respect to Q, K, V)
+# ---------------------------------------------------------------------------------------------------
+def _torch_forward(Q, K, V, Phi, Phi_v, S_l, B_l, thetas, Psi, scale):
+    """The forward written with torch float64 ops, for autograd (an independent derivation of the gradient)."""
+    import torch
+    Kt, Vt = Phi @ K, Phi_v @ V
+    A = torch.softmax(scale * (Q @ Kt.T), dim=1)
+    Z = A @ Vt
+    alpha = torch.zeros_like(Z)
+    out = Z
+    for S_t, B_t, th in zip(S_l, B_l, thetas):
+        x = alpha @ S_t + Z @ B_t
+        alpha = torch.sign(x) * torch.relu(torch.abs(x) - th)
+        out = alpha
+    if Psi is not None and len(thetas) > 0:
+        out = out @ Psi.T
+    return out
+
+
+def _backward_case(seed, T, with_psi, separate, untied):
+    import torch
+    r = np.random.default_rng(seed)
+    n, nq, d, m = 14, 6, 5, 7
+    Q, K, V = r.standard_normal((nq, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    Phi = r.standard_normal((m, n)) / np.sqrt(m)
+    Phi_v = r.standard_normal((m, n)) / np.sqrt(m) if separate else None
+    Psi = (np.eye(d) + 0.3 * r.standard_normal((d, d))) if with_psi else None
+    G = r.standard_normal((nq, d))
+    lam = 0.15
+    if untied:
+        S = 0.5 * np.eye(d) + 0.2 * r.standard_normal((T, d, d))
+        Bm = 0.5 * r.standard_normal((T, d, d))
+        thetas = list(0.02 + 0.05 * r.random(T))
+        weights = (S, Bm, thetas)
+        S_l, B_l = list(S), list(Bm)
+    else:
+        weights = None
+        Dm = orc.default_decoder_matrix(Phi if Phi_v is None else Phi_v, d)
+        M = Dm if Psi is None else Dm @ Psi
+        S_dec, B_dec, theta, _ = orc.decoder_setup(M, lam)
+        S_l, B_l, thetas = [S_dec] * T, [B_dec] * T, [float(theta)] * T
+    st = {}
+    got = orc.csat_backward_head(Q, K, V, Phi, G, T=T, lam=lam, Psi=Psi, weights=weights, Phi_v_h=Phi_v, stages=st)
+    tq, tk, tv = (torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in (Q, K, V))
+    t = lambda x: None if x is None else torch.tensor(x, dtype=torch.float64)
+    out = _torch_forward(tq, tk, tv, t(Phi), t(Phi if Phi_v is None else Phi_v), [t(x) for x in S_l], [t(x) for x in B_l],
+                         thetas, t(Psi), 1.0 / np.sqrt(d))
+    # the torch forward is the oracle's forward
+    ref_out = orc.csat_forward_head(Q, K, V, Phi, T=T, lam=lam, Psi=Psi, weights=weights, Phi_v_h=Phi_v)
+    assert np.allclose(out.detach().numpy(), ref_out, rtol=0, atol=1e-12)
+    (out * t(G)).sum().backward()
+    for name, g, ref in zip("QKV", got, (tq.grad, tk.grad, tv.grad)):
+        assert np.allclose(g, ref.numpy(), rtol=1e-10, atol=1e-12), (name, seed, T)
+    return Q, K, V, Phi, Phi_v, Psi, G, lam, weights, got, st
+
+
+def test_backward_matches_autograd():
+    for seed, T, with_psi, separate, untied in [(81, 0, False, False, False), (82, 1, False, False, False),
+                                                (83, 4, True, False, False), (84, 3, False, True, False),
+                                                (85, 5, True, True, True), (86, 2, False, False, True)]:
+        _backward_case(seed, T, with_psi, separate, untied)
+
+
+def test_backward_matches_central_differences():
+    """dL/dx_k by (L(x + h e_k) - L(x - h e_k)) / 2h with L = sum(out o G), along random directions, on a case
+    whose iterates keep clear of the kinks of eta by far more than the step."""
+    Q, K, V, Phi, Phi_v, Psi, G, lam, weights, got, st = _backward_case(87, 4, True, False, False)
+    assert st["min_margin"].min() > 1e-4
+    r = np.random.default_rng(88)
+    L = lambda q, k, v: float((orc.csat_forward_head(q, k, v, Phi, T=4, lam=lam, Psi=Psi, weights=weights) * G).sum())
+    h = 1e-6
+    for which in range(3):
+        for _ in range(4):
+            dirs = [np.zeros_like(Q), np.zeros_like(K), np.zeros_like(V)]
+            dirs[which] = r.standard_normal(dirs[which].shape)
+            fd = (L(Q + h * dirs[0], K + h * dirs[1], V + h * dirs[2]) - L(Q - h * dirs[0], K - h * dirs[1], V - h * dirs[2])) / (2 * h)
+            an = float((got[which] * dirs[which]).sum())
+            assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (which, fd, an)
+
+
+def test_backward_special_cases():
+    r = np.random.default_rng(89)
+    n, nq, d, m = 9, 4, 3, 5
+    Q, K, V = r.standard_normal((nq, d)), r.standard_normal((n, d)), r.standard_normal((n, d))
+    Phi = r.standard_normal((m, n))
+    G = r.standard_normal((nq, d))
+    # T = 0 and m = 1: the softmax over one measurement is 1, out = Phi V for every query: dQ = 0, dK = 0,
+    # dV = Phi^T (sum of the rows of G)
+    dQ, dK, dV = orc.csat_backward_head(Q, K, V, Phi[:1], G, T=0, lam=0.0)
+    assert np.allclose(dQ, 0, atol=1e-15) and np.allclose(dK, 0, atol=1e-15)
+    assert np.allclose(dV, Phi[:1].T @ G.sum(axis=0, keepdims=True), rtol=1e-12, atol=1e-14)
+    # a threshold above every |x|: the output is 0 and so is every gradient
+    big = (np.zeros((d, d)), np.eye(d), [1e6, 1e6])
+    for g in orc.csat_backward_head(Q, K, V, Phi, G, T=2, lam=0.0, weights=big):
+        assert not g.any()
+    # theta = 0, S = 0, B = I, one layer: the decoder is the identity, the gradient is the T = 0 gradient
+    ident = (np.zeros((d, d)), np.eye(d), [0.0])
+    a = orc.csat_backward_head(Q, K, V, Phi, G, T=1, lam=0.0, weights=ident)
+    b = orc.csat_backward_head(Q, K, V, Phi, G, T=0, lam=0.0)
+    for x, y in zip(a, b):
+        assert np.allclose(x, y, rtol=1e-12, atol=1e-14)
+    # whole-batch wrapper = the heads one by one
+    Qb, Kb, Vb = (r.standard_normal((2, 2, s, d)) for s in (nq, n, n))
+    Phib = r.standard_normal((2, m, n))
+    Gb = r.standard_normal((2, 2, nq, d))
+    full = orc.csat_backward(Qb, Kb, Vb, Phib, Gb, T=2, lam=0.1)
+    one = orc.csat_backward_head(Qb[1, 0], Kb[1, 0], Vb[1, 0], Phib[0], Gb[1, 0], T=2, lam=0.1)
+    for x, y in zip(full, one):
+        assert np.array_equal(x[1, 0], y)
