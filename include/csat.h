@@ -164,6 +164,21 @@ int csat_set_lista_weights(csat_ctx* ctx, const void* S, const void* Bm, const f
 int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, const float* theta, int layers,
                                  void* stream);
 
+/* csat_backward -- gradients of csat_forward with respect to its inputs.  The paper's decoder is an
+ * unrolled network meant to be trained by backpropagation (its section on the sparse decoder), but the paper
+ * prints no backward pass; this is the chain rule through the forward's equations in reverse order, with the
+ * derivative of eta_theta taken as 1 where |x| > theta and 0 elsewhere.  Phi, Psi and the decoder weights are
+ * constants.
+ *   Q [B,H,n_q,d], K, V [B,H,n,d]   the forward's inputs          (context dtype, device)
+ *   dOut [B,H,n_q,d]                gradient of the loss with respect to csat_forward's output
+ *   dQ [B,H,n_q,d], dK, dV [B,H,n,d]  outputs (context dtype)
+ * Nothing of an earlier csat_forward is reused: the call compresses K, V again and recomputes what it needs in
+ * float32.  Its first call allocates float32 scratch (B H (n_q (d + 2) + 2 m d) floats, counted by
+ * csat_workspace_bytes).  CSAT_T <= 32 and d <= 256, else CSAT_ERR_UNSUPPORTED.  This first version runs on plain
+ * FFMA kernels for both storage types. */
+int csat_backward(csat_ctx* ctx, const void* Q, const void* K, const void* V, const void* dOut, void* dQ, void* dK,
+                  void* dV, void* stream);
+
 /* csat_project_qkv -- paper: the projection equation Q = X W^Q, K = X W^K, V = X W^V ("Mathematical Framework"),
  * for all heads at once, written in the layout csat_forward reads.
  *   Xq   [B, n_q, d_model]  tokens the queries come from           (context dtype, device)

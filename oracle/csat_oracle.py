@@ -251,12 +251,15 @@ def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=Non
 # backward: d out / d (Q, K, V), chain rule through the forward's equations in reverse order
 # ----------------------------------------------------------------------------
 def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None, scale=None, weights=None,
-                       Phi_v_h=None, stages: dict | None = None):
+                       Phi_v_h=None, stages: dict | None = None, kv_round=None):
     """Vector-Jacobian product of csat_forward_head for one (batch, head): given G = dL/d out [n_q,d], returns
     (dL/dQ [n_q,d], dL/dK [n,d], dL/dV [n,d]).  Phi, Psi and the decoder weights are constants.
     The shrinkage eta_theta has derivative 1 where |x| > theta and 0 elsewhere (0 is taken at |x| = theta).
     stages (optional dict) receives min_margin [n_q] = min over layers and columns of | |x_t| - theta_t |, which
-    tells how close a row came to a kink of eta."""
+    tells how close a row came to a kink of eta.
+    kv_round (optional callable) is applied to K~ and V~ before they are used: a library that keeps them in a
+    16-bit workspace takes its shrinkage decisions from the rounded values, and so must the reference.  The
+    gradient then treats the rounding as the identity."""
     Q = np.asarray(Q, F64)
     K = np.asarray(K, F64)
     V = np.asarray(V, F64)
@@ -268,6 +271,8 @@ def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None
     # forward, keeping what the backward needs
     Kt = compress(Phi_h, K)
     Vt = compress(Phi_v, V)
+    if kv_round is not None:
+        Kt, Vt = np.asarray(kv_round(Kt), F64), np.asarray(kv_round(Vt), F64)
     A = softmax_rows(compressed_scores(Q, Kt, scale))
     Z = compressed_output(A, Vt)
     margin = np.full(Q.shape[0], np.inf)
@@ -316,7 +321,7 @@ def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None
 
 
 def csat_backward(Q, K, V, Phi, G, *, T, lam, Psi=None, D=None, step=None, scale=None, weights=None, Phi_V=None,
-                  stages: list | None = None):
+                  stages: list | None = None, kv_round=None):
     """Vector-Jacobian product of csat_forward: G [B,H,n_q,d] -> (dQ [B,H,n_q,d], dK [B,H,n,d], dV [B,H,n,d])."""
     Q = np.asarray(Q)
     B, H, nq, d = Q.shape
@@ -336,7 +341,7 @@ def csat_backward(Q, K, V, Phi, G, *, T, lam, Psi=None, D=None, step=None, scale
             st = {} if stages is not None else None
             dQ[b, h], dK[b, h], dV[b, h] = csat_backward_head(
                 Q[b, h], K[b, h], V[b, h], Phi[h], G[b, h], T=T, lam=lam, Psi=psi_h, D=D_h, step=step, scale=scale,
-                weights=w_h, Phi_v_h=None if Phi_V is None else Phi_V[h], stages=st)
+                weights=w_h, Phi_v_h=None if Phi_V is None else Phi_V[h], stages=st, kv_round=kv_round)
             if stages is not None:
                 stages.append(st)
     return dQ, dK, dV

@@ -41,6 +41,7 @@ SIGNATURES = {
     "csat_set_lista_layer_weights": (_int, [_vp, _vp, _vp, _vp, _int, _vp]),
     "csat_project_qkv": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp]),
     "csat_forward": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "csat_backward": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_forward_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
     "csat_get_decoder": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
@@ -167,6 +168,11 @@ def csat_project_qkv(h, Xq, Xkv, W, d_model, Q, K, V, stream=None):
 
 def csat_forward(h, Q, K, V, out, stream=None):
     _check(h, load().csat_forward(h, _ptr(Q), _ptr(K), _ptr(V), _ptr(out), _stream(stream)))
+
+
+def csat_backward(h, Q, K, V, dOut, dQ, dK, dV, stream=None):
+    _check(h, load().csat_backward(h, _ptr(Q), _ptr(K), _ptr(V), _ptr(dOut), _ptr(dQ), _ptr(dK), _ptr(dV),
+                                   _stream(stream)))
 
 
 def csat_forward_host(h, Qh, Kh, Vh, outh, stream=None):
@@ -332,6 +338,12 @@ class Csat:
         assert S.shape == (self.H, self.d, self.d) and Bm.shape == S.shape and S.dtype == self.torch_dtype == Bm.dtype
         theta = theta.reshape(-1, self.H).to(torch.float32).contiguous()
         csat_set_lista_weights(self.h, S.contiguous(), Bm.contiguous(), theta, theta.shape[0])
+
+    def backward(self, Q, K, V, dOut):
+        """Gradients of forward(Q, K, V) with respect to Q, K, V for the output gradient dOut."""
+        dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+        csat_backward(self.h, Q, K, V, dOut, dQ, dK, dV)
+        return dQ, dK, dV
 
     def project_qkv(self, X, W, Xkv=None):
         """Q, K, V [B,H,tokens,d] from tokens X [B,n_q,d_model] (and Xkv [B,n,d_model] for cross-attention; default X)

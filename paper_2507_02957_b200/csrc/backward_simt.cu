@@ -1,0 +1,392 @@
+// Backward of the CSAT forward with respect to Q, K, V: the chain rule through the paper's equations, last to
+// first (reconstruction C^ = Psi alpha, the unrolled recurrence alpha^{t+1} = eta_theta(alpha^t S + z B), the
+// compressed output Z = A~ V~, the softmax, the scores S = Q K~^T / sqrt(d_k), the compression K~ = Phi K,
+// V~ = Phi V).  The paper trains through the unrolled decoder but prints no backward pass; eta_theta has derivative
+// 1 where |x| > theta and 0 elsewhere.
+//
+// First CUDA version: plain FFMA kernels, float32 arithmetic, nothing stored by the forward.  After the
+// compression (the forward's own kernel) three kernels run:
+//   bwd_rows_kernel : one warp per query row.  Recomputes the row's scores, softmax statistics and Z, runs the
+//                     recurrence forward keeping one bit per layer and column (|x_t| > theta_t), then backward:
+//                     d alpha_T = G Psi, dx_t = d alpha_{t+1} o mask_t, dZ += dx_t B_t^T, d alpha_t = dx_t S_t^T.
+//                     Stores dZ, L = log sum exp of the row's scores and D = <dZ, Z>, then sweeps K~|V~ again:
+//                     p = exp(s - L), dS = p (dZ . V~_r - D), dQ = scale sum_r dS_r K~_r.
+//   bwd_cols_kernel : one warp per measurement r, all query rows in turn (deterministic, no atomics):
+//                     dK~_r = scale sum_i dS_ir Q_i,  dV~_r = sum_i p_ir dZ_i.
+//   bwd_phiT_kernel : dK = Phi^T dK~, dV = Phi_V^T dV~.
+#include "csat_internal.h"
+
+namespace csat {
+namespace {
+
+constexpr int kRowWarps = 8;
+constexpr int kColWarps = 8;
+constexpr int kColRows = 16;      // query rows staged per step of bwd_cols_kernel
+
+template <typename T> __device__ __forceinline__ float ldf(const T* p, int64_t i);
+template <> __device__ __forceinline__ float ldf<float>(const float* p, int64_t i) { return p[i]; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p, int64_t i) {
+  return __bfloat162float(p[i]);
+}
+template <typename T> __device__ __forceinline__ void stf(T* p, int64_t i, float v);
+template <> __device__ __forceinline__ void stf<float>(float* p, int64_t i, float v) { p[i] = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p, int64_t i, float v) {
+  p[i] = __float2bfloat16_rn(v);
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// lane owns columns lane + 32 j.  y[col] = sum_k x[k] W[k][col]
+template <int DC>
+__device__ __forceinline__ void row_times(const float (&x)[DC], float (&y)[DC], const float* __restrict__ W, int d, int lane) {
+#pragma unroll
+  for (int j = 0; j < DC; ++j) y[j] = 0.f;
+#pragma unroll
+  for (int jk = 0; jk < DC; ++jk)
+    for (int l = 0; l < 32; ++l) {
+      const int k = 32 * jk + l;
+      const float xk = __shfl_sync(0xffffffffu, x[jk], l);
+      if (k < d) {
+#pragma unroll
+        for (int j = 0; j < DC; ++j) {
+          const int col = lane + 32 * j;
+          if (col < d) y[j] = fmaf(xk, W[(int64_t)k * d + col], y[j]);
+        }
+      }
+    }
+}
+// y[k] = sum_c x[c] W[k][c]   (x times the transpose of W)
+template <int DC>
+__device__ __forceinline__ void row_times_T(const float (&x)[DC], float (&y)[DC], const float* __restrict__ W, int d, int lane) {
+#pragma unroll
+  for (int j = 0; j < DC; ++j) y[j] = 0.f;
+#pragma unroll
+  for (int jc = 0; jc < DC; ++jc)
+    for (int l = 0; l < 32; ++l) {
+      const int c = 32 * jc + l;
+      const float xc = __shfl_sync(0xffffffffu, x[jc], l);
+      if (c < d) {
+#pragma unroll
+        for (int j = 0; j < DC; ++j) {
+          const int k = lane + 32 * j;
+          if (k < d) y[j] = fmaf(xc, W[(int64_t)k * d + c], y[j]);
+        }
+      }
+    }
+}
+
+template <typename T, int DC>   // DC = ceil(d / 32)
+__global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
+    T* __restrict__ dQ, float* __restrict__ ws_dZ, float* __restrict__ ws_LD, const T* __restrict__ Q,
+    const T* __restrict__ G, const T* __restrict__ kv, const float* __restrict__ S_dec, const float* __restrict__ B_dec,
+    int64_t layer_stride, const float* __restrict__ theta, int theta_stride, const float* __restrict__ psi_f32,
+    int64_t nq, int64_t m, int d, int H, int T_iters, float scale) {
+  extern __shared__ float smem[];
+  const int d2 = 2 * d, ldk = d2 + 1;
+  float* kvs = smem;                               // [32][2d+1]
+  float* qs = smem + 32 * ldk;                     // [warps][d]
+  float* dzs = qs + kRowWarps * d;                 // [warps][d]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, h = bh % H;
+  const int64_t row = (int64_t)blockIdx.x * kRowWarps + warp;
+  const bool live = row < nq;
+  const int64_t grow = (int64_t)bh * nq + (live ? row : 0);
+  const T* kvb = kv + (int64_t)bh * m * d2;
+  float* q = qs + warp * d;
+  float* dzr = dzs + warp * d;
+  for (int c = lane; c < d; c += 32) q[c] = live ? ldf(Q, grow * d + c) : 0.f;
+
+  // ---- forward: scores, softmax statistics, Z ----
+  float z[DC];
+#pragma unroll
+  for (int j = 0; j < DC; ++j) z[j] = 0.f;
+  float run_max = -INFINITY, run_sum = 0.f;
+  for (int64_t r0 = 0; r0 < m; r0 += 32) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < 32 * d2; i += kRowWarps * 32) {
+      const int rr = i / d2, c = i % d2;
+      kvs[rr * ldk + c] = (r0 + rr < m) ? ldf(kvb, (r0 + rr) * d2 + c) : 0.f;
+    }
+    __syncthreads();
+    float s = 0.f;
+    const float* kr = kvs + lane * ldk;
+    for (int c = 0; c < d; ++c) s = fmaf(q[c], kr[c], s);
+    s = (r0 + lane < m) ? s * scale : -INFINITY;
+    const float new_max = fmaxf(run_max, warp_max(s));
+    const float corr = expf(run_max - new_max);
+    const float p = expf(s - new_max);
+    run_sum = run_sum * corr + warp_sum(p);
+    run_max = new_max;
+#pragma unroll
+    for (int j = 0; j < DC; ++j) z[j] *= corr;
+    for (int rr = 0; rr < 32; ++rr) {
+      const float pr = __shfl_sync(0xffffffffu, p, rr);
+      const float* vr = kvs + rr * ldk + d;
+#pragma unroll
+      for (int j = 0; j < DC; ++j) {
+        const int col = lane + 32 * j;
+        if (col < d) z[j] = fmaf(pr, vr[col], z[j]);
+      }
+    }
+  }
+  const float inv = 1.f / run_sum;
+#pragma unroll
+  for (int j = 0; j < DC; ++j) z[j] *= inv;
+  const float L = run_max + logf(run_sum);          // log sum exp of the row's scaled scores
+
+  // ---- recurrence forward (masks), then backward: dZ ----
+  float g[DC], dz[DC];
+#pragma unroll
+  for (int j = 0; j < DC; ++j) {
+    const int col = lane + 32 * j;
+    g[j] = (live && col < d) ? ldf(G, grow * d + col) : 0.f;
+  }
+  if (T_iters == 0) {
+#pragma unroll
+    for (int j = 0; j < DC; ++j) dz[j] = g[j];
+  } else {
+    const float* Sh = S_dec + (int64_t)h * d * d;
+    const float* Bh = B_dec + (int64_t)h * d * d;
+    uint32_t mask[DC];
+    float a[DC], c[DC], t[DC];
+#pragma unroll
+    for (int j = 0; j < DC; ++j) { mask[j] = 0u; a[j] = 0.f; }
+    for (int it = 0; it < T_iters; ++it) {
+      const float th = theta[(int64_t)it * theta_stride + h];
+      if (it == 0 || layer_stride != 0) row_times<DC>(z, c, Bh + layer_stride * it, d, lane);      // z B_t
+      if (it > 0) row_times<DC>(a, t, Sh + layer_stride * it, d, lane);
+#pragma unroll
+      for (int j = 0; j < DC; ++j) {
+        const float x = (it > 0 ? t[j] : 0.f) + c[j];
+        if (fabsf(x) > th) mask[j] |= 1u << it;
+        a[j] = x - fminf(fmaxf(x, -th), th);
+      }
+    }
+    float da[DC], dx[DC];
+    if (psi_f32) row_times<DC>(g, da, psi_f32 + (int64_t)h * d * d, d, lane);     // d alpha_T = G Psi
+    else {
+#pragma unroll
+      for (int j = 0; j < DC; ++j) da[j] = g[j];
+    }
+#pragma unroll
+    for (int j = 0; j < DC; ++j) dz[j] = 0.f;
+    for (int it = T_iters - 1; it >= 0; --it) {
+#pragma unroll
+      for (int j = 0; j < DC; ++j) dx[j] = ((mask[j] >> it) & 1u) ? da[j] : 0.f;
+      row_times_T<DC>(dx, t, Bh + layer_stride * it, d, lane);                    // dZ += dx B_t^T
+#pragma unroll
+      for (int j = 0; j < DC; ++j) dz[j] += t[j];
+      if (it > 0) row_times_T<DC>(dx, da, Sh + layer_stride * it, d, lane);       // d alpha_t = dx S_t^T
+    }
+  }
+  float part = 0.f;
+#pragma unroll
+  for (int j = 0; j < DC; ++j) part = fmaf(dz[j], z[j], part);
+  const float Dr = warp_sum(part);                                                // <dZ, Z> = rowsum(dA o A)
+#pragma unroll
+  for (int j = 0; j < DC; ++j) {
+    const int col = lane + 32 * j;
+    if (col < d) {
+      dzr[col] = dz[j];
+      if (live) ws_dZ[grow * d + col] = dz[j];
+    }
+  }
+  if (live && lane == 0) { ws_LD[grow * 2] = L; ws_LD[grow * 2 + 1] = Dr; }
+
+  // ---- second sweep: dS, dQ ----
+  float dq[DC];
+#pragma unroll
+  for (int j = 0; j < DC; ++j) dq[j] = 0.f;
+  for (int64_t r0 = 0; r0 < m; r0 += 32) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < 32 * d2; i += kRowWarps * 32) {
+      const int rr = i / d2, c = i % d2;
+      kvs[rr * ldk + c] = (r0 + rr < m) ? ldf(kvb, (r0 + rr) * d2 + c) : 0.f;
+    }
+    __syncthreads();
+    const float* kr = kvs + lane * ldk;
+    float s = 0.f, dA = 0.f;
+    for (int c = 0; c < d; ++c) {
+      s = fmaf(q[c], kr[c], s);
+      dA = fmaf(dzr[c], kr[d + c], dA);
+    }
+    const float p = (r0 + lane < m) ? expf(s * scale - L) : 0.f;
+    const float dS = p * (dA - Dr);
+    for (int rr = 0; rr < 32; ++rr) {
+      const float ds = __shfl_sync(0xffffffffu, dS, rr);
+      const float* krr = kvs + rr * ldk;
+#pragma unroll
+      for (int j = 0; j < DC; ++j) {
+        const int col = lane + 32 * j;
+        if (col < d) dq[j] = fmaf(ds, krr[col], dq[j]);
+      }
+    }
+  }
+  if (live) {
+#pragma unroll
+    for (int j = 0; j < DC; ++j) {
+      const int col = lane + 32 * j;
+      if (col < d) stf(dQ, grow * d + col, dq[j] * scale);
+    }
+  }
+}
+
+template <typename T, int DC>
+__global__ void __launch_bounds__(kColWarps * 32) bwd_cols_kernel(
+    float* __restrict__ ws_dKV, const T* __restrict__ Q, const T* __restrict__ kv, const float* __restrict__ ws_dZ,
+    const float* __restrict__ ws_LD, int64_t nq, int64_t m, int d, float scale) {
+  extern __shared__ float smem[];
+  float* qt = smem;                                // [kColRows][d]
+  float* dzt = qt + kColRows * d;                  // [kColRows][d]
+  float* ldt = dzt + kColRows * d;                 // [kColRows][2]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y;
+  const int64_t r = (int64_t)blockIdx.x * kColWarps + warp;
+  const bool live = r < m;
+  const T* kvr = kv + ((int64_t)bh * m + (live ? r : 0)) * 2 * d;
+  float kr[DC], vr[DC], ak[DC], av[DC];
+#pragma unroll
+  for (int j = 0; j < DC; ++j) {
+    const int col = lane + 32 * j;
+    kr[j] = (col < d) ? ldf(kvr, col) : 0.f;
+    vr[j] = (col < d) ? ldf(kvr, d + col) : 0.f;
+    ak[j] = av[j] = 0.f;
+  }
+  for (int64_t i0 = 0; i0 < nq; i0 += kColRows) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < kColRows * d; i += kColWarps * 32) {
+      const int ii = i / d, c = i % d;
+      const bool ok = i0 + ii < nq;
+      const int64_t gi = (int64_t)bh * nq + i0 + ii;
+      qt[i] = ok ? ldf(Q, gi * d + c) : 0.f;
+      dzt[i] = ok ? ws_dZ[gi * d + c] : 0.f;
+    }
+    if (threadIdx.x < kColRows * 2) {
+      const int ii = threadIdx.x >> 1;
+      ldt[threadIdx.x] = (i0 + ii < nq) ? ws_LD[((int64_t)bh * nq + i0 + ii) * 2 + (threadIdx.x & 1)] : 0.f;
+    }
+    __syncthreads();
+    const int cnt = (int)((nq - i0 < kColRows) ? nq - i0 : kColRows);
+    for (int ii = 0; ii < cnt; ++ii) {
+      float s = 0.f, dA = 0.f;
+#pragma unroll
+      for (int j = 0; j < DC; ++j) {
+        const int col = lane + 32 * j;
+        if (col < d) {
+          s = fmaf(qt[ii * d + col], kr[j], s);
+          dA = fmaf(dzt[ii * d + col], vr[j], dA);
+        }
+      }
+      s = warp_sum(s);
+      dA = warp_sum(dA);
+      const float p = expf(s * scale - ldt[2 * ii]);
+      const float dS = p * (dA - ldt[2 * ii + 1]);
+#pragma unroll
+      for (int j = 0; j < DC; ++j) {
+        const int col = lane + 32 * j;
+        if (col < d) {
+          ak[j] = fmaf(dS, qt[ii * d + col], ak[j]);
+          av[j] = fmaf(p, dzt[ii * d + col], av[j]);
+        }
+      }
+    }
+  }
+  if (live) {
+    float* o = ws_dKV + ((int64_t)bh * m + r) * 2 * d;
+#pragma unroll
+    for (int j = 0; j < DC; ++j) {
+      const int col = lane + 32 * j;
+      if (col < d) { o[col] = ak[j] * scale; o[d + col] = av[j]; }
+    }
+  }
+}
+
+// dK[j][c] = sum_r Phi_K[r][j] dK~[r][c],  dV[j][c] = sum_r Phi_V[r][j] dV~[r][c]; one block per token j,
+// thread = column of K|V
+template <typename T>
+__global__ void bwd_phiT_kernel(T* __restrict__ dK, T* __restrict__ dV, const T* __restrict__ phi,
+                                const float* __restrict__ ws_dKV, int64_t n, int64_t n_pad, int64_t m, int d, int H,
+                                int phi_v_head0) {
+  const int64_t j = blockIdx.x;
+  const int bh = blockIdx.y, h = bh % H;
+  const int c2 = threadIdx.x;
+  if (c2 >= 2 * d) return;
+  const bool is_v = c2 >= d;
+  const T* ph = phi + (int64_t)((is_v ? phi_v_head0 : 0) + h) * m * n_pad + j;
+  const float* g = ws_dKV + (int64_t)bh * m * 2 * d + c2;
+  float acc = 0.f;
+  for (int64_t r = 0; r < m; ++r) acc = fmaf(ldf(ph, r * n_pad), g[r * 2 * d], acc);
+  if (is_v) stf(dV, ((int64_t)bh * n + j) * d + (c2 - d), acc);
+  else stf(dK, ((int64_t)bh * n + j) * d + c2, acc);
+}
+
+template <typename T>
+cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, void* dV, cudaStream_t s, int* launches) {
+  const Params& p = c->p;
+  const int d = (int)p.d, dc = (d + 31) / 32;
+  const float scale = (float)(p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)d));
+  const unsigned BH = (unsigned)(p.B * p.H);
+  const float* Sd = c->w_untied ? c->Sl_dec : c->S_dec;
+  const float* Bd = c->w_untied ? c->Bl_dec : c->B_dec;
+  const int64_t lstride = c->w_untied ? (int64_t)(p.H * p.d * p.d) : 0;
+  cudaError_t e = cudaSuccess;
+  {
+    const dim3 grid((unsigned)((p.nq + kRowWarps - 1) / kRowWarps), BH);
+    const size_t sm = (size_t)(32 * (2 * d + 1) + 2 * kRowWarps * d) * sizeof(float);
+#define CSAT_BWD_ROWS(DC)                                                                                            \
+  do {                                                                                                               \
+    if (sm > 48 * 1024)                                                                                              \
+      e = cudaFuncSetAttribute(bwd_rows_kernel<T, DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);        \
+    if (e == cudaSuccess)                                                                                            \
+      bwd_rows_kernel<T, DC><<<grid, kRowWarps * 32, sm, s>>>(                                                       \
+          (T*)dQ, c->bw_dZ, c->bw_LD, (const T*)Q, (const T*)G, (const T*)c->kv, Sd, Bd, lstride, c->thr(),          \
+          c->thr_stride(), c->psi ? c->psi_f32 : nullptr, p.nq, p.m, d, (int)p.H, p.T, scale);                       \
+  } while (0)
+    if (dc <= 2) CSAT_BWD_ROWS(2);
+    else if (dc <= 4) CSAT_BWD_ROWS(4);
+    else CSAT_BWD_ROWS(8);
+#undef CSAT_BWD_ROWS
+    if (e != cudaSuccess) return e;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  {
+    const dim3 grid((unsigned)((p.m + kColWarps - 1) / kColWarps), BH);
+    const size_t sm = (size_t)(2 * kColRows * d + 2 * kColRows) * sizeof(float);
+#define CSAT_BWD_COLS(DC)                                                                                            \
+  bwd_cols_kernel<T, DC><<<grid, kColWarps * 32, sm, s>>>(c->bw_dKV, (const T*)Q, (const T*)c->kv, c->bw_dZ, c->bw_LD, \
+                                                         p.nq, p.m, d, scale)
+    if (dc <= 2) CSAT_BWD_COLS(2);
+    else if (dc <= 4) CSAT_BWD_COLS(4);
+    else CSAT_BWD_COLS(8);
+#undef CSAT_BWD_COLS
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  {
+    const dim3 grid((unsigned)p.n, BH);
+    const int threads = ((2 * d + 31) / 32) * 32;
+    bwd_phiT_kernel<T><<<grid, threads, 0, s>>>((T*)dK, (T*)dV, (const T*)c->phi, c->bw_dKV, p.n, p.n_pad, p.m, d,
+                                                (int)p.H, p.separate_phi ? (int)p.H : 0);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  *launches += 3;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+// K~|V~ must already be in the workspace (the forward's compression of the same K, V)
+cudaError_t launch_backward(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, void* dV, cudaStream_t s,
+                            int* launches) {
+  return c->p.dtype == CSAT_DTYPE_FP32 ? run<float>(c, Q, G, dQ, dK, dV, s, launches)
+                                       : run<__nv_bfloat16>(c, Q, G, dQ, dK, dV, s, launches);
+}
+
+}  // namespace csat

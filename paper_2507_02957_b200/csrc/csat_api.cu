@@ -66,6 +66,13 @@ void free_lista(csat_ctx* c) {
   c->w_untied = false;
 }
 
+void free_backward(csat_ctx* c) {
+  dev_free(c, &c->bw_dZ, c->bw_bytes_dZ);
+  dev_free(c, &c->bw_LD, c->bw_bytes_LD);
+  dev_free(c, &c->bw_dKV, c->bw_bytes_dKV);
+  c->bw_bytes_dZ = c->bw_bytes_LD = c->bw_bytes_dKV = 0;
+}
+
 void free_staging(csat_ctx* c) {
   dev_free(c, &c->stage_q, c->stage_bytes_q);
   dev_free(c, &c->stage_o, c->stage_bytes_q);
@@ -90,6 +97,7 @@ void free_all(csat_ctx* c) {
   dev_free(c, &c->mats_bf16, 3 * dd_bytes(p, 2));
   free_lista(c);
   free_staging(c);
+  free_backward(c);
   prof_destroy(c);
   if (c->pipe_ready) {
     for (int i = 0; i < 3; ++i) cudaStreamDestroy(c->pipe_stream[i]);
@@ -518,6 +526,51 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   if (e != cudaSuccess) return fail_cuda(c, e, "attend/recover launch");
   prof_mark(c, s, CSAT_KERNEL_ATTEND_RECOVER);
   if (c->prof_slots) ++c->prof_calls;
+  c->have_forward = true;
+  c->last_launches = launches;
+  return CSAT_OK;
+}
+
+int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, const void* dOut, void* dQ, void* dK,
+                  void* dV, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !dOut || !dQ || !dK || !dV) return fail(c, CSAT_ERR_INVALID_ARG, "csat_backward: NULL pointer");
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dOut) || !aligned16(dQ) || !aligned16(dK) ||
+      !aligned16(dV))
+    return fail(c, CSAT_ERR_INVALID_ARG, "csat_backward: pointers must be 16-byte aligned");
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  if (*(volatile int*)c->status != 0)
+    return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
+  const csat::Params& p = c->p;
+  if (p.T > 32) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward keeps one mask bit per layer: CSAT_T <= 32");
+  if (p.d > 256) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: d <= 256");
+  if (p.T > 0 && c->w_S && (c->w_layers != 1 || c->w_untied) && c->w_layers != p.T)
+    return fail(c, CSAT_ERR_STATE, "the supplied LISTA weights are for a number of layers other than CSAT_T");
+  cudaStream_t s = (cudaStream_t)stream;
+  int launches = 0;
+  if (p.T > 0) {
+    int rc = ensure_decoder(c, s, &launches);
+    if (rc != CSAT_OK) return rc;
+  }
+  const size_t bz = (size_t)(p.B * p.H * p.nq * p.d) * 4, bl = (size_t)(p.B * p.H * p.nq * 2) * 4,
+               bk = (size_t)(p.B * p.H * p.m * 2 * p.d) * 4;
+  if (c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk) {
+    cudaDeviceSynchronize();
+    free_backward(c);
+    c->bw_bytes_dZ = bz; c->bw_bytes_LD = bl; c->bw_bytes_dKV = bk;
+    if (dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
+        dev_alloc(c, &c->bw_dKV, bk) != cudaSuccess) {
+      free_backward(c);
+      return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(backward scratch) failed");
+    }
+  }
+  const bool tc_compress = c->tmap_phi_valid && c->force_simt != 1;
+  cudaError_t e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches)
+                              : csat::launch_simt_compress(c, K, V, s, &launches);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward: compress launch");
+  e = csat::launch_backward(c, Q, dOut, dQ, dK, dV, s, &launches);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward launch");
   c->have_forward = true;
   c->last_launches = launches;
   return CSAT_OK;

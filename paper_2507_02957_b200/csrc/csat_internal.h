@@ -70,6 +70,10 @@ struct csat_ctx {
   size_t w_mat_count() const { return (size_t)(w_untied ? w_layers : 1) * (size_t)(p.H * p.d * p.d); }
   float* mu = nullptr;        // [H]
   int* status = nullptr;      // device status word (0 = ok)
+  // float32 scratch of csat_backward, allocated by its first call: dZ [B,H,n_q,d], (L, D) [B,H,n_q,2],
+  // dK~|dV~ [B,H,m,2d]
+  float* bw_dZ = nullptr; float* bw_LD = nullptr; float* bw_dKV = nullptr;
+  size_t bw_bytes_dZ = 0, bw_bytes_LD = 0, bw_bytes_dKV = 0;
   // staging for csat_forward_host
   void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
   size_t stage_bytes_q = 0, stage_bytes_kv = 0;
@@ -132,6 +136,10 @@ cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, c
 // X [B, n_tok, dm] and writes the heads of Q / K / V those columns belong to
 cudaError_t launch_project(csat_ctx* c, const void* X, const void* W, int64_t n_tok, int64_t dm, int col0, int ncols,
                            void* Q, void* K, void* V, cudaStream_t s, int* launches);
+
+// backward_simt.cu : gradients with respect to Q, K, V; K~|V~ of the same K, V must be in the workspace
+cudaError_t launch_backward(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, void* dV, cudaStream_t s,
+                            int* launches);
 
 // copies K~ or V~ out of the interleaved workspace: dst [B,H,m,d]
 cudaError_t launch_split_kv(const csat_ctx* c, void* kt, void* vt, cudaStream_t s);

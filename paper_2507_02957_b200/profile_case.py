@@ -4,6 +4,7 @@
     python -m paper_2507_02957_b200.profile_case workload c1|c2|c3|c4|c5 [--iters I]
     python -m paper_2507_02957_b200.profile_case ensembles N M D H        (regenerates Phi with every ensemble)
     python -m paper_2507_02957_b200.profile_case project N D B H DMODEL [--iters I]   (the Q, K, V projections)
+    python -m paper_2507_02957_b200.profile_case backward c1|c2|c3|c4|c5 [--iters I]   (csat_backward on a workload)
 
 A small driver to put under a profiler (ncu -k regex:<kernel> ...): 3 warm-up forwards, then I timed ones.
 Inputs are seeded random tensors (N(0, 1/d) for `forward`, the workload's own recipe for `workload`).
@@ -56,6 +57,9 @@ def main():
     for name in ("n", "d", "B", "H", "dm"):
         pj.add_argument(name, type=int)
     pj.add_argument("--iters", type=int, default=10)
+    bw = sub.add_parser("backward")
+    bw.add_argument("name")
+    bw.add_argument("--iters", type=int, default=3)
     a = ap.parse_args()
 
     if a.cmd == "forward":
@@ -84,6 +88,28 @@ def main():
         if inp["Psi"] is not None:
             ctx.set_dictionary(torch.from_numpy(inp["Psi"]).cuda().to(dt))
         print(w.name, _timed_forwards(ctx, Q, K, V, a.iters))
+        ctx.close()
+    elif a.cmd == "backward":
+        w = wl.CONFIGS[a.name]
+        inp = wl.make_inputs(w)
+        dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        Q, K, V = (torch.from_numpy(inp[k]).cuda().to(dt) for k in "QKV")
+        ctx = binding.Csat(w.n, w.m, w.d, w.H, w.phi_seed, B=w.B, n_q=w.n_q, dtype=w.dtype, T=w.T, lam=w.lam)
+        if inp["Psi"] is not None:
+            ctx.set_dictionary(torch.from_numpy(inp["Psi"]).cuda().to(dt))
+        G = torch.randn_like(Q)
+        dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
+        binding.csat_backward(ctx.h, Q, K, V, G, dQ, dK, dV)
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(a.iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            binding.csat_backward(ctx.h, Q, K, V, G, dQ, dK, dV)
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+        print(w.name, {"backward_ms": round(float(np.median(times)), 4)})
         ctx.close()
     elif a.cmd == "project":
         g = torch.Generator(device="cuda")

@@ -1,0 +1,107 @@
+"""GPU parity of csat_backward (gradients with respect to Q, K, V) against the float64 oracle.
+
+The derivative of the shrinkage is discontinuous at |x| = theta, so a row whose iterates come within rounding
+distance of a threshold may take the other branch on the GPU.  The oracle reports each row's smallest distance to
+a kink, and the output gradient of the rows closer than 5e-5 theta is set to zero on both sides (they then
+contribute to no gradient).  With bf16 storage the library keeps K~|V~ in bf16, and its shrinkage decisions follow
+the rounded values: the oracle is given the same rounding for its own K~, V~ (kv_round); the few masks that still
+differ (float32 against float64 accumulation under the rounding) change single terms, so there the comparison is
+the relative Frobenius error of each gradient."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import csat_oracle as orc
+from paper_2507_02957_b200 import binding, workloads as wl
+from gpu_util import device_inputs, make_ctx, rel_err, to_dev, to_np
+
+pytestmark = pytest.mark.gpu
+C = wl.CONFIGS
+
+
+def fro_err(got, ref):
+    return float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
+
+
+CASES = {
+    "c1_fp32": lambda: C["c1"],
+    "fp32_T0": lambda: wl.shrink(C["c1"], n=96, n_q=40, m=32, T=0),
+    "fp32_cross_d32": lambda: wl.shrink(C["c1"], B=2, H=2, n=100, n_q=37, m=40, d=32, T=6),
+    "bf16_d64": lambda: wl.shrink(C["c2"], B=2, H=3, n_q=150),
+    "bf16_d128": lambda: wl.shrink(C["c5"], B=1, H=2, n=512, n_q=200, m=160, T=8, lam=0.002),
+}
+
+
+@pytest.mark.parametrize("name", sorted(CASES))
+@pytest.mark.parametrize("variant", ["default", "psi_separate_untied"])
+def test_backward_matches_oracle(name, variant):
+    w = CASES[name]()
+    if variant != "default" and (w.T == 0 or name == "bf16_d128"):
+        pytest.skip("one variant is enough here")
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    r = np.random.default_rng(97)
+    d, H, T = w.d, w.H, w.T
+    kw = dict(T=T, lam=w.lam)
+    if variant == "psi_separate_untied":
+        Psi = wl.round_to_storage((np.eye(d) + 0.3 * r.standard_normal((d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        ctx.set_dictionary(to_dev(Psi, w.dtype))
+        ctx.set(separate_phi=True)
+        S = wl.round_to_storage((0.6 * np.eye(d) + 0.4 * r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        Bm = wl.round_to_storage((r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        st0 = []
+        orc.csat_forward(inp["Q"][:1], inp["K"][:1], inp["V"][:1], to_np(ctx.get_phi())[:H], T=0, lam=0.0, stages=st0)
+        th0 = float(np.median(np.abs(st0[0]["Z"] @ Bm[0, 0].astype(np.float64))))
+        thetas = (th0 * r.uniform(0.2, 1.5, size=(T, H))).astype(np.float32)
+        ctx.set_lista_layer_weights(to_dev(S, w.dtype), to_dev(Bm, w.dtype), torch.from_numpy(thetas).cuda())
+        kw.update(Psi=Psi.astype(np.float64), weights=(S.astype(np.float64), Bm.astype(np.float64), list(thetas.astype(np.float64))))
+    phi = to_np(ctx.get_phi())
+    if variant == "psi_separate_untied":
+        kw.update(Phi_V=phi[H:])
+        phi = phi[:H]
+    G = wl.round_to_storage(r.standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    if w.dtype == "bf16":
+        kw.update(kv_round=lambda x: wl.round_to_storage(x.astype(np.float32), "bf16"))
+    if T > 0:
+        # rows that come within 5e-5 theta of a kink of eta: no output gradient on either side
+        stages = []
+        orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, stages=stages, **kw)
+        margins = np.stack([s["min_margin"] for s in stages]).reshape(G.shape[:3])
+        th_ref = max(float(np.max(kw["weights"][2])) if "weights" in kw else 0.0, 1e-12)
+        if "weights" not in kw:
+            st1 = []
+            orc.csat_forward(inp["Q"][:1], inp["K"][:1], inp["V"][:1], phi, T=1, lam=w.lam, stages=st1)
+            th_ref = max(s["theta"] for s in st1)
+        near = margins < 5e-5 * th_ref
+        assert near.mean() < 0.2
+        G = G * (~near)[..., None]
+    ref = orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, **kw)
+    got = ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    assert binding.csat_last_launch_count(ctx.h) >= 4
+    for nm, g, rf in zip(("dQ", "dK", "dV"), got, ref):
+        g = to_np(g)
+        assert np.isfinite(g).all()
+        assert np.abs(rf).max() > 0
+        if w.dtype == "fp32":
+            err = rel_err(g, rf)
+            assert err <= 2e-5, (name, variant, nm, err)            # measured ~1e-6
+        else:
+            err = fro_err(g, rf)
+            assert err <= 6e-3, (name, variant, nm, err)            # measured ~2e-3: the bf16 rounding of the outputs
+    # deterministic (no atomics)
+    again = ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    for a, b in zip(got, again):
+        assert torch.equal(a, b)
+    ctx.close()
+
+
+def test_backward_refuses_what_it_does_not_cover():
+    ctx = binding.Csat(64, 16, 8, 1, 0, dtype="fp32", T=33)
+    x = torch.zeros(1, 1, 64, 8, device="cuda")
+    with pytest.raises(binding.CsatError) as ei:
+        ctx.backward(x, x, x, x)
+    assert ei.value.code == 5
+    ctx.set(T=2)
+    ctx.backward(x, x, x, x)                     # the context stays usable
+    ctx.close()
