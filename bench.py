@@ -287,6 +287,28 @@ def time_projection(w: wl.Workload, iters: int = 10, warmup: int = 3) -> dict:
     return {"ms": ms, "tflops": f / (ms * 1e-3) / 1e12, "gflop": f / 1e9, "d_model": dm}
 
 
+def time_backward(w: wl.Workload, iters: int = 2) -> dict:
+    """csat_backward (gradients with respect to Q, K, V; first version on FFMA kernels) on a workload."""
+    import torch
+    from paper_2507_02957_b200 import binding
+    host, dev, psi = device_tensors(w)
+    ctx = make_ctx(w, psi)
+    G = torch.randn_like(dev["Q"])
+    dQ, dK, dV = torch.empty_like(dev["Q"]), torch.empty_like(dev["K"]), torch.empty_like(dev["V"])
+    binding.csat_backward(ctx.h, dev["Q"], dev["K"], dev["V"], G, dQ, dK, dV)
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(iters):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        binding.csat_backward(ctx.h, dev["Q"], dev["K"], dev["V"], G, dQ, dK, dV)
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1))
+    ctx.close()
+    return {"ms": float(np.median(times)), "kernels": "ffma, float32 arithmetic"}
+
+
 def run_csat(args, w: wl.Workload) -> dict:
     import torch
     import torch.distributed as dist
@@ -398,6 +420,7 @@ def run_csat(args, w: wl.Workload) -> dict:
                 extra[f"{w.name}_untied_layers"] = time_small(w, untied=True)
             if w.dtype == "bf16" and w.n == w.n_q:
                 extra[f"{w.name}_qkv_projection"] = time_projection(w)
+            extra["backward"] = {wl.CONFIGS[k].name: time_backward(wl.CONFIGS[k]) for k in ("c1", "c2", "c3", "c4")}
             result["other_workloads"] = extra
         if not args.no_cpu_baseline:
             inp = {k: host[k].float().numpy() for k in "QKV"}

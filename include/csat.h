@@ -173,8 +173,8 @@ int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, c
  *   dOut [B,H,n_q,d]                gradient of the loss with respect to csat_forward's output
  *   dQ [B,H,n_q,d], dK, dV [B,H,n,d]  outputs (context dtype)
  * Nothing of an earlier csat_forward is reused: the call compresses K, V again and recomputes what it needs in
- * float32.  Its first call allocates float32 scratch (B H (n_q (d + 2) + 2 m d) floats, counted by
- * csat_workspace_bytes).  CSAT_T <= 32 and d <= 256, else CSAT_ERR_UNSUPPORTED.  This first version runs on plain
+ * float32.  Its first call allocates float32 scratch (B H (n_q (d + 2) + 2 m d) floats and transposed
+ * copies of the decoder matrices, counted by csat_workspace_bytes).  CSAT_T <= 32 and d <= 256, else CSAT_ERR_UNSUPPORTED.  This first version runs on plain
  * FFMA kernels for both storage types. */
 int csat_backward(csat_ctx* ctx, const void* Q, const void* K, const void* V, const void* dOut, void* dQ, void* dK,
                   void* dV, void* stream);

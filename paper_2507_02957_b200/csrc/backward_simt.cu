@@ -6,9 +6,12 @@
 //
 // First CUDA version: plain FFMA kernels, float32 arithmetic, nothing stored by the forward.  After the
 // compression (the forward's own kernel) three kernels run:
+//   transpose_kernel: float32 transposes of the decoder matrices S_t, B_t, so that every product below reads its
+//                     matrix row by row (coalesced).
 //   bwd_rows_kernel : one warp per query row.  Recomputes the row's scores, softmax statistics and Z, runs the
 //                     recurrence forward keeping one bit per layer and column (|x_t| > theta_t), then backward:
-//                     d alpha_T = G Psi, dx_t = d alpha_{t+1} o mask_t, dZ += dx_t B_t^T, d alpha_t = dx_t S_t^T.
+//                     d alpha_T = G Psi, dx_t = d alpha_{t+1} o mask_t, dZ += dx_t B_t^T, d alpha_t = dx_t S_t^T
+//                     (with one B for all layers dZ = (sum_t dx_t) B^T is a single product at the end).
 //                     Stores dZ, L = log sum exp of the row's scores and D = <dZ, Z>, then sweeps K~|V~ again:
 //                     p = exp(s - L), dS = p (dZ . V~_r - D), dQ = scale sum_r dS_r K~_r.
 //   bwd_cols_kernel : one warp per measurement r, all query rows in turn (deterministic, no atomics):
@@ -63,31 +66,21 @@ __device__ __forceinline__ void row_times(const float (&x)[DC], float (&y)[DC], 
       }
     }
 }
-// y[k] = sum_c x[c] W[k][c]   (x times the transpose of W)
-template <int DC>
-__device__ __forceinline__ void row_times_T(const float (&x)[DC], float (&y)[DC], const float* __restrict__ W, int d, int lane) {
-#pragma unroll
-  for (int j = 0; j < DC; ++j) y[j] = 0.f;
-#pragma unroll
-  for (int jc = 0; jc < DC; ++jc)
-    for (int l = 0; l < 32; ++l) {
-      const int c = 32 * jc + l;
-      const float xc = __shfl_sync(0xffffffffu, x[jc], l);
-      if (c < d) {
-#pragma unroll
-        for (int j = 0; j < DC; ++j) {
-          const int k = lane + 32 * j;
-          if (k < d) y[j] = fmaf(xc, W[(int64_t)k * d + c], y[j]);
-        }
-      }
-    }
+// out[mat][a][b] = in[mat][b][a] for every d x d matrix
+__global__ void transpose_kernel(float* __restrict__ out, const float* __restrict__ in, int d, int64_t mats) {
+  const int64_t total = mats * d * d;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t mat = i / (d * d);
+    const int a = (int)((i / d) % d), b = (int)(i % d);
+    out[i] = in[mat * d * d + (int64_t)b * d + a];
+  }
 }
 
 template <typename T, int DC>   // DC = ceil(d / 32)
 __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
     T* __restrict__ dQ, float* __restrict__ ws_dZ, float* __restrict__ ws_LD, const T* __restrict__ Q,
     const T* __restrict__ G, const T* __restrict__ kv, const float* __restrict__ S_dec, const float* __restrict__ B_dec,
-    int64_t layer_stride, const float* __restrict__ theta, int theta_stride, const float* __restrict__ psi_f32,
+    const float* __restrict__ S_decT, const float* __restrict__ B_decT, int64_t layer_stride, const float* __restrict__ theta, int theta_stride, const float* __restrict__ psi_f32,
     int64_t nq, int64_t m, int d, int H, int T_iters, float scale) {
   extern __shared__ float smem[];
   const int d2 = 2 * d, ldk = d2 + 1;
@@ -155,6 +148,8 @@ __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
   } else {
     const float* Sh = S_dec + (int64_t)h * d * d;
     const float* Bh = B_dec + (int64_t)h * d * d;
+    const float* ShT = S_decT + (int64_t)h * d * d;             // transposes: x W^T = row_times(x, W^T)
+    const float* BhT = B_decT + (int64_t)h * d * d;
     uint32_t mask[DC];
     float a[DC], c[DC], t[DC];
 #pragma unroll
@@ -181,10 +176,20 @@ __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
     for (int it = T_iters - 1; it >= 0; --it) {
 #pragma unroll
       for (int j = 0; j < DC; ++j) dx[j] = ((mask[j] >> it) & 1u) ? da[j] : 0.f;
-      row_times_T<DC>(dx, t, Bh + layer_stride * it, d, lane);                    // dZ += dx B_t^T
+      if (layer_stride != 0) {
+        row_times<DC>(dx, t, BhT + layer_stride * it, d, lane);                   // dZ += dx B_t^T
 #pragma unroll
-      for (int j = 0; j < DC; ++j) dz[j] += t[j];
-      if (it > 0) row_times_T<DC>(dx, da, Sh + layer_stride * it, d, lane);       // d alpha_t = dx S_t^T
+        for (int j = 0; j < DC; ++j) dz[j] += t[j];
+      } else {
+#pragma unroll
+        for (int j = 0; j < DC; ++j) dz[j] += dx[j];                              // one B: sum the dx first
+      }
+      if (it > 0) row_times<DC>(dx, da, ShT + layer_stride * it, d, lane);        // d alpha_t = dx S_t^T
+    }
+    if (layer_stride == 0) {
+#pragma unroll
+      for (int j = 0; j < DC; ++j) dx[j] = dz[j];
+      row_times<DC>(dx, dz, BhT, d, lane);                                        // dZ = (sum_t dx_t) B^T
     }
   }
   float part = 0.f;
@@ -338,6 +343,17 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   const float* Bd = c->w_untied ? c->Bl_dec : c->B_dec;
   const int64_t lstride = c->w_untied ? (int64_t)(p.H * p.d * p.d) : 0;
   cudaError_t e = cudaSuccess;
+  const int64_t mats = (c->w_untied ? c->w_layers : 1) * p.H;
+  float* SdT = c->bw_WT;
+  float* BdT = c->bw_WT + mats * d * d;
+  if (p.T > 0) {
+    const int64_t total = mats * d * d;
+    const unsigned tg = (unsigned)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+    transpose_kernel<<<tg, 256, 0, s>>>(SdT, Sd, d, mats);
+    transpose_kernel<<<tg, 256, 0, s>>>(BdT, Bd, d, mats);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    *launches += 2;
+  }
   {
     const dim3 grid((unsigned)((p.nq + kRowWarps - 1) / kRowWarps), BH);
     const size_t sm = (size_t)(32 * (2 * d + 1) + 2 * kRowWarps * d) * sizeof(float);
@@ -347,7 +363,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
       e = cudaFuncSetAttribute(bwd_rows_kernel<T, DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);        \
     if (e == cudaSuccess)                                                                                            \
       bwd_rows_kernel<T, DC><<<grid, kRowWarps * 32, sm, s>>>(                                                       \
-          (T*)dQ, c->bw_dZ, c->bw_LD, (const T*)Q, (const T*)G, (const T*)c->kv, Sd, Bd, lstride, c->thr(),          \
+          (T*)dQ, c->bw_dZ, c->bw_LD, (const T*)Q, (const T*)G, (const T*)c->kv, Sd, Bd, SdT, BdT, lstride, c->thr(), \
           c->thr_stride(), c->psi ? c->psi_f32 : nullptr, p.nq, p.m, d, (int)p.H, p.T, scale);                       \
   } while (0)
     if (dc <= 2) CSAT_BWD_ROWS(2);

@@ -72,8 +72,9 @@ struct csat_ctx {
   int* status = nullptr;      // device status word (0 = ok)
   // float32 scratch of csat_backward, allocated by its first call: dZ [B,H,n_q,d], (L, D) [B,H,n_q,2],
   // dK~|dV~ [B,H,m,2d]
-  float* bw_dZ = nullptr; float* bw_LD = nullptr; float* bw_dKV = nullptr;
-  size_t bw_bytes_dZ = 0, bw_bytes_LD = 0, bw_bytes_dKV = 0;
+  // and the float32 transposes of the decoder matrices [2][layers or 1][H][d][d]
+  float* bw_dZ = nullptr; float* bw_LD = nullptr; float* bw_dKV = nullptr; float* bw_WT = nullptr;
+  size_t bw_bytes_dZ = 0, bw_bytes_LD = 0, bw_bytes_dKV = 0, bw_bytes_WT = 0;
   // staging for csat_forward_host
   void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
   size_t stage_bytes_q = 0, stage_bytes_kv = 0;
