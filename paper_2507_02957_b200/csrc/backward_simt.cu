@@ -314,23 +314,58 @@ __global__ void __launch_bounds__(kColWarps * 32) bwd_cols_kernel(
   }
 }
 
-// dK[j][c] = sum_r Phi_K[r][j] dK~[r][c],  dV[j][c] = sum_r Phi_V[r][j] dV~[r][c]; one block per token j,
-// thread = column of K|V
+// dK[j][c] = sum_r Phi_K[r][j] dK~[r][c],  dV[j][c] = sum_r Phi_V[r][j] dV~[r][c].
+// Block = 64 tokens x 32 columns of K (blockIdx.z even) or V (odd); 256 threads, 4 tokens x 2 columns each;
+// Phi and dK~|dV~ pass through shared memory 32 measurement rows at a time (Phi rows are read along the tokens).
+constexpr int kPtTok = 64, kPtCol = 32, kPtRows = 32;
 template <typename T>
-__global__ void bwd_phiT_kernel(T* __restrict__ dK, T* __restrict__ dV, const T* __restrict__ phi,
-                                const float* __restrict__ ws_dKV, int64_t n, int64_t n_pad, int64_t m, int d, int H,
-                                int phi_v_head0) {
-  const int64_t j = blockIdx.x;
-  const int bh = blockIdx.y, h = bh % H;
-  const int c2 = threadIdx.x;
-  if (c2 >= 2 * d) return;
-  const bool is_v = c2 >= d;
-  const T* ph = phi + (int64_t)((is_v ? phi_v_head0 : 0) + h) * m * n_pad + j;
-  const float* g = ws_dKV + (int64_t)bh * m * 2 * d + c2;
-  float acc = 0.f;
-  for (int64_t r = 0; r < m; ++r) acc = fmaf(ldf(ph, r * n_pad), g[r * 2 * d], acc);
-  if (is_v) stf(dV, ((int64_t)bh * n + j) * d + (c2 - d), acc);
-  else stf(dK, ((int64_t)bh * n + j) * d + c2, acc);
+__global__ void __launch_bounds__(256) bwd_phiT_kernel(T* __restrict__ dK, T* __restrict__ dV, const T* __restrict__ phi,
+                                                       const float* __restrict__ ws_dKV, int64_t n, int64_t n_pad,
+                                                       int64_t m, int d, int H, int phi_v_head0) {
+  __shared__ float ps[kPtRows][kPtTok + 1];
+  __shared__ float gs[kPtRows][kPtCol + 1];
+  const int bh = blockIdx.z >> 1, is_v = blockIdx.z & 1, h = bh % H;
+  const int64_t j0 = (int64_t)blockIdx.x * kPtTok;
+  const int c0 = blockIdx.y * kPtCol;
+  const T* ph = phi + (int64_t)((is_v ? phi_v_head0 : 0) + h) * m * n_pad;
+  const float* g = ws_dKV + (int64_t)bh * m * 2 * d + (is_v ? d : 0);
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;       // columns 2 tx, 2 tx + 1; tokens 4 ty .. 4 ty + 3
+  float acc[4][2];
+#pragma unroll
+  for (int a = 0; a < 4; ++a) acc[a][0] = acc[a][1] = 0.f;
+  for (int64_t r0 = 0; r0 < m; r0 += kPtRows) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < kPtRows * kPtTok; i += 256) {
+      const int rr = i / kPtTok, jj = i % kPtTok;
+      ps[rr][jj] = (r0 + rr < m && j0 + jj < n) ? ldf(ph, (r0 + rr) * n_pad + j0 + jj) : 0.f;
+    }
+    for (int i = threadIdx.x; i < kPtRows * kPtCol; i += 256) {
+      const int rr = i / kPtCol, cc = i % kPtCol;
+      gs[rr][cc] = (r0 + rr < m && c0 + cc < d) ? g[(r0 + rr) * 2 * d + c0 + cc] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int rr = 0; rr < kPtRows; ++rr) {
+      const float g0 = gs[rr][2 * tx], g1 = gs[rr][2 * tx + 1];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const float pv = ps[rr][4 * ty + a];
+        acc[a][0] = fmaf(pv, g0, acc[a][0]);
+        acc[a][1] = fmaf(pv, g1, acc[a][1]);
+      }
+    }
+  }
+  T* dst = is_v ? dV : dK;
+#pragma unroll
+  for (int a = 0; a < 4; ++a) {
+    const int64_t j = j0 + 4 * ty + a;
+    if (j >= n) continue;
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int c = c0 + 2 * tx + u;
+      if (c < d) stf(dst, ((int64_t)bh * n + j) * d + c, acc[a][u]);
+    }
+  }
 }
 
 template <typename T>
@@ -386,9 +421,8 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   {
-    const dim3 grid((unsigned)p.n, BH);
-    const int threads = ((2 * d + 31) / 32) * 32;
-    bwd_phiT_kernel<T><<<grid, threads, 0, s>>>((T*)dK, (T*)dV, (const T*)c->phi, c->bw_dKV, p.n, p.n_pad, p.m, d,
+    const dim3 grid((unsigned)((p.n + kPtTok - 1) / kPtTok), (unsigned)((d + kPtCol - 1) / kPtCol), BH * 2);
+    bwd_phiT_kernel<T><<<grid, 256, 0, s>>>((T*)dK, (T*)dV, (const T*)c->phi, c->bw_dKV, p.n, p.n_pad, p.m, d,
                                                 (int)p.H, p.separate_phi ? (int)p.H : 0);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }

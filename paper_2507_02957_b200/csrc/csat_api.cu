@@ -546,6 +546,7 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   const csat::Params& p = c->p;
   if (p.T > 32) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward keeps one mask bit per layer: CSAT_T <= 32");
   if (p.d > 256) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: d <= 256");
+  if (p.B * p.H > 32767) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: B * H <= 32767");
   if (p.T > 0 && c->w_S && (c->w_layers != 1 || c->w_untied) && c->w_layers != p.T)
     return fail(c, CSAT_ERR_STATE, "the supplied LISTA weights are for a number of layers other than CSAT_T");
   cudaStream_t s = (cudaStream_t)stream;
