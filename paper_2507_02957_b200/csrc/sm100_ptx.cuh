@@ -1,5 +1,5 @@
 // Thin inline-PTX wrappers for the sm_100a features the tensor-core kernels use: mbarrier, TMA
-// (cp.async.bulk.tensor, no multicast anywhere), tcgen05 (TMEM allocation, MMA, commit, load) and the
+// (cp.async.bulk.tensor; every copy lands in the issuing CTA's own shared memory), tcgen05 (TMEM allocation, MMA, commit, load) and the
 // shared-memory / instruction descriptors of tcgen05.mma.
 //
 // Every wait is bounded: it gives up after kWaitTimeoutNs, records where in the status word and returns
