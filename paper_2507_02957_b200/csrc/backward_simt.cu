@@ -16,7 +16,8 @@
 //                     p = exp(s - L), dS = p (dZ . V~_r - D), dQ = scale sum_r dS_r K~_r.
 //   bwd_cols_kernel : one warp per measurement r, all query rows in turn (deterministic, no atomics):
 //                     dK~_r = scale sum_i dS_ir Q_i,  dV~_r = sum_i p_ir dZ_i.
-//   bwd_phiT_kernel : dK = Phi^T dK~, dV = Phi_V^T dV~.
+//   bwd_phiT_kernel : dK = Phi^T dK~, dV = Phi_V^T dV~  (bf16 contexts with d in {64, 128} run this product on the
+//                     tensor cores instead: phiT_sm100.cu, from a bf16 copy of dK~|dV~).
 #include "csat_internal.h"
 
 namespace csat {
@@ -246,8 +247,8 @@ __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
 
 template <typename T, int DC>
 __global__ void __launch_bounds__(kColWarps * 32) bwd_cols_kernel(
-    float* __restrict__ ws_dKV, const T* __restrict__ Q, const T* __restrict__ kv, const float* __restrict__ ws_dZ,
-    const float* __restrict__ ws_LD, int64_t nq, int64_t m, int d, float scale) {
+    float* __restrict__ ws_dKV, __nv_bfloat16* __restrict__ ws_dKV16, const T* __restrict__ Q, const T* __restrict__ kv,
+    const float* __restrict__ ws_dZ, const float* __restrict__ ws_LD, int64_t nq, int64_t m, int d, float scale) {
   extern __shared__ float smem[];
   float* qt = smem;                                // [kColRows][d]
   float* dzt = qt + kColRows * d;                  // [kColRows][d]
@@ -309,7 +310,15 @@ __global__ void __launch_bounds__(kColWarps * 32) bwd_cols_kernel(
 #pragma unroll
     for (int j = 0; j < DC; ++j) {
       const int col = lane + 32 * j;
-      if (col < d) { o[col] = ak[j] * scale; o[d + col] = av[j]; }
+      if (col < d) {
+        o[col] = ak[j] * scale;
+        o[d + col] = av[j];
+        if (ws_dKV16) {                        // operand copy for the tensor-core Phi^T product
+          __nv_bfloat16* o16 = ws_dKV16 + ((int64_t)bh * m + r) * 2 * d;
+          o16[col] = __float2bfloat16_rn(ak[j] * scale);
+          o16[d + col] = __float2bfloat16_rn(av[j]);
+        }
+      }
     }
   }
 }
@@ -378,6 +387,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   const float* Bd = c->w_untied ? c->Bl_dec : c->B_dec;
   const int64_t lstride = c->w_untied ? (int64_t)(p.H * p.d * p.d) : 0;
   cudaError_t e = cudaSuccess;
+  const bool tc_phiT = c->bw_dKV16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
   const int64_t mats = (c->w_untied ? c->w_layers : 1) * p.H;
   float* SdT = c->bw_WT;
   float* BdT = c->bw_WT + mats * d * d;
@@ -412,13 +422,18 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
     const dim3 grid((unsigned)((p.m + kColWarps - 1) / kColWarps), BH);
     const size_t sm = (size_t)(2 * kColRows * d + 2 * kColRows) * sizeof(float);
 #define CSAT_BWD_COLS(DC)                                                                                            \
-  bwd_cols_kernel<T, DC><<<grid, kColWarps * 32, sm, s>>>(c->bw_dKV, (const T*)Q, (const T*)c->kv, c->bw_dZ, c->bw_LD, \
-                                                         p.nq, p.m, d, scale)
+  bwd_cols_kernel<T, DC><<<grid, kColWarps * 32, sm, s>>>(c->bw_dKV, tc_phiT ? c->bw_dKV16 : nullptr, (const T*)Q,  \
+                                                         (const T*)c->kv, c->bw_dZ, c->bw_LD, p.nq, p.m, d, scale)
     if (dc <= 2) CSAT_BWD_COLS(2);
     else if (dc <= 4) CSAT_BWD_COLS(4);
     else CSAT_BWD_COLS(8);
 #undef CSAT_BWD_COLS
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  if (tc_phiT) {
+    if ((e = launch_sm100_phiT(c, c->bw_dKV16, dK, dV, s, launches)) != cudaSuccess) return e;
+    *launches += 2;
+    return cudaSuccess;
   }
   {
     const dim3 grid((unsigned)((p.n + kPtTok - 1) / kPtTok), (unsigned)((d + kPtCol - 1) / kPtCol), BH * 2);
