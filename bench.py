@@ -306,7 +306,8 @@ def time_backward(w: wl.Workload, iters: int = 2) -> dict:
         e1.synchronize()
         times.append(e0.elapsed_time(e1))
     ctx.close()
-    return {"ms": float(np.median(times)), "kernels": "ffma, float32 arithmetic"}
+    return {"ms": float(np.median(times)),
+            "kernels": "per-row stage on ffma kernels (float32); dK~|dV~ and Phi^T on tcgen05 for bf16"}
 
 
 def run_csat(args, w: wl.Workload) -> dict:

@@ -175,8 +175,9 @@ int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, c
  * Nothing of an earlier csat_forward is reused: the call compresses K, V again and recomputes what it needs in
  * float32.  Its first call allocates float32 scratch (B H (n_q (d + 2) + 2 m d) floats and transposed
  * copies of the decoder matrices, counted by csat_workspace_bytes).  CSAT_T <= 32, d <= 256 and B H <= 32767, else CSAT_ERR_UNSUPPORTED.  This first
- * version runs on plain FFMA kernels for both storage types, except the last product (Phi^T times the gradients of
- * K~|V~), which bf16 contexts with d in {64, 128} run on the tensor cores from a bf16 copy of those gradients. */
+ * version recomputes each query row (scores, recurrence, its backward, dQ) on plain FFMA kernels in float32; bf16
+ * contexts with d in {64, 128} then run the gradients of K~|V~ (P^T dZ, dS^T Q) and the product with Phi^T on the
+ * tensor cores with bf16 operands, everything else stays on FFMA kernels. */
 int csat_backward(csat_ctx* ctx, const void* Q, const void* K, const void* V, const void* dOut, void* dQ, void* dK,
                   void* dV, void* stream);
 

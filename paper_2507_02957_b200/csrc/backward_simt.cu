@@ -15,7 +15,8 @@
 //                     Stores dZ, L = log sum exp of the row's scores and D = <dZ, Z>, then sweeps K~|V~ again:
 //                     p = exp(s - L), dS = p (dZ . V~_r - D), dQ = scale sum_r dS_r K~_r.
 //   bwd_cols_kernel : one warp per measurement r, all query rows in turn (deterministic, no atomics):
-//                     dK~_r = scale sum_i dS_ir Q_i,  dV~_r = sum_i p_ir dZ_i.
+//                     dK~_r = scale sum_i dS_ir Q_i,  dV~_r = sum_i p_ir dZ_i  (bf16 contexts with d in {64, 128}
+//                     run this stage on the tensor cores instead: bwd_cols_sm100.cu).
 //   bwd_phiT_kernel : dK = Phi^T dK~, dV = Phi_V^T dV~  (bf16 contexts with d in {64, 128} run this product on the
 //                     tensor cores instead: phiT_sm100.cu, from a bf16 copy of dK~|dV~).
 #include "csat_internal.h"
@@ -79,7 +80,8 @@ __global__ void transpose_kernel(float* __restrict__ out, const float* __restric
 
 template <typename T, int DC>   // DC = ceil(d / 32)
 __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
-    T* __restrict__ dQ, float* __restrict__ ws_dZ, float* __restrict__ ws_LD, const T* __restrict__ Q,
+    T* __restrict__ dQ, float* __restrict__ ws_dZ, __nv_bfloat16* __restrict__ ws_dZ16, float* __restrict__ ws_LD,
+    const T* __restrict__ Q,
     const T* __restrict__ G, const T* __restrict__ kv, const float* __restrict__ S_dec, const float* __restrict__ B_dec,
     const float* __restrict__ S_decT, const float* __restrict__ B_decT, int64_t layer_stride, const float* __restrict__ theta, int theta_stride, const float* __restrict__ psi_f32,
     int64_t nq, int64_t m, int d, int H, int T_iters, float scale) {
@@ -202,7 +204,10 @@ __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
     const int col = lane + 32 * j;
     if (col < d) {
       dzr[col] = dz[j];
-      if (live) ws_dZ[grow * d + col] = dz[j];
+      if (live) {
+        ws_dZ[grow * d + col] = dz[j];
+        if (ws_dZ16) ws_dZ16[grow * d + col] = __float2bfloat16_rn(dz[j]);     // operand of the tensor-core stage
+      }
     }
   }
   if (live && lane == 0) { ws_LD[grow * 2] = L; ws_LD[grow * 2 + 1] = Dr; }
@@ -387,7 +392,8 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   const float* Bd = c->w_untied ? c->Bl_dec : c->B_dec;
   const int64_t lstride = c->w_untied ? (int64_t)(p.H * p.d * p.d) : 0;
   cudaError_t e = cudaSuccess;
-  const bool tc_phiT = c->bw_dKV16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
+  // bf16 with d in {64, 128}: the stages after the per-row kernel run on the tensor cores
+  const bool tc_phiT = c->bw_dKV16 != nullptr && c->bw_dZ16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
   const int64_t mats = (c->w_untied ? c->w_layers : 1) * p.H;
   float* SdT = c->bw_WT;
   float* BdT = c->bw_WT + mats * d * d;
@@ -408,7 +414,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
       e = cudaFuncSetAttribute(bwd_rows_kernel<T, DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);        \
     if (e == cudaSuccess)                                                                                            \
       bwd_rows_kernel<T, DC><<<grid, kRowWarps * 32, sm, s>>>(                                                       \
-          (T*)dQ, c->bw_dZ, c->bw_LD, (const T*)Q, (const T*)G, (const T*)c->kv, Sd, Bd, SdT, BdT, lstride, c->thr(), \
+          (T*)dQ, c->bw_dZ, tc_phiT ? c->bw_dZ16 : nullptr, c->bw_LD, (const T*)Q, (const T*)G, (const T*)c->kv, Sd, Bd, SdT, BdT, lstride, c->thr(), \
           c->thr_stride(), c->psi ? c->psi_f32 : nullptr, p.nq, p.m, d, (int)p.H, p.T, scale);                       \
   } while (0)
     if (dc <= 2) CSAT_BWD_ROWS(2);
@@ -418,22 +424,24 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
     if (e != cudaSuccess) return e;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
+  if (tc_phiT) {
+    // dK~, dV~ and dK, dV on the tensor cores
+    if ((e = launch_sm100_bwd_cols(c, Q, s, launches)) != cudaSuccess) return e;
+    if ((e = launch_sm100_phiT(c, c->bw_dKV16, dK, dV, s, launches)) != cudaSuccess) return e;
+    *launches += 1;
+    return cudaSuccess;
+  }
   {
     const dim3 grid((unsigned)((p.m + kColWarps - 1) / kColWarps), BH);
     const size_t sm = (size_t)(2 * kColRows * d + 2 * kColRows) * sizeof(float);
 #define CSAT_BWD_COLS(DC)                                                                                            \
-  bwd_cols_kernel<T, DC><<<grid, kColWarps * 32, sm, s>>>(c->bw_dKV, tc_phiT ? c->bw_dKV16 : nullptr, (const T*)Q,  \
-                                                         (const T*)c->kv, c->bw_dZ, c->bw_LD, p.nq, p.m, d, scale)
+  bwd_cols_kernel<T, DC><<<grid, kColWarps * 32, sm, s>>>(c->bw_dKV, nullptr, (const T*)Q, (const T*)c->kv, c->bw_dZ,   \
+                                                         c->bw_LD, p.nq, p.m, d, scale)
     if (dc <= 2) CSAT_BWD_COLS(2);
     else if (dc <= 4) CSAT_BWD_COLS(4);
     else CSAT_BWD_COLS(8);
 #undef CSAT_BWD_COLS
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  }
-  if (tc_phiT) {
-    if ((e = launch_sm100_phiT(c, c->bw_dKV16, dK, dV, s, launches)) != cudaSuccess) return e;
-    *launches += 2;
-    return cudaSuccess;
   }
   {
     const dim3 grid((unsigned)((p.n + kPtTok - 1) / kPtTok), (unsigned)((d + kPtCol - 1) / kPtCol), BH * 2);

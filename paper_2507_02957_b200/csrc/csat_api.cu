@@ -72,7 +72,8 @@ void free_backward(csat_ctx* c) {
   dev_free(c, &c->bw_dKV, c->bw_bytes_dKV);
   dev_free(c, &c->bw_WT, c->bw_bytes_WT);
   dev_free(c, &c->bw_dKV16, c->bw_bytes_dKV16);
-  c->bw_bytes_dZ = c->bw_bytes_LD = c->bw_bytes_dKV = c->bw_bytes_WT = c->bw_bytes_dKV16 = 0;
+  dev_free(c, &c->bw_dZ16, c->bw_bytes_dZ16);
+  c->bw_bytes_dZ = c->bw_bytes_LD = c->bw_bytes_dKV = c->bw_bytes_WT = c->bw_bytes_dKV16 = c->bw_bytes_dZ16 = 0;
 }
 
 void free_staging(csat_ctx* c) {
@@ -559,15 +560,16 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   const size_t bz = (size_t)(p.B * p.H * p.nq * p.d) * 4, bl = (size_t)(p.B * p.H * p.nq * 2) * 4,
                bk = (size_t)(p.B * p.H * p.m * 2 * p.d) * 4,
                bw = (size_t)(2 * (c->w_untied ? c->w_layers : 1) * p.H * p.d * p.d) * 4,
-               b16 = c->tmap_phi_valid ? bk / 2 : 0;
+               b16 = c->tmap_phi_valid ? bk / 2 : 0, z16 = c->tmap_phi_valid ? bz / 2 : 0;
   if (c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
-      c->bw_bytes_dKV16 != b16) {
+      c->bw_bytes_dKV16 != b16 || c->bw_bytes_dZ16 != z16) {
     cudaDeviceSynchronize();
     free_backward(c);
     c->bw_bytes_dZ = bz; c->bw_bytes_LD = bl; c->bw_bytes_dKV = bk; c->bw_bytes_WT = bw; c->bw_bytes_dKV16 = b16;
+    c->bw_bytes_dZ16 = z16;
     if (dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
         dev_alloc(c, &c->bw_dKV, bk) != cudaSuccess || dev_alloc(c, &c->bw_WT, bw) != cudaSuccess ||
-        dev_alloc(c, &c->bw_dKV16, b16) != cudaSuccess) {
+        dev_alloc(c, &c->bw_dKV16, b16) != cudaSuccess || dev_alloc(c, &c->bw_dZ16, z16) != cudaSuccess) {
       free_backward(c);
       return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(backward scratch) failed");
     }

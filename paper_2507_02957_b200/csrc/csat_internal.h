@@ -75,7 +75,8 @@ struct csat_ctx {
   // and the float32 transposes of the decoder matrices [2][layers or 1][H][d][d]
   float* bw_dZ = nullptr; float* bw_LD = nullptr; float* bw_dKV = nullptr; float* bw_WT = nullptr;
   __nv_bfloat16* bw_dKV16 = nullptr;     // bf16 copy of dK~|dV~ (operand of the tensor-core Phi^T product)
-  size_t bw_bytes_dZ = 0, bw_bytes_LD = 0, bw_bytes_dKV = 0, bw_bytes_WT = 0, bw_bytes_dKV16 = 0;
+  __nv_bfloat16* bw_dZ16 = nullptr;      // bf16 copy of dZ (operand of the tensor-core dK~|dV~ stage)
+  size_t bw_bytes_dZ = 0, bw_bytes_LD = 0, bw_bytes_dKV = 0, bw_bytes_WT = 0, bw_bytes_dKV16 = 0, bw_bytes_dZ16 = 0;
   // staging for csat_forward_host
   void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
   size_t stage_bytes_q = 0, stage_bytes_kv = 0;
@@ -142,6 +143,10 @@ cudaError_t launch_project(csat_ctx* c, const void* X, const void* W, int64_t n_
 // backward_simt.cu : gradients with respect to Q, K, V; K~|V~ of the same K, V must be in the workspace
 cudaError_t launch_backward(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, void* dV, cudaStream_t s,
                             int* launches);
+
+// bwd_cols_sm100.cu : dK~ = scale dS^T Q, dV~ = P^T dZ on the tensor cores (bf16, d in {64, 128}); reads bw_dZ16,
+// bw_LD and the K~|V~ workspace, writes bw_dKV and bw_dKV16
+cudaError_t launch_sm100_bwd_cols(csat_ctx* c, const void* Q, cudaStream_t s, int* launches);
 
 // phiT_sm100.cu : dK = Phi_K^T dK~, dV = Phi_V^T dV~ on the tensor cores (bf16, d in {64, 128}); g16 = dK~|dV~ as bf16
 cudaError_t launch_sm100_phiT(csat_ctx* c, const void* g16, void* dK, void* dV, cudaStream_t s, int* launches);
