@@ -252,8 +252,8 @@ __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
 
 template <typename T, int DC>
 __global__ void __launch_bounds__(kColWarps * 32) bwd_cols_kernel(
-    float* __restrict__ ws_dKV, __nv_bfloat16* __restrict__ ws_dKV16, const T* __restrict__ Q, const T* __restrict__ kv,
-    const float* __restrict__ ws_dZ, const float* __restrict__ ws_LD, int64_t nq, int64_t m, int d, float scale) {
+    float* __restrict__ ws_dKV, const T* __restrict__ Q, const T* __restrict__ kv, const float* __restrict__ ws_dZ,
+    const float* __restrict__ ws_LD, int64_t nq, int64_t m, int d, float scale) {
   extern __shared__ float smem[];
   float* qt = smem;                                // [kColRows][d]
   float* dzt = qt + kColRows * d;                  // [kColRows][d]
@@ -315,15 +315,7 @@ __global__ void __launch_bounds__(kColWarps * 32) bwd_cols_kernel(
 #pragma unroll
     for (int j = 0; j < DC; ++j) {
       const int col = lane + 32 * j;
-      if (col < d) {
-        o[col] = ak[j] * scale;
-        o[d + col] = av[j];
-        if (ws_dKV16) {                        // operand copy for the tensor-core Phi^T product
-          __nv_bfloat16* o16 = ws_dKV16 + ((int64_t)bh * m + r) * 2 * d;
-          o16[col] = __float2bfloat16_rn(ak[j] * scale);
-          o16[d + col] = __float2bfloat16_rn(av[j]);
-        }
-      }
+      if (col < d) { o[col] = ak[j] * scale; o[d + col] = av[j]; }
     }
   }
 }
@@ -393,7 +385,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   const int64_t lstride = c->w_untied ? (int64_t)(p.H * p.d * p.d) : 0;
   cudaError_t e = cudaSuccess;
   // bf16 with d in {64, 128}: the stages after the per-row kernel run on the tensor cores
-  const bool tc_phiT = c->bw_dKV16 != nullptr && c->bw_dZ16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
+  const bool tc_stages = c->bw_dKV16 != nullptr && c->bw_dZ16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
   const int64_t mats = (c->w_untied ? c->w_layers : 1) * p.H;
   float* SdT = c->bw_WT;
   float* BdT = c->bw_WT + mats * d * d;
@@ -414,7 +406,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
       e = cudaFuncSetAttribute(bwd_rows_kernel<T, DC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);        \
     if (e == cudaSuccess)                                                                                            \
       bwd_rows_kernel<T, DC><<<grid, kRowWarps * 32, sm, s>>>(                                                       \
-          (T*)dQ, c->bw_dZ, tc_phiT ? c->bw_dZ16 : nullptr, c->bw_LD, (const T*)Q, (const T*)G, (const T*)c->kv, Sd, Bd, SdT, BdT, lstride, c->thr(), \
+          (T*)dQ, c->bw_dZ, tc_stages ? c->bw_dZ16 : nullptr, c->bw_LD, (const T*)Q, (const T*)G, (const T*)c->kv, Sd, Bd, SdT, BdT, lstride, c->thr(), \
           c->thr_stride(), c->psi ? c->psi_f32 : nullptr, p.nq, p.m, d, (int)p.H, p.T, scale);                       \
   } while (0)
     if (dc <= 2) CSAT_BWD_ROWS(2);
@@ -424,7 +416,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
     if (e != cudaSuccess) return e;
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
-  if (tc_phiT) {
+  if (tc_stages) {
     // dK~, dV~ and dK, dV on the tensor cores
     if ((e = launch_sm100_bwd_cols(c, Q, s, launches)) != cudaSuccess) return e;
     if ((e = launch_sm100_phiT(c, c->bw_dKV16, dK, dV, s, launches)) != cudaSuccess) return e;
@@ -435,8 +427,8 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
     const dim3 grid((unsigned)((p.m + kColWarps - 1) / kColWarps), BH);
     const size_t sm = (size_t)(2 * kColRows * d + 2 * kColRows) * sizeof(float);
 #define CSAT_BWD_COLS(DC)                                                                                            \
-  bwd_cols_kernel<T, DC><<<grid, kColWarps * 32, sm, s>>>(c->bw_dKV, nullptr, (const T*)Q, (const T*)c->kv, c->bw_dZ,   \
-                                                         c->bw_LD, p.nq, p.m, d, scale)
+  bwd_cols_kernel<T, DC><<<grid, kColWarps * 32, sm, s>>>(c->bw_dKV, (const T*)Q, (const T*)c->kv, c->bw_dZ, c->bw_LD, \
+                                                         p.nq, p.m, d, scale)
     if (dc <= 2) CSAT_BWD_COLS(2);
     else if (dc <= 4) CSAT_BWD_COLS(4);
     else CSAT_BWD_COLS(8);
