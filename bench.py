@@ -217,8 +217,7 @@ def make_ctx(w: wl.Workload, psi):
 
 def kernel_flops(w: wl.Workload) -> dict:
     f = wl.flops(w)
-    return {"compress": f["compress"], "attend_recover": f["attend"] + f["recover"], "decoder_setup": 0,
-            "split_reduce": 0}
+    return {"compress": f["compress"], "attend_recover": f["attend"] + f["recover"], "decoder_setup": 0}
 
 
 def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3, untied: bool = False) -> dict:

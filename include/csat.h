@@ -83,8 +83,7 @@ enum {
 enum {
   CSAT_KERNEL_DECODER_SETUP = 0, /* the three small set-up launches, timed together      */
   CSAT_KERNEL_COMPRESS = 1,      /* K~|V~ = Phi [K|V]                                    */
-  CSAT_KERNEL_ATTEND_RECOVER = 2,/* softmax(Q K~^T) V~, recovery iterations, Psi         */
-  CSAT_KERNEL_SPLIT_REDUCE = 3   /* fixed-order sum of token-axis partial K~|V~ tiles    */
+  CSAT_KERNEL_ATTEND_RECOVER = 2 /* softmax(Q K~^T) V~, recovery iterations, Psi         */
 };
 enum { CSAT_DTYPE_BF16 = 0, CSAT_DTYPE_FP32 = 1 };
 enum { CSAT_ENSEMBLE_GAUSSIAN = 0, CSAT_ENSEMBLE_RADEMACHER = 1, CSAT_ENSEMBLE_HADAMARD = 2 };
@@ -117,7 +116,11 @@ int csat_destroy(csat_ctx* ctx);
 /* Tunables m, t, Phi, Psi of the paper ("Interpretation and Benefits") that are not fixed at
  * creation.  Setters validate and record; dependent decoder quantities (S, B, theta) are
  * re-derived by the next csat_forward on that call's stream.  Must not be called while a
- * forward of the same context is still running on the device. */
+ * forward of the same context is still running on the device.
+ * CSAT_BATCH, CSAT_DTYPE and CSAT_SEPARATE_PHI re-allocate.  If that fails (CSAT_ERR_ALLOC) the context keeps
+ * the new value but holds no usable buffers: csat_forward, csat_forward_host, csat_backward, csat_set_phi and the
+ * getters of device data return CSAT_ERR_STATE until one of those three setters succeeds (setting the same value
+ * again retries the allocation). */
 int csat_set_i64(csat_ctx* ctx, int key, int64_t value);
 int csat_get_i64(const csat_ctx* ctx, int key, int64_t* value_host);
 int csat_set_f64(csat_ctx* ctx, int key, double value);
@@ -198,7 +201,7 @@ int csat_project_qkv(csat_ctx* ctx, const void* Xq, const void* Xkv, const void*
  * csat_forward -- paper: compression, approximate attention matrix, compressed output,
  * LISTA recurrence and reconstruction equations (all of the hot path).
  *   Q   [B, H, n_q, d]   K, V [B, H, n, d]   out [B, H, n_q, d]   device, context dtype.
- * out must not overlap Q, K or V.  Launch-only: no allocation, no synchronisation, no host
+ * out must not overlap Q, K or V (checked on the byte ranges: CSAT_ERR_INVALID_ARG).  Launch-only: no allocation, no synchronisation, no host
  * access to the tensors.  The n_q x m attention matrix and the recovery iterates never reach
  * global memory; K~|V~ (m x 2d per (b,h)) live in the context's workspace.
  * Errors: CSAT_ERR_INVALID_ARG (NULL/misaligned), CSAT_ERR_SHAPE (default D with m < d or
@@ -211,8 +214,8 @@ int csat_forward(csat_ctx* ctx, const void* Q, const void* K, const void* V, voi
  * csat_forward_host -- same computation with HOST buffers (same layouts and dtype; pinned memory gives
  * asynchronous copies).  Copies Q, K, V to staging buffers the context owns (allocated by the first call, so
  * that call also allocates), computes, copies out back and returns once `stream` has reached the end of all of
- * it.  On the tensor-core path (and with CSAT_PROFILE off) the job is pipelined in chunks of a few heads of one
- * batch element over three internal streams (copy in, compute, copy out) ordered after `stream`, so that the
+ * it.  On the tensor-core path (and with CSAT_PROFILE off) the job is pipelined in runs of consecutive
+ * (batch, head) pairs (about four runs per batch element, at most 64 in all) over three internal streams (copy in, compute, copy out) ordered after `stream`, so that the
  * copies overlap the compute and each other; otherwise everything runs in order on `stream`.
  */
 int csat_forward_host(csat_ctx* ctx, const void* Q_host, const void* K_host, const void* V_host,
@@ -280,6 +283,12 @@ int csat_attend_noalloc(const void* Q, const void* K, const void* V, const void*
  * status word and returns the code it held (0 = none). */
 int csat_selftest_wait_timeout(csat_ctx* ctx, int64_t limit_us, void* stream);
 int csat_clear_status(csat_ctx* ctx, int* code_host);
+
+/* csat_debug_fail_alloc -- test aid, no counterpart in the paper.  Makes the countdown-th device allocation any
+ * context of this process attempts from now on fail as if the device were out of memory (0 switches the aid off;
+ * it also switches itself off after firing).  Lets a test drive the CSAT_ERR_ALLOC paths without exhausting a
+ * GPU.  Process-wide; not for production use. */
+int csat_debug_fail_alloc(int countdown);
 
 /* Bytes of device memory the context currently owns (Phi, workspace, decoder matrices, staging). */
 size_t csat_workspace_bytes(const csat_ctx* ctx);

@@ -18,7 +18,7 @@ ERR_NAMES = {1: "CSAT_ERR_INVALID_ARG", 2: "CSAT_ERR_SHAPE", 3: "CSAT_ERR_ALLOC"
              5: "CSAT_ERR_UNSUPPORTED", 6: "CSAT_ERR_STATE", 7: "CSAT_ERR_TIMEOUT"}
 CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE, CSAT_ENSEMBLE, CSAT_SEPARATE_PHI = 1, 2, 3, 4, 5, 6, 7, 8
 CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER, CSAT_ENSEMBLE_HADAMARD = 0, 1, 2
-KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover", 3: "split_reduce"}
+KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1
 CSAT_LAMBDA, CSAT_STEP, CSAT_SCALE = 1, 2, 3
 
@@ -50,6 +50,7 @@ SIGNATURES = {
                                    C.c_char_p, C.c_size_t]),
     "csat_selftest_wait_timeout": (_int, [_vp, _i64, _vp]),
     "csat_clear_status": (_int, [_vp, C.POINTER(_int)]),
+    "csat_debug_fail_alloc": (_int, [_int]),
     "csat_workspace_bytes": (C.c_size_t, [_vp]),
     "csat_last_launch_count": (_int, [_vp]),
     "csat_last_error": (C.c_char_p, [_vp]),
@@ -222,6 +223,11 @@ def csat_clear_status(h) -> int:
     code = _int()
     _check(h, load().csat_clear_status(h, C.byref(code)))
     return code.value
+
+
+def csat_debug_fail_alloc(countdown: int) -> int:
+    """Test aid: the countdown-th device allocation from now on fails (0 = off)."""
+    return load().csat_debug_fail_alloc(int(countdown))
 
 
 def csat_workspace_bytes(h) -> int:

@@ -891,13 +891,10 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   const uint32_t qb[3] = {64, (uint32_t)kRows, 1};
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
-  static bool attr_set = false;
-  if (!attr_set) {
-    e = cudaFuncSetAttribute(attend_recover_sm100_kernel<D, kUntied>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)C::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static DeviceFlags smem_opt_in;
+  if ((e = ensure_dynamic_smem(attend_recover_sm100_kernel<D, kUntied>, (int)C::kSmemBytes, c->device, smem_opt_in)) !=
+      cudaSuccess)
+    return e;
   const double scale = p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)D);
   const float scale_log2 = (float)(scale * 1.4426950408889634);
   // persistent CTAs, one per SM, each walking the work items (256 queries of one (batch, head)) it owns
@@ -905,13 +902,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   const int64_t items_x = (p.nq + rows_per_item - 1) / rows_per_item;
   const int64_t n_items = items_x * (c->bh_cnt ? c->bh_cnt : p.B * p.H);    // all (batch, head) pairs, or a sub-range
   if (n_items > (int64_t)1 << 30) return cudaErrorInvalidValue;
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-      sms = 148;
-  }
+  const int sms = c->sms;
   const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
   attend_recover_sm100_kernel<D, kUntied><<<grid, kThreads, C::kSmemBytes, s>>>(
       tq, c->tmap_kv, kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, p.T,

@@ -233,12 +233,8 @@ cudaError_t launch(csat_ctx* c, const void* Q, cudaStream_t s) {
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
   if ((e = make_tmap_bf16_3d(&tz, c->bw_dZ16, qd, qs, qb)) != cudaSuccess) return e;
-  static bool attr_set = false;
-  if (!attr_set) {
-    e = cudaFuncSetAttribute(bwd_cols_sm100_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static DeviceFlags smem_opt_in;
+  if ((e = ensure_dynamic_smem(bwd_cols_sm100_kernel<D>, (int)C::kSmemBytes, c->device, smem_opt_in)) != cudaSuccess) return e;
   const float scale = (float)(p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)D));
   const dim3 grid((unsigned)((p.m + kRows - 1) / kRows), (unsigned)(p.B * p.H));
   bwd_cols_sm100_kernel<D><<<grid, kThreads, C::kSmemBytes, s>>>(tq, tz, c->tmap_kv, c->bw_dKV, c->bw_dKV16, c->bw_LD,

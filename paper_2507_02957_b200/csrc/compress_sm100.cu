@@ -115,7 +115,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
       if (!ok) {
         // gave up: let copies that are still in flight land before the CTA's shared memory goes away
         for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
-          mbar_wait(&full[i % C::kStages], (i / C::kStages) & 1, status, 102, cta_abort);
+          mbar_wait_drain(&full[i % C::kStages], (i / C::kStages) & 1);
       }
     }
   } else if (warp == 1) {
@@ -198,12 +198,9 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tk, K, kd, ks, kb)) != cudaSuccess) return e;
   if ((e = make_tmap_bf16_3d(&tv, V, kd, ks, kb)) != cudaSuccess) return e;
-  static bool attr_set = false;
-  if (!attr_set) {
-    e = cudaFuncSetAttribute(compress_sm100_kernel<D, SEP, BG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static DeviceFlags smem_opt_in;
+  if ((e = ensure_dynamic_smem(compress_sm100_kernel<D, SEP, BG>, (int)C::kSmemBytes, c->device, smem_opt_in)) != cudaSuccess)
+    return e;
   // whole batch, or a range of heads of one batch element
   const int64_t Bl = c->bh_cnt ? 1 : p.B, Hl = c->bh_cnt ? c->bh_cnt : p.H;
   const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(((Bl + BG - 1) / BG) * Hl));

@@ -3,6 +3,8 @@
 #include <cstring>
 #include <new>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "csat_internal.h"
 
 namespace {
@@ -21,10 +23,26 @@ int fail_cuda(csat_ctx* c, cudaError_t e, const char* what) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// byte ranges [a, a + na) and [b, b + nb) share at least one byte
+bool ranges_overlap(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+  return a0 < b0 + nb && b0 < a0 + na;
+}
+
+// An NVTX range around a host call (visible in a timeline tool; a no-op when none is attached).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+};
+
+// csat_debug_fail_alloc: the k-th device allocation from now on fails (0 = off)
+std::atomic<int> g_fail_alloc_countdown{0};
+
 template <typename T>
 cudaError_t dev_alloc(csat_ctx* c, T** p, size_t bytes) {
   *p = nullptr;
   if (bytes == 0) return cudaSuccess;
+  if (g_fail_alloc_countdown.load() > 0 && g_fail_alloc_countdown.fetch_sub(1) == 1) return cudaErrorMemoryAllocation;
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), bytes);
   if (e == cudaSuccess) c->bytes += bytes;
   return e;
@@ -117,8 +135,14 @@ void free_all(csat_ctx* c) {
 int allocate_and_generate(csat_ctx* c) {
   const csat::Params& p = c->p;
   cudaError_t e;
+  // Until everything below has succeeded the context holds no usable Phi / workspace: compute calls are refused.
+  c->broken = true;
+  c->tmap_phi_valid = false;
   if ((e = dev_alloc(c, &c->phi, phi_bytes(p))) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(Phi) failed");
-  if ((e = dev_alloc(c, &c->kv, kv_bytes(p))) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(K~|V~) failed");
+  if ((e = dev_alloc(c, &c->kv, kv_bytes(p))) != cudaSuccess) {
+    dev_free(c, &c->phi, phi_bytes(p));
+    return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(K~|V~) failed");
+  }
   if ((e = csat::launch_phi_gen(c->phi, gen_params(p), 0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen launch");
   if ((e = cudaStreamSynchronize(0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen");
   c->tmap_phi_valid = false;
@@ -129,7 +153,20 @@ int allocate_and_generate(csat_ctx* c) {
   }
   c->decoder_dirty = true;
   c->have_forward = false;
+  c->broken = false;
   return CSAT_OK;
+}
+
+// refusal of compute calls and getters after a failed re-allocation
+const char* kBrokenMsg =
+    "an earlier setter failed to re-allocate the context's buffers; set CSAT_BATCH, CSAT_DTYPE or CSAT_SEPARATE_PHI "
+    "again (successfully) before using the context";
+
+int allocate_and_generate_with_batch(csat_ctx* c, int64_t B) {
+  dev_free(c, &c->phi, phi_bytes(c->p));
+  dev_free(c, &c->kv, kv_bytes(c->p));
+  c->p.B = B;
+  return allocate_and_generate(c);
 }
 
 void prof_destroy(csat_ctx* c) {
@@ -174,6 +211,7 @@ extern "C" {
 int csat_version(void) { return 100; }
 
 csat_ctx* csat_create(int64_t n, int64_t m, int64_t d, int64_t H, uint64_t seed) {
+  NvtxRange range("csat_create");
   if (n < 1 || m < 1 || m > n || d < 1 || H < 1) {
     fail(nullptr, CSAT_ERR_SHAPE, "csat_create: need 1 <= m <= n, d >= 1, H >= 1");
     return nullptr;
@@ -198,6 +236,7 @@ csat_ctx* csat_create(int64_t n, int64_t m, int64_t d, int64_t H, uint64_t seed)
     return nullptr;
   }
   cudaGetDevice(&c->device);
+  if (cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->sms <= 0) c->sms = 148;
   csat::Params& p = c->p;
   p.n = n; p.m = m; p.d = d; p.H = H; p.B = 1; p.nq = n;
   p.n_pad = csat::round_up(n, csat::kPhiColPad);
@@ -244,17 +283,18 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
   switch (key) {
     case CSAT_BATCH: {
       if (v < 1 || v > (1 << 20)) return fail(c, CSAT_ERR_SHAPE, "CSAT_BATCH must be >= 1");
-      if (v == p.B) return CSAT_OK;
+      if (v == p.B && !c->broken) return CSAT_OK;
       cudaDeviceSynchronize();
+      if (!c->phi) return allocate_and_generate_with_batch(c, v);   // after a failed re-allocation: start over
       dev_free(c, &c->kv, kv_bytes(p));
       free_staging(c);
       p.B = v;
       c->have_forward = false;
+      c->broken = true;
       if (dev_alloc(c, &c->kv, kv_bytes(p)) != cudaSuccess) return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(K~|V~) failed");
-      if (c->tmap_phi_valid && csat::make_attend_tmaps(c) != cudaSuccess) {
-        c->tmap_phi_valid = false;
+      if (c->tmap_phi_valid && csat::make_attend_tmaps(c) != cudaSuccess)
         return fail(c, CSAT_ERR_CUDA, "tensor maps for K~|V~");
-      }
+      c->broken = false;
       return CSAT_OK;
     }
     case CSAT_NQ:
@@ -264,7 +304,7 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       return CSAT_OK;
     case CSAT_DTYPE: {
       if (v != CSAT_DTYPE_BF16 && v != CSAT_DTYPE_FP32) return fail(c, CSAT_ERR_INVALID_ARG, "unknown CSAT_DTYPE");
-      if ((int)v == p.dtype) return CSAT_OK;
+      if ((int)v == p.dtype && !c->broken) return CSAT_OK;
       cudaDeviceSynchronize();
       dev_free(c, &c->phi, phi_bytes(p));
       dev_free(c, &c->kv, kv_bytes(p));
@@ -279,6 +319,7 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       if (v != CSAT_ENSEMBLE_GAUSSIAN && v != CSAT_ENSEMBLE_RADEMACHER && v != CSAT_ENSEMBLE_HADAMARD)
         return fail(c, CSAT_ERR_INVALID_ARG, "unknown CSAT_ENSEMBLE");
       if ((int)v == p.ensemble) return CSAT_OK;
+      if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
       cudaDeviceSynchronize();
       p.ensemble = (int)v;
       cudaError_t e = csat::launch_phi_gen(c->phi, gen_params(p), 0);   // a Phi set by csat_set_phi is replaced as well
@@ -289,7 +330,7 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
     }
     case CSAT_SEPARATE_PHI: {
       if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_SEPARATE_PHI must be 0 or 1");
-      if ((int)v == p.separate_phi) return CSAT_OK;
+      if ((int)v == p.separate_phi && !c->broken) return CSAT_OK;
       cudaDeviceSynchronize();
       dev_free(c, &c->phi, phi_bytes(p));
       dev_free(c, &c->kv, kv_bytes(p));
@@ -374,6 +415,7 @@ int csat_get_f64(const csat_ctx* c, int key, double* out) {
 int csat_set_phi(csat_ctx* c, const void* phi, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
   if (!phi || !aligned16(phi)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_phi: NULL or misaligned pointer");
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
   std::string why;
   if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
   cudaError_t e = csat::launch_phi_pack(c->phi, phi, gen_params(c->p), (cudaStream_t)stream);
@@ -386,6 +428,7 @@ int csat_get_phi(const csat_ctx* c, void* phi_out, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
   csat_ctx* mc = const_cast<csat_ctx*>(c);
   if (!phi_out || !aligned16(phi_out)) return fail(mc, CSAT_ERR_INVALID_ARG, "csat_get_phi: NULL or misaligned pointer");
+  if (c->broken) return fail(mc, CSAT_ERR_STATE, kBrokenMsg);
   std::string why;
   if (!on_device(c, &why)) return fail(mc, CSAT_ERR_STATE, why);
   cudaError_t e = csat::launch_phi_unpack(phi_out, c->phi, gen_params(c->p), (cudaStream_t)stream);
@@ -501,7 +544,15 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   if (!Q || !K || !V || !out) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward: NULL tensor pointer");
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(out))
     return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward: tensor pointers must be 16-byte aligned");
-  if (out == Q || out == K || out == V) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward: out aliases an input");
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
+  NvtxRange range("csat_forward");
+  {
+    const csat::Params& p = c->p;
+    const size_t es = csat::elt_size(p.dtype);
+    const size_t bq = (size_t)(p.B * p.H * p.nq * p.d) * es, bkv = (size_t)(p.B * p.H * p.n * p.d) * es;
+    if (ranges_overlap(out, bq, Q, bq) || ranges_overlap(out, bq, K, bkv) || ranges_overlap(out, bq, V, bkv))
+      return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward: out overlaps an input");
+  }
   std::string why;
   if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
   if (*(volatile int*)c->status != 0)
@@ -541,6 +592,8 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(dOut) || !aligned16(dQ) || !aligned16(dK) ||
       !aligned16(dV))
     return fail(c, CSAT_ERR_INVALID_ARG, "csat_backward: pointers must be 16-byte aligned");
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
+  NvtxRange range("csat_backward");
   std::string why;
   if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
   if (*(volatile int*)c->status != 0)
@@ -600,6 +653,8 @@ static int ensure_pipeline(csat_ctx* c) {
 int csat_forward_host(csat_ctx* c, const void* Qh, const void* Kh, const void* Vh, void* outh, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
   if (!Qh || !Kh || !Vh || !outh) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward_host: NULL pointer");
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
+  NvtxRange range("csat_forward_host");
   const csat::Params& p = c->p;
   const size_t es = csat::elt_size(p.dtype);
   const size_t bq = (size_t)(p.B * p.H * p.nq * p.d) * es, bkv = (size_t)(p.B * p.H * p.n * p.d) * es;
@@ -651,32 +706,33 @@ int csat_forward_host(csat_ctx* c, const void* Qh, const void* Kh, const void* V
     rc = ensure_decoder(c, s_run, &launches);
     if (rc != CSAT_OK) return rc;
   }
-  int64_t hg = (p.H + 3) / 4;                         // heads per chunk: about four chunks per batch element
-  const int max_chunks = (csat_ctx::kPipeEvents - 2) / 2;
-  while (p.B * ((p.H + hg - 1) / hg) > max_chunks) ++hg;
+  // Chunks are runs of consecutive (batch, head) pairs (contiguous in every tensor; a run may cross from one batch
+  // element into the next): about four per batch element, fewer when that would need more events than there are.
+  const int64_t pairs = p.B * p.H;
+  const int64_t max_chunks = (csat_ctx::kPipeEvents - 2) / 2;
+  int64_t per_chunk = (p.H + 3) / 4;
+  if ((pairs + per_chunk - 1) / per_chunk > max_chunks) per_chunk = (pairs + max_chunks - 1) / max_chunks;
   int chunk = 0;
-  for (int64_t b = 0; b < p.B; ++b) {
-    for (int64_t h0 = 0; h0 < p.H; h0 += hg, ++chunk) {
-      const int64_t cnt = p.H - h0 < hg ? p.H - h0 : hg, bh0 = b * p.H + h0;
-      const size_t oq = (size_t)(bh0 * p.nq * p.d) * es, okv = (size_t)(bh0 * p.n * p.d) * es;
-      const size_t nq_b = (size_t)(cnt * p.nq * p.d) * es, nkv_b = (size_t)(cnt * p.n * p.d) * es;
-      cudaEvent_t ev_in = c->pipe_event[2 + 2 * chunk], ev_run = c->pipe_event[3 + 2 * chunk];
-      if ((e = cudaMemcpyAsync((char*)c->stage_k + okv, (const char*)Kh + okv, nkv_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
-          (e = cudaMemcpyAsync((char*)c->stage_v + okv, (const char*)Vh + okv, nkv_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
-          (e = cudaMemcpyAsync((char*)c->stage_q + oq, (const char*)Qh + oq, nq_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
-          (e = cudaEventRecord(ev_in, s_in)) != cudaSuccess || (e = cudaStreamWaitEvent(s_run, ev_in, 0)) != cudaSuccess)
-        return fail_cuda(c, e, "csat_forward_host: host->device copy");
-      c->bh0 = bh0;
-      c->bh_cnt = cnt;
-      e = csat::launch_sm100_compress(c, c->stage_k, c->stage_v, s_run, &launches);
-      if (e == cudaSuccess) e = csat::launch_sm100_attend_recover(c, c->stage_q, c->stage_o, s_run, &launches);
-      c->bh0 = 0;
-      c->bh_cnt = 0;
-      if (e != cudaSuccess) return fail_cuda(c, e, "csat_forward_host: launch");
-      if ((e = cudaEventRecord(ev_run, s_run)) != cudaSuccess || (e = cudaStreamWaitEvent(s_out, ev_run, 0)) != cudaSuccess ||
-          (e = cudaMemcpyAsync((char*)outh + oq, (const char*)c->stage_o + oq, nq_b, cudaMemcpyDeviceToHost, s_out)) != cudaSuccess)
-        return fail_cuda(c, e, "csat_forward_host: device->host copy");
-    }
+  for (int64_t bh0 = 0; bh0 < pairs; bh0 += per_chunk, ++chunk) {
+    const int64_t cnt = pairs - bh0 < per_chunk ? pairs - bh0 : per_chunk;
+    const size_t oq = (size_t)(bh0 * p.nq * p.d) * es, okv = (size_t)(bh0 * p.n * p.d) * es;
+    const size_t nq_b = (size_t)(cnt * p.nq * p.d) * es, nkv_b = (size_t)(cnt * p.n * p.d) * es;
+    cudaEvent_t ev_in = c->pipe_event[2 + 2 * chunk], ev_run = c->pipe_event[3 + 2 * chunk];
+    if ((e = cudaMemcpyAsync((char*)c->stage_k + okv, (const char*)Kh + okv, nkv_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
+        (e = cudaMemcpyAsync((char*)c->stage_v + okv, (const char*)Vh + okv, nkv_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
+        (e = cudaMemcpyAsync((char*)c->stage_q + oq, (const char*)Qh + oq, nq_b, cudaMemcpyHostToDevice, s_in)) != cudaSuccess ||
+        (e = cudaEventRecord(ev_in, s_in)) != cudaSuccess || (e = cudaStreamWaitEvent(s_run, ev_in, 0)) != cudaSuccess)
+      return fail_cuda(c, e, "csat_forward_host: host->device copy");
+    c->bh0 = bh0;
+    c->bh_cnt = cnt;
+    e = csat::launch_sm100_compress(c, c->stage_k, c->stage_v, s_run, &launches);
+    if (e == cudaSuccess) e = csat::launch_sm100_attend_recover(c, c->stage_q, c->stage_o, s_run, &launches);
+    c->bh0 = 0;
+    c->bh_cnt = 0;
+    if (e != cudaSuccess) return fail_cuda(c, e, "csat_forward_host: launch");
+    if ((e = cudaEventRecord(ev_run, s_run)) != cudaSuccess || (e = cudaStreamWaitEvent(s_out, ev_run, 0)) != cudaSuccess ||
+        (e = cudaMemcpyAsync((char*)outh + oq, (const char*)c->stage_o + oq, nq_b, cudaMemcpyDeviceToHost, s_out)) != cudaSuccess)
+      return fail_cuda(c, e, "csat_forward_host: device->host copy");
   }
   // the caller's stream continues after the last copy; this call returns once everything has landed
   if ((e = cudaEventRecord(ev_done, s_out)) != cudaSuccess || (e = cudaStreamWaitEvent(s, ev_done, 0)) != cudaSuccess ||
@@ -695,6 +751,7 @@ int csat_project_qkv(csat_ctx* c, const void* Xq, const void* Xkv, const void* W
   if (!aligned16(Xq) || !aligned16(Xkv) || !aligned16(W) || !aligned16(Q) || !aligned16(K) || !aligned16(V))
     return fail(c, CSAT_ERR_INVALID_ARG, "csat_project_qkv: pointers must be 16-byte aligned");
   if (d_model < 1 || d_model > (1 << 20)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_project_qkv: d_model out of range");
+  NvtxRange range("csat_project_qkv");
   std::string why;
   if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
   if (*(volatile int*)c->status != 0)
@@ -719,6 +776,7 @@ int csat_project_qkv(csat_ctx* c, const void* Xq, const void* Xkv, const void* W
 int csat_get_compressed(const csat_ctx* c, void* kt, void* vt, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
   csat_ctx* mc = const_cast<csat_ctx*>(c);
+  if (c->broken) return fail(mc, CSAT_ERR_STATE, kBrokenMsg);
   if (!c->have_forward) return fail(mc, CSAT_ERR_STATE, "csat_get_compressed: no forward has run yet");
   if ((kt && !aligned16(kt)) || (vt && !aligned16(vt)))
     return fail(mc, CSAT_ERR_INVALID_ARG, "csat_get_compressed: misaligned pointer");
@@ -729,6 +787,7 @@ int csat_get_compressed(const csat_ctx* c, void* kt, void* vt, void* stream) {
 
 int csat_get_decoder(csat_ctx* c, float* S_out, float* B_out, float* theta_out, float* mu_out, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
   cudaStream_t s = (cudaStream_t)stream;
   int launches = 0;
   int rc = ensure_decoder(c, s, &launches);
@@ -782,6 +841,12 @@ int csat_clear_status(csat_ctx* c, int* code_host) {
   if (code_host) *code_host = *(volatile int*)c->status;
   *(volatile int*)c->status = 0;
   c->err.clear();
+  return CSAT_OK;
+}
+
+int csat_debug_fail_alloc(int countdown) {
+  if (countdown < 0) return CSAT_ERR_INVALID_ARG;
+  g_fail_alloc_countdown.store(countdown);
   return CSAT_OK;
 }
 

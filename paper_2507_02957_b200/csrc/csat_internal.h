@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
+#include <atomic>
 #include <string>
 #include <vector>
 
@@ -16,6 +17,23 @@ namespace csat {
 constexpr int64_t kPhiColPad = 64;
 
 inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+// The opt-in to large dynamic shared memory is a per-device attribute of a kernel: one flag per device ordinal
+// (kernels keep one DeviceFlags each).  Beyond kMaxTracked ordinals the attribute is simply set on every launch.
+struct DeviceFlags {
+  static constexpr int kMaxTracked = 64;
+  std::atomic<uint64_t> done{0};
+  bool test(int dev) const { return dev >= 0 && dev < kMaxTracked && ((done.load(std::memory_order_acquire) >> dev) & 1u); }
+  void set(int dev) { if (dev >= 0 && dev < kMaxTracked) done.fetch_or((uint64_t)1 << dev, std::memory_order_release); }
+};
+
+template <typename Kernel>
+cudaError_t ensure_dynamic_smem(Kernel* kernel, int bytes, int device, DeviceFlags& flags) {
+  if (flags.test(device)) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) flags.set(device);
+  return e;
+}
 
 struct Params {            // plain values kernels need
   int64_t n, m, d, H, B, nq;
@@ -34,6 +52,8 @@ struct csat_ctx {
   csat::Params p;
   int64_t phi_heads() const { return p.H * (p.separate_phi ? 2 : 1); }   // matrices stored in phi
   int device = 0;
+  int sms = 148;              // multiprocessors of `device` (grid size of the persistent kernels)
+  bool broken = false;        // a setter's re-allocation failed: compute calls are refused until a setter succeeds
   int force_simt = 0;         // diagnostic: 1 = FFMA kernels for everything, 2 = for attention/recovery only
 
   // library-owned device memory
@@ -99,7 +119,7 @@ struct csat_ctx {
   int thr_stride() const { return (w_S && w_layers > 1) ? (int)p.H : 0; }
 
   // (batch, head) pairs [bh0, bh0 + bh_cnt) the next kernel launches cover; bh_cnt = 0 means all B*H.  A sub-range
-  // lies inside one batch element (csat_forward_host pipelines copies and compute chunk by chunk)
+  // may cross from one batch element into the next (csat_forward_host pipelines copies and compute run by run)
   int64_t bh0 = 0, bh_cnt = 0;
 
   bool decoder_dirty = true;

@@ -170,12 +170,8 @@ cudaError_t launch(csat_ctx* c, const void* g16, void* dK, void* dV, cudaStream_
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tphi, c->phi, pd, ps, pb)) != cudaSuccess) return e;
   if ((e = make_tmap_bf16_3d(&tg, g16, gd, gs, gb)) != cudaSuccess) return e;
-  static bool attr_set = false;
-  if (!attr_set) {
-    e = cudaFuncSetAttribute(phiT_sm100_kernel<D, SEP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static DeviceFlags smem_opt_in;
+  if ((e = ensure_dynamic_smem(phiT_sm100_kernel<D, SEP>, (int)C::kSmemBytes, c->device, smem_opt_in)) != cudaSuccess) return e;
   const dim3 grid((unsigned)((p.n + kTileM - 1) / kTileM), (unsigned)(p.B * p.H));
   phiT_sm100_kernel<D, SEP><<<grid, kThreads, C::kSmemBytes, s>>>(tphi, tg, (__nv_bfloat16*)dK, (__nv_bfloat16*)dV,
                                                                   (int)p.m, (int)p.n, (int)p.H, c->status);

@@ -235,27 +235,15 @@ cudaError_t launch_project(csat_ctx* c, const void* X, const void* W, int64_t n_
   a.ntiles = (ncols + kTileN - 1) / kTileN;
   const int64_t n_tiles = (int64_t)a.B * a.mtiles * a.ntiles;
   if (n_tiles > (int64_t)1 << 30) return cudaErrorInvalidValue;
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
-      sms = 148;
-  }
+  const int sms = c->sms;
   const unsigned grid = (unsigned)(n_tiles < sms ? n_tiles : sms);
   if (p.d == 64) {
-    static bool attr64 = false;
-    if (!attr64) {
-      if ((e = cudaFuncSetAttribute(project_sm100_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes)) != cudaSuccess) return e;
-      attr64 = true;
-    }
+    static DeviceFlags opt_in64;
+    if ((e = ensure_dynamic_smem(project_sm100_kernel<64>, (int)kSmemBytes, c->device, opt_in64)) != cudaSuccess) return e;
     project_sm100_kernel<64><<<grid, kThreads, kSmemBytes, s>>>(tx, tw, a, c->status);
   } else {
-    static bool attr128 = false;
-    if (!attr128) {
-      if ((e = cudaFuncSetAttribute(project_sm100_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes)) != cudaSuccess) return e;
-      attr128 = true;
-    }
+    static DeviceFlags opt_in128;
+    if ((e = ensure_dynamic_smem(project_sm100_kernel<128>, (int)kSmemBytes, c->device, opt_in128)) != cudaSuccess) return e;
     project_sm100_kernel<128><<<grid, kThreads, kSmemBytes, s>>>(tx, tw, a, c->status);
   }
   return cudaGetLastError();

@@ -187,7 +187,12 @@ def test_abi_errors_and_determinism():
     assert lib.csat_forward(ctx.h, None, p(K), p(V), p(out2), s) == 1
     assert lib.csat_forward(ctx.h, p(Q) + 2, p(K), p(V), p(out2), s) == 1     # misaligned
     assert lib.csat_forward(ctx.h, p(Q), p(K), p(V), p(Q), s) == 1            # out aliases Q
-    assert "alias" in binding.csat_last_error(ctx.h)
+    assert "overlap" in binding.csat_last_error(ctx.h)
+    big = torch.empty(2 * Q.numel(), dtype=Q.dtype, device="cuda")
+    big[: Q.numel()].copy_(Q.reshape(-1))
+    shifted = big[64: 64 + Q.numel()]                                         # 128 bytes into the copy of Q
+    assert lib.csat_forward(ctx.h, p(big), p(K), p(V), p(shifted), s) == 1    # out overlaps Q without equal pointers
+    assert "overlap" in binding.csat_last_error(ctx.h)
     assert lib.csat_set_i64(ctx.h, 99, 1) == 1
     assert lib.csat_set_i64(ctx.h, binding.CSAT_T, -1) == 1
     assert lib.csat_set_f64(ctx.h, binding.CSAT_LAMBDA, -0.5) == 1
