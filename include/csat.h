@@ -74,6 +74,8 @@ enum {
                           same seeded generator, the decoder's default D is the block of Phi_V, and
                           csat_set_phi / csat_get_phi then move [2H, m, n]: the H matrices Phi_K, then the H
                           matrices Phi_V.  Changing it regenerates both from the seed                 */
+  CSAT_KEEP_MASKS = 9, /* 1: csat_backward also keeps its shrinkage decisions (one 32-bit word per (b, h, query,
+                          column); needs CSAT_T <= 32) for csat_get_backward_masks.  0 (default): not kept  */
   CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls
                           (0 = off, default; at most 4096).  Setting it creates/destroys
                           events, so set it outside the timed region                    */
@@ -177,12 +179,21 @@ int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, c
  *   dQ [B,H,n_q,d], dK, dV [B,H,n,d]  outputs (context dtype)
  * Nothing of an earlier csat_forward is reused: the call compresses K, V again and recomputes what it needs in
  * float32.  Its first call allocates float32 scratch (B H (n_q (d + 2) + 2 m d) floats and transposed
- * copies of the decoder matrices, counted by csat_workspace_bytes).  CSAT_T <= 32, d <= 256 and B H <= 32767, else CSAT_ERR_UNSUPPORTED.  This first
+ * copies of the decoder matrices, plus B H n_q d words with CSAT_KEEP_MASKS, counted by csat_workspace_bytes).  CSAT_T <= 32, d <= 256 and B H <= 32767, else CSAT_ERR_UNSUPPORTED.  This first
  * version recomputes each query row (scores, recurrence, its backward, dQ) on plain FFMA kernels in float32; bf16
  * contexts with d in {64, 128} then run the gradients of K~|V~ (P^T dZ, dS^T Q) and the product with Phi^T on the
  * tensor cores with bf16 operands, everything else stays on FFMA kernels. */
 int csat_backward(csat_ctx* ctx, const void* Q, const void* K, const void* V, const void* dOut, void* dQ, void* dK,
                   void* dV, void* stream);
+
+/* csat_get_backward_masks -- the decisions |x_t| > theta_t the most recent csat_backward took in the layers of the
+ * LISTA recurrence (the derivative of eta_theta is 1 or 0 by that decision; the paper prints no backward pass).
+ *   masks_out [B, H, n_q, d] uint32, device: bit t of a word = the decision of layer t for that query and column.
+ * The derivative of eta_theta is discontinuous, so two implementations in different precisions may decide an entry
+ * within rounding distance of its threshold differently; a reference that is given these decisions can be compared
+ * with csat_backward's gradients element by element.  Needs CSAT_KEEP_MASKS = 1 before that csat_backward and
+ * CSAT_T >= 1, else CSAT_ERR_STATE.  Copied on `stream`. */
+int csat_get_backward_masks(const csat_ctx* ctx, uint32_t* masks_out, void* stream);
 
 /* csat_project_qkv -- paper: the projection equation Q = X W^Q, K = X W^K, V = X W^V ("Mathematical Framework"),
  * for all heads at once, written in the layout csat_forward reads.

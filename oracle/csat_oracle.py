@@ -251,15 +251,22 @@ def csat_forward(Q, K, V, Phi, *, T, lam, Psi=None, D=None, step=None, scale=Non
 # backward: d out / d (Q, K, V), chain rule through the forward's equations in reverse order
 # ----------------------------------------------------------------------------
 def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None, scale=None, weights=None,
-                       Phi_v_h=None, stages: dict | None = None, kv_round=None):
+                       Phi_v_h=None, stages: dict | None = None, masks=None):
     """Vector-Jacobian product of csat_forward_head for one (batch, head): given G = dL/d out [n_q,d], returns
-    (dL/dQ [n_q,d], dL/dK [n,d], dL/dV [n,d]).  Phi, Psi and the decoder weights are constants.
-    The shrinkage eta_theta has derivative 1 where |x| > theta and 0 elsewhere (0 is taken at |x| = theta).
-    stages (optional dict) receives min_margin [n_q] = min over layers and columns of | |x_t| - theta_t |, which
-    tells how close a row came to a kink of eta.
-    kv_round (optional callable) is applied to K~ and V~ before they are used: a library that keeps them in a
-    16-bit workspace takes its shrinkage decisions from the rounded values, and so must the reference.  The
-    gradient then treats the rounding as the identity."""
+    (dL/dQ [n_q,d], dL/dK [n,d], dL/dV [n,d]).  Phi is a constant.
+    The shrinkage eta_theta(x) = x - theta sign(x) where |x| > theta and 0 elsewhere; its derivative with respect
+    to x is 1 where |x| > theta and 0 elsewhere (0 is taken at |x| = theta), with respect to theta it is -sign(x)
+    where |x| > theta.
+    masks (optional, bool [T,n_q,d]): the decisions |x_t| > theta_t taken elsewhere.  The derivative of eta is
+    discontinuous, so an implementation in lower precision may decide an entry within rounding distance of its
+    threshold the other way; both sides of a comparison then have to use the same decisions.  With masks given,
+    layer t differentiates alpha^{t+1} = masks[t] o (x_t - theta_t sign(x_t)); the forward values stay this
+    function's own.
+    stages (optional dict) receives: xs [T,n_q,d] (the pre-activations x_t), masks [T,n_q,d] (this function's own
+    decisions), min_margin [n_q] = min over layers and columns of | |x_t| - theta_t |, dZ, A, Z, and the gradients
+    with respect to the decoder's parameters as used in layer t: dS [T,d,d], dB [T,d,d], dtheta [T] (with weights
+    shared by the layers the gradient of the shared matrix is the sum over t) and dPsi [d,d] of the
+    reconstruction out = alpha Psi^T (None without a dictionary)."""
     Q = np.asarray(Q, F64)
     K = np.asarray(K, F64)
     V = np.asarray(V, F64)
@@ -271,49 +278,62 @@ def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None
     # forward, keeping what the backward needs
     Kt = compress(Phi_h, K)
     Vt = compress(Phi_v, V)
-    if kv_round is not None:
-        Kt, Vt = np.asarray(kv_round(Kt), F64), np.asarray(kv_round(Vt), F64)
     A = softmax_rows(compressed_scores(Q, Kt, scale))
     Z = compressed_output(A, Vt)
     margin = np.full(Q.shape[0], np.inf)
-    if int(T) == 0:
+    T = int(T)
+    if T == 0:
         dZ = G.copy()
+        if stages is not None:
+            stages.update(xs=np.zeros((0,) + Z.shape), masks=np.zeros((0,) + Z.shape, dtype=bool),
+                          dS=np.zeros((0, d, d)), dB=np.zeros((0, d, d)), dtheta=np.zeros(0), dPsi=None)
     else:
         if weights is not None:
             S_w, B_w, thetas = weights
             S_w, B_w = np.asarray(S_w, F64), np.asarray(B_w, F64)
-            S_l = [S_w[t] if S_w.ndim == 3 else S_w for t in range(int(T))]
-            B_l = [B_w[t] if B_w.ndim == 3 else B_w for t in range(int(T))]
+            S_l = [S_w[t] if S_w.ndim == 3 else S_w for t in range(T)]
+            B_l = [B_w[t] if B_w.ndim == 3 else B_w for t in range(T)]
             thetas = [float(th) for th in thetas]
         else:
             Dm = default_decoder_matrix(Phi_v, d) if D is None else np.asarray(D, F64)
             M = Dm if Psi is None else Dm @ np.asarray(Psi, F64)
             S_dec, B_dec, theta, _ = decoder_setup(M, lam, step)
-            S_l, B_l, thetas = [S_dec] * int(T), [B_dec] * int(T), [float(theta)] * int(T)
+            S_l, B_l, thetas = [S_dec] * T, [B_dec] * T, [float(theta)] * T
         alpha = np.zeros_like(Z)
-        xs = []
-        for t in range(int(T)):
+        alphas, xs = [], []
+        for t in range(T):
             x = alpha @ S_l[t] + Z @ B_l[t]
+            alphas.append(alpha)
             xs.append(x)
             margin = np.minimum(margin, np.abs(np.abs(x) - thetas[t]).min(axis=1))
             alpha = soft_threshold(x, thetas[t])
-        # out = alpha Psi^T  ->  d alpha = G Psi
+        own_masks = np.stack([np.abs(xs[t]) > thetas[t] for t in range(T)])
+        use = own_masks if masks is None else np.asarray(masks, dtype=bool)
+        assert use.shape == own_masks.shape
+        # out = alpha Psi^T  ->  d alpha = G Psi, d Psi = G^T alpha
         d_alpha = G if Psi is None else G @ np.asarray(Psi, F64)
+        dPsi = None if Psi is None else G.T @ alpha
         dZ = np.zeros_like(Z)
-        for t in range(int(T) - 1, -1, -1):
-            dx = d_alpha * (np.abs(xs[t]) > thetas[t])          # through eta_theta
-            dZ += dx @ B_l[t].T                                  # x_t = alpha_t S_t + Z B_t
+        dS, dB, dth = np.zeros((T, d, d)), np.zeros((T, d, d)), np.zeros(T)
+        for t in range(T - 1, -1, -1):
+            dx = d_alpha * use[t]                                # through eta_theta, with respect to x_t
+            dth[t] = -(dx * np.sign(xs[t])).sum()                # ... and with respect to theta_t
+            dS[t] = alphas[t].T @ dx                             # x_t = alpha_t S_t + Z B_t
+            dB[t] = Z.T @ dx
+            dZ += dx @ B_l[t].T
             d_alpha = dx @ S_l[t].T
+        if stages is not None:
+            stages.update(xs=np.stack(xs), masks=own_masks, dS=dS, dB=dB, dtheta=dth, dPsi=dPsi)
     if stages is not None:
         stages.update(min_margin=margin, dZ=dZ, A=A, Z=Z)
     # Z = A~ V~
     dA = dZ @ Vt.T
     dVt = A.T @ dZ
     # A~ = softmax(S) row-wise:  dS = A o (dA - rowsum(dA o A))
-    dS = A * (dA - (dA * A).sum(axis=1, keepdims=True))
+    dS_scores = A * (dA - (dA * A).sum(axis=1, keepdims=True))
     # S = sc Q K~^T
-    dQ = sc * (dS @ Kt)
-    dKt = sc * (dS.T @ Q)
+    dQ = sc * (dS_scores @ Kt)
+    dKt = sc * (dS_scores.T @ Q)
     # K~ = Phi K, V~ = Phi_V V
     dK = Phi_h.T @ dKt
     dV = Phi_v.T @ dVt
@@ -321,8 +341,9 @@ def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None
 
 
 def csat_backward(Q, K, V, Phi, G, *, T, lam, Psi=None, D=None, step=None, scale=None, weights=None, Phi_V=None,
-                  stages: list | None = None, kv_round=None):
-    """Vector-Jacobian product of csat_forward: G [B,H,n_q,d] -> (dQ [B,H,n_q,d], dK [B,H,n,d], dV [B,H,n,d])."""
+                  stages: list | None = None, masks=None):
+    """Vector-Jacobian product of csat_forward: G [B,H,n_q,d] -> (dQ [B,H,n_q,d], dK [B,H,n,d], dV [B,H,n,d]).
+    masks (optional, bool [B,H,T,n_q,d]): shrinkage decisions to differentiate with, see csat_backward_head."""
     Q = np.asarray(Q)
     B, H, nq, d = Q.shape
     n = np.asarray(K).shape[2]
@@ -341,7 +362,8 @@ def csat_backward(Q, K, V, Phi, G, *, T, lam, Psi=None, D=None, step=None, scale
             st = {} if stages is not None else None
             dQ[b, h], dK[b, h], dV[b, h] = csat_backward_head(
                 Q[b, h], K[b, h], V[b, h], Phi[h], G[b, h], T=T, lam=lam, Psi=psi_h, D=D_h, step=step, scale=scale,
-                weights=w_h, Phi_v_h=None if Phi_V is None else Phi_V[h], stages=st, kv_round=kv_round)
+                weights=w_h, Phi_v_h=None if Phi_V is None else Phi_V[h], stages=st,
+                masks=None if masks is None else np.asarray(masks)[b, h])
             if stages is not None:
                 stages.append(st)
     return dQ, dK, dV

@@ -17,6 +17,7 @@ CSAT_OK = 0
 ERR_NAMES = {1: "CSAT_ERR_INVALID_ARG", 2: "CSAT_ERR_SHAPE", 3: "CSAT_ERR_ALLOC", 4: "CSAT_ERR_CUDA",
              5: "CSAT_ERR_UNSUPPORTED", 6: "CSAT_ERR_STATE", 7: "CSAT_ERR_TIMEOUT"}
 CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE, CSAT_ENSEMBLE, CSAT_SEPARATE_PHI = 1, 2, 3, 4, 5, 6, 7, 8
+CSAT_KEEP_MASKS = 9
 CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER, CSAT_ENSEMBLE_HADAMARD = 0, 1, 2
 KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1
@@ -45,6 +46,7 @@ SIGNATURES = {
     "csat_forward_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
     "csat_get_decoder": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "csat_get_backward_masks": (_int, [_vp, _vp, _vp]),
     "csat_get_profile": (_int, [_vp, _i64, _int, C.POINTER(_int), C.POINTER(C.c_float), C.POINTER(_int)]),
     "csat_attend_noalloc": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _i64, _i64, _int, _dbl, _vp,
                                    C.c_char_p, C.c_size_t]),
@@ -186,6 +188,10 @@ def csat_get_compressed(h, kt_out, vt_out, stream=None):
 
 def csat_get_decoder(h, S_out, B_out, theta_out, mu_out, stream=None):
     _check(h, load().csat_get_decoder(h, _ptr(S_out), _ptr(B_out), _ptr(theta_out), _ptr(mu_out), _stream(stream)))
+
+
+def csat_get_backward_masks(h, masks_out, stream=None):
+    _check(h, load().csat_get_backward_masks(h, _ptr(masks_out), _stream(stream)))
 
 
 def csat_get_profile(h, call_index):
@@ -350,6 +356,13 @@ class Csat:
         dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
         csat_backward(self.h, Q, K, V, dOut, dQ, dK, dV)
         return dQ, dK, dV
+
+    def backward_masks(self):
+        """The shrinkage decisions of the most recent backward (CSAT_KEEP_MASKS = 1): int32 [B,H,n_q,d], bit t of a
+        word = |x_t| > theta_t."""
+        out = self._new(self.B, self.H, self.n_q, self.d, dtype=torch.int32)
+        csat_get_backward_masks(self.h, out)
+        return out
 
     def project_qkv(self, X, W, Xkv=None):
         """Q, K, V [B,H,tokens,d] from tokens X [B,n_q,d_model] (and Xkv [B,n,d_model] for cross-attention; default X)

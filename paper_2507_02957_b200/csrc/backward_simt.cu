@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
     const T* __restrict__ Q,
     const T* __restrict__ G, const T* __restrict__ kv, const float* __restrict__ S_dec, const float* __restrict__ B_dec,
     const float* __restrict__ S_decT, const float* __restrict__ B_decT, int64_t layer_stride, const float* __restrict__ theta, int theta_stride, const float* __restrict__ psi_f32,
-    int64_t nq, int64_t m, int d, int H, int T_iters, float scale) {
+    int64_t nq, int64_t m, int d, int H, int T_iters, float scale, uint32_t* __restrict__ ws_masks) {
   extern __shared__ float smem[];
   const int d2 = 2 * d, ldk = d2 + 1;
   float* kvs = smem;                               // [32][2d+1]
@@ -166,6 +166,13 @@ __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
         const float x = (it > 0 ? t[j] : 0.f) + c[j];
         if (fabsf(x) > th) mask[j] |= 1u << it;
         a[j] = x - fminf(fmaxf(x, -th), th);
+      }
+    }
+    if (ws_masks && live) {
+#pragma unroll
+      for (int j = 0; j < DC; ++j) {
+        const int col = lane + 32 * j;
+        if (col < d) ws_masks[grow * d + col] = mask[j];          // bit t: |x_t| > theta_t
       }
     }
     float da[DC], dx[DC];
@@ -407,7 +414,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
     if (e == cudaSuccess)                                                                                            \
       bwd_rows_kernel<T, DC><<<grid, kRowWarps * 32, sm, s>>>(                                                       \
           (T*)dQ, c->bw_dZ, tc_stages ? c->bw_dZ16 : nullptr, c->bw_LD, (const T*)Q, (const T*)G, (const T*)c->kv, Sd, Bd, SdT, BdT, lstride, c->thr(), \
-          c->thr_stride(), c->psi ? c->psi_f32 : nullptr, p.nq, p.m, d, (int)p.H, p.T, scale);                       \
+          c->thr_stride(), c->psi ? c->psi_f32 : nullptr, p.nq, p.m, d, (int)p.H, p.T, scale, c->bw_masks);          \
   } while (0)
     if (dc <= 2) CSAT_BWD_ROWS(2);
     else if (dc <= 4) CSAT_BWD_ROWS(4);

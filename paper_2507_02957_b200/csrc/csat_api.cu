@@ -91,6 +91,9 @@ void free_backward(csat_ctx* c) {
   dev_free(c, &c->bw_WT, c->bw_bytes_WT);
   dev_free(c, &c->bw_dKV16, c->bw_bytes_dKV16);
   dev_free(c, &c->bw_dZ16, c->bw_bytes_dZ16);
+  dev_free(c, &c->bw_masks, c->bw_bytes_masks);
+  c->bw_bytes_masks = 0;
+  c->have_masks = false;
   c->bw_bytes_dZ = c->bw_bytes_LD = c->bw_bytes_dKV = c->bw_bytes_WT = c->bw_bytes_dKV16 = c->bw_bytes_dZ16 = 0;
 }
 
@@ -345,6 +348,11 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       if (v < 0 || v > 2) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_FORCE_SIMT must be 0, 1 or 2");
       c->force_simt = (int)v;
       return CSAT_OK;
+    case CSAT_KEEP_MASKS:
+      if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_KEEP_MASKS must be 0 or 1");
+      if ((v != 0) != c->keep_masks) { cudaDeviceSynchronize(); free_backward(c); }
+      c->keep_masks = v != 0;
+      return CSAT_OK;
     case CSAT_PROFILE: {
       if (v < 0 || v > 4096) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_PROFILE must be in [0, 4096]");
       cudaDeviceSynchronize();
@@ -380,6 +388,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
     case CSAT_SEPARATE_PHI: *out = c->p.separate_phi; return CSAT_OK;
     case CSAT_FORCE_SIMT: *out = c->force_simt; return CSAT_OK;
     case CSAT_PROFILE: *out = c->prof_slots; return CSAT_OK;
+    case CSAT_KEEP_MASKS: *out = c->keep_masks ? 1 : 0; return CSAT_OK;
     default: return CSAT_ERR_INVALID_ARG;
   }
 }
@@ -613,14 +622,16 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   const size_t bz = (size_t)(p.B * p.H * p.nq * p.d) * 4, bl = (size_t)(p.B * p.H * p.nq * 2) * 4,
                bk = (size_t)(p.B * p.H * p.m * 2 * p.d) * 4,
                bw = (size_t)(2 * (c->w_untied ? c->w_layers : 1) * p.H * p.d * p.d) * 4,
-               b16 = c->tmap_phi_valid ? bk / 2 : 0, z16 = c->tmap_phi_valid ? bz / 2 : 0;
-  if (c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
+               b16 = c->tmap_phi_valid ? bk / 2 : 0, z16 = c->tmap_phi_valid ? bz / 2 : 0,
+               bm = c->keep_masks && p.T > 0 ? bz : 0;
+  if (c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
       c->bw_bytes_dKV16 != b16 || c->bw_bytes_dZ16 != z16) {
     cudaDeviceSynchronize();
     free_backward(c);
     c->bw_bytes_dZ = bz; c->bw_bytes_LD = bl; c->bw_bytes_dKV = bk; c->bw_bytes_WT = bw; c->bw_bytes_dKV16 = b16;
     c->bw_bytes_dZ16 = z16;
-    if (dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
+    c->bw_bytes_masks = bm;
+    if (dev_alloc(c, &c->bw_masks, bm) != cudaSuccess || dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
         dev_alloc(c, &c->bw_dKV, bk) != cudaSuccess || dev_alloc(c, &c->bw_WT, bw) != cudaSuccess ||
         dev_alloc(c, &c->bw_dKV16, b16) != cudaSuccess || dev_alloc(c, &c->bw_dZ16, z16) != cudaSuccess) {
       free_backward(c);
@@ -633,6 +644,7 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward: compress launch");
   e = csat::launch_backward(c, Q, dOut, dQ, dK, dV, s, &launches);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward launch");
+  c->have_masks = c->bw_masks != nullptr;
   c->have_forward = true;
   c->last_launches = launches;
   return CSAT_OK;
@@ -799,6 +811,17 @@ int csat_get_decoder(csat_ctx* c, float* S_out, float* B_out, float* theta_out, 
   if (theta_out && e == cudaSuccess) e = cudaMemcpyAsync(theta_out, c->thr(), (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
   if (mu_out && e == cudaSuccess) e = cudaMemcpyAsync(mu_out, c->mu, (size_t)p.H * 4, cudaMemcpyDeviceToDevice, s);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_get_decoder");
+  return CSAT_OK;
+}
+
+int csat_get_backward_masks(const csat_ctx* c, uint32_t* masks_out, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  csat_ctx* mc = const_cast<csat_ctx*>(c);
+  if (!masks_out || !aligned16(masks_out)) return fail(mc, CSAT_ERR_INVALID_ARG, "csat_get_backward_masks: NULL or misaligned pointer");
+  if (!c->have_masks)
+    return fail(mc, CSAT_ERR_STATE, "csat_get_backward_masks: no csat_backward with CSAT_KEEP_MASKS = 1 and CSAT_T > 0 has run");
+  cudaError_t e = cudaMemcpyAsync(masks_out, c->bw_masks, c->bw_bytes_masks, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
+  if (e != cudaSuccess) return fail_cuda(mc, e, "csat_get_backward_masks");
   return CSAT_OK;
 }
 

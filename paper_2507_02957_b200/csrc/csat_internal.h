@@ -97,6 +97,12 @@ struct csat_ctx {
   __nv_bfloat16* bw_dKV16 = nullptr;     // bf16 copy of dK~|dV~ (operand of the tensor-core Phi^T product)
   __nv_bfloat16* bw_dZ16 = nullptr;      // bf16 copy of dZ (operand of the tensor-core dK~|dV~ stage)
   size_t bw_bytes_dZ = 0, bw_bytes_LD = 0, bw_bytes_dKV = 0, bw_bytes_WT = 0, bw_bytes_dKV16 = 0, bw_bytes_dZ16 = 0;
+  // CSAT_KEEP_MASKS: the shrinkage decisions of the most recent csat_backward, one word per (b, h, query, column),
+  // bit t = |x_t| > theta_t
+  bool keep_masks = false;
+  bool have_masks = false;
+  uint32_t* bw_masks = nullptr;
+  size_t bw_bytes_masks = 0;
   // staging for csat_forward_host
   void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
   size_t stage_bytes_q = 0, stage_bytes_kv = 0;

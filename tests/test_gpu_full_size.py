@@ -1,9 +1,11 @@
 """GPU parity at the full workload sizes, in the launch configuration bench.py times.
 
 The float64 oracle cannot run a whole workload in seconds, but every (batch, head) pair is independent, so a
-few sampled pairs are checked in full, element by element, against the oracle (same seeded inputs, the
-library's exported Phi), with recovery disabled, at the workload's own (T, lambda) and at lambda = 0 (dense
-output).  Properties that hold at any size cover the rest: no NaN/Inf anywhere, and bit-identical reruns.
+few sampled pairs (first and last batch element, first and last head, one in between) are checked in full, element
+by element, against the oracle (same seeded inputs, the library's exported Phi), with recovery disabled, at the
+workload's own (T, lambda), at lambda = 0 (dense output) and at the lambda that shrinks about half of the first
+layer's coefficients.  Properties that hold at any size cover the rest: no NaN/Inf anywhere, and bit-identical
+reruns.
 """
 import numpy as np
 import pytest
@@ -15,7 +17,10 @@ from gpu_util import TOL, device_inputs, make_ctx, rel_err, to_np
 
 pytestmark = pytest.mark.gpu
 
-SAMPLES = {"c2": [(0, 0), (17, 5), (31, 11)], "c3": [(0, 0), (7, 11)], "c4": [(0, 0), (15, 7)], "c5": [(1, 9)]}
+SAMPLES = {"c2": [(0, 0), (17, 5), (31, 11), (0, 11), (31, 0)],
+           "c3": [(0, 0), (7, 11), (0, 11), (7, 0), (3, 5)],
+           "c4": [(0, 0), (15, 7), (0, 7), (15, 0), (8, 3)],
+           "c5": [(0, 0), (1, 15), (0, 15), (1, 0), (1, 9)]}
 
 
 @pytest.mark.parametrize("key", sorted(SAMPLES))
@@ -29,7 +34,11 @@ def test_sampled_pairs_of_the_full_workload(key):
     phi = ctx.get_phi()
     tol = TOL[w.dtype]
     psi64 = None if inp["Psi"] is None else inp["Psi"].astype(np.float64)
-    for T, lam in [(0, w.lam), (w.T, w.lam), (w.T, 0.0)]:
+    # lambda that keeps about half of the first layer's coefficients, from the oracle alone (pair (0, 0))
+    st = {}
+    orc.csat_forward_head(inp["Q"][0, 0], inp["K"][0, 0], inp["V"][0, 0], to_np(phi[0]), T=1, lam=0.0, Psi=psi64, stages=st)
+    lam_med = float(np.median(np.abs(st["Z"] @ st["B_dec"])) / st["mu"])
+    for T, lam in [(0, w.lam), (w.T, w.lam), (w.T, 0.0), (w.T, lam_med)]:
         ctx.set(T=T, lam=lam)
         out = ctx.forward(Q, K, V)
         assert torch.isfinite(out).all()
@@ -40,6 +49,9 @@ def test_sampled_pairs_of_the_full_workload(key):
             ref = orc.csat_forward_head(inp["Q"][b, h], inp["K"][b, h], inp["V"][b, h], to_np(phi[h]), T=T, lam=lam,
                                         Psi=psi64, stages=st)
             got = to_np(out[b, h])
+            if (T, lam) == (w.T, lam_med):
+                frac = float((st["alpha"] != 0).mean())
+                assert 0.2 < frac < 0.8, (key, b, h, frac)          # the setting really is the half-shrunk one
             if np.abs(ref).max() == 0.0:
                 assert np.abs(got).max() <= st["theta"] * tol, (key, b, h, T, lam)
             else:

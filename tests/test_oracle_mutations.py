@@ -155,6 +155,33 @@ def _backward_softmax_without_row_term(Q, K, V, Phi_h, G, **kw):
     return sc * dS @ Kt, Phi_h.T @ (sc * dS.T @ np.asarray(Q, F64)), Phi_v.T @ (st["A"].T @ st["dZ"])
 
 
+def _backward_masks_of_the_wrong_layer(Q, K, V, Phi_h, G, **kw):
+    # supplied decisions applied one layer late (the natural ones are left alone)
+    if kw.get("masks") is not None:
+        kw = {**kw, "masks": np.roll(np.asarray(kw["masks"]), 1, axis=0)}
+    return _orig_backward_head(Q, K, V, Phi_h, G, **kw)
+
+
+def _backward_masks_ignored(Q, K, V, Phi_h, G, **kw):
+    return _orig_backward_head(Q, K, V, Phi_h, G, **{**kw, "masks": None})
+
+
+def _backward_dtheta_without_sign(Q, K, V, Phi_h, G, **kw):
+    st = kw.get("stages")
+    out = _orig_backward_head(Q, K, V, Phi_h, G, **kw)
+    if st is not None and len(st["dtheta"]):
+        st["dtheta"] = -np.abs(st["dtheta"])
+    return out
+
+
+def _backward_dS_from_the_next_iterate(Q, K, V, Phi_h, G, **kw):
+    st = kw.get("stages")
+    out = _orig_backward_head(Q, K, V, Phi_h, G, **kw)
+    if st is not None and len(st["dS"]) > 1:
+        st["dS"] = np.roll(st["dS"], -1, axis=0)
+    return out
+
+
 _orig_lista = orc.lista
 _orig_project = orc.project_qkv
 _orig_backward_head = orc.csat_backward_head
@@ -186,6 +213,10 @@ MUTATIONS = {
     "project: queries and keys exchanged": ("project_qkv", _project_W_transposed_per_head),
     "backward: score scale dropped": ("csat_backward_head", _backward_scale_dropped),
     "backward: softmax Jacobian without the row term": ("csat_backward_head", _backward_softmax_without_row_term),
+    "backward: supplied decisions one layer late": ("csat_backward_head", _backward_masks_of_the_wrong_layer),
+    "backward: supplied decisions ignored": ("csat_backward_head", _backward_masks_ignored),
+    "backward: d theta loses the sign of x": ("csat_backward_head", _backward_dtheta_without_sign),
+    "backward: d S_t taken from the layer after": ("csat_backward_head", _backward_dS_from_the_next_iterate),
     "compress: |Phi|": ("compress", _compress_abs),
     "output: weights ignored": ("compressed_output", _output_uses_unweighted),
 }

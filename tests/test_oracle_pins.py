@@ -650,17 +650,22 @@ def test_project_qkv_matches_scalar_loops_and_layout():
 # ---------------------------------------------------------------------------------------------------
 # backward (vector-Jacobian product of the forward with respect to Q, K, V)
 # ---------------------------------------------------------------------------------------------------
-def _torch_forward(Q, K, V, Phi, Phi_v, S_l, B_l, thetas, Psi, scale):
-    """The forward written with torch float64 ops, for autograd (an independent derivation of the gradient)."""
+def _torch_forward(Q, K, V, Phi, Phi_v, S_l, B_l, thetas, Psi, scale, forced_masks=None):
+    """The forward written with torch float64 ops, for autograd (an independent derivation of the gradient).
+    forced_masks [T,n_q,d]: layer t computes masks[t] o (x - theta sign(x)) instead of the shrinkage, i.e. the
+    shrinkage with its decisions |x| > theta taken from outside."""
     import torch
     Kt, Vt = Phi @ K, Phi_v @ V
     A = torch.softmax(scale * (Q @ Kt.T), dim=1)
     Z = A @ Vt
     alpha = torch.zeros_like(Z)
     out = Z
-    for S_t, B_t, th in zip(S_l, B_l, thetas):
+    for t, (S_t, B_t, th) in enumerate(zip(S_l, B_l, thetas)):
         x = alpha @ S_t + Z @ B_t
-        alpha = torch.sign(x) * torch.relu(torch.abs(x) - th)
+        if forced_masks is None:
+            alpha = torch.sign(x) * torch.relu(torch.abs(x) - th)
+        else:
+            alpha = forced_masks[t] * (x - th * torch.sign(x))
         out = alpha
     if Psi is not None and len(thetas) > 0:
         out = out @ Psi.T
@@ -693,15 +698,74 @@ def _backward_case(seed, T, with_psi, separate, untied):
     got = orc.csat_backward_head(Q, K, V, Phi, G, T=T, lam=lam, Psi=Psi, weights=weights, Phi_v_h=Phi_v, stages=st)
     tq, tk, tv = (torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in (Q, K, V))
     t = lambda x: None if x is None else torch.tensor(x, dtype=torch.float64)
-    out = _torch_forward(tq, tk, tv, t(Phi), t(Phi if Phi_v is None else Phi_v), [t(x) for x in S_l], [t(x) for x in B_l],
-                         thetas, t(Psi), 1.0 / np.sqrt(d))
+    # one leaf per layer for every decoder parameter, so that autograd gives the per-layer gradients
+    tS = [torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in S_l]
+    tB = [torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in B_l]
+    tth = [torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in thetas]
+    tPsi = None if Psi is None else torch.tensor(Psi, dtype=torch.float64, requires_grad=True)
+    out = _torch_forward(tq, tk, tv, t(Phi), t(Phi if Phi_v is None else Phi_v), tS, tB, tth, tPsi, 1.0 / np.sqrt(d))
     # the torch forward is the oracle's forward
     ref_out = orc.csat_forward_head(Q, K, V, Phi, T=T, lam=lam, Psi=Psi, weights=weights, Phi_v_h=Phi_v)
     assert np.allclose(out.detach().numpy(), ref_out, rtol=0, atol=1e-12)
     (out * t(G)).sum().backward()
     for name, g, ref in zip("QKV", got, (tq.grad, tk.grad, tv.grad)):
         assert np.allclose(g, ref.numpy(), rtol=1e-10, atol=1e-12), (name, seed, T)
+    # gradients with respect to the decoder's parameters, layer by layer
+    assert st["dS"].shape == (T, d, d) and st["dB"].shape == (T, d, d) and st["dtheta"].shape == (T,)
+    for l in range(T):
+        gS = tS[l].grad.numpy() if tS[l].grad is not None else np.zeros((d, d))     # layer 0 multiplies alpha^0 = 0
+        assert np.allclose(st["dS"][l], gS, rtol=1e-10, atol=1e-12), ("dS", seed, l)
+        assert np.allclose(st["dB"][l], tB[l].grad.numpy(), rtol=1e-10, atol=1e-12), ("dB", seed, l)
+        assert np.allclose(st["dtheta"][l], tth[l].grad.numpy(), rtol=1e-10, atol=1e-12), ("dtheta", seed, l)
+    if Psi is not None and T > 0:
+        assert np.allclose(st["dPsi"], tPsi.grad.numpy(), rtol=1e-10, atol=1e-12), ("dPsi", seed)
+    if T > 0:
+        assert st["masks"].shape == (T, nq, d) and st["xs"].shape == (T, nq, d)
+        assert np.array_equal(st["masks"], np.abs(st["xs"]) > np.asarray(thetas)[:, None, None])
     return Q, K, V, Phi, Phi_v, Psi, G, lam, weights, got, st
+
+
+def test_backward_with_supplied_shrinkage_decisions():
+    """masks= replaces the oracle's own decisions |x_t| > theta_t.  Pinned by autograd through a forward whose
+    layers compute masks[t] o (x - theta sign(x)) with RANDOM masks (so that layer, row and column indices all
+    matter); the gradients with respect to Q, K, V depend on the masks and on constant matrices only, so they must
+    agree exactly.  The oracle's own masks passed back in change nothing."""
+    import torch
+    for seed, T, with_psi, separate, untied in [(91, 3, False, False, False), (92, 4, True, True, True)]:
+        Q, K, V, Phi, Phi_v, Psi, G, lam, weights, got, st = _backward_case(seed, T, with_psi, separate, untied)
+        kw = dict(T=T, lam=lam, Psi=Psi, weights=weights, Phi_v_h=Phi_v)
+        same = orc.csat_backward_head(Q, K, V, Phi, G, masks=st["masks"], **kw)
+        for a, b in zip(got, same):
+            assert np.array_equal(a, b)
+        r = np.random.default_rng(seed + 100)
+        forced = r.random(st["masks"].shape) < 0.6
+        assert (forced != st["masks"]).any() and len({forced[l].tobytes() for l in range(T)}) == T
+        d = Q.shape[1]
+        if weights is None:
+            Dm = orc.default_decoder_matrix(Phi if Phi_v is None else Phi_v, d)
+            S_dec, B_dec, theta, _ = orc.decoder_setup(Dm if Psi is None else Dm @ Psi, lam)
+            S_l, B_l, thetas = [S_dec] * T, [B_dec] * T, [float(theta)] * T
+        else:
+            S_l, B_l, thetas = list(weights[0]), list(weights[1]), list(weights[2])
+        t = lambda x: None if x is None else torch.tensor(x, dtype=torch.float64)
+        tq, tk, tv = (torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in (Q, K, V))
+        out = _torch_forward(tq, tk, tv, t(Phi), t(Phi if Phi_v is None else Phi_v), [t(x) for x in S_l],
+                             [t(x) for x in B_l], thetas, t(Psi), 1.0 / np.sqrt(d),
+                             forced_masks=torch.tensor(forced, dtype=torch.float64))
+        (out * t(G)).sum().backward()
+        with_forced = orc.csat_backward_head(Q, K, V, Phi, G, masks=forced, **kw)
+        for name, g, ref in zip("QKV", with_forced, (tq.grad, tk.grad, tv.grad)):
+            assert np.allclose(g, ref.numpy(), rtol=1e-10, atol=1e-12), (name, seed)
+        # whole-batch wrapper hands every (batch, head) its own masks
+        Qb, Kb, Vb, Gb = (np.stack([x, x[::-1]])[None] for x in (Q, K, V, G))          # B = 1, H = 2
+        Phib = np.stack([Phi, Phi])
+        wb = None if weights is None else (np.stack([weights[0]] * 2, axis=1), np.stack([weights[1]] * 2, axis=1),
+                                           [[th, th] for th in weights[2]])
+        mb = np.stack([forced, st["masks"][:, ::-1]])[None]
+        full = orc.csat_backward(Qb, Kb, Vb, Phib, Gb, T=T, lam=lam, Psi=Psi, weights=wb,
+                                 Phi_V=None if Phi_v is None else np.stack([Phi_v, Phi_v]), masks=mb)
+        for x, y in zip(full, with_forced):
+            assert np.array_equal(x[0, 0], y)
 
 
 def test_backward_matches_autograd():

@@ -5,7 +5,8 @@ take cudaMalloc's implicit synchronisation, processes with a fixed memory budget
 csat_create/csat_forward, whose K~|V~ workspace is allocated.  The entry point keeps that scratch in a
 fixed array inside the library.  This test calls it through the C-ABI twice in a row (the array is shared
 and keeps the previous call's contents, so the second call must not be disturbed by the first) and checks
-each result against csat_forward with recovery disabled on the same inputs and the same Phi.
+each result against csat_forward with recovery disabled on the same inputs and the same Phi, and (so that the
+agreement of two CUDA paths is not the only evidence) against the float64 oracle's compressed attention.
 
 The file name sorts last so that a run that stops at the first failure has already run every other test.
 """
@@ -13,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import csat_oracle as orc
 from paper_2507_02957_b200 import binding, workloads as wl
 from gpu_util import TOL, device_inputs, make_ctx, rel_err, to_np
 
@@ -35,11 +37,13 @@ def test_two_calls_in_a_row_match_the_allocating_entry_point():
         ctx.close()
         out = torch.full_like(Q, float("nan"))
         binding.csat_attend_noalloc(Q, K, V, phi, out)
-        got.append((w, out))
+        got.append((w, out, inp, to_np(phi)))
     torch.cuda.synchronize()
-    for (w, out), ref in zip(got, expected):
+    for (w, out, inp, phi), ref in zip(got, expected):
         assert torch.isfinite(out).all()
         assert rel_err(to_np(out), to_np(ref)) <= TOL[w.dtype], w.name
+        oracle = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=0, lam=0.0)
+        assert rel_err(to_np(out), oracle) <= TOL[w.dtype], w.name
 
 
 def test_sizes_beyond_the_built_in_scratch_are_refused():
