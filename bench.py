@@ -54,6 +54,47 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+FFMA_LANES_PER_SM, SMS = 128, 148
+
+
+def fp32_ffma_peak_tflops(peaks: dict) -> float:
+    """Peak of the plain-ALU (FFMA) path, from the unit counts: SMs x fp32 lanes x 2 flop x the SM clock."""
+    return SMS * FFMA_LANES_PER_SM * 2 * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+
+
+def choose_tensor_peak(peaks: dict, region_ms: float, clocks: dict | None) -> tuple[str, float]:
+    """Burst or sustained bf16 peak, whichever matches how the kernel was timed: the burst figure for a short timed
+    region at full clocks with no power cap, the sustained one for a long region or one that ran under the cap."""
+    burst = float(peaks["bf16_tflops"])
+    sustained = float(peaks.get("bf16_tflops_sustained") or burst)
+    capped = bool(clocks) and "sw_power_cap" in (clocks.get("reasons") or [])
+    slow = bool(clocks) and clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] < 0.95 * clocks["sm_max_mhz"]
+    if region_ms > 500.0 or capped or slow:
+        return "sustained", sustained
+    return "burst", burst
+
+
+def roofline_fractions(w: wl.Workload, ms: float, flop: float, peaks: dict) -> dict:
+    """Achieved throughput of one whole forward against both rooflines (tensor or ALU, and HBM)."""
+    es = 4 if w.dtype == "fp32" else 2
+    bytes_alg = input_bytes(w) + w.H * w.m * w.n * es
+    t = ms * 1e-3
+    hbm = float(peaks["hbm_gbs"])
+    out = {"hbm_gbs": bytes_alg / t / 1e9, "frac_hbm": bytes_alg / t / 1e9 / hbm}
+    if w.dtype == "fp32":
+        pk = fp32_ffma_peak_tflops(peaks)
+        out.update(bound="alu", frac_alu_peak=flop / t / 1e12 / pk, peak_tflops=pk)
+        t_roof = max(flop / (pk * 1e12), bytes_alg / (hbm * 1e9))
+    else:
+        burst, sus = float(peaks["bf16_tflops"]), float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
+        out.update(bound="tensor", frac_burst=flop / t / 1e12 / burst, frac_sustained=flop / t / 1e12 / sus,
+                   frac_nominal_2250=flop / t / 1e12 / 2250.0)
+        t_roof = max(flop / (burst * 1e12), bytes_alg / (hbm * 1e9))
+    out["roofline_us"] = t_roof * 1e6            # the slower of the two limits (burst peak, measured HBM)
+    out["frac_of_roofline"] = t_roof / t
+    return out
+
+
 def workload_config(w: wl.Workload, n_gpus: int) -> dict:
     return {"workload": w.name, "B_per_gpu": w.B, "H": w.H, "n": w.n, "n_q": w.n_q, "d": w.d, "m": w.m,
             "T": w.T, "lambda": w.lam, "storage": w.dtype, "parallelism": f"batch-sharded x{n_gpus}",
@@ -220,7 +261,8 @@ def kernel_flops(w: wl.Workload) -> dict:
     return {"compress": f["compress"], "attend_recover": f["attend"] + f["recover"], "decoder_setup": 0}
 
 
-def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3, untied: bool = False) -> dict:
+def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3, untied: bool = False, peaks: dict | None = None,
+               device_index: int = 0) -> dict:
     """Per-iteration CUDA-event timing with an L2 flush between iterations (workloads that fit in L2).
     untied: random LISTA weights with one S_t, B_t per layer instead of the ISTA-derived decoder."""
     import torch
@@ -239,7 +281,10 @@ def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3, untied: bool = 
     for _ in range(warmup):
         ctx.forward(dev["Q"], dev["K"], dev["V"], out)
     times = []
-    for _ in range(iters):
+    # at least `iters` iterations and long enough (0.25 s) for the clock sampler to see the GPU under this load
+    sampler = ClockSampler(device_index) if peaks is not None else None
+    t_start = time.perf_counter()
+    while len(times) < iters or (sampler is not None and time.perf_counter() - t_start < 0.25 and len(times) < 2000):
         flush.zero_()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -247,13 +292,18 @@ def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3, untied: bool = 
         e1.record()
         e1.synchronize()
         times.append(e0.elapsed_time(e1))
+    clocks = sampler.stop() if sampler is not None else None
     ctx.close()
     ms = float(np.median(times))
     f = wl.flops(w)["total"]
     if untied:
         f += 2 * w.n_q * w.d * w.d * (w.T - 1) * w.B * w.H      # z B_t in every layer after the first
-    return {"ms": ms, "tokens_per_s": w.query_tokens / (ms * 1e-3), "tflops": f / (ms * 1e-3) / 1e12,
-            "gflop": f / 1e9}
+    res = {"ms": ms, "iters": len(times), "tokens_per_s": w.query_tokens / (ms * 1e-3), "tflops": f / (ms * 1e-3) / 1e12,
+           "gflop": f / 1e9}
+    if peaks is not None:
+        res["roofline"] = roofline_fractions(w, ms, f, peaks)
+        res["clocks"] = clocks
+    return res
 
 
 def time_projection(w: wl.Workload, iters: int = 10, warmup: int = 3) -> dict:
@@ -371,13 +421,27 @@ def run_csat(args, w: wl.Workload) -> dict:
         tf = kf.get(name, 0) / (avg * 1e-3) / 1e12
         kernels.append({"kernel": name, "launch_groups": cnt, "avg_ms": avg, "share": ms / tot_ms, "tflops": tf})
     top = kernels[0]
-    peak_tf = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
+    burst_tf = float(peaks["bf16_tflops"])
+    sustained_tf = float(peaks.get("bf16_tflops_sustained") or burst_tf)
     if w.dtype == "fp32":
-        peak_tf = peak_tf / 32.0   # FFMA path: no fp32 tensor-core kernel; fp32 FMA peak taken as 1/32 of the bf16 tensor peak
-    roofline = {"kernel": top["kernel"], "bound": "tensor", "achieved": top["tflops"], "peak": peak_tf,
-                "unit": "TFLOP/s", "frac": top["tflops"] / peak_tf, "peak_source": f"{peak_kind} bf16 sustained",
-                "traffic": NCU_TRAFFIC_BYTES.get((top["kernel"], w.name)),
-                "flops_per_launch": kf.get(top["kernel"], 0), "avg_launch_ms": top["avg_ms"]}
+        # FFMA path (no fp32 tensor-core kernel): plain ALU bound, peak from the unit counts and the clock
+        peak_tf = fp32_ffma_peak_tflops(peaks)
+        roofline = {"kernel": top["kernel"], "bound": "alu", "achieved": top["tflops"], "peak": peak_tf,
+                    "unit": "TFLOP/s", "frac": top["tflops"] / peak_tf,
+                    "peak_source": "148 SMs x 128 fp32 lanes x 2 flop x max SM clock", "traffic": None,
+                    "flops_per_launch": kf.get(top["kernel"], 0), "avg_launch_ms": top["avg_ms"]}
+    else:
+        which, peak_tf = choose_tensor_peak(peaks, ms_total, clocks)
+        roofline = {"kernel": top["kernel"], "bound": "tensor", "achieved": top["tflops"], "peak": peak_tf,
+                    "unit": "TFLOP/s", "frac": top["tflops"] / peak_tf,
+                    "peak_source": f"{peak_kind} bf16 {which} (timed region {ms_total:.0f} ms)",
+                    "frac_burst": top["tflops"] / burst_tf, "frac_sustained": top["tflops"] / sustained_tf,
+                    "frac_nominal_2250": top["tflops"] / 2250.0,
+                    "traffic": NCU_TRAFFIC_BYTES.get((top["kernel"], w.name)),
+                    "flops_per_launch": kf.get(top["kernel"], 0), "avg_launch_ms": top["avg_ms"]}
+        for k in kernels:
+            k["frac_burst"] = k["tflops"] / burst_tf
+            k["frac_sustained"] = k["tflops"] / sustained_tf
 
     # end to end through the host-buffer entry point (copies inside the timed region)
     oh = torch.empty_like(host["Q"]).pin_memory()
@@ -399,7 +463,8 @@ def run_csat(args, w: wl.Workload) -> dict:
         "warmup": W, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic", "config": workload_config(w, world),
         "tflops": fl["total"] * world / (ms_step * 1e-3) / 1e12,
-        "frac_of_bf16_peak": {"measured_sustained": fl["total"] / (ms_step * 1e-3) / 1e12 / peak_tf,
+        "frac_of_bf16_peak": {"measured_burst": fl["total"] / (ms_step * 1e-3) / 1e12 / burst_tf,
+                              "measured_sustained": fl["total"] / (ms_step * 1e-3) / 1e12 / sustained_tf,
                               "nominal_2250": fl["total"] / (ms_step * 1e-3) / 1e12 / 2250.0},
         "hbm_gbs_algorithmic": (input_bytes(w) + w.H * w.m * w.n * (4 if w.dtype == "fp32" else 2))
         / (ms_step * 1e-3) / 1e9,
@@ -413,14 +478,15 @@ def run_csat(args, w: wl.Workload) -> dict:
         if not args.no_extra:
             extra = {}
             for key in ("c1", "c2", "c3", "c4"):
-                extra[wl.CONFIGS[key].name] = time_small(wl.CONFIGS[key])
-            for n in (2048, 4096, 8192):
-                extra[f"c5_sweep_n{n}"] = time_small(wl.sweep_config(n))
+                extra[wl.CONFIGS[key].name] = time_small(wl.CONFIGS[key], peaks=peaks, device_index=local)
+            for n in (2048, 4096, 8192, 16384):
+                extra[f"c5_sweep_n{n}"] = time_small(wl.sweep_config(n), peaks=peaks, device_index=local)
             if w.T > 1 and w.dtype == "bf16":
                 extra[f"{w.name}_untied_layers"] = time_small(w, untied=True)
             if w.dtype == "bf16" and w.n == w.n_q:
                 extra[f"{w.name}_qkv_projection"] = time_projection(w)
-            extra["backward"] = {wl.CONFIGS[k].name: time_backward(wl.CONFIGS[k]) for k in ("c1", "c2", "c3", "c4")}
+            extra["backward"] = {wl.CONFIGS[k].name: time_backward(wl.CONFIGS[k], iters=1 if k == "c5" else 2)
+                                 for k in ("c1", "c2", "c3", "c4", "c5")}
             result["other_workloads"] = extra
         if not args.no_cpu_baseline:
             inp = {k: host[k].float().numpy() for k in "QKV"}

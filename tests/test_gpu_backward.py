@@ -8,7 +8,13 @@ parts, as for any result where floating point takes a discrete decision:
      (the parity tolerance times max |x_t|), and such entries must be few;
   2. the gradients: the oracle differentiates with the library's decisions (its forward values stay its own) and
      every gradient is compared element by element, max |gpu - oracle| / max |oracle| <= the forward's tolerance
-     (2e-2 with bf16 storage; float32: 2e-5, measured ~1e-6)."""
+     (2e-2 with bf16 storage; float32: 2e-5, measured ~1e-6).
+The output gradient G is random.  dK~ and dV~ are sums over the query rows, so with an unlucky draw the column sums
+of dZ cancel far below their typical 1/sqrt(n_q) of the sum of magnitudes; the gradient is then a difference of
+nearly equal terms and magnifies the bf16 rounding of its operands (one of ten draws did for the sparse case: 1 %
+cancellation, 4 % error from rounding P alone in float64 emulation, 0.3-0.9 % for the other nine).  The test
+asserts, from the oracle alone, that the draw's cancellation is typical, so that the bar measures the kernel and
+not the draw."""
 import numpy as np
 import pytest
 import torch
@@ -32,6 +38,7 @@ CASES = {
 
 
 BWD_TOL = {"bf16": 2e-2, "fp32": 2e-5}
+G_SEED = 103
 
 
 @pytest.mark.parametrize("name", sorted(CASES))
@@ -63,7 +70,7 @@ def test_backward_matches_oracle(name, variant):
     if variant == "psi_separate_untied":
         kw.update(Phi_V=phi[H:])
         phi = phi[:H]
-    G = wl.round_to_storage(r.standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    G = wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
     got = ctx.backward(Q, K, V, to_dev(G, w.dtype))
     assert binding.csat_last_launch_count(ctx.h) >= 4
     tol = BWD_TOL[w.dtype]
@@ -82,6 +89,10 @@ def test_backward_matches_oracle(name, variant):
             st1 = []
             orc.csat_forward(inp["Q"][:1], inp["K"][:1], inp["V"][:1], phi, T=1, lam=w.lam, stages=st1)
             th = np.asarray([s["theta"] for s in st1])[None, :, None, None, None]
+        for st in stages:                     # the draw of G is not a degenerate one (see the file header)
+            col_abs = np.abs(st["dZ"]).sum(axis=0).max()
+            if col_abs > 0:
+                assert np.abs(st["dZ"].sum(axis=0)).max() / col_abs >= 0.25 / np.sqrt(w.n_q), (name, variant)
         differ = masks != own
         assert differ.mean() <= (2e-2 if w.dtype == "bf16" else 1e-4), (name, variant, differ.mean())
         bar = TOL[w.dtype] * np.abs(xs).max(axis=(3, 4), keepdims=True)               # per (b, h, layer)
