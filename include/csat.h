@@ -222,6 +222,33 @@ int csat_project_qkv(csat_ctx* ctx, const void* Xq, const void* Xkv, const void*
 int csat_forward(csat_ctx* ctx, const void* Q, const void* K, const void* V, void* out, void* stream);
 
 /*
+ * Token-sharded forward -- paper: "Efficiency and Scaling" (sequences beyond one device) and the compression
+ * equation, whose sum over the n tokens splits over shards: Phi K = sum over shards s of Phi[:, shard s] K[shard s].
+ * When the keys and values of one (batch, head) pair are spread over several GPUs, every GPU
+ *   1. csat_compress_partial: multiplies its token shard by the matching columns of Phi (every GPU generates the
+ *      same Phi from the seed) and gets the float32 partial sums for K~|V~;
+ *   2. exchanges the partials with the other GPUs (the caller's collective, e.g. an all-gather: the library takes no
+ *      communicator) and
+ *   3. csat_reduce_partials: adds them in the order given -- the same order on every GPU, so all hold bit-identical
+ *      K~|V~ -- into the context's workspace, rounded once to the context dtype;
+ *   4. csat_attend: attention and recovery for its own queries (the context's CSAT_NQ = the number of local
+ *      queries); no further exchange.
+ *
+ *   K_shard, V_shard [B, H, n_len, d]   tokens n0 .. n0 + n_len - 1 of the sequence (context dtype, device)
+ *   partial_out      [B, H, m, 2d]      float32, device: row r = K~_r | V~_r partial sums
+ *   partials         [count][B, H, m, 2d] float32, device, contiguous: the shards' partials in the agreed order
+ *   Q, out           [B, H, n_q, d]     as for csat_forward
+ * n0 must be a multiple of 8 (shard boundaries at multiples of 64 keep every load aligned to a 128-byte line) and
+ * [n0, n0 + n_len) inside [0, n): else CSAT_ERR_SHAPE.  Launch-only, no allocation.  csat_attend needs a workspace
+ * filled by csat_reduce_partials or csat_forward (CSAT_ERR_STATE otherwise).  One shard covering all n tokens
+ * followed by csat_reduce_partials(count = 1) and csat_attend equals csat_forward up to the rounding of the sums.
+ */
+int csat_compress_partial(csat_ctx* ctx, const void* K_shard, const void* V_shard, int64_t n0, int64_t n_len,
+                          float* partial_out, void* stream);
+int csat_reduce_partials(csat_ctx* ctx, const float* partials, int count, void* stream);
+int csat_attend(csat_ctx* ctx, const void* Q, void* out, void* stream);
+
+/*
  * csat_forward_host -- same computation with HOST buffers (same layouts and dtype; pinned memory gives
  * asynchronous copies).  Copies Q, K, V to staging buffers the context owns (allocated by the first call, so
  * that call also allocates), computes, copies out back and returns once `stream` has reached the end of all of

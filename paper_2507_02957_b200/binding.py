@@ -42,6 +42,9 @@ SIGNATURES = {
     "csat_set_lista_layer_weights": (_int, [_vp, _vp, _vp, _vp, _int, _vp]),
     "csat_project_qkv": (_int, [_vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _vp]),
     "csat_forward": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "csat_compress_partial": (_int, [_vp, _vp, _vp, _i64, _i64, _vp, _vp]),
+    "csat_reduce_partials": (_int, [_vp, _vp, _int, _vp]),
+    "csat_attend": (_int, [_vp, _vp, _vp, _vp]),
     "csat_backward": (_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_forward_host": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
@@ -171,6 +174,19 @@ def csat_project_qkv(h, Xq, Xkv, W, d_model, Q, K, V, stream=None):
 
 def csat_forward(h, Q, K, V, out, stream=None):
     _check(h, load().csat_forward(h, _ptr(Q), _ptr(K), _ptr(V), _ptr(out), _stream(stream)))
+
+
+def csat_compress_partial(h, K_shard, V_shard, n0, n_len, partial_out, stream=None):
+    _check(h, load().csat_compress_partial(h, _ptr(K_shard), _ptr(V_shard), int(n0), int(n_len), _ptr(partial_out),
+                                           _stream(stream)))
+
+
+def csat_reduce_partials(h, partials, count, stream=None):
+    _check(h, load().csat_reduce_partials(h, _ptr(partials), int(count), _stream(stream)))
+
+
+def csat_attend(h, Q, out, stream=None):
+    _check(h, load().csat_attend(h, _ptr(Q), _ptr(out), _stream(stream)))
 
 
 def csat_backward(h, Q, K, V, dOut, dQ, dK, dV, stream=None):
@@ -350,6 +366,30 @@ class Csat:
         assert S.shape == (self.H, self.d, self.d) and Bm.shape == S.shape and S.dtype == self.torch_dtype == Bm.dtype
         theta = theta.reshape(-1, self.H).to(torch.float32).contiguous()
         csat_set_lista_weights(self.h, S.contiguous(), Bm.contiguous(), theta, theta.shape[0])
+
+    def compress_partial(self, K_shard, V_shard, n0):
+        """float32 partial sums [B,H,m,2d] of K~|V~ for the token shard that starts at token n0."""
+        assert K_shard.shape == V_shard.shape and K_shard.shape[:2] == (self.B, self.H) and K_shard.shape[3] == self.d
+        out = self._new(self.B, self.H, self.m, 2 * self.d, dtype=torch.float32)
+        csat_compress_partial(self.h, K_shard, V_shard, n0, K_shard.shape[2], out)
+        return out
+
+    def reduce_partials(self, partials):
+        """partials [count,B,H,m,2d] float32, summed in the order given into the workspace."""
+        assert partials.dtype == torch.float32 and partials.shape[1:] == (self.B, self.H, self.m, 2 * self.d)
+        csat_reduce_partials(self.h, partials.contiguous(), partials.shape[0])
+
+    def attend(self, Q, out=None):
+        """Attention and recovery for Q [B,H,n_q,d] against the K~|V~ in the workspace."""
+        assert Q.shape == (self.B, self.H, self.n_q, self.d) and Q.dtype == self.torch_dtype and Q.is_cuda
+        if out is None:
+            out = self._new(self.B, self.H, self.n_q, self.d)
+        csat_attend(self.h, Q, out)
+        return out
+
+    def set_n_q(self, n_q):
+        csat_set_i64(self.h, CSAT_NQ, n_q)
+        self.n_q = n_q
 
     def backward(self, Q, K, V, dOut):
         """Gradients of forward(Q, K, V) with respect to Q, K, V for the output gradient dOut."""

@@ -11,6 +11,9 @@
 //   warps 2-5: epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), round to bf16, store
 //              row r of the tile as K~_r | V~_r into the workspace.
 // Rows of Phi beyond m and tokens beyond n are zero-filled by TMA (and Phi's padded columns hold zeros).
+// Token-sharded use: the same kernel over a token range [phi_j0, phi_j0 + n) of Phi against a shard of K, V that
+// holds only those n tokens; the epilogue then writes the float32 partial sums to `partial` instead of the
+// workspace (they are summed over the shards, in a fixed order, before anything reads them).
 #include "csat_internal.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -46,7 +49,7 @@ template <int D, bool SEP, int BG>
 __global__ void __launch_bounds__(kThreads, 1)
 compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, __nv_bfloat16* __restrict__ kv, int m, int n, int H,
-                      int B, int bh0, int* status) {
+                      int B, int bh0, int* status, int phi_j0, float* __restrict__ partial) {
   using C = Cfg<D, SEP, BG>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -101,8 +104,8 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
         ok = mbar_wait(&empty[s], ((i / C::kStages) & 1) ^ 1, status, 101, cta_abort);
         if (!ok) break;
         mbar_arrive_expect_tx(&full[s], C::kStageBytes);
-        tma_load_3d(a_buf + s * C::kATiles * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, hphi);
-        if (SEP) tma_load_3d(a_buf + (s * C::kATiles + 1) * kABytes, &tmap_phi, &full[s], i * kChunk, mtile * kTileM, H + hphi);
+        tma_load_3d(a_buf + s * C::kATiles * kABytes, &tmap_phi, &full[s], phi_j0 + i * kChunk, mtile * kTileM, hphi);
+        if (SEP) tma_load_3d(a_buf + (s * C::kATiles + 1) * kABytes, &tmap_phi, &full[s], phi_j0 + i * kChunk, mtile * kTileM, H + hphi);
 #pragma unroll
         for (int g = 0; g < C::kBoxes; ++g) {
           const bool is_v = g >= C::kBoxes / 2;
@@ -152,7 +155,13 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
         tmem_wait_ld();
         // accumulator column c0: K half or V half, batch element e of the group, feature column
         const int half = c0 / (C::kN / 2), e = (c0 % (C::kN / 2)) / D, col = c0 % D;
-        if (row < m && b0 + e < B) {
+        if (row < m && b0 + e < B && partial != nullptr) {
+          float4* o = reinterpret_cast<float4*>(partial + ((int64_t)bh_of(e) * m + row) * (2 * D) + half * D + col);
+#pragma unroll
+          for (int v = 0; v < 8; ++v)
+            o[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                               __uint_as_float(r[4 * v + 3]));
+        } else if (row < m && b0 + e < B) {
           uint4* o = reinterpret_cast<uint4*>(kv + ((int64_t)bh_of(e) * m + row) * (2 * D) + half * D + col);
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
@@ -187,13 +196,16 @@ __global__ void wait_timeout_selftest_kernel(int* status, unsigned long long lim
   }
 }
 
+// n_len tokens of K, V (a shard that starts at token phi_j0 of the sequence, or the whole sequence); partial: float32
+// destination of a shard's sums, null = the workspace
 template <int D, bool SEP, int BG>
-cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
+cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int64_t phi_j0, int64_t n_len,
+                   float* partial) {
   using C = Cfg<D, SEP, BG>;
   const Params& p = c->p;
   CUtensorMap tk, tv;
-  const uint64_t kd[3] = {(uint64_t)D, (uint64_t)p.n, (uint64_t)(p.B * p.H)};
-  const uint64_t ks[2] = {(uint64_t)D * 2, (uint64_t)p.n * D * 2};
+  const uint64_t kd[3] = {(uint64_t)D, (uint64_t)n_len, (uint64_t)(p.B * p.H)};
+  const uint64_t ks[2] = {(uint64_t)D * 2, (uint64_t)n_len * D * 2};
   const uint32_t kb[3] = {64, (uint32_t)kChunk, 1};
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tk, K, kd, ks, kb)) != cudaSuccess) return e;
@@ -205,7 +217,8 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
   const int64_t Bl = c->bh_cnt ? 1 : p.B, Hl = c->bh_cnt ? c->bh_cnt : p.H;
   const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(((Bl + BG - 1) / BG) * Hl));
   compress_sm100_kernel<D, SEP, BG><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
-                                                                 (int)p.n, (int)p.H, (int)Bl, (int)c->bh0, c->status);
+                                                                 (int)n_len, (int)p.H, (int)Bl, (int)c->bh0, c->status,
+                                                                 (int)phi_j0, partial);
   return cudaGetLastError();
 }
 
@@ -224,13 +237,19 @@ cudaError_t make_phi_tmap(csat_ctx* c) {
   return make_tmap_bf16_3d(&c->tmap_phi, c->phi, d, st, b);
 }
 
-cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches) {
+cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches,
+                                  int64_t phi_j0, int64_t n_len, float* partial) {
   *launches += 1;
+  if (n_len <= 0) n_len = c->p.n;
   // d = 64: two batch elements per CTA where the batch has them (N = 256 MMAs)
   if (c->p.d == 64 && c->p.B >= 2 && c->bh_cnt == 0)
-    return c->p.separate_phi ? launch<64, true, 2>(c, K, V, s) : launch<64, false, 2>(c, K, V, s);
-  if (c->p.separate_phi) return c->p.d == 64 ? launch<64, true, 1>(c, K, V, s) : launch<128, true, 1>(c, K, V, s);
-  return c->p.d == 64 ? launch<64, false, 1>(c, K, V, s) : launch<128, false, 1>(c, K, V, s);
+    return c->p.separate_phi ? launch<64, true, 2>(c, K, V, s, phi_j0, n_len, partial)
+                             : launch<64, false, 2>(c, K, V, s, phi_j0, n_len, partial);
+  if (c->p.separate_phi)
+    return c->p.d == 64 ? launch<64, true, 1>(c, K, V, s, phi_j0, n_len, partial)
+                        : launch<128, true, 1>(c, K, V, s, phi_j0, n_len, partial);
+  return c->p.d == 64 ? launch<64, false, 1>(c, K, V, s, phi_j0, n_len, partial)
+                      : launch<128, false, 1>(c, K, V, s, phi_j0, n_len, partial);
 }
 
 }  // namespace csat

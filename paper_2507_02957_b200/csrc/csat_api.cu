@@ -594,6 +594,81 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   return CSAT_OK;
 }
 
+// ---- token-sharded use: one (batch, head) pair's keys and values spread over several GPUs ----------------------
+int csat_compress_partial(csat_ctx* c, const void* K_shard, const void* V_shard, int64_t n0, int64_t n_len,
+                          float* partial_out, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!K_shard || !V_shard || !partial_out) return fail(c, CSAT_ERR_INVALID_ARG, "csat_compress_partial: NULL pointer");
+  if (!aligned16(K_shard) || !aligned16(V_shard) || !aligned16(partial_out))
+    return fail(c, CSAT_ERR_INVALID_ARG, "csat_compress_partial: pointers must be 16-byte aligned");
+  const csat::Params& p = c->p;
+  if (n0 < 0 || n_len < 1 || n0 + n_len > p.n)
+    return fail(c, CSAT_ERR_SHAPE, "csat_compress_partial: the shard [n0, n0 + n_len) must lie inside [0, n)");
+  if (n0 % 8 != 0) return fail(c, CSAT_ERR_SHAPE, "csat_compress_partial: n0 must be a multiple of 8");
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  if (*(volatile int*)c->status != 0)
+    return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
+  NvtxRange range("csat_compress_partial");
+  cudaStream_t s = (cudaStream_t)stream;
+  int launches = 0;
+  const bool tc = c->tmap_phi_valid && c->force_simt != 1;
+  cudaError_t e = tc ? csat::launch_sm100_compress(c, K_shard, V_shard, s, &launches, n0, n_len, partial_out)
+                     : csat::launch_simt_compress(c, K_shard, V_shard, s, &launches, n0, n_len, partial_out);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_compress_partial launch");
+  c->last_launches = launches;
+  return CSAT_OK;
+}
+
+int csat_reduce_partials(csat_ctx* c, const float* partials, int count, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!partials || !aligned16(partials)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_reduce_partials: NULL or misaligned pointer");
+  if (count < 1 || count > 4096) return fail(c, CSAT_ERR_INVALID_ARG, "csat_reduce_partials: count must be in [1, 4096]");
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  int launches = 0;
+  cudaError_t e = csat::launch_reduce_partials(c, partials, count, (cudaStream_t)stream, &launches);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_reduce_partials launch");
+  c->have_forward = true;                 // the workspace now holds K~|V~
+  c->last_launches = launches;
+  return CSAT_OK;
+}
+
+int csat_attend(csat_ctx* c, const void* Q, void* out, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!Q || !out) return fail(c, CSAT_ERR_INVALID_ARG, "csat_attend: NULL tensor pointer");
+  if (!aligned16(Q) || !aligned16(out)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_attend: tensor pointers must be 16-byte aligned");
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
+  if (!c->have_forward)
+    return fail(c, CSAT_ERR_STATE, "csat_attend: the workspace holds no K~|V~ yet (csat_reduce_partials or csat_forward first)");
+  {
+    const csat::Params& p = c->p;
+    const size_t bq = (size_t)(p.B * p.H * p.nq * p.d) * csat::elt_size(p.dtype);
+    if (ranges_overlap(out, bq, Q, bq)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_attend: out overlaps Q");
+  }
+  std::string why;
+  if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
+  if (*(volatile int*)c->status != 0)
+    return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
+  if (c->p.T > 0 && c->w_S && (c->w_layers != 1 || c->w_untied) && c->w_layers != c->p.T)
+    return fail(c, CSAT_ERR_STATE, "the supplied LISTA weights are for a number of layers other than CSAT_T");
+  NvtxRange range("csat_attend");
+  cudaStream_t s = (cudaStream_t)stream;
+  int launches = 0;
+  if (c->p.T > 0) {
+    int rc = ensure_decoder(c, s, &launches);
+    if (rc != CSAT_OK) return rc;
+  }
+  const bool tc_attend = c->tmap_phi_valid && c->force_simt == 0;
+  cudaError_t e = tc_attend ? csat::launch_sm100_attend_recover(c, Q, out, s, &launches)
+                            : csat::launch_simt_attend_recover(c, Q, out, s, &launches);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_attend launch");
+  c->last_launches = launches;
+  return CSAT_OK;
+}
+
 int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, const void* dOut, void* dQ, void* dK,
                   void* dV, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;

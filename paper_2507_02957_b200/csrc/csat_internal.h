@@ -148,13 +148,19 @@ cudaError_t launch_phi_unpack(void* phi_dense, const void* phi_padded, const Par
 cudaError_t launch_decoder_setup(csat_ctx* c, cudaStream_t s, int* launches);
 
 // simt_forward.cu : plain FFMA path (fp32 accumulate), both storage types
-cudaError_t launch_simt_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches);
+// (phi_j0, n_len, partial): token-sharded use, see compress_sm100.cu; defaults = the whole sequence into the workspace
+cudaError_t launch_simt_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches,
+                                 int64_t phi_j0 = 0, int64_t n_len = 0, float* partial = nullptr);
+// workspace := sum over r < R of partials[r] (float32 [B,H,m,2d] each), added in the order r = 0, 1, ..., rounded
+// once to the context's storage type
+cudaError_t launch_reduce_partials(csat_ctx* c, const float* partials, int R, cudaStream_t s, int* launches);
 cudaError_t launch_simt_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
 
 // compress_sm100.cu : tcgen05 / TMEM / TMA compression (bf16, d in {64, 128})
 cudaError_t make_phi_tmap(csat_ctx* c);
 cudaError_t launch_wait_timeout_selftest(csat_ctx* c, unsigned long long limit_ns, cudaStream_t s);
-cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches);
+cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches,
+                                  int64_t phi_j0 = 0, int64_t n_len = 0, float* partial = nullptr);
 
 // attend_recover_sm100.cu : tcgen05 compressed attention + recovery (bf16, d in {64, 128})
 cudaError_t make_attend_tmaps(csat_ctx* c);

@@ -61,6 +61,71 @@ __global__ void phi_gen_kernel(T* __restrict__ phi, int64_t total, int64_t n, in
   }
 }
 
+// bf16 storage, n % 8 == 0: the same Philox stream and the same Box-Muller pairing, with arithmetic sized for a
+// 16-bit result (the stored value has 8 bits of mantissa; everything below is accurate to ~1e-6 relative, so the
+// rounded value differs from the exactly computed one only where that lies within 1e-6 of a rounding boundary):
+//   radius  sqrt(-2 ln u / m) = sqrt.approx(c log2 u), c = -2 ln 2 / m (the 1/sqrt(m) scale folded in);
+//   angle   x = 2 u in (0, 2) half-turns: k = nearest multiple of 1/2, f = x - k / 2 in [-1/4, 1/4] (exact),
+//           sin(pi f), cos(pi f) by odd / even polynomials in y = pi f (relative accuracy also next to the zeros,
+//           where the value is f itself), quadrant k selects and signs them.
+// A thread produces eight consecutive elements (two Philox blocks) and writes them with one 16-byte store; rows
+// are walked by stepping (one 64-bit division per thread, outside the loop).
+// Cost: Philox4x32-10 alone is 20 wide multiplies, 20 three-input xors and 20 key additions per four elements, so
+// the kernel is bound by integer arithmetic, not by the 2 bytes it writes per element.
+__device__ __forceinline__ void box_muller_bf16(uint32_t ua, uint32_t ub, float c, float& g0, float& g1) {
+  float r;
+  {
+    const float r2 = c * __log2f(uniform23(ua));
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(r2));
+  }
+  const float x = 2.0f * uniform23(ub);
+  const float kf = rintf(2.0f * x);
+  const float y = 3.14159265358979f * fmaf(kf, -0.5f, x);
+  const float y2 = y * y;
+  float sn = fmaf(y2, -1.9841270e-4f, 8.3333333e-3f);
+  sn = fmaf(sn, y2, -1.6666667e-1f);
+  sn = fmaf(sn * y2, y, y);
+  float cs = fmaf(y2, 2.4801587e-5f, -1.3888889e-3f);
+  cs = fmaf(cs, y2, 4.1666667e-2f);
+  cs = fmaf(cs, y2, -0.5f);
+  cs = fmaf(cs, y2, 1.0f);
+  const int k = (int)kf;
+  const float sa = (k & 1) ? cs : sn, ca = (k & 1) ? sn : cs;
+  // quadrant 0: (s, c); 1: (c, -s); 2: (-s, -c); 3: (-c, s)
+  const float s_out = (k & 2) ? -sa : sa;
+  const float c_out = ((k + 1) & 2) ? -ca : ca;
+  g0 = r * c_out;
+  g1 = r * s_out;
+}
+
+__global__ void phi_gen_bf16_vec_kernel(__nv_bfloat16* __restrict__ phi, int64_t total, int64_t n, int64_t n_pad, float c,
+                                        uint32_t k0, uint32_t k1) {
+  const int64_t noct = total >> 3;                       // total % 8 == 0
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int64_t o = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (o >= noct) return;
+  int64_t row = (o << 3) / n, j = (o << 3) - row * n;
+  const int64_t drow = (stride << 3) / n, dj = (stride << 3) - drow * n;
+  for (; o < noct; o += stride) {
+    uint32_t w[4];
+#pragma unroll
+    for (int b = 0; b < 2; ++b) {
+      const int64_t q = 2 * o + b;
+      const U4 u = philox4x32_10(U4{(uint32_t)q, (uint32_t)(q >> 32), 0u, 0u}, k0, k1);
+      float g0, g1, g2, g3;
+      box_muller_bf16(u.x, u.y, c, g0, g1);
+      box_muller_bf16(u.z, u.w, c, g2, g3);
+      __nv_bfloat162 p0 = __floats2bfloat162_rn(g0, g1), p1 = __floats2bfloat162_rn(g2, g3);
+      w[2 * b] = *reinterpret_cast<uint32_t*>(&p0);
+      w[2 * b + 1] = *reinterpret_cast<uint32_t*>(&p1);
+    }
+    *reinterpret_cast<uint4*>(phi + row * n_pad + j) = make_uint4(w[0], w[1], w[2], w[3]);
+    row += drow;
+    j += dj;
+    if (j >= n) { j -= n; ++row; }
+  }
+}
+
 // Rademacher ensemble: one sign bit per element of the unpadded index space, 128 elements per Philox block,
 // counter (q, 0, 1, 0) as (low, high, third, fourth) words.  A warp takes 32 consecutive blocks (4096
 // elements): lane l computes block l, and in step s the word (s % 4) of lane s / 4 is broadcast so that lane l
@@ -225,6 +290,12 @@ cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s) {
       else
         phi_rademacher_kernel<__nv_bfloat16><<<rg, rb, 0, s>>>((__nv_bfloat16*)phi, total, p.n, p.n_pad, inv, k0, k1);
     }
+    return cudaGetLastError();
+  }
+  if (p.dtype == CSAT_DTYPE_BF16 && p.n % 8 == 0) {
+    const int block = 256, grid = grid_for(total / 8, block);
+    const float c = (float)(-2.0 * 0.6931471805599453 / (double)p.m);
+    phi_gen_bf16_vec_kernel<<<grid, block, 0, s>>>((__nv_bfloat16*)phi, total, p.n, p.n_pad, c, k0, k1);
     return cudaGetLastError();
   }
   const int block = 256, grid = grid_for((total + 3) / 4, block);

@@ -27,10 +27,13 @@ template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16* p,
 // ---------------------------------------------------------------------------------------------
 constexpr int kCmpRows = 32, kCmpChunk = 16;
 
-template <typename T, int KC>   // KC = ceil(2d / 32) column slots per lane
-__global__ void __launch_bounds__(256) compress_kernel(T* __restrict__ kv, const T* __restrict__ phi,
+// Token-sharded use: K, V hold the n tokens [phi_j0, phi_j0 + n) of the sequence and the sums go out as float32
+// partials (TO = float) that are added over the shards before anything reads them.
+template <typename T, typename TO, int KC>   // KC = ceil(2d / 32) column slots per lane
+__global__ void __launch_bounds__(256) compress_kernel(TO* __restrict__ kv, const T* __restrict__ phi,
                                                        const T* __restrict__ K, const T* __restrict__ V, int64_t n,
-                                                       int64_t n_pad, int64_t m, int d, int H, int phi_v_head0) {
+                                                       int64_t n_pad, int64_t m, int d, int H, int phi_v_head0,
+                                                       int64_t phi_j0) {
   // phi_v_head0: index of the first Phi_V matrix in phi (0 when Phi_V = Phi_K, H when they are separate)
   extern __shared__ float smem[];
   float* phis = smem;                              // [2][32][17]: Phi_K tile, Phi_V tile
@@ -54,8 +57,9 @@ __global__ void __launch_bounds__(256) compress_kernel(T* __restrict__ kv, const
     for (int i = threadIdx.x; i < kCmpRows * kCmpChunk; i += 256) {
       const int rr = i / kCmpChunk, jj = i % kCmpChunk;
       const int64_t r = r0 + rr;
-      phis[rr * (kCmpChunk + 1) + jj] = (r < m) ? ldf(Ph, r * n_pad + j0 + jj) : 0.f;   // padded columns hold 0
-      phiv[rr * (kCmpChunk + 1) + jj] = (r < m) ? ldf(Pv, r * n_pad + j0 + jj) : 0.f;
+      const bool in = r < m && j0 + jj < n;              // a shard's last chunk must not reach into the next shard
+      phis[rr * (kCmpChunk + 1) + jj] = in ? ldf(Ph, r * n_pad + phi_j0 + j0 + jj) : 0.f;
+      phiv[rr * (kCmpChunk + 1) + jj] = in ? ldf(Pv, r * n_pad + phi_j0 + j0 + jj) : 0.f;
     }
     for (int i = threadIdx.x; i < kCmpChunk * d2; i += 256) {
       const int jj = i / d2, c = i % d2;
@@ -83,7 +87,7 @@ __global__ void __launch_bounds__(256) compress_kernel(T* __restrict__ kv, const
     }
     __syncthreads();
   }
-  T* dst = kv + (int64_t)bh * m * d2;
+  TO* dst = kv + (int64_t)bh * m * d2;
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const int64_t r = r0 + ty * 4 + i;
@@ -93,6 +97,20 @@ __global__ void __launch_bounds__(256) compress_kernel(T* __restrict__ kv, const
       const int c = tx + 32 * k;
       if (c < d2) stf(dst, r * d2 + c, acc[i][k]);
     }
+  }
+}
+
+// workspace[i] = sum over r < R of partials[r][i], added in the order r = 0, 1, ..., R-1 (the same on every rank
+// and in every run), rounded once to the storage type
+template <typename T>
+__global__ void reduce_partials_kernel(T* __restrict__ kv, const float* __restrict__ partials, int64_t count, int R) {
+  for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * 4; i < count; i += (int64_t)gridDim.x * blockDim.x * 4) {
+    float4 a = *reinterpret_cast<const float4*>(partials + i);
+    for (int r = 1; r < R; ++r) {
+      const float4 b = *reinterpret_cast<const float4*>(partials + (int64_t)r * count + i);
+      a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+    }
+    stf(kv, i, a.x); stf(kv, i + 1, a.y); stf(kv, i + 2, a.z); stf(kv, i + 3, a.w);
   }
 }
 
@@ -259,15 +277,24 @@ __global__ void split_kv_kernel(T* __restrict__ kt, T* __restrict__ vt, const T*
 }
 
 template <typename T>
-cudaError_t compress_t(csat_ctx* c, const void* K, const void* V, cudaStream_t s) {
+cudaError_t compress_t(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int64_t phi_j0, int64_t n_len,
+                       float* partial) {
   const Params& p = c->p;
   const int d = (int)p.d;
   const dim3 grid((unsigned)((p.m + kCmpRows - 1) / kCmpRows), (unsigned)(p.B * p.H));
   const size_t sm = (size_t)(2 * kCmpRows * (kCmpChunk + 1) + kCmpChunk * 2 * d) * sizeof(float);
   const int kc = (2 * d + 31) / 32;
-#define CSAT_CMP(KC)                                                                                         \
-  compress_kernel<T, KC><<<grid, 256, sm, s>>>((T*)c->kv, (const T*)c->phi, (const T*)K, (const T*)V, p.n, \
-                                               p.n_pad, p.m, d, (int)p.H, p.separate_phi ? (int)p.H : 0)
+#define CSAT_CMP(KC)                                                                                                  \
+  do {                                                                                                                \
+    if (partial)                                                                                                      \
+      compress_kernel<T, float, KC><<<grid, 256, sm, s>>>(partial, (const T*)c->phi, (const T*)K, (const T*)V, n_len, \
+                                                          p.n_pad, p.m, d, (int)p.H, p.separate_phi ? (int)p.H : 0,  \
+                                                          phi_j0);                                                    \
+    else                                                                                                              \
+      compress_kernel<T, T, KC><<<grid, 256, sm, s>>>((T*)c->kv, (const T*)c->phi, (const T*)K, (const T*)V, n_len,  \
+                                                      p.n_pad, p.m, d, (int)p.H, p.separate_phi ? (int)p.H : 0,      \
+                                                      phi_j0);                                                        \
+  } while (0)
   if (kc <= 4) CSAT_CMP(4);
   else if (kc <= 8) CSAT_CMP(8);
   else CSAT_CMP(16);
@@ -305,9 +332,25 @@ cudaError_t attend_t(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
 
 }  // namespace
 
-cudaError_t launch_simt_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches) {
+cudaError_t launch_simt_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches,
+                                 int64_t phi_j0, int64_t n_len, float* partial) {
   *launches += 1;
-  return c->p.dtype == CSAT_DTYPE_FP32 ? compress_t<float>(c, K, V, s) : compress_t<__nv_bfloat16>(c, K, V, s);
+  if (n_len <= 0) n_len = c->p.n;
+  return c->p.dtype == CSAT_DTYPE_FP32 ? compress_t<float>(c, K, V, s, phi_j0, n_len, partial)
+                                       : compress_t<__nv_bfloat16>(c, K, V, s, phi_j0, n_len, partial);
+}
+
+cudaError_t launch_reduce_partials(csat_ctx* c, const float* partials, int R, cudaStream_t s, int* launches) {
+  *launches += 1;
+  const Params& p = c->p;
+  const int64_t count = p.B * p.H * p.m * 2 * p.d;       // a multiple of 16 (d % 8 == 0)
+  int64_t g = (count / 4 + 255) / 256;
+  if (g > 148 * 16) g = 148 * 16;
+  if (p.dtype == CSAT_DTYPE_FP32)
+    reduce_partials_kernel<float><<<(unsigned)g, 256, 0, s>>>((float*)c->kv, partials, count, R);
+  else
+    reduce_partials_kernel<__nv_bfloat16><<<(unsigned)g, 256, 0, s>>>((__nv_bfloat16*)c->kv, partials, count, R);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_simt_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches) {
