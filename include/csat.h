@@ -74,6 +74,11 @@ enum {
                           same seeded generator, the decoder's default D is the block of Phi_V, and
                           csat_set_phi / csat_get_phi then move [2H, m, n]: the H matrices Phi_K, then the H
                           matrices Phi_V.  Changing it regenerates both from the seed                 */
+  CSAT_HADAMARD_TRANSFORM = 10, /* 1: with CSAT_ENSEMBLE_HADAMARD (seeded, not replaced by csat_set_phi) and n <= 16384,
+                          csat_forward compresses by a fast Walsh-Hadamard transform over the tokens followed by a
+                          gather of the m selected rows (n log n additions per column instead of m n multiply-adds; the
+                          same K~, V~ up to the order of the float32 sums).  0 (default): the dense product.  Other
+                          ensembles, supplied matrices and longer sequences keep the dense product either way      */
   CSAT_KEEP_MASKS = 9, /* 1: csat_backward also keeps its shrinkage decisions (one 32-bit word per (b, h, query,
                           column); needs CSAT_T <= 32) for csat_get_backward_masks.  0 (default): not kept  */
   CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls

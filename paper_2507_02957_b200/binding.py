@@ -18,6 +18,7 @@ ERR_NAMES = {1: "CSAT_ERR_INVALID_ARG", 2: "CSAT_ERR_SHAPE", 3: "CSAT_ERR_ALLOC"
              5: "CSAT_ERR_UNSUPPORTED", 6: "CSAT_ERR_STATE", 7: "CSAT_ERR_TIMEOUT"}
 CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE, CSAT_ENSEMBLE, CSAT_SEPARATE_PHI = 1, 2, 3, 4, 5, 6, 7, 8
 CSAT_KEEP_MASKS = 9
+CSAT_HADAMARD_TRANSFORM = 10
 CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER, CSAT_ENSEMBLE_HADAMARD = 0, 1, 2
 KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1
@@ -300,7 +301,10 @@ class Csat:
         except Exception:
             pass
 
-    def set(self, *, T=None, lam=None, step=None, scale=None, force_simt=None, ensemble=None, separate_phi=None):
+    def set(self, *, T=None, lam=None, step=None, scale=None, force_simt=None, ensemble=None, separate_phi=None,
+            hadamard_transform=None):
+        if hadamard_transform is not None:
+            csat_set_i64(self.h, CSAT_HADAMARD_TRANSFORM, int(bool(hadamard_transform)))
         if separate_phi is not None:
             csat_set_i64(self.h, CSAT_SEPARATE_PHI, int(bool(separate_phi)))
             self.phi_heads = self.H * (2 if separate_phi else 1)

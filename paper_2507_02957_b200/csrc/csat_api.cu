@@ -84,6 +84,30 @@ void free_lista(csat_ctx* c) {
   c->w_untied = false;
 }
 
+void free_hadamard_tables(csat_ctx* c) {
+  dev_free(c, &c->had_signs, c->had_bytes_signs);
+  dev_free(c, &c->had_ab, c->had_bytes_ab);
+  c->had_bytes_signs = c->had_bytes_ab = 0;
+}
+
+// the fast-transform compression's tables, (re)written whenever the structured Hadamard ensemble is generated
+int make_hadamard_tables(csat_ctx* c) {
+  free_hadamard_tables(c);
+  if (c->p.ensemble != CSAT_ENSEMBLE_HADAMARD) return CSAT_OK;
+  const csat::Params g = gen_params(c->p);
+  const size_t bs = (size_t)((g.H * g.n + 31) / 32) * 4, ba = (size_t)g.H * 8;
+  if (dev_alloc(c, &c->had_signs, bs) != cudaSuccess || dev_alloc(c, &c->had_ab, ba) != cudaSuccess) {
+    free_hadamard_tables(c);
+    return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(Hadamard tables) failed");
+  }
+  c->had_bytes_signs = bs;
+  c->had_bytes_ab = ba;
+  cudaError_t e = csat::launch_hadamard_tables(c->had_signs, c->had_ab, g, 0);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(0);
+  if (e != cudaSuccess) return fail_cuda(c, e, "Hadamard tables");
+  return CSAT_OK;
+}
+
 void free_backward(csat_ctx* c) {
   dev_free(c, &c->bw_dZ, c->bw_bytes_dZ);
   dev_free(c, &c->bw_LD, c->bw_bytes_LD);
@@ -119,6 +143,7 @@ void free_all(csat_ctx* c) {
   dev_free(c, &c->theta, (size_t)p.H * 4);
   dev_free(c, &c->mu, (size_t)p.H * 4);
   dev_free(c, &c->mats_bf16, 3 * dd_bytes(p, 2));
+  free_hadamard_tables(c);
   free_lista(c);
   free_staging(c);
   free_backward(c);
@@ -148,6 +173,8 @@ int allocate_and_generate(csat_ctx* c) {
   }
   if ((e = csat::launch_phi_gen(c->phi, gen_params(p), 0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen launch");
   if ((e = cudaStreamSynchronize(0)) != cudaSuccess) return fail_cuda(c, e, "phi_gen");
+  c->phi_generated = true;
+  if (int rc = make_hadamard_tables(c)) return rc;
   c->tmap_phi_valid = false;
   if (p.dtype == CSAT_DTYPE_BF16 && (p.d == 64 || p.d == 128)) {
     if ((e = csat::make_phi_tmap(c)) != cudaSuccess) return fail_cuda(c, e, "tensor map for Phi");
@@ -328,9 +355,14 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       cudaError_t e = csat::launch_phi_gen(c->phi, gen_params(p), 0);   // a Phi set by csat_set_phi is replaced as well
       if (e == cudaSuccess) e = cudaStreamSynchronize(0);
       if (e != cudaSuccess) return fail_cuda(c, e, "phi_gen");
+      c->phi_generated = true;
       c->decoder_dirty = true;
-      return CSAT_OK;
+      return make_hadamard_tables(c);
     }
+    case CSAT_HADAMARD_TRANSFORM:
+      if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_HADAMARD_TRANSFORM must be 0 or 1");
+      c->hadamard_transform = (int)v;
+      return CSAT_OK;
     case CSAT_SEPARATE_PHI: {
       if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_SEPARATE_PHI must be 0 or 1");
       if ((int)v == p.separate_phi && !c->broken) return CSAT_OK;
@@ -389,6 +421,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
     case CSAT_FORCE_SIMT: *out = c->force_simt; return CSAT_OK;
     case CSAT_PROFILE: *out = c->prof_slots; return CSAT_OK;
     case CSAT_KEEP_MASKS: *out = c->keep_masks ? 1 : 0; return CSAT_OK;
+    case CSAT_HADAMARD_TRANSFORM: *out = c->hadamard_transform; return CSAT_OK;
     default: return CSAT_ERR_INVALID_ARG;
   }
 }
@@ -429,6 +462,7 @@ int csat_set_phi(csat_ctx* c, const void* phi, void* stream) {
   if (!on_device(c, &why)) return fail(c, CSAT_ERR_STATE, why);
   cudaError_t e = csat::launch_phi_pack(c->phi, phi, gen_params(c->p), (cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_set_phi");
+  c->phi_generated = false;                // a supplied matrix has no structure the fast transform could use
   c->decoder_dirty = true;
   return CSAT_OK;
 }
@@ -581,7 +615,10 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   // float32 contexts, and head sizes without a tensor-core kernel, take the FFMA kernels
   const bool tc_compress = c->tmap_phi_valid && c->force_simt != 1;
   const bool tc_attend = c->tmap_phi_valid && c->force_simt == 0;
-  e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
+  if (c->hadamard_transform && csat::fwht_compress_supported(c))
+    e = csat::launch_fwht_compress(c, K, V, s, &launches);   // structured ensemble: transform instead of the dense product
+  else
+    e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
   if (e != cudaSuccess) return fail_cuda(c, e, "compress launch");
   prof_mark(c, s, CSAT_KERNEL_COMPRESS);
   e = tc_attend ? csat::launch_sm100_attend_recover(c, Q, out, s, &launches)

@@ -62,6 +62,14 @@ struct csat_ctx {
   void* psi = nullptr;        // [Hpsi, d, d] dtype (user dictionary), null = identity
   void* dmat = nullptr;       // [H, d, d] dtype (user decoder matrix), null = Phi block
   bool psi_per_head = false;
+  bool phi_generated = true;  // phi holds the seeded ensemble (false once csat_set_phi replaced it)
+  // structured Hadamard ensemble: what the fast-transform compression needs instead of the dense matrix.
+  // had_signs: the column-sign bit stream (bit e % 32 of word e / 32, e = head * n + column); had_ab: (u0, u1) per
+  // head, row r of Phi_h is row ((2 u0 + 1) r + u1) mod N of the Hadamard matrix.  Written with the ensemble.
+  uint32_t* had_signs = nullptr;
+  uint32_t* had_ab = nullptr;
+  size_t had_bytes_signs = 0, had_bytes_ab = 0;
+  int hadamard_transform = 0; // CSAT_HADAMARD_TRANSFORM
   CUtensorMap tmap_phi;       // TMA view of phi for the tensor-core compress kernel (bf16, d in {64,128})
   bool tmap_phi_valid = false;
   CUtensorMap tmap_kv;        // TMA view of the K~|V~ workspace
@@ -141,6 +149,12 @@ size_t elt_size(int dtype);
 
 // phi_gen.cu
 cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s);
+// sign stream words [ceil(heads n / 32)] and (u0, u1) per head [2 heads] of the structured Hadamard ensemble
+cudaError_t launch_hadamard_tables(uint32_t* sign_words, uint32_t* ab, const Params& p, cudaStream_t s);
+
+// fwht_compress.cu : K~|V~ of the structured Hadamard ensemble by a fast Walsh-Hadamard transform
+bool fwht_compress_supported(const csat_ctx* c);
+cudaError_t launch_fwht_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches);
 cudaError_t launch_phi_pack(void* phi_padded, const void* phi_dense, const Params& p, cudaStream_t s);
 cudaError_t launch_phi_unpack(void* phi_dense, const void* phi_padded, const Params& p, cudaStream_t s);
 

@@ -237,6 +237,25 @@ __global__ void phi_hadamard_kernel(T* __restrict__ phi, int64_t n, int64_t n_pa
   }
 }
 
+// word k of the column-sign stream = word k % 4 of the Philox block with counter (k / 4, 0, 2, 0); (u0, u1) of head h
+// = the first two words of block (h, 0, 3, 0): the same blocks phi_hadamard_kernel draws from
+__global__ void hadamard_tables_kernel(uint32_t* __restrict__ sign_words, uint32_t* __restrict__ ab, int64_t nwords,
+                                       int heads, uint32_t k0, uint32_t k1) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const int64_t nblocks = (nwords + 3) >> 2;
+  if (i < nblocks) {
+    const U4 u = philox4x32_10(U4{(uint32_t)i, (uint32_t)(i >> 32), 2u, 0u}, k0, k1);
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+    for (int q = 0; q < 4; ++q)
+      if (4 * i + q < nwords) sign_words[4 * i + q] = w[q];
+  }
+  if (i < heads) {
+    const U4 u = philox4x32_10(U4{(uint32_t)i, 0u, 3u, 0u}, k0, k1);
+    ab[2 * i] = u.x;
+    ab[2 * i + 1] = u.y;
+  }
+}
+
 template <typename T>
 __global__ void phi_pack_kernel(T* __restrict__ dst, const T* __restrict__ src, int64_t rows, int64_t n,
                                 int64_t n_pad, bool to_padded) {
@@ -303,6 +322,15 @@ cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s) {
     phi_gen_kernel<float><<<grid, block, 0, s>>>((float*)phi, total, p.n, p.n_pad, inv, k0, k1);
   else
     phi_gen_kernel<__nv_bfloat16><<<grid, block, 0, s>>>((__nv_bfloat16*)phi, total, p.n, p.n_pad, inv, k0, k1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_hadamard_tables(uint32_t* sign_words, uint32_t* ab, const Params& p, cudaStream_t s) {
+  const int64_t nwords = (p.H * p.n + 31) / 32;            // p.H counts every generated matrix (2 H with separate Phi_V)
+  const int64_t nblocks = (nwords + 3) / 4;
+  const int64_t work = nblocks > p.H ? nblocks : p.H;
+  const uint32_t k0 = (uint32_t)(p.seed & 0xFFFFFFFFull), k1 = (uint32_t)(p.seed >> 32);
+  hadamard_tables_kernel<<<(unsigned)((work + 127) / 128), 128, 0, s>>>(sign_words, ab, nwords, (int)p.H, k0, k1);
   return cudaGetLastError();
 }
 

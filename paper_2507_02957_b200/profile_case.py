@@ -5,6 +5,8 @@
     python -m paper_2507_02957_b200.profile_case ensembles N M D H        (regenerates Phi with every ensemble)
     python -m paper_2507_02957_b200.profile_case project N D B H DMODEL [--iters I]   (the Q, K, V projections)
     python -m paper_2507_02957_b200.profile_case backward c1|c2|c3|c4|c5 [--iters I]   (csat_backward on a workload)
+    python -m paper_2507_02957_b200.profile_case hadamard N D B H [--iters I]   (compression of the structured Hadamard
+                       ensemble, dense product against fast transform, for m / n in {1/16, 1/8, 1/4, 1/2})
 
 A small driver to put under a profiler (ncu -k regex:<kernel> ...): 3 warm-up forwards, then I timed ones.
 Inputs are seeded random tensors (N(0, 1/d) for `forward`, the workload's own recipe for `workload`).
@@ -60,6 +62,10 @@ def main():
     bw = sub.add_parser("backward")
     bw.add_argument("name")
     bw.add_argument("--iters", type=int, default=3)
+    hd = sub.add_parser("hadamard")
+    for name in ("n", "d", "B", "H"):
+        hd.add_argument(name, type=int)
+    hd.add_argument("--iters", type=int, default=10)
     a = ap.parse_args()
 
     if a.cmd == "forward":
@@ -111,6 +117,32 @@ def main():
             times.append(e0.elapsed_time(e1))
         print(w.name, {"backward_ms": round(float(np.median(times)), 4)})
         ctx.close()
+    elif a.cmd == "hadamard":
+        g = torch.Generator(device="cuda")
+        g.manual_seed(1)
+        s = 1.0 / np.sqrt(a.d)
+        Q, K, V = ((torch.randn(a.B, a.H, a.n, a.d, device="cuda", generator=g) * s).to(torch.bfloat16) for _ in range(3))
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        for frac in (16, 8, 4, 2):
+            ctx = binding.Csat(a.n, a.n // frac, a.d, a.H, 0, B=a.B, dtype="bf16", T=0)
+            ctx.set(ensemble="hadamard")
+            out = torch.empty_like(Q)
+            row = {}
+            for mode in ("dense", "transform"):
+                ctx.set(hadamard_transform=(mode == "transform"))
+                for _ in range(3):
+                    ctx.forward(Q, K, V, out)
+                torch.cuda.synchronize()
+                binding.csat_set_i64(ctx.h, binding.CSAT_PROFILE, a.iters)
+                for _ in range(a.iters):
+                    flush.zero_()
+                    ctx.forward(Q, K, V, out)
+                torch.cuda.synchronize()
+                ts = [ms for i in range(a.iters) for kid, ms in binding.csat_get_profile(ctx.h, i) if kid == 1]
+                binding.csat_set_i64(ctx.h, binding.CSAT_PROFILE, 0)
+                row[mode] = round(float(np.median(ts)), 5)
+            print(f"n={a.n} d={a.d} B={a.B} H={a.H} m=n/{frac}={a.n // frac}: compress ms", row)
+            ctx.close()
     elif a.cmd == "project":
         g = torch.Generator(device="cuda")
         g.manual_seed(1)

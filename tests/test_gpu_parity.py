@@ -603,3 +603,48 @@ def test_project_qkv_matches_oracle(case):
     ref = orc.csat_forward(to_np(Q), to_np(K), to_np(V), to_np(ctx.get_phi()), T=0, lam=0.0)
     assert rel_err(out, ref) <= TOL[dt]
     ctx.close()
+
+
+FWHT_CASES = {
+    "bf16_d64_n4096_m1024": wl.Workload("fwht_a", 2, 2, 4096, 300, 64, 1024, "bf16", 3, 0.01, "iid", 71),
+    "bf16_d64_ragged_n197": wl.Workload("fwht_b", 2, 3, 197, 197, 64, 64, "bf16", 3, 0.01, "iid", 72),
+    "fp32_d72_n1000": wl.Workload("fwht_c", 1, 2, 1000, 100, 72, 250, "fp32", 2, 0.01, "iid", 73),
+    "bf16_d128_n5000": wl.Workload("fwht_d", 1, 2, 5000, 200, 128, 320, "bf16", 2, 0.01, "iid", 74),
+    "bf16_d64_n16384": wl.Workload("fwht_e", 1, 1, 16384, 256, 64, 1024, "bf16", 0, 0.0, "iid", 75),
+}
+
+
+@pytest.mark.parametrize("name", sorted(FWHT_CASES))
+@pytest.mark.parametrize("separate", [False, True])
+def test_hadamard_fast_transform_matches_oracle_and_dense_product(name, separate):
+    """CSAT_HADAMARD_TRANSFORM: K~, V~ by a fast Walsh-Hadamard transform and a gather of the selected rows.  The
+    reference is the oracle's compression with the dense matrix the library exports for the same ensemble; the dense
+    tensor-core / FFMA product of the same context must agree as well, and so must the whole forward."""
+    w = FWHT_CASES[name]
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    ctx.set(ensemble="hadamard")
+    if separate:
+        ctx.set(separate_phi=True)
+    phi = to_np(ctx.get_phi())
+    phi_k, phi_v = phi[:w.H], (phi[w.H:] if separate else phi[:w.H])
+    dense_out = ctx.forward(Q, K, V).clone()
+    kt_d, vt_d = (to_np(t) for t in ctx.get_compressed())
+    ctx.set(hadamard_transform=True)
+    assert binding.csat_get_i64(ctx.h, binding.CSAT_HADAMARD_TRANSFORM) == 1
+    fast_out = ctx.forward(Q, K, V)
+    kt_f, vt_f = (to_np(t) for t in ctx.get_compressed())
+    kt_ref = np.stack([[orc.compress(phi_k[h], inp["K"][b, h]) for h in range(w.H)] for b in range(w.B)])
+    vt_ref = np.stack([[orc.compress(phi_v[h], inp["V"][b, h]) for h in range(w.H)] for b in range(w.B)])
+    tol_kv = 4e-3 if w.dtype == "bf16" else 2e-6
+    assert rel_err(kt_f, kt_ref) <= tol_kv and rel_err(vt_f, vt_ref) <= tol_kv, name
+    assert rel_err(kt_f, kt_d) <= 2 * tol_kv and rel_err(vt_f, vt_d) <= 2 * tol_kv, name
+    ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi_k, T=w.T, lam=w.lam, Phi_V=phi_v if separate else None)
+    assert rel_err(to_np(fast_out), ref) <= TOL[w.dtype], name
+    assert rel_err(to_np(fast_out), to_np(dense_out)) <= TOL[w.dtype], name
+    assert torch.equal(fast_out, ctx.forward(Q, K, V))               # deterministic
+    # a supplied matrix has no structure to transform: the dense product takes over again
+    ctx.set_phi(ctx.get_phi())
+    assert torch.equal(ctx.forward(Q, K, V), dense_out)
+    ctx.close()
