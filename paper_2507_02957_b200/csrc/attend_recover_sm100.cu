@@ -202,7 +202,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
-                            int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status) {
+                            int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status,
+                            float* __restrict__ lse_out, int lse_stride) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
@@ -637,6 +638,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         float s0, s1;
         unpack2(sum2, s0, s1);
         inv = 1.f / (s0 + s1);
+        // the backward pass asks for the row's log sum exp of the scaled scores (natural logarithm)
+        if (lse_out != nullptr && row0 + t * kRows + row < nq)
+          lse_out[((int64_t)bh * nq + row0 + t * kRows + row) * lse_stride] = (ref + __log2f(s0 + s1)) * 0.69314718056f;
       }
       w.wait(&bars->zc_full[t], (cb + nchunks - 1) & 1, 222);   // every P V~ product has been added
       cb += nchunks;
@@ -882,7 +886,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
 }
 
 template <int D, bool kUntied>
-cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
+cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T, float* lse_out, int lse_stride) {
   using C = Cfg<D>;
   const Params& p = c->p;
   CUtensorMap tq;
@@ -905,8 +909,8 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s) {
   const int sms = c->sms;
   const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
   attend_recover_sm100_kernel<D, kUntied><<<grid, kThreads, C::kSmemBytes, s>>>(
-      tq, c->tmap_kv, kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, p.T,
-      c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, (int)c->bh0, c->status);
+      tq, c->tmap_kv, kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, T,
+      c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, (int)c->bh0, c->status, lse_out, lse_stride);
   return cudaGetLastError();
 }
 
@@ -939,8 +943,16 @@ cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, c
   *launches += 1;
   // with untied layers and T > 0 the per-layer kernel; the set-up has then built its operands for exactly T layers
   if (c->w_S && c->w_untied && c->p.T > 0)
-    return c->p.d == 64 ? launch<64, true>(c, Q, out, s) : launch<128, true>(c, Q, out, s);
-  return c->p.d == 64 ? launch<64, false>(c, Q, out, s) : launch<128, false>(c, Q, out, s);
+    return c->p.d == 64 ? launch<64, true>(c, Q, out, s, c->p.T, nullptr, 0) : launch<128, true>(c, Q, out, s, c->p.T, nullptr, 0);
+  return c->p.d == 64 ? launch<64, false>(c, Q, out, s, c->p.T, nullptr, 0) : launch<128, false>(c, Q, out, s, c->p.T, nullptr, 0);
+}
+
+// Z = A~ V~ (recovery disabled whatever CSAT_T says) and the rows' log sum exp, for the backward pass
+cudaError_t launch_sm100_attend_lse(csat_ctx* c, const void* Q, void* z_out, float* lse_out, int lse_stride,
+                                    cudaStream_t s, int* launches) {
+  *launches += 1;
+  return c->p.d == 64 ? launch<64, false>(c, Q, z_out, s, 0, lse_out, lse_stride)
+                      : launch<128, false>(c, Q, z_out, s, 0, lse_out, lse_stride);
 }
 
 }  // namespace csat

@@ -393,6 +393,15 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   cudaError_t e = cudaSuccess;
   // bf16 with d in {64, 128}: the stages after the per-row kernel run on the tensor cores
   const bool tc_stages = c->bw_dKV16 != nullptr && c->bw_dZ16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
+  // ... and with one S, B for all layers the per-query stages too: the forward's attention phase leaves Z and the
+  // rows' log sum exp, then the recurrence (forward with its decisions recorded, and backward) and dQ
+  if (tc_stages && !c->w_untied && c->bw_Z16 != nullptr) {
+    if ((e = launch_sm100_attend_lse(c, Q, c->bw_Z16, c->bw_LD, 2, s, launches)) != cudaSuccess) return e;
+    if ((e = launch_sm100_bwd_recur(c, G, s, launches)) != cudaSuccess) return e;
+    if ((e = launch_sm100_bwd_dq(c, Q, dQ, s, launches)) != cudaSuccess) return e;
+    if ((e = launch_sm100_bwd_cols(c, Q, s, launches)) != cudaSuccess) return e;
+    return launch_sm100_phiT(c, c->bw_dKV16, dK, dV, s, launches);
+  }
   const int64_t mats = (c->w_untied ? c->w_layers : 1) * p.H;
   float* SdT = c->bw_WT;
   float* BdT = c->bw_WT + mats * d * d;

@@ -1,0 +1,619 @@
+// The per-query stages of the backward pass on the sm_100a tensor cores (bf16 storage, d in {64, 128}, one S, B for
+// all layers).  The paper trains through its unrolled decoder but prints no backward pass: this is the chain rule
+// through the LISTA recurrence alpha^{t+1} = eta_theta(alpha^t S + z B), the reconstruction C^ = Psi alpha, the
+// compressed output Z = A~ V~ and the softmax over the measurements, with the derivative of eta_theta taken as 1
+// where |x| > theta and 0 elsewhere.
+//
+// Before these kernels the forward's own kernels have left K~|V~ in the workspace, Z (bf16, as the forward rounds it
+// for its first product) in bw_Z16 and every row's log sum exp L in bw_LD.
+//
+// bwd_recur_sm100_kernel, one CTA per tile of 128 queries (TMEM lane = query row, one thread per row):
+//   1. the forward recurrence exactly as the forward kernel runs it (increment form: the accumulator holds
+//      r_t = theta + z B - a^_t (mu G), the registers b_t = alpha^t - theta; bf16 increments feed one MMA per layer),
+//      recording the decision |x_t| > theta_t of every layer as bit t of a word per (row, column) in tensor memory;
+//   2. d alpha_T = G Psi (one MMA; G itself without a dictionary), then for t = T-1 .. 0
+//        dx_t = d alpha_{t+1} o mask_t,   dZ += dx_t B^T,   d alpha_t = dx_t S^T = dx_t + dx_t (S - I)^T :
+//      dx_t goes to tensor memory as the bf16 A operand of two MMAs, whose B operands are the forward's own
+//      shared-memory tiles of S - I and B read as MN-major operands (a d x d tile with 128-byte rows is K-major when
+//      its rows are the output columns and MN-major when they are the reduction index: the transposed product needs
+//      no transposed copy); the identity part of S^T stays exact in float32 registers;
+//   3. dZ (bf16, the operand of the stages that follow) and D = <dZ, Z>.
+//
+// bwd_dq_sm100_kernel, one CTA per tile of 128 queries, K~|V~ streamed in chunks of 64 measurements:
+//        S_j = Q K~_j^T,  dA_j = dZ V~_j^T                        (two SS MMAs into tensor memory)
+//        dS_j = scale * exp(scale S_j - L) o (dA_j - D)           (one thread per row; bf16 back into tensor memory)
+//        dQ  += dS_j K~_j                                         (TS MMA, K~_j read as an MN-major operand)
+//   the structure of the forward's attention phase with the roles of the operands changed.
+//
+// Every wait is bounded (see sm100_ptx.cuh); a time-out sets the context's status word and the CTA winds down.
+#include "csat_internal.h"
+#include "sm100_ptx.cuh"
+#include "tma_host.h"
+
+namespace csat {
+namespace {
+
+using namespace ptx;
+
+constexpr int kRows = 128;
+constexpr int kMC = 64;
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&p);
+}
+__device__ __forceinline__ float fma_sat(float a, float b, float c) {   // clamps the result to [0, 1]
+  float y;
+  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+struct Waiter {
+  int* status;
+  int* cta_abort;
+  bool dead = false;
+  __device__ __forceinline__ void wait(uint64_t* bar, uint32_t parity, int code) {
+    if (dead) return;
+    if (!mbar_wait(bar, parity, status, code, cta_abort)) dead = true;
+  }
+};
+
+// ====================================================================================================================
+// recurrence forward (masks) and backward
+// ====================================================================================================================
+template <int D> struct RCfg {
+  static constexpr int kDBoxes = D / 64;
+  static constexpr uint32_t kMatBoxBytes = D * 128;               // one 64-column box of a d x d bf16 matrix
+  static constexpr uint32_t kMatBytes = kDBoxes * kMatBoxBytes;
+  static constexpr uint32_t kOffMat = 0;                          // [3]: S - I | B^T | Psi, as the forward stages them
+  static constexpr uint32_t kOffBar = 3 * kMatBytes;
+  static constexpr uint32_t kSmemBytes = kOffBar + 128 + 1024 /*alignment slack*/;
+  // TMEM columns: accumulator | dZ accumulator | masks (one word per column) | bf16 operand (two per column)
+  static constexpr uint32_t kColAcc = 0, kColDz = D, kColMask = 2 * D, kColOp = 3 * D;
+  static constexpr uint32_t kTmemCols = (D == 64) ? 256 : 512;
+  static_assert(3 * D + D / 2 <= kTmemCols, "TMEM budget");
+};
+
+struct RBars {
+  uint64_t mats_full, a_full, r_full;
+  uint32_t tmem_slot;
+  int abort;
+};
+
+constexpr int kRThreads = 160;      // warps 0-3: one thread per query row; warp 4: TMA and MMA issue
+
+template <int D>
+__global__ void __launch_bounds__(kRThreads, 1)
+bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv_bfloat16* __restrict__ Z16,
+                       const __nv_bfloat16* __restrict__ G, __nv_bfloat16* __restrict__ dZ16, float* __restrict__ ws_LD,
+                       uint32_t* __restrict__ ws_masks, const float* __restrict__ theta, int theta_stride, int nq, int H,
+                       int T, int has_psi, int* status) {
+  using C = RCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  RBars* bars = reinterpret_cast<RBars*>(smem + C::kOffBar);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, h = bh % H, row0 = blockIdx.x * kRows;
+  Waiter w{status, &bars->abort};
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tmap_mats);
+    mbar_init(&bars->mats_full, 1);
+    mbar_init(&bars->a_full, kRows);
+    mbar_init(&bars->r_full, 1);
+    bars->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(&bars->tmem_slot, C::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_slot;
+
+  if (warp == 4) {
+    if (T > 0 && elect_one()) {
+      // ---- the decoder matrices of this head, then one MMA group per operand the threads publish ----
+      const int nmats = has_psi ? 3 : 2;
+      mbar_arrive_expect_tx(&bars->mats_full, nmats * C::kMatBytes);
+      for (int mat = 0; mat < nmats; ++mat)
+        for (int gx = 0; gx < C::kDBoxes; ++gx)
+          tma_load_3d(smem + C::kOffMat + mat * C::kMatBytes + gx * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, gx * 64,
+                      0, h * 3 + mat);
+      constexpr uint32_t idesc_f = make_idesc_bf16(kRows, D, false, false);   // forward products: B K-major
+      constexpr uint32_t idesc_t = make_idesc_bf16(kRows, D, false, true);    // transposed products: B MN-major
+      auto mat_k = [&](int mat) { return make_smem_desc(smem_u32(smem + C::kOffMat + mat * C::kMatBytes), 16, 1024); };
+      auto mat_mn = [&](int mat) {
+        return make_smem_desc(smem_u32(smem + C::kOffMat + mat * C::kMatBytes), C::kMatBoxBytes, 1024);
+      };
+      const uint32_t op = tmem + C::kColOp, acc = tmem + C::kColAcc, dz = tmem + C::kColDz;
+      // product with the matrix as the forward stores it (K-major): K step k lies in box k / 4, 32 (k % 4) bytes in
+      auto mma_fwd = [&](uint32_t d_t, int mat, uint32_t accumulate) {
+        const uint64_t bd = mat_k(mat);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          mma_f16_ts(d_t, op + k * 8, bd + (uint64_t)((k / 4) * (C::kMatBoxBytes >> 4) + (k % 4) * 2), idesc_f,
+                     k == 0 ? accumulate : 1u);
+      };
+      // product with its transpose: the tile's rows are the reduction index, 16 rows (2048 bytes) per K step
+      auto mma_tr = [&](uint32_t d_t, int mat, uint32_t accumulate) {
+        const uint64_t bd = mat_mn(mat);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k) mma_f16_ts(d_t, op + k * 8, bd + (uint64_t)(k * 128), idesc_t, k == 0 ? accumulate : 1u);
+      };
+      uint32_t n_ops = 0;
+      auto operand_ready = [&]() {
+        w.wait(&bars->a_full, n_ops & 1, 601);
+        ++n_ops;
+        tc_fence_after();
+      };
+      w.wait(&bars->mats_full, 0, 600);
+      // forward: r_0 = kappa + z B, then T - 1 increments times S - I
+      operand_ready();
+      mma_fwd(acc, 1, 1u);
+      mma_commit(&bars->r_full);
+      for (int it = 0; it + 1 < T; ++it) {
+        operand_ready();
+        mma_fwd(acc, 0, 1u);
+        mma_commit(&bars->r_full);
+      }
+      // backward: d alpha_T = G Psi
+      if (has_psi) {
+        operand_ready();
+        mma_tr(acc, 2, 0u);
+        mma_commit(&bars->r_full);
+      }
+      for (int t = T - 1; t >= 0; --t) {
+        operand_ready();
+        if (t > 0) mma_tr(acc, 0, 0u);                       // dx_t (S - I)^T
+        mma_tr(dz, 1, t == T - 1 ? 0u : 1u);                 // dZ += dx_t B^T
+        mma_commit(&bars->r_full);
+      }
+      if (w.dead) mbar_wait_drain(&bars->mats_full, 0);
+    }
+  } else {
+    // ---------------------------------------------- one thread per query row ----------------------------------------
+    const int row = warp * 32 + lane;
+    const int grow = row0 + row;
+    const bool live = grow < nq;
+    const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t acc_addr = tbase + C::kColAcc, dz_addr = tbase + C::kColDz, mask_addr = tbase + C::kColMask,
+                   op_addr = tbase + C::kColOp;
+    const int64_t goff = ((int64_t)bh * nq + (live ? grow : 0)) * D;
+    int phase = 0;
+    float v[D];                                   // b_t = alpha^t - kappa, later d alpha / dx
+    auto publish_bf16 = [&]() {                   // v as the bf16 A operand
+#pragma unroll
+      for (int c0 = 0; c0 < D; c0 += 16) {
+        uint32_t pk[8];
+#pragma unroll
+        for (int e = 0; e < 16; e += 2) pk[e >> 1] = pack_bf16(v[c0 + e], v[c0 + e + 1]);
+        tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars->a_full);
+    };
+    auto load_row = [&](const __nv_bfloat16* src) {       // v := the row of a [B,H,n_q,d] bf16 tensor (0 beyond n_q)
+      const uint4* p = reinterpret_cast<const uint4*>(src + goff);
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) {
+        const uint4 q = live ? p[c] : make_uint4(0, 0, 0, 0);
+        v[8 * c + 0] = bf16_lo(q.x); v[8 * c + 1] = bf16_hi(q.x);
+        v[8 * c + 2] = bf16_lo(q.y); v[8 * c + 3] = bf16_hi(q.y);
+        v[8 * c + 4] = bf16_lo(q.z); v[8 * c + 5] = bf16_hi(q.z);
+        v[8 * c + 6] = bf16_lo(q.w); v[8 * c + 7] = bf16_hi(q.w);
+      }
+    };
+    if (T == 0) {
+      // no decoder: dZ = G, D = <G, Z>
+      load_row(G);
+      float dsum = 0.f;
+      const uint4* zp = reinterpret_cast<const uint4*>(Z16 + goff);
+      uint4* out = reinterpret_cast<uint4*>(dZ16 + goff);
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) {
+        const uint4 z = live ? zp[c] : make_uint4(0, 0, 0, 0);
+        dsum = fmaf(v[8 * c + 0], bf16_lo(z.x), dsum); dsum = fmaf(v[8 * c + 1], bf16_hi(z.x), dsum);
+        dsum = fmaf(v[8 * c + 2], bf16_lo(z.y), dsum); dsum = fmaf(v[8 * c + 3], bf16_hi(z.y), dsum);
+        dsum = fmaf(v[8 * c + 4], bf16_lo(z.z), dsum); dsum = fmaf(v[8 * c + 5], bf16_hi(z.z), dsum);
+        dsum = fmaf(v[8 * c + 6], bf16_lo(z.w), dsum); dsum = fmaf(v[8 * c + 7], bf16_hi(z.w), dsum);
+        if (live)
+          out[c] = make_uint4(pack_bf16(v[8 * c], v[8 * c + 1]), pack_bf16(v[8 * c + 2], v[8 * c + 3]),
+                              pack_bf16(v[8 * c + 4], v[8 * c + 5]), pack_bf16(v[8 * c + 6], v[8 * c + 7]));
+      }
+      if (live) ws_LD[((int64_t)bh * nq + grow) * 2 + 1] = dsum;
+    } else {
+      // ---- forward recurrence, as the forward kernel runs it, with the decisions recorded ----
+      const float kappa = theta[h];
+      {
+        uint32_t tb[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) tb[e] = __float_as_uint(kappa);
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) tmem_st_32x32b_x16(acc_addr + c0, tb);      // accumulator := kappa
+      }
+      load_row(Z16);
+      publish_bf16();                                                                 // z as the A operand of z B
+#pragma unroll
+      for (int i = 0; i < D; ++i) v[i] = -kappa;                                      // alpha^0 = 0
+      for (int it = 0; it < T; ++it) {
+        const float th = theta[(int64_t)it * theta_stride + h];
+        const bool last = it == T - 1;
+        const float inv2th = th > 0.f ? 0.5f / th : 0.f;
+        const float dk = th - kappa;
+        w.wait(&bars->r_full, phase & 1, 610); ++phase;
+        tc_fence_after();
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t r[16], mk[16];
+          tmem_ld_32x32b_x16(acc_addr + c0, r);
+          if (it > 0) tmem_ld_32x32b_x16(mask_addr + c0, mk);
+          tmem_wait_ld();
+          uint32_t pk[8];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const float rr = __uint_as_float(r[e]);
+            const float x = v[c0 + e] + rr;                     // alpha^t S + z B - (kappa - kappa)
+            uint32_t bit;
+            float inc;
+            if (!last) {
+              // saturating form, as in the forward: s in {0, 1} exactly where |x| >= theta
+              const float s = fma_sat(x, inv2th, 0.5f);
+              const float bn = fmaf(s, -2.f * th, x) + dk;      // eta_theta(x) - kappa
+              inc = fmaf(s, -2.f * th, rr) + dk;                // alpha^{t+1} - alpha^t
+              v[c0 + e] = bn;
+              bit = (__float_as_uint(s) - 1u >= 0x3f7fffffu) ? 1u : 0u;
+              if (th == 0.f) bit = 1u;                          // eta_0 is the identity
+            } else {
+              inc = 0.f;
+              bit = fabsf(x) > th ? 1u : 0u;
+            }
+            if (e & 1) pk[e >> 1] = pack_bf16(__uint_as_float(pk[e >> 1]), inc); else pk[e >> 1] = __float_as_uint(inc);
+            mk[e] = (it > 0 ? mk[e] : 0u) | (bit << it);
+          }
+          tmem_st_32x32b_x16(mask_addr + c0, mk);
+          if (!last) tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+        }
+        tmem_wait_st();
+        if (!last) {
+          tc_fence_before();
+          mbar_arrive(&bars->a_full);
+        }
+      }
+      if (ws_masks != nullptr) {              // (the tensor-memory loads are warp-wide: every lane takes part)
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t mk[16];
+          tmem_ld_32x32b_x16(mask_addr + c0, mk);
+          tmem_wait_ld();
+          if (live) {
+            uint4* o = reinterpret_cast<uint4*>(ws_masks + goff + c0);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) o[q] = make_uint4(mk[4 * q], mk[4 * q + 1], mk[4 * q + 2], mk[4 * q + 3]);
+          }
+        }
+      }
+      // ---- backward recurrence ----
+      load_row(G);                                              // d out
+      if (has_psi) {
+        publish_bf16();                                         // G is bf16 already: nothing is lost
+        w.wait(&bars->r_full, phase & 1, 611); ++phase;
+        tc_fence_after();
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(acc_addr + c0, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 16; ++e) v[c0 + e] = __uint_as_float(r[e]);          // d alpha_T = G Psi
+        }
+      }
+      for (int t = T - 1; t >= 0; --t) {
+        // dx_t = d alpha_{t+1} o mask_t, published as the operand of both products
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t mk[16];
+          tmem_ld_32x32b_x16(mask_addr + c0, mk);
+          tmem_wait_ld();
+          uint32_t pk[8];
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) {
+            const float a0 = ((mk[e] >> t) & 1u) ? v[c0 + e] : 0.f, a1 = ((mk[e + 1] >> t) & 1u) ? v[c0 + e + 1] : 0.f;
+            v[c0 + e] = a0;
+            v[c0 + e + 1] = a1;
+            pk[e >> 1] = pack_bf16(a0, a1);
+          }
+          tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+        }
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(&bars->a_full);
+        w.wait(&bars->r_full, phase & 1, 612); ++phase;
+        tc_fence_after();
+        if (t > 0) {
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld_32x32b_x16(acc_addr + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) v[c0 + e] += __uint_as_float(r[e]);        // d alpha_t = dx_t + dx_t (S - I)^T
+          }
+        }
+      }
+      // ---- dZ and D = <dZ, Z> ----
+      float dsum = 0.f;
+      const uint4* zp = reinterpret_cast<const uint4*>(Z16 + goff);
+      uint4* out = reinterpret_cast<uint4*>(dZ16 + goff);
+#pragma unroll
+      for (int c0 = 0; c0 < D; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(dz_addr + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          const uint4 z = live ? zp[c0 / 8 + half] : make_uint4(0, 0, 0, 0);
+          const float* f = reinterpret_cast<const float*>(r) + 8 * half;
+          dsum = fmaf(f[0], bf16_lo(z.x), dsum); dsum = fmaf(f[1], bf16_hi(z.x), dsum);
+          dsum = fmaf(f[2], bf16_lo(z.y), dsum); dsum = fmaf(f[3], bf16_hi(z.y), dsum);
+          dsum = fmaf(f[4], bf16_lo(z.z), dsum); dsum = fmaf(f[5], bf16_hi(z.z), dsum);
+          dsum = fmaf(f[6], bf16_lo(z.w), dsum); dsum = fmaf(f[7], bf16_hi(z.w), dsum);
+          if (live && !w.dead)
+            out[c0 / 8 + half] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
+                                            pack_bf16(f[6], f[7]));
+        }
+      }
+      if (live && !w.dead) ws_LD[((int64_t)bh * nq + grow) * 2 + 1] = dsum;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) tmem_dealloc(tmem, C::kTmemCols);
+}
+
+// ====================================================================================================================
+// dQ
+// ====================================================================================================================
+template <int D> struct QCfg {
+  static constexpr int kDBoxes = D / 64;
+  static constexpr int kStages = 3;
+  static constexpr uint32_t kTileBoxBytes = kRows * 128;            // 128 rows x 64 columns
+  static constexpr uint32_t kTileBytes = kDBoxes * kTileBoxBytes;   // Q tile, dZ tile
+  static constexpr uint32_t kBoxBytes = kMC * 128;                  // one 64-column box of a K~ or V~ chunk
+  static constexpr uint32_t kSlotBytes = kDBoxes * kBoxBytes;
+  static constexpr uint32_t kOffQ = 0, kOffZ = kTileBytes, kOffRing = 2 * kTileBytes;   // ring: [stage][K~ slot | V~ slot]
+  static constexpr uint32_t kOffBar = kOffRing + kStages * 2 * kSlotBytes;
+  static constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024 /*alignment slack*/;
+  // TMEM columns: S[2] | dA[2] | dQ accumulator; dS_j (bf16) overlays the first half of S[j & 1]
+  static constexpr uint32_t kColS = 0, kColA = 2 * kMC, kColQ = 4 * kMC, kTmemCols = 512;
+  static_assert(4 * kMC + D <= 512, "TMEM budget");
+};
+
+struct QBars {
+  uint64_t qz_full, full[3], empty[3], s_full[2], p_full[2], acc_done;
+  uint32_t tmem_slot;
+  int abort;
+};
+
+constexpr int kQThreads = 192;      // warps 0-3: one thread per query row; warp 4: TMA; warp 5: MMA issue
+
+template <int D>
+__global__ void __launch_bounds__(kQThreads, 1)
+bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_z,
+                    const __grid_constant__ CUtensorMap tmap_kv, __nv_bfloat16* __restrict__ dQ,
+                    const float* __restrict__ ws_LD, int nq, int m, float scale, int* status) {
+  using C = QCfg<D>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  QBars* bars = reinterpret_cast<QBars*>(smem + C::kOffBar);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int bh = blockIdx.y, row0 = blockIdx.x * kRows;
+  const int nchunks = (m + kMC - 1) / kMC;
+  Waiter w{status, &bars->abort};
+  auto k_slot = [&](int s) { return smem + C::kOffRing + (2 * s) * C::kSlotBytes; };
+  auto v_slot = [&](int s) { return smem + C::kOffRing + (2 * s + 1) * C::kSlotBytes; };
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tmap_q);
+    prefetch_tmap(&tmap_z);
+    prefetch_tmap(&tmap_kv);
+    mbar_init(&bars->qz_full, 1);
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(&bars->s_full[b], 1); mbar_init(&bars->p_full[b], kRows); }
+    mbar_init(&bars->acc_done, 1);
+    bars->abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 5) {
+    tmem_alloc(&bars->tmem_slot, C::kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = bars->tmem_slot;
+
+  if (warp == 4) {
+    if (elect_one()) {
+      mbar_arrive_expect_tx(&bars->qz_full, 2 * C::kTileBytes);
+      for (int gx = 0; gx < C::kDBoxes; ++gx) {
+        tma_load_3d(smem + C::kOffQ + gx * C::kTileBoxBytes, &tmap_q, &bars->qz_full, gx * 64, row0, bh);
+        tma_load_3d(smem + C::kOffZ + gx * C::kTileBoxBytes, &tmap_z, &bars->qz_full, gx * 64, row0, bh);
+      }
+      int issued = 0;
+      for (int j = 0; j < nchunks && !w.dead; ++j) {
+        const int s = j % C::kStages;
+        if (j >= C::kStages) w.wait(&bars->empty[s], (j / C::kStages - 1) & 1, 701);
+        if (w.dead) break;
+        mbar_arrive_expect_tx(&bars->full[s], 2 * C::kSlotBytes);
+        for (int gx = 0; gx < C::kDBoxes; ++gx) {
+          tma_load_3d(k_slot(s) + gx * C::kBoxBytes, &tmap_kv, &bars->full[s], gx * 64, j * kMC, bh);
+          tma_load_3d(v_slot(s) + gx * C::kBoxBytes, &tmap_kv, &bars->full[s], D + gx * 64, j * kMC, bh);
+        }
+        ++issued;
+      }
+      if (w.dead) {
+        mbar_wait_drain(&bars->qz_full, 0);
+        for (int i = issued > C::kStages ? issued - C::kStages : 0; i < issued; ++i)
+          mbar_wait_drain(&bars->full[i % C::kStages], (i / C::kStages) & 1);
+      }
+    }
+  } else if (warp == 5) {
+    if (elect_one()) {
+      constexpr uint32_t idesc_s = make_idesc_bf16(kRows, kMC, false, false);   // S, dA: both operands K-major
+      constexpr uint32_t idesc_q = make_idesc_bf16(kRows, D, false, true);      // dQ += dS K~: K~ is MN-major
+      auto kstep = [](int k, uint32_t box_bytes) { return (uint64_t)((k / 4) * (box_bytes >> 4) + (k % 4) * 2); };
+      const uint64_t qd = make_smem_desc(smem_u32(smem + C::kOffQ), 16, 1024);
+      const uint64_t zd = make_smem_desc(smem_u32(smem + C::kOffZ), 16, 1024);
+      auto issue_sd = [&](int j) {
+        const int s = j % C::kStages, b = j & 1;
+        w.wait(&bars->full[s], (j / C::kStages) & 1, 711);
+        tc_fence_after();
+        const uint64_t kd = make_smem_desc(smem_u32(k_slot(s)), 16, 1024);
+        const uint64_t vd = make_smem_desc(smem_u32(v_slot(s)), 16, 1024);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          mma_f16_ss(tmem + C::kColS + b * kMC, qd + kstep(k, C::kTileBoxBytes), kd + kstep(k, C::kBoxBytes), idesc_s, k != 0);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          mma_f16_ss(tmem + C::kColA + b * kMC, zd + kstep(k, C::kTileBoxBytes), vd + kstep(k, C::kBoxBytes), idesc_s, k != 0);
+        mma_commit(&bars->s_full[b]);
+      };
+      w.wait(&bars->qz_full, 0, 710);
+      issue_sd(0);
+      for (int j = 0; j < nchunks; ++j) {
+        // S_{j+1}, dA_{j+1} run while the threads work on chunk j; they overwrite the buffers dS_{j-1} was read from
+        // by the dQ product of chunk j-1, which was issued earlier and therefore executes first
+        if (j + 1 < nchunks) issue_sd(j + 1);
+        const int s = j % C::kStages, b = j & 1;
+        w.wait(&bars->p_full[b], (j >> 1) & 1, 712);
+        tc_fence_after();
+        const uint64_t kd = make_smem_desc(smem_u32(k_slot(s)), C::kBoxBytes, 1024);      // MN-major: rows = reduction
+#pragma unroll
+        for (int k = 0; k < kMC / 16; ++k)
+          mma_f16_ts(tmem + C::kColQ, tmem + C::kColS + b * kMC + k * 8, kd + (uint64_t)(k * 128), idesc_q, (uint32_t)((j | k) != 0));
+        mma_commit(&bars->empty[s]);
+      }
+      mma_commit(&bars->acc_done);
+    }
+  } else {
+    const int row = warp * 32 + lane, grow = row0 + row;
+    const bool live = grow < nq;
+    const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16);
+    const float l2e = 1.4426950408889634f;
+    const float L2 = live ? ws_LD[((int64_t)bh * nq + grow) * 2] * l2e : 0.f;
+    const float Dv = live ? ws_LD[((int64_t)bh * nq + grow) * 2 + 1] : 0.f;
+    const float scale_log2 = scale * l2e;
+    for (int j = 0; j < nchunks; ++j) {
+      const int b = j & 1;
+      w.wait(&bars->s_full[b], (j >> 1) & 1, 720);
+      tc_fence_after();
+#pragma unroll
+      for (int hlf = 0; hlf < 2; ++hlf) {
+        uint32_t sv[32], av[32];
+        tmem_ld_32x32b_x32(tbase + C::kColS + b * kMC + hlf * 32, sv);
+        tmem_ld_32x32b_x32(tbase + C::kColA + b * kMC + hlf * 32, av);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const float p0 = ex2f(fmaf(__uint_as_float(sv[e]), scale_log2, -L2));
+          const float p1 = ex2f(fmaf(__uint_as_float(sv[e + 1]), scale_log2, -L2));
+          const float d0 = live ? scale * p0 * (__uint_as_float(av[e]) - Dv) : 0.f;
+          const float d1 = live ? scale * p1 * (__uint_as_float(av[e + 1]) - Dv) : 0.f;
+          pk[e >> 1] = pack_bf16(d0, d1);
+        }
+        // dS over the first 32 columns of S[b]: the first half's 16 packed columns are written after both of its
+        // S columns groups ... the second half's S columns (32..63) are read before columns 16..31 are overwritten
+        if (hlf == 0) {
+          // columns 0..15 of S[b] hold scores this thread has already read (they are in sv)
+          tmem_st_32x32b_x16(tbase + C::kColS + b * kMC, pk);
+        } else {
+          tmem_st_32x32b_x16(tbase + C::kColS + b * kMC + 16, pk);
+        }
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(&bars->p_full[b]);
+    }
+    w.wait(&bars->acc_done, 0, 721);
+    tc_fence_after();
+    {
+      // the tensor-memory loads are warp-wide (every lane takes part); only the stores depend on the row
+      const bool store = live && !w.dead && *(volatile int*)&bars->abort == 0;
+      uint4* o = reinterpret_cast<uint4*>(dQ + ((int64_t)bh * nq + (live ? grow : 0)) * D);
+#pragma unroll
+      for (int c0 = 0; c0 < D; c0 += 16) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(tbase + C::kColQ + c0, r);
+        tmem_wait_ld();
+        const float* f = reinterpret_cast<const float*>(r);
+        if (store) {
+          o[c0 / 8] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+          o[c0 / 8 + 1] = make_uint4(pack_bf16(f[8], f[9]), pack_bf16(f[10], f[11]), pack_bf16(f[12], f[13]), pack_bf16(f[14], f[15]));
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 5) tmem_dealloc(tmem, C::kTmemCols);
+}
+
+template <int D>
+cudaError_t launch_recur(csat_ctx* c, const void* G, cudaStream_t s) {
+  using C = RCfg<D>;
+  const Params& p = c->p;
+  static DeviceFlags smem_opt_in;
+  cudaError_t e = ensure_dynamic_smem(bwd_recur_sm100_kernel<D>, (int)C::kSmemBytes, c->device, smem_opt_in);
+  if (e != cudaSuccess) return e;
+  const dim3 grid((unsigned)((p.nq + kRows - 1) / kRows), (unsigned)(p.B * p.H));
+  bwd_recur_sm100_kernel<D><<<grid, kRThreads, C::kSmemBytes, s>>>(
+      c->tmap_mats, c->bw_Z16, (const __nv_bfloat16*)G, c->bw_dZ16, c->bw_LD, c->bw_masks, c->thr(), c->thr_stride(),
+      (int)p.nq, (int)p.H, p.T, c->psi ? 1 : 0, c->status);
+  return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch_dq(csat_ctx* c, const void* Q, void* dQ, cudaStream_t s) {
+  using C = QCfg<D>;
+  const Params& p = c->p;
+  CUtensorMap tq, tz;
+  const uint64_t qd[3] = {(uint64_t)D, (uint64_t)p.nq, (uint64_t)(p.B * p.H)};
+  const uint64_t qs[2] = {(uint64_t)D * 2, (uint64_t)p.nq * D * 2};
+  const uint32_t qb[3] = {64, (uint32_t)kRows, 1};
+  cudaError_t e;
+  if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
+  if ((e = make_tmap_bf16_3d(&tz, c->bw_dZ16, qd, qs, qb)) != cudaSuccess) return e;
+  static DeviceFlags smem_opt_in;
+  if ((e = ensure_dynamic_smem(bwd_dq_sm100_kernel<D>, (int)C::kSmemBytes, c->device, smem_opt_in)) != cudaSuccess) return e;
+  const float scale = (float)(p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)D));
+  const dim3 grid((unsigned)((p.nq + kRows - 1) / kRows), (unsigned)(p.B * p.H));
+  bwd_dq_sm100_kernel<D><<<grid, kQThreads, C::kSmemBytes, s>>>(tq, tz, c->tmap_kv, (__nv_bfloat16*)dQ, c->bw_LD, (int)p.nq,
+                                                              (int)p.m, scale, c->status);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_sm100_bwd_recur(csat_ctx* c, const void* G, cudaStream_t s, int* launches) {
+  *launches += 1;
+  return c->p.d == 64 ? launch_recur<64>(c, G, s) : launch_recur<128>(c, G, s);
+}
+
+cudaError_t launch_sm100_bwd_dq(csat_ctx* c, const void* Q, void* dQ, cudaStream_t s, int* launches) {
+  *launches += 1;
+  return c->p.d == 64 ? launch_dq<64>(c, Q, dQ, s) : launch_dq<128>(c, Q, dQ, s);
+}
+
+}  // namespace csat

@@ -104,6 +104,8 @@ struct csat_ctx {
   float* bw_dZ = nullptr; float* bw_LD = nullptr; float* bw_dKV = nullptr; float* bw_WT = nullptr;
   __nv_bfloat16* bw_dKV16 = nullptr;     // bf16 copy of dK~|dV~ (operand of the tensor-core Phi^T product)
   __nv_bfloat16* bw_dZ16 = nullptr;      // bf16 copy of dZ (operand of the tensor-core dK~|dV~ stage)
+  __nv_bfloat16* bw_Z16 = nullptr;       // Z = A~ V~ as the forward rounds it (tensor-core per-query stages)
+  size_t bw_bytes_Z16 = 0;
   size_t bw_bytes_dZ = 0, bw_bytes_LD = 0, bw_bytes_dKV = 0, bw_bytes_WT = 0, bw_bytes_dKV16 = 0, bw_bytes_dZ16 = 0;
   // CSAT_KEEP_MASKS: the shrinkage decisions of the most recent csat_backward, one word per (b, h, query, column),
   // bit t = |x_t| > theta_t
@@ -180,6 +182,15 @@ cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cud
 cudaError_t make_attend_tmaps(csat_ctx* c);
 cudaError_t make_layer_weights_tmap(csat_ctx* c);
 cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
+// the attention phase alone: z_out [B,H,n_q,d] bf16 = Z, lse_out[row * lse_stride] = log sum exp of the row's scores
+cudaError_t launch_sm100_attend_lse(csat_ctx* c, const void* Q, void* z_out, float* lse_out, int lse_stride,
+                                    cudaStream_t s, int* launches);
+
+// bwd_rows_sm100.cu : the per-query stages of the backward on the tensor cores (bf16, d in {64, 128}, one S, B
+// for all layers).  recur: Z, G -> dZ (bf16 into bw_dZ16), D = <dZ, Z> (into bw_LD), optionally the masks;
+// dq: Q, dZ, L, D, K~|V~ -> dQ
+cudaError_t launch_sm100_bwd_recur(csat_ctx* c, const void* G, cudaStream_t s, int* launches);
+cudaError_t launch_sm100_bwd_dq(csat_ctx* c, const void* Q, void* dQ, cudaStream_t s, int* launches);
 
 // project_sm100.cu : input projections; one launch applies columns [col0, col0 + ncols) of W [dm, 3 H d] to
 // X [B, n_tok, dm] and writes the heads of Q / K / V those columns belong to

@@ -76,20 +76,31 @@ __global__ void __launch_bounds__(kThreads) fwht_compress_kernel(T* __restrict__
   const bool is_v = col0 >= d;
   const T* src = (is_v ? V : K) + (int64_t)bh * n * d + (is_v ? col0 - d : col0);
   const int hp = (is_v && sep) ? H + h : h;                // the generator's head: Phi_V of head h is head H + h
-  for (int j = threadIdx.x; j < N; j += kThreads) {
-    float v[CG];
-    if (j < n) {
-      const Vec<T, CG> in = *reinterpret_cast<const Vec<T, CG>*>(src + (int64_t)j * d);
-      const int64_t e = (int64_t)hp * n + j;
-      const bool neg = (sign_words[e >> 5] >> (e & 31)) & 1u;
+  // four token rows per thread and step: the loads are independent and all in flight together
+  constexpr int kU = 4;
+  for (int j0 = threadIdx.x; j0 < N; j0 += kThreads * kU) {
+    Vec<T, CG> in[kU];
+    uint32_t sw[kU];
 #pragma unroll
-      for (int c = 0; c < CG; ++c) v[c] = neg ? -to_f<T>(in.v[c]) : to_f<T>(in.v[c]);
-    } else {
-#pragma unroll
-      for (int c = 0; c < CG; ++c) v[c] = 0.f;
+    for (int u = 0; u < kU; ++u) {
+      const int j = j0 + u * kThreads;
+      if (j < n) {
+        in[u] = *reinterpret_cast<const Vec<T, CG>*>(src + (int64_t)j * d);
+        const int64_t e = (int64_t)hp * n + j;
+        sw[u] = sign_words[e >> 5] >> (e & 31);
+      }
     }
 #pragma unroll
-    for (int c = 0; c < CG; ++c) xs[c * Np + pad(j)] = v[c];
+    for (int u = 0; u < kU; ++u) {
+      const int j = j0 + u * kThreads;
+      if (j >= N) continue;
+      const bool live = j < n, neg = live && (sw[u] & 1u);
+#pragma unroll
+      for (int c = 0; c < CG; ++c) {
+        const float x = live ? to_f<T>(in[u].v[c]) : 0.f;
+        xs[c * Np + pad(j)] = neg ? -x : x;
+      }
+    }
   }
   __syncthreads();
   int s = 0;
@@ -132,9 +143,9 @@ cudaError_t launch_cg(csat_ctx* c, const void* K, const void* V, cudaStream_t s,
 
 template <typename T>
 cudaError_t launch_t(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int log2N) {
-  // columns per CTA: as many as keep the CTA's [CG][N] float32 tile within shared memory (<= 136 KB here)
-  if (log2N <= 12) return launch_cg<T, 8>(c, K, V, s, log2N);
-  if (log2N == 13) return launch_cg<T, 4>(c, K, V, s, log2N);
+  // columns per CTA: the CTA's [CG][N] float32 tile takes ~68 KB (three CTAs per SM), 136 KB at N = 16384
+  if (log2N <= 11) return launch_cg<T, 8>(c, K, V, s, log2N);
+  if (log2N == 12) return launch_cg<T, 4>(c, K, V, s, log2N);
   return launch_cg<T, 2>(c, K, V, s, log2N);
 }
 

@@ -72,14 +72,23 @@ __global__ void phi_gen_kernel(T* __restrict__ phi, int64_t total, int64_t n, in
 // are walked by stepping (one 64-bit division per thread, outside the loop).
 // Cost: Philox4x32-10 alone is 20 wide multiplies, 20 three-input xors and 20 key additions per four elements, so
 // the kernel is bound by integer arithmetic, not by the 2 bytes it writes per element.
+// ((u >> 9) + 0.5) * 2^-23 without an integer-to-float conversion: 1 + k 2^-23 is the float with mantissa field k,
+// and subtracting 1 - 2^-24 from it is exact
+__device__ __forceinline__ float uniform23_bits(uint32_t u) {
+  return __uint_as_float(0x3f800000u | (u >> 9)) - 0.99999994039535522461f;
+}
+
 __device__ __forceinline__ void box_muller_bf16(uint32_t ua, uint32_t ub, float c, float& g0, float& g1) {
   float r;
   {
-    const float r2 = c * __log2f(uniform23(ua));
+    const float r2 = c * __log2f(uniform23_bits(ua));
     asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(r2));
   }
-  const float x = 2.0f * uniform23(ub);
-  const float kf = rintf(2.0f * x);
+  const float x = 2.0f * uniform23_bits(ub);
+  // k = nearest integer to 2 x (0 .. 4): the low mantissa bits of 2 x + 1.5 * 2^23 hold it
+  const float tk = fmaf(2.0f, x, 12582912.f);
+  const float kf = tk - 12582912.f;
+  const uint32_t k = __float_as_uint(tk);
   const float y = 3.14159265358979f * fmaf(kf, -0.5f, x);
   const float y2 = y * y;
   float sn = fmaf(y2, -1.9841270e-4f, 8.3333333e-3f);
@@ -89,11 +98,10 @@ __device__ __forceinline__ void box_muller_bf16(uint32_t ua, uint32_t ub, float 
   cs = fmaf(cs, y2, 4.1666667e-2f);
   cs = fmaf(cs, y2, -0.5f);
   cs = fmaf(cs, y2, 1.0f);
-  const int k = (int)kf;
-  const float sa = (k & 1) ? cs : sn, ca = (k & 1) ? sn : cs;
-  // quadrant 0: (s, c); 1: (c, -s); 2: (-s, -c); 3: (-c, s)
-  const float s_out = (k & 2) ? -sa : sa;
-  const float c_out = ((k + 1) & 2) ? -ca : ca;
+  const float sa = (k & 1u) ? cs : sn, ca = (k & 1u) ? sn : cs;
+  // quadrant 0: (s, c); 1: (c, -s); 2: (-s, -c); 3: (-c, s): the sign bits come from bit 1 of k and of k + 1
+  const float s_out = __uint_as_float(__float_as_uint(sa) ^ ((k & 2u) << 30));
+  const float c_out = __uint_as_float(__float_as_uint(ca) ^ (((k + 1u) & 2u) << 30));
   g0 = r * c_out;
   g1 = r * s_out;
 }
@@ -206,12 +214,12 @@ __global__ void phi_rademacher_vec_kernel(T* __restrict__ phi, int64_t total, in
 // block (e / 128, 0, 2, 0), e = h n + j.  One thread per V consecutive columns of one row (V = 8 when n % 8 == 0:
 // the eight sign bits are one byte of one word, and the store is one 16-byte vector for bf16).
 template <typename T, int V>
-__global__ void phi_hadamard_kernel(T* __restrict__ phi, int64_t n, int64_t n_pad, int64_t m, uint32_t log2N,
-                                    float inv_sqrt_m, uint32_t k0, uint32_t k1) {
-  const int64_t row = blockIdx.y;                        // h * m + r
-  const int64_t h = row / m, r = row - h * m;
+__global__ void phi_hadamard_kernel(T* __restrict__ phi, int64_t n, int64_t n_pad, int64_t m, int64_t rows,
+                                    uint32_t log2N, float inv_sqrt_m, uint32_t k0, uint32_t k1) {
   const int64_t j0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * V;
   if (j0 >= n) return;
+  for (int64_t row = blockIdx.y; row < rows; row += gridDim.y) {     // row = h * m + r
+  const int64_t h = row / m, r = row - h * m;
   const U4 ab = philox4x32_10(U4{(uint32_t)h, 0u, 3u, 0u}, k0, k1);
   const uint64_t a = 2ull * ab.x + 1ull, b = ab.y;
   const uint32_t ir = (uint32_t)((a * (uint64_t)r + b) & ((1ull << log2N) - 1ull));
@@ -234,6 +242,7 @@ __global__ void phi_hadamard_kernel(T* __restrict__ phi, int64_t n, int64_t n_pa
     if (sizeof(T) == 4) reinterpret_cast<uint4*>(dst)[1] = src[1];
   } else {
     dst[0] = v[0];
+  }
   }
 }
 
@@ -279,7 +288,9 @@ size_t elt_size(int dtype) { return dtype == CSAT_DTYPE_FP32 ? 4 : 2; }
 
 cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s) {
   const int64_t total = p.H * p.m * p.n;
-  cudaError_t e = cudaMemsetAsync(phi, 0, (size_t)(p.H * p.m * p.n_pad) * elt_size(p.dtype), s);
+  cudaError_t e = cudaSuccess;
+  if (p.n_pad != p.n)      // the padding columns must hold zeros; without padding every element is written below
+    e = cudaMemsetAsync(phi, 0, (size_t)(p.H * p.m * p.n_pad) * elt_size(p.dtype), s);
   if (e != cudaSuccess) return e;
   const float inv = (float)(1.0 / sqrt((double)p.m));
   const uint32_t k0 = (uint32_t)(p.seed & 0xFFFFFFFFull), k1 = (uint32_t)(p.seed >> 32);
@@ -287,11 +298,10 @@ cudaError_t launch_phi_gen(void* phi, const Params& p, cudaStream_t s) {
     uint32_t log2N = 0;
     while (((int64_t)1 << log2N) < p.n) ++log2N;
     const int64_t rows = p.H * p.m;
-    if (rows > 65535) return cudaErrorInvalidValue;      // one grid row per row of Phi
     const bool vec = p.n % 8 == 0;
     const int64_t per_row = vec ? p.n / 8 : p.n;
-    const dim3 grid((unsigned)((per_row + 127) / 128), (unsigned)rows);
-#define CSAT_HAD(T, V) phi_hadamard_kernel<T, V><<<grid, 128, 0, s>>>((T*)phi, p.n, p.n_pad, p.m, log2N, inv, k0, k1)
+    const dim3 grid((unsigned)((per_row + 127) / 128), (unsigned)(rows < 65535 ? rows : 65535));   // rows beyond: strided
+#define CSAT_HAD(T, V) phi_hadamard_kernel<T, V><<<grid, 128, 0, s>>>((T*)phi, p.n, p.n_pad, p.m, rows, log2N, inv, k0, k1)
     if (p.dtype == CSAT_DTYPE_FP32) { if (vec) CSAT_HAD(float, 8); else CSAT_HAD(float, 1); }
     else { if (vec) CSAT_HAD(__nv_bfloat16, 8); else CSAT_HAD(__nv_bfloat16, 1); }
 #undef CSAT_HAD
