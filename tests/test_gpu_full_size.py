@@ -129,3 +129,52 @@ def test_untied_layers_at_the_full_workload_shape(key, pairs):
     torch.cuda.synchronize()
     assert torch.equal(oh, out.cpu())
     ctx.close()
+
+
+@pytest.mark.parametrize("key,pairs", [("c3", [(0, 0), (7, 11)]), ("c4", [(15, 7)]), ("c2", [(0, 0), (31, 11)])])
+def test_backward_at_the_full_workload_shape(key, pairs):
+    """csat_backward on the whole workload (thousands of query tiles through the tensor-core stages): sampled
+    (batch, head) pairs against the oracle, which differentiates with the library's own shrinkage decisions (see
+    tests/test_gpu_backward.py for why); no NaN/Inf anywhere; bit-identical rerun.  lambda is the one that keeps about
+    half of the first layer's coefficients, so that the decoder's backward has work to do."""
+    from paper_2507_02957_b200 import binding
+    from gpu_util import to_dev
+    w = wl.CONFIGS[key]
+    inp = wl.make_inputs(w)
+    Q, K, V, Psi = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    if Psi is not None:
+        ctx.set_dictionary(Psi)
+    binding.csat_set_i64(ctx.h, binding.CSAT_KEEP_MASKS, 1)
+    phi = ctx.get_phi()
+    psi64 = None if inp["Psi"] is None else inp["Psi"].astype(np.float64)
+    st = {}
+    orc.csat_forward_head(inp["Q"][0, 0], inp["K"][0, 0], inp["V"][0, 0], to_np(phi[0]), T=1, lam=0.0, Psi=psi64, stages=st)
+    lam = float(np.median(np.abs(st["Z"] @ st["B_dec"])) / st["mu"])
+    ctx.set(lam=lam)
+    G = wl.round_to_storage(np.random.default_rng(303).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    Gd = to_dev(G, w.dtype)
+    dQ, dK, dV = ctx.backward(Q, K, V, Gd)
+    for t in (dQ, dK, dV):
+        assert torch.isfinite(t).all()
+    words = ctx.backward_masks()
+    again = ctx.backward(Q, K, V, Gd)
+    assert all(torch.equal(a, b) for a, b in zip((dQ, dK, dV), again))
+    for (b, h) in pairs:
+        mw = words[b, h].cpu().numpy().astype(np.uint32)
+        masks = np.stack([(mw >> t) & 1 for t in range(w.T)]).astype(bool)
+        stg = {}
+        ref = orc.csat_backward_head(inp["Q"][b, h], inp["K"][b, h], inp["V"][b, h], to_np(phi[h]), G[b, h], T=w.T, lam=lam,
+                                     Psi=psi64, masks=masks, stages=stg)
+        differ = masks != stg["masks"]
+        assert differ.mean() <= 2e-2, (key, b, h, differ.mean())
+        bar = TOL[w.dtype] * np.abs(stg["xs"]).max(axis=(1, 2), keepdims=True)
+        st1 = {}
+        orc.csat_forward_head(inp["Q"][b, h][:1], inp["K"][b, h], inp["V"][b, h], to_np(phi[h]), T=1, lam=lam, Psi=psi64, stages=st1)
+        dist = np.abs(np.abs(stg["xs"]) - st1["theta"])
+        assert (dist[differ] <= np.broadcast_to(bar, dist.shape)[differ]).all(), (key, b, h)
+        for nm, g, rf in zip(("dQ", "dK", "dV"), (dQ, dK, dV), ref):
+            assert np.abs(rf).max() > 0
+            err = rel_err(to_np(g[b, h]), rf)
+            assert err <= TOL[w.dtype], (key, b, h, nm, err)
+    ctx.close()
