@@ -197,13 +197,17 @@ struct Waiter {
   }
 };
 
-template <int D, bool kUntied>
+// kMasks (backward pass only, one S, B for all layers): besides the output the kernel leaves what the backward needs:
+// Z (bf16, as fed to the first product), every row's log sum exp, and the decision |x_t| > theta_t of every layer,
+// one bit per column: word c / 32 of (layer, row), bit 31 - c % 32.
+template <int D, bool kUntied, bool kMasks>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
                             int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status,
-                            float* __restrict__ lse_out, int lse_stride) {
+                            float* __restrict__ lse_out, int lse_stride, __nv_bfloat16* __restrict__ z_out,
+                            uint32_t* __restrict__ mask_out) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
@@ -659,6 +663,25 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           for (int e = 0; e < 16; e += 2) v2[(c0 + e) >> 1] = mul2(pack2u(a[e], a[e + 1]), inv2);
         }
       }
+      const int grow_m = row0 + t * kRows + row;                // this thread's query (may lie beyond n_q)
+      if (kMasks && z_out != nullptr && grow_m < nq) {
+        uint4* zo = reinterpret_cast<uint4*>(z_out + ((int64_t)bh * nq + grow_m) * D);
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+          float x[8];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) unpack2(v2[c * 4 + u], x[2 * u], x[2 * u + 1]);
+          zo[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+        }
+      }
+      uint32_t mw[D / 32];                                      // kMasks: the current layer's decisions
+      auto store_masks = [&](int layer) {
+        if (kMasks && mask_out != nullptr && grow_m < nq) {
+          uint32_t* mo = mask_out + (((int64_t)bh * T + layer) * nq + grow_m) * (D / 32);
+          if (D == 128) *reinterpret_cast<uint4*>(mo) = make_uint4(mw[0], mw[1], mw[2], mw[D / 32 - 1]);
+          else *reinterpret_cast<uint2*>(mo) = make_uint2(mw[0], mw[1]);
+        }
+      };
       auto publish = [&](uint32_t col) {                        // v2 as a bf16 A operand, from column col of S on
         const uint32_t op_addr = tbase + C::kColS + col;
 #pragma unroll
@@ -791,6 +814,10 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                 const uint64_t x2 = add2(v2[(c0 + e) >> 1], r2);               // alpha^t S + z B
                 float x0, x1;
                 unpack2(x2, x0, x1);
+                if (kMasks) {                                                  // the sign bit of theta - |x| is the decision
+                  mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x0)), mw[c0 >> 5], 1);
+                  mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x1)), mw[c0 >> 5], 1);
+                }
                 const uint64_t t2 = pack2(fma_sat(x0, inv2th, 0.5f), fma_sat(x1, inv2th, 0.5f));
                 uint64_t bn = fma2(t2, m2th2, x2);                             // eta_theta(x) - theta
                 uint64_t dn = fma2(t2, m2th2, r2);                             // alpha^{t+1} - alpha^t
@@ -816,6 +843,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(&bars->a_full[t]);
+            store_masks(it);
           }
         };
         if (theta_stride != 0) iterate(std::true_type{}); else iterate(std::false_type{});
@@ -833,9 +861,14 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             float b0, b1;
             unpack2(v2[(c0 + e) >> 1], b0, b1);
             const float x0 = b0 + __uint_as_float(r[e]), x1 = b1 + __uint_as_float(r[e + 1]);
+            if (kMasks) {
+              mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x0)), mw[c0 >> 5], 1);
+              mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x1)), mw[c0 >> 5], 1);
+            }
             v2[(c0 + e) >> 1] = pack2(x0 - fminf(fmaxf(x0, -th), th), x1 - fminf(fmaxf(x1, -th), th));
           }
         }
+        store_masks(T - 1);
         if (has_psi) {
           publish(0);
           w.wait(&bars->r_full[t], phase & 1, 232); ++phase;
@@ -851,7 +884,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         }
       }
       const int grow = row0 + t * kRows + row;
-      if (grow < nq && !w.dead && *(volatile int*)&bars->abort == 0) {
+      if (out != nullptr && grow < nq && !w.dead && *(volatile int*)&bars->abort == 0) {
         // a row is a multiple of 128 bytes; where the output is 32-byte aligned every store covers whole
         // 32-byte sectors (the lanes of a warp write different rows), otherwise 16-byte stores
         __nv_bfloat16* orow = out + ((int64_t)bh * nq + grow) * D;
@@ -885,8 +918,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   if (warp == kMmaWarp) tmem_dealloc(tmem, C::kTmemCols);
 }
 
-template <int D, bool kUntied>
-cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T, float* lse_out, int lse_stride) {
+template <int D, bool kUntied, bool kMasks = false>
+cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T, float* lse_out, int lse_stride,
+                   __nv_bfloat16* z_out = nullptr, uint32_t* mask_out = nullptr) {
   using C = Cfg<D>;
   const Params& p = c->p;
   CUtensorMap tq;
@@ -896,7 +930,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
   static DeviceFlags smem_opt_in;
-  if ((e = ensure_dynamic_smem(attend_recover_sm100_kernel<D, kUntied>, (int)C::kSmemBytes, c->device, smem_opt_in)) !=
+  if ((e = ensure_dynamic_smem(attend_recover_sm100_kernel<D, kUntied, kMasks>, (int)C::kSmemBytes, c->device, smem_opt_in)) !=
       cudaSuccess)
     return e;
   const double scale = p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)D);
@@ -908,9 +942,9 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   if (n_items > (int64_t)1 << 30) return cudaErrorInvalidValue;
   const int sms = c->sms;
   const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
-  attend_recover_sm100_kernel<D, kUntied><<<grid, kThreads, C::kSmemBytes, s>>>(
+  attend_recover_sm100_kernel<D, kUntied, kMasks><<<grid, kThreads, C::kSmemBytes, s>>>(
       tq, c->tmap_kv, kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, T,
-      c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, (int)c->bh0, c->status, lse_out, lse_stride);
+      c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out);
   return cudaGetLastError();
 }
 
@@ -947,12 +981,13 @@ cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, c
   return c->p.d == 64 ? launch<64, false>(c, Q, out, s, c->p.T, nullptr, 0) : launch<128, false>(c, Q, out, s, c->p.T, nullptr, 0);
 }
 
-// Z = A~ V~ (recovery disabled whatever CSAT_T says) and the rows' log sum exp, for the backward pass
-cudaError_t launch_sm100_attend_lse(csat_ctx* c, const void* Q, void* z_out, float* lse_out, int lse_stride,
-                                    cudaStream_t s, int* launches) {
+// The forward with what the backward pass needs as its only outputs: Z (bf16), the rows' log sum exp and the layers'
+// shrinkage decisions (one S, B for all layers; the decoded output itself is not stored)
+cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bfloat16* z_out, float* lse_out,
+                                             int lse_stride, uint32_t* mask_out, cudaStream_t s, int* launches) {
   *launches += 1;
-  return c->p.d == 64 ? launch<64, false>(c, Q, z_out, s, 0, lse_out, lse_stride)
-                      : launch<128, false>(c, Q, z_out, s, 0, lse_out, lse_stride);
+  return c->p.d == 64 ? launch<64, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out)
+                      : launch<128, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out);
 }
 
 }  // namespace csat

@@ -78,6 +78,22 @@ __global__ void transpose_kernel(float* __restrict__ out, const float* __restric
   }
 }
 
+// out[(bh, row, c)] = sum over layers t of bit_t << t, from the forward kernel's record [bh][t][row][d / 32] in which
+// column c is bit 31 - c % 32 of word c / 32
+__global__ void expand_masks_kernel(uint32_t* __restrict__ out, const uint32_t* __restrict__ bits, int64_t total,
+                                    int64_t nq, int d, int T) {
+  const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int c = (int)(i % d);
+  const int64_t row = (i / d) % nq, bh = i / (d * nq);
+  uint32_t wv = 0;
+  for (int t = 0; t < T; ++t) {
+    const uint32_t m = bits[((bh * T + t) * nq + row) * (d / 32) + (c >> 5)];
+    wv |= ((m >> (31 - (c & 31))) & 1u) << t;
+  }
+  out[i] = wv;
+}
+
 template <typename T, int DC>   // DC = ceil(d / 32)
 __global__ void __launch_bounds__(kRowWarps * 32) bwd_rows_kernel(
     T* __restrict__ dQ, float* __restrict__ ws_dZ, __nv_bfloat16* __restrict__ ws_dZ16, float* __restrict__ ws_LD,
@@ -395,8 +411,14 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   const bool tc_stages = c->bw_dKV16 != nullptr && c->bw_dZ16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
   // ... and with one S, B for all layers the per-query stages too: the forward's attention phase leaves Z and the
   // rows' log sum exp, then the recurrence (forward with its decisions recorded, and backward) and dQ
-  if (tc_stages && !c->w_untied && c->bw_Z16 != nullptr) {
-    if ((e = launch_sm100_attend_lse(c, Q, c->bw_Z16, c->bw_LD, 2, s, launches)) != cudaSuccess) return e;
+  if (tc_stages && !c->w_untied && c->bw_Z16 != nullptr && (p.T == 0 || c->bw_maskbits != nullptr)) {
+    if ((e = launch_sm100_attend_for_backward(c, Q, c->bw_Z16, c->bw_LD, 2, c->bw_maskbits, s, launches)) != cudaSuccess) return e;
+    if (c->bw_masks != nullptr && p.T > 0) {           // CSAT_KEEP_MASKS: the decisions in the exported layout
+      const int64_t total = p.B * p.H * p.nq * p.d;
+      expand_masks_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(c->bw_masks, c->bw_maskbits, total, p.nq, d, p.T);
+      if ((e = cudaGetLastError()) != cudaSuccess) return e;
+      *launches += 1;
+    }
     if ((e = launch_sm100_bwd_recur(c, G, s, launches)) != cudaSuccess) return e;
     if ((e = launch_sm100_bwd_dq(c, Q, dQ, s, launches)) != cudaSuccess) return e;
     if ((e = launch_sm100_bwd_cols(c, Q, s, launches)) != cudaSuccess) return e;

@@ -5,19 +5,19 @@
 // where |x| > theta and 0 elsewhere.
 //
 // Before these kernels the forward's own kernels have left K~|V~ in the workspace, Z (bf16, as the forward rounds it
-// for its first product) in bw_Z16 and every row's log sum exp L in bw_LD.
+// for its first product) in bw_Z16, every row's log sum exp L in bw_LD and the layers' shrinkage decisions in
+// bw_maskbits.
 //
-// bwd_recur_sm100_kernel, one CTA per tile of 128 queries (TMEM lane = query row, one thread per row):
-//   1. the forward recurrence exactly as the forward kernel runs it (increment form: the accumulator holds
-//      r_t = theta + z B - a^_t (mu G), the registers b_t = alpha^t - theta; bf16 increments feed one MMA per layer),
-//      recording the decision |x_t| > theta_t of every layer as bit t of a word per (row, column) in tensor memory;
-//   2. d alpha_T = G Psi (one MMA; G itself without a dictionary), then for t = T-1 .. 0
+// bwd_recur_sm100_kernel, one CTA per tile of 128 queries (TMEM lane = query row, one thread per row): the recurrence
+// run backwards.  The decisions |x_t| > theta_t are the forward kernel's own (it records them, one bit per column and
+// layer, when it runs for the backward pass), so nothing of the forward recurrence is repeated here:
+//   d alpha_T = G Psi (one MMA; G itself without a dictionary), then for t = T-1 .. 0
 //        dx_t = d alpha_{t+1} o mask_t,   dZ += dx_t B^T,   d alpha_t = dx_t S^T = dx_t + dx_t (S - I)^T :
-//      dx_t goes to tensor memory as the bf16 A operand of two MMAs, whose B operands are the forward's own
-//      shared-memory tiles of S - I and B read as MN-major operands (a d x d tile with 128-byte rows is K-major when
-//      its rows are the output columns and MN-major when they are the reduction index: the transposed product needs
-//      no transposed copy); the identity part of S^T stays exact in float32 registers;
-//   3. dZ (bf16, the operand of the stages that follow) and D = <dZ, Z>.
+//   dx_t goes to tensor memory as the bf16 A operand of two MMAs, whose B operands are the forward's own
+//   shared-memory tiles of S - I and B read as MN-major operands (a d x d tile with 128-byte rows is K-major when
+//   its rows are the output columns and MN-major when they are the reduction index: the transposed product needs
+//   no transposed copy); the identity part of S^T stays exact in float32 registers;
+//   at the end dZ (bf16, the operand of the stages that follow) and D = <dZ, Z>.
 //
 // bwd_dq_sm100_kernel, one CTA per tile of 128 queries, K~|V~ streamed in chunks of 64 measurements:
 //        S_j = Q K~_j^T,  dA_j = dZ V~_j^T                        (two SS MMAs into tensor memory)
@@ -66,7 +66,7 @@ struct Waiter {
 };
 
 // ====================================================================================================================
-// recurrence forward (masks) and backward
+// recurrence backward
 // ====================================================================================================================
 template <int D> struct RCfg {
   static constexpr int kDBoxes = D / 64;
@@ -75,10 +75,10 @@ template <int D> struct RCfg {
   static constexpr uint32_t kOffMat = 0;                          // [3]: S - I | B^T | Psi, as the forward stages them
   static constexpr uint32_t kOffBar = 3 * kMatBytes;
   static constexpr uint32_t kSmemBytes = kOffBar + 128 + 1024 /*alignment slack*/;
-  // TMEM columns: accumulator | dZ accumulator | masks (one word per column) | bf16 operand (two per column)
-  static constexpr uint32_t kColAcc = 0, kColDz = D, kColMask = 2 * D, kColOp = 3 * D;
+  // TMEM columns: accumulator | dZ accumulator | bf16 operand (two per column)
+  static constexpr uint32_t kColAcc = 0, kColDz = D, kColOp = 2 * D;
   static constexpr uint32_t kTmemCols = (D == 64) ? 256 : 512;
-  static_assert(3 * D + D / 2 <= kTmemCols, "TMEM budget");
+  static_assert(2 * D + D / 2 <= kTmemCols, "TMEM budget");
 };
 
 struct RBars {
@@ -93,8 +93,7 @@ template <int D>
 __global__ void __launch_bounds__(kRThreads, 1)
 bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv_bfloat16* __restrict__ Z16,
                        const __nv_bfloat16* __restrict__ G, __nv_bfloat16* __restrict__ dZ16, float* __restrict__ ws_LD,
-                       uint32_t* __restrict__ ws_masks, const float* __restrict__ theta, int theta_stride, int nq, int H,
-                       int T, int has_psi, int* status) {
+                       const uint32_t* __restrict__ maskbits, int nq, int H, int T, int has_psi, int* status) {
   using C = RCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -129,24 +128,12 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
         for (int gx = 0; gx < C::kDBoxes; ++gx)
           tma_load_3d(smem + C::kOffMat + mat * C::kMatBytes + gx * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, gx * 64,
                       0, h * 3 + mat);
-      constexpr uint32_t idesc_f = make_idesc_bf16(kRows, D, false, false);   // forward products: B K-major
       constexpr uint32_t idesc_t = make_idesc_bf16(kRows, D, false, true);    // transposed products: B MN-major
-      auto mat_k = [&](int mat) { return make_smem_desc(smem_u32(smem + C::kOffMat + mat * C::kMatBytes), 16, 1024); };
-      auto mat_mn = [&](int mat) {
-        return make_smem_desc(smem_u32(smem + C::kOffMat + mat * C::kMatBytes), C::kMatBoxBytes, 1024);
-      };
       const uint32_t op = tmem + C::kColOp, acc = tmem + C::kColAcc, dz = tmem + C::kColDz;
-      // product with the matrix as the forward stores it (K-major): K step k lies in box k / 4, 32 (k % 4) bytes in
-      auto mma_fwd = [&](uint32_t d_t, int mat, uint32_t accumulate) {
-        const uint64_t bd = mat_k(mat);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k)
-          mma_f16_ts(d_t, op + k * 8, bd + (uint64_t)((k / 4) * (C::kMatBoxBytes >> 4) + (k % 4) * 2), idesc_f,
-                     k == 0 ? accumulate : 1u);
-      };
-      // product with its transpose: the tile's rows are the reduction index, 16 rows (2048 bytes) per K step
+      // product with the transpose of a matrix the forward stores [output column][k]: the tile's rows are now the
+      // reduction index, 16 rows (2048 bytes) per K step, the next 64 output columns one box further
       auto mma_tr = [&](uint32_t d_t, int mat, uint32_t accumulate) {
-        const uint64_t bd = mat_mn(mat);
+        const uint64_t bd = make_smem_desc(smem_u32(smem + C::kOffMat + mat * C::kMatBytes), C::kMatBoxBytes, 1024);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) mma_f16_ts(d_t, op + k * 8, bd + (uint64_t)(k * 128), idesc_t, k == 0 ? accumulate : 1u);
       };
@@ -157,25 +144,15 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
         tc_fence_after();
       };
       w.wait(&bars->mats_full, 0, 600);
-      // forward: r_0 = kappa + z B, then T - 1 increments times S - I
-      operand_ready();
-      mma_fwd(acc, 1, 1u);
-      mma_commit(&bars->r_full);
-      for (int it = 0; it + 1 < T; ++it) {
-        operand_ready();
-        mma_fwd(acc, 0, 1u);
-        mma_commit(&bars->r_full);
-      }
-      // backward: d alpha_T = G Psi
-      if (has_psi) {
+      if (has_psi) {                                           // d alpha_T = G Psi
         operand_ready();
         mma_tr(acc, 2, 0u);
         mma_commit(&bars->r_full);
       }
       for (int t = T - 1; t >= 0; --t) {
         operand_ready();
-        if (t > 0) mma_tr(acc, 0, 0u);                       // dx_t (S - I)^T
-        mma_tr(dz, 1, t == T - 1 ? 0u : 1u);                 // dZ += dx_t B^T
+        if (t > 0) mma_tr(acc, 0, 0u);                         // dx_t (S - I)^T
+        mma_tr(dz, 1, t == T - 1 ? 0u : 1u);                   // dZ += dx_t B^T
         mma_commit(&bars->r_full);
       }
       if (w.dead) mbar_wait_drain(&bars->mats_full, 0);
@@ -186,11 +163,10 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
     const int grow = row0 + row;
     const bool live = grow < nq;
     const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16);
-    const uint32_t acc_addr = tbase + C::kColAcc, dz_addr = tbase + C::kColDz, mask_addr = tbase + C::kColMask,
-                   op_addr = tbase + C::kColOp;
+    const uint32_t acc_addr = tbase + C::kColAcc, dz_addr = tbase + C::kColDz, op_addr = tbase + C::kColOp;
     const int64_t goff = ((int64_t)bh * nq + (live ? grow : 0)) * D;
     int phase = 0;
-    float v[D];                                   // b_t = alpha^t - kappa, later d alpha / dx
+    float v[D];                                   // d alpha_{t+1}, then dx_t
     auto publish_bf16 = [&]() {                   // v as the bf16 A operand
 #pragma unroll
       for (int c0 = 0; c0 < D; c0 += 16) {
@@ -203,8 +179,8 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
       tc_fence_before();
       mbar_arrive(&bars->a_full);
     };
-    auto load_row = [&](const __nv_bfloat16* src) {       // v := the row of a [B,H,n_q,d] bf16 tensor (0 beyond n_q)
-      const uint4* p = reinterpret_cast<const uint4*>(src + goff);
+    {                                             // v := the row of the output gradient (0 beyond n_q)
+      const uint4* p = reinterpret_cast<const uint4*>(G + goff);
 #pragma unroll
       for (int c = 0; c < D / 8; ++c) {
         const uint4 q = live ? p[c] : make_uint4(0, 0, 0, 0);
@@ -213,98 +189,8 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
         v[8 * c + 4] = bf16_lo(q.z); v[8 * c + 5] = bf16_hi(q.z);
         v[8 * c + 6] = bf16_lo(q.w); v[8 * c + 7] = bf16_hi(q.w);
       }
-    };
-    if (T == 0) {
-      // no decoder: dZ = G, D = <G, Z>
-      load_row(G);
-      float dsum = 0.f;
-      const uint4* zp = reinterpret_cast<const uint4*>(Z16 + goff);
-      uint4* out = reinterpret_cast<uint4*>(dZ16 + goff);
-#pragma unroll
-      for (int c = 0; c < D / 8; ++c) {
-        const uint4 z = live ? zp[c] : make_uint4(0, 0, 0, 0);
-        dsum = fmaf(v[8 * c + 0], bf16_lo(z.x), dsum); dsum = fmaf(v[8 * c + 1], bf16_hi(z.x), dsum);
-        dsum = fmaf(v[8 * c + 2], bf16_lo(z.y), dsum); dsum = fmaf(v[8 * c + 3], bf16_hi(z.y), dsum);
-        dsum = fmaf(v[8 * c + 4], bf16_lo(z.z), dsum); dsum = fmaf(v[8 * c + 5], bf16_hi(z.z), dsum);
-        dsum = fmaf(v[8 * c + 6], bf16_lo(z.w), dsum); dsum = fmaf(v[8 * c + 7], bf16_hi(z.w), dsum);
-        if (live)
-          out[c] = make_uint4(pack_bf16(v[8 * c], v[8 * c + 1]), pack_bf16(v[8 * c + 2], v[8 * c + 3]),
-                              pack_bf16(v[8 * c + 4], v[8 * c + 5]), pack_bf16(v[8 * c + 6], v[8 * c + 7]));
-      }
-      if (live) ws_LD[((int64_t)bh * nq + grow) * 2 + 1] = dsum;
-    } else {
-      // ---- forward recurrence, as the forward kernel runs it, with the decisions recorded ----
-      const float kappa = theta[h];
-      {
-        uint32_t tb[16];
-#pragma unroll
-        for (int e = 0; e < 16; ++e) tb[e] = __float_as_uint(kappa);
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 16) tmem_st_32x32b_x16(acc_addr + c0, tb);      // accumulator := kappa
-      }
-      load_row(Z16);
-      publish_bf16();                                                                 // z as the A operand of z B
-#pragma unroll
-      for (int i = 0; i < D; ++i) v[i] = -kappa;                                      // alpha^0 = 0
-      for (int it = 0; it < T; ++it) {
-        const float th = theta[(int64_t)it * theta_stride + h];
-        const bool last = it == T - 1;
-        const float inv2th = th > 0.f ? 0.5f / th : 0.f;
-        const float dk = th - kappa;
-        w.wait(&bars->r_full, phase & 1, 610); ++phase;
-        tc_fence_after();
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 16) {
-          uint32_t r[16], mk[16];
-          tmem_ld_32x32b_x16(acc_addr + c0, r);
-          if (it > 0) tmem_ld_32x32b_x16(mask_addr + c0, mk);
-          tmem_wait_ld();
-          uint32_t pk[8];
-#pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const float rr = __uint_as_float(r[e]);
-            const float x = v[c0 + e] + rr;                     // alpha^t S + z B - (kappa - kappa)
-            uint32_t bit;
-            float inc;
-            if (!last) {
-              // saturating form, as in the forward: s in {0, 1} exactly where |x| >= theta
-              const float s = fma_sat(x, inv2th, 0.5f);
-              const float bn = fmaf(s, -2.f * th, x) + dk;      // eta_theta(x) - kappa
-              inc = fmaf(s, -2.f * th, rr) + dk;                // alpha^{t+1} - alpha^t
-              v[c0 + e] = bn;
-              bit = (__float_as_uint(s) - 1u >= 0x3f7fffffu) ? 1u : 0u;
-              if (th == 0.f) bit = 1u;                          // eta_0 is the identity
-            } else {
-              inc = 0.f;
-              bit = fabsf(x) > th ? 1u : 0u;
-            }
-            if (e & 1) pk[e >> 1] = pack_bf16(__uint_as_float(pk[e >> 1]), inc); else pk[e >> 1] = __float_as_uint(inc);
-            mk[e] = (it > 0 ? mk[e] : 0u) | (bit << it);
-          }
-          tmem_st_32x32b_x16(mask_addr + c0, mk);
-          if (!last) tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
-        }
-        tmem_wait_st();
-        if (!last) {
-          tc_fence_before();
-          mbar_arrive(&bars->a_full);
-        }
-      }
-      if (ws_masks != nullptr) {              // (the tensor-memory loads are warp-wide: every lane takes part)
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 16) {
-          uint32_t mk[16];
-          tmem_ld_32x32b_x16(mask_addr + c0, mk);
-          tmem_wait_ld();
-          if (live) {
-            uint4* o = reinterpret_cast<uint4*>(ws_masks + goff + c0);
-#pragma unroll
-            for (int q = 0; q < 4; ++q) o[q] = make_uint4(mk[4 * q], mk[4 * q + 1], mk[4 * q + 2], mk[4 * q + 3]);
-          }
-        }
-      }
-      // ---- backward recurrence ----
-      load_row(G);                                              // d out
+    }
+    if (T > 0) {
       if (has_psi) {
         publish_bf16();                                         // G is bf16 already: nothing is lost
         w.wait(&bars->r_full, phase & 1, 611); ++phase;
@@ -319,25 +205,17 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
         }
       }
       for (int t = T - 1; t >= 0; --t) {
-        // dx_t = d alpha_{t+1} o mask_t, published as the operand of both products
+        // dx_t = d alpha_{t+1} o mask_t (the forward's decisions: column c is bit 31 - c % 32 of word c / 32)
+        uint32_t mwd[D / 32];
+        {
+          const uint32_t* mp = maskbits + (((int64_t)bh * T + t) * nq + (live ? grow : 0)) * (D / 32);
 #pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 16) {
-          uint32_t mk[16];
-          tmem_ld_32x32b_x16(mask_addr + c0, mk);
-          tmem_wait_ld();
-          uint32_t pk[8];
-#pragma unroll
-          for (int e = 0; e < 16; e += 2) {
-            const float a0 = ((mk[e] >> t) & 1u) ? v[c0 + e] : 0.f, a1 = ((mk[e + 1] >> t) & 1u) ? v[c0 + e + 1] : 0.f;
-            v[c0 + e] = a0;
-            v[c0 + e + 1] = a1;
-            pk[e >> 1] = pack_bf16(a0, a1);
-          }
-          tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+          for (int q = 0; q < D / 32; ++q) mwd[q] = live ? mp[q] : 0u;
         }
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(&bars->a_full);
+#pragma unroll
+        for (int c = 0; c < D; ++c)
+          v[c] = ((mwd[c >> 5] >> (31 - (c & 31))) & 1u) ? v[c] : 0.f;
+        publish_bf16();
         w.wait(&bars->r_full, phase & 1, 612); ++phase;
         tc_fence_after();
         if (t > 0) {
@@ -351,30 +229,35 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
           }
         }
       }
-      // ---- dZ and D = <dZ, Z> ----
-      float dsum = 0.f;
-      const uint4* zp = reinterpret_cast<const uint4*>(Z16 + goff);
-      uint4* out = reinterpret_cast<uint4*>(dZ16 + goff);
+    }
+    // ---- dZ (the accumulated products; G itself without a decoder) and D = <dZ, Z> ----
+    float dsum = 0.f;
+    const uint4* zp = reinterpret_cast<const uint4*>(Z16 + goff);
+    uint4* out = reinterpret_cast<uint4*>(dZ16 + goff);
 #pragma unroll
-      for (int c0 = 0; c0 < D; c0 += 16) {
-        uint32_t r[16];
+    for (int c0 = 0; c0 < D; c0 += 16) {
+      uint32_t r[16];
+      if (T > 0) {                                              // uniform over the CTA: every lane takes part
         tmem_ld_32x32b_x16(dz_addr + c0, r);
         tmem_wait_ld();
+      } else {
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          const uint4 z = live ? zp[c0 / 8 + half] : make_uint4(0, 0, 0, 0);
-          const float* f = reinterpret_cast<const float*>(r) + 8 * half;
-          dsum = fmaf(f[0], bf16_lo(z.x), dsum); dsum = fmaf(f[1], bf16_hi(z.x), dsum);
-          dsum = fmaf(f[2], bf16_lo(z.y), dsum); dsum = fmaf(f[3], bf16_hi(z.y), dsum);
-          dsum = fmaf(f[4], bf16_lo(z.z), dsum); dsum = fmaf(f[5], bf16_hi(z.z), dsum);
-          dsum = fmaf(f[6], bf16_lo(z.w), dsum); dsum = fmaf(f[7], bf16_hi(z.w), dsum);
-          if (live && !w.dead)
-            out[c0 / 8 + half] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
-                                            pack_bf16(f[6], f[7]));
-        }
+        for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(v[c0 + e]);
       }
-      if (live && !w.dead) ws_LD[((int64_t)bh * nq + grow) * 2 + 1] = dsum;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint4 z = live ? zp[c0 / 8 + half] : make_uint4(0, 0, 0, 0);
+        const float* f = reinterpret_cast<const float*>(r) + 8 * half;
+        dsum = fmaf(f[0], bf16_lo(z.x), dsum); dsum = fmaf(f[1], bf16_hi(z.x), dsum);
+        dsum = fmaf(f[2], bf16_lo(z.y), dsum); dsum = fmaf(f[3], bf16_hi(z.y), dsum);
+        dsum = fmaf(f[4], bf16_lo(z.z), dsum); dsum = fmaf(f[5], bf16_hi(z.z), dsum);
+        dsum = fmaf(f[6], bf16_lo(z.w), dsum); dsum = fmaf(f[7], bf16_hi(z.w), dsum);
+        if (live && !w.dead)
+          out[c0 / 8 + half] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]),
+                                          pack_bf16(f[6], f[7]));
+      }
     }
+    if (live && !w.dead) ws_LD[((int64_t)bh * nq + grow) * 2 + 1] = dsum;
   }
   tc_fence_before();
   __syncthreads();
@@ -579,8 +462,8 @@ cudaError_t launch_recur(csat_ctx* c, const void* G, cudaStream_t s) {
   if (e != cudaSuccess) return e;
   const dim3 grid((unsigned)((p.nq + kRows - 1) / kRows), (unsigned)(p.B * p.H));
   bwd_recur_sm100_kernel<D><<<grid, kRThreads, C::kSmemBytes, s>>>(
-      c->tmap_mats, c->bw_Z16, (const __nv_bfloat16*)G, c->bw_dZ16, c->bw_LD, c->bw_masks, c->thr(), c->thr_stride(),
-      (int)p.nq, (int)p.H, p.T, c->psi ? 1 : 0, c->status);
+      c->tmap_mats, c->bw_Z16, (const __nv_bfloat16*)G, c->bw_dZ16, c->bw_LD, c->bw_maskbits, (int)p.nq, (int)p.H, p.T,
+      c->psi ? 1 : 0, c->status);
   return cudaGetLastError();
 }
 

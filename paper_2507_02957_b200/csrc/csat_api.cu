@@ -117,7 +117,8 @@ void free_backward(csat_ctx* c) {
   dev_free(c, &c->bw_dZ16, c->bw_bytes_dZ16);
   dev_free(c, &c->bw_masks, c->bw_bytes_masks);
   dev_free(c, &c->bw_Z16, c->bw_bytes_Z16);
-  c->bw_bytes_Z16 = 0;
+  dev_free(c, &c->bw_maskbits, c->bw_bytes_maskbits);
+  c->bw_bytes_Z16 = c->bw_bytes_maskbits = 0;
   c->bw_bytes_masks = 0;
   c->have_masks = false;
   c->bw_bytes_dZ = c->bw_bytes_LD = c->bw_bytes_dKV = c->bw_bytes_WT = c->bw_bytes_dKV16 = c->bw_bytes_dZ16 = 0;
@@ -737,8 +738,9 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
                bk = (size_t)(p.B * p.H * p.m * 2 * p.d) * 4,
                bw = (size_t)(2 * (c->w_untied ? c->w_layers : 1) * p.H * p.d * p.d) * 4,
                b16 = c->tmap_phi_valid ? bk / 2 : 0, z16 = c->tmap_phi_valid ? bz / 2 : 0,
-               bm = c->keep_masks && p.T > 0 ? bz : 0;
-  if (c->bw_bytes_Z16 != z16 || c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
+               bm = c->keep_masks && p.T > 0 ? bz : 0,
+               bmb = c->tmap_phi_valid ? (size_t)(p.B * p.H * p.T * p.nq * (p.d / 32)) * 4 : 0;
+  if (c->bw_bytes_maskbits != bmb || c->bw_bytes_Z16 != z16 || c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
       c->bw_bytes_dKV16 != b16 || c->bw_bytes_dZ16 != z16) {
     cudaDeviceSynchronize();
     free_backward(c);
@@ -746,7 +748,8 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
     c->bw_bytes_dZ16 = z16;
     c->bw_bytes_masks = bm;
     c->bw_bytes_Z16 = z16;
-    if (dev_alloc(c, &c->bw_Z16, z16) != cudaSuccess || dev_alloc(c, &c->bw_masks, bm) != cudaSuccess || dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
+    c->bw_bytes_maskbits = bmb;
+    if (dev_alloc(c, &c->bw_maskbits, bmb) != cudaSuccess || dev_alloc(c, &c->bw_Z16, z16) != cudaSuccess || dev_alloc(c, &c->bw_masks, bm) != cudaSuccess || dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
         dev_alloc(c, &c->bw_dKV, bk) != cudaSuccess || dev_alloc(c, &c->bw_WT, bw) != cudaSuccess ||
         dev_alloc(c, &c->bw_dKV16, b16) != cudaSuccess || dev_alloc(c, &c->bw_dZ16, z16) != cudaSuccess) {
       free_backward(c);

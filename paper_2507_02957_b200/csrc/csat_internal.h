@@ -105,7 +105,8 @@ struct csat_ctx {
   __nv_bfloat16* bw_dKV16 = nullptr;     // bf16 copy of dK~|dV~ (operand of the tensor-core Phi^T product)
   __nv_bfloat16* bw_dZ16 = nullptr;      // bf16 copy of dZ (operand of the tensor-core dK~|dV~ stage)
   __nv_bfloat16* bw_Z16 = nullptr;       // Z = A~ V~ as the forward rounds it (tensor-core per-query stages)
-  size_t bw_bytes_Z16 = 0;
+  uint32_t* bw_maskbits = nullptr;       // the forward's decisions, one bit per (b, h, layer, query, column)
+  size_t bw_bytes_Z16 = 0, bw_bytes_maskbits = 0;
   size_t bw_bytes_dZ = 0, bw_bytes_LD = 0, bw_bytes_dKV = 0, bw_bytes_WT = 0, bw_bytes_dKV16 = 0, bw_bytes_dZ16 = 0;
   // CSAT_KEEP_MASKS: the shrinkage decisions of the most recent csat_backward, one word per (b, h, query, column),
   // bit t = |x_t| > theta_t
@@ -182,9 +183,10 @@ cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cud
 cudaError_t make_attend_tmaps(csat_ctx* c);
 cudaError_t make_layer_weights_tmap(csat_ctx* c);
 cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
-// the attention phase alone: z_out [B,H,n_q,d] bf16 = Z, lse_out[row * lse_stride] = log sum exp of the row's scores
-cudaError_t launch_sm100_attend_lse(csat_ctx* c, const void* Q, void* z_out, float* lse_out, int lse_stride,
-                                    cudaStream_t s, int* launches);
+// the forward run for the backward pass: z_out [B,H,n_q,d] bf16 = Z, lse_out[row * lse_stride] = log sum exp of the
+// row's scores, mask_out [B,H,T,n_q,d/32] = the layers' decisions |x_t| > theta_t (column c: word c / 32, bit 31 - c % 32)
+cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bfloat16* z_out, float* lse_out,
+                                             int lse_stride, uint32_t* mask_out, cudaStream_t s, int* launches);
 
 // bwd_rows_sm100.cu : the per-query stages of the backward on the tensor cores (bf16, d in {64, 128}, one S, B
 // for all layers).  recur: Z, G -> dZ (bf16 into bw_dZ16), D = <dZ, Z> (into bw_LD), optionally the masks;
