@@ -39,9 +39,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture of that kernel and workload exists)
 NCU_TRAFFIC_BYTES = {
-    # profiles/dram_traffic_c5_long.txt: 153.8 MB read + 91.1 MB written (part of the 134 MB output is still in L2
+    # profiles/dram_traffic_c5_long.txt: 153.9 MB read + 91.5 MB written (part of the 134 MB output is still in L2
     # when the kernel ends); algorithmic: Q 134.2 + out 134.2 + K~|V~ 16.8 MB
-    ("attend_recover", "c5_long"): 244896256,
+    ("attend_recover", "c5_long"): 245424640,
 }
 
 
@@ -337,7 +337,7 @@ def time_projection(w: wl.Workload, iters: int = 10, warmup: int = 3) -> dict:
 
 
 def time_backward(w: wl.Workload, iters: int = 2) -> dict:
-    """csat_backward (gradients with respect to Q, K, V; first version on FFMA kernels) on a workload."""
+    """csat_backward (gradients with respect to Q, K, V) on a workload."""
     import torch
     from paper_2507_02957_b200 import binding
     host, dev, psi = device_tensors(w)
@@ -356,7 +356,8 @@ def time_backward(w: wl.Workload, iters: int = 2) -> dict:
         times.append(e0.elapsed_time(e1))
     ctx.close()
     return {"ms": float(np.median(times)),
-            "kernels": "per-row stage on ffma kernels (float32); dK~|dV~ and Phi^T on tcgen05 for bf16"}
+            "kernels": "bf16: every stage on tcgen05 (forward with decisions recorded, recurrence backward, dQ, dK~|dV~, "
+                       "Phi^T); float32: ffma kernels"}
 
 
 def run_csat(args, w: wl.Workload) -> dict:
