@@ -66,6 +66,7 @@ constexpr int kTileThreads = 128;
 constexpr int kThreads = 384;          // three warpgroups: tile A, tile B, control
 constexpr int kMmaWarp = 8, kTmaWarp = 9, kMmaWarpB = 10;   // tile A's MMA issuer, TMA producer, tile B's MMA issuer
 constexpr int kMaxStages = 6;
+constexpr int kComputeRegs = 224, kControlRegs = 56;   // registers per thread after setmaxnreg (checked on the host)
 constexpr int kPolyEvery = 4;          // every 4th pair of scores takes the polynomial exp2 (measured best of 1, 2, 3, 4, none)
 
 template <int D> struct Cfg {
@@ -262,7 +263,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
 
   // 2 x 128 x 224 + 128 x 56 = 64512 registers; each branch below starts with its own setmaxnreg
   if (warp >= kMmaWarp) {
-  reg_dealloc<56>();
+  reg_dealloc<kControlRegs>();
   if (warp == kTmaWarp) {
     // ------------------------------------------------ TMA producer ------------------------------------------------
     // Ring position g counts the chunks loaded so far (stage g % kStages, use g / kStages).  After an item's
@@ -293,6 +294,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             ++q_loads[t];
           }
         }
+        // K~|V~ come from the compression kernel before this one in the stream: with a programmatic dependent launch
+        // this kernel may have started (and loaded its first Q tiles) before that one finished
+        if (items_done == 0) pdl_wait();
         for (int j = 0; j < nchunks && !w.dead; ++j, ++g) {
           const int s = g % C::kStages;
           ring_wait_k(g, 201);
@@ -533,7 +537,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     }
   }
   } else {
-    reg_alloc<224>();
+    reg_alloc<kComputeRegs>();
     // ------------------------------------------------ compute threads ---------------------------------------------
     const int t = warp >> 2, wq = warp & 3;                     // tile, lane quarter
     const int row = wq * 32 + lane;                             // row of the tile = TMEM lane
@@ -930,6 +934,14 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
   static DeviceFlags smem_opt_in;
+  if (!smem_opt_in.test(c->device)) {
+    // setmaxnreg moves registers inside the pool the CTA is launched with (threads x the compiled register count); the
+    // kernel asks for 2 x 128 x 224 + 128 x 56 of them, and a request the pool cannot satisfy would wait forever
+    cudaFuncAttributes fa;
+    if ((e = cudaFuncGetAttributes(&fa, attend_recover_sm100_kernel<D, kUntied, kMasks>)) != cudaSuccess) return e;
+    if ((int64_t)fa.numRegs * kThreads < (int64_t)kTiles * kTileThreads * kComputeRegs + 128 * kControlRegs)
+      return cudaErrorLaunchOutOfResources;
+  }
   if ((e = ensure_dynamic_smem(attend_recover_sm100_kernel<D, kUntied, kMasks>, (int)C::kSmemBytes, c->device, smem_opt_in)) !=
       cudaSuccess)
     return e;
@@ -942,10 +954,21 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   if (n_items > (int64_t)1 << 30) return cudaErrorInvalidValue;
   const int sms = c->sms;
   const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
-  attend_recover_sm100_kernel<D, kUntied, kMasks><<<grid, kThreads, C::kSmemBytes, s>>>(
-      tq, c->tmap_kv, kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(), (int)p.nq, (int)p.m, (int)p.H, T,
-      c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items, (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out);
-  return cudaGetLastError();
+  // programmatic dependent launch: the kernel may be scheduled while the compression kernel before it still runs
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kMasks>, tq, c->tmap_kv,
+                            kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
+                            (int)p.nq, (int)p.m, (int)p.H, T, c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items,
+                            (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out);
 }
 
 }  // namespace

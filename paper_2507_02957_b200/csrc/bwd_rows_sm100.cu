@@ -47,11 +47,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 p = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&p);
 }
-__device__ __forceinline__ float fma_sat(float a, float b, float c) {   // clamps the result to [0, 1]
-  float y;
-  asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
-  return y;
-}
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
@@ -75,14 +70,14 @@ template <int D> struct RCfg {
   static constexpr uint32_t kOffMat = 0;                          // [3]: S - I | B^T | Psi, as the forward stages them
   static constexpr uint32_t kOffBar = 3 * kMatBytes;
   static constexpr uint32_t kSmemBytes = kOffBar + 128 + 1024 /*alignment slack*/;
-  // TMEM columns: accumulator | dZ accumulator | bf16 operand (two per column)
-  static constexpr uint32_t kColAcc = 0, kColDz = D, kColOp = 2 * D;
+  // TMEM columns: accumulator | dZ accumulator | two bf16 operand buffers (two values per column)
+  static constexpr uint32_t kColAcc = 0, kColDz = D, kColOp = 2 * D, kOpCols = D / 2;
   static constexpr uint32_t kTmemCols = (D == 64) ? 256 : 512;
-  static_assert(2 * D + D / 2 <= kTmemCols, "TMEM budget");
+  static_assert(2 * D + 2 * kOpCols <= kTmemCols, "TMEM budget");
 };
 
 struct RBars {
-  uint64_t mats_full, a_full, r_full;
+  uint64_t mats_full, a_full, r_full, op_free[2];
   uint32_t tmem_slot;
   int abort;
 };
@@ -107,6 +102,8 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
     mbar_init(&bars->mats_full, 1);
     mbar_init(&bars->a_full, kRows);
     mbar_init(&bars->r_full, 1);
+    mbar_init(&bars->op_free[0], 1);
+    mbar_init(&bars->op_free[1], 1);
     bars->abort = 0;
     fence_mbar_init();
   }
@@ -129,10 +126,11 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
           tma_load_3d(smem + C::kOffMat + mat * C::kMatBytes + gx * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, gx * 64,
                       0, h * 3 + mat);
       constexpr uint32_t idesc_t = make_idesc_bf16(kRows, D, false, true);    // transposed products: B MN-major
-      const uint32_t op = tmem + C::kColOp, acc = tmem + C::kColAcc, dz = tmem + C::kColDz;
+      const uint32_t acc = tmem + C::kColAcc, dz = tmem + C::kColDz;
       // product with the transpose of a matrix the forward stores [output column][k]: the tile's rows are now the
-      // reduction index, 16 rows (2048 bytes) per K step, the next 64 output columns one box further
-      auto mma_tr = [&](uint32_t d_t, int mat, uint32_t accumulate) {
+      // reduction index, 16 rows (2048 bytes) per K step, the next 64 output columns one box further.  The operands
+      // alternate between two buffers (publication n uses buffer n & 1).
+      auto mma_tr = [&](uint32_t d_t, uint32_t op, int mat, uint32_t accumulate) {
         const uint64_t bd = make_smem_desc(smem_u32(smem + C::kOffMat + mat * C::kMatBytes), C::kMatBoxBytes, 1024);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) mma_f16_ts(d_t, op + k * 8, bd + (uint64_t)(k * 128), idesc_t, k == 0 ? accumulate : 1u);
@@ -144,16 +142,25 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
         tc_fence_after();
       };
       w.wait(&bars->mats_full, 0, 600);
+      // The threads only wait for the product they need next (r_full); the dZ product trails it and releases the
+      // operand buffer (op_free) when it has read it.
       if (has_psi) {                                           // d alpha_T = G Psi
+        const uint32_t op = tmem + C::kColOp + (n_ops & 1) * C::kOpCols;
         operand_ready();
-        mma_tr(acc, 2, 0u);
+        mma_tr(acc, op, 2, 0u);
         mma_commit(&bars->r_full);
+        mma_commit(&bars->op_free[(n_ops - 1) & 1]);
       }
       for (int t = T - 1; t >= 0; --t) {
+        const uint32_t op = tmem + C::kColOp + (n_ops & 1) * C::kOpCols;
         operand_ready();
-        if (t > 0) mma_tr(acc, 0, 0u);                         // dx_t (S - I)^T
-        mma_tr(dz, 1, t == T - 1 ? 0u : 1u);                   // dZ += dx_t B^T
-        mma_commit(&bars->r_full);
+        if (t > 0) {
+          mma_tr(acc, op, 0, 0u);                              // dx_t (S - I)^T
+          mma_commit(&bars->r_full);
+        }
+        mma_tr(dz, op, 1, t == T - 1 ? 0u : 1u);               // dZ += dx_t B^T
+        if (t == 0) mma_commit(&bars->r_full);                 // the last result the threads wait for is dZ itself
+        mma_commit(&bars->op_free[(n_ops - 1) & 1]);
       }
       if (w.dead) mbar_wait_drain(&bars->mats_full, 0);
     }
@@ -163,11 +170,16 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
     const int grow = row0 + row;
     const bool live = grow < nq;
     const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16);
-    const uint32_t acc_addr = tbase + C::kColAcc, dz_addr = tbase + C::kColDz, op_addr = tbase + C::kColOp;
+    const uint32_t acc_addr = tbase + C::kColAcc, dz_addr = tbase + C::kColDz;
     const int64_t goff = ((int64_t)bh * nq + (live ? grow : 0)) * D;
     int phase = 0;
+    uint32_t n_pub = 0;                           // operands published so far (buffer n_pub & 1)
     float v[D];                                   // d alpha_{t+1}, then dx_t
     auto publish_bf16 = [&]() {                   // v as the bf16 A operand
+      const uint32_t op_addr = tbase + C::kColOp + (n_pub & 1) * C::kOpCols;
+      // the buffer's previous operand (two publications ago) has been read by its trailing product
+      if (n_pub >= 2) w.wait(&bars->op_free[n_pub & 1], ((n_pub >> 1) - 1) & 1, 613);
+      ++n_pub;
 #pragma unroll
       for (int c0 = 0; c0 < D; c0 += 16) {
         uint32_t pk[8];
@@ -204,20 +216,25 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
           for (int e = 0; e < 16; ++e) v[c0 + e] = __uint_as_float(r[e]);          // d alpha_T = G Psi
         }
       }
-      for (int t = T - 1; t >= 0; --t) {
-        // dx_t = d alpha_{t+1} o mask_t (the forward's decisions: column c is bit 31 - c % 32 of word c / 32)
-        uint32_t mwd[D / 32];
-        {
-          const uint32_t* mp = maskbits + (((int64_t)bh * T + t) * nq + (live ? grow : 0)) * (D / 32);
+      // the forward's decisions of layer t: column c is bit 31 - c % 32 of word c / 32 (loaded one layer ahead)
+      auto load_masks = [&](int t, uint32_t (&m)[D / 32]) {
+        const uint32_t* mp = maskbits + (((int64_t)bh * T + t) * nq + (live ? grow : 0)) * (D / 32);
 #pragma unroll
-          for (int q = 0; q < D / 32; ++q) mwd[q] = live ? mp[q] : 0u;
-        }
+        for (int q = 0; q < D / 32; ++q) m[q] = live ? mp[q] : 0u;
+      };
+      uint32_t mwd[D / 32], mnext[D / 32];
+      load_masks(T - 1, mwd);
+      for (int t = T - 1; t >= 0; --t) {
+        // dx_t = d alpha_{t+1} o mask_t
 #pragma unroll
         for (int c = 0; c < D; ++c)
           v[c] = ((mwd[c >> 5] >> (31 - (c & 31))) & 1u) ? v[c] : 0.f;
         publish_bf16();
+        if (t > 0) load_masks(t - 1, mnext);
         w.wait(&bars->r_full, phase & 1, 612); ++phase;
         tc_fence_after();
+#pragma unroll
+        for (int q = 0; q < D / 32; ++q) mwd[q] = mnext[q];
         if (t > 0) {
 #pragma unroll
           for (int c0 = 0; c0 < D; c0 += 16) {

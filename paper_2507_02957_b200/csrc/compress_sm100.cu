@@ -94,6 +94,9 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // the kernel after this one in the stream (attention / recovery) may be scheduled as SMs free up: its prologue
+  // and its Q loads overlap this kernel's tail; it waits for this grid before it reads K~|V~
+  pdl_launch_dependents();
 
   if (warp == 0) {
     if (elect_one()) {
