@@ -135,3 +135,65 @@ def test_backward_refuses_what_it_does_not_cover():
     ctx.set(T=2)
     ctx.backward(x, x, x, x)                     # the context stays usable
     ctx.close()
+
+
+EDGE = {
+    # (workload, tied LISTA weights with one threshold per layer?)
+    "one_layer": (wl.shrink(C["c2"], B=1, H=2, n_q=130, T=1, lam=0.01), False),
+    "thirty_two_layers": (wl.shrink(C["c2"], B=1, H=1, n_q=64, T=32, lam=0.01), False),
+    "zero_threshold": (wl.shrink(C["c2"], B=1, H=2, n_q=77, T=3, lam=0.0), False),
+    "single_query_d128": (wl.shrink(C["c5"], B=1, H=2, n=256, n_q=1, m=128, T=4, lam=0.002), False),
+    "per_layer_thresholds_d128": (wl.shrink(C["c5"], B=2, H=1, n=320, n_q=129, m=192, T=5, lam=0.002), True),
+}
+
+
+@pytest.mark.parametrize("name", sorted(EDGE))
+def test_backward_edge_cases_on_the_tensor_core_path(name):
+    """Depths 1 and 32, a zero threshold (eta is the identity: every decision is 1), a single query, 129 queries (a
+    second tile with one live row), and supplied tied weights with one threshold per layer: all bf16 with d in
+    {64, 128}, i.e. the tensor-core kernels.  Same two-part comparison as above."""
+    w, per_layer = EDGE[name]
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    binding.csat_set_i64(ctx.h, binding.CSAT_KEEP_MASKS, 1)
+    r = np.random.default_rng(11)
+    d, H, T = w.d, w.H, w.T
+    kw = dict(T=T, lam=w.lam)
+    phi = to_np(ctx.get_phi())
+    if per_layer:
+        S = wl.round_to_storage((0.6 * np.eye(d) + 0.4 * r.standard_normal((H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        Bm = wl.round_to_storage((r.standard_normal((H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        st0 = []
+        orc.csat_forward(inp["Q"][:1], inp["K"][:1], inp["V"][:1], phi, T=0, lam=0.0, stages=st0)
+        th0 = float(np.median(np.abs(st0[0]["Z"] @ Bm[0].astype(np.float64))))
+        thetas = (th0 * r.uniform(0.2, 1.5, size=(T, H))).astype(np.float32)
+        ctx.set_lista_weights(to_dev(S, w.dtype), to_dev(Bm, w.dtype), torch.from_numpy(thetas).cuda())
+        kw.update(weights=(S.astype(np.float64), Bm.astype(np.float64), list(thetas.astype(np.float64))))
+    G = wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    got = ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    words = ctx.backward_masks().cpu().numpy().astype(np.uint32)
+    masks = np.stack([(words >> t) & 1 for t in range(T)], axis=2).astype(bool)
+    stages = []
+    orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, stages=stages, **kw)
+    own = np.stack([s["masks"] for s in stages]).reshape(masks.shape)
+    xs = np.stack([s["xs"] for s in stages]).reshape(masks.shape)
+    differ = masks != own
+    if name == "zero_threshold":
+        assert masks.all()
+    assert differ.mean() <= 2e-2, (name, differ.mean())
+    if "weights" in kw:
+        th = np.asarray(kw["weights"][2], dtype=np.float64).T[None, :, :, None, None]
+    else:
+        st1 = []
+        orc.csat_forward(inp["Q"][:1], inp["K"][:1], inp["V"][:1], phi, T=1, lam=w.lam, stages=st1)
+        th = np.asarray([s["theta"] for s in st1])[None, :, None, None, None]
+    bar = TOL[w.dtype] * np.abs(xs).max(axis=(3, 4), keepdims=True)
+    dist = np.abs(np.abs(xs) - th)
+    assert (dist[differ] <= np.broadcast_to(bar, dist.shape)[differ]).all(), name
+    ref = orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, masks=masks, **kw)
+    for nm, g, rf in zip(("dQ", "dK", "dV"), got, ref):
+        assert np.abs(rf).max() > 0
+        err = rel_err(to_np(g), rf)
+        assert err <= BWD_TOL[w.dtype], (name, nm, err)
+    ctx.close()
