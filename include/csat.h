@@ -79,6 +79,9 @@ enum {
                           gather of the m selected rows (n log n additions per column instead of m n multiply-adds; the
                           same K~, V~ up to the order of the float32 sums).  0 (default): the dense product.  Other
                           ensembles, supplied matrices and longer sequences keep the dense product either way      */
+  CSAT_DEBUG_CANARY = 11, /* debugging aid: 1 fills the K~|V~ workspace with NaN bit patterns (one extra memset on the
+                          call's stream) before csat_forward / csat_backward compress, so that a row the compression
+                          failed to write shows as NaN in the output instead of reusing an earlier call's values  */
   CSAT_KEEP_MASKS = 9, /* 1: csat_backward also keeps its shrinkage decisions (one 32-bit word per (b, h, query,
                           column); needs CSAT_T <= 32) for csat_get_backward_masks.  0 (default): not kept  */
   CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls

@@ -19,6 +19,7 @@ ERR_NAMES = {1: "CSAT_ERR_INVALID_ARG", 2: "CSAT_ERR_SHAPE", 3: "CSAT_ERR_ALLOC"
 CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE, CSAT_ENSEMBLE, CSAT_SEPARATE_PHI = 1, 2, 3, 4, 5, 6, 7, 8
 CSAT_KEEP_MASKS = 9
 CSAT_HADAMARD_TRANSFORM = 10
+CSAT_DEBUG_CANARY = 11
 CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER, CSAT_ENSEMBLE_HADAMARD = 0, 1, 2
 KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1

@@ -362,6 +362,10 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       c->decoder_dirty = true;
       return make_hadamard_tables(c);
     }
+    case CSAT_DEBUG_CANARY:
+      if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_DEBUG_CANARY must be 0 or 1");
+      c->debug_canary = (int)v;
+      return CSAT_OK;
     case CSAT_HADAMARD_TRANSFORM:
       if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_HADAMARD_TRANSFORM must be 0 or 1");
       c->hadamard_transform = (int)v;
@@ -425,6 +429,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
     case CSAT_PROFILE: *out = c->prof_slots; return CSAT_OK;
     case CSAT_KEEP_MASKS: *out = c->keep_masks ? 1 : 0; return CSAT_OK;
     case CSAT_HADAMARD_TRANSFORM: *out = c->hadamard_transform; return CSAT_OK;
+    case CSAT_DEBUG_CANARY: *out = c->debug_canary; return CSAT_OK;
     default: return CSAT_ERR_INVALID_ARG;
   }
 }
@@ -618,6 +623,8 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
   // float32 contexts, and head sizes without a tensor-core kernel, take the FFMA kernels
   const bool tc_compress = c->tmap_phi_valid && c->force_simt != 1;
   const bool tc_attend = c->tmap_phi_valid && c->force_simt == 0;
+  if (c->debug_canary && (e = cudaMemsetAsync(c->kv, 0xFF, kv_bytes(c->p), s)) != cudaSuccess)
+    return fail_cuda(c, e, "canary fill");
   if (c->hadamard_transform && csat::fwht_compress_supported(c))
     e = csat::launch_fwht_compress(c, K, V, s, &launches);   // structured ensemble: transform instead of the dense product
   else
@@ -757,8 +764,9 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
     }
   }
   const bool tc_compress = c->tmap_phi_valid && c->force_simt != 1;
-  cudaError_t e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches)
-                              : csat::launch_simt_compress(c, K, V, s, &launches);
+  cudaError_t e = c->debug_canary ? cudaMemsetAsync(c->kv, 0xFF, kv_bytes(p), s) : cudaSuccess;
+  if (e != cudaSuccess) return fail_cuda(c, e, "canary fill");
+  e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward: compress launch");
   e = csat::launch_backward(c, Q, dOut, dQ, dK, dV, s, &launches);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward launch");

@@ -70,6 +70,7 @@ struct csat_ctx {
   uint32_t* had_ab = nullptr;
   size_t had_bytes_signs = 0, had_bytes_ab = 0;
   int hadamard_transform = 0; // CSAT_HADAMARD_TRANSFORM
+  int debug_canary = 0;       // CSAT_DEBUG_CANARY: the K~|V~ workspace is filled with NaN bit patterns before every compression
   CUtensorMap tmap_phi;       // TMA view of phi for the tensor-core compress kernel (bf16, d in {64,128})
   bool tmap_phi_valid = false;
   CUtensorMap tmap_kv;        // TMA view of the K~|V~ workspace

@@ -55,3 +55,28 @@ def test_failed_reallocation_is_refused_until_a_setter_succeeds():
             torch.cuda.synchronize()
             assert torch.equal(ctx.forward(Q, K, V), ref), (key, countdown)
     ctx.close()
+
+
+@pytest.mark.parametrize("shape", [(1, 3, 131, 67, 64, 67), (2, 2, 203, 37, 128, 139), (3, 1, 392, 200, 64, 200),
+                                   (1, 2, 100, 50, 40, 41)])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_workspace_canary_finds_no_unwritten_row(shape, dtype):
+    """CSAT_DEBUG_CANARY fills the K~|V~ workspace with NaN before every compression: on ragged shapes (measurement and
+    token counts that are no multiples of the tiles, odd batches, both kernel families) the forward and the backward
+    must stay finite and give the same bits as without the canary, i.e. every workspace row that is read was
+    written by the same call."""
+    B, H, n, nq, d, m = shape
+    w = wl.Workload("canary", B, H, n, nq, d, m, dtype, 3, 0.01, "iid", 57)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    ref = ctx.forward(Q, K, V).clone()
+    G = torch.randn_like(Q)
+    gref = [t.clone() for t in ctx.backward(Q, K, V, G)]
+    binding.csat_set_i64(ctx.h, binding.CSAT_DEBUG_CANARY, 1)
+    assert binding.csat_get_i64(ctx.h, binding.CSAT_DEBUG_CANARY) == 1
+    out = ctx.forward(Q, K, V)
+    assert torch.isfinite(out).all() and torch.equal(out, ref)
+    for a, b in zip(ctx.backward(Q, K, V, G), gref):
+        assert torch.isfinite(a).all() and torch.equal(a, b)
+    ctx.close()
