@@ -127,53 +127,29 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&r)[8]) {
                "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
                : "memory");
 }
-// two-element packed fp32 arithmetic (one instruction for both halves of a 64-bit register pair)
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-  return r;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
+// two-element packed fp32 arithmetic (one instruction for both halves of a register pair): the compiler's float2
+// builtins, so that it sees the register pairs (inline assembly on 64-bit registers cost extra moves and spills)
+using F2 = float2;
+__device__ __forceinline__ F2 pack2(float lo, float hi) { return make_float2(lo, hi); }
+__device__ __forceinline__ F2 pack2u(uint32_t lo, uint32_t hi) { return make_float2(__uint_as_float(lo), __uint_as_float(hi)); }
+__device__ __forceinline__ void unpack2(F2 v, float& lo, float& hi) { lo = v.x; hi = v.y; }
+__device__ __forceinline__ F2 fma2(F2 a, F2 b, F2 c) { return __ffma2_rn(a, b, c); }
+__device__ __forceinline__ F2 add2(F2 a, F2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ F2 sub2(F2 a, F2 b) { return __fadd2_rn(a, make_float2(-b.x, -b.y)); }
+__device__ __forceinline__ F2 mul2(F2 a, F2 b) { return __fmul2_rn(a, b); }
 
 // exp2 of both halves on the FMA pipe (the MUFU unit is the bottleneck of the softmax: 4 lanes per clock and
 // sub-core).  x <= ~9; anything below -120 (masked columns are -inf) gives 2^-120.  Round-to-nearest split
 // x = i + f, f in [-1/2, 1/2]; 2^f by a cubic fitted to 7.5e-5 relative error (P is rounded to bf16, 3.9e-3,
 // and the row sum tolerates far more); 2^i by adding i to the exponent field.
-__device__ __forceinline__ void exp2_poly2(uint64_t x2, float& p0, float& p1) {
+__device__ __forceinline__ void exp2_poly2(F2 x2, float& p0, float& p1) {
   float x0, x1;
   unpack2(x2, x0, x1);
   x2 = pack2(fmaxf(x0, -120.f), fmaxf(x1, -120.f));
-  const uint64_t magic = pack2(12582912.f, 12582912.f);          // 1.5 * 2^23: the sum's low mantissa bits hold i
-  const uint64_t t2 = add2(x2, magic);
-  const uint64_t f2 = sub2(x2, sub2(t2, magic));
-  uint64_t q2 = fma2(f2, pack2(0.055171459913253784f, 0.055171459913253784f), pack2(0.2426108568906784f, 0.2426108568906784f));
+  const F2 magic = pack2(12582912.f, 12582912.f);          // 1.5 * 2^23: the sum's low mantissa bits hold i
+  const F2 t2 = add2(x2, magic);
+  const F2 f2 = sub2(x2, sub2(t2, magic));
+  F2 q2 = fma2(f2, pack2(0.055171459913253784f, 0.055171459913253784f), pack2(0.2426108568906784f, 0.2426108568906784f));
   q2 = fma2(q2, f2, pack2(0.6932609677314758f, 0.6932609677314758f));
   q2 = fma2(q2, f2, pack2(0.9999281167984009f, 0.9999281167984009f));
   float t0, t1, q0, q1;
@@ -543,7 +519,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     const int row = wq * 32 + lane;                             // row of the tile = TMEM lane
     const uint32_t tbase = tmem + ((uint32_t)(wq * 32) << 16) + t * C::kTileCols;
     const uint32_t acc_addr = tbase + C::kColAcc;
-    const uint64_t sc2 = pack2(scale_log2, scale_log2);
+    const F2 sc2 = pack2(scale_log2, scale_log2);
     uint32_t cb = 0;                                            // chunks of this tile's earlier items
     uint32_t zc_seen = 0;                                       // phases of zc_full[t] this thread has waited for
     int phase = 0;                                              // phases of r_full[t] this thread has waited for
@@ -551,7 +527,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       const int bh = bh0 + item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
       if (t >= ((nq - row0 > kRows) ? 2 : 1)) continue;         // this item has no second tile
       float ref = -INFINITY;                                    // reference maximum of the row (log2 domain)
-      uint64_t sum2 = pack2(0.f, 0.f);                          // running sum of P, two partial sums
+      F2 sum2 = pack2(0.f, 0.f);                          // running sum of P, two partial sums
       const float kappa = T > 0 ? theta[h] : 0.f;               // loaded now, needed after the attention phase
 
       for (int j = 0; j < nchunks; ++j) {
@@ -607,13 +583,13 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             }
           }
         }
-        const uint64_t nref2 = pack2(-ref, -ref);
+        const F2 nref2 = pack2(-ref, -ref);
         // P_j over the first 32 columns of S[b] (two bf16 per column)
         auto exp_half = [&](const uint32_t (&r)[32], uint32_t col) {
           uint32_t pk[16];
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
-            const uint64_t x2 = fma2(pack2u(r[e], r[e + 1]), sc2, nref2);
+            const F2 x2 = fma2(pack2u(r[e], r[e + 1]), sc2, nref2);
             float p0, p1;
             if ((e >> 1) % kPolyEvery == kPolyEvery - 1) {       // this pair on the FMA pipe, the others on the MUFU
               exp2_poly2(x2, p0, p1);
@@ -655,9 +631,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       zc_seen = cb;
       tc_fence_after();
       // v2 holds, in turn: Z, b_t = alpha^t - theta, alpha^T, Psi alpha^T  (pairs of adjacent columns)
-      uint64_t v2[D / 2];
+      F2 v2[D / 2];
       {
-        const uint64_t inv2 = pack2(inv, inv);
+        const F2 inv2 = pack2(inv, inv);
 #pragma unroll
         for (int c0 = 0; c0 < D; c0 += 16) {
           uint32_t a[16];
@@ -719,19 +695,19 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           const float th = theta[(int64_t)it * theta_stride + h];
           const float thn = it + 2 < T ? theta[(int64_t)(it + 1) * theta_stride + h] : 0.f;
           const float inv2th = th > 0.f ? 0.5f / th : 0.f;          // theta = 0: sat(0) = 0 and eta(x) = x
-          const uint64_t m2th2 = pack2(-2.f * th, -2.f * th);
-          const uint64_t nx2 = pack2(thn, thn);
+          const F2 m2th2 = pack2(-2.f * th, -2.f * th);
+          const F2 nx2 = pack2(thn, thn);
           w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
           tc_fence_after();
           auto shrink16 = [&](const uint32_t (&r)[16], int c0) {
             uint32_t pk[8];
 #pragma unroll
             for (int e = 0; e < 16; e += 2) {
-              const uint64_t y2 = add2(v2[(c0 + e) >> 1], pack2u(r[e], r[e + 1]));   // alpha^t S_t + z B_t + theta_t
+              const F2 y2 = add2(v2[(c0 + e) >> 1], pack2u(r[e], r[e + 1]));   // alpha^t S_t + z B_t + theta_t
               float y0, y1;
               unpack2(y2, y0, y1);
-              const uint64_t t2 = pack2(fma_sat(y0, inv2th, 0.f), fma_sat(y1, inv2th, 0.f));
-              const uint64_t an = fma2(t2, m2th2, y2);                               // alpha^{t+1} = eta_theta(x)
+              const F2 t2 = pack2(fma_sat(y0, inv2th, 0.f), fma_sat(y1, inv2th, 0.f));
+              const F2 an = fma2(t2, m2th2, y2);                               // alpha^{t+1} = eta_theta(x)
               v2[(c0 + e) >> 1] = add2(an, nx2);
               float a0, a1;
               unpack2(an, a0, a1);
@@ -805,8 +781,8 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           for (int it = 0; it + 1 < T; ++it) {
             const float th = per_layer.value ? theta[(int64_t)it * theta_stride + h] : kappa;
             const float inv2th = th > 0.f ? 0.5f / th : 0.f;        // theta = 0: sat(1/2) = 1/2 and eta(x) = x
-            const uint64_t m2th2 = pack2(-2.f * th, -2.f * th);
-            const uint64_t dk2 = pack2(th - kappa, th - kappa);
+            const F2 m2th2 = pack2(-2.f * th, -2.f * th);
+            const F2 dk2 = pack2(th - kappa, th - kappa);
             w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
             tc_fence_after();
             // 16 columns at a time, the next piece's TMEM load in flight while this one is shrunk
@@ -814,17 +790,17 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
               uint32_t pk[8];
 #pragma unroll
               for (int e = 0; e < 16; e += 2) {
-                const uint64_t r2 = pack2u(r[e], r[e + 1]);
-                const uint64_t x2 = add2(v2[(c0 + e) >> 1], r2);               // alpha^t S + z B
+                const F2 r2 = pack2u(r[e], r[e + 1]);
+                const F2 x2 = add2(v2[(c0 + e) >> 1], r2);               // alpha^t S + z B
                 float x0, x1;
                 unpack2(x2, x0, x1);
                 if (kMasks) {                                                  // the sign bit of theta - |x| is the decision
                   mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x0)), mw[c0 >> 5], 1);
                   mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x1)), mw[c0 >> 5], 1);
                 }
-                const uint64_t t2 = pack2(fma_sat(x0, inv2th, 0.5f), fma_sat(x1, inv2th, 0.5f));
-                uint64_t bn = fma2(t2, m2th2, x2);                             // eta_theta(x) - theta
-                uint64_t dn = fma2(t2, m2th2, r2);                             // alpha^{t+1} - alpha^t
+                const F2 t2 = pack2(fma_sat(x0, inv2th, 0.5f), fma_sat(x1, inv2th, 0.5f));
+                F2 bn = fma2(t2, m2th2, x2);                             // eta_theta(x) - theta
+                F2 dn = fma2(t2, m2th2, r2);                             // alpha^{t+1} - alpha^t
                 if (per_layer.value) { bn = add2(bn, dk2); dn = add2(dn, dk2); }   // ... - kappa
                 v2[(c0 + e) >> 1] = bn;
                 float d0, d1;
