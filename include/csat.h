@@ -185,12 +185,16 @@ int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, c
  *   Q [B,H,n_q,d], K, V [B,H,n,d]   the forward's inputs          (context dtype, device)
  *   dOut [B,H,n_q,d]                gradient of the loss with respect to csat_forward's output
  *   dQ [B,H,n_q,d], dK, dV [B,H,n,d]  outputs (context dtype)
- * Nothing of an earlier csat_forward is reused: the call compresses K, V again and recomputes what it needs in
- * float32.  Its first call allocates float32 scratch (B H (n_q (d + 2) + 2 m d) floats and transposed
- * copies of the decoder matrices, plus B H n_q d words with CSAT_KEEP_MASKS, counted by csat_workspace_bytes).  CSAT_T <= 32, d <= 256 and B H <= 32767, else CSAT_ERR_UNSUPPORTED.  This first
- * version recomputes each query row (scores, recurrence, its backward, dQ) on plain FFMA kernels in float32; bf16
- * contexts with d in {64, 128} then run the gradients of K~|V~ (P^T dZ, dS^T Q) and the product with Phi^T on the
- * tensor cores with bf16 operands, everything else stays on FFMA kernels. */
+ * Nothing of an earlier csat_forward is reused: the call compresses K, V again and recomputes what it needs.  Its
+ * first call allocates scratch (B H (n_q (d + 2) + 2 m d) floats and transposed copies of the decoder matrices;
+ * bf16 copies of Z, dZ and dK~|dV~ and B H T n_q d / 32 decision words on the tensor-core path; B H n_q d words
+ * more with CSAT_KEEP_MASKS; all counted by csat_workspace_bytes).
+ * Two paths.  bf16 contexts with d in {64, 128} and tied layers run every stage on the tensor cores: the forward
+ * kernel once more (it keeps Z, the softmax statistics and one decision bit per layer, query and column), the
+ * backward recurrence, dQ, the gradients of K~|V~ (P^T dZ, dS^T Q) and the product with Phi^T, all with bf16
+ * operands and float32 accumulation; any CSAT_T.  Everything else (float32 contexts, other d, untied layers) runs
+ * float32 FFMA kernels that recompute each query row and keep the decisions of one (query, column) in one word:
+ * CSAT_T <= 32 there and with CSAT_KEEP_MASKS.  d <= 256 and B H <= 32767.  Otherwise CSAT_ERR_UNSUPPORTED. */
 int csat_backward(csat_ctx* ctx, const void* Q, const void* K, const void* V, const void* dOut, void* dQ, void* dK,
                   void* dV, void* stream);
 

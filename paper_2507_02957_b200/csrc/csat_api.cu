@@ -730,7 +730,11 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   if (*(volatile int*)c->status != 0)
     return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
   const csat::Params& p = c->p;
-  if (p.T > 32) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward keeps one mask bit per layer: CSAT_T <= 32");
+  const bool tc_all_stages = c->tmap_phi_valid && c->force_simt == 0 && !c->w_untied && !c->keep_masks;
+  if (p.T > 32 && !tc_all_stages)
+    return fail(c, CSAT_ERR_UNSUPPORTED,
+                "csat_backward: the float32 kernels and CSAT_KEEP_MASKS keep one decision bit per layer in a 32-bit "
+                "word: CSAT_T <= 32");
   if (p.d > 256) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: d <= 256");
   if (p.B * p.H > 32767) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: B * H <= 32767");
   if (p.T > 0 && c->w_S && (c->w_layers != 1 || c->w_untied) && c->w_layers != p.T)

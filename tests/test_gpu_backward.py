@@ -137,6 +137,26 @@ def test_backward_refuses_what_it_does_not_cover():
     ctx.close()
 
 
+def test_backward_tensor_core_path_takes_more_than_32_layers():
+    """The tensor-core path keeps its decisions per layer, so CSAT_T is not bounded by a word's 32 bits there.  With
+    lambda = 0 every decision is |x| > 0, the same on both sides, so the oracle needs no decisions supplied."""
+    w = wl.shrink(C["c2"], B=1, H=2, n_q=150, T=40, lam=0.0)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    phi = to_np(ctx.get_phi())
+    G = wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    got = ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    ref = orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, T=w.T, lam=0.0)
+    for nm, g, rf in zip(("dQ", "dK", "dV"), got, ref):
+        assert rel_err(to_np(g), rf) <= BWD_TOL["bf16"], nm
+    binding.csat_set_i64(ctx.h, binding.CSAT_KEEP_MASKS, 1)          # one word per entry: 32 layers at most
+    with pytest.raises(binding.CsatError) as ei:
+        ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    assert ei.value.code == 5
+    ctx.close()
+
+
 EDGE = {
     # (workload, tied LISTA weights with one threshold per layer?)
     "one_layer": (wl.shrink(C["c2"], B=1, H=2, n_q=130, T=1, lam=0.01), False),

@@ -648,3 +648,42 @@ def test_hadamard_fast_transform_matches_oracle_and_dense_product(name, separate
     ctx.set_phi(ctx.get_phi())
     assert torch.equal(ctx.forward(Q, K, V), dense_out)
     ctx.close()
+
+
+def _random_shapes():
+    """Seeded random shapes: both kernel families (bf16 with d in {64, 128} on the tensor cores, everything else on
+    the FFMA kernels), token / query / measurement counts that are no multiples of any tile, odd batches."""
+    r = np.random.default_rng(2024)
+    out = []
+    for i in range(16):
+        tc = i % 2 == 0
+        dtype = "bf16" if (tc or i % 4 == 1) else "fp32"
+        d = int(r.choice([64, 128])) if tc else int(r.choice([8, 16, 24, 40, 72]))
+        m = int(r.integers(d, 3 * d + 40))
+        n = int(r.integers(m, m + 600))
+        nq = int(r.integers(1, 420))
+        out.append(wl.Workload(f"rand{i}", int(r.integers(1, 4)), int(r.integers(1, 4)), n, nq, d, m, dtype,
+                               int(r.integers(0, 6)), float(r.choice([0.0, 0.005, 0.02])), "iid", 500 + i))
+    return out
+
+
+@pytest.mark.parametrize("w", _random_shapes(), ids=lambda w: f"{w.name}_{w.dtype}_B{w.B}H{w.H}_n{w.n}_nq{w.n_q}_d{w.d}_m{w.m}_T{w.T}")
+def test_random_shapes_match_oracle(w):
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    phi = to_np(ctx.get_phi())
+    out = to_np(ctx.forward(Q, K, V))
+    stages = []
+    ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], phi, T=w.T, lam=w.lam, stages=stages)
+    assert np.isfinite(out).all()
+    if np.abs(ref).max() == 0.0:
+        assert np.abs(out).max() <= max(s["theta"] for s in stages) * TOL[w.dtype]
+    else:
+        assert rel_err(out, ref) <= TOL[w.dtype], w
+    # the host-buffer entry point runs the same kernels over sub-ranges of (batch, head) pairs
+    Qh, Kh, Vh = (t.cpu().pin_memory() for t in (Q, K, V))
+    oh = torch.empty_like(Qh).pin_memory()
+    ctx.forward_host(Qh, Kh, Vh, oh)
+    assert torch.equal(oh, ctx.forward(Q, K, V).cpu())
+    ctx.close()
