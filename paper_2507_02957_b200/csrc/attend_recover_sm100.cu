@@ -521,7 +521,6 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     const uint32_t acc_addr = tbase + C::kColAcc;
     const F2 sc2 = pack2(scale_log2, scale_log2);
     uint32_t cb = 0;                                            // chunks of this tile's earlier items
-    uint32_t zc_seen = 0;                                       // phases of zc_full[t] this thread has waited for
     int phase = 0;                                              // phases of r_full[t] this thread has waited for
     for (int item = blockIdx.x; item < n_items && !w.dead; item += gridDim.x) {
       const int bh = bh0 + item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
@@ -566,8 +565,10 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           const bool raise = mx > ref + 8.f;
           if (__any_sync(0xffffffffu, raise)) {
             // rare: rescale this warp's rows of the accumulator (factor 1 for rows that keep their reference)
+            // A parity wait is only safe when the barrier is in the awaited phase or the one after it.  It is:
+            // S_j's commit (observed above) completes after every MMA its thread issued before, P_{j-2} V~_{j-2}
+            // among them, so phases up to c - 2 are over; phase c cannot end before this thread's arrival below.
             w.wait(&bars->zc_full[t], (c - 1) & 1, 221);        // P_{j-1} V~_{j-1} has been added
-            zc_seen = c;
             tc_fence_after();
             const float f = raise ? ex2(ref - mx) : 1.f;
             if (raise) ref = mx;
@@ -608,13 +609,10 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         exp_half(rb, 16);
         tmem_wait_st();                                         // also covers a rescale's stores
         tc_fence_before();
-        // A parity wait is only safe when the waiter is at most one phase behind, so every phase of zc_full is
-        // observed in order: phase j-1 here (it cannot be two ahead, since P_j V~_j needs the arrival below;
-        // normally it completed long ago), phase j after the next chunk, the last one after the loop.
-        if (j > 0 && zc_seen < c) {
-          w.wait(&bars->zc_full[t], (c - 1) & 1, 223);
-          zc_seen = c;
-        }
+        // The item's last two phases of zc_full are observed in order, the first of them before the arrival that
+        // lets the last product start (afterwards the barrier may be two phases on, which a parity wait cannot tell
+        // from none).
+        if (j == nchunks - 1 && j > 0) w.wait(&bars->zc_full[t], (c - 1) & 1, 223);
         mbar_arrive(&bars->p_full[t][b]);
       }
       float inv;
@@ -628,7 +626,6 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       }
       w.wait(&bars->zc_full[t], (cb + nchunks - 1) & 1, 222);   // every P V~ product has been added
       cb += nchunks;
-      zc_seen = cb;
       tc_fence_after();
       // v2 holds, in turn: Z, b_t = alpha^t - theta, alpha^T, Psi alpha^T  (pairs of adjacent columns)
       F2 v2[D / 2];
