@@ -1,22 +1,30 @@
 // Backward of the compressed attention with respect to the compressed keys and values, on the sm_100a tensor cores:
 //   dV~ = P^T dZ,   dK~ = scale dS^T Q,   P = exp(scale Q K~^T - L),   dS = P o (dZ V~^T - D)
 // (chain rule through Z = A~ V~ and A~ = softmax(Q K~^T / sqrt(d_k)); L = log-sum-exp of a row's scores and
-// D = <dZ, Z> come from the per-row kernel of the backward, like dZ itself).
+// D = <dZ, Z> come from the per-row stage of the backward, like dZ itself).
 //
 // One CTA owns 128 measurements of one (batch, head): K~ and V~ of the block stay in shared memory, the two
-// accumulators dK~ and dV~ [128 x d] in tensor memory, and the CTA walks the query tiles (128 rows):
-//   warp 0   : TMA producer: Q tile and dZ tile (bf16) of the next query tile.
+// accumulators dK~ and dV~ [128 x d] in tensor memory, and the CTA walks the queries in tiles of 64.  The scores are
+// formed TRANSPOSED, S^T = K~ Q^T (rows = measurements), so that the thread that owns a measurement's row of S^T
+// writes its row of P^T straight back into tensor memory, where it is the A operand (M = measurements, K = queries)
+// of the second pair of products: neither P nor dS passes through shared memory.
+//   warp 0   : TMA producer: Q and dZ tiles (bf16, 64 queries x d) and the queries' L, D (one untiled bulk copy) into
+//              a ring of kStages stages.
 //   warp 1   : allocates tensor memory; one elected thread issues the MMAs:
-//                S  = Q  K~^T   (A = Q tile, K-major; B = K~ block, K-major)      -> TMEM, 128 columns
-//                dA = dZ V~^T   (A = dZ tile, K-major; B = V~ block, K-major)     -> TMEM, 128 columns
-//              and, once the threads have written P and dS:
-//                dV~ += P^T  dZ (A = P  in shared memory, MN-major: rows = queries; B = the dZ tile, MN-major)
-//                dK~ += dS^T Q  (A = dS in shared memory, MN-major;                 B = the Q tile,  MN-major)
-//              The Q and dZ tiles are read twice without being moved: a tile of 128 rows x d with 128-byte rows is
-//              a K-major operand when its rows are the M index and an MN-major operand when they are the K index.
-//   warps 2-5: one thread per query row: reads its row of S and dA, forms P and dS (zero for rows beyond n_q and
-//              measurements beyond m), writes them as bf16 into the two operand tiles; at the end the same threads
-//              (TMEM lane = measurement) store the accumulators as float32 and as the bf16 operand of Phi^T.
+//                S^T  = K~ Q^T    (A = K~ block, K-major; B = Q tile, K-major)       -> set[i & 1], 64 columns
+//                dA^T = V~ dZ^T   (A = V~ block, K-major; B = dZ tile, K-major)      -> set[i & 1], 64 columns
+//              and, once the threads have written P^T and dS^T over them (bf16, two per column):
+//                dV~ += P^T  dZ   (A = P^T  in tensor memory; B = the dZ tile, MN-major: rows = queries = K index)
+//                dK~ += dS^T Q    (A = dS^T in tensor memory; B = the Q tile,  MN-major)
+//              The Q and dZ tiles are read twice without being moved: a tile of 64 rows x d with 128-byte rows is a
+//              K-major operand when its rows are the N index and an MN-major operand when they are the K index.
+//              Two sets of S^T | dA^T: the products of tile i + 1 run while the threads work on tile i.  The MMAs of
+//              one thread execute in issue order, so tile i + 2's scores overwrite set[i & 1] only after tile i's
+//              second pair of products has read it.
+//   warps 2-9: TMEM lane = measurement; warps 2-5 take the tile's queries [0, 32), warps 6-9 the queries [32, 64):
+//              P = exp2(S^T scale log2 e - L log2 e), dS = scale P (dA^T - D) with the queries' L, D read from global
+//              memory (the same address in every lane), zero for queries beyond n_q.  At the end the same threads
+//              store the accumulators as float32 and as the bf16 operand of the product with Phi^T.
 #include "csat_internal.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -26,27 +34,46 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kRows = 128;       // query rows per tile = measurements per block
-constexpr int kThreads = 192;
-constexpr uint32_t kPBytes = 2 * kRows * 128;          // P or dS: 128 queries x 128 measurements bf16, two 64-wide boxes
+constexpr int kRows = 128;       // measurements per block
+constexpr int kQT = 64;          // queries per tile
+constexpr int kStages = 4;       // Q | dZ tiles in flight
+constexpr int kSimtWarps = 8;
+constexpr int kThreads = (2 + kSimtWarps) * 32;
 
 template <int D> struct Cfg {
   static constexpr int kDBoxes = D / 64;
-  static constexpr uint32_t kBoxBytes = kRows * 128;                  // 128 rows x 64 columns
-  static constexpr uint32_t kTileBytes = kDBoxes * kBoxBytes;         // 128 rows x d
-  static constexpr uint32_t kOffK = 0, kOffV = kTileBytes, kOffQ = 2 * kTileBytes, kOffZ = 3 * kTileBytes;
-  static constexpr uint32_t kOffP = 4 * kTileBytes, kOffS = kOffP + kPBytes, kOffBar = kOffS + kPBytes;
+  static constexpr uint32_t kKvBoxBytes = kRows * 128;                // 128 rows x 64 columns
+  static constexpr uint32_t kKvBytes = kDBoxes * kKvBoxBytes;         // K~ block (= V~ block)
+  static constexpr uint32_t kInBoxBytes = kQT * 128;                  // 64 rows x 64 columns
+  static constexpr uint32_t kInBytes = kDBoxes * kInBoxBytes;         // Q tile (= dZ tile)
+  static constexpr uint32_t kOffK = 0, kOffV = kKvBytes, kOffIn = 2 * kKvBytes;   // stage s: Q at kOffIn + 2 s kInBytes, dZ after it
+  // L, D of a tile's queries: 64 pairs of floats copied from the 16-byte boundary at or below the first, so 66 pairs
+  static constexpr uint32_t kLdBytes = (kQT + 2) * 8, kLdStride = 544;
+  static constexpr uint32_t kOffLd = kOffIn + kStages * 2 * kInBytes;
+  static constexpr uint32_t kOffBar = kOffLd + kStages * kLdStride;
   static constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024 /*alignment slack*/;
-  static constexpr uint32_t kColS = 0, kColA = 128, kColV = 256, kColK = 256 + D, kTmemCols = 512;
-  static_assert(256 + 2 * D <= 512, "TMEM budget");
+  // TMEM columns: set s at 128 s: S^T (64) | dA^T (64); then the accumulators
+  static constexpr uint32_t kSetCols = 2 * kQT, kColA = kQT, kColV = 2 * kSetCols, kColK = kColV + D, kTmemCols = 512;
+  static_assert(2 * kSetCols + 2 * D <= 512, "TMEM budget");
   static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 };
 
 struct Bars {
-  uint64_t kv_full, in_full, in_free, sd_full, pm_full, acc_done;
+  uint64_t kv_full, in_full[kStages], in_free[kStages], sd_full[2], pd_full[2], acc_done;
   uint32_t tmem_slot;
   int abort;
 };
+static_assert(sizeof(Bars) <= 256, "barrier block");
+
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// packed column (two bf16 per 32-bit column) of K step k (16 queries) inside S^T or dA^T: the warps of the first
+// half write over the first 16 columns of their own 32 scores, the second half over columns [32, 48)
+__device__ __forceinline__ constexpr uint32_t pcol(int k) { return (uint32_t)((k >> 1) * 32 + (k & 1) * 8); }
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -60,17 +87,15 @@ bwd_cols_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   Bars* bars = reinterpret_cast<Bars*>(smem + C::kOffBar);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int mb = blockIdx.x, bh = blockIdx.y;
-  const int ntiles = (nq + kRows - 1) / kRows;
+  const int ntiles = (nq + kQT - 1) / kQT;
 
   if (threadIdx.x == 0) {
     prefetch_tmap(&tmap_q);
     prefetch_tmap(&tmap_z);
     prefetch_tmap(&tmap_kv);
     mbar_init(&bars->kv_full, 1);
-    mbar_init(&bars->in_full, 1);
-    mbar_init(&bars->in_free, 1);
-    mbar_init(&bars->sd_full, 1);
-    mbar_init(&bars->pm_full, 4 * 32);
+    for (int s = 0; s < kStages; ++s) { mbar_init(&bars->in_full[s], 1); mbar_init(&bars->in_free[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&bars->sd_full[s], 1); mbar_init(&bars->pd_full[s], kSimtWarps * 32); }
     mbar_init(&bars->acc_done, 1);
     bars->abort = 0;
     fence_mbar_init();
@@ -87,132 +112,167 @@ bwd_cols_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   if (warp == 0) {
     if (elect_one()) {
       // K~ and V~ of the block: the workspace rows are K~_r | V~_r; boxes of 64 columns x 64 rows
-      mbar_arrive_expect_tx(&bars->kv_full, 2 * C::kTileBytes);
+      mbar_arrive_expect_tx(&bars->kv_full, 2 * C::kKvBytes);
       for (int gx = 0; gx < C::kDBoxes; ++gx)
         for (int half = 0; half < 2; ++half) {
-          tma_load_3d(smem + C::kOffK + gx * C::kBoxBytes + half * 64 * 128, &tmap_kv, &bars->kv_full, gx * 64,
+          tma_load_3d(smem + C::kOffK + gx * C::kKvBoxBytes + half * 64 * 128, &tmap_kv, &bars->kv_full, gx * 64,
                       mb * kRows + half * 64, bh);
-          tma_load_3d(smem + C::kOffV + gx * C::kBoxBytes + half * 64 * 128, &tmap_kv, &bars->kv_full, D + gx * 64,
+          tma_load_3d(smem + C::kOffV + gx * C::kKvBoxBytes + half * 64 * 128, &tmap_kv, &bars->kv_full, D + gx * 64,
                       mb * kRows + half * 64, bh);
         }
       bool ok = true;
       int issued = 0;
+      const float2* LDg = reinterpret_cast<const float2*>(ws_LD) + (int64_t)bh * nq;
       for (int i = 0; i < ntiles && ok; ++i) {
-        ok = mbar_wait(&bars->in_free, (i & 1) ^ 1, status, 501, &bars->abort);   // the MMAs of tile i-1 have read Q, dZ
+        const int s = i % kStages;
+        // the second pair of products of tile i - kStages has read the stage
+        if (i >= kStages) ok = mbar_wait(&bars->in_free[s], ((i / kStages) & 1) ^ 1, status, 501, &bars->abort);
         if (!ok) break;
-        mbar_arrive_expect_tx(&bars->in_full, 2 * C::kTileBytes);
+        uint8_t* qs = smem + C::kOffIn + (uint32_t)s * 2 * C::kInBytes;
+        mbar_arrive_expect_tx(&bars->in_full[s], 2 * C::kInBytes + C::kLdBytes);
+        // (the copy may run up to 65 pairs past the rows of this (batch, head), into the next one's or into the slack
+        // the buffer is allocated with; those queries are masked)
+        bulk_load_1d(smem + C::kOffLd + (uint32_t)s * C::kLdStride,
+                     reinterpret_cast<const uint8_t*>((reinterpret_cast<uintptr_t>(LDg + i * kQT)) & ~uintptr_t(15)),
+                     C::kLdBytes, &bars->in_full[s]);
         for (int gx = 0; gx < C::kDBoxes; ++gx) {
-          tma_load_3d(smem + C::kOffQ + gx * C::kBoxBytes, &tmap_q, &bars->in_full, gx * 64, i * kRows, bh);
-          tma_load_3d(smem + C::kOffZ + gx * C::kBoxBytes, &tmap_z, &bars->in_full, gx * 64, i * kRows, bh);
+          tma_load_3d(qs + gx * C::kInBoxBytes, &tmap_q, &bars->in_full[s], gx * 64, i * kQT, bh);
+          tma_load_3d(qs + C::kInBytes + gx * C::kInBoxBytes, &tmap_z, &bars->in_full[s], gx * 64, i * kQT, bh);
         }
         ++issued;
       }
-      if (!ok) {
+      if (!ok) {                                  // gave up: let the copies in flight land before the CTA exits
         mbar_wait_drain(&bars->kv_full, 0);
-        if (issued > 0) mbar_wait_drain(&bars->in_full, (issued - 1) & 1);
+        for (int i = issued > kStages ? issued - kStages : 0; i < issued; ++i)
+          mbar_wait_drain(&bars->in_full[i % kStages], (i / kStages) & 1);
       }
     }
   } else if (warp == 1) {
     if (elect_one()) {
-      constexpr uint32_t idesc_s = make_idesc_bf16(kRows, kRows, false, false);   // S, dA: both operands K-major
-      constexpr uint32_t idesc_g = make_idesc_bf16(kRows, D, true, true);         // dV~, dK~: both operands MN-major
-      // K-major tile of 128 rows: K step k (16 columns) lies in 64-column box k / 4, 32 (k % 4) bytes into each row
-      auto kstep = [](int k) { return (uint64_t)((k / 4) * (C::kBoxBytes >> 4) + (k % 4) * 2); };
+      constexpr uint32_t idesc_s = make_idesc_bf16(kRows, kQT, false, false);    // S^T, dA^T: both operands K-major
+      constexpr uint32_t idesc_g = make_idesc_bf16(kRows, D, false, true);       // dV~, dK~: A in TMEM, B MN-major
+      // K-major tile: K step k (16 columns) lies in 64-column box k / 4, 32 (k % 4) bytes into each row
+      auto kstep = [](int k, uint32_t box_bytes) { return (uint64_t)((k / 4) * (box_bytes >> 4) + (k % 4) * 2); };
       const uint64_t kd = make_smem_desc(smem_u32(smem + C::kOffK), 16, 1024);
       const uint64_t vd = make_smem_desc(smem_u32(smem + C::kOffV), 16, 1024);
-      const uint64_t qd = make_smem_desc(smem_u32(smem + C::kOffQ), 16, 1024);
-      const uint64_t zd = make_smem_desc(smem_u32(smem + C::kOffZ), 16, 1024);
-      // MN-major: the next 64 elements along M / N start one box (128 rows x 128 bytes) further; 16 k rows = 2048 B
-      const uint64_t pm = make_smem_desc(smem_u32(smem + C::kOffP), kRows * 128, 1024);
-      const uint64_t sm = make_smem_desc(smem_u32(smem + C::kOffS), kRows * 128, 1024);
-      const uint64_t qn = make_smem_desc(smem_u32(smem + C::kOffQ), C::kBoxBytes, 1024);
-      const uint64_t zn = make_smem_desc(smem_u32(smem + C::kOffZ), C::kBoxBytes, 1024);
+      // stage 0's tiles; stage s lies 2 kInBytes s further.  K-major view (rows = N index) and MN-major view
+      // (rows = K index: the next 64 elements along N start one box further; 16 k rows = 2048 B) of the same bytes
+      const uint64_t qk0 = make_smem_desc(smem_u32(smem + C::kOffIn), 16, 1024);
+      const uint64_t zk0 = make_smem_desc(smem_u32(smem + C::kOffIn + C::kInBytes), 16, 1024);
+      const uint64_t qn0 = make_smem_desc(smem_u32(smem + C::kOffIn), C::kInBoxBytes, 1024);
+      const uint64_t zn0 = make_smem_desc(smem_u32(smem + C::kOffIn + C::kInBytes), C::kInBoxBytes, 1024);
+      constexpr uint64_t kStageStep = (2 * C::kInBytes) >> 4;
       bool ok = mbar_wait(&bars->kv_full, 0, status, 502, &bars->abort);
+      auto issue_scores = [&](int i) {            // S^T and dA^T of tile i
+        const int s = i % kStages;
+        ok = mbar_wait(&bars->in_full[s], (i / kStages) & 1, status, 503, &bars->abort);
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t ts = tmem + (uint32_t)(i & 1) * C::kSetCols;
+        const uint64_t st = (uint64_t)s * kStageStep;
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          mma_f16_ss(ts, kd + kstep(k, C::kKvBoxBytes), qk0 + st + kstep(k, C::kInBoxBytes), idesc_s, k != 0);
+#pragma unroll
+        for (int k = 0; k < D / 16; ++k)
+          mma_f16_ss(ts + C::kColA, vd + kstep(k, C::kKvBoxBytes), zk0 + st + kstep(k, C::kInBoxBytes), idesc_s, k != 0);
+        mma_commit(&bars->sd_full[i & 1]);
+      };
+      if (ok) issue_scores(0);
+      if (ok && ntiles > 1) issue_scores(1);
       for (int i = 0; i < ntiles && ok; ++i) {
-        ok = mbar_wait(&bars->in_full, i & 1, status, 503, &bars->abort);
+        ok = mbar_wait(&bars->pd_full[i & 1], (i >> 1) & 1, status, 504, &bars->abort);   // P^T and dS^T are written
         if (!ok) break;
         tc_fence_after();
+        const uint32_t ts = tmem + (uint32_t)(i & 1) * C::kSetCols;
+        const uint64_t st = (uint64_t)(i % kStages) * kStageStep;
 #pragma unroll
-        for (int k = 0; k < D / 16; ++k) mma_f16_ss(tmem + C::kColS, qd + kstep(k), kd + kstep(k), idesc_s, k != 0);
-#pragma unroll
-        for (int k = 0; k < D / 16; ++k) mma_f16_ss(tmem + C::kColA, zd + kstep(k), vd + kstep(k), idesc_s, k != 0);
-        mma_commit(&bars->sd_full);
-        ok = mbar_wait(&bars->pm_full, i & 1, status, 504, &bars->abort);       // P and dS are in shared memory
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll
-        for (int k = 0; k < kRows / 16; ++k) {
-          mma_f16_ss(tmem + C::kColV, pm + (uint64_t)(k * 128), zn + (uint64_t)(k * 128), idesc_g, (i | k) != 0);
-          mma_f16_ss(tmem + C::kColK, sm + (uint64_t)(k * 128), qn + (uint64_t)(k * 128), idesc_g, (i | k) != 0);
+        for (int k = 0; k < kQT / 16; ++k) {
+          mma_f16_ts(tmem + C::kColV, ts + pcol(k), zn0 + st + (uint64_t)(k * 128), idesc_g, (i | k) != 0);
+          mma_f16_ts(tmem + C::kColK, ts + C::kColA + pcol(k), qn0 + st + (uint64_t)(k * 128), idesc_g, (i | k) != 0);
         }
-        mma_commit(&bars->in_free);               // Q, dZ, P and dS may be overwritten
+        mma_commit(&bars->in_free[i % kStages]);  // the stage may be overwritten
+        if (i + 2 < ntiles) issue_scores(i + 2);
       }
-      mma_commit(&bars->acc_done);
+      if (ok) mma_commit(&bars->acc_done);
     }
   } else {
-    const int q = warp & 3;                       // TMEM lanes [32q, 32q+32)
-    const int row = q * 32 + lane;                // query row of the tile, later measurement of the block
+    const int q = warp & 3;                       // TMEM lanes [32q, 32q+32): a warp reaches only its own quarter
+    const int hf = (warp - 2) >> 2;               // which 32 of the tile's 64 queries
     const uint32_t tbase = tmem + ((uint32_t)(q * 32) << 16);
     const float scale_log2 = scale * 1.4426950408889634f;
-    uint8_t* prow = smem + C::kOffP + row * 128;
-    uint8_t* srow = smem + C::kOffS + row * 128;
+    // first pair of the tile within its staged copy: 0 or 1 (the same for every tile: 64 pairs are 512 bytes)
+    const int ld_off = (int)((reinterpret_cast<uintptr_t>(reinterpret_cast<const float2*>(ws_LD) + (int64_t)bh * nq) >> 3) & 1);
     bool ok = true;
     for (int i = 0; i < ntiles && ok; ++i) {
-      const int gq = i * kRows + row;
-      const bool live = gq < nq;
-      const float L = live ? ws_LD[((int64_t)bh * nq + gq) * 2] * 1.4426950408889634f : 0.f;   // log2 domain
-      const float Dr = live ? ws_LD[((int64_t)bh * nq + gq) * 2 + 1] : 0.f;
-      ok = mbar_wait(&bars->sd_full, i & 1, status, 505, &bars->abort);
+      const uint32_t ts = tbase + (uint32_t)(i & 1) * C::kSetCols;
+      // the TMEM loads and stores below are warp-wide: the whole warp gives up together
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->sd_full[i & 1], (i >> 1) & 1, status, 505, &bars->abort));
       if (!ok) break;
+      // The scores' commit follows the stage's arrival in the MMA thread's program order, but this thread reads the
+      // staged L, D itself, so it observes the stage's barrier too (complete by now: no waiting).
+      ok = __all_sync(0xffffffffu, mbar_wait(&bars->in_full[i % kStages], (i / kStages) & 1, status, 507, &bars->abort));
+      if (!ok) break;
+      const float2* ldq = reinterpret_cast<const float2*>(smem + C::kOffLd + (uint32_t)(i % kStages) * C::kLdStride) + ld_off;
       tc_fence_after();
-      // P and dS of tile i-1 have been read: sd_full of tile i follows the commit of tile i-1's last MMAs
-#pragma unroll 1
-      for (int c0 = 0; c0 < kRows; c0 += 16) {
+#pragma unroll
+      for (int sp = 0; sp < 2; ++sp) {            // 16 queries at a time
+        const int c0 = hf * 32 + sp * 16;         // first of them within the tile = column of S^T
         uint32_t s[16], a[16];
-        tmem_ld_32x32b_x16(tbase + C::kColS + c0, s);
-        tmem_ld_32x32b_x16(tbase + C::kColA + c0, a);
+        tmem_ld_32x32b_x16(ts + c0, s);
+        tmem_ld_32x32b_x16(ts + C::kColA + c0, a);
+        float2 ld[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const int gq = i * kQT + c0 + e;
+          ld[e] = gq < nq ? ldq[c0 + e] : make_float2(INFINITY, 0.f);         // beyond n_q: P = exp2(-inf) = 0
+        }
         tmem_wait_ld();
         uint32_t pw[8], dw[8];
 #pragma unroll
         for (int e = 0; e < 16; e += 2) {
-          float p0 = 0.f, p1 = 0.f;
-          if (live && mb * kRows + c0 + e < m) p0 = exp2f(fmaf(__uint_as_float(s[e]), scale_log2, -L));
-          if (live && mb * kRows + c0 + e + 1 < m) p1 = exp2f(fmaf(__uint_as_float(s[e + 1]), scale_log2, -L));
-          const float d0 = p0 * (__uint_as_float(a[e]) - Dr) * scale, d1 = p1 * (__uint_as_float(a[e + 1]) - Dr) * scale;
+          const float p0 = ex2f(fmaf(__uint_as_float(s[e]), scale_log2, -ld[e].x * 1.4426950408889634f));
+          const float p1 = ex2f(fmaf(__uint_as_float(s[e + 1]), scale_log2, -ld[e + 1].x * 1.4426950408889634f));
+          const float d0 = p0 * (__uint_as_float(a[e]) - ld[e].y) * scale;
+          const float d1 = p1 * (__uint_as_float(a[e + 1]) - ld[e + 1].y) * scale;
           __nv_bfloat162 pp = __floats2bfloat162_rn(p0, p1), dd = __floats2bfloat162_rn(d0, d1);
           pw[e >> 1] = *reinterpret_cast<uint32_t*>(&pp);
           dw[e >> 1] = *reinterpret_cast<uint32_t*>(&dd);
         }
-        // measurements c0 .. c0 + 15 of this query row: box c0 / 64, two 16-byte pieces swizzled by the row
-        const uint32_t box = (uint32_t)(c0 / 64) * (kRows * 128), piece = (uint32_t)((c0 % 64) / 8);
-#pragma unroll
-        for (int h2 = 0; h2 < 2; ++h2) {
-          const uint32_t off = box + (((piece + h2) ^ (uint32_t)(row & 7)) << 4);
-          *reinterpret_cast<uint4*>(prow + off) = make_uint4(pw[4 * h2], pw[4 * h2 + 1], pw[4 * h2 + 2], pw[4 * h2 + 3]);
-          *reinterpret_cast<uint4*>(srow + off) = make_uint4(dw[4 * h2], dw[4 * h2 + 1], dw[4 * h2 + 2], dw[4 * h2 + 3]);
-        }
+        // over the scores this thread has already read (see pcol)
+        tmem_st_32x32b_x8(ts + hf * 32 + sp * 8, pw);
+        tmem_st_32x32b_x8(ts + C::kColA + hf * 32 + sp * 8, dw);
       }
-      fence_proxy_async();                        // the tensor cores read what these threads wrote
+      tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(&bars->pm_full);
+      mbar_arrive(&bars->pd_full[i & 1]);
     }
-    if (ok && mbar_wait(&bars->acc_done, 0, status, 506, &bars->abort) && *(volatile int*)&bars->abort == 0) {
+    if (__all_sync(0xffffffffu, ok && mbar_wait(&bars->acc_done, 0, status, 506, &bars->abort) &&
+                                    *(volatile int*)&bars->abort == 0)) {
       tc_fence_after();
-      const int r = mb * kRows + row;             // measurement
+      const int r = mb * kRows + q * 32 + lane;   // measurement
+      // workspace row: dK~ | dV~; the first half of the warps stores dK~, the second dV~
+      const uint32_t acc = tbase + (hf == 0 ? C::kColK : C::kColV);
+      float* o = ws_dKV + ((int64_t)bh * m + r) * 2 * D + hf * D;
+      __nv_bfloat16* o16 = ws_dKV16 + ((int64_t)bh * m + r) * 2 * D + hf * D;
 #pragma unroll 1
-      for (int c0 = 0; c0 < 2 * D; c0 += 16) {
+      for (int c0 = 0; c0 < D; c0 += 16) {
         uint32_t v[16];
-        // accumulator columns: dV~ at kColV, dK~ at kColK; workspace row: dK~ | dV~
-        tmem_ld_32x32b_x16(tbase + (c0 < D ? C::kColK + c0 : C::kColV + (c0 - D)), v);
+        tmem_ld_32x32b_x16(acc + c0, v);          // the whole warp takes part in the load
         tmem_wait_ld();
         if (r < m) {
-          float* o = ws_dKV + ((int64_t)bh * m + r) * 2 * D + c0;
-          __nv_bfloat16* o16 = ws_dKV16 + ((int64_t)bh * m + r) * 2 * D + c0;
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            o[e] = __uint_as_float(v[e]);
-            o16[e] = __float2bfloat16_rn(__uint_as_float(v[e]));
+          for (int e = 0; e < 16; e += 4)
+            *reinterpret_cast<float4*>(o + c0 + e) = make_float4(__uint_as_float(v[e]), __uint_as_float(v[e + 1]),
+                                                                 __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
+          uint32_t h[8];
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) {
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+            h[e >> 1] = *reinterpret_cast<uint32_t*>(&b2);
           }
+          *reinterpret_cast<uint4*>(o16 + c0) = make_uint4(h[0], h[1], h[2], h[3]);
+          *reinterpret_cast<uint4*>(o16 + c0 + 8) = make_uint4(h[4], h[5], h[6], h[7]);
         }
       }
     }
@@ -229,7 +289,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, cudaStream_t s) {
   CUtensorMap tq, tz;
   const uint64_t qd[3] = {(uint64_t)D, (uint64_t)p.nq, (uint64_t)(p.B * p.H)};
   const uint64_t qs[2] = {(uint64_t)D * 2, (uint64_t)p.nq * D * 2};
-  const uint32_t qb[3] = {64, (uint32_t)kRows, 1};
+  const uint32_t qb[3] = {64, (uint32_t)kQT, 1};
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
   if ((e = make_tmap_bf16_3d(&tz, c->bw_dZ16, qd, qs, qb)) != cudaSuccess) return e;
@@ -244,7 +304,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, cudaStream_t s) {
 
 }  // namespace
 
-// needs dZ as bf16 (bw_dZ16), L and D (bw_LD) from the per-row kernel, and K~|V~ in the workspace
+// needs dZ as bf16 (bw_dZ16), L and D (bw_LD) from the per-row stage, and K~|V~ in the workspace
 cudaError_t launch_sm100_bwd_cols(csat_ctx* c, const void* Q, cudaStream_t s, int* launches) {
   *launches += 1;
   return c->p.d == 64 ? launch<64>(c, Q, s) : launch<128>(c, Q, s);

@@ -745,7 +745,7 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
     int rc = ensure_decoder(c, s, &launches);
     if (rc != CSAT_OK) return rc;
   }
-  const size_t bz = (size_t)(p.B * p.H * p.nq * p.d) * 4, bl = (size_t)(p.B * p.H * p.nq * 2) * 4,
+  const size_t bz = (size_t)(p.B * p.H * p.nq * p.d) * 4, bl = (size_t)(p.B * p.H * p.nq * 2) * 4 + 1024 /* read past the end by whole-tile copies */,
                bk = (size_t)(p.B * p.H * p.m * 2 * p.d) * 4,
                bw = (size_t)(2 * (c->w_untied ? c->w_layers : 1) * p.H * p.d * p.d) * 4,
                b16 = c->tmap_phi_valid ? bk / 2 : 0, z16 = c->tmap_phi_valid ? bz / 2 : 0,
