@@ -116,6 +116,11 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
+__device__ __forceinline__ float add_sat(float a, float b) {            // clamps the result to [0, 1]
+  float y;
+  asm("add.sat.f32 %0, %1, %2;" : "=f"(y) : "f"(a), "f"(b));
+  return y;
+}
 __device__ __forceinline__ float fma_sat(float a, float b, float c) {   // clamps the result to [0, 1]
   float y;
   asm("fma.rn.sat.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
@@ -757,7 +762,93 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
       }
-      if (!kUntied && T > 0) {
+      // One positive threshold for all layers (the ISTA-derived decoder), no decisions to record: the same recurrence
+      // in units of 2 theta, which saves one instruction per pair of elements.  Registers c = alpha / (2 theta),
+      // accumulator r' = 1/2 + (z B - a^ mu G) / (2 theta) (the threads store 1/2, z is published divided by 2 theta):
+      //   s = sat(c + r') (= sat(x / (2 theta) + 1/2), one saturating add);  increment = r' - s;  c += increment.
+      const bool scaled_units = !kUntied && !kMasks && T > 0 && theta_stride == 0 && kappa > 0.f;
+      if (scaled_units) {
+        const uint32_t op_addr = tbase + C::kColS;
+        {
+          uint32_t tb[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e) tb[e] = __float_as_uint(0.5f);
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) tmem_st_32x32b_x16(acc_addr + c0, tb);
+          const float inv2th = 0.5f / kappa;
+          const F2 i2 = pack2(inv2th, inv2th);
+#pragma unroll
+          for (int i = 0; i < D / 2; ++i) v2[i] = mul2(v2[i], i2);
+        }
+        publish(0);
+#pragma unroll
+        for (int i = 0; i < D / 2; ++i) v2[i] = pack2(0.f, 0.f);      // alpha^0 = 0
+        const F2 m1 = pack2(-1.f, -1.f);
+        for (int it = 0; it + 1 < T; ++it) {
+          w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
+          tc_fence_after();
+          auto shrink16 = [&](const uint32_t (&r)[16], int c0) {
+            uint32_t pk[8];
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) {
+              float a0, a1;
+              unpack2(v2[(c0 + e) >> 1], a0, a1);
+              const F2 s2 = pack2(add_sat(a0, __uint_as_float(r[e])), add_sat(a1, __uint_as_float(r[e + 1])));
+              const F2 dn = fma2(s2, m1, pack2u(r[e], r[e + 1]));     // (alpha^{t+1} - alpha^t) / (2 theta)
+              v2[(c0 + e) >> 1] = add2(v2[(c0 + e) >> 1], dn);
+              float d0, d1;
+              unpack2(dn, d0, d1);
+              pk[e >> 1] = pack_bf16(d0, d1);
+            }
+            tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+          };
+          uint32_t r0[16], r1[16];
+          tmem_ld_32x32b_x16(acc_addr, r0);
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            tmem_wait_ld();
+            tmem_ld_32x32b_x16(acc_addr + c0 + 16, r1);
+            shrink16(r0, c0);
+            tmem_wait_ld();
+            if (c0 + 32 < D) tmem_ld_32x32b_x16(acc_addr + c0 + 32, r0);
+            shrink16(r1, c0 + 16);
+          }
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(&bars->a_full[t]);
+        }
+        // last iteration, exact shrinkage, back in the data's units: alpha^T = 2 theta eta_{1/2}(c + r' - 1/2)
+        w.wait(&bars->r_full[t], phase & 1, 231); ++phase;
+        tc_fence_after();
+        const float two_th = 2.f * kappa;
+#pragma unroll
+        for (int c0 = 0; c0 < D; c0 += 16) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(acc_addr + c0, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) {
+            float a0, a1;
+            unpack2(v2[(c0 + e) >> 1], a0, a1);
+            const float y0 = a0 + __uint_as_float(r[e]) - 0.5f, y1 = a1 + __uint_as_float(r[e + 1]) - 0.5f;
+            v2[(c0 + e) >> 1] = pack2((y0 - fminf(fmaxf(y0, -0.5f), 0.5f)) * two_th, (y1 - fminf(fmaxf(y1, -0.5f), 0.5f)) * two_th);
+          }
+        }
+        if (has_psi) {
+          publish(0);
+          w.wait(&bars->r_full[t], phase & 1, 232); ++phase;
+          tc_fence_after();
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) {
+            uint32_t r[16];
+            tmem_ld_32x32b_x16(acc_addr + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) v2[(c0 + e) >> 1] = pack2u(r[e], r[e + 1]);
+          }
+        }
+      }
+      if (!kUntied && T > 0 && !scaled_units) {
         // layer t uses theta[t * theta_stride + h] (stride 0: one threshold for all layers).  The accumulator is
         // biased by kappa = theta of layer 0 and the registers hold b = alpha - kappa throughout.
         const uint32_t op_addr = tbase + C::kColS;
