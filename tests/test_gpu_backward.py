@@ -217,3 +217,36 @@ def test_backward_edge_cases_on_the_tensor_core_path(name):
         err = rel_err(to_np(g), rf)
         assert err <= BWD_TOL[w.dtype], (name, nm, err)
     ctx.close()
+
+
+def _random_backward_shapes():
+    """Seeded random shapes for both backward paths (bf16 with d in {64, 128}: tensor cores; the rest: FFMA kernels):
+    query, token and measurement counts that are no multiples of any tile, lambda = 0 so that every decision is
+    |x| > 0 on both sides and the oracle needs no decisions supplied."""
+    r = np.random.default_rng(4048)
+    out = []
+    for i in range(10):
+        tc = i % 2 == 0
+        dtype = "bf16" if tc else "fp32"
+        d = (64, 128)[(i // 2) % 2] if tc else int(r.choice([8, 24, 40]))
+        m = int(r.integers(d, 2 * d + 70))
+        n = int(r.integers(m, m + 400))
+        out.append(wl.Workload(f"bwrand{i}", int(r.integers(1, 3)), int(r.integers(1, 4)), n, int(r.integers(1, 300)), d, m,
+                               dtype, int(r.integers(0, 5)), 0.0, "iid", 700 + i))
+    return out
+
+
+@pytest.mark.parametrize("w", _random_backward_shapes(), ids=lambda w: f"{w.name}_{w.dtype}_B{w.B}H{w.H}_n{w.n}_nq{w.n_q}_d{w.d}_m{w.m}_T{w.T}")
+def test_backward_random_shapes_match_oracle(w):
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    phi = to_np(ctx.get_phi())
+    G = wl.round_to_storage(np.random.default_rng(G_SEED + 1).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    got = ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    ref = orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, T=w.T, lam=0.0)
+    for nm, g, rf in zip(("dQ", "dK", "dV"), got, ref):
+        g = to_np(g)
+        assert np.isfinite(g).all()
+        assert rel_err(g, rf) <= BWD_TOL[w.dtype], (w, nm, rel_err(g, rf))
+    ctx.close()
