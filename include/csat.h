@@ -82,6 +82,11 @@ enum {
   CSAT_DEBUG_CANARY = 11, /* debugging aid: 1 fills the K~|V~ workspace with NaN bit patterns (one extra memset on the
                           call's stream) before csat_forward / csat_backward compress, so that a row the compression
                           failed to write shows as NaN in the output instead of reusing an earlier call's values  */
+  CSAT_WEIGHT_GRADS = 12, /* 1: csat_backward also forms the gradients with respect to the decoder's parameters (S, B,
+                          the thresholds, the dictionary) for csat_get_weight_grads; tensor-core path only (bf16, d in
+                          {64, 128}, one S, B for all layers, CSAT_T >= 1), else csat_backward returns
+                          CSAT_ERR_UNSUPPORTED.  It then keeps every layer's iterate and its gradient as bf16:
+                          (2 T + 1) B H n_q d more 16-bit values of scratch.  0 (default): not formed  */
   CSAT_KEEP_MASKS = 9, /* 1: csat_backward also keeps its shrinkage decisions (one 32-bit word per (b, h, query,
                           column); needs CSAT_T <= 32) for csat_get_backward_masks.  0 (default): not kept  */
   CSAT_PROFILE = 6     /* keep per-kernel CUDA-event times of the last v forward calls
@@ -206,6 +211,21 @@ int csat_backward(csat_ctx* ctx, const void* Q, const void* K, const void* V, co
  * with csat_backward's gradients element by element.  Needs CSAT_KEEP_MASKS = 1 before that csat_backward and
  * CSAT_T >= 1, else CSAT_ERR_STATE.  Copied on `stream`. */
 int csat_get_backward_masks(const csat_ctx* ctx, uint32_t* masks_out, void* stream);
+
+/* csat_get_weight_grads -- gradients of the loss with respect to the decoder's parameters, formed by the most recent
+ * csat_backward with CSAT_WEIGHT_GRADS = 1.  The paper trains S, B, theta (its LISTA recurrence
+ * alpha^{t+1} = eta_theta(S alpha^t + B Z_i)) and the dictionary Psi (C^_i = Psi alpha^_i) by backpropagation and
+ * prints no backward pass; this is the chain rule with x_t = alpha^t S + Z B in the row-vector form the library
+ * computes in (csat_set_lista_weights takes S, B in the same form):
+ *   dS     [H, d, d] float32  = sum over layers, queries, batch of (alpha^t)^T dx_t
+ *   dB     [H, d, d] float32  = ... of Z^T dx_t
+ *   dtheta [T, H]    float32  = per layer: - sum of sign(x_t) o dx_t   (one threshold for all layers: add the rows)
+ *   dPsi   [d, d]    float32  = sum over heads too of G^T alpha^T (C^ = alpha^T Psi^T); zeros without a dictionary;
+ *                               may be NULL
+ * with dx_t = d alpha^{t+1} where |x_t| > theta_t, 0 elsewhere.  All device pointers, copied on `stream`.  The
+ * products take the iterates and the dx_t rounded to bf16 and accumulate in float32, in a fixed order (the same bits
+ * on every run).  CSAT_ERR_STATE if no such csat_backward has run. */
+int csat_get_weight_grads(const csat_ctx* ctx, float* dS, float* dB, float* dtheta, float* dPsi, void* stream);
 
 /* csat_project_qkv -- paper: the projection equation Q = X W^Q, K = X W^K, V = X W^V ("Mathematical Framework"),
  * for all heads at once, written in the layout csat_forward reads.

@@ -20,6 +20,7 @@ CSAT_BATCH, CSAT_NQ, CSAT_DTYPE, CSAT_T, CSAT_FORCE_SIMT, CSAT_PROFILE, CSAT_ENS
 CSAT_KEEP_MASKS = 9
 CSAT_HADAMARD_TRANSFORM = 10
 CSAT_DEBUG_CANARY = 11
+CSAT_WEIGHT_GRADS = 12
 CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER, CSAT_ENSEMBLE_HADAMARD = 0, 1, 2
 KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1
@@ -52,6 +53,7 @@ SIGNATURES = {
     "csat_get_compressed": (_int, [_vp, _vp, _vp, _vp]),
     "csat_get_decoder": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_backward_masks": (_int, [_vp, _vp, _vp]),
+    "csat_get_weight_grads": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_profile": (_int, [_vp, _i64, _int, C.POINTER(_int), C.POINTER(C.c_float), C.POINTER(_int)]),
     "csat_attend_noalloc": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _i64, _i64, _int, _dbl, _vp,
                                    C.c_char_p, C.c_size_t]),
@@ -210,6 +212,11 @@ def csat_get_decoder(h, S_out, B_out, theta_out, mu_out, stream=None):
 
 def csat_get_backward_masks(h, masks_out, stream=None):
     _check(h, load().csat_get_backward_masks(h, _ptr(masks_out), _stream(stream)))
+
+
+def csat_get_weight_grads(h, dS, dB, dtheta, dPsi=None, stream=None):
+    _check(h, load().csat_get_weight_grads(h, _ptr(dS), _ptr(dB), _ptr(dtheta), _ptr(dPsi) if dPsi is not None else None,
+                                           _stream(stream)))
 
 
 def csat_get_profile(h, call_index):
@@ -408,6 +415,17 @@ class Csat:
         out = self._new(self.B, self.H, self.n_q, self.d, dtype=torch.int32)
         csat_get_backward_masks(self.h, out)
         return out
+
+    def weight_grads(self):
+        """Gradients with respect to the decoder's parameters from the most recent backward (CSAT_WEIGHT_GRADS = 1):
+        dS [H,d,d], dB [H,d,d], dtheta [T,H], dPsi [d,d] (float32)."""
+        T = csat_get_i64(self.h, CSAT_T)
+        dS = self._new(self.H, self.d, self.d, dtype=torch.float32)
+        dB = self._new(self.H, self.d, self.d, dtype=torch.float32)
+        dth = self._new(T, self.H, dtype=torch.float32)
+        dPsi = self._new(self.d, self.d, dtype=torch.float32)
+        csat_get_weight_grads(self.h, dS, dB, dth, dPsi)
+        return dS, dB, dth, dPsi
 
     def project_qkv(self, X, W, Xkv=None):
         """Q, K, V [B,H,tokens,d] from tokens X [B,n_q,d_model] (and Xkv [B,n,d_model] for cross-attention; default X)

@@ -181,7 +181,9 @@ struct Waiter {
 
 // kMasks (backward pass only, one S, B for all layers): besides the output the kernel leaves what the backward needs:
 // Z (bf16, as fed to the first product), every row's log sum exp, and the decision |x_t| > theta_t of every layer,
-// one bit per column: word c / 32 of (layer, row), bit 31 - c % 32.
+// one bit per column: word c / 32 of (layer, row), bit 31 - c % 32.  With alpha_out (the gradients of the decoder's
+// weights need them) also the iterates alpha^1 .. alpha^T as bf16: alpha^t of (b, h, row) at slot t of alpha_slot
+// elements each (slot 0, alpha^0 = 0, is the caller's to clear).
 template <int D, bool kUntied, bool kMasks>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
@@ -189,7 +191,8 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
                             int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status,
                             float* __restrict__ lse_out, int lse_stride, __nv_bfloat16* __restrict__ z_out,
-                            uint32_t* __restrict__ mask_out) {
+                            uint32_t* __restrict__ mask_out, __nv_bfloat16* __restrict__ alpha_out,
+                            int64_t alpha_slot) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
@@ -656,6 +659,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           zo[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
         }
       }
+      // kMasks: this row's place in slot 0 of the iterates (rows of 2 D bytes from a 256-byte aligned base: 32-byte stores)
+      __nv_bfloat16* arow = (kMasks && alpha_out != nullptr && grow_m < nq)
+                                ? alpha_out + ((int64_t)bh * nq + grow_m) * D : nullptr;
       uint32_t mw[D / 32];                                      // kMasks: the current layer's decisions
       auto store_masks = [&](int layer) {
         if (kMasks && mask_out != nullptr && grow_m < nq) {
@@ -896,6 +902,16 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                 pk[e >> 1] = pack_bf16(d0, d1);
               }
               tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+              if (kMasks && arow != nullptr) {                                 // alpha^{t+1} = b + kappa
+                uint32_t pa[8];
+#pragma unroll
+                for (int e = 0; e < 16; e += 2) {
+                  float a0, a1;
+                  unpack2(v2[(c0 + e) >> 1], a0, a1);
+                  pa[e >> 1] = pack_bf16(a0 + kappa, a1 + kappa);
+                }
+                st_global_v8(arow + (int64_t)(it + 1) * alpha_slot + c0, pa);
+              }
             };
             uint32_t r0[16], r1[16];
             tmem_ld_32x32b_x16(acc_addr, r0);
@@ -937,6 +953,19 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
         store_masks(T - 1);
+        if (kMasks && arow != nullptr) {
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) {
+            uint32_t pa[8];
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) {
+              float a0, a1;
+              unpack2(v2[(c0 + e) >> 1], a0, a1);
+              pa[e >> 1] = pack_bf16(a0, a1);
+            }
+            st_global_v8(arow + (int64_t)T * alpha_slot + c0, pa);
+          }
+        }
         if (has_psi) {
           publish(0);
           w.wait(&bars->r_full[t], phase & 1, 232); ++phase;
@@ -988,7 +1017,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
 
 template <int D, bool kUntied, bool kMasks = false>
 cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T, float* lse_out, int lse_stride,
-                   __nv_bfloat16* z_out = nullptr, uint32_t* mask_out = nullptr) {
+                   __nv_bfloat16* z_out = nullptr, uint32_t* mask_out = nullptr, __nv_bfloat16* alpha_out = nullptr) {
   using C = Cfg<D>;
   const Params& p = c->p;
   CUtensorMap tq;
@@ -1032,7 +1061,8 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kMasks>, tq, c->tmap_kv,
                             kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
                             (int)p.nq, (int)p.m, (int)p.H, T, c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items,
-                            (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out);
+                            (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out, alpha_out,
+                            (int64_t)(p.B * p.H * p.nq * p.d));
 }
 
 }  // namespace
@@ -1071,10 +1101,12 @@ cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, c
 // The forward with what the backward pass needs as its only outputs: Z (bf16), the rows' log sum exp and the layers'
 // shrinkage decisions (one S, B for all layers; the decoded output itself is not stored)
 cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bfloat16* z_out, float* lse_out,
-                                             int lse_stride, uint32_t* mask_out, cudaStream_t s, int* launches) {
+                                             int lse_stride, uint32_t* mask_out, __nv_bfloat16* alpha_out,
+                                             cudaStream_t s, int* launches) {
   *launches += 1;
-  return c->p.d == 64 ? launch<64, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out)
-                      : launch<128, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out);
+  return c->p.d == 64
+             ? launch<64, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
+             : launch<128, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out);
 }
 
 }  // namespace csat

@@ -412,7 +412,11 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   // ... and with one S, B for all layers the per-query stages too: the forward's attention phase leaves Z and the
   // rows' log sum exp, then the recurrence (forward with its decisions recorded, and backward) and dQ
   if (tc_stages && !c->w_untied && c->bw_Z16 != nullptr && (p.T == 0 || c->bw_maskbits != nullptr)) {
-    if ((e = launch_sm100_attend_for_backward(c, Q, c->bw_Z16, c->bw_LD, 2, c->bw_maskbits, s, launches)) != cudaSuccess) return e;
+    const bool wg = c->weight_grads && p.T > 0 && c->bw_alpha16 != nullptr;
+    if (wg && (e = cudaMemsetAsync(c->bw_alpha16, 0, (size_t)(p.B * p.H * p.nq * p.d) * 2, s)) != cudaSuccess) return e;   // alpha^0
+    if ((e = launch_sm100_attend_for_backward(c, Q, c->bw_Z16, c->bw_LD, 2, c->bw_maskbits, wg ? c->bw_alpha16 : nullptr, s,
+                                              launches)) != cudaSuccess)
+      return e;
     if (c->bw_masks != nullptr && p.T > 0) {           // CSAT_KEEP_MASKS: the decisions in the exported layout
       const int64_t total = p.B * p.H * p.nq * p.d;
       expand_masks_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(c->bw_masks, c->bw_maskbits, total, p.nq, d, p.T);
@@ -420,6 +424,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
       *launches += 1;
     }
     if ((e = launch_sm100_bwd_recur(c, G, s, launches)) != cudaSuccess) return e;
+    if (wg && (e = launch_sm100_wgrad(c, G, s, launches)) != cudaSuccess) return e;
     if ((e = launch_sm100_bwd_dq(c, Q, dQ, s, launches)) != cudaSuccess) return e;
     if ((e = launch_sm100_bwd_cols(c, Q, s, launches)) != cudaSuccess) return e;
     return launch_sm100_phiT(c, c->bw_dKV16, dK, dV, s, launches);

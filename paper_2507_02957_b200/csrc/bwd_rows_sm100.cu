@@ -88,7 +88,8 @@ template <int D>
 __global__ void __launch_bounds__(kRThreads, 1)
 bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv_bfloat16* __restrict__ Z16,
                        const __nv_bfloat16* __restrict__ G, __nv_bfloat16* __restrict__ dZ16, float* __restrict__ ws_LD,
-                       const uint32_t* __restrict__ maskbits, int nq, int H, int T, int has_psi, int* status) {
+                       const uint32_t* __restrict__ maskbits, int nq, int H, int T, int has_psi, int* status,
+                       __nv_bfloat16* __restrict__ dx_out, int64_t dx_slot) {
   using C = RCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -175,7 +176,8 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
     int phase = 0;
     uint32_t n_pub = 0;                           // operands published so far (buffer n_pub & 1)
     float v[D];                                   // d alpha_{t+1}, then dx_t
-    auto publish_bf16 = [&]() {                   // v as the bf16 A operand
+    // v as the bf16 A operand; with `keep` also to global memory (dx_t, for the gradients of the decoder's weights)
+    auto publish_bf16 = [&](__nv_bfloat16* keep = nullptr) {
       const uint32_t op_addr = tbase + C::kColOp + (n_pub & 1) * C::kOpCols;
       // the buffer's previous operand (two publications ago) has been read by its trailing product
       if (n_pub >= 2) w.wait(&bars->op_free[n_pub & 1], ((n_pub >> 1) - 1) & 1, 613);
@@ -186,6 +188,11 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
 #pragma unroll
         for (int e = 0; e < 16; e += 2) pk[e >> 1] = pack_bf16(v[c0 + e], v[c0 + e + 1]);
         tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
+        if (keep != nullptr) {
+          uint4* kp = reinterpret_cast<uint4*>(keep + c0);
+          kp[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          kp[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+        }
       }
       tmem_wait_st();
       tc_fence_before();
@@ -229,7 +236,7 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
 #pragma unroll
         for (int c = 0; c < D; ++c)
           v[c] = ((mwd[c >> 5] >> (31 - (c & 31))) & 1u) ? v[c] : 0.f;
-        publish_bf16();
+        publish_bf16(dx_out != nullptr && live && !w.dead ? dx_out + (int64_t)t * dx_slot + goff : nullptr);
         if (t > 0) load_masks(t - 1, mnext);
         w.wait(&bars->r_full, phase & 1, 612); ++phase;
         tc_fence_after();
@@ -480,7 +487,7 @@ cudaError_t launch_recur(csat_ctx* c, const void* G, cudaStream_t s) {
   const dim3 grid((unsigned)((p.nq + kRows - 1) / kRows), (unsigned)(p.B * p.H));
   bwd_recur_sm100_kernel<D><<<grid, kRThreads, C::kSmemBytes, s>>>(
       c->tmap_mats, c->bw_Z16, (const __nv_bfloat16*)G, c->bw_dZ16, c->bw_LD, c->bw_maskbits, (int)p.nq, (int)p.H, p.T,
-      c->psi ? 1 : 0, c->status);
+      c->psi ? 1 : 0, c->status, c->weight_grads ? c->bw_dx16 : nullptr, (int64_t)(p.B * p.H * p.nq * p.d));
   return cudaGetLastError();
 }
 

@@ -118,6 +118,13 @@ void free_backward(csat_ctx* c) {
   dev_free(c, &c->bw_masks, c->bw_bytes_masks);
   dev_free(c, &c->bw_Z16, c->bw_bytes_Z16);
   dev_free(c, &c->bw_maskbits, c->bw_bytes_maskbits);
+  dev_free(c, &c->bw_alpha16, c->bw_bytes_alpha16);
+  dev_free(c, &c->bw_dx16, c->bw_bytes_dx16);
+  dev_free(c, &c->bw_wpart, c->bw_bytes_wpart);
+  dev_free(c, &c->bw_thpart, c->bw_bytes_thpart);
+  dev_free(c, &c->bw_wgrad, c->bw_bytes_wgrad);
+  c->bw_bytes_alpha16 = c->bw_bytes_dx16 = c->bw_bytes_wpart = c->bw_bytes_thpart = c->bw_bytes_wgrad = 0;
+  c->have_wgrads = false;
   c->bw_bytes_Z16 = c->bw_bytes_maskbits = 0;
   c->bw_bytes_masks = 0;
   c->have_masks = false;
@@ -392,6 +399,11 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       if ((v != 0) != c->keep_masks) { cudaDeviceSynchronize(); free_backward(c); }
       c->keep_masks = v != 0;
       return CSAT_OK;
+    case CSAT_WEIGHT_GRADS:
+      if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_WEIGHT_GRADS must be 0 or 1");
+      if ((v != 0) != c->weight_grads) { cudaDeviceSynchronize(); free_backward(c); }
+      c->weight_grads = v != 0;
+      return CSAT_OK;
     case CSAT_PROFILE: {
       if (v < 0 || v > 4096) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_PROFILE must be in [0, 4096]");
       cudaDeviceSynchronize();
@@ -428,6 +440,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
     case CSAT_FORCE_SIMT: *out = c->force_simt; return CSAT_OK;
     case CSAT_PROFILE: *out = c->prof_slots; return CSAT_OK;
     case CSAT_KEEP_MASKS: *out = c->keep_masks ? 1 : 0; return CSAT_OK;
+    case CSAT_WEIGHT_GRADS: *out = c->weight_grads ? 1 : 0; return CSAT_OK;
     case CSAT_HADAMARD_TRANSFORM: *out = c->hadamard_transform; return CSAT_OK;
     case CSAT_DEBUG_CANARY: *out = c->debug_canary; return CSAT_OK;
     default: return CSAT_ERR_INVALID_ARG;
@@ -736,6 +749,10 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
                 "csat_backward: the float32 kernels and CSAT_KEEP_MASKS keep one decision bit per layer in a 32-bit "
                 "word: CSAT_T <= 32");
   if (p.d > 256) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: d <= 256");
+  if (c->weight_grads && !(c->tmap_phi_valid && c->force_simt == 0 && !c->w_untied && p.T > 0))
+    return fail(c, CSAT_ERR_UNSUPPORTED,
+                "CSAT_WEIGHT_GRADS: the gradients of the decoder's parameters are formed on the tensor-core path only "
+                "(bf16, d in {64, 128}, one S, B for all layers, CSAT_T > 0)");
   if (p.B * p.H > 32767) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: B * H <= 32767");
   if (p.T > 0 && c->w_S && (c->w_layers != 1 || c->w_untied) && c->w_layers != p.T)
     return fail(c, CSAT_ERR_STATE, "the supplied LISTA weights are for a number of layers other than CSAT_T");
@@ -750,8 +767,14 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
                bw = (size_t)(2 * (c->w_untied ? c->w_layers : 1) * p.H * p.d * p.d) * 4,
                b16 = c->tmap_phi_valid ? bk / 2 : 0, z16 = c->tmap_phi_valid ? bz / 2 : 0,
                bm = c->keep_masks && p.T > 0 ? bz : 0,
-               bmb = c->tmap_phi_valid ? (size_t)(p.B * p.H * p.T * p.nq * (p.d / 32)) * 4 : 0;
-  if (c->bw_bytes_maskbits != bmb || c->bw_bytes_Z16 != z16 || c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
+               bmb = c->tmap_phi_valid ? (size_t)(p.B * p.H * p.T * p.nq * (p.d / 32)) * 4 : 0,
+               bal = c->weight_grads ? (size_t)((p.T + 1) * p.B * p.H * p.nq * p.d) * 2 : 0,
+               bdx = c->weight_grads ? (size_t)(p.T * p.B * p.H * p.nq * p.d) * 2 : 0,
+               bwp = c->weight_grads ? (size_t)(csat::wgrad_splits(c) * p.H * 2 * p.d * p.d) * 4 : 0,
+               bth = c->weight_grads ? (size_t)(64 * p.T * p.H) * 4 : 0,
+               bwg = c->weight_grads ? (size_t)((2 * p.H + 1) * p.d * p.d + p.T * p.H) * 4 : 0;
+  if (c->bw_bytes_alpha16 != bal || c->bw_bytes_dx16 != bdx || c->bw_bytes_wpart != bwp || c->bw_bytes_thpart != bth ||
+      c->bw_bytes_wgrad != bwg || c->bw_bytes_maskbits != bmb || c->bw_bytes_Z16 != z16 || c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
       c->bw_bytes_dKV16 != b16 || c->bw_bytes_dZ16 != z16) {
     cudaDeviceSynchronize();
     free_backward(c);
@@ -760,7 +783,10 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
     c->bw_bytes_masks = bm;
     c->bw_bytes_Z16 = z16;
     c->bw_bytes_maskbits = bmb;
-    if (dev_alloc(c, &c->bw_maskbits, bmb) != cudaSuccess || dev_alloc(c, &c->bw_Z16, z16) != cudaSuccess || dev_alloc(c, &c->bw_masks, bm) != cudaSuccess || dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
+    c->bw_bytes_alpha16 = bal; c->bw_bytes_dx16 = bdx; c->bw_bytes_wpart = bwp; c->bw_bytes_thpart = bth; c->bw_bytes_wgrad = bwg;
+    if (dev_alloc(c, &c->bw_alpha16, bal) != cudaSuccess || dev_alloc(c, &c->bw_dx16, bdx) != cudaSuccess ||
+        dev_alloc(c, &c->bw_wpart, bwp) != cudaSuccess || dev_alloc(c, &c->bw_thpart, bth) != cudaSuccess ||
+        dev_alloc(c, &c->bw_wgrad, bwg) != cudaSuccess || dev_alloc(c, &c->bw_maskbits, bmb) != cudaSuccess || dev_alloc(c, &c->bw_Z16, z16) != cudaSuccess || dev_alloc(c, &c->bw_masks, bm) != cudaSuccess || dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
         dev_alloc(c, &c->bw_dKV, bk) != cudaSuccess || dev_alloc(c, &c->bw_WT, bw) != cudaSuccess ||
         dev_alloc(c, &c->bw_dKV16, b16) != cudaSuccess || dev_alloc(c, &c->bw_dZ16, z16) != cudaSuccess) {
       free_backward(c);
@@ -775,6 +801,7 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   e = csat::launch_backward(c, Q, dOut, dQ, dK, dV, s, &launches);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward launch");
   c->have_masks = c->bw_masks != nullptr;
+  c->have_wgrads = c->weight_grads && c->bw_wgrad != nullptr;
   c->have_forward = true;
   c->last_launches = launches;
   return CSAT_OK;
@@ -952,6 +979,24 @@ int csat_get_backward_masks(const csat_ctx* c, uint32_t* masks_out, void* stream
     return fail(mc, CSAT_ERR_STATE, "csat_get_backward_masks: no csat_backward with CSAT_KEEP_MASKS = 1 and CSAT_T > 0 has run");
   cudaError_t e = cudaMemcpyAsync(masks_out, c->bw_masks, c->bw_bytes_masks, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(mc, e, "csat_get_backward_masks");
+  return CSAT_OK;
+}
+
+int csat_get_weight_grads(const csat_ctx* c, float* dS, float* dB, float* dtheta, float* dPsi, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  csat_ctx* mc = const_cast<csat_ctx*>(c);
+  if (!dS || !dB || !dtheta) return fail(mc, CSAT_ERR_INVALID_ARG, "csat_get_weight_grads: NULL pointer");
+  if (!c->have_wgrads)
+    return fail(mc, CSAT_ERR_STATE, "csat_get_weight_grads: no csat_backward with CSAT_WEIGHT_GRADS = 1 has run");
+  const csat::Params& p = c->p;
+  const size_t dd = (size_t)(p.d * p.d), hdd = (size_t)p.H * dd;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaError_t e = cudaMemcpyAsync(dS, c->bw_wgrad, hdd * 4, cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dB, c->bw_wgrad + hdd, hdd * 4, cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess && dPsi) e = cudaMemcpyAsync(dPsi, c->bw_wgrad + 2 * hdd, dd * 4, cudaMemcpyDeviceToDevice, s);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(dtheta, c->bw_wgrad + 2 * hdd + dd, (size_t)(p.T * p.H) * 4, cudaMemcpyDeviceToDevice, s);
+  if (e != cudaSuccess) return fail_cuda(mc, e, "csat_get_weight_grads");
   return CSAT_OK;
 }
 

@@ -115,6 +115,15 @@ struct csat_ctx {
   bool have_masks = false;
   uint32_t* bw_masks = nullptr;
   size_t bw_bytes_masks = 0;
+  // CSAT_WEIGHT_GRADS: csat_backward also forms the gradients of the decoder's parameters.  The forward kernel leaves
+  // the iterates alpha^0 .. alpha^T (bf16 [T+1][B,H,n_q,d]) and the recurrence kernel the dx_t (bf16 [T][B,H,n_q,d]);
+  // bw_wpart = per-CTA partial sums [splits][H][2][d][d], bw_thpart = [chunks][T][H],
+  // bw_wgrad = dS [H,d,d] | dB [H,d,d] | dPsi [d,d] | dtheta [T,H]
+  bool weight_grads = false;
+  bool have_wgrads = false;
+  __nv_bfloat16* bw_alpha16 = nullptr; __nv_bfloat16* bw_dx16 = nullptr;
+  float* bw_wpart = nullptr; float* bw_thpart = nullptr; float* bw_wgrad = nullptr;
+  size_t bw_bytes_alpha16 = 0, bw_bytes_dx16 = 0, bw_bytes_wpart = 0, bw_bytes_thpart = 0, bw_bytes_wgrad = 0;
   // staging for csat_forward_host
   void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
   size_t stage_bytes_q = 0, stage_bytes_kv = 0;
@@ -186,8 +195,15 @@ cudaError_t make_layer_weights_tmap(csat_ctx* c);
 cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int* launches);
 // the forward run for the backward pass: z_out [B,H,n_q,d] bf16 = Z, lse_out[row * lse_stride] = log sum exp of the
 // row's scores, mask_out [B,H,T,n_q,d/32] = the layers' decisions |x_t| > theta_t (column c: word c / 32, bit 31 - c % 32)
+// alpha_out (may be null): the iterates alpha^1 .. alpha^T as bf16 into slots 1 .. T of [T+1][B,H,n_q,d]
 cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bfloat16* z_out, float* lse_out,
-                                             int lse_stride, uint32_t* mask_out, cudaStream_t s, int* launches);
+                                             int lse_stride, uint32_t* mask_out, __nv_bfloat16* alpha_out,
+                                             cudaStream_t s, int* launches);
+
+// wgrad_sm100.cu : gradients of the decoder's parameters from the stored iterates and dx_t (bf16, d in {64, 128}, one
+// S, B for all layers) into bw_wgrad; wgrad_splits = CTAs per head of its contraction kernel
+int wgrad_splits(const csat_ctx* c);
+cudaError_t launch_sm100_wgrad(csat_ctx* c, const void* G, cudaStream_t s, int* launches);
 
 // bwd_rows_sm100.cu : the per-query stages of the backward on the tensor cores (bf16, d in {64, 128}, one S, B
 // for all layers).  recur: Z, G -> dZ (bf16 into bw_dZ16), D = <dZ, Z> (into bw_LD), optionally the masks;

@@ -250,3 +250,81 @@ def test_backward_random_shapes_match_oracle(w):
         assert np.isfinite(g).all()
         assert rel_err(g, rf) <= BWD_TOL[w.dtype], (w, nm, rel_err(g, rf))
     ctx.close()
+
+
+WGRAD_CASES = {
+    "bf16_d64": lambda: wl.shrink(C["c2"], B=2, H=3, n_q=150, lam=0.01),
+    "bf16_d64_T1": lambda: wl.shrink(C["c2"], B=1, H=2, n_q=77, T=1, lam=0.01),
+    "bf16_d128": lambda: wl.shrink(C["c5"], B=2, H=2, n=512, n_q=200, m=160, T=8, lam=0.002),
+}
+
+
+@pytest.mark.parametrize("name", sorted(WGRAD_CASES))
+@pytest.mark.parametrize("with_psi", [False, True], ids=["identity", "dictionary"])
+def test_weight_gradients_match_oracle(name, with_psi):
+    """Gradients with respect to the decoder's S, B, thresholds and dictionary (CSAT_WEIGHT_GRADS), against the oracle's
+    per-layer gradients summed over the layers (one S, B for all layers) and over the batch, with the library's own
+    shrinkage decisions (the same protocol as for dQ, dK, dV) and the same tolerance."""
+    w = WGRAD_CASES[name]()
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    binding.csat_set_i64(ctx.h, binding.CSAT_KEEP_MASKS, 1)
+    binding.csat_set_i64(ctx.h, binding.CSAT_WEIGHT_GRADS, 1)
+    d, H, T, B = w.d, w.H, w.T, w.B
+    kw = dict(T=T, lam=w.lam)
+    if with_psi:
+        r = np.random.default_rng(97)
+        Psi = wl.round_to_storage((np.eye(d) + 0.3 * r.standard_normal((d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        ctx.set_dictionary(to_dev(Psi, w.dtype))
+        kw.update(Psi=Psi.astype(np.float64))
+    phi = to_np(ctx.get_phi())
+    G = wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    got_in = ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    words = ctx.backward_masks().cpu().numpy().astype(np.uint32)
+    masks = np.stack([(words >> t) & 1 for t in range(T)], axis=2).astype(bool)
+    stages = []
+    ref_in = orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, masks=masks, stages=stages, **kw)
+    assert len(stages) == B * H
+    dS = np.zeros((H, d, d)); dB = np.zeros((H, d, d)); dth = np.zeros((T, H)); dPsi = np.zeros((d, d))
+    for b in range(B):
+        for h in range(H):
+            st = stages[b * H + h]
+            dS[h] += st["dS"].sum(axis=0)
+            dB[h] += st["dB"].sum(axis=0)
+            dth[:, h] += st["dtheta"]
+            if with_psi:
+                dPsi += st["dPsi"]
+    gS, gB, gth, gPsi = (x.cpu().numpy().astype(np.float64) for x in ctx.weight_grads())
+    tol = BWD_TOL[w.dtype]
+    for nm, g, rf in (("dS", gS, dS), ("dB", gB, dB), ("dtheta", gth, dth)) + ((("dPsi", gPsi, dPsi),) if with_psi else ()):
+        assert np.isfinite(g).all()
+        if T == 1 and nm == "dS":                 # alpha^0 = 0: the only layer has no input iterate
+            assert np.abs(rf).max() == 0.0 and np.abs(g).max() == 0.0
+            continue
+        assert np.abs(rf).max() > 0, nm
+        assert rel_err(g, rf) <= tol, (name, with_psi, nm, rel_err(g, rf))
+    if not with_psi:
+        assert np.abs(gPsi).max() == 0.0
+    # the input gradients are what they are without the key
+    for g, rf in zip(got_in, ref_in):
+        assert rel_err(to_np(g), rf) <= tol
+    # bit-identical on a second run (fixed-order sums)
+    ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    for a, b_ in zip((gS, gB, gth, gPsi), ctx.weight_grads()):
+        assert np.array_equal(a, b_.cpu().numpy().astype(np.float64))
+    ctx.close()
+
+
+def test_weight_gradients_need_the_key_and_the_tensor_core_path():
+    ctx = binding.Csat(64, 16, 8, 1, 0, dtype="fp32", T=2)
+    x = torch.zeros(1, 1, 64, 8, device="cuda")
+    ctx.backward(x, x, x, x)
+    with pytest.raises(binding.CsatError) as ei:
+        ctx.weight_grads()
+    assert ei.value.code == 6
+    binding.csat_set_i64(ctx.h, binding.CSAT_WEIGHT_GRADS, 1)
+    with pytest.raises(binding.CsatError) as ei:
+        ctx.backward(x, x, x, x)                # float32 context: FFMA kernels
+    assert ei.value.code == 5
+    ctx.close()
