@@ -336,12 +336,15 @@ def time_projection(w: wl.Workload, iters: int = 10, warmup: int = 3) -> dict:
     return {"ms": ms, "tflops": f / (ms * 1e-3) / 1e12, "gflop": f / 1e9, "d_model": dm}
 
 
-def time_backward(w: wl.Workload, iters: int = 2) -> dict:
-    """csat_backward (gradients with respect to Q, K, V) on a workload."""
+def time_backward(w: wl.Workload, iters: int = 2, weight_grads: bool = False) -> dict:
+    """csat_backward (gradients with respect to Q, K, V; with weight_grads also to the decoder's S, B, thresholds and
+    dictionary) on a workload."""
     import torch
     from paper_2507_02957_b200 import binding
     host, dev, psi = device_tensors(w)
     ctx = make_ctx(w, psi)
+    if weight_grads:
+        binding.csat_set_i64(ctx.h, binding.CSAT_WEIGHT_GRADS, 1)
     G = torch.randn_like(dev["Q"])
     dQ, dK, dV = torch.empty_like(dev["Q"]), torch.empty_like(dev["K"]), torch.empty_like(dev["V"])
     binding.csat_backward(ctx.h, dev["Q"], dev["K"], dev["V"], G, dQ, dK, dV)
@@ -355,6 +358,9 @@ def time_backward(w: wl.Workload, iters: int = 2) -> dict:
         e1.synchronize()
         times.append(e0.elapsed_time(e1))
     ctx.close()
+    if weight_grads:
+        return {"ms": float(np.median(times)), "kernels": "as backward, plus the iterates and dx_t kept as bf16, a tcgen05 "
+                "contraction over them (dS, dB, dPsi) and a streaming sum (dtheta)"}
     return {"ms": float(np.median(times)),
             "kernels": "bf16: every stage on tcgen05 (forward with decisions recorded, recurrence backward, dQ, dK~|dV~, "
                        "Phi^T); float32: ffma kernels"}
@@ -488,6 +494,9 @@ def run_csat(args, w: wl.Workload) -> dict:
                 extra[f"{w.name}_qkv_projection"] = time_projection(w)
             extra["backward"] = {wl.CONFIGS[k].name: time_backward(wl.CONFIGS[k], iters=1 if k == "c5" else 2)
                                  for k in ("c1", "c2", "c3", "c4", "c5")}
+            extra["backward_with_weight_gradients"] = {
+                wl.CONFIGS[k].name: time_backward(wl.CONFIGS[k], iters=1 if k == "c5" else 2, weight_grads=True)
+                for k in ("c2", "c3", "c4", "c5")}
             result["other_workloads"] = extra
         if not args.no_cpu_baseline:
             inp = {k: host[k].float().numpy() for k in "QKV"}

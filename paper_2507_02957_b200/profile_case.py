@@ -62,6 +62,7 @@ def main():
     bw = sub.add_parser("backward")
     bw.add_argument("name")
     bw.add_argument("--iters", type=int, default=3)
+    bw.add_argument("--weight-grads", action="store_true", help="also form the gradients of the decoder's parameters")
     hd = sub.add_parser("hadamard")
     for name in ("n", "d", "B", "H"):
         hd.add_argument(name, type=int)
@@ -103,6 +104,8 @@ def main():
         ctx = binding.Csat(w.n, w.m, w.d, w.H, w.phi_seed, B=w.B, n_q=w.n_q, dtype=w.dtype, T=w.T, lam=w.lam)
         if inp["Psi"] is not None:
             ctx.set_dictionary(torch.from_numpy(inp["Psi"]).cuda().to(dt))
+        if a.weight_grads:
+            binding.csat_set_i64(ctx.h, binding.CSAT_WEIGHT_GRADS, 1)
         G = torch.randn_like(Q)
         dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
         binding.csat_backward(ctx.h, Q, K, V, G, dQ, dK, dV)
@@ -115,7 +118,7 @@ def main():
             e1.record()
             e1.synchronize()
             times.append(e0.elapsed_time(e1))
-        print(w.name, {"backward_ms": round(float(np.median(times)), 4)})
+        print(w.name, {"backward_ms": round(float(np.median(times)), 4), "weight_grads": bool(a.weight_grads)})
         ctx.close()
     elif a.cmd == "hadamard":
         g = torch.Generator(device="cuda")

@@ -178,3 +178,43 @@ def test_backward_at_the_full_workload_shape(key, pairs):
             err = rel_err(to_np(g[b, h]), rf)
             assert err <= TOL[w.dtype], (key, b, h, nm, err)
     ctx.close()
+
+
+def test_weight_gradients_at_the_full_workload_shape():
+    """CSAT_WEIGHT_GRADS on the whole c3 workload (1248 query tiles, 20 layers): the sums for head 0 against the oracle
+    run over all eight batch elements of that head with the library's decisions; dPsi sums over every head, so it is
+    only checked to be finite.  Same median-survivor lambda as above."""
+    from paper_2507_02957_b200 import binding
+    from gpu_util import to_dev
+    w = wl.CONFIGS["c3"]
+    inp = wl.make_inputs(w)
+    Q, K, V, Psi = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    if Psi is not None:
+        ctx.set_dictionary(Psi)
+    binding.csat_set_i64(ctx.h, binding.CSAT_KEEP_MASKS, 1)
+    binding.csat_set_i64(ctx.h, binding.CSAT_WEIGHT_GRADS, 1)
+    phi = ctx.get_phi()
+    psi64 = None if inp["Psi"] is None else inp["Psi"].astype(np.float64)
+    st = {}
+    orc.csat_forward_head(inp["Q"][0, 0], inp["K"][0, 0], inp["V"][0, 0], to_np(phi[0]), T=1, lam=0.0, Psi=psi64, stages=st)
+    lam = float(np.median(np.abs(st["Z"] @ st["B_dec"])) / st["mu"])
+    ctx.set(lam=lam)
+    G = wl.round_to_storage(np.random.default_rng(303).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    words = ctx.backward_masks()
+    gS, gB, gth, gPsi = (x.cpu().numpy().astype(np.float64) for x in ctx.weight_grads())
+    assert all(np.isfinite(x).all() for x in (gS, gB, gth, gPsi))
+    h = 0
+    dS = np.zeros((w.d, w.d)); dB = np.zeros((w.d, w.d)); dth = np.zeros(w.T)
+    for b in range(w.B):
+        mw = words[b, h].cpu().numpy().astype(np.uint32)
+        masks = np.stack([(mw >> t) & 1 for t in range(w.T)]).astype(bool)
+        stg = {}
+        orc.csat_backward_head(inp["Q"][b, h], inp["K"][b, h], inp["V"][b, h], to_np(phi[h]), G[b, h], T=w.T, lam=lam,
+                               Psi=psi64, masks=masks, stages=stg)
+        dS += stg["dS"].sum(axis=0); dB += stg["dB"].sum(axis=0); dth += stg["dtheta"]
+    for nm, g, rf in (("dS", gS[h], dS), ("dB", gB[h], dB), ("dtheta", gth[:, h], dth)):
+        assert np.abs(rf).max() > 0
+        assert rel_err(g, rf) <= TOL[w.dtype], (nm, rel_err(g, rf))
+    ctx.close()
