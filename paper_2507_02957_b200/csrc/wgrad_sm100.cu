@@ -260,7 +260,7 @@ cudaError_t launch_gram(csat_ctx* c, const CUtensorMap& a1, const CUtensorMap& a
 int wgrad_splits(const csat_ctx* c) {
   const Params& p = c->p;
   const int64_t units = p.B * ((p.nq + kRows - 1) / kRows);
-  int64_t s = (c->sms + p.H - 1) / p.H;
+  int64_t s = c->sms / p.H;                     // one wave: at most sms CTAs in all
   if (s > units) s = units;
   return (int)(s < 1 ? 1 : s);
 }
