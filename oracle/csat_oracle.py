@@ -266,7 +266,9 @@ def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None
     decisions), min_margin [n_q] = min over layers and columns of | |x_t| - theta_t |, dZ, A, Z, and the gradients
     with respect to the decoder's parameters as used in layer t: dS [T,d,d], dB [T,d,d], dtheta [T] (with weights
     shared by the layers the gradient of the shared matrix is the sum over t) and dPsi [d,d] of the
-    reconstruction out = alpha Psi^T (None without a dictionary)."""
+    reconstruction out = alpha Psi^T (None without a dictionary); and dPhi_K = dK~ K^T, dPhi_V = dV~ V^T [m,n], the
+    gradients with respect to the measurement matrices through the compression K~ = Phi K, V~ = Phi_V V with the
+    decoder's matrices held fixed (a Phi shared by keys and values receives their sum)."""
     Q = np.asarray(Q, F64)
     K = np.asarray(K, F64)
     V = np.asarray(V, F64)
@@ -337,6 +339,10 @@ def csat_backward_head(Q, K, V, Phi_h, G, *, T, lam, Psi=None, D=None, step=None
     # K~ = Phi K, V~ = Phi_V V
     dK = Phi_h.T @ dKt
     dV = Phi_v.T @ dVt
+    if stages is not None:
+        # ... and with respect to the measurement matrices themselves (a learned Phi), the decoder's matrices held
+        # fixed: d Phi_K = dK~ K^T, d Phi_V = dV~ V^T, each [m,n]; one shared Phi receives their sum
+        stages.update(dPhi_K=dKt @ K.T, dPhi_V=dVt @ V.T)
     return dQ, dK, dV
 
 

@@ -182,6 +182,23 @@ def _backward_dS_from_the_next_iterate(Q, K, V, Phi_h, G, **kw):
     return out
 
 
+def _backward_dPhi_keys_and_values_exchanged(Q, K, V, Phi_h, G, **kw):
+    st = kw.get("stages")
+    out = _orig_backward_head(Q, K, V, Phi_h, G, **kw)
+    if st is not None:
+        st["dPhi_K"], st["dPhi_V"] = st["dPhi_V"], st["dPhi_K"]
+    return out
+
+
+def _backward_dPhi_transposed_product(Q, K, V, Phi_h, G, **kw):
+    # K~^T-like slip: the gradient of K~ = Phi K taken against the rows of K in reverse order
+    st = kw.get("stages")
+    out = _orig_backward_head(Q, K, V, Phi_h, G, **kw)
+    if st is not None:
+        st["dPhi_K"] = st["dPhi_K"][:, ::-1]
+    return out
+
+
 _orig_lista = orc.lista
 _orig_project = orc.project_qkv
 _orig_backward_head = orc.csat_backward_head
@@ -217,6 +234,8 @@ MUTATIONS = {
     "backward: supplied decisions ignored": ("csat_backward_head", _backward_masks_ignored),
     "backward: d theta loses the sign of x": ("csat_backward_head", _backward_dtheta_without_sign),
     "backward: d S_t taken from the layer after": ("csat_backward_head", _backward_dS_from_the_next_iterate),
+    "backward: d Phi_K and d Phi_V exchanged": ("csat_backward_head", _backward_dPhi_keys_and_values_exchanged),
+    "backward: d Phi_K against the tokens in reverse order": ("csat_backward_head", _backward_dPhi_transposed_product),
     "compress: |Phi|": ("compress", _compress_abs),
     "output: weights ignored": ("compressed_output", _output_uses_unweighted),
 }

@@ -703,7 +703,10 @@ def _backward_case(seed, T, with_psi, separate, untied):
     tB = [torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in B_l]
     tth = [torch.tensor(x, dtype=torch.float64, requires_grad=True) for x in thetas]
     tPsi = None if Psi is None else torch.tensor(Psi, dtype=torch.float64, requires_grad=True)
-    out = _torch_forward(tq, tk, tv, t(Phi), t(Phi if Phi_v is None else Phi_v), tS, tB, tth, tPsi, 1.0 / np.sqrt(d))
+    # the measurement matrices as leaves too (the decoder's matrices above are constants for autograd, i.e. held fixed)
+    tPhi = torch.tensor(Phi, dtype=torch.float64, requires_grad=True)
+    tPhiv = tPhi if Phi_v is None else torch.tensor(Phi_v, dtype=torch.float64, requires_grad=True)
+    out = _torch_forward(tq, tk, tv, tPhi, tPhiv, tS, tB, tth, tPsi, 1.0 / np.sqrt(d))
     # the torch forward is the oracle's forward
     ref_out = orc.csat_forward_head(Q, K, V, Phi, T=T, lam=lam, Psi=Psi, weights=weights, Phi_v_h=Phi_v)
     assert np.allclose(out.detach().numpy(), ref_out, rtol=0, atol=1e-12)
@@ -719,6 +722,11 @@ def _backward_case(seed, T, with_psi, separate, untied):
         assert np.allclose(st["dtheta"][l], tth[l].grad.numpy(), rtol=1e-10, atol=1e-12), ("dtheta", seed, l)
     if Psi is not None and T > 0:
         assert np.allclose(st["dPsi"], tPsi.grad.numpy(), rtol=1e-10, atol=1e-12), ("dPsi", seed)
+    if Phi_v is None:
+        assert np.allclose(st["dPhi_K"] + st["dPhi_V"], tPhi.grad.numpy(), rtol=1e-10, atol=1e-12), ("dPhi", seed)
+    else:
+        assert np.allclose(st["dPhi_K"], tPhi.grad.numpy(), rtol=1e-10, atol=1e-12), ("dPhi_K", seed)
+        assert np.allclose(st["dPhi_V"], tPhiv.grad.numpy(), rtol=1e-10, atol=1e-12), ("dPhi_V", seed)
     if T > 0:
         assert st["masks"].shape == (T, nq, d) and st["xs"].shape == (T, nq, d)
         assert np.array_equal(st["masks"], np.abs(st["xs"]) > np.asarray(thetas)[:, None, None])
