@@ -357,11 +357,26 @@ def time_backward(w: wl.Workload, iters: int = 2, weight_grads: bool = False) ->
         e1.record()
         e1.synchronize()
         times.append(e0.elapsed_time(e1))
+    phi_ms = None
+    if w.dtype == "bf16" and w.d in (64, 128) and not weight_grads:
+        # the gradient with respect to the measurement matrices, from the dK~|dV~ that call left
+        dPhi = torch.empty(w.H, w.m, w.n, dtype=torch.float32, device="cuda")
+        binding.csat_backward_phi(ctx.h, dev["K"], dev["V"], dPhi)
+        torch.cuda.synchronize()
+        tp = []
+        for _ in range(iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            binding.csat_backward_phi(ctx.h, dev["K"], dev["V"], dPhi)
+            e1.record()
+            e1.synchronize()
+            tp.append(e0.elapsed_time(e1))
+        phi_ms = float(np.median(tp))
     ctx.close()
     if weight_grads:
         return {"ms": float(np.median(times)), "kernels": "as backward, plus the iterates and dx_t kept as bf16, a tcgen05 "
                 "contraction over them (dS, dB, dPsi) and a streaming sum (dtheta)"}
-    return {"ms": float(np.median(times)),
+    return {"ms": float(np.median(times)), "backward_phi_ms": phi_ms,
             "kernels": "bf16: every stage on tcgen05 (forward with decisions recorded, recurrence backward, dQ, dK~|dV~, "
                        "Phi^T); float32: ffma kernels"}
 

@@ -227,6 +227,17 @@ int csat_get_backward_masks(const csat_ctx* ctx, uint32_t* masks_out, void* stre
  * on every run).  CSAT_ERR_STATE if no such csat_backward has run. */
 int csat_get_weight_grads(const csat_ctx* ctx, float* dS, float* dB, float* dtheta, float* dPsi, void* stream);
 
+/* csat_backward_phi -- gradient of the loss with respect to the measurement matrices, for a Phi that is learned (the
+ * paper allows fixed or learned sensing matrices and prints no backward pass): the chain rule through the
+ * compression K~ = Phi K, V~ = Phi V with the decoder's matrices held fixed,
+ *   dPhi [H, m, n] float32 = sum over the batch of dK~ K^T + dV~ V^T      (one Phi per head), or
+ *   dPhi [2H, m, n]: the H matrices dPhi_K = sum dK~ K^T, then the H matrices dPhi_V = sum dV~ V^T (CSAT_SEPARATE_PHI).
+ * dK~, dV~ are the ones the most recent csat_backward of this context formed (kept as bf16); K, V [B,H,n,d] (device,
+ * context dtype) must be the tensors that call was given.  One tensor-core product per head with float32
+ * accumulation, written once (H m n floats: size the call for it).  Only after a csat_backward on the tensor-core path
+ * (bf16, d in {64, 128}), else CSAT_ERR_STATE. */
+int csat_backward_phi(csat_ctx* ctx, const void* K, const void* V, float* dPhi, void* stream);
+
 /* csat_project_qkv -- paper: the projection equation Q = X W^Q, K = X W^K, V = X W^V ("Mathematical Framework"),
  * for all heads at once, written in the layout csat_forward reads.
  *   Xq   [B, n_q, d_model]  tokens the queries come from           (context dtype, device)

@@ -54,6 +54,7 @@ SIGNATURES = {
     "csat_get_decoder": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
     "csat_get_backward_masks": (_int, [_vp, _vp, _vp]),
     "csat_get_weight_grads": (_int, [_vp, _vp, _vp, _vp, _vp, _vp]),
+    "csat_backward_phi": (_int, [_vp, _vp, _vp, _vp, _vp]),
     "csat_get_profile": (_int, [_vp, _i64, _int, C.POINTER(_int), C.POINTER(C.c_float), C.POINTER(_int)]),
     "csat_attend_noalloc": (_int, [_vp, _vp, _vp, _vp, _vp, _i64, _i64, _i64, _i64, _i64, _i64, _int, _dbl, _vp,
                                    C.c_char_p, C.c_size_t]),
@@ -217,6 +218,10 @@ def csat_get_backward_masks(h, masks_out, stream=None):
 def csat_get_weight_grads(h, dS, dB, dtheta, dPsi=None, stream=None):
     _check(h, load().csat_get_weight_grads(h, _ptr(dS), _ptr(dB), _ptr(dtheta), _ptr(dPsi) if dPsi is not None else None,
                                            _stream(stream)))
+
+
+def csat_backward_phi(h, K, V, dPhi, stream=None):
+    _check(h, load().csat_backward_phi(h, _ptr(K), _ptr(V), _ptr(dPhi), _stream(stream)))
 
 
 def csat_get_profile(h, call_index):
@@ -414,6 +419,14 @@ class Csat:
         word = |x_t| > theta_t."""
         out = self._new(self.B, self.H, self.n_q, self.d, dtype=torch.int32)
         csat_get_backward_masks(self.h, out)
+        return out
+
+    def backward_phi(self, K, V):
+        """Gradient with respect to the measurement matrices from the most recent backward's dK~, dV~ and the same K, V:
+        float32 [H, m, n] ([2H, m, n] with separate Phi_K / Phi_V)."""
+        heads = self.H * (2 if csat_get_i64(self.h, CSAT_SEPARATE_PHI) else 1)
+        out = self._new(heads, self.m, self.n, dtype=torch.float32)
+        csat_backward_phi(self.h, K, V, out)
         return out
 
     def weight_grads(self):

@@ -125,6 +125,7 @@ void free_backward(csat_ctx* c) {
   dev_free(c, &c->bw_wgrad, c->bw_bytes_wgrad);
   c->bw_bytes_alpha16 = c->bw_bytes_dx16 = c->bw_bytes_wpart = c->bw_bytes_thpart = c->bw_bytes_wgrad = 0;
   c->have_wgrads = false;
+  c->have_dkv16 = false;
   c->bw_bytes_Z16 = c->bw_bytes_maskbits = 0;
   c->bw_bytes_masks = 0;
   c->have_masks = false;
@@ -802,6 +803,7 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward launch");
   c->have_masks = c->bw_masks != nullptr;
   c->have_wgrads = c->weight_grads && c->bw_wgrad != nullptr;
+  c->have_dkv16 = c->bw_dKV16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
   c->have_forward = true;
   c->last_launches = launches;
   return CSAT_OK;
@@ -979,6 +981,25 @@ int csat_get_backward_masks(const csat_ctx* c, uint32_t* masks_out, void* stream
     return fail(mc, CSAT_ERR_STATE, "csat_get_backward_masks: no csat_backward with CSAT_KEEP_MASKS = 1 and CSAT_T > 0 has run");
   cudaError_t e = cudaMemcpyAsync(masks_out, c->bw_masks, c->bw_bytes_masks, cudaMemcpyDeviceToDevice, (cudaStream_t)stream);
   if (e != cudaSuccess) return fail_cuda(mc, e, "csat_get_backward_masks");
+  return CSAT_OK;
+}
+
+int csat_backward_phi(csat_ctx* c, const void* K, const void* V, float* dPhi, void* stream) {
+  if (!c) return CSAT_ERR_INVALID_ARG;
+  if (!K || !V || !dPhi) return fail(c, CSAT_ERR_INVALID_ARG, "csat_backward_phi: NULL pointer");
+  if (!aligned16(K) || !aligned16(V) || !aligned16(dPhi))
+    return fail(c, CSAT_ERR_INVALID_ARG, "csat_backward_phi: pointers must be 16-byte aligned");
+  if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
+  if (!c->have_dkv16)
+    return fail(c, CSAT_ERR_STATE,
+                "csat_backward_phi: no csat_backward on the tensor-core path (bf16, d in {64, 128}) has run on this context");
+  if (*(volatile int*)c->status != 0)
+    return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
+  NvtxRange range("csat_backward_phi");
+  int launches = 0;
+  cudaError_t e = csat::launch_sm100_phigrad(c, K, V, dPhi, (cudaStream_t)stream, &launches);
+  if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward_phi launch");
+  c->last_launches = launches;
   return CSAT_OK;
 }
 

@@ -121,6 +121,7 @@ struct csat_ctx {
   // bw_wgrad = dS [H,d,d] | dB [H,d,d] | dPsi [d,d] | dtheta [T,H]
   bool weight_grads = false;
   bool have_wgrads = false;
+  bool have_dkv16 = false;       // bw_dKV16 holds dK~|dV~ of the most recent csat_backward (tensor-core path)
   __nv_bfloat16* bw_alpha16 = nullptr; __nv_bfloat16* bw_dx16 = nullptr;
   float* bw_wpart = nullptr; float* bw_thpart = nullptr; float* bw_wgrad = nullptr;
   size_t bw_bytes_alpha16 = 0, bw_bytes_dx16 = 0, bw_bytes_wpart = 0, bw_bytes_thpart = 0, bw_bytes_wgrad = 0;
@@ -226,6 +227,9 @@ cudaError_t launch_sm100_bwd_cols(csat_ctx* c, const void* Q, cudaStream_t s, in
 
 // phiT_sm100.cu : dK = Phi_K^T dK~, dV = Phi_V^T dV~ on the tensor cores (bf16, d in {64, 128}); g16 = dK~|dV~ as bf16
 cudaError_t launch_sm100_phiT(csat_ctx* c, const void* g16, void* dK, void* dV, cudaStream_t s, int* launches);
+
+// phigrad_sm100.cu : dPhi [H or 2H, m, n] float32 = sum over the batch of dK~ K^T (+ dV~ V^T), from bw_dKV16
+cudaError_t launch_sm100_phigrad(csat_ctx* c, const void* K, const void* V, float* dPhi, cudaStream_t s, int* launches);
 
 // copies K~ or V~ out of the interleaved workspace: dst [B,H,m,d]
 cudaError_t launch_split_kv(const csat_ctx* c, void* kt, void* vt, cudaStream_t s);

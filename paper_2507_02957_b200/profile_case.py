@@ -63,6 +63,7 @@ def main():
     bw.add_argument("name")
     bw.add_argument("--iters", type=int, default=3)
     bw.add_argument("--weight-grads", action="store_true", help="also form the gradients of the decoder's parameters")
+    bw.add_argument("--phi-grad", action="store_true", help="also time csat_backward_phi (reported separately)")
     hd = sub.add_parser("hadamard")
     for name in ("n", "d", "B", "H"):
         hd.add_argument(name, type=int)
@@ -118,7 +119,21 @@ def main():
             e1.record()
             e1.synchronize()
             times.append(e0.elapsed_time(e1))
-        print(w.name, {"backward_ms": round(float(np.median(times)), 4), "weight_grads": bool(a.weight_grads)})
+        res = {"backward_ms": round(float(np.median(times)), 4), "weight_grads": bool(a.weight_grads)}
+        if a.phi_grad:
+            dPhi = torch.empty(w.H, w.m, w.n, dtype=torch.float32, device="cuda")
+            binding.csat_backward_phi(ctx.h, K, V, dPhi)
+            torch.cuda.synchronize()
+            tp = []
+            for _ in range(a.iters):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                binding.csat_backward_phi(ctx.h, K, V, dPhi)
+                e1.record()
+                e1.synchronize()
+                tp.append(e0.elapsed_time(e1))
+            res["backward_phi_ms"] = round(float(np.median(tp)), 4)
+        print(w.name, res)
         ctx.close()
     elif a.cmd == "hadamard":
         g = torch.Generator(device="cuda")

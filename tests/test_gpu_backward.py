@@ -328,3 +328,65 @@ def test_weight_gradients_need_the_key_and_the_tensor_core_path():
         ctx.backward(x, x, x, x)                # float32 context: FFMA kernels
     assert ei.value.code == 5
     ctx.close()
+
+
+PHIGRAD_CASES = {
+    "bf16_d64": lambda: wl.shrink(C["c2"], B=2, H=3, n_q=150, lam=0.01),                            # n = 197: ragged, odd
+    "bf16_d128": lambda: wl.shrink(C["c5"], B=2, H=2, n=520, n_q=200, m=160, T=8, lam=0.002),       # m, n ragged tiles
+    "bf16_d64_T0": lambda: wl.shrink(C["c2"], B=1, H=2, n=300, n_q=77, m=130, T=0),
+}
+
+
+@pytest.mark.parametrize("name", sorted(PHIGRAD_CASES))
+@pytest.mark.parametrize("separate", [False, True], ids=["shared_phi", "separate_phi"])
+def test_measurement_matrix_gradient_matches_oracle(name, separate):
+    """csat_backward_phi (d Phi = sum over the batch of dK~ K^T + dV~ V^T, decoder held fixed) against the oracle's
+    dPhi_K, dPhi_V summed the same way, with the library's shrinkage decisions; element by element, the tolerance of
+    every other gradient."""
+    w = PHIGRAD_CASES[name]()
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    if separate:
+        ctx.set(separate_phi=True)
+    binding.csat_set_i64(ctx.h, binding.CSAT_KEEP_MASKS, 1)
+    H, T, B = w.H, w.T, w.B
+    phi = to_np(ctx.get_phi())
+    kw = dict(T=T, lam=w.lam)
+    if separate:
+        kw.update(Phi_V=phi[H:])
+        phi = phi[:H]
+    G = wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    masks = None
+    if T > 0:
+        words = ctx.backward_masks().cpu().numpy().astype(np.uint32)
+        masks = np.stack([(words >> t) & 1 for t in range(T)], axis=2).astype(bool)
+    got = ctx.backward_phi(K, V).cpu().numpy().astype(np.float64)
+    stages = []
+    orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, masks=masks, stages=stages, **kw)
+    ref = np.zeros_like(got)
+    for b in range(B):
+        for h in range(H):
+            st = stages[b * H + h]
+            if separate:
+                ref[h] += st["dPhi_K"]
+                ref[H + h] += st["dPhi_V"]
+            else:
+                ref[h] += st["dPhi_K"] + st["dPhi_V"]
+    assert got.shape == ((2 * H if separate else H), w.m, w.n)
+    assert np.isfinite(got).all() and np.abs(ref).max() > 0
+    assert rel_err(got, ref) <= BWD_TOL[w.dtype], (name, separate, rel_err(got, ref))
+    assert torch.equal(ctx.backward_phi(K, V), torch.from_numpy(got.astype(np.float32)).cuda())
+    ctx.close()
+
+
+def test_measurement_matrix_gradient_needs_a_backward_first():
+    w = wl.shrink(C["c2"], B=1, H=1, n_q=64, T=2)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    with pytest.raises(binding.CsatError) as ei:
+        ctx.backward_phi(K, V)
+    assert ei.value.code == 6
+    ctx.close()

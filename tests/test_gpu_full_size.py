@@ -183,7 +183,8 @@ def test_backward_at_the_full_workload_shape(key, pairs):
 def test_weight_gradients_at_the_full_workload_shape():
     """CSAT_WEIGHT_GRADS on the whole c3 workload (1248 query tiles, 20 layers): the sums for head 0 against the oracle
     run over all eight batch elements of that head with the library's decisions; dPsi sums over every head, so it is
-    only checked to be finite.  Same median-survivor lambda as above."""
+    only checked to be finite.  The same oracle calls give head 0's gradient of the measurement matrix
+    (csat_backward_phi).  Same median-survivor lambda as above."""
     from paper_2507_02957_b200 import binding
     from gpu_util import to_dev
     w = wl.CONFIGS["c3"]
@@ -205,8 +206,10 @@ def test_weight_gradients_at_the_full_workload_shape():
     words = ctx.backward_masks()
     gS, gB, gth, gPsi = (x.cpu().numpy().astype(np.float64) for x in ctx.weight_grads())
     assert all(np.isfinite(x).all() for x in (gS, gB, gth, gPsi))
+    gPhi = ctx.backward_phi(K, V)
+    assert gPhi.shape == (w.H, w.m, w.n) and torch.isfinite(gPhi).all()
     h = 0
-    dS = np.zeros((w.d, w.d)); dB = np.zeros((w.d, w.d)); dth = np.zeros(w.T)
+    dS = np.zeros((w.d, w.d)); dB = np.zeros((w.d, w.d)); dth = np.zeros(w.T); dPhi = np.zeros((w.m, w.n))
     for b in range(w.B):
         mw = words[b, h].cpu().numpy().astype(np.uint32)
         masks = np.stack([(mw >> t) & 1 for t in range(w.T)]).astype(bool)
@@ -214,7 +217,9 @@ def test_weight_gradients_at_the_full_workload_shape():
         orc.csat_backward_head(inp["Q"][b, h], inp["K"][b, h], inp["V"][b, h], to_np(phi[h]), G[b, h], T=w.T, lam=lam,
                                Psi=psi64, masks=masks, stages=stg)
         dS += stg["dS"].sum(axis=0); dB += stg["dB"].sum(axis=0); dth += stg["dtheta"]
-    for nm, g, rf in (("dS", gS[h], dS), ("dB", gB[h], dB), ("dtheta", gth[:, h], dth)):
+        dPhi += stg["dPhi_K"] + stg["dPhi_V"]
+    for nm, g, rf in (("dS", gS[h], dS), ("dB", gB[h], dB), ("dtheta", gth[:, h], dth),
+                      ("dPhi", gPhi[h].cpu().numpy().astype(np.float64), dPhi)):
         assert np.abs(rf).max() > 0
         assert rel_err(g, rf) <= TOL[w.dtype], (nm, rel_err(g, rf))
     ctx.close()
