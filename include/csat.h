@@ -194,10 +194,11 @@ int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, c
  * first call allocates scratch (B H (n_q (d + 2) + 2 m d) floats and transposed copies of the decoder matrices;
  * bf16 copies of Z, dZ and dK~|dV~ and B H T n_q d / 32 decision words on the tensor-core path; B H n_q d words
  * more with CSAT_KEEP_MASKS; all counted by csat_workspace_bytes).
- * Two paths.  bf16 contexts with d in {64, 128} and tied layers run every stage on the tensor cores: the forward
+ * Two paths.  bf16 contexts with d in {64, 128} run every stage on the tensor cores (one S, B for all layers, or one
+ * pair per layer streamed through shared memory from the last layer to the first): the forward
  * kernel once more (it keeps Z, the softmax statistics and one decision bit per layer, query and column), the
  * backward recurrence, dQ, the gradients of K~|V~ (P^T dZ, dS^T Q) and the product with Phi^T, all with bf16
- * operands and float32 accumulation; any CSAT_T.  Everything else (float32 contexts, other d, untied layers) runs
+ * operands and float32 accumulation; any CSAT_T.  Everything else (float32 contexts, other d) runs
  * float32 FFMA kernels that recompute each query row and keep the decisions of one (query, column) in one word:
  * CSAT_T <= 32 there and with CSAT_KEEP_MASKS.  d <= 256 and B H <= 32767.  Otherwise CSAT_ERR_UNSUPPORTED. */
 int csat_backward(csat_ctx* ctx, const void* Q, const void* K, const void* V, const void* dOut, void* dQ, void* dK,

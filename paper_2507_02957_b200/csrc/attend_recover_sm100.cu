@@ -704,6 +704,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           const float thn = it + 2 < T ? theta[(int64_t)(it + 1) * theta_stride + h] : 0.f;
           const float inv2th = th > 0.f ? 0.5f / th : 0.f;          // theta = 0: sat(0) = 0 and eta(x) = x
           const F2 m2th2 = pack2(-2.f * th, -2.f * th);
+          const F2 p2th2 = pack2(2.f * th, 2.f * th);
           const F2 nx2 = pack2(thn, thn);
           w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
           tc_fence_after();
@@ -714,6 +715,13 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
               const F2 y2 = add2(v2[(c0 + e) >> 1], pack2u(r[e], r[e + 1]));   // alpha^t S_t + z B_t + theta_t
               float y0, y1;
               unpack2(y2, y0, y1);
+              if (kMasks) {
+                // |x| > theta  <=>  y < 0 or y > 2 theta  <=>  y (2 theta - y) < 0: its sign bit is the decision
+                float g0, g1;
+                unpack2(mul2(y2, fma2(y2, pack2(-1.f, -1.f), p2th2)), g0, g1);
+                mw[c0 >> 5] = __funnelshift_l(__float_as_uint(g0), mw[c0 >> 5], 1);
+                mw[c0 >> 5] = __funnelshift_l(__float_as_uint(g1), mw[c0 >> 5], 1);
+              }
               const F2 t2 = pack2(fma_sat(y0, inv2th, 0.f), fma_sat(y1, inv2th, 0.f));
               const F2 an = fma2(t2, m2th2, y2);                               // alpha^{t+1} = eta_theta(x)
               v2[(c0 + e) >> 1] = add2(an, nx2);
@@ -737,6 +745,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           tmem_wait_st();
           tc_fence_before();
           mbar_arrive(&bars->a_full[t]);
+          store_masks(it);
         }
         const float th = theta[(int64_t)(T - 1) * theta_stride + h];
         w.wait(&bars->r_full[t], phase & 1, 231); ++phase;
@@ -751,9 +760,14 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             float b0, b1;
             unpack2(v2[(c0 + e) >> 1], b0, b1);
             const float x0 = b0 + __uint_as_float(r[e]), x1 = b1 + __uint_as_float(r[e + 1]);
+            if (kMasks) {
+              mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x0)), mw[c0 >> 5], 1);
+              mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x1)), mw[c0 >> 5], 1);
+            }
             v2[(c0 + e) >> 1] = pack2(x0 - fminf(fmaxf(x0, -th), th), x1 - fminf(fmaxf(x1, -th), th));
           }
         }
+        store_masks(T - 1);
         if (has_psi) {
           publish(D / 2);
           w.wait(&bars->r_full[t], phase & 1, 232); ++phase;
@@ -1104,6 +1118,9 @@ cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bf
                                              int lse_stride, uint32_t* mask_out, __nv_bfloat16* alpha_out,
                                              cudaStream_t s, int* launches) {
   *launches += 1;
+  if (c->w_S && c->w_untied && c->p.T > 0)      // one S_t, B_t per layer (no iterates kept: alpha_out is for tied layers)
+    return c->p.d == 64 ? launch<64, true, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out)
+                        : launch<128, true, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out);
   return c->p.d == 64
              ? launch<64, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
              : launch<128, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out);

@@ -411,7 +411,7 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   const bool tc_stages = c->bw_dKV16 != nullptr && c->bw_dZ16 != nullptr && c->tmap_phi_valid && c->force_simt == 0;
   // ... and with one S, B for all layers the per-query stages too: the forward's attention phase leaves Z and the
   // rows' log sum exp, then the recurrence (forward with its decisions recorded, and backward) and dQ
-  if (tc_stages && !c->w_untied && c->bw_Z16 != nullptr && (p.T == 0 || c->bw_maskbits != nullptr)) {
+  if (tc_stages && c->bw_Z16 != nullptr && (p.T == 0 || c->bw_maskbits != nullptr)) {
     const bool wg = c->weight_grads && p.T > 0 && c->bw_alpha16 != nullptr;
     if (wg && (e = cudaMemsetAsync(c->bw_alpha16, 0, (size_t)(p.B * p.H * p.nq * p.d) * 2, s)) != cudaSuccess) return e;   // alpha^0
     if ((e = launch_sm100_attend_for_backward(c, Q, c->bw_Z16, c->bw_LD, 2, c->bw_maskbits, wg ? c->bw_alpha16 : nullptr, s,

@@ -63,12 +63,14 @@ struct Waiter {
 // ====================================================================================================================
 // recurrence backward
 // ====================================================================================================================
-template <int D> struct RCfg {
+// kUntied: one S_t, B_t per layer: the pair of the layer at work and the pair of the next one (two stages), then Psi
+template <int D, bool kUntied = false> struct RCfg {
   static constexpr int kDBoxes = D / 64;
   static constexpr uint32_t kMatBoxBytes = D * 128;               // one 64-column box of a d x d bf16 matrix
   static constexpr uint32_t kMatBytes = kDBoxes * kMatBoxBytes;
-  static constexpr uint32_t kOffMat = 0;                          // [3]: S - I | B^T | Psi, as the forward stages them
-  static constexpr uint32_t kOffBar = 3 * kMatBytes;
+  static constexpr uint32_t kOffMat = 0;                          // [3]: S - I | B | Psi, as the forward stages them
+  static constexpr int kMats = kUntied ? 5 : 3;                   // untied: [stage 0: S_t - I | B_t][stage 1: ...][Psi]
+  static constexpr uint32_t kOffBar = kMats * kMatBytes;
   static constexpr uint32_t kSmemBytes = kOffBar + 128 + 1024 /*alignment slack*/;
   // TMEM columns: accumulator | dZ accumulator | two bf16 operand buffers (two values per column)
   static constexpr uint32_t kColAcc = 0, kColDz = D, kColOp = 2 * D, kOpCols = D / 2;
@@ -78,19 +80,20 @@ template <int D> struct RCfg {
 
 struct RBars {
   uint64_t mats_full, a_full, r_full, op_free[2];
+  uint64_t lm_full[2], lm_free[2];   // untied layers: a stage's pair of matrices has landed / has been read
   uint32_t tmem_slot;
   int abort;
 };
 
 constexpr int kRThreads = 160;      // warps 0-3: one thread per query row; warp 4: TMA and MMA issue
 
-template <int D>
+template <int D, bool kUntied>
 __global__ void __launch_bounds__(kRThreads, 1)
 bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv_bfloat16* __restrict__ Z16,
                        const __nv_bfloat16* __restrict__ G, __nv_bfloat16* __restrict__ dZ16, float* __restrict__ ws_LD,
                        const uint32_t* __restrict__ maskbits, int nq, int H, int T, int has_psi, int* status,
                        __nv_bfloat16* __restrict__ dx_out, int64_t dx_slot) {
-  using C = RCfg<D>;
+  using C = RCfg<D, kUntied>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   RBars* bars = reinterpret_cast<RBars*>(smem + C::kOffBar);
@@ -105,6 +108,7 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
     mbar_init(&bars->r_full, 1);
     mbar_init(&bars->op_free[0], 1);
     mbar_init(&bars->op_free[1], 1);
+    for (int s2 = 0; s2 < 2; ++s2) { mbar_init(&bars->lm_full[s2], 1); mbar_init(&bars->lm_free[s2], 1); }
     bars->abort = 0;
     fence_mbar_init();
   }
@@ -120,19 +124,39 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
   if (warp == 4) {
     if (T > 0 && elect_one()) {
       // ---- the decoder matrices of this head, then one MMA group per operand the threads publish ----
-      const int nmats = has_psi ? 3 : 2;
-      mbar_arrive_expect_tx(&bars->mats_full, nmats * C::kMatBytes);
-      for (int mat = 0; mat < nmats; ++mat)
+      // one S, B for all layers: tiles S - I | B | Psi of head h, loaded once.  One pair per layer (kUntied): the
+      // tensor holds, per head, S_0 - I, B_0, S_1 - I, B_1, ..., then Psi; the layers are walked from the last to the
+      // first through two stages, the pair of layer t - 2 loaded into the stage layer t's products have just read.
+      const int mat0 = kUntied ? h * (2 * T + 1) : h * 3;
+      auto load_mat = [&](int slot, int index, uint64_t* bar) {
         for (int gx = 0; gx < C::kDBoxes; ++gx)
-          tma_load_3d(smem + C::kOffMat + mat * C::kMatBytes + gx * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, gx * 64,
-                      0, h * 3 + mat);
+          tma_load_3d(smem + C::kOffMat + slot * C::kMatBytes + gx * C::kMatBoxBytes, &tmap_mats, bar, gx * 64, 0, index);
+      };
+      auto load_layer = [&](int t) {              // into stage (T - 1 - t) & 1
+        const int st = (T - 1 - t) & 1;
+        mbar_arrive_expect_tx(&bars->lm_full[st], 2 * C::kMatBytes);
+        load_mat(2 * st, mat0 + 2 * t, &bars->lm_full[st]);
+        load_mat(2 * st + 1, mat0 + 2 * t + 1, &bars->lm_full[st]);
+      };
+      if (kUntied) {
+        if (has_psi) {
+          mbar_arrive_expect_tx(&bars->mats_full, C::kMatBytes);
+          load_mat(4, mat0 + 2 * T, &bars->mats_full);
+        }
+        load_layer(T - 1);
+        if (T > 1) load_layer(T - 2);
+      } else {
+        const int nmats = has_psi ? 3 : 2;
+        mbar_arrive_expect_tx(&bars->mats_full, nmats * C::kMatBytes);
+        for (int mat = 0; mat < nmats; ++mat) load_mat(mat, mat0 + mat, &bars->mats_full);
+      }
       constexpr uint32_t idesc_t = make_idesc_bf16(kRows, D, false, true);    // transposed products: B MN-major
       const uint32_t acc = tmem + C::kColAcc, dz = tmem + C::kColDz;
       // product with the transpose of a matrix the forward stores [output column][k]: the tile's rows are now the
       // reduction index, 16 rows (2048 bytes) per K step, the next 64 output columns one box further.  The operands
       // alternate between two buffers (publication n uses buffer n & 1).
-      auto mma_tr = [&](uint32_t d_t, uint32_t op, int mat, uint32_t accumulate) {
-        const uint64_t bd = make_smem_desc(smem_u32(smem + C::kOffMat + mat * C::kMatBytes), C::kMatBoxBytes, 1024);
+      auto mma_tr = [&](uint32_t d_t, uint32_t op, int slot, uint32_t accumulate) {
+        const uint64_t bd = make_smem_desc(smem_u32(smem + C::kOffMat + slot * C::kMatBytes), C::kMatBoxBytes, 1024);
 #pragma unroll
         for (int k = 0; k < D / 16; ++k) mma_f16_ts(d_t, op + k * 8, bd + (uint64_t)(k * 128), idesc_t, k == 0 ? accumulate : 1u);
       };
@@ -142,28 +166,43 @@ bwd_recur_sm100_kernel(const __grid_constant__ CUtensorMap tmap_mats, const __nv
         ++n_ops;
         tc_fence_after();
       };
-      w.wait(&bars->mats_full, 0, 600);
+      if (!kUntied || has_psi) w.wait(&bars->mats_full, 0, 600);
       // The threads only wait for the product they need next (r_full); the dZ product trails it and releases the
       // operand buffer (op_free) when it has read it.
       if (has_psi) {                                           // d alpha_T = G Psi
         const uint32_t op = tmem + C::kColOp + (n_ops & 1) * C::kOpCols;
         operand_ready();
-        mma_tr(acc, op, 2, 0u);
+        mma_tr(acc, op, kUntied ? 4 : 2, 0u);
         mma_commit(&bars->r_full);
         mma_commit(&bars->op_free[(n_ops - 1) & 1]);
       }
       for (int t = T - 1; t >= 0; --t) {
         const uint32_t op = tmem + C::kColOp + (n_ops & 1) * C::kOpCols;
+        const int li = T - 1 - t, st = li & 1;                 // untied: this layer's stage
         operand_ready();
+        if (kUntied) {
+          w.wait(&bars->lm_full[st], (li >> 1) & 1, 602);
+          tc_fence_after();
+        }
+        const int sS = kUntied ? 2 * st : 0, sB = kUntied ? 2 * st + 1 : 1;
         if (t > 0) {
-          mma_tr(acc, op, 0, 0u);                              // dx_t (S - I)^T
+          mma_tr(acc, op, sS, 0u);                             // dx_t (S_t - I)^T
           mma_commit(&bars->r_full);
         }
-        mma_tr(dz, op, 1, t == T - 1 ? 0u : 1u);               // dZ += dx_t B^T
+        mma_tr(dz, op, sB, t == T - 1 ? 0u : 1u);              // dZ += dx_t B_t^T
         if (t == 0) mma_commit(&bars->r_full);                 // the last result the threads wait for is dZ itself
         mma_commit(&bars->op_free[(n_ops - 1) & 1]);
+        if (kUntied && t >= 2) {                               // the stage is free once these products have read it
+          mma_commit(&bars->lm_free[st]);
+          w.wait(&bars->lm_free[st], (li >> 1) & 1, 603);
+          if (!w.dead) load_layer(t - 2);
+        }
       }
-      if (w.dead) mbar_wait_drain(&bars->mats_full, 0);
+      if (w.dead && kUntied) {                                 // gave up: let the copies in flight land
+        mbar_wait_drain(&bars->lm_full[0], 0);                 // (whichever phase: a bounded wait either way)
+        mbar_wait_drain(&bars->lm_full[1], 0);
+      }
+      if (w.dead && (!kUntied || has_psi)) mbar_wait_drain(&bars->mats_full, 0);
     }
   } else {
     // ---------------------------------------------- one thread per query row ----------------------------------------
@@ -477,16 +516,16 @@ bwd_dq_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
   if (warp == 5) tmem_dealloc(tmem, C::kTmemCols);
 }
 
-template <int D>
+template <int D, bool kUntied>
 cudaError_t launch_recur(csat_ctx* c, const void* G, cudaStream_t s) {
-  using C = RCfg<D>;
+  using C = RCfg<D, kUntied>;
   const Params& p = c->p;
   static DeviceFlags smem_opt_in;
-  cudaError_t e = ensure_dynamic_smem(bwd_recur_sm100_kernel<D>, (int)C::kSmemBytes, c->device, smem_opt_in);
+  cudaError_t e = ensure_dynamic_smem(bwd_recur_sm100_kernel<D, kUntied>, (int)C::kSmemBytes, c->device, smem_opt_in);
   if (e != cudaSuccess) return e;
   const dim3 grid((unsigned)((p.nq + kRows - 1) / kRows), (unsigned)(p.B * p.H));
-  bwd_recur_sm100_kernel<D><<<grid, kRThreads, C::kSmemBytes, s>>>(
-      c->tmap_mats, c->bw_Z16, (const __nv_bfloat16*)G, c->bw_dZ16, c->bw_LD, c->bw_maskbits, (int)p.nq, (int)p.H, p.T,
+  bwd_recur_sm100_kernel<D, kUntied><<<grid, kRThreads, C::kSmemBytes, s>>>(
+      kUntied ? c->tmap_lmats : c->tmap_mats, c->bw_Z16, (const __nv_bfloat16*)G, c->bw_dZ16, c->bw_LD, c->bw_maskbits, (int)p.nq, (int)p.H, p.T,
       c->psi ? 1 : 0, c->status, c->weight_grads ? c->bw_dx16 : nullptr, (int64_t)(p.B * p.H * p.nq * p.d));
   return cudaGetLastError();
 }
@@ -515,7 +554,9 @@ cudaError_t launch_dq(csat_ctx* c, const void* Q, void* dQ, cudaStream_t s) {
 
 cudaError_t launch_sm100_bwd_recur(csat_ctx* c, const void* G, cudaStream_t s, int* launches) {
   *launches += 1;
-  return c->p.d == 64 ? launch_recur<64>(c, G, s) : launch_recur<128>(c, G, s);
+  if (c->w_S && c->w_untied && c->p.T > 0)
+    return c->p.d == 64 ? launch_recur<64, true>(c, G, s) : launch_recur<128, true>(c, G, s);
+  return c->p.d == 64 ? launch_recur<64, false>(c, G, s) : launch_recur<128, false>(c, G, s);
 }
 
 cudaError_t launch_sm100_bwd_dq(csat_ctx* c, const void* Q, void* dQ, cudaStream_t s, int* launches) {

@@ -744,7 +744,7 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
   if (*(volatile int*)c->status != 0)
     return fail(c, CSAT_ERR_TIMEOUT, "a bounded device-side wait of an earlier launch gave up; its output is invalid");
   const csat::Params& p = c->p;
-  const bool tc_all_stages = c->tmap_phi_valid && c->force_simt == 0 && !c->w_untied && !c->keep_masks;
+  const bool tc_all_stages = c->tmap_phi_valid && c->force_simt == 0 && !c->keep_masks;
   if (p.T > 32 && !tc_all_stages)
     return fail(c, CSAT_ERR_UNSUPPORTED,
                 "csat_backward: the float32 kernels and CSAT_KEEP_MASKS keep one decision bit per layer in a 32-bit "

@@ -64,6 +64,7 @@ def main():
     bw.add_argument("--iters", type=int, default=3)
     bw.add_argument("--weight-grads", action="store_true", help="also form the gradients of the decoder's parameters")
     bw.add_argument("--phi-grad", action="store_true", help="also time csat_backward_phi (reported separately)")
+    bw.add_argument("--untied", action="store_true", help="one random S_t, B_t per layer instead of the ISTA-derived pair")
     hd = sub.add_parser("hadamard")
     for name in ("n", "d", "B", "H"):
         hd.add_argument(name, type=int)
@@ -107,6 +108,13 @@ def main():
             ctx.set_dictionary(torch.from_numpy(inp["Psi"]).cuda().to(dt))
         if a.weight_grads:
             binding.csat_set_i64(ctx.h, binding.CSAT_WEIGHT_GRADS, 1)
+        if a.untied and w.T > 0:
+            g = torch.Generator(device="cuda")
+            g.manual_seed(1)
+            sc = 1.0 / np.sqrt(w.d)
+            S = (0.6 * torch.eye(w.d, device="cuda") + 0.4 * sc * torch.randn(w.T, w.H, w.d, w.d, device="cuda", generator=g)).to(dt)
+            Bm = (sc * torch.randn(w.T, w.H, w.d, w.d, device="cuda", generator=g)).to(dt)
+            ctx.set_lista_layer_weights(S, Bm, torch.full((w.T, w.H), 0.02, device="cuda"))
         G = torch.randn_like(Q)
         dQ, dK, dV = torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V)
         binding.csat_backward(ctx.h, Q, K, V, G, dQ, dK, dV)
@@ -119,7 +127,7 @@ def main():
             e1.record()
             e1.synchronize()
             times.append(e0.elapsed_time(e1))
-        res = {"backward_ms": round(float(np.median(times)), 4), "weight_grads": bool(a.weight_grads)}
+        res = {"backward_ms": round(float(np.median(times)), 4), "weight_grads": bool(a.weight_grads), "untied": bool(a.untied)}
         if a.phi_grad:
             dPhi = torch.empty(w.H, w.m, w.n, dtype=torch.float32, device="cuda")
             binding.csat_backward_phi(ctx.h, K, V, dPhi)
