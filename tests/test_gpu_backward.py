@@ -390,3 +390,44 @@ def test_measurement_matrix_gradient_needs_a_backward_first():
         ctx.backward_phi(K, V)
     assert ei.value.code == 6
     ctx.close()
+
+
+@pytest.mark.parametrize("T", [1, 2, 3, 5])
+@pytest.mark.parametrize("with_psi", [False, True], ids=["identity", "dictionary"])
+def test_backward_with_per_layer_weights_small_depths(T, with_psi):
+    """One S_t, B_t per layer on the tensor-core path at the depths where its two-stage ring of layer matrices starts,
+    wraps and ends (1, 2, 3, 5 layers), with and without a dictionary; the usual two-part comparison."""
+    w = wl.shrink(C["c2"], B=1, H=2, n_q=100, T=T, lam=0.01)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    binding.csat_set_i64(ctx.h, binding.CSAT_KEEP_MASKS, 1)
+    r = np.random.default_rng(11 + T)
+    d, H = w.d, w.H
+    kw = dict(T=T, lam=w.lam)
+    if with_psi:
+        Psi = wl.round_to_storage((np.eye(d) + 0.3 * r.standard_normal((d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        ctx.set_dictionary(to_dev(Psi, w.dtype))
+        kw.update(Psi=Psi.astype(np.float64))
+    S = wl.round_to_storage((0.6 * np.eye(d) + 0.4 * r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+    Bm = wl.round_to_storage((r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+    phi = to_np(ctx.get_phi())
+    st0 = []
+    orc.csat_forward(inp["Q"][:1], inp["K"][:1], inp["V"][:1], phi, T=0, lam=0.0, stages=st0)
+    th0 = float(np.median(np.abs(st0[0]["Z"] @ Bm[0, 0].astype(np.float64))))
+    thetas = (th0 * r.uniform(0.2, 1.5, size=(T, H))).astype(np.float32)
+    ctx.set_lista_layer_weights(to_dev(S, w.dtype), to_dev(Bm, w.dtype), torch.from_numpy(thetas).cuda())
+    kw.update(weights=(S.astype(np.float64), Bm.astype(np.float64), list(thetas.astype(np.float64))))
+    G = wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    got = ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    # the six tensor-core kernels and the mask export, plus the operand set-up on the first call
+    assert binding.csat_last_launch_count(ctx.h) in (7, 8)
+    words = ctx.backward_masks().cpu().numpy().astype(np.uint32)
+    masks = np.stack([(words >> t) & 1 for t in range(T)], axis=2).astype(bool)
+    stages = []
+    ref = orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, masks=masks, stages=stages, **kw)
+    own = np.stack([s["masks"] for s in stages]).reshape(masks.shape)
+    assert (masks != own).mean() <= 2e-2
+    for nm, g, rf in zip(("dQ", "dK", "dV"), got, ref):
+        assert rel_err(to_np(g), rf) <= BWD_TOL[w.dtype], (T, with_psi, nm, rel_err(to_np(g), rf))
+    ctx.close()
