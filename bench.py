@@ -372,11 +372,28 @@ def time_backward(w: wl.Workload, iters: int = 2, weight_grads: bool = False) ->
             e1.synchronize()
             tp.append(e0.elapsed_time(e1))
         phi_ms = float(np.median(tp))
+    saved = None
+    if w.dtype == "bf16" and w.d in (64, 128) and not weight_grads:
+        # the training pattern: a forward that saves for the backward, then a backward that reuses it
+        binding.csat_set_i64(ctx.h, binding.CSAT_SAVE_FOR_BACKWARD, 1)
+        out = torch.empty_like(dev["Q"])
+        tf, tb = [], []
+        for _ in range(iters + 1):
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record()
+            binding.csat_forward(ctx.h, dev["Q"], dev["K"], dev["V"], out)
+            e1.record()
+            binding.csat_backward(ctx.h, dev["Q"], dev["K"], dev["V"], G, dQ, dK, dV)
+            e2.record()
+            e2.synchronize()
+            tf.append(e0.elapsed_time(e1))
+            tb.append(e1.elapsed_time(e2))
+        saved = {"forward_ms": float(np.median(tf[1:])), "backward_ms": float(np.median(tb[1:]))}
     ctx.close()
     if weight_grads:
         return {"ms": float(np.median(times)), "kernels": "as backward, plus the iterates and dx_t kept as bf16, a tcgen05 "
                 "contraction over them (dS, dB, dPsi) and a streaming sum (dtheta)"}
-    return {"ms": float(np.median(times)), "backward_phi_ms": phi_ms,
+    return {"ms": float(np.median(times)), "backward_phi_ms": phi_ms, "with_save_for_backward": saved,
             "kernels": "bf16: every stage on tcgen05 (forward with decisions recorded, recurrence backward, dQ, dK~|dV~, "
                        "Phi^T); float32: ffma kernels"}
 

@@ -82,6 +82,13 @@ enum {
   CSAT_DEBUG_CANARY = 11, /* debugging aid: 1 fills the K~|V~ workspace with NaN bit patterns (one extra memset on the
                           call's stream) before csat_forward / csat_backward compress, so that a row the compression
                           failed to write shows as NaN in the output instead of reusing an earlier call's values  */
+  CSAT_SAVE_FOR_BACKWARD = 13, /* 1: csat_forward (tensor-core path: bf16, d in {64, 128}) also keeps what csat_backward
+                          needs from it (K~|V~ stay in the workspace; Z, the rows' softmax statistics and one decision
+                          bit per layer, query and column go to the backward's scratch, which this then allocates),
+                          and the next csat_backward on the same Q, K, V skips its own compression and forward pass
+                          (about a third of its time).  The saved state is dropped by any setter and by any other
+                          compute call in between; it is the caller's contract that Q, K, V are unchanged.  The
+                          forward then costs about a third more.  0 (default): csat_backward recomputes  */
   CSAT_WEIGHT_GRADS = 12, /* 1: csat_backward also forms the gradients with respect to the decoder's parameters (S, B,
                           the thresholds, the dictionary) for csat_get_weight_grads; tensor-core path only (bf16, d in
                           {64, 128}, one S, B for all layers, CSAT_T >= 1), else csat_backward returns

@@ -21,6 +21,7 @@ CSAT_KEEP_MASKS = 9
 CSAT_HADAMARD_TRANSFORM = 10
 CSAT_DEBUG_CANARY = 11
 CSAT_WEIGHT_GRADS = 12
+CSAT_SAVE_FOR_BACKWARD = 13
 CSAT_ENSEMBLE_GAUSSIAN, CSAT_ENSEMBLE_RADEMACHER, CSAT_ENSEMBLE_HADAMARD = 0, 1, 2
 KERNEL_NAMES = {0: "decoder_setup", 1: "compress", 2: "attend_recover"}
 CSAT_DTYPE_BF16, CSAT_DTYPE_FP32 = 0, 1

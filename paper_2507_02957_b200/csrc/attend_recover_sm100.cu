@@ -1116,14 +1116,14 @@ cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, c
 // shrinkage decisions (one S, B for all layers; the decoded output itself is not stored)
 cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bfloat16* z_out, float* lse_out,
                                              int lse_stride, uint32_t* mask_out, __nv_bfloat16* alpha_out,
-                                             cudaStream_t s, int* launches) {
+                                             cudaStream_t s, int* launches, void* out) {
   *launches += 1;
   if (c->w_S && c->w_untied && c->p.T > 0)      // one S_t, B_t per layer (no iterates kept: alpha_out is for tied layers)
-    return c->p.d == 64 ? launch<64, true, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out)
-                        : launch<128, true, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out);
+    return c->p.d == 64 ? launch<64, true, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out)
+                        : launch<128, true, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out);
   return c->p.d == 64
-             ? launch<64, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
-             : launch<128, false, true>(c, Q, nullptr, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out);
+             ? launch<64, false, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
+             : launch<128, false, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out);
 }
 
 }  // namespace csat

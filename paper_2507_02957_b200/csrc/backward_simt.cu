@@ -413,10 +413,12 @@ cudaError_t run(csat_ctx* c, const void* Q, const void* G, void* dQ, void* dK, v
   // rows' log sum exp, then the recurrence (forward with its decisions recorded, and backward) and dQ
   if (tc_stages && c->bw_Z16 != nullptr && (p.T == 0 || c->bw_maskbits != nullptr)) {
     const bool wg = c->weight_grads && p.T > 0 && c->bw_alpha16 != nullptr;
-    if (wg && (e = cudaMemsetAsync(c->bw_alpha16, 0, (size_t)(p.B * p.H * p.nq * p.d) * 2, s)) != cudaSuccess) return e;   // alpha^0
-    if ((e = launch_sm100_attend_for_backward(c, Q, c->bw_Z16, c->bw_LD, 2, c->bw_maskbits, wg ? c->bw_alpha16 : nullptr, s,
-                                              launches)) != cudaSuccess)
-      return e;
+    if (!c->reuse_saved) {        // otherwise a csat_forward with CSAT_SAVE_FOR_BACKWARD has left all of it
+      if (wg && (e = cudaMemsetAsync(c->bw_alpha16, 0, (size_t)(p.B * p.H * p.nq * p.d) * 2, s)) != cudaSuccess) return e;   // alpha^0
+      if ((e = launch_sm100_attend_for_backward(c, Q, c->bw_Z16, c->bw_LD, 2, c->bw_maskbits, wg ? c->bw_alpha16 : nullptr,
+                                                s, launches)) != cudaSuccess)
+        return e;
+    }
     if (c->bw_masks != nullptr && p.T > 0) {           // CSAT_KEEP_MASKS: the decisions in the exported layout
       const int64_t total = p.B * p.H * p.nq * p.d;
       expand_masks_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(c->bw_masks, c->bw_maskbits, total, p.nq, d, p.T);

@@ -126,6 +126,7 @@ void free_backward(csat_ctx* c) {
   c->bw_bytes_alpha16 = c->bw_bytes_dx16 = c->bw_bytes_wpart = c->bw_bytes_thpart = c->bw_bytes_wgrad = 0;
   c->have_wgrads = false;
   c->have_dkv16 = false;
+  c->saved_valid = false;
   c->bw_bytes_Z16 = c->bw_bytes_maskbits = 0;
   c->bw_bytes_masks = 0;
   c->have_masks = false;
@@ -320,6 +321,7 @@ int csat_destroy(csat_ctx* c) {
 
 int csat_set_i64(csat_ctx* c, int key, int64_t v) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   csat::Params& p = c->p;
   switch (key) {
     case CSAT_BATCH: {
@@ -400,6 +402,10 @@ int csat_set_i64(csat_ctx* c, int key, int64_t v) {
       if ((v != 0) != c->keep_masks) { cudaDeviceSynchronize(); free_backward(c); }
       c->keep_masks = v != 0;
       return CSAT_OK;
+    case CSAT_SAVE_FOR_BACKWARD:
+      if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_SAVE_FOR_BACKWARD must be 0 or 1");
+      c->save_for_backward = v != 0;
+      return CSAT_OK;
     case CSAT_WEIGHT_GRADS:
       if (v != 0 && v != 1) return fail(c, CSAT_ERR_INVALID_ARG, "CSAT_WEIGHT_GRADS must be 0 or 1");
       if ((v != 0) != c->weight_grads) { cudaDeviceSynchronize(); free_backward(c); }
@@ -442,6 +448,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
     case CSAT_PROFILE: *out = c->prof_slots; return CSAT_OK;
     case CSAT_KEEP_MASKS: *out = c->keep_masks ? 1 : 0; return CSAT_OK;
     case CSAT_WEIGHT_GRADS: *out = c->weight_grads ? 1 : 0; return CSAT_OK;
+    case CSAT_SAVE_FOR_BACKWARD: *out = c->save_for_backward ? 1 : 0; return CSAT_OK;
     case CSAT_HADAMARD_TRANSFORM: *out = c->hadamard_transform; return CSAT_OK;
     case CSAT_DEBUG_CANARY: *out = c->debug_canary; return CSAT_OK;
     default: return CSAT_ERR_INVALID_ARG;
@@ -450,6 +457,7 @@ int csat_get_i64(const csat_ctx* c, int key, int64_t* out) {
 
 int csat_set_f64(csat_ctx* c, int key, double v) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   if (!(v == v)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_f64: NaN");
   switch (key) {
     case CSAT_LAMBDA:
@@ -478,6 +486,7 @@ int csat_get_f64(const csat_ctx* c, int key, double* out) {
 
 int csat_set_phi(csat_ctx* c, const void* phi, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   if (!phi || !aligned16(phi)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_phi: NULL or misaligned pointer");
   if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
   std::string why;
@@ -503,6 +512,7 @@ int csat_get_phi(const csat_ctx* c, void* phi_out, void* stream) {
 
 int csat_set_dictionary(csat_ctx* c, const void* psi, int per_head, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   csat::Params& p = c->p;
   const size_t es = csat::elt_size(p.dtype);
   if (psi && !aligned16(psi)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_dictionary: misaligned pointer");
@@ -524,6 +534,7 @@ int csat_set_dictionary(csat_ctx* c, const void* psi, int per_head, void* stream
 
 int csat_set_decoder_matrix(csat_ctx* c, const void* D, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   csat::Params& p = c->p;
   const size_t bytes = dd_bytes(p, csat::elt_size(p.dtype));
   if (D && !aligned16(D)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_set_decoder_matrix: misaligned pointer");
@@ -553,6 +564,7 @@ static int set_weights(csat_ctx* c, const void* S, const void* Bm, const float* 
   if (!aligned16(S) || !aligned16(Bm)) return fail(c, CSAT_ERR_INVALID_ARG, name + ": misaligned pointer");
   if (layers < 1 || layers > 100000) return fail(c, CSAT_ERR_INVALID_ARG, name + ": layers must be >= 1");
   if (c->w_S && (c->w_layers != layers || c->w_untied != untied)) { cudaDeviceSynchronize(); free_lista(c); }
+  c->saved_valid = false;
   const size_t elt = csat::elt_size(p.dtype);
   if (!c->w_S) {
     c->w_layers = layers;
@@ -604,6 +616,8 @@ static int ensure_decoder(csat_ctx* c, cudaStream_t s, int* launches) {
   return CSAT_OK;
 }
 
+static int ensure_backward_scratch(csat_ctx* c);
+
 int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void* out, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
   if (!Q || !K || !V || !out) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward: NULL tensor pointer");
@@ -645,8 +659,21 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
     e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
   if (e != cudaSuccess) return fail_cuda(c, e, "compress launch");
   prof_mark(c, s, CSAT_KERNEL_COMPRESS);
-  e = tc_attend ? csat::launch_sm100_attend_recover(c, Q, out, s, &launches)
-                : csat::launch_simt_attend_recover(c, Q, out, s, &launches);
+  c->saved_valid = false;
+  if (c->save_for_backward && tc_attend && c->p.B * c->p.H <= 32767) {
+    // the recording variant of the same kernel: the output, and Z, the rows' log sum exp, the layers' decisions (and
+    // the iterates with CSAT_WEIGHT_GRADS) where csat_backward will look for them
+    if (int rc = ensure_backward_scratch(c)) return rc;
+    const bool wg = c->weight_grads && c->p.T > 0 && !c->w_untied && c->bw_alpha16 != nullptr;
+    if (wg && (e = cudaMemsetAsync(c->bw_alpha16, 0, (size_t)(c->p.B * c->p.H * c->p.nq * c->p.d) * 2, s)) != cudaSuccess)
+      return fail_cuda(c, e, "memset");
+    e = csat::launch_sm100_attend_for_backward(c, Q, c->bw_Z16, c->bw_LD, 2, c->bw_maskbits, wg ? c->bw_alpha16 : nullptr, s,
+                                               &launches, out);
+    if (e == cudaSuccess) { c->saved_valid = true; c->saved_alpha = wg; }
+  } else {
+    e = tc_attend ? csat::launch_sm100_attend_recover(c, Q, out, s, &launches)
+                  : csat::launch_simt_attend_recover(c, Q, out, s, &launches);
+  }
   if (e != cudaSuccess) return fail_cuda(c, e, "attend/recover launch");
   prof_mark(c, s, CSAT_KERNEL_ATTEND_RECOVER);
   if (c->prof_slots) ++c->prof_calls;
@@ -659,6 +686,7 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
 int csat_compress_partial(csat_ctx* c, const void* K_shard, const void* V_shard, int64_t n0, int64_t n_len,
                           float* partial_out, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   if (!K_shard || !V_shard || !partial_out) return fail(c, CSAT_ERR_INVALID_ARG, "csat_compress_partial: NULL pointer");
   if (!aligned16(K_shard) || !aligned16(V_shard) || !aligned16(partial_out))
     return fail(c, CSAT_ERR_INVALID_ARG, "csat_compress_partial: pointers must be 16-byte aligned");
@@ -684,6 +712,7 @@ int csat_compress_partial(csat_ctx* c, const void* K_shard, const void* V_shard,
 
 int csat_reduce_partials(csat_ctx* c, const float* partials, int count, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   if (!partials || !aligned16(partials)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_reduce_partials: NULL or misaligned pointer");
   if (count < 1 || count > 4096) return fail(c, CSAT_ERR_INVALID_ARG, "csat_reduce_partials: count must be in [1, 4096]");
   if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
@@ -699,6 +728,7 @@ int csat_reduce_partials(csat_ctx* c, const float* partials, int count, void* st
 
 int csat_attend(csat_ctx* c, const void* Q, void* out, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   if (!Q || !out) return fail(c, CSAT_ERR_INVALID_ARG, "csat_attend: NULL tensor pointer");
   if (!aligned16(Q) || !aligned16(out)) return fail(c, CSAT_ERR_INVALID_ARG, "csat_attend: tensor pointers must be 16-byte aligned");
   if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
@@ -727,6 +757,43 @@ int csat_attend(csat_ctx* c, const void* Q, void* out, void* stream) {
                             : csat::launch_simt_attend_recover(c, Q, out, s, &launches);
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_attend launch");
   c->last_launches = launches;
+  return CSAT_OK;
+}
+
+// scratch of csat_backward (and of a csat_forward that saves for it), (re)allocated when a size has changed
+static int ensure_backward_scratch(csat_ctx* c) {
+  const csat::Params& p = c->p;
+  const size_t bz = (size_t)(p.B * p.H * p.nq * p.d) * 4, bl = (size_t)(p.B * p.H * p.nq * 2) * 4 + 1024 /* read past the end by whole-tile copies */,
+               bk = (size_t)(p.B * p.H * p.m * 2 * p.d) * 4,
+               bw = (size_t)(2 * (c->w_untied ? c->w_layers : 1) * p.H * p.d * p.d) * 4,
+               b16 = c->tmap_phi_valid ? bk / 2 : 0, z16 = c->tmap_phi_valid ? bz / 2 : 0,
+               bm = c->keep_masks && p.T > 0 ? bz : 0,
+               bmb = c->tmap_phi_valid ? (size_t)(p.B * p.H * p.T * p.nq * (p.d / 32)) * 4 : 0,
+               bal = c->weight_grads ? (size_t)((p.T + 1) * p.B * p.H * p.nq * p.d) * 2 : 0,
+               bdx = c->weight_grads ? (size_t)(p.T * p.B * p.H * p.nq * p.d) * 2 : 0,
+               bwp = c->weight_grads ? (size_t)(csat::wgrad_splits(c) * p.H * 2 * p.d * p.d) * 4 : 0,
+               bth = c->weight_grads ? (size_t)(64 * p.T * p.H) * 4 : 0,
+               bwg = c->weight_grads ? (size_t)((2 * p.H + 1) * p.d * p.d + p.T * p.H) * 4 : 0;
+  if (c->bw_bytes_alpha16 != bal || c->bw_bytes_dx16 != bdx || c->bw_bytes_wpart != bwp || c->bw_bytes_thpart != bth ||
+      c->bw_bytes_wgrad != bwg || c->bw_bytes_maskbits != bmb || c->bw_bytes_Z16 != z16 || c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
+      c->bw_bytes_dKV16 != b16 || c->bw_bytes_dZ16 != z16) {
+    cudaDeviceSynchronize();
+    free_backward(c);
+    c->bw_bytes_dZ = bz; c->bw_bytes_LD = bl; c->bw_bytes_dKV = bk; c->bw_bytes_WT = bw; c->bw_bytes_dKV16 = b16;
+    c->bw_bytes_dZ16 = z16;
+    c->bw_bytes_masks = bm;
+    c->bw_bytes_Z16 = z16;
+    c->bw_bytes_maskbits = bmb;
+    c->bw_bytes_alpha16 = bal; c->bw_bytes_dx16 = bdx; c->bw_bytes_wpart = bwp; c->bw_bytes_thpart = bth; c->bw_bytes_wgrad = bwg;
+    if (dev_alloc(c, &c->bw_alpha16, bal) != cudaSuccess || dev_alloc(c, &c->bw_dx16, bdx) != cudaSuccess ||
+        dev_alloc(c, &c->bw_wpart, bwp) != cudaSuccess || dev_alloc(c, &c->bw_thpart, bth) != cudaSuccess ||
+        dev_alloc(c, &c->bw_wgrad, bwg) != cudaSuccess || dev_alloc(c, &c->bw_maskbits, bmb) != cudaSuccess || dev_alloc(c, &c->bw_Z16, z16) != cudaSuccess || dev_alloc(c, &c->bw_masks, bm) != cudaSuccess || dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
+        dev_alloc(c, &c->bw_dKV, bk) != cudaSuccess || dev_alloc(c, &c->bw_WT, bw) != cudaSuccess ||
+        dev_alloc(c, &c->bw_dKV16, b16) != cudaSuccess || dev_alloc(c, &c->bw_dZ16, z16) != cudaSuccess) {
+      free_backward(c);
+      return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(backward scratch) failed");
+    }
+  }
   return CSAT_OK;
 }
 
@@ -763,43 +830,21 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
     int rc = ensure_decoder(c, s, &launches);
     if (rc != CSAT_OK) return rc;
   }
-  const size_t bz = (size_t)(p.B * p.H * p.nq * p.d) * 4, bl = (size_t)(p.B * p.H * p.nq * 2) * 4 + 1024 /* read past the end by whole-tile copies */,
-               bk = (size_t)(p.B * p.H * p.m * 2 * p.d) * 4,
-               bw = (size_t)(2 * (c->w_untied ? c->w_layers : 1) * p.H * p.d * p.d) * 4,
-               b16 = c->tmap_phi_valid ? bk / 2 : 0, z16 = c->tmap_phi_valid ? bz / 2 : 0,
-               bm = c->keep_masks && p.T > 0 ? bz : 0,
-               bmb = c->tmap_phi_valid ? (size_t)(p.B * p.H * p.T * p.nq * (p.d / 32)) * 4 : 0,
-               bal = c->weight_grads ? (size_t)((p.T + 1) * p.B * p.H * p.nq * p.d) * 2 : 0,
-               bdx = c->weight_grads ? (size_t)(p.T * p.B * p.H * p.nq * p.d) * 2 : 0,
-               bwp = c->weight_grads ? (size_t)(csat::wgrad_splits(c) * p.H * 2 * p.d * p.d) * 4 : 0,
-               bth = c->weight_grads ? (size_t)(64 * p.T * p.H) * 4 : 0,
-               bwg = c->weight_grads ? (size_t)((2 * p.H + 1) * p.d * p.d + p.T * p.H) * 4 : 0;
-  if (c->bw_bytes_alpha16 != bal || c->bw_bytes_dx16 != bdx || c->bw_bytes_wpart != bwp || c->bw_bytes_thpart != bth ||
-      c->bw_bytes_wgrad != bwg || c->bw_bytes_maskbits != bmb || c->bw_bytes_Z16 != z16 || c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
-      c->bw_bytes_dKV16 != b16 || c->bw_bytes_dZ16 != z16) {
-    cudaDeviceSynchronize();
-    free_backward(c);
-    c->bw_bytes_dZ = bz; c->bw_bytes_LD = bl; c->bw_bytes_dKV = bk; c->bw_bytes_WT = bw; c->bw_bytes_dKV16 = b16;
-    c->bw_bytes_dZ16 = z16;
-    c->bw_bytes_masks = bm;
-    c->bw_bytes_Z16 = z16;
-    c->bw_bytes_maskbits = bmb;
-    c->bw_bytes_alpha16 = bal; c->bw_bytes_dx16 = bdx; c->bw_bytes_wpart = bwp; c->bw_bytes_thpart = bth; c->bw_bytes_wgrad = bwg;
-    if (dev_alloc(c, &c->bw_alpha16, bal) != cudaSuccess || dev_alloc(c, &c->bw_dx16, bdx) != cudaSuccess ||
-        dev_alloc(c, &c->bw_wpart, bwp) != cudaSuccess || dev_alloc(c, &c->bw_thpart, bth) != cudaSuccess ||
-        dev_alloc(c, &c->bw_wgrad, bwg) != cudaSuccess || dev_alloc(c, &c->bw_maskbits, bmb) != cudaSuccess || dev_alloc(c, &c->bw_Z16, z16) != cudaSuccess || dev_alloc(c, &c->bw_masks, bm) != cudaSuccess || dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
-        dev_alloc(c, &c->bw_dKV, bk) != cudaSuccess || dev_alloc(c, &c->bw_WT, bw) != cudaSuccess ||
-        dev_alloc(c, &c->bw_dKV16, b16) != cudaSuccess || dev_alloc(c, &c->bw_dZ16, z16) != cudaSuccess) {
-      free_backward(c);
-      return fail(c, CSAT_ERR_ALLOC, "cudaMalloc(backward scratch) failed");
-    }
-  }
+  if (int rc = ensure_backward_scratch(c)) return rc;
   const bool tc_compress = c->tmap_phi_valid && c->force_simt != 1;
-  cudaError_t e = c->debug_canary ? cudaMemsetAsync(c->kv, 0xFF, kv_bytes(p), s) : cudaSuccess;
-  if (e != cudaSuccess) return fail_cuda(c, e, "canary fill");
-  e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
-  if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward: compress launch");
+  // what a csat_forward with CSAT_SAVE_FOR_BACKWARD left (K~|V~, Z, the softmax statistics, the decisions, the iterates
+  // if asked for) replaces the compression and the forward pass of this call
+  c->reuse_saved = c->save_for_backward && c->saved_valid && c->tmap_phi_valid && c->force_simt == 0 &&
+                   (!c->weight_grads || c->saved_alpha);
+  cudaError_t e = cudaSuccess;
+  if (!c->reuse_saved) {
+    e = c->debug_canary ? cudaMemsetAsync(c->kv, 0xFF, kv_bytes(p), s) : cudaSuccess;
+    if (e != cudaSuccess) return fail_cuda(c, e, "canary fill");
+    e = tc_compress ? csat::launch_sm100_compress(c, K, V, s, &launches) : csat::launch_simt_compress(c, K, V, s, &launches);
+    if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward: compress launch");
+  }
   e = csat::launch_backward(c, Q, dOut, dQ, dK, dV, s, &launches);
+  c->reuse_saved = false;
   if (e != cudaSuccess) return fail_cuda(c, e, "csat_backward launch");
   c->have_masks = c->bw_masks != nullptr;
   c->have_wgrads = c->weight_grads && c->bw_wgrad != nullptr;
@@ -823,6 +868,7 @@ static int ensure_pipeline(csat_ctx* c) {
 
 int csat_forward_host(csat_ctx* c, const void* Qh, const void* Kh, const void* Vh, void* outh, void* stream) {
   if (!c) return CSAT_ERR_INVALID_ARG;
+  c->saved_valid = false;
   if (!Qh || !Kh || !Vh || !outh) return fail(c, CSAT_ERR_INVALID_ARG, "csat_forward_host: NULL pointer");
   if (c->broken) return fail(c, CSAT_ERR_STATE, kBrokenMsg);
   NvtxRange range("csat_forward_host");

@@ -122,6 +122,10 @@ struct csat_ctx {
   bool weight_grads = false;
   bool have_wgrads = false;
   bool have_dkv16 = false;       // bw_dKV16 holds dK~|dV~ of the most recent csat_backward (tensor-core path)
+  // CSAT_SAVE_FOR_BACKWARD: csat_forward runs the recording variant of its kernel and leaves K~|V~, Z, the softmax
+  // statistics and the decisions for the next csat_backward (saved_valid until anything changes them)
+  bool save_for_backward = false, saved_valid = false, saved_alpha = false;
+  bool reuse_saved = false;      // set by csat_backward around launch_backward
   __nv_bfloat16* bw_alpha16 = nullptr; __nv_bfloat16* bw_dx16 = nullptr;
   float* bw_wpart = nullptr; float* bw_thpart = nullptr; float* bw_wgrad = nullptr;
   size_t bw_bytes_alpha16 = 0, bw_bytes_dx16 = 0, bw_bytes_wpart = 0, bw_bytes_thpart = 0, bw_bytes_wgrad = 0;
@@ -197,9 +201,10 @@ cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, c
 // the forward run for the backward pass: z_out [B,H,n_q,d] bf16 = Z, lse_out[row * lse_stride] = log sum exp of the
 // row's scores, mask_out [B,H,T,n_q,d/32] = the layers' decisions |x_t| > theta_t (column c: word c / 32, bit 31 - c % 32)
 // alpha_out (may be null): the iterates alpha^1 .. alpha^T as bf16 into slots 1 .. T of [T+1][B,H,n_q,d]
+// out (may be null): the decoded output as well (a forward that saves for the backward)
 cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bfloat16* z_out, float* lse_out,
                                              int lse_stride, uint32_t* mask_out, __nv_bfloat16* alpha_out,
-                                             cudaStream_t s, int* launches);
+                                             cudaStream_t s, int* launches, void* out = nullptr);
 
 // wgrad_sm100.cu : gradients of the decoder's parameters from the stored iterates and dx_t (bf16, d in {64, 128}, one
 // S, B for all layers) into bw_wgrad; wgrad_splits = CTAs per head of its contraction kernel

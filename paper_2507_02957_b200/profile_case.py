@@ -65,6 +65,7 @@ def main():
     bw.add_argument("--weight-grads", action="store_true", help="also form the gradients of the decoder's parameters")
     bw.add_argument("--phi-grad", action="store_true", help="also time csat_backward_phi (reported separately)")
     bw.add_argument("--untied", action="store_true", help="one random S_t, B_t per layer instead of the ISTA-derived pair")
+    bw.add_argument("--saved", action="store_true", help="time forward (saving for the backward) and backward separately")
     hd = sub.add_parser("hadamard")
     for name in ("n", "d", "B", "H"):
         hd.add_argument(name, type=int)
@@ -128,6 +129,22 @@ def main():
             e1.synchronize()
             times.append(e0.elapsed_time(e1))
         res = {"backward_ms": round(float(np.median(times)), 4), "weight_grads": bool(a.weight_grads), "untied": bool(a.untied)}
+        if a.saved:
+            binding.csat_set_i64(ctx.h, binding.CSAT_SAVE_FOR_BACKWARD, 1)
+            out = torch.empty_like(Q)
+            tf, tb = [], []
+            for _ in range(a.iters + 1):
+                e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+                e0.record()
+                ctx.forward(Q, K, V, out)
+                e1.record()
+                binding.csat_backward(ctx.h, Q, K, V, G, dQ, dK, dV)
+                e2.record()
+                e2.synchronize()
+                tf.append(e0.elapsed_time(e1))
+                tb.append(e1.elapsed_time(e2))
+            res["saving_forward_ms"] = round(float(np.median(tf[1:])), 4)
+            res["backward_after_saving_forward_ms"] = round(float(np.median(tb[1:])), 4)
         if a.phi_grad:
             dPhi = torch.empty(w.H, w.m, w.n, dtype=torch.float32, device="cuda")
             binding.csat_backward_phi(ctx.h, K, V, dPhi)

@@ -431,3 +431,43 @@ def test_backward_with_per_layer_weights_small_depths(T, with_psi):
     for nm, g, rf in zip(("dQ", "dK", "dV"), got, ref):
         assert rel_err(to_np(g), rf) <= BWD_TOL[w.dtype], (T, with_psi, nm, rel_err(to_np(g), rf))
     ctx.close()
+
+
+@pytest.mark.parametrize("name", ["bf16_d64", "bf16_d128"])
+@pytest.mark.parametrize("weights", ["ista", "per_layer"])
+def test_forward_that_saves_for_the_backward(name, weights):
+    """CSAT_SAVE_FOR_BACKWARD: the forward's output still matches the oracle, the backward that follows skips its own
+    compression and forward pass (two launches fewer) and returns the same bits as a backward that recomputes, a second
+    backward still does, and a setter in between makes the backward recompute again."""
+    w = CASES[name]()
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    kw = dict(T=w.T, lam=w.lam)
+    if weights == "per_layer":
+        r = np.random.default_rng(5)
+        d, H, T = w.d, w.H, w.T
+        S = wl.round_to_storage((0.6 * np.eye(d) + 0.4 * r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        Bm = wl.round_to_storage((r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        thetas = np.full((T, H), 0.02, dtype=np.float32)
+        ctx.set_lista_layer_weights(to_dev(S, w.dtype), to_dev(Bm, w.dtype), torch.from_numpy(thetas).cuda())
+        kw.update(weights=(S.astype(np.float64), Bm.astype(np.float64), list(thetas.astype(np.float64))))
+    G = to_dev(wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype), w.dtype)
+    ctx.forward(Q, K, V)                                          # (sets up the decoder's operands)
+    plain = ctx.backward(Q, K, V, G)
+    n_plain = binding.csat_last_launch_count(ctx.h)
+    binding.csat_set_i64(ctx.h, binding.CSAT_SAVE_FOR_BACKWARD, 1)
+    out = to_np(ctx.forward(Q, K, V))
+    ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], to_np(ctx.get_phi()), **kw)
+    assert rel_err(out, ref) <= TOL[w.dtype]
+    saved = ctx.backward(Q, K, V, G)
+    assert binding.csat_last_launch_count(ctx.h) == n_plain - 2
+    again = ctx.backward(Q, K, V, G)
+    for a, b, c_ in zip(plain, saved, again):
+        assert torch.equal(a, b) and torch.equal(a, c_)
+    ctx.set(lam=w.lam)                                            # any setter drops what was saved
+    recomputed = ctx.backward(Q, K, V, G)
+    assert binding.csat_last_launch_count(ctx.h) >= n_plain
+    for a, b in zip(plain, recomputed):
+        assert torch.equal(a, b)
+    ctx.close()
