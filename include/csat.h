@@ -197,7 +197,8 @@ int csat_set_lista_layer_weights(csat_ctx* ctx, const void* S, const void* Bm, c
  *   Q [B,H,n_q,d], K, V [B,H,n,d]   the forward's inputs          (context dtype, device)
  *   dOut [B,H,n_q,d]                gradient of the loss with respect to csat_forward's output
  *   dQ [B,H,n_q,d], dK, dV [B,H,n,d]  outputs (context dtype)
- * Nothing of an earlier csat_forward is reused: the call compresses K, V again and recomputes what it needs.  Its
+ * Unless the last csat_forward ran with CSAT_SAVE_FOR_BACKWARD, nothing of an earlier csat_forward is reused: the
+ * call compresses K, V again and recomputes what it needs.  Its
  * first call allocates scratch (B H (n_q (d + 2) + 2 m d) floats and transposed copies of the decoder matrices;
  * bf16 copies of Z, dZ and dK~|dV~ and B H T n_q d / 32 decision words on the tensor-core path; B H n_q d words
  * more with CSAT_KEEP_MASKS; all counted by csat_workspace_bytes).
