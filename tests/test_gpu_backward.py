@@ -470,4 +470,17 @@ def test_forward_that_saves_for_the_backward(name, weights):
     assert binding.csat_last_launch_count(ctx.h) >= n_plain
     for a, b in zip(plain, recomputed):
         assert torch.equal(a, b)
+    if weights == "ista":
+        # the decoder's gradients too: the saving forward then also keeps the iterates
+        binding.csat_set_i64(ctx.h, binding.CSAT_WEIGHT_GRADS, 1)
+        binding.csat_set_i64(ctx.h, binding.CSAT_SAVE_FOR_BACKWARD, 0)
+        ctx.backward(Q, K, V, G)
+        wg_plain = [x.clone() for x in ctx.weight_grads()]
+        n_wg = binding.csat_last_launch_count(ctx.h)
+        binding.csat_set_i64(ctx.h, binding.CSAT_SAVE_FOR_BACKWARD, 1)
+        ctx.forward(Q, K, V)
+        ctx.backward(Q, K, V, G)
+        assert binding.csat_last_launch_count(ctx.h) == n_wg - 2          # no compression, no forward pass
+        for a, b in zip(wg_plain, ctx.weight_grads()):
+            assert torch.equal(a, b)
     ctx.close()
