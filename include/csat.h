@@ -91,7 +91,7 @@ enum {
                           forward then costs about a third more.  0 (default): csat_backward recomputes  */
   CSAT_WEIGHT_GRADS = 12, /* 1: csat_backward also forms the gradients with respect to the decoder's parameters (S, B,
                           the thresholds, the dictionary) for csat_get_weight_grads; tensor-core path only (bf16, d in
-                          {64, 128}, one S, B for all layers, CSAT_T >= 1), else csat_backward returns
+                          {64, 128}, CSAT_T >= 1), else csat_backward returns
                           CSAT_ERR_UNSUPPORTED.  It then keeps every layer's iterate and its gradient as bf16:
                           (2 T + 1) B H n_q d more 16-bit values of scratch.  0 (default): not formed  */
   CSAT_KEEP_MASKS = 9, /* 1: csat_backward also keeps its shrinkage decisions (one 32-bit word per (b, h, query,
@@ -228,6 +228,7 @@ int csat_get_backward_masks(const csat_ctx* ctx, uint32_t* masks_out, void* stre
  * computes in (csat_set_lista_weights takes S, B in the same form):
  *   dS     [H, d, d] float32  = sum over layers, queries, batch of (alpha^t)^T dx_t
  *   dB     [H, d, d] float32  = ... of Z^T dx_t
+ *          (with one S_t, B_t per layer, csat_set_lista_layer_weights: dS, dB [T, H, d, d], layer by layer, no sum)
  *   dtheta [T, H]    float32  = per layer: - sum of sign(x_t) o dx_t   (one threshold for all layers: add the rows)
  *   dPsi   [d, d]    float32  = sum over heads too of G^T alpha^T (C^ = alpha^T Psi^T); zeros without a dictionary;
  *                               may be NULL

@@ -378,6 +378,7 @@ class Csat:
     def set_lista_weights(self, S, Bm=None, theta=None):
         """Supplied LISTA weights: S, Bm [H,d,d] (context dtype), theta [layers,H] or [H] float32; S=None restores
         the ISTA-derived decoder."""
+        self._per_layer_weights = False
         if S is None:
             csat_set_lista_weights(self.h, None, None, None, 1)
             return
@@ -432,10 +433,11 @@ class Csat:
 
     def weight_grads(self):
         """Gradients with respect to the decoder's parameters from the most recent backward (CSAT_WEIGHT_GRADS = 1):
-        dS [H,d,d], dB [H,d,d], dtheta [T,H], dPsi [d,d] (float32)."""
+        dS [H,d,d], dB [H,d,d] ([T,H,d,d] after set_lista_layer_weights), dtheta [T,H], dPsi [d,d] (float32)."""
         T = csat_get_i64(self.h, CSAT_T)
-        dS = self._new(self.H, self.d, self.d, dtype=torch.float32)
-        dB = self._new(self.H, self.d, self.d, dtype=torch.float32)
+        lead = (T, self.H) if getattr(self, "_per_layer_weights", False) else (self.H,)
+        dS = self._new(*lead, self.d, self.d, dtype=torch.float32)
+        dB = self._new(*lead, self.d, self.d, dtype=torch.float32)
         dth = self._new(T, self.H, dtype=torch.float32)
         dPsi = self._new(self.d, self.d, dtype=torch.float32)
         csat_get_weight_grads(self.h, dS, dB, dth, dPsi)
@@ -461,6 +463,7 @@ class Csat:
         theta = theta.to(torch.float32).contiguous()
         assert theta.shape == (L, self.H)
         csat_set_lista_layer_weights(self.h, S.contiguous(), Bm.contiguous(), theta, L)
+        self._per_layer_weights = True
 
     def get_compressed(self):
         kt = self._new(self.B, self.H, self.m, self.d)

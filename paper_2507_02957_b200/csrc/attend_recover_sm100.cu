@@ -730,6 +730,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
               pk[e >> 1] = pack_bf16(a0, a1);
             }
             tmem_st_32x32b_x8(a_addr + c0 / 2, pk);
+            if (kMasks && arow != nullptr) st_global_v8(arow + (int64_t)(it + 1) * alpha_slot + c0, pk);   // alpha^{t+1}
           };
           uint32_t r0[16], r1[16];
           tmem_ld_32x32b_x16(acc_addr, r0);
@@ -768,6 +769,19 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
         store_masks(T - 1);
+        if (kMasks && arow != nullptr) {
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) {
+            uint32_t pa[8];
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) {
+              float a0, a1;
+              unpack2(v2[(c0 + e) >> 1], a0, a1);
+              pa[e >> 1] = pack_bf16(a0, a1);
+            }
+            st_global_v8(arow + (int64_t)T * alpha_slot + c0, pa);
+          }
+        }
         if (has_psi) {
           publish(D / 2);
           w.wait(&bars->r_full[t], phase & 1, 232); ++phase;
@@ -1118,9 +1132,9 @@ cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bf
                                              int lse_stride, uint32_t* mask_out, __nv_bfloat16* alpha_out,
                                              cudaStream_t s, int* launches, void* out) {
   *launches += 1;
-  if (c->w_S && c->w_untied && c->p.T > 0)      // one S_t, B_t per layer (no iterates kept: alpha_out is for tied layers)
-    return c->p.d == 64 ? launch<64, true, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out)
-                        : launch<128, true, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out);
+  if (c->w_S && c->w_untied && c->p.T > 0)      // one S_t, B_t per layer
+    return c->p.d == 64 ? launch<64, true, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
+                        : launch<128, true, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out);
   return c->p.d == 64
              ? launch<64, false, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
              : launch<128, false, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out);

@@ -664,7 +664,7 @@ int csat_forward(csat_ctx* c, const void* Q, const void* K, const void* V, void*
     // the recording variant of the same kernel: the output, and Z, the rows' log sum exp, the layers' decisions (and
     // the iterates with CSAT_WEIGHT_GRADS) where csat_backward will look for them
     if (int rc = ensure_backward_scratch(c)) return rc;
-    const bool wg = c->weight_grads && c->p.T > 0 && !c->w_untied && c->bw_alpha16 != nullptr;
+    const bool wg = c->weight_grads && c->p.T > 0 && c->bw_alpha16 != nullptr;
     if (wg && (e = cudaMemsetAsync(c->bw_alpha16, 0, (size_t)(c->p.B * c->p.H * c->p.nq * c->p.d) * 2, s)) != cudaSuccess)
       return fail_cuda(c, e, "memset");
     e = csat::launch_sm100_attend_for_backward(c, Q, c->bw_Z16, c->bw_LD, 2, c->bw_maskbits, wg ? c->bw_alpha16 : nullptr, s,
@@ -771,9 +771,10 @@ static int ensure_backward_scratch(csat_ctx* c) {
                bmb = c->tmap_phi_valid ? (size_t)(p.B * p.H * p.T * p.nq * (p.d / 32)) * 4 : 0,
                bal = c->weight_grads ? (size_t)((p.T + 1) * p.B * p.H * p.nq * p.d) * 2 : 0,
                bdx = c->weight_grads ? (size_t)(p.T * p.B * p.H * p.nq * p.d) * 2 : 0,
-               bwp = c->weight_grads ? (size_t)(csat::wgrad_splits(c) * p.H * 2 * p.d * p.d) * 4 : 0,
+               wz = (size_t)(c->w_untied && p.T > 0 ? p.T : 1),      // one dS, dB per layer with per-layer weights
+               bwp = c->weight_grads ? (size_t)(csat::wgrad_splits(c) * p.H * 2 * p.d * p.d) * wz * 4 : 0,
                bth = c->weight_grads ? (size_t)(64 * p.T * p.H) * 4 : 0,
-               bwg = c->weight_grads ? (size_t)((2 * p.H + 1) * p.d * p.d + p.T * p.H) * 4 : 0;
+               bwg = c->weight_grads ? ((size_t)(2 * p.H * p.d * p.d) * wz + (size_t)(p.d * p.d + p.T * p.H)) * 4 : 0;
   if (c->bw_bytes_alpha16 != bal || c->bw_bytes_dx16 != bdx || c->bw_bytes_wpart != bwp || c->bw_bytes_thpart != bth ||
       c->bw_bytes_wgrad != bwg || c->bw_bytes_maskbits != bmb || c->bw_bytes_Z16 != z16 || c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
       c->bw_bytes_dKV16 != b16 || c->bw_bytes_dZ16 != z16) {
@@ -817,10 +818,10 @@ int csat_backward(csat_ctx* c, const void* Q, const void* K, const void* V, cons
                 "csat_backward: the float32 kernels and CSAT_KEEP_MASKS keep one decision bit per layer in a 32-bit "
                 "word: CSAT_T <= 32");
   if (p.d > 256) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: d <= 256");
-  if (c->weight_grads && !(c->tmap_phi_valid && c->force_simt == 0 && !c->w_untied && p.T > 0))
+  if (c->weight_grads && !(c->tmap_phi_valid && c->force_simt == 0 && p.T > 0))
     return fail(c, CSAT_ERR_UNSUPPORTED,
                 "CSAT_WEIGHT_GRADS: the gradients of the decoder's parameters are formed on the tensor-core path only "
-                "(bf16, d in {64, 128}, one S, B for all layers, CSAT_T > 0)");
+                "(bf16, d in {64, 128}, CSAT_T > 0)");
   if (p.B * p.H > 32767) return fail(c, CSAT_ERR_UNSUPPORTED, "csat_backward: B * H <= 32767");
   if (p.T > 0 && c->w_S && (c->w_layers != 1 || c->w_untied) && c->w_layers != p.T)
     return fail(c, CSAT_ERR_STATE, "the supplied LISTA weights are for a number of layers other than CSAT_T");
@@ -1056,7 +1057,7 @@ int csat_get_weight_grads(const csat_ctx* c, float* dS, float* dB, float* dtheta
   if (!c->have_wgrads)
     return fail(mc, CSAT_ERR_STATE, "csat_get_weight_grads: no csat_backward with CSAT_WEIGHT_GRADS = 1 has run");
   const csat::Params& p = c->p;
-  const size_t dd = (size_t)(p.d * p.d), hdd = (size_t)p.H * dd;
+  const size_t dd = (size_t)(p.d * p.d), hdd = (size_t)p.H * dd * (size_t)(c->w_untied && p.T > 0 ? p.T : 1);
   cudaStream_t s = (cudaStream_t)stream;
   cudaError_t e = cudaMemcpyAsync(dS, c->bw_wgrad, hdd * 4, cudaMemcpyDeviceToDevice, s);
   if (e == cudaSuccess) e = cudaMemcpyAsync(dB, c->bw_wgrad + hdd, hdd * 4, cudaMemcpyDeviceToDevice, s);

@@ -91,7 +91,7 @@ wgrad_gram_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
         const int s = i % C::kStages;
         if (i >= C::kStages) ok = mbar_wait(&bars->empty[s], ((i / C::kStages) & 1) ^ 1, status, 701, &bars->abort);
         if (!ok) break;
-        const int u = u0 + i / nt, t = i % nt, b = u / ntiles, tile = u % ntiles;
+        const int u = u0 + i / nt, t = (int)blockIdx.z + i % nt, b = u / ntiles, tile = u % ntiles;
         const int bh = b * H + h;
         uint8_t* st = smem + (uint32_t)s * C::kStageBytes;
         mbar_arrive_expect_tx(&bars->full[s], C::kStageBytes);
@@ -139,7 +139,7 @@ wgrad_gram_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     // epilogue: lane = row of C (d = 128: row i of A1^T B and of A2^T B; d = 64: rows 0-63 A1^T B, 64-127 A2^T B)
     const int row = warp * 32 + lane;
     const uint32_t tbase = tmem + ((uint32_t)(warp * 32) << 16);
-    float* p1 = part + ((int64_t)(split * H + h) * 2) * D * D;       // [2][D][D]
+    float* p1 = part + ((int64_t)((blockIdx.z * gridDim.x + split) * H + h) * 2) * D * D;       // [2][D][D]
     const bool have = steps > 0;
     bool ok = true;
     if (have) ok = mbar_wait(&bars->acc_done, 0, status, 703, &bars->abort) && *(volatile int*)&bars->abort == 0;
@@ -173,11 +173,11 @@ wgrad_gram_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
   if (warp == 5) tmem_dealloc(tmem, C::kTmemCols);
 }
 
-// out[h][i] = sum over the splits, in order, of part[split][h][which][i]   (i over d*d); all heads into out[i] with
-// `over_heads` (the dictionary is shared by the heads)
-__global__ void wgrad_reduce_kernel(float* __restrict__ out, const float* __restrict__ part, int splits, int H, int which,
-                                    int64_t dd, int over_heads) {
-  const int64_t total = (over_heads ? 1 : H) * dd;
+// out[z][h][i] = sum over the splits, in order, of part[z][split][h][which][i]   (i over d*d; z = layer with one pair of
+// matrices per layer, else 0); all heads into out[i] with `over_heads` (the dictionary is shared by the heads)
+__global__ void wgrad_reduce_kernel(float* __restrict__ out, const float* __restrict__ part, int splits, int H, int Z,
+                                    int which, int64_t dd, int over_heads) {
+  const int64_t total = (over_heads ? 1 : (int64_t)Z * H) * dd;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
     const int64_t e = i % dd;
     float acc = 0.f;
@@ -185,8 +185,8 @@ __global__ void wgrad_reduce_kernel(float* __restrict__ out, const float* __rest
       for (int h = 0; h < H; ++h)
         for (int s = 0; s < splits; ++s) acc += part[(((int64_t)s * H + h) * 2 + which) * dd + e];
     } else {
-      const int64_t h = i / dd;
-      for (int s = 0; s < splits; ++s) acc += part[(((int64_t)s * H + h) * 2 + which) * dd + e];
+      const int64_t zh = i / dd, z = zh / H, h = zh % H;
+      for (int s = 0; s < splits; ++s) acc += part[((((int64_t)z * splits + s) * H + h) * 2 + which) * dd + e];
     }
     out[i] = acc;
   }
@@ -244,13 +244,13 @@ cudaError_t slab_map(CUtensorMap* m, const void* base, const Params& p, int64_t 
 
 template <int D>
 cudaError_t launch_gram(csat_ctx* c, const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b, SlabIndex ia1,
-                        SlabIndex ia2, SlabIndex ib, int nt, int splits, int units_per_cta, cudaStream_t s) {
+                        SlabIndex ia2, SlabIndex ib, int nt, int splits, int units_per_cta, cudaStream_t s, int layers_z = 1) {
   using C = GCfg<D>;
   static DeviceFlags smem_opt_in;
   cudaError_t e = ensure_dynamic_smem(wgrad_gram_kernel<D>, (int)C::kSmemBytes, c->device, smem_opt_in);
   if (e != cudaSuccess) return e;
   const Params& p = c->p;
-  wgrad_gram_kernel<D><<<dim3((unsigned)splits, (unsigned)p.H), kThreads, C::kSmemBytes, s>>>(
+  wgrad_gram_kernel<D><<<dim3((unsigned)splits, (unsigned)p.H, (unsigned)layers_z), kThreads, C::kSmemBytes, s>>>(
       a1, a2, b, ia1, ia2, ib, c->bw_wpart, (int)p.nq, (int)p.H, (int)p.B, nt, units_per_cta, c->status);
   return cudaGetLastError();
 }
@@ -260,7 +260,8 @@ cudaError_t launch_gram(csat_ctx* c, const CUtensorMap& a1, const CUtensorMap& a
 int wgrad_splits(const csat_ctx* c) {
   const Params& p = c->p;
   const int64_t units = p.B * ((p.nq + kRows - 1) / kRows);
-  int64_t s = c->sms / p.H;                     // one wave: at most sms CTAs in all
+  // one wave: at most sms CTAs in all; with one pair of matrices per layer every (head, layer) has its own CTAs
+  int64_t s = c->sms / (p.H * (c->w_untied && p.T > 0 ? p.T : 1));
   if (s > units) s = units;
   return (int)(s < 1 ? 1 : s);
 }
@@ -279,18 +280,21 @@ cudaError_t launch_sm100_wgrad(csat_ctx* c, const void* G, cudaStream_t s, int* 
   if ((e = slab_map(&tx, c->bw_dx16, p, p.T * BH)) != cudaSuccess) return e;
   if ((e = slab_map(&tz, c->bw_Z16, p, BH)) != cudaSuccess) return e;
   if ((e = slab_map(&tg, G, p, BH)) != cudaSuccess) return e;
+  // dS [Z,H,d,d] | dB [Z,H,d,d] | dPsi [d,d] | dtheta [T,H]; Z = T with one S_t, B_t per layer, else 1
+  const int Z = (c->w_untied && p.T > 0) ? p.T : 1;
   float* dS = c->bw_wgrad;
-  float* dB = dS + p.H * dd;
-  float* dPsi = dB + p.H * dd;
+  float* dB = dS + (int64_t)Z * p.H * dd;
+  float* dPsi = dB + (int64_t)Z * p.H * dd;
   float* dTh = dPsi + dd;
-  const unsigned rblocks = (unsigned)((p.H * dd + 255) / 256);
-  // dS = sum_t (alpha^t)^T dx_t, dB = sum_t Z^T dx_t
+  const unsigned rblocks = (unsigned)(((int64_t)Z * p.H * dd + 255) / 256);
+  // dS = sum_t (alpha^t)^T dx_t, dB = sum_t Z^T dx_t (per layer: no sum over t, the layer is the grid's z index)
   const SlabIndex ia{0, (int)BH}, iz{0, 0}, ix{0, (int)BH};
-  e = p.d == 64 ? launch_gram<64>(c, ta, tz, tx, ia, iz, ix, p.T, splits, upc, s)
-                : launch_gram<128>(c, ta, tz, tx, ia, iz, ix, p.T, splits, upc, s);
+  const int nt = Z > 1 ? 1 : p.T;
+  e = p.d == 64 ? launch_gram<64>(c, ta, tz, tx, ia, iz, ix, nt, splits, upc, s, Z)
+                : launch_gram<128>(c, ta, tz, tx, ia, iz, ix, nt, splits, upc, s, Z);
   if (e != cudaSuccess) return e;
-  wgrad_reduce_kernel<<<rblocks, 256, 0, s>>>(dS, c->bw_wpart, splits, (int)p.H, 0, dd, 0);
-  wgrad_reduce_kernel<<<rblocks, 256, 0, s>>>(dB, c->bw_wpart, splits, (int)p.H, 1, dd, 0);
+  wgrad_reduce_kernel<<<rblocks, 256, 0, s>>>(dS, c->bw_wpart, splits, (int)p.H, Z, 0, dd, 0);
+  wgrad_reduce_kernel<<<rblocks, 256, 0, s>>>(dB, c->bw_wpart, splits, (int)p.H, Z, 1, dd, 0);
   *launches += 3;
   if (c->psi) {
     // dPsi = G^T alpha^T: A1 = A2 = G, B = slot T of the iterates, one "layer"
@@ -298,7 +302,7 @@ cudaError_t launch_sm100_wgrad(csat_ctx* c, const void* G, cudaStream_t s, int* 
     e = p.d == 64 ? launch_gram<64>(c, tg, tg, ta, ig, ig, iaT, 1, splits, upc, s)
                   : launch_gram<128>(c, tg, tg, ta, ig, ig, iaT, 1, splits, upc, s);
     if (e != cudaSuccess) return e;
-    wgrad_reduce_kernel<<<(unsigned)((dd + 255) / 256), 256, 0, s>>>(dPsi, c->bw_wpart, splits, (int)p.H, 0, dd, 1);
+    wgrad_reduce_kernel<<<(unsigned)((dd + 255) / 256), 256, 0, s>>>(dPsi, c->bw_wpart, splits, (int)p.H, 1, 0, dd, 1);
     *launches += 2;
   } else {
     if ((e = cudaMemsetAsync(dPsi, 0, (size_t)dd * 4, s)) != cudaSuccess) return e;

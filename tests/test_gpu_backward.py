@@ -484,3 +484,58 @@ def test_forward_that_saves_for_the_backward(name, weights):
         for a, b in zip(wg_plain, ctx.weight_grads()):
             assert torch.equal(a, b)
     ctx.close()
+
+
+@pytest.mark.parametrize("name", ["bf16_d64", "bf16_d128"])
+@pytest.mark.parametrize("with_psi", [False, True], ids=["identity", "dictionary"])
+def test_per_layer_weight_gradients_match_oracle(name, with_psi):
+    """CSAT_WEIGHT_GRADS with one S_t, B_t per layer: dS, dB [T,H,d,d] layer by layer (no sum over the layers), dtheta
+    [T,H], dPsi, against the oracle's per-layer gradients summed over the batch, with the library's decisions."""
+    w = WGRAD_CASES[name]()
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    binding.csat_set_i64(ctx.h, binding.CSAT_KEEP_MASKS, 1)
+    binding.csat_set_i64(ctx.h, binding.CSAT_WEIGHT_GRADS, 1)
+    d, H, T, B = w.d, w.H, w.T, w.B
+    r = np.random.default_rng(23)
+    kw = dict(T=T, lam=w.lam)
+    if with_psi:
+        Psi = wl.round_to_storage((np.eye(d) + 0.3 * r.standard_normal((d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+        ctx.set_dictionary(to_dev(Psi, w.dtype))
+        kw.update(Psi=Psi.astype(np.float64))
+    S = wl.round_to_storage((0.6 * np.eye(d) + 0.4 * r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+    Bm = wl.round_to_storage((r.standard_normal((T, H, d, d)) / np.sqrt(d)).astype(np.float32), w.dtype)
+    phi = to_np(ctx.get_phi())
+    st0 = []
+    orc.csat_forward(inp["Q"][:1], inp["K"][:1], inp["V"][:1], phi, T=0, lam=0.0, stages=st0)
+    th0 = float(np.median(np.abs(st0[0]["Z"] @ Bm[0, 0].astype(np.float64))))
+    thetas = (th0 * r.uniform(0.2, 1.5, size=(T, H))).astype(np.float32)
+    ctx.set_lista_layer_weights(to_dev(S, w.dtype), to_dev(Bm, w.dtype), torch.from_numpy(thetas).cuda())
+    kw.update(weights=(S.astype(np.float64), Bm.astype(np.float64), list(thetas.astype(np.float64))))
+    G = wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype)
+    ctx.backward(Q, K, V, to_dev(G, w.dtype))
+    words = ctx.backward_masks().cpu().numpy().astype(np.uint32)
+    masks = np.stack([(words >> t) & 1 for t in range(T)], axis=2).astype(bool)
+    stages = []
+    orc.csat_backward(inp["Q"], inp["K"], inp["V"], phi, G, masks=masks, stages=stages, **kw)
+    dS = np.zeros((T, H, d, d)); dB = np.zeros((T, H, d, d)); dth = np.zeros((T, H)); dPsi = np.zeros((d, d))
+    for b in range(B):
+        for h in range(H):
+            st = stages[b * H + h]
+            dS[:, h] += st["dS"]
+            dB[:, h] += st["dB"]
+            dth[:, h] += st["dtheta"]
+            if with_psi:
+                dPsi += st["dPsi"]
+    gS, gB, gth, gPsi = (x.cpu().numpy().astype(np.float64) for x in ctx.weight_grads())
+    assert gS.shape == (T, H, d, d) and gB.shape == (T, H, d, d)
+    assert np.abs(gS[0]).max() == 0.0                          # alpha^0 = 0
+    tol = BWD_TOL[w.dtype]
+    for nm, g, rf in (("dS", gS, dS), ("dB", gB, dB), ("dtheta", gth, dth)) + ((("dPsi", gPsi, dPsi),) if with_psi else ()):
+        assert np.isfinite(g).all() and np.abs(rf).max() > 0
+        assert rel_err(g, rf) <= tol, (name, with_psi, nm, rel_err(g, rf))
+    # every layer on its own scale too
+    for t in range(1, T):
+        assert rel_err(gS[t], dS[t]) <= 2 * tol and rel_err(gB[t], dB[t]) <= 2 * tol, t
+    ctx.close()
