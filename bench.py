@@ -411,7 +411,19 @@ def run_csat(args, w: wl.Workload) -> dict:
     torch.cuda.set_device(local)
     under_torchrun = "RANK" in os.environ and "MASTER_ADDR" in os.environ
     if world > 1 or under_torchrun:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        # NCCL prints its version banner on stdout (NCCL_DEBUG=VERSION) when the communicator is created, i.e. at the
+        # first collective; stdout carries the one JSON line, so file descriptor 1 points at stderr until then
+        sys.stdout.flush()
+        saved_fd = os.dup(1)
+        os.dup2(2, 1)
+        try:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+            dist.barrier()
+            torch.cuda.synchronize()
+        finally:
+            sys.stdout.flush()
+            os.dup2(saved_fd, 1)
+            os.close(saved_fd)
 
     def barrier():
         if dist.is_initialized():
