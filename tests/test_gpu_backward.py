@@ -539,3 +539,21 @@ def test_per_layer_weight_gradients_match_oracle(name, with_psi):
     for t in range(1, T):
         assert rel_err(gS[t], dS[t]) <= 2 * tol and rel_err(gB[t], dB[t]) <= 2 * tol, t
     ctx.close()
+
+
+def test_saving_forward_without_recovery_layers():
+    """CSAT_SAVE_FOR_BACKWARD at T = 0 (the output is Z itself: nothing but Z and the softmax statistics to keep)."""
+    w = wl.shrink(C["c2"], B=2, H=2, n_q=150, T=0)
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    G = to_dev(wl.round_to_storage(np.random.default_rng(G_SEED).standard_normal(inp["Q"].shape).astype(np.float32), w.dtype), w.dtype)
+    plain = ctx.backward(Q, K, V, G)
+    binding.csat_set_i64(ctx.h, binding.CSAT_SAVE_FOR_BACKWARD, 1)
+    out = ctx.forward(Q, K, V)
+    ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], to_np(ctx.get_phi()), T=0, lam=w.lam)
+    assert rel_err(to_np(out), ref) <= TOL[w.dtype]
+    saved = ctx.backward(Q, K, V, G)
+    for a, b in zip(plain, saved):
+        assert torch.equal(a, b)
+    ctx.close()
