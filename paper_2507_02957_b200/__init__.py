@@ -3,4 +3,4 @@
 `workloads` (seeded synthetic inputs) imports nothing heavy; `binding` loads libcsat.so and
 needs torch + a CUDA device for anything beyond loading.
 """
-__all__ = ["workloads", "binding", "build"]
+__all__ = ["workloads", "binding", "build", "autograd"]
