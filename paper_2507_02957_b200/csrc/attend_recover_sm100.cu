@@ -183,7 +183,8 @@ struct Waiter {
 // Z (bf16, as fed to the first product), every row's log sum exp, and the decision |x_t| > theta_t of every layer,
 // one bit per column: word c / 32 of (layer, row), bit 31 - c % 32.  With alpha_out (the gradients of the decoder's
 // weights need them) also the iterates alpha^1 .. alpha^T as bf16: alpha^t of (b, h, row) at slot t of alpha_slot
-// elements each (slot 0, alpha^0 = 0, is the caller's to clear).
+// elements each (slot 0, alpha^0 = 0, is the caller's to clear), and with sign_out the sign bit of every x_t in the
+// layout of the decisions (the gradient of the thresholds is - sum sign(x_t) o dx_t).
 template <int D, bool kUntied, bool kMasks>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
@@ -192,7 +193,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                             int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status,
                             float* __restrict__ lse_out, int lse_stride, __nv_bfloat16* __restrict__ z_out,
                             uint32_t* __restrict__ mask_out, __nv_bfloat16* __restrict__ alpha_out,
-                            int64_t alpha_slot) {
+                            int64_t alpha_slot, uint32_t* __restrict__ sign_out) {
   using C = Cfg<D>;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
@@ -663,7 +664,14 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       __nv_bfloat16* arow = (kMasks && alpha_out != nullptr && grow_m < nq)
                                 ? alpha_out + ((int64_t)bh * nq + grow_m) * D : nullptr;
       uint32_t mw[D / 32];                                      // kMasks: the current layer's decisions
+      uint32_t sw[D / 32];                                      // kMasks with sign_out: the current layer's sign bits
+      const bool signs = kMasks && sign_out != nullptr;
       auto store_masks = [&](int layer) {
+        if (signs && grow_m < nq) {
+          uint32_t* so = sign_out + (((int64_t)bh * T + layer) * nq + grow_m) * (D / 32);
+          if (D == 128) *reinterpret_cast<uint4*>(so) = make_uint4(sw[0], sw[1], sw[2], sw[D / 32 - 1]);
+          else *reinterpret_cast<uint2*>(so) = make_uint2(sw[0], sw[1]);
+        }
         if (kMasks && mask_out != nullptr && grow_m < nq) {
           uint32_t* mo = mask_out + (((int64_t)bh * T + layer) * nq + grow_m) * (D / 32);
           if (D == 128) *reinterpret_cast<uint4*>(mo) = make_uint4(mw[0], mw[1], mw[2], mw[D / 32 - 1]);
@@ -721,6 +729,10 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                 unpack2(mul2(y2, fma2(y2, pack2(-1.f, -1.f), p2th2)), g0, g1);
                 mw[c0 >> 5] = __funnelshift_l(__float_as_uint(g0), mw[c0 >> 5], 1);
                 mw[c0 >> 5] = __funnelshift_l(__float_as_uint(g1), mw[c0 >> 5], 1);
+                if (signs) {                         // where the decision holds y and x = y - theta have the same sign
+                  sw[c0 >> 5] = __funnelshift_l(__float_as_uint(y0), sw[c0 >> 5], 1);
+                  sw[c0 >> 5] = __funnelshift_l(__float_as_uint(y1), sw[c0 >> 5], 1);
+                }
               }
               const F2 t2 = pack2(fma_sat(y0, inv2th, 0.f), fma_sat(y1, inv2th, 0.f));
               const F2 an = fma2(t2, m2th2, y2);                               // alpha^{t+1} = eta_theta(x)
@@ -764,6 +776,10 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             if (kMasks) {
               mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x0)), mw[c0 >> 5], 1);
               mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x1)), mw[c0 >> 5], 1);
+              if (signs) {
+                sw[c0 >> 5] = __funnelshift_l(__float_as_uint(x0), sw[c0 >> 5], 1);
+                sw[c0 >> 5] = __funnelshift_l(__float_as_uint(x1), sw[c0 >> 5], 1);
+              }
             }
             v2[(c0 + e) >> 1] = pack2(x0 - fminf(fmaxf(x0, -th), th), x1 - fminf(fmaxf(x1, -th), th));
           }
@@ -919,6 +935,10 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                 if (kMasks) {                                                  // the sign bit of theta - |x| is the decision
                   mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x0)), mw[c0 >> 5], 1);
                   mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x1)), mw[c0 >> 5], 1);
+                  if (signs) {
+                    sw[c0 >> 5] = __funnelshift_l(__float_as_uint(x0), sw[c0 >> 5], 1);
+                    sw[c0 >> 5] = __funnelshift_l(__float_as_uint(x1), sw[c0 >> 5], 1);
+                  }
                 }
                 const F2 t2 = pack2(fma_sat(x0, inv2th, 0.5f), fma_sat(x1, inv2th, 0.5f));
                 F2 bn = fma2(t2, m2th2, x2);                             // eta_theta(x) - theta
@@ -976,6 +996,10 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
             if (kMasks) {
               mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x0)), mw[c0 >> 5], 1);
               mw[c0 >> 5] = __funnelshift_l(__float_as_uint(th - fabsf(x1)), mw[c0 >> 5], 1);
+              if (signs) {
+                sw[c0 >> 5] = __funnelshift_l(__float_as_uint(x0), sw[c0 >> 5], 1);
+                sw[c0 >> 5] = __funnelshift_l(__float_as_uint(x1), sw[c0 >> 5], 1);
+              }
             }
             v2[(c0 + e) >> 1] = pack2(x0 - fminf(fmaxf(x0, -th), th), x1 - fminf(fmaxf(x1, -th), th));
           }
@@ -1090,7 +1114,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
                             kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
                             (int)p.nq, (int)p.m, (int)p.H, T, c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items,
                             (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out, alpha_out,
-                            (int64_t)(p.B * p.H * p.nq * p.d));
+                            (int64_t)(p.B * p.H * p.nq * p.d), alpha_out != nullptr ? c->bw_signbits : nullptr);
 }
 
 }  // namespace

@@ -123,6 +123,8 @@ void free_backward(csat_ctx* c) {
   dev_free(c, &c->bw_wpart, c->bw_bytes_wpart);
   dev_free(c, &c->bw_thpart, c->bw_bytes_thpart);
   dev_free(c, &c->bw_wgrad, c->bw_bytes_wgrad);
+  dev_free(c, &c->bw_signbits, c->bw_bytes_signbits);
+  c->bw_bytes_signbits = 0;
   c->bw_bytes_alpha16 = c->bw_bytes_dx16 = c->bw_bytes_wpart = c->bw_bytes_thpart = c->bw_bytes_wgrad = 0;
   c->have_wgrads = false;
   c->have_dkv16 = false;
@@ -773,9 +775,10 @@ static int ensure_backward_scratch(csat_ctx* c) {
                bdx = c->weight_grads ? (size_t)(p.T * p.B * p.H * p.nq * p.d) * 2 : 0,
                wz = (size_t)(c->w_untied && p.T > 0 ? p.T : 1),      // one dS, dB per layer with per-layer weights
                bwp = c->weight_grads ? (size_t)(csat::wgrad_splits(c) * p.H * 2 * p.d * p.d) * wz * 4 : 0,
-               bth = c->weight_grads ? (size_t)(64 * p.T * p.H) * 4 : 0,
+               bsg = c->weight_grads ? bmb : 0,
+               bth = c->weight_grads ? (size_t)((csat::wgrad_splits(c) > 64 ? csat::wgrad_splits(c) : 64) * p.T * p.H) * 4 : 0,
                bwg = c->weight_grads ? ((size_t)(2 * p.H * p.d * p.d) * wz + (size_t)(p.d * p.d + p.T * p.H)) * 4 : 0;
-  if (c->bw_bytes_alpha16 != bal || c->bw_bytes_dx16 != bdx || c->bw_bytes_wpart != bwp || c->bw_bytes_thpart != bth ||
+  if (c->bw_bytes_signbits != bsg || c->bw_bytes_alpha16 != bal || c->bw_bytes_dx16 != bdx || c->bw_bytes_wpart != bwp || c->bw_bytes_thpart != bth ||
       c->bw_bytes_wgrad != bwg || c->bw_bytes_maskbits != bmb || c->bw_bytes_Z16 != z16 || c->bw_bytes_masks != bm || c->bw_bytes_dZ != bz || c->bw_bytes_LD != bl || c->bw_bytes_dKV != bk || c->bw_bytes_WT != bw ||
       c->bw_bytes_dKV16 != b16 || c->bw_bytes_dZ16 != z16) {
     cudaDeviceSynchronize();
@@ -786,7 +789,8 @@ static int ensure_backward_scratch(csat_ctx* c) {
     c->bw_bytes_Z16 = z16;
     c->bw_bytes_maskbits = bmb;
     c->bw_bytes_alpha16 = bal; c->bw_bytes_dx16 = bdx; c->bw_bytes_wpart = bwp; c->bw_bytes_thpart = bth; c->bw_bytes_wgrad = bwg;
-    if (dev_alloc(c, &c->bw_alpha16, bal) != cudaSuccess || dev_alloc(c, &c->bw_dx16, bdx) != cudaSuccess ||
+    c->bw_bytes_signbits = bsg;
+    if (dev_alloc(c, &c->bw_signbits, bsg) != cudaSuccess || dev_alloc(c, &c->bw_alpha16, bal) != cudaSuccess || dev_alloc(c, &c->bw_dx16, bdx) != cudaSuccess ||
         dev_alloc(c, &c->bw_wpart, bwp) != cudaSuccess || dev_alloc(c, &c->bw_thpart, bth) != cudaSuccess ||
         dev_alloc(c, &c->bw_wgrad, bwg) != cudaSuccess || dev_alloc(c, &c->bw_maskbits, bmb) != cudaSuccess || dev_alloc(c, &c->bw_Z16, z16) != cudaSuccess || dev_alloc(c, &c->bw_masks, bm) != cudaSuccess || dev_alloc(c, &c->bw_dZ, bz) != cudaSuccess || dev_alloc(c, &c->bw_LD, bl) != cudaSuccess ||
         dev_alloc(c, &c->bw_dKV, bk) != cudaSuccess || dev_alloc(c, &c->bw_WT, bw) != cudaSuccess ||

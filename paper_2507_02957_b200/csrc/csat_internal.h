@@ -128,7 +128,9 @@ struct csat_ctx {
   bool reuse_saved = false;      // set by csat_backward around launch_backward
   __nv_bfloat16* bw_alpha16 = nullptr; __nv_bfloat16* bw_dx16 = nullptr;
   float* bw_wpart = nullptr; float* bw_thpart = nullptr; float* bw_wgrad = nullptr;
+  uint32_t* bw_signbits = nullptr;       // sign bit of every x_t, in the layout of bw_maskbits (for dtheta)
   size_t bw_bytes_alpha16 = 0, bw_bytes_dx16 = 0, bw_bytes_wpart = 0, bw_bytes_thpart = 0, bw_bytes_wgrad = 0;
+  size_t bw_bytes_signbits = 0;
   // staging for csat_forward_host
   void* stage_q = nullptr; void* stage_k = nullptr; void* stage_v = nullptr; void* stage_o = nullptr;
   size_t stage_bytes_q = 0, stage_bytes_kv = 0;

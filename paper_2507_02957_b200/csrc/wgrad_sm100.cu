@@ -15,7 +15,11 @@
 //   accumulators [128 x 128] in tensor memory; d = 64: A1 | A2 side by side form one M = 128 operand and one
 //   accumulator [128 x 64] holds A1^T B over A2^T B.  The CTA's sums go to a partial buffer; a second kernel adds the
 //   partials in a fixed order (no atomics: the result is the same bits on every run).
-// dtheta_kernel / reduce kernels: plain loads and adds.
+//   dtheta rides along: while a stage's tiles are in shared memory the four epilogue warps (one thread per row of
+//   the tile) read their row of dx_t from it and the row's sign bits of x_t (recorded by the forward kernel, one bit
+//   per column like the decisions), and add sign(x_t) o dx_t into per-layer sums; a stage is released by the MMA
+//   commit and by these four warps.  The sums go to a partial buffer like the matrices.
+// dtheta_partial_kernel (the same sum from the stored iterates' signs) serves depths beyond kMaxFusedLayers.
 #include "csat_internal.h"
 #include "sm100_ptx.cuh"
 #include "tma_host.h"
@@ -27,6 +31,7 @@ using namespace ptx;
 
 constexpr int kRows = 128;
 constexpr int kThreads = 192;          // warps 0-3: epilogue (TMEM lane = row of C), warp 4: TMA, warp 5: MMA
+constexpr int kMaxFusedLayers = 256;   // per-layer sums of sign(x_t) o dx_t kept in shared memory: [layers][4 warps]
 
 template <int D> struct GCfg {
   static constexpr int kDBoxes = D / 64;
@@ -35,7 +40,8 @@ template <int D> struct GCfg {
   static constexpr uint32_t kTileBytes = kDBoxes * kBoxBytes;
   static constexpr uint32_t kStageBytes = 3 * kTileBytes;            // A1 | A2 | B
   static constexpr uint32_t kOffBar = kStages * kStageBytes;
-  static constexpr uint32_t kSmemBytes = kOffBar + 256 + 1024;
+  static constexpr uint32_t kOffTheta = kOffBar + 256;               // float [kMaxFusedLayers][4]
+  static constexpr uint32_t kSmemBytes = kOffTheta + kMaxFusedLayers * 16 + 1024;
   static constexpr uint32_t kTmemCols = (D == 64) ? 64 : 256;
   static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
 };
@@ -53,7 +59,8 @@ template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 wgrad_gram_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_constant__ CUtensorMap tmap_a2,
                   const __grid_constant__ CUtensorMap tmap_b, SlabIndex ia1, SlabIndex ia2, SlabIndex ib,
-                  float* __restrict__ part, int nq, int H, int B, int nt, int units_per_cta, int* status) {
+                  float* __restrict__ part, int nq, int H, int B, int nt, int units_per_cta, int* status,
+                  const uint32_t* __restrict__ signbits, float* __restrict__ thpart, int T) {
   using C = GCfg<D>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -69,7 +76,8 @@ wgrad_gram_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     prefetch_tmap(&tmap_a1);
     prefetch_tmap(&tmap_a2);
     prefetch_tmap(&tmap_b);
-    for (int s = 0; s < C::kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+    // a stage is released by the MMA commit and, where dtheta rides along, by the four epilogue warps
+    for (int s = 0; s < C::kStages; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], signbits ? 5 : 1); }
     mbar_init(&bars->acc_done, 1);
     bars->abort = 0;
     fence_mbar_init();
@@ -142,6 +150,54 @@ wgrad_gram_kernel(const __grid_constant__ CUtensorMap tmap_a1, const __grid_cons
     float* p1 = part + ((int64_t)((blockIdx.z * gridDim.x + split) * H + h) * 2) * D * D;       // [2][D][D]
     const bool have = steps > 0;
     bool ok = true;
+    if (signbits != nullptr) {
+      // ---- dtheta: sum over this thread's row of sign(x_t) o dx_t, per layer ----
+      float* th_s = reinterpret_cast<float*>(smem + C::kOffTheta);           // [nt][4]
+      for (int i = threadIdx.x; i < nt * 4; i += 128) th_s[i] = 0.f;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      for (int i = 0; i < steps; ++i) {
+        const int s = i % C::kStages;
+        const int u = u0 + i / nt, tl = i % nt, t = (int)blockIdx.z + tl, b = u / ntiles, tile = u % ntiles;
+        const int grow = tile * kRows + row;
+        // the row's sign words (column c: word c / 32, bit 31 - c % 32), requested before the stage is waited for
+        uint32_t sg[D / 32];
+        const uint32_t* sp = signbits + ((((int64_t)(b * H + h)) * T + t) * nq + (grow < nq ? grow : 0)) * (D / 32);
+#pragma unroll
+        for (int q = 0; q < D / 32; ++q) sg[q] = grow < nq ? sp[q] : 0u;
+        if (ok) ok = mbar_wait(&bars->full[s], (i / C::kStages) & 1, status, 704, &bars->abort);
+        float acc = 0.f;
+        if (ok) {
+          const uint8_t* xt = smem + (uint32_t)s * C::kStageBytes + 2 * C::kTileBytes;   // the dx_t tile
+#pragma unroll
+          for (int gx = 0; gx < C::kDBoxes; ++gx) {
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {            // 16-byte pieces of the row's 128 bytes, swizzled by the row
+              const uint4 v = *reinterpret_cast<const uint4*>(xt + gx * C::kBoxBytes + row * 128 + ((ch ^ (row & 7)) << 4));
+              const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+              const int c0 = gx * 64 + ch * 8;          // first column of the piece
+              const uint32_t bits = sg[c0 >> 5] << (c0 & 31);            // the piece's 8 sign bits at the top
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                const uint32_t lo = (w4[q] << 16) ^ ((bits << (2 * q)) & 0x80000000u);
+                const uint32_t hi = (w4[q] & 0xffff0000u) ^ ((bits << (2 * q + 1)) & 0x80000000u);
+                acc += __uint_as_float(lo) + __uint_as_float(hi);
+              }
+            }
+          }
+        }
+        // fixed-order sum over the warp's rows, then into the layer's slot of this warp
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) {
+          th_s[tl * 4 + warp] += acc;
+          mbar_arrive(&bars->empty[s]);               // this warp has read the stage
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      for (int tl = threadIdx.x; tl < nt; tl += 128)
+        thpart[((int64_t)split * H + h) * T + (int)blockIdx.z + tl] =
+            th_s[tl * 4] + th_s[tl * 4 + 1] + th_s[tl * 4 + 2] + th_s[tl * 4 + 3];
+    }
     if (have) ok = mbar_wait(&bars->acc_done, 0, status, 703, &bars->abort) && *(volatile int*)&bars->abort == 0;
     ok = __all_sync(0xffffffffu, ok);
     if (have && ok) tc_fence_after();
@@ -227,11 +283,20 @@ dtheta_partial_kernel(float* __restrict__ partial, const __nv_bfloat16* __restri
   if (threadIdx.x == 0) partial[((int64_t)chunk * T + t) * H + h] = -sh[0];
 }
 
-__global__ void dtheta_reduce_kernel(float* __restrict__ out, const float* __restrict__ partial, int chunks, int n) {
+// out[t][h] = sum over the chunks, in order.  from_contraction: partial [chunk][H][T] holds + sum sign(x) o dx (the
+// gradient is its negative); else partial [chunk][T][H] already holds the negative
+__global__ void dtheta_reduce_kernel(float* __restrict__ out, const float* __restrict__ partial, int chunks, int T, int H,
+                                     int from_contraction) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
+  if (i >= T * H) return;
+  const int t = i / H, h = i % H;
   float acc = 0.f;
-  for (int c = 0; c < chunks; ++c) acc += partial[(int64_t)c * n + i];
+  if (from_contraction) {
+    for (int c = 0; c < chunks; ++c) acc += partial[((int64_t)c * H + h) * T + t];
+    acc = -acc;
+  } else {
+    for (int c = 0; c < chunks; ++c) acc += partial[(int64_t)c * T * H + i];
+  }
   out[i] = acc;
 }
 
@@ -244,14 +309,16 @@ cudaError_t slab_map(CUtensorMap* m, const void* base, const Params& p, int64_t 
 
 template <int D>
 cudaError_t launch_gram(csat_ctx* c, const CUtensorMap& a1, const CUtensorMap& a2, const CUtensorMap& b, SlabIndex ia1,
-                        SlabIndex ia2, SlabIndex ib, int nt, int splits, int units_per_cta, cudaStream_t s, int layers_z = 1) {
+                        SlabIndex ia2, SlabIndex ib, int nt, int splits, int units_per_cta, cudaStream_t s, int layers_z = 1,
+                        const uint32_t* signbits = nullptr) {
   using C = GCfg<D>;
   static DeviceFlags smem_opt_in;
   cudaError_t e = ensure_dynamic_smem(wgrad_gram_kernel<D>, (int)C::kSmemBytes, c->device, smem_opt_in);
   if (e != cudaSuccess) return e;
   const Params& p = c->p;
   wgrad_gram_kernel<D><<<dim3((unsigned)splits, (unsigned)p.H, (unsigned)layers_z), kThreads, C::kSmemBytes, s>>>(
-      a1, a2, b, ia1, ia2, ib, c->bw_wpart, (int)p.nq, (int)p.H, (int)p.B, nt, units_per_cta, c->status);
+      a1, a2, b, ia1, ia2, ib, c->bw_wpart, (int)p.nq, (int)p.H, (int)p.B, nt, units_per_cta, c->status, signbits,
+      c->bw_thpart, p.T);
   return cudaGetLastError();
 }
 
@@ -290,8 +357,11 @@ cudaError_t launch_sm100_wgrad(csat_ctx* c, const void* G, cudaStream_t s, int* 
   // dS = sum_t (alpha^t)^T dx_t, dB = sum_t Z^T dx_t (per layer: no sum over t, the layer is the grid's z index)
   const SlabIndex ia{0, (int)BH}, iz{0, 0}, ix{0, (int)BH};
   const int nt = Z > 1 ? 1 : p.T;
-  e = p.d == 64 ? launch_gram<64>(c, ta, tz, tx, ia, iz, ix, nt, splits, upc, s, Z)
-                : launch_gram<128>(c, ta, tz, tx, ia, iz, ix, nt, splits, upc, s, Z);
+  // dtheta rides along where the per-layer sums fit the kernel's shared memory
+  const bool fused_theta = c->bw_signbits != nullptr && nt <= kMaxFusedLayers;
+  const uint32_t* sgn = fused_theta ? c->bw_signbits : nullptr;
+  e = p.d == 64 ? launch_gram<64>(c, ta, tz, tx, ia, iz, ix, nt, splits, upc, s, Z, sgn)
+                : launch_gram<128>(c, ta, tz, tx, ia, iz, ix, nt, splits, upc, s, Z, sgn);
   if (e != cudaSuccess) return e;
   wgrad_reduce_kernel<<<rblocks, 256, 0, s>>>(dS, c->bw_wpart, splits, (int)p.H, Z, 0, dd, 0);
   wgrad_reduce_kernel<<<rblocks, 256, 0, s>>>(dB, c->bw_wpart, splits, (int)p.H, Z, 1, dd, 0);
@@ -307,12 +377,17 @@ cudaError_t launch_sm100_wgrad(csat_ctx* c, const void* G, cudaStream_t s, int* 
   } else {
     if ((e = cudaMemsetAsync(dPsi, 0, (size_t)dd * 4, s)) != cudaSuccess) return e;
   }
-  // dtheta
-  const int chunks = 64;
-  dtheta_partial_kernel<<<dim3(chunks, (unsigned)p.H, (unsigned)p.T), kThThreads, 0, s>>>(
-      c->bw_thpart, c->bw_alpha16, c->bw_dx16, BH * p.nq * p.d, p.nq * p.d, (int)p.B, (int)p.H, p.T);
-  dtheta_reduce_kernel<<<(unsigned)((p.T * p.H + 255) / 256), 256, 0, s>>>(dTh, c->bw_thpart, chunks, (int)(p.T * p.H));
-  *launches += 2;
+  // dtheta [T,H]: the contraction kernel's partial sums [split][H][T], or the streaming kernel's [chunk][T][H]
+  if (fused_theta) {
+    dtheta_reduce_kernel<<<(unsigned)((p.T * p.H + 255) / 256), 256, 0, s>>>(dTh, c->bw_thpart, splits, (int)p.T, (int)p.H, 1);
+    *launches += 1;
+  } else {
+    const int chunks = 64;
+    dtheta_partial_kernel<<<dim3(chunks, (unsigned)p.H, (unsigned)p.T), kThThreads, 0, s>>>(
+        c->bw_thpart, c->bw_alpha16, c->bw_dx16, BH * p.nq * p.d, p.nq * p.d, (int)p.B, (int)p.H, p.T);
+    dtheta_reduce_kernel<<<(unsigned)((p.T * p.H + 255) / 256), 256, 0, s>>>(dTh, c->bw_thpart, chunks, (int)p.T, (int)p.H, 0);
+    *launches += 2;
+  }
   return cudaGetLastError();
 }
 
