@@ -185,7 +185,9 @@ struct Waiter {
 // weights need them) also the iterates alpha^1 .. alpha^T as bf16: alpha^t of (b, h, row) at slot t of alpha_slot
 // elements each (slot 0, alpha^0 = 0, is the caller's to clear), and with sign_out the sign bit of every x_t in the
 // layout of the decisions (the gradient of the thresholds is - sum sign(x_t) o dx_t).
-template <int D, bool kUntied, bool kMasks>
+// kRec: 0 = the plain forward; 1 = also Z, log sum exp and the decisions (kMasks); 2 = also the iterates and the sign
+// bits of x_t (kKeep: only then are alpha_out / sign_out looked at, so that mode 1 carries none of their registers)
+template <int D, bool kUntied, int kRec>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
@@ -195,6 +197,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                             uint32_t* __restrict__ mask_out, __nv_bfloat16* __restrict__ alpha_out,
                             int64_t alpha_slot, uint32_t* __restrict__ sign_out) {
   using C = Cfg<D>;
+  constexpr bool kMasks = kRec >= 1, kKeep = kRec >= 2;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
     if (threadIdx.x == 0) atomicCAS(status, 0, 200);
@@ -661,11 +664,11 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         }
       }
       // kMasks: this row's place in slot 0 of the iterates (rows of 2 D bytes from a 256-byte aligned base: 32-byte stores)
-      __nv_bfloat16* arow = (kMasks && alpha_out != nullptr && grow_m < nq)
+      __nv_bfloat16* arow = (kKeep && alpha_out != nullptr && grow_m < nq)
                                 ? alpha_out + ((int64_t)bh * nq + grow_m) * D : nullptr;
       uint32_t mw[D / 32];                                      // kMasks: the current layer's decisions
       uint32_t sw[D / 32];                                      // kMasks with sign_out: the current layer's sign bits
-      const bool signs = kMasks && sign_out != nullptr;
+      const bool signs = kKeep && sign_out != nullptr;
       auto store_masks = [&](int layer) {
         if (signs && grow_m < nq) {
           uint32_t* so = sign_out + (((int64_t)bh * T + layer) * nq + grow_m) * (D / 32);
@@ -742,7 +745,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
               pk[e >> 1] = pack_bf16(a0, a1);
             }
             tmem_st_32x32b_x8(a_addr + c0 / 2, pk);
-            if (kMasks && arow != nullptr) st_global_v8(arow + (int64_t)(it + 1) * alpha_slot + c0, pk);   // alpha^{t+1}
+            if (kKeep && arow != nullptr) st_global_v8(arow + (int64_t)(it + 1) * alpha_slot + c0, pk);   // alpha^{t+1}
           };
           uint32_t r0[16], r1[16];
           tmem_ld_32x32b_x16(acc_addr, r0);
@@ -785,7 +788,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
         store_masks(T - 1);
-        if (kMasks && arow != nullptr) {
+        if (kKeep && arow != nullptr) {
 #pragma unroll
           for (int c0 = 0; c0 < D; c0 += 16) {
             uint32_t pa[8];
@@ -950,7 +953,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
                 pk[e >> 1] = pack_bf16(d0, d1);
               }
               tmem_st_32x32b_x8(op_addr + c0 / 2, pk);
-              if (kMasks && arow != nullptr) {                                 // alpha^{t+1} = b + kappa
+              if (kKeep && arow != nullptr) {                                 // alpha^{t+1} = b + kappa
                 uint32_t pa[8];
 #pragma unroll
                 for (int e = 0; e < 16; e += 2) {
@@ -1005,7 +1008,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
         store_masks(T - 1);
-        if (kMasks && arow != nullptr) {
+        if (kKeep && arow != nullptr) {
 #pragma unroll
           for (int c0 = 0; c0 < D; c0 += 16) {
             uint32_t pa[8];
@@ -1067,7 +1070,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   if (warp == kMmaWarp) tmem_dealloc(tmem, C::kTmemCols);
 }
 
-template <int D, bool kUntied, bool kMasks = false>
+template <int D, bool kUntied, int kRec = 0>
 cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T, float* lse_out, int lse_stride,
                    __nv_bfloat16* z_out = nullptr, uint32_t* mask_out = nullptr, __nv_bfloat16* alpha_out = nullptr) {
   using C = Cfg<D>;
@@ -1083,11 +1086,11 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
     // setmaxnreg moves registers inside the pool the CTA is launched with (threads x the compiled register count); the
     // kernel asks for 2 x 128 x 224 + 128 x 56 of them, and a request the pool cannot satisfy would wait forever
     cudaFuncAttributes fa;
-    if ((e = cudaFuncGetAttributes(&fa, attend_recover_sm100_kernel<D, kUntied, kMasks>)) != cudaSuccess) return e;
+    if ((e = cudaFuncGetAttributes(&fa, attend_recover_sm100_kernel<D, kUntied, kRec>)) != cudaSuccess) return e;
     if ((int64_t)fa.numRegs * kThreads < (int64_t)kTiles * kTileThreads * kComputeRegs + 128 * kControlRegs)
       return cudaErrorLaunchOutOfResources;
   }
-  if ((e = ensure_dynamic_smem(attend_recover_sm100_kernel<D, kUntied, kMasks>, (int)C::kSmemBytes, c->device, smem_opt_in)) !=
+  if ((e = ensure_dynamic_smem(attend_recover_sm100_kernel<D, kUntied, kRec>, (int)C::kSmemBytes, c->device, smem_opt_in)) !=
       cudaSuccess)
     return e;
   const double scale = p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)D);
@@ -1110,7 +1113,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kMasks>, tq, c->tmap_kv,
+  return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kRec>, tq, c->tmap_kv,
                             kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
                             (int)p.nq, (int)p.m, (int)p.H, T, c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items,
                             (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out, alpha_out,
@@ -1156,12 +1159,17 @@ cudaError_t launch_sm100_attend_for_backward(csat_ctx* c, const void* Q, __nv_bf
                                              int lse_stride, uint32_t* mask_out, __nv_bfloat16* alpha_out,
                                              cudaStream_t s, int* launches, void* out) {
   *launches += 1;
-  if (c->w_S && c->w_untied && c->p.T > 0)      // one S_t, B_t per layer
-    return c->p.d == 64 ? launch<64, true, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
-                        : launch<128, true, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out);
-  return c->p.d == 64
-             ? launch<64, false, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
-             : launch<128, false, true>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out);
+  const bool untied = c->w_S && c->w_untied && c->p.T > 0;      // one S_t, B_t per layer
+  const bool d64 = c->p.d == 64;
+#define CSAT_REC_LAUNCH(DD, UU, RR) \
+  launch<DD, UU, RR>(c, Q, out, s, c->p.T, lse_out, lse_stride, z_out, mask_out, alpha_out)
+  if (alpha_out != nullptr) {                   // with the iterates and the sign bits
+    if (untied) return d64 ? CSAT_REC_LAUNCH(64, true, 2) : CSAT_REC_LAUNCH(128, true, 2);
+    return d64 ? CSAT_REC_LAUNCH(64, false, 2) : CSAT_REC_LAUNCH(128, false, 2);
+  }
+  if (untied) return d64 ? CSAT_REC_LAUNCH(64, true, 1) : CSAT_REC_LAUNCH(128, true, 1);
+  return d64 ? CSAT_REC_LAUNCH(64, false, 1) : CSAT_REC_LAUNCH(128, false, 1);
+#undef CSAT_REC_LAUNCH
 }
 
 }  // namespace csat
