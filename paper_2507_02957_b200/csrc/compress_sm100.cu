@@ -35,22 +35,25 @@ constexpr uint32_t kBoxBytes = 64 * kChunk * 2;       // 8 KB: 64 columns x 64 t
 // operand and the accumulator: [K of element 0 .. K of element BG-1 | V of element 0 .. V of element BG-1].  With
 // d = 64 one element gives an N = 128 MMA, which needs 32 KB of operands per 256 cycles of tensor work: right at
 // what an SM can load; two elements (N = 256) halve the operand bytes per flop and the L2 reads of Phi.
-template <int D, bool SEP, int BG> struct Cfg {
-  static constexpr int kN = 2 * D * BG;               // accumulator columns
+// MT: measurement tiles per CTA (1 or 2; 2 only without SEP).  Two tiles of the same (batch, head) share every K, V
+// chunk: a second A tile per stage and a second accumulator, so the B operand is loaded once for twice the products.
+template <int D, bool SEP, int BG, int MT = 1> struct Cfg {
+  static constexpr int kN = 2 * D * BG;               // accumulator columns (per measurement tile)
   static constexpr int kBoxes = kN / 64;              // B boxes per stage
-  static constexpr int kATiles = SEP ? 2 : 1;
-  static constexpr int kStages = (D == 64 && BG == 1) ? (SEP ? 4 : 6) : (SEP ? 3 : 4);
+  static constexpr int kATiles = SEP ? 2 : MT;
+  static constexpr int kStages = (D == 64 && BG == 1) ? ((SEP || MT == 2) ? 4 : 6) : ((SEP || MT == 2) ? 3 : 4);
   static_assert(kN <= 256, "one MMA covers the accumulator");
+  static_assert(!(SEP && MT == 2) && MT * kN <= 512, "tensor memory");
   static constexpr uint32_t kStageBytes = kATiles * kABytes + kBoxes * kBoxBytes;
   static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <int D, bool SEP, int BG>
+template <int D, bool SEP, int BG, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_k,
                       const __grid_constant__ CUtensorMap tmap_v, __nv_bfloat16* __restrict__ kv, int m, int n, int H,
                       int B, int bh0, int* status, int phi_j0, float* __restrict__ partial) {
-  using C = Cfg<D, SEP, BG>;
+  using C = Cfg<D, SEP, BG, MT>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* a_buf = smem;                                      // [stages][A tiles][16 KB]
@@ -67,7 +70,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
   // (with BG > 1 blockIdx.y counts groups of BG batch elements; a group that runs past the batch repeats its
   // last element and does not store it)
   const int groups = (B + BG - 1) / BG;
-  const int mtile = blockIdx.x, h = blockIdx.y / groups, b0 = (blockIdx.y % groups) * BG;
+  const int mtile = blockIdx.x * MT, h = blockIdx.y / groups, b0 = (blockIdx.y % groups) * BG;   // first of MT tiles
   // bh0: first (batch, head) pair of a sub-range launch (then B = 1 and blockIdx.y counts its heads); 0 otherwise
   const int hl = h;
   auto bh_of = [&](int e) { return bh0 + (b0 + e < B ? b0 + e : B - 1) * H + hl; };
@@ -87,7 +90,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
     fence_mbar_init();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, C::kN);
+    tmem_alloc(tmem_slot, MT * C::kN);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -109,6 +112,8 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
         mbar_arrive_expect_tx(&full[s], C::kStageBytes);
         tma_load_3d(a_buf + s * C::kATiles * kABytes, &tmap_phi, &full[s], phi_j0 + i * kChunk, mtile * kTileM, hphi);
         if (SEP) tma_load_3d(a_buf + (s * C::kATiles + 1) * kABytes, &tmap_phi, &full[s], phi_j0 + i * kChunk, mtile * kTileM, H + hphi);
+        if (MT == 2)   // the next measurement tile of the same head (rows beyond m are zero-filled)
+          tma_load_3d(a_buf + (s * C::kATiles + 1) * kABytes, &tmap_phi, &full[s], phi_j0 + i * kChunk, (mtile + 1) * kTileM, hphi);
 #pragma unroll
         for (int g = 0; g < C::kBoxes; ++g) {
           const bool is_v = g >= C::kBoxes / 2;
@@ -141,6 +146,9 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
           if (SEP)                              // V columns: the second A tile, the V boxes, accumulator columns [d, 2d)
             mma_f16_ss(tmem_base + C::kN / 2, a_desc + (uint64_t)((kABytes >> 4) + k * 2),
                        b_desc + (uint64_t)(((C::kBoxes / 2) * kBoxBytes >> 4) + k * 128), idesc, (i | k) != 0);
+          if (MT == 2)                          // the second measurement tile: its A tile, the same B, its own accumulator
+            mma_f16_ss(tmem_base + C::kN, a_desc + (uint64_t)((kABytes >> 4) + k * 2), b_desc + (uint64_t)(k * 128), idesc,
+                       (i | k) != 0);
         }
         mma_commit(&empty[s]);                  // stage reusable once these MMAs have read it
       }
@@ -150,11 +158,13 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
     const int q = warp & 3;                     // this warp may touch TMEM lanes [32q, 32q+32)
     if (mbar_wait(acc_done, 0, status, 104, cta_abort) && *(volatile int*)cta_abort == 0) {
       tc_fence_after();
-      const int row = mtile * kTileM + q * 32 + lane;
+#pragma unroll 1
+      for (int mt = 0; mt < MT; ++mt) {
+      const int row = (mtile + mt) * kTileM + q * 32 + lane;
 #pragma unroll 1
       for (int c0 = 0; c0 < C::kN; c0 += 32) {
         uint32_t r[32];
-        tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+        tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(mt * C::kN + c0), r);
         tmem_wait_ld();
         // accumulator column c0: K half or V half, batch element e of the group, feature column
         const int half = c0 / (C::kN / 2), e = (c0 % (C::kN / 2)) / D, col = c0 % D;
@@ -179,11 +189,12 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
           }
         }
       }
+      }
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, C::kN);
+  if (warp == 1) tmem_dealloc(tmem_base, MT * C::kN);
 }
 
 // Self-test of the bounded wait: one thread waits on a barrier that nothing arrives at.  The wait gives up after
@@ -201,10 +212,10 @@ __global__ void wait_timeout_selftest_kernel(int* status, unsigned long long lim
 
 // n_len tokens of K, V (a shard that starts at token phi_j0 of the sequence, or the whole sequence); partial: float32
 // destination of a shard's sums, null = the workspace
-template <int D, bool SEP, int BG>
+template <int D, bool SEP, int BG, int MT = 1>
 cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int64_t phi_j0, int64_t n_len,
                    float* partial) {
-  using C = Cfg<D, SEP, BG>;
+  using C = Cfg<D, SEP, BG, MT>;
   const Params& p = c->p;
   CUtensorMap tk, tv;
   const uint64_t kd[3] = {(uint64_t)D, (uint64_t)n_len, (uint64_t)(p.B * p.H)};
@@ -214,12 +225,13 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s, in
   if ((e = make_tmap_bf16_3d(&tk, K, kd, ks, kb)) != cudaSuccess) return e;
   if ((e = make_tmap_bf16_3d(&tv, V, kd, ks, kb)) != cudaSuccess) return e;
   static DeviceFlags smem_opt_in;
-  if ((e = ensure_dynamic_smem(compress_sm100_kernel<D, SEP, BG>, (int)C::kSmemBytes, c->device, smem_opt_in)) != cudaSuccess)
+  if ((e = ensure_dynamic_smem(compress_sm100_kernel<D, SEP, BG, MT>, (int)C::kSmemBytes, c->device, smem_opt_in)) != cudaSuccess)
     return e;
   // whole batch, or a range of heads of one batch element
   const int64_t Bl = c->bh_cnt ? 1 : p.B, Hl = c->bh_cnt ? c->bh_cnt : p.H;
-  const dim3 grid((unsigned)((p.m + kTileM - 1) / kTileM), (unsigned)(((Bl + BG - 1) / BG) * Hl));
-  compress_sm100_kernel<D, SEP, BG><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
+  const int64_t mtiles = (p.m + kTileM - 1) / kTileM;
+  const dim3 grid((unsigned)((mtiles + MT - 1) / MT), (unsigned)(((Bl + BG - 1) / BG) * Hl));
+  compress_sm100_kernel<D, SEP, BG, MT><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
                                                                  (int)n_len, (int)p.H, (int)Bl, (int)c->bh0, c->status,
                                                                  (int)phi_j0, partial);
   return cudaGetLastError();
@@ -251,6 +263,13 @@ cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cud
   if (c->p.separate_phi)
     return c->p.d == 64 ? launch<64, true, 1>(c, K, V, s, phi_j0, n_len, partial)
                         : launch<128, true, 1>(c, K, V, s, phi_j0, n_len, partial);
+  // d = 128: two measurement tiles per CTA where that still leaves at least ~0.8 CTAs per SM
+  {
+    const int64_t mtiles = (c->p.m + kTileM - 1) / kTileM;
+    const int64_t bh = c->bh_cnt ? c->bh_cnt : c->p.B * c->p.H;
+    if (c->p.d == 128 && mtiles >= 2 && ((mtiles + 1) / 2) * bh * 5 >= (int64_t)c->sms * 4)
+      return launch<128, false, 1, 2>(c, K, V, s, phi_j0, n_len, partial);
+  }
   return c->p.d == 64 ? launch<64, false, 1>(c, K, V, s, phi_j0, n_len, partial)
                       : launch<128, false, 1>(c, K, V, s, phi_j0, n_len, partial);
 }
