@@ -256,20 +256,20 @@ cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cud
                                   int64_t phi_j0, int64_t n_len, float* partial) {
   *launches += 1;
   if (n_len <= 0) n_len = c->p.n;
+  // two measurement tiles per CTA where that still leaves at least ~0.8 CTAs per SM
+  const int64_t mtiles = (c->p.m + kTileM - 1) / kTileM;
+  auto pairs_fill = [&](int64_t columns_of_ctas) { return mtiles >= 2 && ((mtiles + 1) / 2) * columns_of_ctas * 5 >= (int64_t)c->sms * 4; };
   // d = 64: two batch elements per CTA where the batch has them (N = 256 MMAs)
-  if (c->p.d == 64 && c->p.B >= 2 && c->bh_cnt == 0)
-    return c->p.separate_phi ? launch<64, true, 2>(c, K, V, s, phi_j0, n_len, partial)
-                             : launch<64, false, 2>(c, K, V, s, phi_j0, n_len, partial);
+  if (c->p.d == 64 && c->p.B >= 2 && c->bh_cnt == 0) {
+    if (c->p.separate_phi) return launch<64, true, 2>(c, K, V, s, phi_j0, n_len, partial);
+    return pairs_fill(((c->p.B + 1) / 2) * c->p.H) ? launch<64, false, 2, 2>(c, K, V, s, phi_j0, n_len, partial)
+                                                  : launch<64, false, 2>(c, K, V, s, phi_j0, n_len, partial);
+  }
   if (c->p.separate_phi)
     return c->p.d == 64 ? launch<64, true, 1>(c, K, V, s, phi_j0, n_len, partial)
                         : launch<128, true, 1>(c, K, V, s, phi_j0, n_len, partial);
-  // d = 128: two measurement tiles per CTA where that still leaves at least ~0.8 CTAs per SM
-  {
-    const int64_t mtiles = (c->p.m + kTileM - 1) / kTileM;
-    const int64_t bh = c->bh_cnt ? c->bh_cnt : c->p.B * c->p.H;
-    if (c->p.d == 128 && mtiles >= 2 && ((mtiles + 1) / 2) * bh * 5 >= (int64_t)c->sms * 4)
-      return launch<128, false, 1, 2>(c, K, V, s, phi_j0, n_len, partial);
-  }
+  if (c->p.d == 128 && pairs_fill(c->bh_cnt ? c->bh_cnt : c->p.B * c->p.H))
+    return launch<128, false, 1, 2>(c, K, V, s, phi_j0, n_len, partial);
   return c->p.d == 64 ? launch<64, false, 1>(c, K, V, s, phi_j0, n_len, partial)
                       : launch<128, false, 1>(c, K, V, s, phi_j0, n_len, partial);
 }
