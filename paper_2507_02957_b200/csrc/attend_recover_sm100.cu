@@ -79,7 +79,9 @@ template <int D> struct Cfg {
   static constexpr uint32_t kMatBytes = kDBoxes * kMatBoxBytes;
   static constexpr uint32_t kOffQ = 0;                            // [tile]
   static constexpr uint32_t kOffRing = kOffQ + kTiles * kQBytes;  // [stage][K~ slot | V~ slot]
-  static constexpr uint32_t kOffBar = kOffRing + kStages * 2 * kSlotBytes;
+  static constexpr uint32_t kOffOut = kOffRing + kStages * 2 * kSlotBytes;   // [compute warp]: 32 rows of one 64-column box of the output
+  static constexpr uint32_t kOutBytes = 32 * 128;
+  static constexpr uint32_t kOffBar = kOffOut + kTiles * 4 * kOutBytes;
   static constexpr uint32_t kBarBytes = 512;
   static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes;     // base must be 1024-byte aligned (checked)
   // TMEM columns per tile (tile t starts at column 256 t): S[0] | S[1] | accumulator (Zacc, then r_t).
@@ -190,7 +192,8 @@ struct Waiter {
 template <int D, bool kUntied, int kRec>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
-                            const __grid_constant__ CUtensorMap tmap_mats, __nv_bfloat16* __restrict__ out,
+                            const __grid_constant__ CUtensorMap tmap_mats,
+                            const __grid_constant__ CUtensorMap tmap_out, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
                             int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status,
                             float* __restrict__ lse_out, int lse_stride, __nv_bfloat16* __restrict__ z_out,
@@ -224,6 +227,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     prefetch_tmap(&tmap_q);
     prefetch_tmap(&tmap_kv);
     prefetch_tmap(&tmap_mats);
+    prefetch_tmap(&tmap_out);
     mbar_init(&bars->mats_full, 1);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], kTiles);     // released by both MMA issuers
@@ -534,7 +538,9 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     const F2 sc2 = pack2(scale_log2, scale_log2);
     uint32_t cb = 0;                                            // chunks of this tile's earlier items
     int phase = 0;                                              // phases of r_full[t] this thread has waited for
-    for (int item = blockIdx.x; item < n_items && !w.dead; item += gridDim.x) {
+    uint8_t* stage = smem + C::kOffOut + warp * C::kOutBytes + lane * 128;   // this row in the warp's staging box
+    // every lane of a warp leaves the loop at the same item (a lane that gave up falls through the item's waits)
+    for (int item = blockIdx.x; item < n_items && !__any_sync(0xffffffffu, w.dead); item += gridDim.x) {
       const int bh = bh0 + item / items_x, row0 = (item % items_x) * (kTiles * kRows), h = bh % H;
       if (t >= ((nq - row0 > kRows) ? 2 : 1)) continue;         // this item has no second tile
       float ref = -INFINITY;                                    // reference maximum of the row (log2 domain)
@@ -653,6 +659,31 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         }
       }
       const int grow_m = row0 + t * kRows + row;                // this thread's query (may lie beyond n_q)
+      // The output leaves through shared memory, one 64-column box of the warp's 32 rows at a time: each thread writes
+      // its 128 bytes in the 128-byte swizzle of the tensor map and lane 0 hands the box to one TMA store, which runs
+      // while the threads go on (storing 32-byte pieces of 32 different rows per instruction straight to global
+      // memory kept them at the stores for ~4000 cycles per item).  Rows beyond n_q are clipped by the tensor map.
+      bool staged = false;
+      auto stage_box = [&](int bx) {
+        if (out == nullptr) return;
+        if (lane == 0) bulk_wait_group_read0();                 // the warp's previous store has read the buffer
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          float x[8];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) unpack2(v2[bx * 32 + c * 4 + u], x[2 * u], x[2 * u + 1]);
+          *reinterpret_cast<uint4*>(stage + ((c ^ (lane & 7)) << 4)) =
+              make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) {
+          if (grow_m < nq && !w.dead && *(volatile int*)&bars->abort == 0)
+            tma_store_3d(&tmap_out, stage, bx * 64, grow_m, bh);
+          bulk_commit_group();
+        }
+      };
       if (kMasks && z_out != nullptr && grow_m < nq) {
         uint4* zo = reinterpret_cast<uint4*>(z_out + ((int64_t)bh * nq + grow_m) * D);
 #pragma unroll
@@ -873,19 +904,35 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         // last iteration, exact shrinkage, back in the data's units: alpha^T = 2 theta eta_{1/2}(c + r' - 1/2)
         w.wait(&bars->r_full[t], phase & 1, 231); ++phase;
         tc_fence_after();
-        const float two_th = 2.f * kappa;
-#pragma unroll
-        for (int c0 = 0; c0 < D; c0 += 16) {
-          uint32_t r[16];
-          tmem_ld_32x32b_x16(acc_addr + c0, r);
-          tmem_wait_ld();
+        const F2 tt2 = pack2(2.f * kappa, 2.f * kappa), mh2 = pack2(-0.5f, -0.5f);
+        auto last16 = [&](const uint32_t (&r)[16], int c0) {
 #pragma unroll
           for (int e = 0; e < 16; e += 2) {
             float a0, a1;
             unpack2(v2[(c0 + e) >> 1], a0, a1);
-            const float y0 = a0 + __uint_as_float(r[e]) - 0.5f, y1 = a1 + __uint_as_float(r[e + 1]) - 0.5f;
-            v2[(c0 + e) >> 1] = pack2((y0 - fminf(fmaxf(y0, -0.5f), 0.5f)) * two_th, (y1 - fminf(fmaxf(y1, -0.5f), 0.5f)) * two_th);
+            // u = c + r' = x / (2 theta) + 1/2;  eta_{1/2}(u - 1/2) = (u - 1/2) - (sat(u) - 1/2): where 0 <= u <= 1 the
+            // two terms are the same float and the difference is an exact zero
+            const F2 u2 = add2(pack2(a0, a1), pack2u(r[e], r[e + 1]));
+            float u0, u1;
+            unpack2(u2, u0, u1);
+            const F2 s2 = pack2(add_sat(u0, 0.f), add_sat(u1, 0.f));
+            v2[(c0 + e) >> 1] = mul2(sub2(add2(u2, mh2), add2(s2, mh2)), tt2);
           }
+        };
+        {
+          uint32_t r0[16], r1[16];
+          tmem_ld_32x32b_x16(acc_addr, r0);
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 32) {
+            tmem_wait_ld();
+            tmem_ld_32x32b_x16(acc_addr + c0 + 16, r1);
+            last16(r0, c0);
+            tmem_wait_ld();
+            if (c0 + 32 < D) tmem_ld_32x32b_x16(acc_addr + c0 + 32, r0);
+            last16(r1, c0 + 16);
+            if (!has_psi && (c0 + 32) % 64 == 0) stage_box(c0 / 64);      // this box of the output is final
+          }
+          staged = !has_psi;
         }
         if (has_psi) {
           publish(0);
@@ -1035,35 +1082,11 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
       }
-      const int grow = row0 + t * kRows + row;
-      if (out != nullptr && grow < nq && !w.dead && *(volatile int*)&bars->abort == 0) {
-        // a row is a multiple of 128 bytes; where the output is 32-byte aligned every store covers whole
-        // 32-byte sectors (the lanes of a warp write different rows), otherwise 16-byte stores
-        __nv_bfloat16* orow = out + ((int64_t)bh * nq + grow) * D;
-        if ((reinterpret_cast<uintptr_t>(out) & 31u) == 0) {
+      if (!staged)
 #pragma unroll
-          for (int c = 0; c < D / 16; ++c) {
-            uint32_t pk[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              float x0, x1;
-              unpack2(v2[c * 8 + u], x0, x1);
-              pk[u] = pack_bf16(x0, x1);
-            }
-            st_global_v8(orow + c * 16, pk);
-          }
-        } else {
-          uint4* o = reinterpret_cast<uint4*>(orow);
-#pragma unroll
-          for (int c = 0; c < D / 8; ++c) {
-            float x[8];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) unpack2(v2[c * 4 + u], x[2 * u], x[2 * u + 1]);
-            o[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
-          }
-        }
-      }
+        for (int bx = 0; bx < C::kDBoxes; ++bx) stage_box(bx);
     }
+    if (lane == 0) bulk_wait_group0();                          // the stores are done before the kernel ends
   }
   tc_fence_before();
   __syncthreads();
@@ -1081,6 +1104,9 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   const uint32_t qb[3] = {64, (uint32_t)kRows, 1};
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
+  CUtensorMap to = tq;                                          // the output has the shape of Q; boxes of one warp's rows
+  const uint32_t ob[3] = {64, 32, 1};
+  if (out != nullptr && (e = make_tmap_bf16_3d(&to, out, qd, qs, ob)) != cudaSuccess) return e;
   static DeviceFlags smem_opt_in;
   if (!smem_opt_in.test(c->device)) {
     // setmaxnreg moves registers inside the pool the CTA is launched with (threads x the compiled register count); the
@@ -1114,7 +1140,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kRec>, tq, c->tmap_kv,
-                            kUntied ? c->tmap_lmats : c->tmap_mats, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
+                            kUntied ? c->tmap_lmats : c->tmap_mats, to, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
                             (int)p.nq, (int)p.m, (int)p.H, T, c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items,
                             (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out, alpha_out,
                             (int64_t)(p.B * p.H * p.nq * p.d), alpha_out != nullptr ? c->bw_signbits : nullptr);
