@@ -193,7 +193,8 @@ template <int D, bool kUntied, int kRec>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats,
-                            const __grid_constant__ CUtensorMap tmap_out, __nv_bfloat16* __restrict__ out,
+                            const __grid_constant__ CUtensorMap tmap_out,
+                            const __grid_constant__ CUtensorMap tmap_z, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
                             int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status,
                             float* __restrict__ lse_out, int lse_stride, __nv_bfloat16* __restrict__ z_out,
@@ -228,6 +229,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     prefetch_tmap(&tmap_kv);
     prefetch_tmap(&tmap_mats);
     prefetch_tmap(&tmap_out);
+    if (kMasks) prefetch_tmap(&tmap_z);
     mbar_init(&bars->mats_full, 1);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], kTiles);     // released by both MMA issuers
@@ -664,8 +666,11 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       // while the threads go on (storing 32-byte pieces of 32 different rows per instruction straight to global
       // memory kept them at the stores for ~4000 cycles per item).  Rows beyond n_q are clipped by the tensor map.
       bool staged = false;
-      auto stage_box = [&](int bx) {
-        if (out == nullptr) return;
+      auto stage_box = [&](int bx, const CUtensorMap* tm = nullptr) {
+        if (tm == nullptr) {
+          if (out == nullptr) return;
+          tm = &tmap_out;
+        }
         if (lane == 0) bulk_wait_group_read0();                 // the warp's previous store has read the buffer
         __syncwarp();
 #pragma unroll
@@ -680,20 +685,13 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         __syncwarp();
         if (lane == 0) {
           if (grow_m < nq && !w.dead && *(volatile int*)&bars->abort == 0)
-            tma_store_3d(&tmap_out, stage, bx * 64, grow_m, bh);
+            tma_store_3d(tm, stage, bx * 64, grow_m, bh);
           bulk_commit_group();
         }
       };
-      if (kMasks && z_out != nullptr && grow_m < nq) {
-        uint4* zo = reinterpret_cast<uint4*>(z_out + ((int64_t)bh * nq + grow_m) * D);
+      if (kMasks && z_out != nullptr)                           // Z as fed to the first product, for the backward pass
 #pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
-          float x[8];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) unpack2(v2[c * 4 + u], x[2 * u], x[2 * u + 1]);
-          zo[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
-        }
-      }
+        for (int bx = 0; bx < C::kDBoxes; ++bx) stage_box(bx, &tmap_z);
       // kMasks: this row's place in slot 0 of the iterates (rows of 2 D bytes from a 256-byte aligned base: 32-byte stores)
       __nv_bfloat16* arow = (kKeep && alpha_out != nullptr && grow_m < nq)
                                 ? alpha_out + ((int64_t)bh * nq + grow_m) * D : nullptr;
@@ -1107,6 +1105,8 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   CUtensorMap to = tq;                                          // the output has the shape of Q; boxes of one warp's rows
   const uint32_t ob[3] = {64, 32, 1};
   if (out != nullptr && (e = make_tmap_bf16_3d(&to, out, qd, qs, ob)) != cudaSuccess) return e;
+  CUtensorMap tz = tq;
+  if (z_out != nullptr && (e = make_tmap_bf16_3d(&tz, z_out, qd, qs, ob)) != cudaSuccess) return e;
   static DeviceFlags smem_opt_in;
   if (!smem_opt_in.test(c->device)) {
     // setmaxnreg moves registers inside the pool the CTA is launched with (threads x the compiled register count); the
@@ -1140,7 +1140,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kRec>, tq, c->tmap_kv,
-                            kUntied ? c->tmap_lmats : c->tmap_mats, to, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
+                            kUntied ? c->tmap_lmats : c->tmap_mats, to, tz, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
                             (int)p.nq, (int)p.m, (int)p.H, T, c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items,
                             (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out, alpha_out,
                             (int64_t)(p.B * p.H * p.nq * p.d), alpha_out != nullptr ? c->bw_signbits : nullptr);
