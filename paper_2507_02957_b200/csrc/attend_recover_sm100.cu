@@ -1156,6 +1156,8 @@ cudaError_t make_attend_tmaps(csat_ctx* c) {
   const uint32_t kb[3] = {64, (uint32_t)kMC, 1};
   cudaError_t e = make_tmap_bf16_3d(&c->tmap_kv, c->kv, kd, ks, kb);
   if (e != cudaSuccess) return e;
+  const uint32_t sb[3] = {64, 32, 1};                           // the compression kernel's stores: one warp's rows
+  if ((e = make_tmap_bf16_3d(&c->tmap_kv_st, c->kv, kd, ks, sb)) != cudaSuccess) return e;
   const uint64_t md[3] = {(uint64_t)p.d, (uint64_t)p.d, (uint64_t)(p.H * 3)};
   const uint64_t ms[2] = {(uint64_t)p.d * 2, (uint64_t)p.d * p.d * 2};
   const uint32_t mb[3] = {64, (uint32_t)p.d, 1};

@@ -8,8 +8,10 @@
 //              them, so no transpose pass is needed), 128-byte swizzle, ring of kStages buffers.
 //   warp 1   : allocates tensor memory; one elected thread issues tcgen05.mma (M=128, N=2d, K=16, bf16
 //              in, fp32 accumulate) and commits to the ring's "empty" barriers.
-//   warps 2-5: epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), round to bf16, store
-//              row r of the tile as K~_r | V~_r into the workspace.
+//   warps 2-5: epilogue: tcgen05.ld the accumulator (each warp its 32-lane quarter), round to bf16, and write
+//              row r of the tile as K~_r | V~_r into the workspace: through boxes of 32 rows x 64 columns in the
+//              ring's shared memory (free once the last MMA has finished) and one TMA store per box, so that no
+//              thread sits at stores of 16-byte pieces of 32 different lines.
 // Rows of Phi beyond m and tokens beyond n are zero-filled by TMA (and Phi's padded columns hold zeros).
 // Token-sharded use: the same kernel over a token range [phi_j0, phi_j0 + n) of Phi against a shard of K, V that
 // holds only those n tokens; the epilogue then writes the float32 partial sums to `partial` instead of the
@@ -46,12 +48,15 @@ template <int D, bool SEP, int BG, int MT = 1> struct Cfg {
   static_assert(!(SEP && MT == 2) && MT * kN <= 512, "tensor memory");
   static constexpr uint32_t kStageBytes = kATiles * kABytes + kBoxes * kBoxBytes;
   static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr uint32_t kOutBoxBytes = 32 * 128;  // epilogue staging: one warp's 32 rows x 64 columns of bf16
+  static_assert(4 * MT * (kN / 64) * kOutBoxBytes <= kStages * kStageBytes, "the epilogue's boxes fit in the ring");
 };
 
 template <int D, bool SEP, int BG, int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_k,
-                      const __grid_constant__ CUtensorMap tmap_v, __nv_bfloat16* __restrict__ kv, int m, int n, int H,
+                      const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_out,
+                      __nv_bfloat16* __restrict__ kv, int m, int n, int H,
                       int B, int bh0, int* status, int phi_j0, float* __restrict__ partial) {
   using C = Cfg<D, SEP, BG, MT>;
   extern __shared__ uint8_t smem_raw[];
@@ -81,6 +86,7 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
     prefetch_tmap(&tmap_phi);
     prefetch_tmap(&tmap_k);
     prefetch_tmap(&tmap_v);
+    prefetch_tmap(&tmap_out);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
@@ -174,8 +180,9 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
           for (int v = 0; v < 8; ++v)
             o[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
                                __uint_as_float(r[4 * v + 3]));
-        } else if (row < m && b0 + e < B) {
-          uint4* o = reinterpret_cast<uint4*>(kv + ((int64_t)bh_of(e) * m + row) * (2 * D) + half * D + col);
+        } else if (partial == nullptr) {
+          // box (mt, c0 / 64) of this warp; this thread's row of it, 16-byte pieces in the 128-byte swizzle
+          uint8_t* box = smem + ((q * MT + mt) * (C::kN / 64) + c0 / 64) * C::kOutBoxBytes;
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             uint32_t w[4];
@@ -185,10 +192,22 @@ compress_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid
                                                        __uint_as_float(r[v * 8 + 2 * j + 1]));
               w[j] = *reinterpret_cast<uint32_t*>(&p);
             }
-            o[v] = make_uint4(w[0], w[1], w[2], w[3]);
+            const int piece = (c0 % 64) / 8 + v;
+            *reinterpret_cast<uint4*>(box + lane * 128 + ((piece ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+          if (c0 % 64 == 32) {                      // the box is complete (rows beyond m are clipped by the tensor map)
+            fence_proxy_async();
+            __syncwarp();
+            const int row0 = (mtile + mt) * kTileM + q * 32;
+            if (lane == 0 && row0 < m && b0 + e < B)
+              tma_store_3d(&tmap_out, box, half * D + (col & ~63), row0, bh_of(e));
           }
         }
       }
+      }
+      if (lane == 0) {
+        bulk_commit_group();
+        bulk_wait_group0();                         // the stores are done before the kernel ends
       }
     }
   }
@@ -231,7 +250,7 @@ cudaError_t launch(csat_ctx* c, const void* K, const void* V, cudaStream_t s, in
   const int64_t Bl = c->bh_cnt ? 1 : p.B, Hl = c->bh_cnt ? c->bh_cnt : p.H;
   const int64_t mtiles = (p.m + kTileM - 1) / kTileM;
   const dim3 grid((unsigned)((mtiles + MT - 1) / MT), (unsigned)(((Bl + BG - 1) / BG) * Hl));
-  compress_sm100_kernel<D, SEP, BG, MT><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, (__nv_bfloat16*)c->kv, (int)p.m,
+  compress_sm100_kernel<D, SEP, BG, MT><<<grid, kThreads, C::kSmemBytes, s>>>(c->tmap_phi, tk, tv, c->tmap_kv_st, (__nv_bfloat16*)c->kv, (int)p.m,
                                                                  (int)n_len, (int)p.H, (int)Bl, (int)c->bh0, c->status,
                                                                  (int)phi_j0, partial);
   return cudaGetLastError();

@@ -74,6 +74,7 @@ struct csat_ctx {
   CUtensorMap tmap_phi;       // TMA view of phi for the tensor-core compress kernel (bf16, d in {64,128})
   bool tmap_phi_valid = false;
   CUtensorMap tmap_kv;        // TMA view of the K~|V~ workspace
+  CUtensorMap tmap_kv_st;     // the same workspace in boxes of 32 rows (the compression kernel's stores)
   CUtensorMap tmap_mats;      // TMA view of mats_bf16
   // bf16 operand copies of the decoder matrices for the tensor-core path: [H][3][d][d], each stored
   // [output column][k] (k contiguous): 0 = -mu G = S - I (symmetric for ISTA), 1 = B^T = (mu M)^T, 2 = Psi
