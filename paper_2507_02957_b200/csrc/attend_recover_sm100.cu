@@ -69,7 +69,9 @@ constexpr int kMaxStages = 6;
 constexpr int kComputeRegs = 224, kControlRegs = 56;   // registers per thread after setmaxnreg (checked on the host)
 constexpr int kPolyEvery = 4;          // every 4th pair of scores takes the polynomial exp2 (measured best of 1, 2, 3, 4, none)
 
-template <int D> struct Cfg {
+// kStaged: the output leaves through shared-memory boxes and TMA stores (the plain forward); the recording variants
+// store directly (they spill more, and the 32 KB of boxes would take the L1 those spills live in)
+template <int D, bool kStaged> struct Cfg {
   static constexpr int kDBoxes = D / 64;                          // 64-column boxes across the head dimension
   static constexpr int kStages = (D == 64) ? 6 : 4;               // K~ / V~ chunks in flight
   static constexpr uint32_t kQBytes = kDBoxes * kRows * 128;      // one Q tile; tile A's buffer later holds B
@@ -81,7 +83,7 @@ template <int D> struct Cfg {
   static constexpr uint32_t kOffRing = kOffQ + kTiles * kQBytes;  // [stage][K~ slot | V~ slot]
   static constexpr uint32_t kOffOut = kOffRing + kStages * 2 * kSlotBytes;   // [compute warp]: 32 rows of one 64-column box of the output
   static constexpr uint32_t kOutBytes = 32 * 128;
-  static constexpr uint32_t kOffBar = kOffOut + kTiles * 4 * kOutBytes;
+  static constexpr uint32_t kOffBar = kOffOut + (kStaged ? kTiles * 4 * kOutBytes : 0);
   static constexpr uint32_t kBarBytes = 512;
   static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes;     // base must be 1024-byte aligned (checked)
   // TMEM columns per tile (tile t starts at column 256 t): S[0] | S[1] | accumulator (Zacc, then r_t).
@@ -193,15 +195,14 @@ template <int D, bool kUntied, int kRec>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats,
-                            const __grid_constant__ CUtensorMap tmap_out,
-                            const __grid_constant__ CUtensorMap tmap_z, __nv_bfloat16* __restrict__ out,
+                            const __grid_constant__ CUtensorMap tmap_out, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
                             int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status,
                             float* __restrict__ lse_out, int lse_stride, __nv_bfloat16* __restrict__ z_out,
                             uint32_t* __restrict__ mask_out, __nv_bfloat16* __restrict__ alpha_out,
                             int64_t alpha_slot, uint32_t* __restrict__ sign_out) {
-  using C = Cfg<D>;
-  constexpr bool kMasks = kRec >= 1, kKeep = kRec >= 2;
+  using C = Cfg<D, kRec == 0>;
+  constexpr bool kMasks = kRec >= 1, kKeep = kRec >= 2, kStaged = kRec == 0;
   extern __shared__ __align__(1024) uint8_t smem[];
   if ((smem_u32(smem) & 1023u) != 0) {          // swizzled tiles need 1024-byte alignment; never seen to fail
     if (threadIdx.x == 0) atomicCAS(status, 0, 200);
@@ -228,8 +229,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     prefetch_tmap(&tmap_q);
     prefetch_tmap(&tmap_kv);
     prefetch_tmap(&tmap_mats);
-    prefetch_tmap(&tmap_out);
-    if (kMasks) prefetch_tmap(&tmap_z);
+    if (kStaged) prefetch_tmap(&tmap_out);
     mbar_init(&bars->mats_full, 1);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], kTiles);     // released by both MMA issuers
@@ -666,11 +666,8 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       // while the threads go on (storing 32-byte pieces of 32 different rows per instruction straight to global
       // memory kept them at the stores for ~4000 cycles per item).  Rows beyond n_q are clipped by the tensor map.
       bool staged = false;
-      auto stage_box = [&](int bx, const CUtensorMap* tm = nullptr) {
-        if (tm == nullptr) {
-          if (out == nullptr) return;
-          tm = &tmap_out;
-        }
+      auto stage_box = [&](int bx) {
+        if (!kStaged || out == nullptr) return;
         if (lane == 0) bulk_wait_group_read0();                 // the warp's previous store has read the buffer
         __syncwarp();
 #pragma unroll
@@ -685,13 +682,20 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         __syncwarp();
         if (lane == 0) {
           if (grow_m < nq && !w.dead && *(volatile int*)&bars->abort == 0)
-            tma_store_3d(tm, stage, bx * 64, grow_m, bh);
+            tma_store_3d(&tmap_out, stage, bx * 64, grow_m, bh);
           bulk_commit_group();
         }
       };
-      if (kMasks && z_out != nullptr)                           // Z as fed to the first product, for the backward pass
+      if (kMasks && z_out != nullptr && grow_m < nq) {          // Z as fed to the first product, for the backward pass
+        uint4* zo = reinterpret_cast<uint4*>(z_out + ((int64_t)bh * nq + grow_m) * D);
 #pragma unroll
-        for (int bx = 0; bx < C::kDBoxes; ++bx) stage_box(bx, &tmap_z);
+        for (int c = 0; c < D / 8; ++c) {
+          float x[8];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) unpack2(v2[c * 4 + u], x[2 * u], x[2 * u + 1]);
+          zo[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+        }
+      }
       // kMasks: this row's place in slot 0 of the iterates (rows of 2 D bytes from a 256-byte aligned base: 32-byte stores)
       __nv_bfloat16* arow = (kKeep && alpha_out != nullptr && grow_m < nq)
                                 ? alpha_out + ((int64_t)bh * nq + grow_m) * D : nullptr;
@@ -1080,11 +1084,38 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
       }
-      if (!staged)
+      if (kStaged && !staged)
 #pragma unroll
         for (int bx = 0; bx < C::kDBoxes; ++bx) stage_box(bx);
+      if (!kStaged && out != nullptr && grow_m < nq && !w.dead && *(volatile int*)&bars->abort == 0) {
+        // a row is a multiple of 128 bytes; where the output is 32-byte aligned every store covers whole
+        // 32-byte sectors (the lanes of a warp write different rows), otherwise 16-byte stores
+        __nv_bfloat16* orow = out + ((int64_t)bh * nq + grow_m) * D;
+        if ((reinterpret_cast<uintptr_t>(out) & 31u) == 0) {
+#pragma unroll
+          for (int c = 0; c < D / 16; ++c) {
+            uint32_t pk[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              float x0, x1;
+              unpack2(v2[c * 8 + u], x0, x1);
+              pk[u] = pack_bf16(x0, x1);
+            }
+            st_global_v8(orow + c * 16, pk);
+          }
+        } else {
+          uint4* o = reinterpret_cast<uint4*>(orow);
+#pragma unroll
+          for (int c = 0; c < D / 8; ++c) {
+            float x[8];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) unpack2(v2[c * 4 + u], x[2 * u], x[2 * u + 1]);
+            o[c] = make_uint4(pack_bf16(x[0], x[1]), pack_bf16(x[2], x[3]), pack_bf16(x[4], x[5]), pack_bf16(x[6], x[7]));
+          }
+        }
+      }
     }
-    if (lane == 0) bulk_wait_group0();                          // the stores are done before the kernel ends
+    if (kStaged && lane == 0) bulk_wait_group0();               // the stores are done before the kernel ends
   }
   tc_fence_before();
   __syncthreads();
@@ -1094,7 +1125,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
 template <int D, bool kUntied, int kRec = 0>
 cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T, float* lse_out, int lse_stride,
                    __nv_bfloat16* z_out = nullptr, uint32_t* mask_out = nullptr, __nv_bfloat16* alpha_out = nullptr) {
-  using C = Cfg<D>;
+  using C = Cfg<D, kRec == 0>;
   const Params& p = c->p;
   CUtensorMap tq;
   const uint64_t qd[3] = {(uint64_t)D, (uint64_t)p.nq, (uint64_t)(p.B * p.H)};
@@ -1104,9 +1135,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   if ((e = make_tmap_bf16_3d(&tq, Q, qd, qs, qb)) != cudaSuccess) return e;
   CUtensorMap to = tq;                                          // the output has the shape of Q; boxes of one warp's rows
   const uint32_t ob[3] = {64, 32, 1};
-  if (out != nullptr && (e = make_tmap_bf16_3d(&to, out, qd, qs, ob)) != cudaSuccess) return e;
-  CUtensorMap tz = tq;
-  if (z_out != nullptr && (e = make_tmap_bf16_3d(&tz, z_out, qd, qs, ob)) != cudaSuccess) return e;
+  if (kRec == 0 && out != nullptr && (e = make_tmap_bf16_3d(&to, out, qd, qs, ob)) != cudaSuccess) return e;
   static DeviceFlags smem_opt_in;
   if (!smem_opt_in.test(c->device)) {
     // setmaxnreg moves registers inside the pool the CTA is launched with (threads x the compiled register count); the
@@ -1140,7 +1169,7 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kRec>, tq, c->tmap_kv,
-                            kUntied ? c->tmap_lmats : c->tmap_mats, to, tz, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
+                            kUntied ? c->tmap_lmats : c->tmap_mats, to, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
                             (int)p.nq, (int)p.m, (int)p.H, T, c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items,
                             (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out, alpha_out,
                             (int64_t)(p.B * p.H * p.nq * p.d), alpha_out != nullptr ? c->bw_signbits : nullptr);
