@@ -550,8 +550,9 @@ def test_untied_lista_layers_match_oracle(name):
 
 
 def test_output_aligned_to_16_bytes_only_gives_the_same_result():
-    """The tensor-core kernel stores 32 bytes per lane where the output allows it and 16 bytes otherwise: an
-    output that starts 16 bytes into an allocation must come out bit-identical."""
+    """The tensor-core kernel's output stores (TMA stores of whole boxes in the plain forward, 32 or 16 bytes per lane
+    in the recording variants) need no more than 16-byte alignment: an output that starts 16 bytes into an
+    allocation must come out bit-identical."""
     for w in (wl.shrink(C["c2"], B=2, H=3, n_q=300), wl.shrink(C["c5"], B=1, H=2, n=1024, n_q=700, m=192)):
         inp = wl.make_inputs(w)
         Q, K, V, _ = device_inputs(w, inp)
@@ -565,6 +566,26 @@ def test_output_aligned_to_16_bytes_only_gives_the_same_result():
         assert torch.equal(out, ref)
         assert float(flat[:8].abs().max()) == 0.0
         ctx.close()
+
+
+def test_output_stores_stay_inside_the_tensor():
+    """Query counts that end inside a warp's 32 rows, a tile's 128 or an item's 256: the output boxes are clipped at
+    n_q, so guard rows before and after the tensor keep their sentinel and every row of the tensor is written."""
+    for d, nqs in ((128, (1, 33, 129, 255, 257)), (64, (31, 160, 385))):
+        for nq in nqs:
+            w = wl.shrink(C["c5"] if d == 128 else C["c2"], B=1, H=2, n=512, n_q=nq, m=192, T=2, lam=0.0)
+            inp = wl.make_inputs(w)
+            Q, K, V, _ = device_inputs(w, inp)
+            ctx = make_ctx(w)
+            guard = 256 * d
+            flat = torch.full((Q.numel() + 2 * guard,), 7.0, dtype=Q.dtype, device="cuda")
+            out = flat[guard:guard + Q.numel()].view(Q.shape)
+            ctx.forward(Q, K, V, out)
+            torch.cuda.synchronize()
+            assert float((flat[:guard] - 7.0).abs().max()) == 0.0 and float((flat[guard + Q.numel():] - 7.0).abs().max()) == 0.0
+            ref = orc.csat_forward(inp["Q"], inp["K"], inp["V"], to_np(ctx.get_phi()), T=w.T, lam=w.lam)
+            assert np.abs(ref).max() > 0 and rel_err(to_np(out), ref) <= TOL["bf16"], (d, nq)
+            ctx.close()
 
 
 @pytest.mark.parametrize("case", ["bf16_d64_self", "bf16_d128_self", "bf16_d64_cross", "bf16_ragged_k", "fp32", "bf16_ffma"])
