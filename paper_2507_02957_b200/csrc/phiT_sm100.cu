@@ -9,7 +9,9 @@
 //              {64 columns x 64 rows} boxes of dK~|dV~ (MN-major B operand), 128-byte swizzle, ring of stages.
 //   warp 1   : allocates tensor memory; one elected thread issues tcgen05.mma (M=128, N=2d, K=16, bf16 in, fp32
 //              accumulate) and commits to the ring's "empty" barriers.
-//   warps 2-5: epilogue: tcgen05.ld the accumulator, round to bf16, store row `token` of dK and of dV.
+//   warps 2-5: epilogue: tcgen05.ld the accumulator, round to bf16, and write the tile's rows of dK and dV through
+//              boxes of 32 tokens x 64 columns in the ring's shared memory (free once the last MMA has finished)
+//              and one TMA store per box (tokens beyond n are clipped by the tensor map).
 // With separate Phi_K / Phi_V a stage holds both A tiles and the K and V halves are two N = d MMAs.
 // Tokens beyond n and measurements beyond m are zero-filled by TMA.
 #include "csat_internal.h"
@@ -36,12 +38,15 @@ template <int D, bool SEP> struct Cfg {
   static constexpr uint32_t kStageBytes = kATiles * kABytes + kBoxes * kBBoxBytes;
   static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
   static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
+  static constexpr uint32_t kOutBoxBytes = 32 * 128;  // epilogue staging: one warp's 32 tokens x 64 columns of bf16
+  static_assert(4 * (kN / 64) * kOutBoxBytes <= kStages * kStageBytes, "the epilogue's boxes fit in the ring");
 };
 
 template <int D, bool SEP>
 __global__ void __launch_bounds__(kThreads, 1)
 phiT_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_g,
-                  __nv_bfloat16* __restrict__ dK, __nv_bfloat16* __restrict__ dV, int m, int n, int H, int* status) {
+                  const __grid_constant__ CUtensorMap tmap_dk, const __grid_constant__ CUtensorMap tmap_dv, int m, int n,
+                  int H, int* status) {
   using C = Cfg<D, SEP>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -60,6 +65,8 @@ phiT_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_con
   if (threadIdx.x == 0) {
     prefetch_tmap(&tmap_phi);
     prefetch_tmap(&tmap_g);
+    prefetch_tmap(&tmap_dk);
+    prefetch_tmap(&tmap_dv);
     for (int s = 0; s < C::kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     mbar_init(acc_done, 1);
     *cta_abort = 0;
@@ -127,27 +134,35 @@ phiT_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_con
     const int q = warp & 3;                       // this warp may touch TMEM lanes [32q, 32q+32)
     if (mbar_wait(acc_done, 0, status, 404, cta_abort) && *(volatile int*)cta_abort == 0) {
       tc_fence_after();
-      const int tok = ttile * kTileM + q * 32 + lane;
+      const int tok0 = ttile * kTileM + q * 32;   // this warp's first token
 #pragma unroll 1
       for (int c0 = 0; c0 < C::kN; c0 += 32) {
         uint32_t r[32];
         tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
         tmem_wait_ld();
-        if (tok < n) {
-          __nv_bfloat16* dst = (c0 < D ? dK : dV) + ((int64_t)bh * n + tok) * D + (c0 % D);
-          uint4* o = reinterpret_cast<uint4*>(dst);
+        // box c0 / 64 of this warp; this thread's token row of it, 16-byte pieces in the 128-byte swizzle
+        uint8_t* box = smem + (q * (C::kN / 64) + c0 / 64) * C::kOutBoxBytes;
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint32_t w[4];
+        for (int v = 0; v < 4; ++v) {
+          uint32_t w[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              __nv_bfloat162 p = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2 * j]),
-                                                       __uint_as_float(r[v * 8 + 2 * j + 1]));
-              w[j] = *reinterpret_cast<uint32_t*>(&p);
-            }
-            o[v] = make_uint4(w[0], w[1], w[2], w[3]);
+          for (int j = 0; j < 4; ++j) {
+            __nv_bfloat162 p = __floats2bfloat162_rn(__uint_as_float(r[v * 8 + 2 * j]),
+                                                     __uint_as_float(r[v * 8 + 2 * j + 1]));
+            w[j] = *reinterpret_cast<uint32_t*>(&p);
           }
+          const int piece = (c0 % 64) / 8 + v;
+          *reinterpret_cast<uint4*>(box + lane * 128 + ((piece ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
+        if (c0 % 64 == 32) {                        // the box is complete
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0 && tok0 < n) tma_store_3d(c0 < D ? &tmap_dk : &tmap_dv, box, (c0 % D) & ~63, tok0, bh);
+        }
+      }
+      if (lane == 0) {
+        bulk_commit_group();
+        bulk_wait_group0();                         // the stores are done before the kernel ends
       }
     }
   }
@@ -170,11 +185,16 @@ cudaError_t launch(csat_ctx* c, const void* g16, void* dK, void* dV, cudaStream_
   cudaError_t e;
   if ((e = make_tmap_bf16_3d(&tphi, c->phi, pd, ps, pb)) != cudaSuccess) return e;
   if ((e = make_tmap_bf16_3d(&tg, g16, gd, gs, gb)) != cudaSuccess) return e;
+  CUtensorMap tdk, tdv;                           // the outputs [B H, n, d] in boxes of one warp's 32 tokens
+  const uint64_t od[3] = {(uint64_t)D, (uint64_t)p.n, (uint64_t)(p.B * p.H)};
+  const uint64_t os[2] = {(uint64_t)D * 2, (uint64_t)p.n * D * 2};
+  const uint32_t ob[3] = {64, 32, 1};
+  if ((e = make_tmap_bf16_3d(&tdk, dK, od, os, ob)) != cudaSuccess) return e;
+  if ((e = make_tmap_bf16_3d(&tdv, dV, od, os, ob)) != cudaSuccess) return e;
   static DeviceFlags smem_opt_in;
   if ((e = ensure_dynamic_smem(phiT_sm100_kernel<D, SEP>, (int)C::kSmemBytes, c->device, smem_opt_in)) != cudaSuccess) return e;
   const dim3 grid((unsigned)((p.n + kTileM - 1) / kTileM), (unsigned)(p.B * p.H));
-  phiT_sm100_kernel<D, SEP><<<grid, kThreads, C::kSmemBytes, s>>>(tphi, tg, (__nv_bfloat16*)dK, (__nv_bfloat16*)dV,
-                                                                  (int)p.m, (int)p.n, (int)p.H, c->status);
+  phiT_sm100_kernel<D, SEP><<<grid, kThreads, C::kSmemBytes, s>>>(tphi, tg, tdk, tdv, (int)p.m, (int)p.n, (int)p.H, c->status);
   return cudaGetLastError();
 }
 
