@@ -34,7 +34,8 @@ template <int D, bool SEP> struct Cfg {
   static constexpr int kN = 2 * D;
   static constexpr int kBoxes = kN / 64;
   static constexpr int kATiles = SEP ? 2 : 1;
-  static constexpr int kStages = (D == 64) ? 4 : (SEP ? 3 : 4);
+  // two CTAs per SM (one's epilogue under the other's products): 2 x 2 stages of 48 KB at d = 128, 2 x 3 of 32 KB at d = 64
+  static constexpr int kStages = SEP ? (D == 64 ? 4 : 3) : (D == 64 ? 3 : 2);
   static constexpr uint32_t kStageBytes = kATiles * kABytes + kBoxes * kBBoxBytes;
   static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
   static_assert(kSmemBytes <= 227 * 1024, "shared memory budget");
@@ -43,7 +44,7 @@ template <int D, bool SEP> struct Cfg {
 };
 
 template <int D, bool SEP>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 phiT_sm100_kernel(const __grid_constant__ CUtensorMap tmap_phi, const __grid_constant__ CUtensorMap tmap_g,
                   const __grid_constant__ CUtensorMap tmap_dk, const __grid_constant__ CUtensorMap tmap_dv, int m, int n,
                   int H, int* status) {
