@@ -19,6 +19,8 @@
 //   warp 9    : one elected thread issues every TMA copy.
 //   warp 10   : one elected thread issues tile B's tcgen05.mma.
 //   warp 11   : idle (it only completes the control warpgroup).
+// Output: each compute warp stages its 32 rows, one 64-column box at a time, in shared memory and lane 0 issues a TMA
+// store of the box (the recording variants of the backward pass, which spill more and need the L1, store directly).
 //
 // Attention phase, per tile and per chunk j of 64 measurements:
 //   S_j = Q K~_j^T            (SS MMA, accumulator S[j&1] in tensor memory)
