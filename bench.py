@@ -261,6 +261,24 @@ def kernel_flops(w: wl.Workload) -> dict:
     return {"compress": f["compress"], "attend_recover": f["attend"] + f["recover"], "decoder_setup": 0}
 
 
+def executed_attend_flops(w: wl.Workload, sms: int) -> int:
+    """Flops the attention / recovery launch group really performs on the tensor cores.  The algorithmic count has
+    T + 1 products of d x d per query (alpha^t S for t = 0 .. T-1 and z B); the kernel skips alpha^0 S = 0, and where
+    the library folds B into the compressed values (ISTA-derived decoder, T >= 2, a positive threshold, at least
+    8 tiles of 128 queries per SM) the n_q products z B become the m products V~ B of the small kernel before it."""
+    bh = w.B * w.H
+    f = wl.flops(w)
+    if w.T <= 0:
+        return f["attend"]
+    psi = f["recover"] - 2 * w.n_q * w.d * w.d * (w.T + 1) * bh
+    ex = f["attend"] + 2 * w.n_q * w.d * w.d * w.T * bh + psi
+    folded = (w.dtype == "bf16" and w.d in (64, 128) and w.T >= 2 and w.lam > 0
+              and -(-w.n_q // 128) * bh >= 8 * sms)
+    if folded:
+        ex += (2 * w.m - 2 * w.n_q) * w.d * w.d * bh
+    return ex
+
+
 def time_small(w: wl.Workload, iters: int = 10, warmup: int = 3, untied: bool = False, peaks: dict | None = None,
                device_index: int = 0) -> dict:
     """Per-iteration CUDA-event timing with an L2 flush between iterations (workloads that fit in L2).
@@ -490,6 +508,11 @@ def run_csat(args, w: wl.Workload) -> dict:
                     "frac_nominal_2250": top["tflops"] / 2250.0,
                     "traffic": NCU_TRAFFIC_BYTES.get((top["kernel"], w.name)),
                     "flops_per_launch": kf.get(top["kernel"], 0), "avg_launch_ms": top["avg_ms"]}
+        if top["kernel"] == "attend_recover":
+            # achieved / frac above count the algorithmic flops; these two count what the tensor cores really did
+            ex = executed_attend_flops(w, torch.cuda.get_device_properties(local).multi_processor_count)
+            roofline["flops_executed_per_launch"] = ex
+            roofline["frac_executed"] = ex / (top["avg_ms"] * 1e-3) / 1e12 / peak_tf
         for k in kernels:
             k["frac_burst"] = k["tflops"] / burst_tf
             k["frac_sustained"] = k["tflops"] / sustained_tf

@@ -193,11 +193,15 @@ struct Waiter {
 // layout of the decisions (the gradient of the thresholds is - sum sign(x_t) o dx_t).
 // kRec: 0 = the plain forward; 1 = also Z, log sum exp and the decisions (kMasks); 2 = also the iterates and the sign
 // bits of x_t (kKeep: only then are alpha_out / sign_out looked at, so that mode 1 carries none of their registers)
-template <int D, bool kUntied, int kRec>
+// kFold (plain forward, one S, B and one positive threshold for all layers, T >= 2): the V~ stream is V~ B (formed
+// once per (batch, head) by vfold_sm100_kernel), so the accumulator of the attention phase already holds z B: there is
+// no product with B, and the first layer's shrinkage follows the normalisation directly.
+template <int D, bool kUntied, int kRec, bool kFold = false>
 __global__ void __launch_bounds__(kThreads, 1)
 attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                             const __grid_constant__ CUtensorMap tmap_mats,
-                            const __grid_constant__ CUtensorMap tmap_out, __nv_bfloat16* __restrict__ out,
+                            const __grid_constant__ CUtensorMap tmap_out,
+                            const __grid_constant__ CUtensorMap tmap_vb, __nv_bfloat16* __restrict__ out,
                             const float* __restrict__ theta, int theta_stride, int nq, int m, int H, int T,
                             int has_psi, float scale_log2, int items_x, int n_items, int bh0, int* status,
                             float* __restrict__ lse_out, int lse_stride, __nv_bfloat16* __restrict__ z_out,
@@ -232,6 +236,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
     prefetch_tmap(&tmap_kv);
     prefetch_tmap(&tmap_mats);
     if (kStaged) prefetch_tmap(&tmap_out);
+    if (kFold) prefetch_tmap(&tmap_vb);
     mbar_init(&bars->mats_full, 1);
     for (int s = 0; s < C::kStages; ++s) {
       mbar_init(&bars->k_full[s], 1); mbar_init(&bars->k_empty[s], kTiles);     // released by both MMA issuers
@@ -306,7 +311,8 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           if (w.dead) { ++g; break; }
           mbar_arrive_expect_tx(&bars->v_full[s], C::kSlotBytes);
           for (int gx = 0; gx < C::kDBoxes; ++gx)
-            tma_load_3d(v_slot(s) + gx * C::kBoxBytes, &tmap_kv, &bars->v_full[s], D + gx * 64, j * kMC, bh);
+            tma_load_3d(v_slot(s) + gx * C::kBoxBytes, kFold ? &tmap_vb : &tmap_kv, &bars->v_full[s],
+                        kFold ? gx * 64 : D + gx * 64, j * kMC, bh);
           v_hist |= 1u;
         }
         if (kUntied && T > 0 && !w.dead) {
@@ -339,7 +345,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           // every S MMA of the item has finished once the last one has: tile A's Q buffer is free for B
           const uint32_t gl = g - 1;
           w.wait(&bars->k_empty[gl % C::kStages], (gl / C::kStages) & 1, 203);
-          if (!w.dead) {
+          if (!w.dead && !kFold) {
             mbar_arrive_expect_tx(&bars->mats_full, C::kMatBytes);
             for (int gx = 0; gx < C::kDBoxes; ++gx)
               tma_load_3d(q_buf + gx * C::kMatBoxBytes, &tmap_mats, &bars->mats_full, gx * 64, 0, h * 3 + 1);
@@ -492,7 +498,8 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
         if (!kUntied && T > 0) {
           const uint32_t gv = g + nchunks;            // ring position of the first box of -mu G / Psi
           const int n_mma = nlayers;                  // r_0 = theta + z B, then T-1 increments with -mu G, then Psi
-          for (int i = 0; i < n_mma; ++i) {
+          if (kFold) release(&bars->q_free[0]);          // no B to stage: tile A's Q buffer is free
+          for (int i = kFold ? 1 : 0; i < n_mma; ++i) {
             const bool first = (i == 0), psi_step = has_psi && i == n_mma - 1;
             if (first) w.wait(&bars->mats_full, items_done & 1, 214);
             if (i == 1 || psi_step)
@@ -503,7 +510,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
               }
             if (active) {
               const uint32_t acc0 = psi_step ? 0u : 1u;
-              w.wait(&bars->a_full[t], (ab + i) & 1, 216);
+              w.wait(&bars->a_full[t], (ab + i - (kFold ? 1 : 0)) & 1, 216);
               tc_fence_after();
 #pragma unroll
               for (int k = 0; k < D / 16; ++k) {
@@ -528,7 +535,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
           }
         }
         g += nchunks + nvirt;
-        if (active) { cb += nchunks; ab += nlayers; }
+        if (active) { cb += nchunks; ab += nlayers - ((kFold && !kUntied && T > 0) ? 1 : 0); }
       }
     }
   }
@@ -854,10 +861,28 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
       // in units of 2 theta, which saves one instruction per pair of elements.  Registers c = alpha / (2 theta),
       // accumulator r' = 1/2 + (z B - a^ mu G) / (2 theta) (the threads store 1/2, z is published divided by 2 theta):
       //   s = sat(c + r') (= sat(x / (2 theta) + 1/2), one saturating add);  increment = r' - s;  c += increment.
-      const bool scaled_units = !kUntied && !kMasks && T > 0 && theta_stride == 0 && kappa > 0.f;
+      const bool scaled_units = kFold || (!kUntied && !kMasks && T > 0 && theta_stride == 0 && kappa > 0.f);
       if (scaled_units) {
         const uint32_t op_addr = tbase + C::kColS;
-        {
+        if (kFold) {
+          // the accumulator held z B (unnormalised): r'_0 = 1/2 + z B / (2 theta) goes back into it, and the first
+          // pass below reads it from there like every later one
+          const float inv2th = 0.5f / kappa;
+          const F2 i2 = pack2(inv2th, inv2th), hf = pack2(0.5f, 0.5f);
+#pragma unroll
+          for (int c0 = 0; c0 < D; c0 += 16) {
+            uint32_t tb[16];
+#pragma unroll
+            for (int e = 0; e < 16; e += 2) {
+              float r0_, r1_;
+              unpack2(fma2(v2[(c0 + e) >> 1], i2, hf), r0_, r1_);
+              tb[e] = __float_as_uint(r0_);
+              tb[e + 1] = __float_as_uint(r1_);
+            }
+            tmem_st_32x32b_x16(acc_addr + c0, tb);
+          }
+          tmem_wait_st();
+        } else {
           uint32_t tb[16];
 #pragma unroll
           for (int e = 0; e < 16; ++e) tb[e] = __float_as_uint(0.5f);
@@ -868,12 +893,12 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
 #pragma unroll
           for (int i = 0; i < D / 2; ++i) v2[i] = mul2(v2[i], i2);
         }
-        publish(0);
+        if (!kFold) publish(0);
 #pragma unroll
         for (int i = 0; i < D / 2; ++i) v2[i] = pack2(0.f, 0.f);      // alpha^0 = 0
         const F2 m1 = pack2(-1.f, -1.f);
         for (int it = 0; it + 1 < T; ++it) {
-          w.wait(&bars->r_full[t], phase & 1, 230); ++phase;
+          if (!kFold || it > 0) { w.wait(&bars->r_full[t], phase & 1, 230); ++phase; }
           tc_fence_after();
           auto shrink16 = [&](const uint32_t (&r)[16], int c0) {
             uint32_t pk[8];
@@ -1124,7 +1149,7 @@ attend_recover_sm100_kernel(const __grid_constant__ CUtensorMap tmap_q, const __
   if (warp == kMmaWarp) tmem_dealloc(tmem, C::kTmemCols);
 }
 
-template <int D, bool kUntied, int kRec = 0>
+template <int D, bool kUntied, int kRec = 0, bool kFold = false>
 cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T, float* lse_out, int lse_stride,
                    __nv_bfloat16* z_out = nullptr, uint32_t* mask_out = nullptr, __nv_bfloat16* alpha_out = nullptr) {
   using C = Cfg<D, kRec == 0>;
@@ -1143,11 +1168,11 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
     // setmaxnreg moves registers inside the pool the CTA is launched with (threads x the compiled register count); the
     // kernel asks for 2 x 128 x 224 + 128 x 56 of them, and a request the pool cannot satisfy would wait forever
     cudaFuncAttributes fa;
-    if ((e = cudaFuncGetAttributes(&fa, attend_recover_sm100_kernel<D, kUntied, kRec>)) != cudaSuccess) return e;
+    if ((e = cudaFuncGetAttributes(&fa, attend_recover_sm100_kernel<D, kUntied, kRec, kFold>)) != cudaSuccess) return e;
     if ((int64_t)fa.numRegs * kThreads < (int64_t)kTiles * kTileThreads * kComputeRegs + 128 * kControlRegs)
       return cudaErrorLaunchOutOfResources;
   }
-  if ((e = ensure_dynamic_smem(attend_recover_sm100_kernel<D, kUntied, kRec>, (int)C::kSmemBytes, c->device, smem_opt_in)) !=
+  if ((e = ensure_dynamic_smem(attend_recover_sm100_kernel<D, kUntied, kRec, kFold>, (int)C::kSmemBytes, c->device, smem_opt_in)) !=
       cudaSuccess)
     return e;
   const double scale = p.scale > 0.0 ? p.scale : 1.0 / sqrt((double)D);
@@ -1170,8 +1195,8 @@ cudaError_t launch(csat_ctx* c, const void* Q, void* out, cudaStream_t s, int T,
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kRec>, tq, c->tmap_kv,
-                            kUntied ? c->tmap_lmats : c->tmap_mats, to, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
+  return cudaLaunchKernelEx(&cfg, attend_recover_sm100_kernel<D, kUntied, kRec, kFold>, tq, c->tmap_kv,
+                            kUntied ? c->tmap_lmats : c->tmap_mats, to, c->tmap_vb, (__nv_bfloat16*)out, c->thr(), c->thr_stride(),
                             (int)p.nq, (int)p.m, (int)p.H, T, c->psi ? 1 : 0, scale_log2, (int)items_x, (int)n_items,
                             (int)c->bh0, c->status, lse_out, lse_stride, z_out, mask_out, alpha_out,
                             (int64_t)(p.B * p.H * p.nq * p.d), alpha_out != nullptr ? c->bw_signbits : nullptr);
@@ -1189,6 +1214,13 @@ cudaError_t make_attend_tmaps(csat_ctx* c) {
   if (e != cudaSuccess) return e;
   const uint32_t sb[3] = {64, 32, 1};                           // the compression kernel's stores: one warp's rows
   if ((e = make_tmap_bf16_3d(&c->tmap_kv_st, c->kv, kd, ks, sb)) != cudaSuccess) return e;
+  // V~ B behind K~|V~: [B H, m, d]
+  const __nv_bfloat16* vb = (const __nv_bfloat16*)c->kv + (size_t)(p.B * p.H * p.m * 2 * p.d);
+  const uint64_t vd[3] = {(uint64_t)p.d, (uint64_t)p.m, (uint64_t)(p.B * p.H)};
+  const uint64_t vs[2] = {(uint64_t)p.d * 2, (uint64_t)p.m * p.d * 2};
+  const uint32_t vbx[3] = {64, (uint32_t)kMC, 1};
+  if ((e = make_tmap_bf16_3d(&c->tmap_vb, vb, vd, vs, vbx)) != cudaSuccess) return e;
+  if ((e = make_tmap_bf16_3d(&c->tmap_vb_st, vb, vd, vs, sb)) != cudaSuccess) return e;
   const uint64_t md[3] = {(uint64_t)p.d, (uint64_t)p.d, (uint64_t)(p.H * 3)};
   const uint64_t ms[2] = {(uint64_t)p.d * 2, (uint64_t)p.d * p.d * 2};
   const uint32_t mb[3] = {64, (uint32_t)p.d, 1};
@@ -1209,6 +1241,17 @@ cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, c
   // with untied layers and T > 0 the per-layer kernel; the set-up has then built its operands for exactly T layers
   if (c->w_S && c->w_untied && c->p.T > 0)
     return c->p.d == 64 ? launch<64, true>(c, Q, out, s, c->p.T, nullptr, 0) : launch<128, true>(c, Q, out, s, c->p.T, nullptr, 0);
+  // Long jobs with the ISTA-derived decoder (one S, B and one positive threshold for all layers) fold B into the
+  // values first: one more small launch, which only pays where the attention kernel walks many items per SM.  The
+  // choice looks at the context's whole job, not at the launch's range of (batch, head) pairs, so that a forward cut
+  // into sub-range launches returns the same bits as one launch.
+  const int64_t tiles = ((c->p.nq + kRows - 1) / kRows) * c->p.B * c->p.H;
+  if (!c->w_S && c->p.T >= 2 && c->p.lambda > 0.0 && tiles >= 8 * (int64_t)c->sms) {
+    cudaError_t e = launch_sm100_vfold(c, s, launches);
+    if (e != cudaSuccess) return e;
+    return c->p.d == 64 ? launch<64, false, 0, true>(c, Q, out, s, c->p.T, nullptr, 0)
+                        : launch<128, false, 0, true>(c, Q, out, s, c->p.T, nullptr, 0);
+  }
   return c->p.d == 64 ? launch<64, false>(c, Q, out, s, c->p.T, nullptr, 0) : launch<128, false>(c, Q, out, s, c->p.T, nullptr, 0);
 }
 

@@ -66,7 +66,12 @@ csat::Params gen_params(const csat::Params& p) {
   g.H = p.H * (p.separate_phi ? 2 : 1);
   return g;
 }
-size_t kv_bytes(const csat::Params& p) { return (size_t)(p.B * p.H * p.m * 2 * p.d) * csat::elt_size(p.dtype); }
+// K~|V~ [B H, m, 2 d]; bf16 contexts keep V~ B [B H, m, d] (the recovery phase's first product, folded into the
+// values) behind it in the same allocation
+size_t kv_bytes(const csat::Params& p) {
+  const int64_t cols = 2 * p.d + (p.dtype == CSAT_DTYPE_BF16 ? p.d : 0);
+  return (size_t)(p.B * p.H * p.m * cols) * csat::elt_size(p.dtype);
+}
 size_t dd_bytes(const csat::Params& p, size_t elt) { return (size_t)(p.H * p.d * p.d) * elt; }
 
 void prof_destroy(csat_ctx* c);

@@ -75,6 +75,8 @@ struct csat_ctx {
   bool tmap_phi_valid = false;
   CUtensorMap tmap_kv;        // TMA view of the K~|V~ workspace
   CUtensorMap tmap_kv_st;     // the same workspace in boxes of 32 rows (the compression kernel's stores)
+  CUtensorMap tmap_vb;        // V~ B [B H, m, d] behind K~|V~ in the same allocation (bf16 contexts), as the attention phase loads it
+  CUtensorMap tmap_vb_st;     // the same in boxes of 32 rows (the stores of the kernel that forms it)
   CUtensorMap tmap_mats;      // TMA view of mats_bf16
   // bf16 operand copies of the decoder matrices for the tensor-core path: [H][3][d][d], each stored
   // [output column][k] (k contiguous): 0 = -mu G = S - I (symmetric for ISTA), 1 = B^T = (mu M)^T, 2 = Psi
@@ -194,6 +196,7 @@ cudaError_t launch_simt_attend_recover(csat_ctx* c, const void* Q, void* out, cu
 // compress_sm100.cu : tcgen05 / TMEM / TMA compression (bf16, d in {64, 128})
 cudaError_t make_phi_tmap(csat_ctx* c);
 cudaError_t launch_wait_timeout_selftest(csat_ctx* c, unsigned long long limit_ns, cudaStream_t s);
+cudaError_t launch_sm100_vfold(csat_ctx* c, cudaStream_t s, int* launches);
 cudaError_t launch_sm100_compress(csat_ctx* c, const void* K, const void* V, cudaStream_t s, int* launches,
                                   int64_t phi_j0 = 0, int64_t n_len = 0, float* partial = nullptr);
 

@@ -131,6 +131,24 @@ def test_untied_layers_at_the_full_workload_shape(key, pairs):
     ctx.close()
 
 
+def test_host_buffer_forward_is_bit_identical_where_b_is_folded_into_the_values():
+    """At c3's size the library forms V~ B before the attention kernel (more than 8 query tiles per SM, ISTA-derived
+    decoder, lambda > 0).  The choice is made for the whole job, so the host-buffer entry point, which cuts the job
+    into sub-range launches, returns the same bits as csat_forward (three launches per range instead of two)."""
+    w = wl.CONFIGS["c3"]
+    inp = wl.make_inputs(w)
+    Q, K, V, _ = device_inputs(w, inp)
+    ctx = make_ctx(w)
+    out = ctx.forward(Q, K, V)
+    assert ctx.launches in (3, 3 + 3)          # compress, V~ B, attention / recovery (+ the decoder set-up at first use)
+    Qh, Kh, Vh = (t.cpu().pin_memory() for t in (Q, K, V))
+    oh = torch.empty_like(Qh).pin_memory()
+    ctx.forward_host(Qh, Kh, Vh, oh)
+    torch.cuda.synchronize()
+    assert torch.equal(oh, out.cpu())
+    ctx.close()
+
+
 @pytest.mark.parametrize("key,pairs", [("c3", [(0, 0), (7, 11)]), ("c4", [(15, 7)]), ("c2", [(0, 0), (31, 11)])])
 def test_backward_at_the_full_workload_shape(key, pairs):
     """csat_backward on the whole workload (thousands of query tiles through the tensor-core stages): sampled
