@@ -39,9 +39,9 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
 # summarised under profiles/ (None until a capture of that kernel and workload exists)
 NCU_TRAFFIC_BYTES = {
-    # profiles/dram_traffic_c5_long.txt: 153.3 MB read + 87.2 MB written (part of the 134 MB output is still in L2
-    # when the kernel ends); algorithmic: Q 134.2 + out 134.2 + K~|V~ 16.8 MB
-    ("attend_recover", "c5_long"): 240465920,
+    # profiles/dram_traffic_c5_long.txt: 152.2 MB read + 86.0 MB written by the attention / recovery kernel (part of
+    # the 134 MB output is still in L2 when the kernel ends); algorithmic: Q 134.2 + out 134.2 + K~|V~ B 16.8 MB
+    ("attend_recover", "c5_long"): 238173952,
 }
 
 
