@@ -426,6 +426,42 @@ def test_tensor_core_edge_shapes():
         ctx.close()
 
 
+def test_values_with_b_folded_in_edge_shapes():
+    """Jobs long enough for the library to form V~ B first (at least 8 query tiles per SM): ragged measurement counts,
+    a dictionary, separate Phi_K / Phi_V, both head sizes, a ragged last query tile; sampled (batch, head) pairs against
+    the oracle, and the exported V~ is still Phi V (V~ B lives beside it)."""
+    cases = [  # B, H, n, n_q, d, m, T, with_psi, separate
+        (2, 5, 600, 15400, 64, 200, 3, True, False),
+        (1, 10, 512, 15900, 128, 136, 2, False, True),
+        (1, 10, 384, 16000, 128, 129, 5, False, False),
+    ]
+    for (B, H, n, nq, d, m, T, with_psi, separate) in cases:
+        w = wl.Workload("folded_edge", B, H, n, nq, d, m, "bf16", T, 0.004, "iid", 9)
+        inp = wl.make_inputs(w)
+        Q, K, V, _ = device_inputs(w, inp)
+        ctx = make_ctx(w)
+        psi = None
+        if with_psi:
+            psi = wl.round_to_storage(wl.orthonormal_basis(d, 7 + d), "bf16")
+            ctx.set_dictionary(to_dev(psi, "bf16"))
+        if separate:
+            ctx.set(separate_phi=True)
+        phi = to_np(ctx.get_phi())
+        out = ctx.forward(Q, K, V)
+        assert ctx.launches >= 3 and torch.isfinite(out).all()
+        assert torch.equal(out, ctx.forward(Q, K, V))
+        kt, vt = (to_np(t) for t in ctx.get_compressed())
+        for (b, h) in [(0, 0), (B - 1, H - 1)]:
+            st = {}
+            ref = orc.csat_forward_head(inp["Q"][b, h], inp["K"][b, h], inp["V"][b, h], phi[h], T=T, lam=w.lam,
+                                        Psi=None if psi is None else psi.astype(np.float64),
+                                        Phi_v_h=phi[H + h] if separate else None, stages=st)
+            assert np.abs(ref).max() > 0
+            assert rel_err(to_np(out[b, h]), ref) <= TOL["bf16"], (B, H, n, nq, d, m, T, b, h)
+            assert rel_err(vt[b, h], st["Vt"]) <= 4e-3
+        ctx.close()
+
+
 @pytest.mark.parametrize("d", [64, 128])
 def test_pipelined_host_forward_is_bit_identical(d):
     """csat_forward_host cuts the job into chunks of heads of one batch element (here 2 + 2 + 1 heads per batch
