@@ -267,7 +267,8 @@ int csat_project_qkv(csat_ctx* ctx, const void* Xq, const void* Xkv, const void*
  *   Q   [B, H, n_q, d]   K, V [B, H, n, d]   out [B, H, n_q, d]   device, context dtype.
  * out must not overlap Q, K or V (checked on the byte ranges: CSAT_ERR_INVALID_ARG).  Launch-only: no allocation, no synchronisation, no host
  * access to the tensors.  The n_q x m attention matrix and the recovery iterates never reach
- * global memory; K~|V~ (m x 2d per (b,h)) live in the context's workspace.
+ * global memory; K~|V~ (m x 2d per (b,h)) live in the context's workspace (bf16 contexts keep m x d more per (b,h)
+ * for V~ B: long jobs with one S, B and one positive threshold for all layers use z B = A~ (V~ B), LISTA recurrence).
  * Errors: CSAT_ERR_INVALID_ARG (NULL/misaligned), CSAT_ERR_SHAPE (default D with m < d or
  * n < d), CSAT_ERR_CUDA (launch failure), CSAT_ERR_TIMEOUT (a previous launch's bounded wait
  * gave up; its output is invalid).
