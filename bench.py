@@ -265,7 +265,8 @@ def executed_attend_flops(w: wl.Workload, sms: int) -> int:
     """Flops the attention / recovery launch group really performs on the tensor cores.  The algorithmic count has
     T + 1 products of d x d per query (alpha^t S for t = 0 .. T-1 and z B); the kernel skips alpha^0 S = 0, and where
     the library folds B into the compressed values (ISTA-derived decoder, T >= 2, a positive threshold, at least
-    8 tiles of 128 queries per SM) the n_q products z B become the m products V~ B of the small kernel before it."""
+    2 tiles of 128 queries per SM at d = 128 and 8 at d = 64) the n_q products z B become the m products V~ B of the
+    small kernel before it."""
     bh = w.B * w.H
     f = wl.flops(w)
     if w.T <= 0:
@@ -273,7 +274,7 @@ def executed_attend_flops(w: wl.Workload, sms: int) -> int:
     psi = f["recover"] - 2 * w.n_q * w.d * w.d * (w.T + 1) * bh
     ex = f["attend"] + 2 * w.n_q * w.d * w.d * w.T * bh + psi
     folded = (w.dtype == "bf16" and w.d in (64, 128) and w.T >= 2 and w.lam > 0
-              and -(-w.n_q // 128) * bh >= 8 * sms)
+              and -(-w.n_q // 128) * bh >= (2 if w.d == 128 else 8) * sms)
     if folded:
         ex += (2 * w.m - 2 * w.n_q) * w.d * w.d * bh
     return ex

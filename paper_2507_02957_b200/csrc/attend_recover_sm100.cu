@@ -1242,11 +1242,12 @@ cudaError_t launch_sm100_attend_recover(csat_ctx* c, const void* Q, void* out, c
   if (c->w_S && c->w_untied && c->p.T > 0)
     return c->p.d == 64 ? launch<64, true>(c, Q, out, s, c->p.T, nullptr, 0) : launch<128, true>(c, Q, out, s, c->p.T, nullptr, 0);
   // Long jobs with the ISTA-derived decoder (one S, B and one positive threshold for all layers) fold B into the
-  // values first: one more small launch, which only pays where the attention kernel walks many items per SM.  The
-  // choice looks at the context's whole job, not at the launch's range of (batch, head) pairs, so that a forward cut
-  // into sub-range launches returns the same bits as one launch.
+  // values first: one more small launch, which only pays where the attention kernel walks several items per SM
+  // (measured: from ~2 tiles of 128 queries per SM at d = 128, where a layer's hand-over chain is long, from ~8 at
+  // d = 64).  The choice looks at the context's whole job, not at the launch's range of (batch, head) pairs, so that
+  // a forward cut into sub-range launches returns the same bits as one launch.
   const int64_t tiles = ((c->p.nq + kRows - 1) / kRows) * c->p.B * c->p.H;
-  if (!c->w_S && c->p.T >= 2 && c->p.lambda > 0.0 && tiles >= 8 * (int64_t)c->sms) {
+  if (!c->w_S && c->p.T >= 2 && c->p.lambda > 0.0 && tiles >= (c->p.d == 128 ? 2 : 8) * (int64_t)c->sms) {
     cudaError_t e = launch_sm100_vfold(c, s, launches);
     if (e != cudaSuccess) return e;
     return c->p.d == 64 ? launch<64, false, 0, true>(c, Q, out, s, c->p.T, nullptr, 0)

@@ -132,7 +132,7 @@ def test_untied_layers_at_the_full_workload_shape(key, pairs):
 
 
 def test_host_buffer_forward_is_bit_identical_where_b_is_folded_into_the_values():
-    """At c3's size the library forms V~ B before the attention kernel (more than 8 query tiles per SM, ISTA-derived
+    """At c3's size the library forms V~ B before the attention kernel (more than 8 query tiles per SM at d = 64, ISTA-derived
     decoder, lambda > 0).  The choice is made for the whole job, so the host-buffer entry point, which cuts the job
     into sub-range launches, returns the same bits as csat_forward (three launches per range instead of two)."""
     w = wl.CONFIGS["c3"]

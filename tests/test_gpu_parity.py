@@ -427,7 +427,7 @@ def test_tensor_core_edge_shapes():
 
 
 def test_values_with_b_folded_in_edge_shapes():
-    """Jobs long enough for the library to form V~ B first (at least 8 query tiles per SM): ragged measurement counts,
+    """Jobs long enough for the library to form V~ B first (at least 8 query tiles per SM at d = 64, 2 at d = 128): ragged measurement counts,
     a dictionary, separate Phi_K / Phi_V, both head sizes, a ragged last query tile; sampled (batch, head) pairs against
     the oracle, and the exported V~ is still Phi V (V~ B lives beside it)."""
     cases = [  # B, H, n, n_q, d, m, T, with_psi, separate
